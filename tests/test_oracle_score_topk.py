@@ -1,0 +1,119 @@
+"""Pins for the oracle's SCORE (Eq. 1, bitcount-xor identity) and TOPK (standard top-k, ties to
+the lowest index): hand-derived fixtures, bit-level brute force, the O(n^2) rank definition and
+invariants.  CPU only."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _lines(name):
+    with open(os.path.join(GOLD, name)) as f:
+        return [ln.strip() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+def test_golden_hamming_cases():
+    for ln in _lines("hamming_cases.txt"):
+        qc, kc, ham, sc = ln.split()
+        s = oracle.score([int(qc, 16)], [int(kc, 16)])
+        assert int(s[0]) == int(sc) == 32 - int(ham), ln
+
+
+def test_score_equals_32_minus_bitwise_hamming_brute_force():
+    rng = np.random.default_rng(10)
+    q = rng.integers(0, 2**32, size=1, dtype=np.uint64).astype(np.uint32)
+    k = rng.integers(0, 2**32, size=5000, dtype=np.uint64).astype(np.uint32)
+    s = oracle.score(q, k)
+    qb = np.unpackbits(q.view(np.uint8)).reshape(1, 32)
+    kb = np.unpackbits(k.view(np.uint8)).reshape(-1, 32)
+    ham = (qb != kb).sum(axis=1)
+    assert np.array_equal(s, 32 - ham)
+    assert s.min() >= 0 and s.max() <= 32
+    # library popcount of the xor
+    assert np.array_equal(s, 32 - np.array([bin(int(a) ^ int(q[0])).count("1") for a in k]))
+
+
+def test_score_special_values_and_invariances():
+    rng = np.random.default_rng(11)
+    k = rng.integers(0, 2**32, size=1000, dtype=np.uint64).astype(np.uint32)
+    q = np.uint32(0x9E3779B9)
+    assert np.all(oracle.score([q], [q]) == 32)
+    assert np.all(oracle.score([q], [~q]) == 0)
+    base = oracle.score([q], k)
+    mask = np.uint32(0xC0FFEE11)
+    assert np.array_equal(oracle.score([q ^ mask], k ^ mask), base)       # common flip mask
+    rot = lambda v: ((v << np.uint32(7)) | (v >> np.uint32(25))).astype(np.uint32)
+    assert np.array_equal(oracle.score([rot(np.array([q]))[0]], rot(k)), base)   # common bit permutation
+    # Hamming distance is symmetric in its two arguments
+    assert all(int(oracle.score([kk], [q])[0]) == int(b) for kk, b in zip(k[:50], base[:50]))
+
+
+def test_group_score_is_max_over_group_and_reduces_to_eq1_for_one_head():
+    rng = np.random.default_rng(12)
+    k = rng.integers(0, 2**32, size=3000, dtype=np.uint64).astype(np.uint32)
+    qs = rng.integers(0, 2**32, size=4, dtype=np.uint64).astype(np.uint32)
+    per_head = np.stack([oracle.score([qq], k) for qq in qs])
+    assert np.array_equal(oracle.score(qs, k), per_head.max(axis=0))
+    assert np.array_equal(oracle.score(qs[:1], k), per_head[0])
+    assert np.array_equal(oracle.score(qs[[2, 0, 3, 1]], k), oracle.score(qs, k))
+
+
+def test_golden_topk_cases():
+    for ln in _lines("topk_cases.txt"):
+        k, scores, sel = [p.strip() for p in ln.split("|")]
+        got = oracle.topk([int(v) for v in scores.split()], int(k))
+        assert got.tolist() == [int(v) for v in sel.split()], ln
+
+
+def _rank_definition(scores, k):
+    n = len(scores)
+    sel = []
+    for i in range(n):
+        better = sum(1 for j in range(n) if scores[j] > scores[i] or (scores[j] == scores[i] and j < i))
+        if better < k:
+            sel.append(i)
+    return sel
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_topk_matches_rank_definition_on_small_inputs(seed):
+    rng = np.random.default_rng(100 + seed)
+    for n in (1, 2, 7, 33, 64):
+        scores = rng.integers(12, 22, size=n)           # narrow range -> heavy ties
+        for k in (0, 1, n // 2, n - 1, n, n + 3):
+            assert oracle.topk(scores, k).tolist() == _rank_definition(scores.tolist(), k)
+
+
+def test_topk_properties_on_large_tied_input():
+    rng = np.random.default_rng(13)
+    n = 20000
+    scores = np.clip(np.rint(rng.normal(18, 1.8, size=n)), 0, 32).astype(np.int32)
+    prev = set()
+    for k in (1, 50, 625, 626, 5000, n):
+        idx = oracle.topk(scores, k)
+        assert len(idx) == min(k, n) and np.all(np.diff(idx) > 0)
+        sel = np.zeros(n, bool)
+        sel[idx] = True
+        if k < n:
+            t = scores[sel].min()
+            assert t >= scores[~sel].max()
+            tied_sel = np.nonzero(sel & (scores == t))[0]
+            tied_not = np.nonzero(~sel & (scores == t))[0]
+            if len(tied_sel) and len(tied_not):
+                assert tied_sel.max() < tied_not.min()
+        assert prev <= set(idx.tolist())                 # nesting I_k subset I_k'
+        prev = set(idx.tolist())
+    # library sort: lexsort by (index asc) within (score desc)
+    order = np.lexsort((np.arange(n), -scores))
+    assert sorted(order[:625].tolist()) == oracle.topk(scores, 625).tolist()
+    assert np.bincount(scores, minlength=33).sum() == n
+
+
+def test_topk_all_equal_scores_takes_lowest_indices():
+    assert oracle.topk(np.full(100, 17), 10).tolist() == list(range(10))
+    assert oracle.topk(np.full(5, 0), 10).tolist() == list(range(5))
+    assert oracle.topk(np.array([], dtype=np.int32), 4).tolist() == []
