@@ -1,0 +1,184 @@
+/*
+ * hashattn.h — C ABI of the B200 (sm_100a) HashAttention decode library.
+ *
+ * The library implements the decode-time sparse-attention recipe of the HashAttention paper
+ * (arXiv 2412.14468, Section 4): ENCODE the query and the newly appended key into 32-bit
+ * signatures with the learned mappings (Eq. 2), SCORE every cached token by the Hamming
+ * distance between signatures (Eq. 1, computed as bitcount(xor), Section 4.1
+ * "Implementation"), take the standard TOPK per KV head, and run GATHER-ATT — exact softmax
+ * attention restricted to the selected tokens (Section 4), reading K/V rows by index without
+ * compacting them (Section 4.4).
+ *
+ * General conventions
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller and
+ *     must stay valid until the work enqueued on `stream` has completed.  bf16 values are passed
+ *     as uint16_t bit patterns.  `stream` is a cudaStream_t passed as void* (NULL = legacy
+ *     default stream).
+ *   - Calls only enqueue work on `stream`: no host synchronisation and no allocation, except
+ *     where stated (ha_read_device_status, ha_sparse_decode_host).
+ *   - Scratch memory is one caller-owned workspace of at least ha_workspace_bytes(...) bytes,
+ *     256-byte aligned, prepared once with ha_workspace_init.  Calls that share a workspace must
+ *     be ordered on one stream.
+ *   - Return value: HA_OK, or an HA_ERR_* code for errors detectable on the host (nothing is
+ *     enqueued in that case).  Errors only visible on the device (an index outside the sequence)
+ *     set a bit in the workspace status word, are skipped, and never trap.
+ *   - Fixed by the method's configuration (Section 5.2; abstract): head_dim = 128, signature
+ *     width b = 32 bits, mapping network 128x128 - 128x128 - 128x32.  Other values return
+ *     HA_ERR_UNSUPPORTED.  n_q_heads must be a multiple of n_kv_heads with a group size
+ *     G = n_q_heads / n_kv_heads <= 8; query head j uses KV head j / G.
+ */
+#ifndef HASHATTN_H
+#define HASHATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HA_OK 0
+#define HA_ERR_INVALID_ARG 1 /* NULL where a pointer is required, negative size, bad stride */
+#define HA_ERR_UNSUPPORTED 2 /* head_dim != 128, n_bits != 32, group size > 8, ... */
+#define HA_ERR_WORKSPACE 3   /* workspace NULL, misaligned or smaller than ha_workspace_bytes */
+#define HA_ERR_CUDA 4        /* a CUDA runtime call failed (launch error, bad stream) */
+
+/* bits of the device status word (ha_read_device_status) */
+#define HA_DEV_BAD_INDEX 1u /* an idx entry >= seq_len was met and skipped */
+#define HA_DEV_TIMEOUT 2u   /* reserved: a bounded wait gave up (no kernel here spins) */
+
+#define HA_HEAD_DIM 128
+#define HA_N_BITS 32
+#define HA_HIST_BINS 33 /* scores 0..32 */
+
+/* Problem shape of one layer-step. sm_scale multiplies the logits (1/sqrt(d) in the SDPA
+ * definition, Section 3.1). */
+typedef struct ha_shape {
+    int32_t batch;
+    int32_t n_q_heads;
+    int32_t n_kv_heads;
+    int32_t head_dim; /* must be 128 */
+    float sm_scale;
+} ha_shape;
+
+/* One side's mapping networks (phi_q or phi_kv of Eq. 2), one network per KV head.
+ * y = x W + b with W stored [in][out] row-major; hidden activation ReLU; bit o of the signature
+ * is 1 iff output o of the last layer is > 0.  Biases may be NULL (= zeros). */
+typedef struct ha_mapping {
+    int32_t n_kv_heads;
+    int32_t in_dim;  /* 128 */
+    int32_t hid_dim; /* 128 */
+    int32_t n_bits;  /* 32 */
+    const uint16_t *w1; /* bf16 [n_kv_heads][128][128] */
+    const uint16_t *w2; /* bf16 [n_kv_heads][128][128] */
+    const uint16_t *w3; /* bf16 [n_kv_heads][128][32]  */
+    const float *b1;    /* fp32 [n_kv_heads][128] or NULL */
+    const float *b2;    /* fp32 [n_kv_heads][128] or NULL */
+    const float *b3;    /* fp32 [n_kv_heads][32]  or NULL */
+} ha_mapping;
+
+/* A bf16 tensor [batch][heads][tokens][128] addressed by element strides; the last dimension is
+ * contiguous and every row must start on a 16-byte boundary (strides multiples of 8). */
+typedef struct ha_tensor {
+    const void *ptr;
+    int64_t stride_b;
+    int64_t stride_h;
+    int64_t stride_n;
+} ha_tensor;
+
+/* Bytes of workspace needed by every entry point for shapes up to (shape, max_seq_len, max_k).
+ * Returns 0 if the shape is unsupported. */
+size_t ha_workspace_bytes(const ha_shape *shape, int32_t max_seq_len, int32_t max_k);
+
+/* Clears the workspace header (device status word).  Call once after allocating the workspace
+ * and whenever the status should be reset. */
+int ha_workspace_init(void *workspace, size_t ws_bytes, void *stream);
+
+/* ENCODE — Eq. 2: codes = pack(sign(F(x)) > 0) with F the Section 5.2 network; phi_kv takes the
+ * key only (Section 4.1).  Arithmetic: fp32 fused multiply-add chain per output, ascending input
+ * index, started from the bias; hidden activations stay fp32.
+ *   x             bf16 [batch][n_heads][n_tokens][128] (strides in x)
+ *   heads_per_kv  head h uses network h / heads_per_kv (G for the query side, 1 for the key side)
+ *   codes         out: codes[b*c_stride_b + h*c_stride_h + t] for t < n_tokens, or, when `slot`
+ *                 is given (n_tokens must be 1), codes[b*c_stride_b + h*c_stride_h + slot[b]]
+ *                 (the append of Section 4.1: slot[b] = seq_len[b] - 1); slot[b] < 0 skips b. */
+int ha_encode(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, int32_t batch,
+              int32_t n_heads, int32_t n_tokens, uint32_t *codes, int64_t c_stride_b,
+              int64_t c_stride_h, const int32_t *slot, void *stream);
+
+/* SCORE + TOPK — Eq. 1 as s = 32 - bitcount(k_code xor q_code) (Section 4.1), group score =
+ * max over the G query heads of the KV head, then the standard top-k (Section 4) with ties
+ * broken towards the lowest token index.
+ *   q_codes    u32 [batch][n_q_heads]
+ *   k_codes    u32 [batch][n_kv_heads][>= seq_len], token-contiguous, rows 16-byte aligned
+ *   seq_lens   i32 [batch]
+ *   k_per_seq  i32 [batch] or NULL (then k_uniform is used for every sequence)
+ *   idx        out i32 [batch][n_kv_heads][k_max] (strides given), ascending token index,
+ *              entries count..k_max-1 set to -1; k_max = max budget = the k passed to
+ *              ha_workspace_bytes or less
+ *   count      out i32 [batch][n_kv_heads] = min(k_b, seq_len_b)
+ *   hist_out   optional out i32 [batch][n_kv_heads][33]: histogram of the group scores */
+int ha_score_topk(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes,
+                  int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens,
+                  const int32_t *k_per_seq, int32_t k_uniform, int32_t max_seq_len, int32_t k_max,
+                  int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
+                  int32_t *hist_out, void *workspace, size_t ws_bytes, void *stream);
+
+/* GATHER-ATT — Section 4: out_j = sum_{i in I} softmax_I(sm_scale <q_j, k_i>) v_i for every
+ * query head j, I = idx[b][j / G][0..count).  K/V rows are read in place through the indices
+ * (Section 4.4).  fp32 accumulation, one rounding to bf16.
+ *   idx entries < 0 are padding and skipped; entries >= seq_len are skipped and raise
+ *   HA_DEV_BAD_INDEX.  An empty list gives out = 0, lse = -inf.
+ *   out bf16 [batch][n_q_heads][128]; lse fp32 [batch][n_q_heads] or NULL. */
+int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
+                   const ha_tensor *V, const int32_t *seq_lens, const int32_t *idx,
+                   int64_t idx_stride_b, int64_t idx_stride_h, const int32_t *count, int32_t k_max,
+                   uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream);
+
+/* Dense decode attention — single-query SDPA over all seq_len tokens (Section 3.1): the
+ * computation the sparse path replaces, provided as the same-run comparator. */
+int ha_dense_decode(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
+                    const ha_tensor *V, const int32_t *seq_lens, int32_t max_seq_len,
+                    uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream);
+
+/* One whole layer-step (Section 4 recipe; Section 4.1 "Implementation"): signature of the new
+ * key appended at slot seq_len-1 (skipped if k_new is NULL), query signatures, SCORE, TOPK,
+ * GATHER-ATT.  Same semantics as ha_encode (x2) + ha_score_topk + ha_gather_attn.
+ *   k_new    bf16 [batch][n_kv_heads][128] contiguous or NULL
+ *   q_codes  out u32 [batch][n_q_heads]; k_codes is read and, if k_new, written at the slot. */
+int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
+                     const uint16_t *q, const uint16_t *k_new, const ha_tensor *K,
+                     const ha_tensor *V, uint32_t *k_codes, int64_t kc_stride_b,
+                     int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
+                     int32_t k_uniform, int32_t max_seq_len, int32_t k_max, uint32_t *q_codes,
+                     int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
+                     uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream);
+
+/* The same layer-step driven from HOST buffers (the per-step inputs of a decoder: the new
+ * query, key and value vectors; Section 4.1): copies q_host, k_new_host, v_new_host to the device
+ * (staging inside the workspace), writes the new K/V rows into the resident cache at slot
+ * seq_len-1, runs ha_sparse_decode, copies `out` back to out_host and SYNCHRONISES the stream.
+ * Host buffers should be pinned.  K, V, k_codes, seq_lens, k_per_seq, idx, count stay device
+ * pointers (resident state).  K and V must be writable. */
+int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
+                          const uint16_t *q_host, const uint16_t *k_new_host,
+                          const uint16_t *v_new_host, const ha_tensor *K, const ha_tensor *V,
+                          uint32_t *k_codes, int64_t kc_stride_b, int64_t kc_stride_h,
+                          const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                          int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
+                          int64_t idx_stride_h, int32_t *count, uint16_t *out_host,
+                          void *workspace, size_t ws_bytes, void *stream);
+
+/* Copies the device status word to *flags (host) and clears nothing; synchronises `stream`. */
+int ha_read_device_status(void *workspace, void *stream, uint32_t *flags);
+
+/* Number of kernels this library has launched in this process (host-side counter). */
+uint64_t ha_kernel_launches(void);
+
+const char *ha_status_string(int status);
+const char *ha_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HASHATTN_H */

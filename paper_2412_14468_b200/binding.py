@@ -1,0 +1,248 @@
+"""Thin ctypes binding over libhashattn.so: argument marshalling only.
+
+Every function has the name and semantics of the C entry point declared in include/hashattn.h;
+tensors are torch tensors used purely as device (or pinned host) memory handles.  There is no
+fallback: if the CUDA library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libhashattn.so")
+
+HA_OK = 0
+HA_ERR_INVALID_ARG, HA_ERR_UNSUPPORTED, HA_ERR_WORKSPACE, HA_ERR_CUDA = 1, 2, 3, 4
+HA_DEV_BAD_INDEX, HA_DEV_TIMEOUT = 1, 2
+HIST_BINS = 33
+
+EXPORTS = [
+    "ha_workspace_bytes", "ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn",
+    "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
+    "ha_kernel_launches", "ha_status_string", "ha_version",
+]
+
+
+class ha_shape(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("sm_scale", C.c_float)]
+
+
+class ha_mapping(C.Structure):
+    _fields_ = [("n_kv_heads", C.c_int32), ("in_dim", C.c_int32), ("hid_dim", C.c_int32), ("n_bits", C.c_int32),
+                ("w1", C.c_void_p), ("w2", C.c_void_p), ("w3", C.c_void_p),
+                ("b1", C.c_void_p), ("b2", C.c_void_p), ("b3", C.c_void_p)]
+
+
+class ha_tensor(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_n", C.c_int64)]
+
+
+class HashAttnError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__(f"{fn} failed: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libhashattn.so (built by paper_2412_14468_b200/build.py).  Raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: run `python -m paper_2412_14468_b200.build` "
+                               "(nvcc, sm_100a); this package has no CPU fallback")
+        L = C.CDLL(LIB_PATH)
+        P, I32, I64, SZ = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+        L.ha_workspace_bytes.restype = SZ
+        L.ha_workspace_bytes.argtypes = [P, I32, I32]
+        L.ha_workspace_init.argtypes = [P, SZ, P]
+        L.ha_encode.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, P, P]
+        L.ha_score_topk.argtypes = [P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64, P, P, P, SZ, P]
+        L.ha_gather_attn.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P, SZ, P]
+        L.ha_dense_decode.argtypes = [P, P, P, P, P, I32, P, P, P, SZ, P]
+        L.ha_sparse_decode.argtypes = [P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, P, I64, I64, P,
+                                       P, P, P, SZ, P]
+        L.ha_sparse_decode_host.argtypes = [P, P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64,
+                                            P, P, P, SZ, P]
+        L.ha_read_device_status.argtypes = [P, P, P]
+        L.ha_kernel_launches.restype = C.c_uint64
+        L.ha_status_string.restype = C.c_char_p
+        L.ha_status_string.argtypes = [C.c_int]
+        L.ha_version.restype = C.c_char_p
+        for fn in ("ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn", "ha_dense_decode",
+                   "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status"):
+            getattr(L, fn).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().ha_status_string(int(status)).decode()
+
+
+def ha_version() -> str:
+    return lib().ha_version().decode()
+
+
+def ha_kernel_launches() -> int:
+    return int(lib().ha_kernel_launches())
+
+
+def _check(fn: str, status: int) -> None:
+    if status != HA_OK:
+        raise HashAttnError(fn, status)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype:
+        raise TypeError(f"{name}: expected a CUDA tensor of {dtype}, got {t.dtype} on {t.device}")
+    return t
+
+
+def make_shape(batch: int, n_q_heads: int, n_kv_heads: int, sm_scale: float, head_dim: int = 128) -> ha_shape:
+    return ha_shape(batch, n_q_heads, n_kv_heads, head_dim, float(sm_scale))
+
+
+def make_tensor(t: torch.Tensor) -> ha_tensor:
+    """bf16 [B,H,N,128] tensor (any strides with a contiguous last dim) -> ha_tensor."""
+    _dev(t, torch.bfloat16, "tensor")
+    if t.dim() == 3:                       # [B,H,128]: one token per head
+        t = t.unsqueeze(2)
+    if t.dim() != 4 or t.stride(3) != 1:
+        raise ValueError("expected [B,H,N,128] with a contiguous last dimension")
+    return ha_tensor(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2) if t.shape[2] > 1 else max(t.stride(2), 128))
+
+
+class Mapping:
+    """Device-resident weights of one side's mapping networks + the ha_mapping struct over them."""
+
+    def __init__(self, weights: Dict[str, torch.Tensor]):
+        self.t = {}
+        for k in ("w1", "w2", "w3"):
+            self.t[k] = _dev(weights[k], torch.bfloat16, k).contiguous()
+        for k in ("b1", "b2", "b3"):
+            b = weights.get(k)
+            self.t[k] = None if b is None else _dev(b, torch.float32, k).contiguous()
+        hkv = self.t["w1"].shape[0]
+        assert tuple(self.t["w1"].shape) == (hkv, 128, 128) and tuple(self.t["w2"].shape) == (hkv, 128, 128)
+        assert tuple(self.t["w3"].shape) == (hkv, 128, 32)
+        self.struct = ha_mapping(hkv, 128, 128, 32, _ptr(self.t["w1"]), _ptr(self.t["w2"]), _ptr(self.t["w3"]),
+                                 _ptr(self.t["b1"]), _ptr(self.t["b2"]), _ptr(self.t["b3"]))
+
+    @property
+    def ref(self):
+        return C.byref(self.struct)
+
+
+def ha_workspace_bytes(shape: ha_shape, max_seq_len: int, max_k: int) -> int:
+    n = int(lib().ha_workspace_bytes(C.byref(shape), max_seq_len, max_k))
+    if n == 0:
+        raise HashAttnError("ha_workspace_bytes", HA_ERR_UNSUPPORTED)
+    return n
+
+
+def ha_workspace_init(workspace: torch.Tensor, stream=None) -> None:
+    _check("ha_workspace_init", lib().ha_workspace_init(workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                                       _stream(stream)))
+
+
+def alloc_workspace(shape: ha_shape, max_seq_len: int, max_k: int, device="cuda") -> torch.Tensor:
+    """Convenience for callers and tests: a uint8 workspace of the right size, already initialised."""
+    ws = torch.empty(ha_workspace_bytes(shape, max_seq_len, max_k), dtype=torch.uint8, device=device)
+    ha_workspace_init(ws)
+    return ws
+
+
+def _ws(ws: torch.Tensor):
+    return ws.data_ptr(), ws.numel() * ws.element_size()
+
+
+def ha_encode(mapping: Mapping, heads_per_kv: int, x: torch.Tensor, codes: torch.Tensor,
+              slot: Optional[torch.Tensor] = None, stream=None) -> None:
+    """x: bf16 [B,H,T,128] (or [B,H,128]); codes: int32/uint32-as-int32 [B,H,>=T] (last dim contiguous)."""
+    xt = make_tensor(x)
+    B, H = x.shape[0], x.shape[1]
+    T = 1 if x.dim() == 3 else x.shape[2]
+    _dev(codes, torch.int32, "codes")
+    assert codes.dim() == 3 and codes.stride(2) == 1
+    _check("ha_encode", lib().ha_encode(mapping.ref, heads_per_kv, C.byref(xt), B, H, T, codes.data_ptr(),
+                                        codes.stride(0), codes.stride(1), _ptr(slot), _stream(stream)))
+
+
+def ha_score_topk(shape: ha_shape, q_codes, k_codes, seq_lens, k_per_seq, k_uniform: int, max_seq_len: int,
+                  k_max: int, idx, count, workspace, hist_out=None, stream=None) -> None:
+    """q_codes int32 [B,Hq]; k_codes int32 [B,Hkv,N]; idx int32 [B,Hkv,k_max]; count int32 [B,Hkv]."""
+    p, n = _ws(workspace)
+    _check("ha_score_topk", lib().ha_score_topk(
+        C.byref(shape), q_codes.data_ptr(), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1),
+        seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform, max_seq_len, k_max, idx.data_ptr(), idx.stride(0),
+        idx.stride(1), count.data_ptr(), _ptr(hist_out), p, n, _stream(stream)))
+
+
+def ha_gather_attn(shape: ha_shape, q, K, V, seq_lens, idx, count, k_max: int, out, workspace, lse=None,
+                   stream=None) -> None:
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K), make_tensor(V)
+    _check("ha_gather_attn", lib().ha_gather_attn(
+        C.byref(shape), q.data_ptr(), C.byref(kt), C.byref(vt), seq_lens.data_ptr(), idx.data_ptr(), idx.stride(0),
+        idx.stride(1), count.data_ptr(), k_max, out.data_ptr(), _ptr(lse), p, n, _stream(stream)))
+
+
+def ha_dense_decode(shape: ha_shape, q, K, V, seq_lens, max_seq_len: int, out, workspace, lse=None,
+                    stream=None) -> None:
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K), make_tensor(V)
+    _check("ha_dense_decode", lib().ha_dense_decode(
+        C.byref(shape), q.data_ptr(), C.byref(kt), C.byref(vt), seq_lens.data_ptr(), max_seq_len, out.data_ptr(),
+        _ptr(lse), p, n, _stream(stream)))
+
+
+def ha_sparse_decode(shape: ha_shape, map_q: Mapping, map_k: Optional[Mapping], q, k_new, K, V, k_codes, seq_lens,
+                     k_per_seq, k_uniform: int, max_seq_len: int, k_max: int, q_codes, idx, count, out, workspace,
+                     lse=None, stream=None) -> None:
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K), make_tensor(V)
+    _check("ha_sparse_decode", lib().ha_sparse_decode(
+        C.byref(shape), map_q.ref, None if map_k is None else map_k.ref, q.data_ptr(), _ptr(k_new), C.byref(kt),
+        C.byref(vt), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1), seq_lens.data_ptr(), _ptr(k_per_seq),
+        k_uniform, max_seq_len, k_max, q_codes.data_ptr(), idx.data_ptr(), idx.stride(0), idx.stride(1),
+        count.data_ptr(), out.data_ptr(), _ptr(lse), p, n, _stream(stream)))
+
+
+def ha_sparse_decode_host(shape: ha_shape, map_q: Mapping, map_k: Mapping, q_host, k_new_host, v_new_host, K, V,
+                          k_codes, seq_lens, k_per_seq, k_uniform: int, max_seq_len: int, k_max: int, idx, count,
+                          out_host, workspace, stream=None) -> None:
+    """q_host/k_new_host/v_new_host/out_host: pinned CPU bf16 tensors; everything else on the device."""
+    for t in (q_host, k_new_host, v_new_host, out_host):
+        if t.is_cuda or not t.is_contiguous():
+            raise TypeError("host buffers must be contiguous CPU tensors")
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K), make_tensor(V)
+    _check("ha_sparse_decode_host", lib().ha_sparse_decode_host(
+        C.byref(shape), map_q.ref, map_k.ref, q_host.data_ptr(), k_new_host.data_ptr(), v_new_host.data_ptr(),
+        C.byref(kt), C.byref(vt), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1), seq_lens.data_ptr(),
+        _ptr(k_per_seq), k_uniform, max_seq_len, k_max, idx.data_ptr(), idx.stride(0), idx.stride(1),
+        count.data_ptr(), out_host.data_ptr(), p, n, _stream(stream)))
+
+
+def ha_read_device_status(workspace, stream=None) -> int:
+    flags = C.c_uint32(0)
+    _check("ha_read_device_status", lib().ha_read_device_status(workspace.data_ptr(), _stream(stream), C.byref(flags)))
+    return int(flags.value)

@@ -1,0 +1,278 @@
+// C-ABI entry points: argument validation, workspace carving, kernel sequencing.
+// See include/hashattn.h for the contract of every function.
+#include <atomic>
+
+#include "ha_common.cuh"
+
+namespace ha {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static int check_shape(const ha_shape *s) {
+    if (!s) return HA_ERR_INVALID_ARG;
+    if (s->batch < 0 || s->n_q_heads <= 0 || s->n_kv_heads <= 0) return HA_ERR_INVALID_ARG;
+    if (s->head_dim != kD) return HA_ERR_UNSUPPORTED;
+    if (s->n_q_heads % s->n_kv_heads != 0) return HA_ERR_UNSUPPORTED;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return HA_ERR_UNSUPPORTED;
+    if (s->n_kv_heads > 65535 || s->batch > 65535) return HA_ERR_UNSUPPORTED;
+    if (!(s->sm_scale == s->sm_scale)) return HA_ERR_INVALID_ARG;
+    return HA_OK;
+}
+
+static int check_mapping(const ha_mapping *m, int n_kv_heads) {
+    if (!m || !m->w1 || !m->w2 || !m->w3) return HA_ERR_INVALID_ARG;
+    if (m->in_dim != kD || m->hid_dim != kHid || m->n_bits != kBits) return HA_ERR_UNSUPPORTED;
+    if (m->n_kv_heads <= 0 || (n_kv_heads > 0 && m->n_kv_heads != n_kv_heads)) return HA_ERR_INVALID_ARG;
+    if (((uintptr_t)m->w1 | (uintptr_t)m->w2 | (uintptr_t)m->w3) & 15) return HA_ERR_INVALID_ARG;
+    return HA_OK;
+}
+
+static int check_tensor(const ha_tensor *t) {
+    if (!t || !t->ptr) return HA_ERR_INVALID_ARG;
+    if (((uintptr_t)t->ptr & 15) || (t->stride_b & 7) || (t->stride_h & 7) || (t->stride_n & 7))
+        return HA_ERR_INVALID_ARG;
+    if (t->stride_n < kD) return HA_ERR_INVALID_ARG;
+    return HA_OK;
+}
+
+static int check_workspace(const ha_shape *s, void *ws, size_t bytes, WorkspaceLayout *L) {
+    if (!ws || ((uintptr_t)ws & 255)) return HA_ERR_WORKSPACE;
+    *L = make_layout(s->batch, s->n_q_heads, s->n_kv_heads);
+    if (bytes < L->total) return HA_ERR_WORKSPACE;
+    return HA_OK;
+}
+
+static TensorView view(const ha_tensor *t) {
+    return TensorView{reinterpret_cast<const uint16_t *>(t->ptr), (long long)t->stride_b, (long long)t->stride_h,
+                      (long long)t->stride_n};
+}
+
+static MapView view(const ha_mapping *m) { return MapView{m->w1, m->w2, m->w3, m->b1, m->b2, m->b3}; }
+
+template <typename T>
+static T *ws_ptr(void *ws, size_t off) { return reinterpret_cast<T *>(reinterpret_cast<char *>(ws) + off); }
+
+} // namespace ha
+
+using namespace ha;
+
+#define HA_TRY(expr)                      \
+    do {                                  \
+        int _st = (expr);                 \
+        if (_st != HA_OK) return _st;     \
+    } while (0)
+#define HA_CUDA(expr)                              \
+    do {                                           \
+        if ((expr) != cudaSuccess) return HA_ERR_CUDA; \
+    } while (0)
+
+extern "C" {
+
+size_t ha_workspace_bytes(const ha_shape *shape, int32_t max_seq_len, int32_t max_k) {
+    if (check_shape(shape) != HA_OK || max_seq_len < 0 || max_k < 0) return 0;
+    return make_layout(shape->batch, shape->n_q_heads, shape->n_kv_heads).total;
+}
+
+int ha_workspace_init(void *workspace, size_t ws_bytes, void *stream) {
+    if (!workspace || ((uintptr_t)workspace & 255) || ws_bytes < kHeaderBytes) return HA_ERR_WORKSPACE;
+    HA_CUDA(cudaMemsetAsync(workspace, 0, kHeaderBytes, (cudaStream_t)stream));
+    return HA_OK;
+}
+
+int ha_encode(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, int32_t batch, int32_t n_heads,
+              int32_t n_tokens, uint32_t *codes, int64_t c_stride_b, int64_t c_stride_h, const int32_t *slot,
+              void *stream) {
+    HA_TRY(check_mapping(map, 0));
+    HA_TRY(check_tensor(x));
+    if (!codes || batch < 0 || n_heads <= 0 || n_tokens < 0 || heads_per_kv <= 0) return HA_ERR_INVALID_ARG;
+    if (n_heads % heads_per_kv != 0 || n_heads / heads_per_kv != map->n_kv_heads) return HA_ERR_INVALID_ARG;
+    if (slot && n_tokens != 1) return HA_ERR_INVALID_ARG;
+    if (batch > 65535 || n_heads > 65535) return HA_ERR_UNSUPPORTED;
+    if (batch == 0 || n_tokens == 0) return HA_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n_tokens == 1) {
+        EncodeJob a{};
+        a.x = reinterpret_cast<const uint16_t *>(x->ptr);
+        a.x_sb = x->stride_b; a.x_sh = x->stride_h;
+        a.codes = codes; a.c_sb = c_stride_b; a.c_sh = c_stride_h;
+        a.slot = slot; a.slot_minus_one = 0;
+        a.n_heads = n_heads; a.heads_per_kv = heads_per_kv; a.n_vec = batch * n_heads;
+        a.map = view(map);
+        EncodeJob none{};
+        HA_CUDA(launch_encode_vectors(a, none, st));
+    } else {
+        HA_CUDA(launch_encode_bulk(view(map), heads_per_kv, view(x), batch, n_heads, n_tokens, codes, c_stride_b,
+                                   c_stride_h, st));
+    }
+    return HA_OK;
+}
+
+static int check_score_args(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes,
+                            int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens, int32_t k_uniform,
+                            const int32_t *k_per_seq, int32_t max_seq_len, int32_t k_max, int32_t *idx,
+                            int32_t *count) {
+    HA_TRY(check_shape(shape));
+    if (!q_codes || !k_codes || !seq_lens || !idx || !count) return HA_ERR_INVALID_ARG;
+    if (max_seq_len < 0 || k_max < 0 || (!k_per_seq && k_uniform < 0)) return HA_ERR_INVALID_ARG;
+    if (((uintptr_t)k_codes & 15) || (kc_stride_b & 3) || (kc_stride_h & 3)) return HA_ERR_INVALID_ARG;
+    return HA_OK;
+}
+
+int ha_score_topk(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes, int64_t kc_stride_b,
+                  int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                  int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h,
+                  int32_t *count, int32_t *hist_out, void *workspace, size_t ws_bytes, void *stream) {
+    HA_TRY(check_score_args(shape, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_uniform, k_per_seq,
+                            max_seq_len, k_max, idx, count));
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    if (shape->batch == 0) return HA_OK;
+    HA_CUDA(launch_score_topk(shape->batch, shape->n_q_heads, shape->n_kv_heads, q_codes, k_codes, kc_stride_b,
+                              kc_stride_h, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx, idx_stride_b,
+                              idx_stride_h, count, hist_out, ws_ptr<int32_t>(workspace, L.off_hist),
+                              (cudaStream_t)stream));
+    return HA_OK;
+}
+
+int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K, const ha_tensor *V,
+                   const int32_t *seq_lens, const int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h,
+                   const int32_t *count, int32_t k_max, uint16_t *out, float *lse, void *workspace, size_t ws_bytes,
+                   void *stream) {
+    HA_TRY(check_shape(shape));
+    HA_TRY(check_tensor(K));
+    HA_TRY(check_tensor(V));
+    if (!q || !seq_lens || !idx || !count || !out || k_max < 0) return HA_ERR_INVALID_ARG;
+    if ((uintptr_t)q & 15) return HA_ERR_INVALID_ARG;
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    if (shape->batch == 0) return HA_OK;
+    HA_CUDA(launch_attention(true, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K),
+                             view(V), seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
+                             ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),
+                             ws_ptr<uint32_t>(workspace, 0), (cudaStream_t)stream));
+    return HA_OK;
+}
+
+int ha_dense_decode(const ha_shape *shape, const uint16_t *q, const ha_tensor *K, const ha_tensor *V,
+                    const int32_t *seq_lens, int32_t max_seq_len, uint16_t *out, float *lse, void *workspace,
+                    size_t ws_bytes, void *stream) {
+    HA_TRY(check_shape(shape));
+    HA_TRY(check_tensor(K));
+    HA_TRY(check_tensor(V));
+    if (!q || !seq_lens || !out || max_seq_len < 0) return HA_ERR_INVALID_ARG;
+    if ((uintptr_t)q & 15) return HA_ERR_INVALID_ARG;
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    if (shape->batch == 0) return HA_OK;
+    HA_CUDA(launch_attention(false, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K),
+                             view(V), seq_lens, nullptr, 0, 0, nullptr, max_seq_len, out, lse,
+                             ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),
+                             ws_ptr<uint32_t>(workspace, 0), (cudaStream_t)stream));
+    return HA_OK;
+}
+
+int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k, const uint16_t *q,
+                     const uint16_t *k_new, const ha_tensor *K, const ha_tensor *V, uint32_t *k_codes,
+                     int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
+                     int32_t k_uniform, int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx,
+                     int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse,
+                     void *workspace, size_t ws_bytes, void *stream) {
+    HA_TRY(check_score_args(shape, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_uniform, k_per_seq,
+                            max_seq_len, k_max, idx, count));
+    HA_TRY(check_mapping(map_q, shape->n_kv_heads));
+    if (k_new) HA_TRY(check_mapping(map_k, shape->n_kv_heads));
+    HA_TRY(check_tensor(K));
+    HA_TRY(check_tensor(V));
+    if (!q || !out || ((uintptr_t)q & 15)) return HA_ERR_INVALID_ARG;
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    if (shape->batch == 0) return HA_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int B = shape->batch, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
+
+    EncodeJob jq{};
+    jq.x = q; jq.x_sb = (long long)Hq * kD; jq.x_sh = kD;
+    jq.codes = q_codes; jq.c_sb = Hq; jq.c_sh = 1;
+    jq.slot = nullptr; jq.slot_minus_one = 0;
+    jq.n_heads = Hq; jq.heads_per_kv = Hq / Hkv; jq.n_vec = B * Hq;
+    jq.map = view(map_q);
+    EncodeJob jk{};
+    if (k_new) {
+        jk.x = k_new; jk.x_sb = (long long)Hkv * kD; jk.x_sh = kD;
+        jk.codes = k_codes; jk.c_sb = kc_stride_b; jk.c_sh = kc_stride_h;
+        jk.slot = seq_lens; jk.slot_minus_one = 1;
+        jk.n_heads = Hkv; jk.heads_per_kv = 1; jk.n_vec = B * Hkv;
+        jk.map = view(map_k);
+    }
+    HA_CUDA(launch_encode_vectors(jq, jk, st));
+    HA_CUDA(launch_score_topk(B, Hq, Hkv, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
+                              max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, nullptr,
+                              ws_ptr<int32_t>(workspace, L.off_hist), st));
+    HA_CUDA(launch_attention(true, B, Hq, Hkv, shape->sm_scale, q, view(K), view(V), seq_lens, idx, idx_stride_b,
+                             idx_stride_h, count, k_max, out, lse, ws_ptr<float>(workspace, L.off_part_ml),
+                             ws_ptr<float>(workspace, L.off_part_acc), ws_ptr<uint32_t>(workspace, 0), st));
+    return HA_OK;
+}
+
+int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
+                          const uint16_t *q_host, const uint16_t *k_new_host, const uint16_t *v_new_host,
+                          const ha_tensor *K, const ha_tensor *V, uint32_t *k_codes, int64_t kc_stride_b,
+                          int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                          int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
+                          int64_t idx_stride_h, int32_t *count, uint16_t *out_host, void *workspace, size_t ws_bytes,
+                          void *stream) {
+    HA_TRY(check_shape(shape));
+    if (!q_host || !k_new_host || !v_new_host || !out_host) return HA_ERR_INVALID_ARG;
+    HA_TRY(check_tensor(K));
+    HA_TRY(check_tensor(V));
+    HA_TRY(check_mapping(map_q, shape->n_kv_heads));
+    HA_TRY(check_mapping(map_k, shape->n_kv_heads));
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    HA_TRY(check_score_args(shape, ws_ptr<uint32_t>(workspace, L.off_qcodes), k_codes, kc_stride_b, kc_stride_h,
+                            seq_lens, k_uniform, k_per_seq, max_seq_len, k_max, idx, count));
+    if (shape->batch == 0) return HA_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int B = shape->batch, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
+    uint16_t *dq = ws_ptr<uint16_t>(workspace, L.off_stage_q);
+    uint16_t *dk = ws_ptr<uint16_t>(workspace, L.off_stage_k);
+    uint16_t *dv = ws_ptr<uint16_t>(workspace, L.off_stage_v);
+    uint16_t *dout = ws_ptr<uint16_t>(workspace, L.off_stage_out);
+    uint32_t *dqc = ws_ptr<uint32_t>(workspace, L.off_qcodes);
+    HA_CUDA(cudaMemcpyAsync(dq, q_host, (size_t)B * Hq * kD * 2, cudaMemcpyHostToDevice, st));
+    HA_CUDA(cudaMemcpyAsync(dk, k_new_host, (size_t)B * Hkv * kD * 2, cudaMemcpyHostToDevice, st));
+    HA_CUDA(cudaMemcpyAsync(dv, v_new_host, (size_t)B * Hkv * kD * 2, cudaMemcpyHostToDevice, st));
+    HA_CUDA(launch_append_kv(B, Hkv, dk, dv, view(K), view(V), seq_lens, st));
+    HA_TRY(ha_sparse_decode(shape, map_q, map_k, dq, dk, K, V, k_codes, kc_stride_b, kc_stride_h, seq_lens,
+                            k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx, idx_stride_b, idx_stride_h, count,
+                            dout, nullptr, workspace, ws_bytes, stream));
+    HA_CUDA(cudaMemcpyAsync(out_host, dout, (size_t)B * Hq * kD * 2, cudaMemcpyDeviceToHost, st));
+    HA_CUDA(cudaStreamSynchronize(st));
+    return HA_OK;
+}
+
+int ha_read_device_status(void *workspace, void *stream, uint32_t *flags) {
+    if (!workspace || !flags) return HA_ERR_INVALID_ARG;
+    HA_CUDA(cudaMemcpyAsync(flags, workspace, sizeof(uint32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    HA_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    return HA_OK;
+}
+
+uint64_t ha_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *ha_status_string(int status) {
+    switch (status) {
+        case HA_OK: return "ok";
+        case HA_ERR_INVALID_ARG: return "invalid argument";
+        case HA_ERR_UNSUPPORTED: return "unsupported configuration";
+        case HA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case HA_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown status";
+    }
+}
+
+const char *ha_version(void) { return "hashattn-b200 0.1 (sm_100a)"; }
+
+} // extern "C"

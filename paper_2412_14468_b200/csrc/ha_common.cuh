@@ -1,0 +1,107 @@
+// Internal declarations shared by the translation units of libhashattn (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hashattn.h"
+
+namespace ha {
+
+constexpr int kD = HA_HEAD_DIM;     // head dimension, mapping input width
+constexpr int kHid = 128;           // mapping hidden width
+constexpr int kBits = HA_N_BITS;    // signature width b
+constexpr int kBins = HA_HIST_BINS; // score levels 0..32
+constexpr int kMaxChunks = 128;     // chunks of the code scan per (sequence, KV head)
+constexpr int kMaxSplits = 64;      // split-K partials per query head
+constexpr int kMaxGroup = 8;        // query heads per KV head
+constexpr size_t kHeaderBytes = 256;
+
+// Where each scratch region lives inside the caller's workspace.  Sizes depend on the head counts
+// and the batch only, so a workspace sized once serves every smaller call.
+struct WorkspaceLayout {
+    size_t off_hist;      // i32 [B][Hkv][kMaxChunks][33]   per-chunk score histograms
+    size_t off_part_ml;   // f32 [B][Hq][kMaxSplits][2]     split-K running max (log2 domain) and sum
+    size_t off_part_acc;  // f32 [B][Hq][kMaxSplits][128]   split-K unnormalised outputs
+    size_t off_stage_q;   // bf16 [B][Hq][128]              host-entry staging
+    size_t off_stage_k;   // bf16 [B][Hkv][128]
+    size_t off_stage_v;   // bf16 [B][Hkv][128]
+    size_t off_stage_out; // bf16 [B][Hq][128]
+    size_t off_qcodes;    // u32 [B][Hq]
+    size_t total;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline WorkspaceLayout make_layout(int B, int Hq, int Hkv) {
+    WorkspaceLayout L;
+    size_t o = kHeaderBytes;
+    L.off_hist = o;      o = align_up(o + (size_t)B * Hkv * kMaxChunks * kBins * 4, 256);
+    L.off_part_ml = o;   o = align_up(o + (size_t)B * Hq * kMaxSplits * 2 * 4, 256);
+    L.off_part_acc = o;  o = align_up(o + (size_t)B * Hq * kMaxSplits * kD * 4, 256);
+    L.off_stage_q = o;   o = align_up(o + (size_t)B * Hq * kD * 2, 256);
+    L.off_stage_k = o;   o = align_up(o + (size_t)B * Hkv * kD * 2, 256);
+    L.off_stage_v = o;   o = align_up(o + (size_t)B * Hkv * kD * 2, 256);
+    L.off_stage_out = o; o = align_up(o + (size_t)B * Hq * kD * 2, 256);
+    L.off_qcodes = o;    o = align_up(o + (size_t)B * Hq * 4, 256);
+    L.total = o;
+    return L;
+}
+
+// Tokens of the code cache scanned by one CTA: 2048, doubled until a sequence of max_seq_len
+// tokens needs at most kMaxChunks chunks.
+inline int chunk_tokens_for(int max_seq_len) {
+    long long c = 2048;
+    while ((max_seq_len + c - 1) / c > kMaxChunks) c *= 2;
+    return (int)c;
+}
+
+// Tokens of the index list handled by one CTA of the attention kernel.
+int split_tokens_for(int n_units, int max_items);
+
+void count_launch(int n = 1);
+
+struct TensorView {
+    const uint16_t *ptr;
+    long long sb, sh, sn;
+};
+
+struct MapView {
+    const uint16_t *w1, *w2, *w3;
+    const float *b1, *b2, *b3;
+};
+
+// One batch of vectors to encode: vector v = (b, h) with b = v / n_heads.
+struct EncodeJob {
+    const uint16_t *x;       // bf16, vector (b,h) at x + b*x_sb + h*x_sh
+    long long x_sb, x_sh;
+    uint32_t *codes;         // written at codes + b*c_sb + h*c_sh + slot
+    long long c_sb, c_sh;
+    const int32_t *slot;     // per-sequence slot (device) or NULL = 0
+    int slot_minus_one;      // 1: slot[] holds sequence lengths, write at slot[b] - 1
+    int n_heads, heads_per_kv, n_vec;
+    MapView map;
+};
+
+// ---- launchers (each enqueues kernels on `st` and returns the last CUDA error) ----
+cudaError_t launch_encode_vectors(const EncodeJob &a, const EncodeJob &b, cudaStream_t st);
+cudaError_t launch_encode_bulk(const MapView &map, int heads_per_kv, TensorView x, int B, int H, int T,
+                               uint32_t *codes, long long c_sb, long long c_sh, cudaStream_t st);
+
+cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes,
+                              long long kc_sb, long long kc_sh, const int32_t *seq_lens,
+                              const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max,
+                              int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
+                              int32_t *hist_out, int32_t *ws_hist, cudaStream_t st);
+
+cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale, const uint16_t *q,
+                             TensorView K, TensorView V, const int32_t *seq_lens, const int32_t *idx,
+                             long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
+                             uint16_t *out, float *lse, float *part_ml, float *part_acc,
+                             uint32_t *status, cudaStream_t st);
+
+cudaError_t launch_append_kv(int B, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
+                             TensorView V, const int32_t *seq_lens, cudaStream_t st);
+
+} // namespace ha

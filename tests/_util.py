@@ -1,0 +1,56 @@
+"""Helpers shared by the GPU parity tests: move seeded inputs between torch (device) and the
+numpy views the oracle takes, and run the oracle's pieces per (sequence, KV head)."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2412_14468_b200 import workloads as wl
+
+OUT_TOL = 1e-2      # max-abs tolerance on bf16 attention outputs (fp32 accumulate, bf16 I/O)
+OUT_AIM = 2e-3      # what the kernels are expected to reach on N(0,1) values
+
+
+def u16(t: torch.Tensor) -> np.ndarray:
+    return wl.as_u16(t)
+
+
+def codes_np(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().contiguous().numpy().view(np.uint32)
+
+
+def bf16_to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().to(torch.float64).numpy()
+
+
+def oracle_key_codes(K: torch.Tensor, map_k, lens) -> np.ndarray:
+    """Signature cache [B,Hkv,n_cap] from the oracle's ENCODE."""
+    Ku = u16(K)
+    mk = wl.mapping_numpy(map_k)
+    B, Hkv, n_cap, _ = Ku.shape
+    out = np.zeros((B, Hkv, n_cap), np.uint32)
+    for b in range(B):
+        for g in range(Hkv):
+            n = lens[b]
+            if n:
+                out[b, g, :n] = oracle.encode(Ku[b, g, :n], mk["w1"][g], mk["w2"][g], mk["w3"][g],
+                                              mk["b1"][g], mk["b2"][g], mk["b3"][g])
+    return out
+
+
+def oracle_query_codes(q: torch.Tensor, map_q, n_kv_heads: int) -> np.ndarray:
+    qu = u16(q)
+    mq = wl.mapping_numpy(map_q)
+    B, Hq, _ = qu.shape
+    G = Hq // n_kv_heads
+    out = np.zeros((B, Hq), np.uint32)
+    for b in range(B):
+        for g in range(n_kv_heads):
+            out[b, g * G:(g + 1) * G] = oracle.encode(qu[b, g * G:(g + 1) * G], mq["w1"][g], mq["w2"][g], mq["w3"][g],
+                                                      mq["b1"][g], mq["b2"][g], mq["b3"][g])
+    return out
+
+
+def max_abs_diff_bf16(a_bits: np.ndarray, b_bits: np.ndarray) -> float:
+    return float(np.max(np.abs(oracle.bf16_bits_to_f64(a_bits) - oracle.bf16_bits_to_f64(b_bits)))) if a_bits.size else 0.0

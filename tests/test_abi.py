@@ -1,0 +1,104 @@
+"""Boundary tests that need no GPU: the C-ABI library loads, exports every function the header
+declares, sizes its workspace on the host, and rejects bad arguments with error codes before
+touching CUDA."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2412_14468_b200 import binding as ha
+from paper_2412_14468_b200 import build as ha_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    ha_build.build()
+    return ha.lib()
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "hashattn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ha_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_functions()
+    assert set(names) == set(ha.EXPORTS), (names, ha.EXPORTS)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_binding_has_same_names():
+    for n in ha.EXPORTS:
+        if n == "ha_status_string":
+            assert hasattr(ha, "status_string")
+        else:
+            assert hasattr(ha, n), n
+
+
+def test_version_and_status_strings(lib):
+    assert "sm_100a" in ha.ha_version()
+    assert ha.status_string(0) == "ok"
+    assert len({ha.status_string(i) for i in range(6)}) == 6
+
+
+def test_workspace_bytes_is_host_only_and_monotone_in_batch(lib):
+    s1 = ha.make_shape(1, 32, 8, 0.088)
+    s16 = ha.make_shape(16, 32, 8, 0.088)
+    a, b = ha.ha_workspace_bytes(s1, 32768, 1024), ha.ha_workspace_bytes(s16, 32768, 2048)
+    assert 0 < a < b and a % 256 == 0
+    assert ha.ha_workspace_bytes(s1, 524288, 16384) == a          # sized by head counts and batch only
+    for bad in (ha.make_shape(1, 32, 8, 0.1, head_dim=64), ha.make_shape(1, 30, 8, 0.1), ha.make_shape(1, 24, 8, 0.1),
+                ha.make_shape(-1, 32, 8, 0.1)):
+        assert lib.ha_workspace_bytes(C.byref(bad), 100, 10) == 0
+
+
+def test_bad_arguments_are_rejected_on_the_host(lib):
+    s = ha.make_shape(1, 32, 8, 0.088)
+    fake = 0x1000          # never dereferenced: validation fails first
+    # NULL pointers
+    assert lib.ha_score_topk(C.byref(s), None, fake, 0, 0, fake, None, 4, 16, 4, fake, 0, 0, fake, None, fake, 1 << 30, None) \
+        == ha.HA_ERR_INVALID_ARG
+    # unsupported head_dim
+    s64 = ha.make_shape(1, 32, 8, 0.1, head_dim=64)
+    assert lib.ha_score_topk(C.byref(s64), fake, fake, 0, 0, fake, None, 4, 16, 4, fake, 0, 0, fake, None, fake, 1 << 30, None) \
+        == ha.HA_ERR_UNSUPPORTED
+    # misaligned code cache row stride
+    assert lib.ha_score_topk(C.byref(s), fake, fake, 6, 3, fake, None, 4, 16, 4, fake, 0, 0, fake, None, fake, 1 << 30, None) \
+        == ha.HA_ERR_INVALID_ARG
+    # workspace too small / misaligned / missing
+    assert lib.ha_score_topk(C.byref(s), fake, fake, 16, 16, fake, None, 4, 16, 4, fake, 0, 0, fake, None, fake, 512, None) \
+        == ha.HA_ERR_WORKSPACE
+    assert lib.ha_score_topk(C.byref(s), fake, fake, 16, 16, fake, None, 4, 16, 4, fake, 0, 0, fake, None, fake + 8, 1 << 30, None) \
+        == ha.HA_ERR_WORKSPACE
+    assert lib.ha_score_topk(C.byref(s), fake, fake, 16, 16, fake, None, 4, 16, 4, fake, 0, 0, fake, None, None, 0, None) \
+        == ha.HA_ERR_WORKSPACE
+    # negative budget
+    assert lib.ha_score_topk(C.byref(s), fake, fake, 16, 16, fake, None, -1, 16, 4, fake, 0, 0, fake, None, fake, 1 << 30, None) \
+        == ha.HA_ERR_INVALID_ARG
+    # mapping with the wrong widths / tensors with bad strides
+    m = ha.ha_mapping(8, 128, 64, 32, fake, fake, fake, None, None, None)
+    t = ha.ha_tensor(fake, 1024, 128, 128)
+    assert lib.ha_encode(C.byref(m), 1, C.byref(t), 1, 8, 1, fake, 8, 1, None, None) == ha.HA_ERR_UNSUPPORTED
+    m = ha.ha_mapping(8, 128, 128, 32, fake, fake, fake, None, None, None)
+    tbad = ha.ha_tensor(fake, 1024, 128, 100)
+    assert lib.ha_encode(C.byref(m), 1, C.byref(tbad), 1, 8, 1, fake, 8, 1, None, None) == ha.HA_ERR_INVALID_ARG
+    assert lib.ha_encode(C.byref(m), 3, C.byref(t), 1, 8, 1, fake, 8, 1, None, None) == ha.HA_ERR_INVALID_ARG
+    assert lib.ha_gather_attn(C.byref(s), fake, C.byref(tbad), C.byref(t), fake, fake, 0, 0, fake, 4, fake, None, fake, 1 << 30, None) \
+        == ha.HA_ERR_INVALID_ARG
+    assert lib.ha_dense_decode(C.byref(s), None, C.byref(t), C.byref(t), fake, 16, fake, None, fake, 1 << 30, None) \
+        == ha.HA_ERR_INVALID_ARG
+    # empty batch is a no-op that succeeds without touching the device
+    s0 = ha.make_shape(0, 32, 8, 0.088)
+    assert lib.ha_dense_decode(C.byref(s0), fake, C.byref(t), C.byref(t), fake, 16, fake, None, fake, 1 << 30, None) == ha.HA_OK
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(ha, "_lib", None)
+    monkeypatch.setattr(ha, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        ha.lib()

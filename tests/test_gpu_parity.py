@@ -1,0 +1,345 @@
+"""GPU parity: every C-ABI entry point against the CPU oracle on the same seeded inputs.
+Codes, scores (through the histogram), counts and index sets must match bit for bit; attention
+outputs within 1e-2 max-abs (fp32 accumulate, bf16 I/O)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2412_14468_b200 import binding as ha
+from paper_2412_14468_b200 import workloads as wl
+from tests._util import OUT_AIM, OUT_TOL, bf16_to_f64, codes_np, max_abs_diff_bf16, oracle_key_codes, \
+    oracle_query_codes, u16
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _mapping(hkv, seed):
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed)
+    return wl.make_mapping(hkv, g, DEV)
+
+
+# ---------------------------------------------------------------------------- ENCODE
+
+@pytest.mark.parametrize("T", [1, 2, 63, 64, 65, 200])
+def test_encode_bulk_and_single_bit_exact(T):
+    B, H = 2, 4
+    mp = _mapping(H, 100 + T)
+    x = torch.randn(B, H, T, 128, device=DEV, generator=torch.Generator(DEV).manual_seed(T)).to(torch.bfloat16)
+    codes = torch.zeros(B, H, T + 3, dtype=torch.int32, device=DEV)
+    ha.ha_encode(ha.Mapping(mp), 1, x, codes)
+    torch.cuda.synchronize()
+    got = codes_np(codes)
+    m = wl.mapping_numpy(mp)
+    xu = u16(x)
+    for b in range(B):
+        for h in range(H):
+            exp = oracle.encode(xu[b, h], m["w1"][h], m["w2"][h], m["w3"][h], m["b1"][h], m["b2"][h], m["b3"][h])
+            assert np.array_equal(got[b, h, :T], exp)
+            assert not got[b, h, T:].any()          # nothing written past the tokens
+
+
+def test_encode_query_side_group_sharing_and_append_slot():
+    B, Hq, Hkv = 3, 8, 2
+    mp = _mapping(Hkv, 7)
+    q = torch.randn(B, Hq, 128, device=DEV).to(torch.bfloat16)
+    qc = torch.zeros(B, Hq, 1, dtype=torch.int32, device=DEV)
+    ha.ha_encode(ha.Mapping(mp), Hq // Hkv, q, qc)
+    assert np.array_equal(codes_np(qc)[:, :, 0], oracle_query_codes(q, mp, Hkv))
+    # append: code of k_new lands in slot[b]; a negative slot skips the sequence
+    k_new = torch.randn(B, Hkv, 128, device=DEV).to(torch.bfloat16)
+    cache = torch.full((B, Hkv, 40), 0x55, dtype=torch.int32, device=DEV)
+    slot = torch.tensor([0, 39, -1], dtype=torch.int32, device=DEV)
+    ha.ha_encode(ha.Mapping(mp), 1, k_new, cache, slot=slot)
+    got = codes_np(cache)
+    exp = oracle_query_codes(k_new, mp, Hkv)        # heads_per_kv = 1 on the key side
+    assert np.array_equal(got[0, :, 0], exp[0]) and np.array_equal(got[1, :, 39], exp[1])
+    got[0, :, 0] = 0x55
+    got[1, :, 39] = 0x55
+    assert np.all(got == 0x55)
+
+
+def test_encode_without_biases_and_strided_input():
+    H, T = 2, 70
+    mp = _mapping(H, 9)
+    nb = {k: v for k, v in mp.items() if k.startswith("w")}
+    big = torch.randn(1, T, H, 256, device=DEV).to(torch.bfloat16)
+    x = big[..., :128].permute(0, 2, 1, 3)           # [1,H,T,128] view with token stride H*256
+    codes = torch.zeros(1, H, T, dtype=torch.int32, device=DEV)
+    ha.ha_encode(ha.Mapping(nb), 1, x, codes)
+    m = wl.mapping_numpy(nb)
+    xu = u16(x.contiguous())
+    for h in range(H):
+        assert np.array_equal(codes_np(codes)[0, h], oracle.encode(xu[0, h], m["w1"][h], m["w2"][h], m["w3"][h]))
+
+
+# ---------------------------------------------------------------------------- SCORE + TOPK
+
+def _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, k_uniform=None):
+    B = len(lens)
+    n_cap = kc_np.shape[2]
+    k_max = max(max(ks), 1)
+    shape = ha.make_shape(B, Hq, Hkv, 1.0)
+    ws = ha.alloc_workspace(shape, n_cap, k_max)
+    qc = torch.from_numpy(qc_np.view(np.int32)).to(DEV)
+    kc = torch.from_numpy(kc_np.view(np.int32)).to(DEV)
+    sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    kp = None if k_uniform is not None else torch.tensor(ks, dtype=torch.int32, device=DEV)
+    idx = torch.full((B, Hkv, k_max), -7, dtype=torch.int32, device=DEV)
+    cnt = torch.full((B, Hkv), -7, dtype=torch.int32, device=DEV)
+    hist = torch.full((B, Hkv, 33), -7, dtype=torch.int32, device=DEV)
+    ha.ha_score_topk(shape, qc, kc, sl, kp, k_uniform if k_uniform is not None else 0, n_cap, k_max, idx, cnt, ws,
+                     hist_out=hist)
+    torch.cuda.synchronize()
+    return idx.cpu().numpy(), cnt.cpu().numpy(), hist.cpu().numpy()
+
+
+def _check_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, **kw):
+    idx, cnt, hist = _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, **kw)
+    G = Hq // Hkv
+    for b, (n, k) in enumerate(zip(lens, ks)):
+        for g in range(Hkv):
+            s = oracle.score(qc_np[b, g * G:(g + 1) * G], kc_np[b, g, :n])
+            exp = oracle.topk(s, k)
+            assert cnt[b, g] == len(exp) == min(k, n)
+            assert np.array_equal(idx[b, g, :len(exp)], exp), (b, g, n, k)
+            assert np.all(idx[b, g, len(exp):] == -1)
+            assert np.array_equal(hist[b, g], np.bincount(s, minlength=33))
+
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_score_topk_sizes_ragged_tail_and_budgets(G):
+    rng = np.random.default_rng(5 + G)
+    Hkv, Hq = 2, 2 * G
+    lens = [0, 1, 5, 1023, 2047, 2048, 2049, 5000, 70001]
+    n_cap = 70004
+    kc = rng.integers(0, 2 ** 32, size=(len(lens), Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    qc = rng.integers(0, 2 ** 32, size=(len(lens), Hq), dtype=np.uint64).astype(np.uint32)
+    for ks in ([n // 16 for n in lens], [n for n in lens], [n + 5 for n in lens], [1] * len(lens), [0] * len(lens),
+               [min(n, 777) for n in lens]):
+        _check_score_topk(qc, kc, lens, ks, Hq, Hkv)
+
+
+def test_score_topk_heavy_ties():
+    rng = np.random.default_rng(11)
+    Hq, Hkv, n = 8, 2, 9000
+    # few distinct codes -> huge tie blocks; all-equal codes -> lowest indices win
+    pool = rng.integers(0, 2 ** 32, size=6, dtype=np.uint64).astype(np.uint32)
+    kc = pool[rng.integers(0, 6, size=(3, Hkv, n))]
+    kc[2] = 0xABCDEF01
+    qc = rng.integers(0, 2 ** 32, size=(3, Hq), dtype=np.uint64).astype(np.uint32)
+    qc[1, :4] = pool[0]                                # exact matches: score 32
+    for k in (1, 100, 1500, 4500, 8999):
+        _check_score_topk(qc, kc, [n, n - 13, n], [k, k, k], Hq, Hkv, k_uniform=k)
+
+
+def test_score_topk_biased_bits_like_random_init_mappings():
+    # narrow score distribution (many tokens on the threshold level), as random-init ReLU nets give
+    rng = np.random.default_rng(12)
+    Hq, Hkv, n = 32, 8, 32768
+    p1 = rng.uniform(0.02, 0.98, size=32)
+    bits = rng.random((1, Hkv, n, 32)) < p1
+    kc = (bits * (1 << np.arange(32, dtype=np.uint64))).sum(-1).astype(np.uint32)
+    qbits = rng.random((1, Hq, 32)) < p1
+    qc = (qbits * (1 << np.arange(32, dtype=np.uint64))).sum(-1).astype(np.uint32)
+    _check_score_topk(qc, kc, [n], [1024], Hq, Hkv)
+
+
+# ---------------------------------------------------------------------------- GATHER-ATT / dense
+
+def _attn_inputs(B, Hq, Hkv, n_cap, seed, scale=1.0):
+    g = torch.Generator(DEV).manual_seed(seed)
+    q = torch.randn(B, Hq, 128, device=DEV, generator=g).to(torch.bfloat16)
+    K = (scale * torch.randn(B, Hkv, n_cap, 128, device=DEV, generator=g)).to(torch.bfloat16)
+    V = torch.randn(B, Hkv, n_cap, 128, device=DEV, generator=g).to(torch.bfloat16)
+    return q, K, V
+
+
+def _check_gather(q, K, V, lens, idx_np, cnt_np, sm_scale, expect_flag=0):
+    B, Hq, _ = q.shape
+    Hkv = K.shape[1]
+    G = Hq // Hkv
+    k_max = idx_np.shape[2]
+    shape = ha.make_shape(B, Hq, Hkv, sm_scale)
+    ws = ha.alloc_workspace(shape, K.shape[2], k_max)
+    out = torch.full((B, Hq, 128), 7.0, dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((B, Hq), 7.0, dtype=torch.float32, device=DEV)
+    ha.ha_gather_attn(shape, q, K, V, torch.tensor(lens, dtype=torch.int32, device=DEV),
+                      torch.from_numpy(idx_np).to(DEV), torch.from_numpy(cnt_np).to(DEV), k_max, out, ws, lse=lse)
+    assert ha.ha_read_device_status(ws) == expect_flag
+    qu, Ku, Vu, ou = u16(q), u16(K), u16(V), u16(out)
+    lse_np = lse.cpu().numpy()
+    worst = 0.0
+    for b in range(B):
+        for h in range(Hq):
+            g = h // G
+            eo, el, _ = oracle.gather_attn(qu[b, h], Ku[b, g], Vu[b, g], idx_np[b, g, :cnt_np[b, g]],
+                                           sm_scale=sm_scale, n_valid=lens[b])
+            worst = max(worst, max_abs_diff_bf16(ou[b, h], eo))
+            if math.isinf(el):
+                assert lse_np[b, h] == -math.inf and not ou[b, h].any()
+            else:
+                assert abs(lse_np[b, h] - el) < 1e-3 * max(1.0, abs(el))
+    assert worst <= OUT_TOL
+    return worst
+
+
+@pytest.mark.parametrize("G", [1, 4, 8])
+def test_gather_attn_random_lists(G):
+    Hkv, Hq, n_cap = 2, 2 * G, 3000
+    B = 3
+    lens = [3000, 1777, 64]
+    q, K, V = _attn_inputs(B, Hq, Hkv, n_cap, 40 + G)
+    rng = np.random.default_rng(41)
+    k_max = 700
+    idx = np.full((B, Hkv, k_max), -1, np.int32)
+    cnt = np.zeros((B, Hkv), np.int32)
+    for b in range(B):
+        for g in range(Hkv):
+            c = [700, 333, 17][b] if g == 0 else [1, 64, 0][b]
+            c = min(c, lens[b])
+            cnt[b, g] = c
+            idx[b, g, :c] = np.sort(rng.choice(lens[b], size=c, replace=False))
+    worst = _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128))
+    assert worst <= OUT_AIM
+
+
+def test_gather_attn_padding_invalid_and_unsorted_indices():
+    Hq, Hkv, n_cap = 8, 2, 500
+    q, K, V = _attn_inputs(1, Hq, Hkv, n_cap, 50, scale=2.0)
+    idx = np.full((1, Hkv, 64), -1, np.int32)
+    idx[0, 0, :10] = [499, 3, 3, -1, 250, 7, -1, 0, 42, 499]       # padding inside, duplicates, unsorted
+    idx[0, 1, :6] = [5, 400, 450, 10, 399, 1]                       # 400, 450 are beyond seq_len = 400
+    cnt = np.array([[10, 6]], np.int32)
+    _check_gather(q, K, V, [400 + 100], idx[:, :, :], np.array([[10, 0]], np.int32), 0.2)
+    _check_gather(q, K, V, [400], np.where(idx == 499, 399, idx), cnt, 0.2, expect_flag=ha.HA_DEV_BAD_INDEX)
+
+
+def test_single_index_returns_value_row_exactly_and_k_equals_n_is_dense():
+    Hq, Hkv, n = 8, 2, 1234
+    q, K, V = _attn_inputs(1, Hq, Hkv, n, 60)
+    shape = ha.make_shape(1, Hq, Hkv, 1.0 / math.sqrt(128))
+    ws = ha.alloc_workspace(shape, n, n)
+    sl = torch.tensor([n], dtype=torch.int32, device=DEV)
+    one = torch.tensor([[[777], [5]]], dtype=torch.int32, device=DEV)
+    out = torch.zeros(1, Hq, 128, dtype=torch.bfloat16, device=DEV)
+    ha.ha_gather_attn(shape, q, K, V, sl, one, torch.ones(1, Hkv, dtype=torch.int32, device=DEV), 1, out, ws)
+    assert torch.equal(out[0, :4], V[0, 0, 777].expand(4, 128)) and torch.equal(out[0, 4:], V[0, 1, 5].expand(4, 128))
+    # k = n through the gather kernel equals the dense kernel equals the oracle
+    full = torch.arange(n, dtype=torch.int32, device=DEV).expand(1, Hkv, n).contiguous()
+    cnt = torch.full((1, Hkv), n, dtype=torch.int32, device=DEV)
+    o_sparse = torch.zeros_like(out)
+    o_dense = torch.zeros_like(out)
+    l_s = torch.zeros(1, Hq, device=DEV)
+    l_d = torch.zeros(1, Hq, device=DEV)
+    ha.ha_gather_attn(shape, q, K, V, sl, full, cnt, n, o_sparse, ws, lse=l_s)
+    ha.ha_dense_decode(shape, q, K, V, sl, n, o_dense, ws, lse=l_d)
+    assert float((o_sparse.float() - o_dense.float()).abs().max()) <= OUT_AIM
+    assert float((l_s - l_d).abs().max()) < 1e-4
+    qu, Ku, Vu = u16(q), u16(K), u16(V)
+    for h in range(Hq):
+        eo, el, _ = oracle.dense(qu[0, h], Ku[0, h // 4], Vu[0, h // 4])
+        assert max_abs_diff_bf16(u16(o_dense)[0, h], eo) <= OUT_AIM
+        assert abs(float(l_d[0, h]) - el) < 1e-3
+
+
+@pytest.mark.parametrize("lens", [[1], [33, 4097], [20000, 1, 0]])
+def test_dense_decode_matches_oracle(lens):
+    Hq, Hkv = 8, 2
+    B, n_cap = len(lens), max(max(lens), 1)
+    q, K, V = _attn_inputs(B, Hq, Hkv, n_cap, 70 + len(lens))
+    shape = ha.make_shape(B, Hq, Hkv, 1.0 / math.sqrt(128))
+    ws = ha.alloc_workspace(shape, n_cap, n_cap)
+    out = torch.full((B, Hq, 128), 3.0, dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(B, Hq, device=DEV)
+    ha.ha_dense_decode(shape, q, K, V, torch.tensor(lens, dtype=torch.int32, device=DEV), n_cap, out, ws, lse=lse)
+    qu, Ku, Vu, ou = u16(q), u16(K), u16(V), u16(out)
+    for b in range(B):
+        for h in range(Hq):
+            eo, el, _ = oracle.dense(qu[b, h], Ku[b, h // 4], Vu[b, h // 4], n=lens[b])
+            assert max_abs_diff_bf16(ou[b, h], eo) <= OUT_AIM
+            if lens[b] == 0:
+                assert float(lse[b, h]) == -math.inf
+            else:
+                assert abs(float(lse[b, h]) - el) < 1e-3
+
+
+# ---------------------------------------------------------------------------- whole step
+
+def _run_step(w, host=False):
+    cfg = w["cfg"]
+    B, Hq, Hkv = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
+    ws = ha.alloc_workspace(shape, w["n_cap"], w["k_max"])
+    mq, mk = ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"])
+    kc = torch.zeros(B, Hkv, (w["n_cap"] + 3) // 4 * 4, dtype=torch.int32, device=DEV)
+    ha.ha_encode(mk, 1, w["K"], kc)                                  # signature cache of the prompt
+    for b in range(B):
+        if w["lens"][b] > 0:
+            kc[b, :, w["lens"][b] - 1] = 0x7FFFFFFF                  # the step must rewrite the appended slot
+    qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+    idx = torch.zeros(B, Hkv, w["k_max"], dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=DEV)
+    out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(B, Hq, device=DEV)
+    if host:
+        K2, V2 = w["K"].clone(), w["V"].clone()
+        for b in range(B):
+            if w["lens"][b] > 0:
+                K2[b, :, w["lens"][b] - 1] = 0
+                V2[b, :, w["lens"][b] - 1] = 0
+        hq, hk, hv = (w[x].cpu().pin_memory() for x in ("q", "k_new", "v_new"))
+        ho = torch.zeros(B, Hq, 128, dtype=torch.bfloat16).pin_memory()
+        ha.ha_sparse_decode_host(shape, mq, mk, hq, hk, hv, K2, V2, kc, w["seq_lens"], w["k_per_seq"], 0, w["n_cap"],
+                                 w["k_max"], idx, cnt, ho, ws)
+        assert torch.equal(K2, w["K"]) and torch.equal(V2, w["V"])   # the new rows were appended in place
+        out = ho.to(DEV)
+        lse = None
+    else:
+        ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
+                            w["n_cap"], w["k_max"], qc, idx, cnt, out, ws, lse=lse)
+    torch.cuda.synchronize()
+    assert ha.ha_read_device_status(ws) == 0
+    return dict(kc=kc, qc=qc, idx=idx, cnt=cnt, out=out, lse=lse)
+
+
+@pytest.mark.parametrize("cfg", [
+    wl.Config("tiny-ragged", 50, 3, [300, 2049, 1], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8),
+    wl.Config("tiny-g1", 51, 2, [700, 64], 32, 0.05, n_q_heads=2, n_kv_heads=2, sparsity=8),
+    wl.CONFIGS["c1"],
+])
+def test_sparse_decode_step_matches_oracle(cfg):
+    w = wl.make_workload(cfg, DEV)
+    r = _run_step(w)
+    Kc = oracle_key_codes(w["K"], w["map_k"], w["lens"])
+    B, Hkv = cfg.batch, cfg.n_kv_heads
+    n_cap = w["n_cap"]
+    assert np.array_equal(codes_np(r["kc"])[:, :, :n_cap] * (np.arange(n_cap)[None, None, :] < np.array(w["lens"])[:, None, None]),
+                          Kc)
+    ref = oracle.decode_step(u16(w["q"]), u16(w["k_new"]), u16(w["K"]), u16(w["V"]), Kc.copy(),
+                             wl.mapping_numpy(w["map_q"]), wl.mapping_numpy(w["map_k"]), w["lens"], w["ks"],
+                             sm_scale=w["sm_scale"], n_threads=4)
+    assert np.array_equal(codes_np(r["qc"]), ref["qcodes"])
+    assert np.array_equal(r["cnt"].cpu().numpy(), ref["count"])
+    assert np.array_equal(r["idx"].cpu().numpy(), ref["idx"])
+    assert max_abs_diff_bf16(u16(r["out"]), ref["out"]) <= OUT_AIM
+    assert np.max(np.abs(r["lse"].cpu().numpy().astype(np.float64) - ref["lse"])) < 1e-3
+    # the host-buffer entry point gives the same result
+    rh = _run_step(w, host=True)
+    assert torch.equal(rh["idx"], r["idx"]) and torch.equal(rh["out"], r["out"])
+
+
+def test_k_equals_n_sparse_step_equals_dense_kernel():
+    cfg = wl.Config("k=n", 52, 2, [1500, 900], None, 0.0, n_q_heads=8, n_kv_heads=2, sparsity=1)
+    w = wl.make_workload(cfg, DEV)
+    r = _run_step(w)
+    shape = ha.make_shape(2, 8, 2, w["sm_scale"])
+    ws = ha.alloc_workspace(shape, w["n_cap"], w["n_cap"])
+    dense = torch.zeros_like(r["out"])
+    ha.ha_dense_decode(shape, w["q"], w["K"], w["V"], w["seq_lens"], w["n_cap"], dense, ws)
+    assert float((dense.float() - r["out"].float()).abs().max()) <= OUT_AIM
+    assert r["cnt"].cpu().tolist() == [[1500, 1500], [900, 900]]
