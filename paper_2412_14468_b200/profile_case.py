@@ -1,0 +1,59 @@
+"""Small, self-ending run of the decode path for profiler captures (ncu) and quick timing.
+
+    python -m paper_2412_14468_b200.profile_case --config c3 --batch 4 --steps 3
+
+Runs `steps` plain (un-graphed) layer-steps on one replica; inputs are larger than L2 for c3/c4
+style shapes but stay within a few GB.  Prints the CUDA-event time per step."""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+
+import torch
+
+from . import binding as ha
+from . import workloads as wl
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default="c3")
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--dense", action="store_true", help="also run the dense comparator each step")
+    args = ap.parse_args()
+    cfg = wl.CONFIGS[args.config]
+    if args.batch is not None:
+        cfg = dataclasses.replace(cfg, batch=args.batch)
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    w = wl.make_workload(cfg, dev)
+    B, Hq, Hkv = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
+    ws = ha.alloc_workspace(shape, w["n_cap"], w["k_max"], device=dev)
+    mq, mk = ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"])
+    kc = torch.zeros(B, Hkv, (w["n_cap"] + 3) // 4 * 4, dtype=torch.int32, device=dev)
+    ha.ha_encode(mk, 1, w["K"], kc)
+    qc = torch.zeros(B, Hq, dtype=torch.int32, device=dev)
+    idx = torch.zeros(B, Hkv, w["k_max"], dtype=torch.int32, device=dev)
+    cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
+    out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+    for s in range(args.steps):
+        flush.fill_(s & 0xFF)                      # evict L2 between steps
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
+                            w["n_cap"], w["k_max"], qc, idx, cnt, out, ws)
+        e1.record()
+        if args.dense:
+            ha.ha_dense_decode(shape, w["q"], w["K"], w["V"], w["seq_lens"], w["n_cap"], out, ws)
+        torch.cuda.synchronize()
+        print(f"step {s}: {e0.elapsed_time(e1) * 1e3:.1f} us (plain launches, L2 flushed)")
+    assert ha.ha_read_device_status(ws) == 0
+    print("algorithmic bytes per step:", wl.algorithmic_bytes(w["lens"], w["ks"], Hq, Hkv))
+
+
+if __name__ == "__main__":
+    main()
