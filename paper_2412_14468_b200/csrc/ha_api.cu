@@ -17,6 +17,7 @@ static int check_shape(const ha_shape *s) {
     const int G = s->n_q_heads / s->n_kv_heads;
     if (G != 1 && G != 2 && G != 4 && G != 8) return HA_ERR_UNSUPPORTED;
     if (s->n_kv_heads > 65535 || s->batch > 65535) return HA_ERR_UNSUPPORTED;
+    if ((long long)s->n_kv_heads * s->batch > kMaxUnits) return HA_ERR_UNSUPPORTED;
     if (!(s->sm_scale == s->sm_scale)) return HA_ERR_INVALID_ARG;
     return HA_OK;
 }
@@ -77,7 +78,10 @@ size_t ha_workspace_bytes(const ha_shape *shape, int32_t max_seq_len, int32_t ma
 
 int ha_workspace_init(void *workspace, size_t ws_bytes, void *stream) {
     if (!workspace || ((uintptr_t)workspace & 255) || ws_bytes < kHeaderBytes) return HA_ERR_WORKSPACE;
-    HA_CUDA(cudaMemsetAsync(workspace, 0, kHeaderBytes, (cudaStream_t)stream));
+    // status word and the ticket counters (which every call leaves at zero again)
+    size_t n = kHeaderBytes + (size_t)kMaxUnits * 4;
+    if (n > ws_bytes) n = ws_bytes;
+    HA_CUDA(cudaMemsetAsync(workspace, 0, n, (cudaStream_t)stream));
     return HA_OK;
 }
 
@@ -151,7 +155,8 @@ int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
     HA_CUDA(launch_attention(true, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K),
                              view(V), seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
                              ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),
-                             ws_ptr<uint32_t>(workspace, 0), (cudaStream_t)stream));
+                             ws_ptr<int32_t>(workspace, L.off_tickets), ws_ptr<uint32_t>(workspace, 0),
+                             (cudaStream_t)stream));
     return HA_OK;
 }
 
@@ -169,7 +174,8 @@ int ha_dense_decode(const ha_shape *shape, const uint16_t *q, const ha_tensor *K
     HA_CUDA(launch_attention(false, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K),
                              view(V), seq_lens, nullptr, 0, 0, nullptr, max_seq_len, out, lse,
                              ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),
-                             ws_ptr<uint32_t>(workspace, 0), (cudaStream_t)stream));
+                             ws_ptr<int32_t>(workspace, L.off_tickets), ws_ptr<uint32_t>(workspace, 0),
+                             (cudaStream_t)stream));
     return HA_OK;
 }
 
@@ -212,7 +218,8 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
                               ws_ptr<int32_t>(workspace, L.off_hist), st));
     HA_CUDA(launch_attention(true, B, Hq, Hkv, shape->sm_scale, q, view(K), view(V), seq_lens, idx, idx_stride_b,
                              idx_stride_h, count, k_max, out, lse, ws_ptr<float>(workspace, L.off_part_ml),
-                             ws_ptr<float>(workspace, L.off_part_acc), ws_ptr<uint32_t>(workspace, 0), st));
+                             ws_ptr<float>(workspace, L.off_part_acc), ws_ptr<int32_t>(workspace, L.off_tickets),
+                             ws_ptr<uint32_t>(workspace, 0), st));
     return HA_OK;
 }
 

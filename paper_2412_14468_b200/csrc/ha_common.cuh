@@ -16,11 +16,13 @@ constexpr int kBins = HA_HIST_BINS; // score levels 0..32
 constexpr int kMaxChunks = 128;     // chunks of the code scan per (sequence, KV head)
 constexpr int kMaxSplits = 64;      // split-K partials per query head
 constexpr int kMaxGroup = 8;        // query heads per KV head
-constexpr size_t kHeaderBytes = 256;
+constexpr size_t kHeaderBytes = 256;   // device status word (+ padding)
+constexpr int kMaxUnits = 65536;       // (sequence, KV head) pairs: bounds the ticket region
 
 // Where each scratch region lives inside the caller's workspace.  Sizes depend on the head counts
 // and the batch only, so a workspace sized once serves every smaller call.
 struct WorkspaceLayout {
+    size_t off_tickets;   // i32 [B][Hkv]  arrival counters of the split-K merge; zero between calls
     size_t off_hist;      // i32 [B][Hkv][kMaxChunks][33]   per-chunk score histograms
     size_t off_part_ml;   // f32 [B][Hq][kMaxSplits][2]     split-K running max (log2 domain) and sum
     size_t off_part_acc;  // f32 [B][Hq][kMaxSplits][128]   split-K unnormalised outputs
@@ -37,6 +39,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline WorkspaceLayout make_layout(int B, int Hq, int Hkv) {
     WorkspaceLayout L;
     size_t o = kHeaderBytes;
+    L.off_tickets = o;   o = align_up(o + (size_t)B * Hkv * 4, 256);
     L.off_hist = o;      o = align_up(o + (size_t)B * Hkv * kMaxChunks * kBins * 4, 256);
     L.off_part_ml = o;   o = align_up(o + (size_t)B * Hq * kMaxSplits * 2 * 4, 256);
     L.off_part_acc = o;  o = align_up(o + (size_t)B * Hq * kMaxSplits * kD * 4, 256);
@@ -98,7 +101,7 @@ cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, c
 cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale, const uint16_t *q,
                              TensorView K, TensorView V, const int32_t *seq_lens, const int32_t *idx,
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
-                             uint16_t *out, float *lse, float *part_ml, float *part_acc,
+                             uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
                              uint32_t *status, cudaStream_t st);
 
 cudaError_t launch_append_kv(int B, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,

@@ -38,10 +38,10 @@ def main():
     idx = torch.zeros(B, Hkv, w["k_max"], dtype=torch.int32, device=dev)
     cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
     out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=dev)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
     torch.cuda.synchronize()
     for s in range(args.steps):
-        flush.fill_(s & 0xFF)                      # evict L2 between steps
+        _ = int(flush.sum())                       # read 256 MB: evicts L2 and leaves only clean lines
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
