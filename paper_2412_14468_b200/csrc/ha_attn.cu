@@ -1,22 +1,22 @@
-// GATHER-ATT (Section 4) and dense single-query SDPA (Section 3.1) as one split-K flash-decode
-// kernel.  A CTA owns a slice of the index list (or of the sequence) of one (sequence, KV head) and
-// serves all G query heads of that KV head, so every selected K/V row is read from HBM once; the
-// 256-byte bf16 rows are read in place through the indices (Section 4.4: no gather into a buffer).
+// GATHER-ATT (Section 4) and dense single-query SDPA (Section 3.1) as one persistent split-K
+// flash-decode kernel.  The 256-byte bf16 K/V rows are read in place through the indices
+// (Section 4.4: no gather into a buffer) and every row is read from HBM once for all G query heads
+// of its KV head.
 //
-// Data path per warp and per block of 16 list entries (8 KB of K/V rows, all loads issued before
-// the first use so that a warp keeps 8 KB in flight):
-//   * K rows go straight from global memory into mma.sync B fragments: four lanes share a row and
-//     each takes 16-byte chunks, which fixes a permutation of the head dimension; the query
-//     fragments are loaded with the same permutation, so the dot products are unchanged.
-//   * S[head][token] = Q K^T on the tensor cores (m16n8k16, bf16 in, fp32 out), online softmax in
-//     fp32 in the log2 domain; the C fragment of S is already the B fragment of P^T.
-//   * V rows go from global memory into A fragments of V^T (two tokens are paired per register
-//     with a byte permute), O^T[d][head] += V^T P^T with P split into bf16 hi + lo parts so that
-//     the weights keep ~16 bits.
-// The slices' states (running max, sum, unnormalised output) are merged by whichever CTA of the
-// (sequence, KV head) finishes last (a ticket counter in the workspace; nobody waits), which
-// normalises and rounds once to bf16.  The arithmetic intensity is ~4 FLOP/B: the kernel is bound
-// by HBM, the tensor cores only keep the instruction count out of the way.
+// Scheduling.  The index lists of all (sequence, KV head) units are cut into blocks of 16 entries;
+// the blocks of all units, laid end to end, are divided evenly over a fixed number of CTAs (two per
+// SM), whatever the batch size and however ragged the lists are.  A CTA walks its range unit by
+// unit; where a unit is shared by several CTAs each publishes its running (max, sum, output) state
+// and the CTA that arrives last (a ticket counter; nobody waits) merges them, normalises and
+// rounds once to bf16.
+//
+// Data path per warp: a private ring in shared memory holds kStages blocks of rows; rows are
+// fetched with 16-byte cp.async (a half-warp per 256-byte row) two blocks ahead of their use, the
+// list entries one block further ahead.  S[head][token] = Q K^T and O^T[d][head] += V^T P^T run on
+// the tensor cores from ldmatrix fragments (mma.sync m16n8k16, bf16 in, fp32 accumulate; P is
+// split into bf16 hi + lo parts so the weights keep ~16 bits), softmax online in fp32 in the log2
+// domain.  At ~4 FLOP/B the kernel is bound by HBM; the tensor cores only keep the instruction
+// count out of the way.
 #include "ha_common.cuh"
 
 #include <math_constants.h>
@@ -25,16 +25,33 @@ namespace ha {
 
 constexpr int kAttnWarps = 4;
 constexpr int kAttnThreads = kAttnWarps * 32;
-constexpr int kBlockTokens = 16;   // list entries per warp iteration
+constexpr int kBlockTokens = 16;              // list entries per warp iteration
+constexpr int kStages = 3;                    // blocks of rows in flight per warp (ring in shared memory)
+constexpr int kRowBytes = kD * 2 + 16;        // 256-byte row + 16 bytes so that ldmatrix rows hit distinct banks
+constexpr int kTileBytes = kBlockTokens * kRowBytes;   // one block of K (or V) rows
+constexpr int kStageBytes = 2 * kTileBytes;            // K tile followed by V tile
+constexpr int kWarpRingBytes = kStages * kStageBytes;
+constexpr int kAttnSmemBytes = kAttnWarps * kWarpRingBytes;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-__device__ __forceinline__ uint4 ld_stream16(const void *p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// 16-byte asynchronous global->shared copy; src_bytes = 0 writes zeros without reading
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -51,264 +68,443 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
-__device__ __forceinline__ uint32_t reg_of(const uint4 &v, int w) {
-    return w == 0 ? v.x : (w == 1 ? v.y : (w == 2 ? v.z : v.w));
-}
+struct AttnArgs {
+    const uint16_t *q;
+    TensorView K, V;
+    const int32_t *seq_lens, *idx, *count;
+    long long idx_sb, idx_sh;
+    int max_items, Hq, Hkv, n_units, balanced;
+    float scale_log2;
+    float *part_ml, *part_acc;
+    int32_t *tickets;
+    uint32_t *status;
+    uint16_t *out;
+    float *lse;
+};
 
 template <int G, bool kGather>
-__global__ void __launch_bounds__(kAttnThreads, 3) attn_splitk_kernel(
-    const uint16_t *__restrict__ q, TensorView K, TensorView V, const int32_t *__restrict__ seq_lens,
-    const int32_t *__restrict__ idx, long long idx_sb, long long idx_sh, const int32_t *__restrict__ count,
-    int max_items, int Hq, int Hkv, float scale_log2, int split_tokens, float *__restrict__ part_ml,
-    float *__restrict__ part_acc, int32_t *__restrict__ tickets, uint32_t *__restrict__ status,
-    uint16_t *__restrict__ out, float *__restrict__ lse) {
+__global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];   // kAttnWarps private rings, then the block prefix
     __shared__ float s_m[kAttnWarps][8], s_l[kAttnWarps][8];
-    __shared__ float s_acc[kAttnWarps][G][kD];
+    __shared__ uint32_t s_mask[kAttnWarps][kStages];
     __shared__ int s_last;
+    int *s_pref = reinterpret_cast<int *>(ring + kAttnSmemBytes);   // [n_units + 1] in balanced mode
 
-    const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, c = lane & 3;
-    const int n = seq_lens[b];
-    const int cnt = max(0, min(kGather ? count[b * Hkv + kvh] : n, max_items));
-    const int n_splits = (cnt + split_tokens - 1) / split_tokens;
-    const long long head0 = (long long)b * Hq + (long long)kvh * G;
-    if (cnt == 0) {   // empty selection: out = 0, lse = -inf
-        if (split == 0) {
-            for (int i = tid; i < G * kD; i += kAttnThreads) out[head0 * kD + i] = 0;
-            if (lse && tid < G) lse[head0 + tid] = -CUDART_INF_F;
-        }
-        return;
-    }
-    const int start = split * split_tokens;
-    if (start >= cnt) return;
-    const int end = min(cnt, start + split_tokens);
-
-    // query fragments: lane (g, c) holds chunks 4i + c (16 bytes each) of head g's row, zero for g >= G
-    uint4 qa[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) qa[i] = make_uint4(0, 0, 0, 0);
-    if (g < G) {
-        const uint4 *qp = reinterpret_cast<const uint4 *>(q + (head0 + g) * kD);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) qa[i] = __ldg(qp + 4 * i + c);
-    }
-
-    float acc[8][4];
-#pragma unroll
-    for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[mt][e] = 0.0f;
-    float m_run = -CUDART_INF_F, l_run = 0.0f;
-
-    const uint16_t *Kb = K.ptr + (long long)b * K.sb + (long long)kvh * K.sh;
-    const uint16_t *Vb = V.ptr + (long long)b * V.sb + (long long)kvh * V.sh;
-    const int32_t *list = kGather ? idx + (long long)b * idx_sb + (long long)kvh * idx_sh : nullptr;
+    const int cta = blockIdx.x, P = gridDim.x;
+    const int Hq = a.Hq, Hkv = a.Hkv;
+    unsigned char *my_ring = ring + warp * kWarpRingBytes;
+    const uint32_t ring_u32 = smem_u32(my_ring);
     bool bad = false;
 
-    auto token_at = [&](int p) -> int {
-        if (p >= end) return -1;
-        int t = kGather ? __ldg(list + p) : p;
-        if (t >= n) { bad = true; t = -1; }
-        return t;
+    auto unit_count = [&](int u) -> int {
+        const int b = u / Hkv;
+        return max(0, min(kGather ? a.count[u] : a.seq_lens[b], a.max_items));
+    };
+    auto write_empty = [&](int u) {   // empty selection: out = 0, lse = -inf
+        const long long h0 = (long long)(u / Hkv) * Hq + (long long)(u % Hkv) * G;
+        for (int i = tid; i < G * kD; i += kAttnThreads) a.out[h0 * kD + i] = 0;
+        if (a.lse && tid < G) a.lse[h0 + tid] = -CUDART_INF_F;
     };
 
-    for (int p0 = start + warp * kBlockTokens; p0 < end; p0 += kAttnWarps * kBlockTokens) {
-        // ---- which rows this lane fetches
-        const int tk0 = token_at(p0 + g), tk1 = token_at(p0 + 8 + g);
-        int tv[4];
-        tv[0] = token_at(p0 + 2 * c);
-        tv[1] = token_at(p0 + 2 * c + 1);
-        tv[2] = token_at(p0 + 2 * c + 8);
-        tv[3] = token_at(p0 + 2 * c + 9);
-
-        // ---- issue every load of the block: K rows tk0, tk1 (chunks 4i+c), V rows tv[u] (chunks 8j+g)
-        uint4 k0[4], k1[4], v[4][2];
-        {
-            const uint4 *kp0 = reinterpret_cast<const uint4 *>(Kb + (long long)max(tk0, 0) * K.sn);
-            const uint4 *kp1 = reinterpret_cast<const uint4 *>(Kb + (long long)max(tk1, 0) * K.sn);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                k0[i] = (tk0 >= 0) ? ld_stream16(kp0 + 4 * i + c) : make_uint4(0, 0, 0, 0);
-                k1[i] = (tk1 >= 0) ? ld_stream16(kp1 + 4 * i + c) : make_uint4(0, 0, 0, 0);
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint4 *vp = reinterpret_cast<const uint4 *>(Vb + (long long)max(tv[u], 0) * V.sn);
-#pragma unroll
-                for (int j = 0; j < 2; ++j)
-                    v[u][j] = (tv[u] >= 0) ? ld_stream16(vp + 8 * j + g) : make_uint4(0, 0, 0, 0);
-            }
-        }
-
-        // ---- S[head g][tokens 2c, 2c+1, 8+2c, 8+2c+1] = Q K^T
-        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            mma_bf16_16816(s0, qa[i].x, 0u, qa[i].y, 0u, k0[i].x, k0[i].y);
-            mma_bf16_16816(s0, qa[i].z, 0u, qa[i].w, 0u, k0[i].z, k0[i].w);
-            mma_bf16_16816(s1, qa[i].x, 0u, qa[i].y, 0u, k1[i].x, k1[i].y);
-            mma_bf16_16816(s1, qa[i].z, 0u, qa[i].w, 0u, k1[i].z, k1[i].w);
-        }
-
-        // ---- online softmax for head g (log2 domain); masked entries contribute nothing
-        float sv[4];
-        sv[0] = (tv[0] >= 0) ? s0[0] * scale_log2 : -CUDART_INF_F;
-        sv[1] = (tv[1] >= 0) ? s0[1] * scale_log2 : -CUDART_INF_F;
-        sv[2] = (tv[2] >= 0) ? s1[0] * scale_log2 : -CUDART_INF_F;
-        sv[3] = (tv[3] >= 0) ? s1[1] * scale_log2 : -CUDART_INF_F;
-        float bm = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
-        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
-        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
-        const float m_new = fmaxf(m_run, bm);
-        const float m_use = (m_new == -CUDART_INF_F) ? 0.0f : m_new;
-        const float corr = exp2f(m_run - m_use);
-        float p[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) p[u] = exp2f(sv[u] - m_use);
-        l_run = fmaf(l_run, corr, (p[0] + p[1]) + (p[2] + p[3]));
-        m_run = m_new;
-        float ph[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) ph[u] = bf16_round(p[u]);
-        const uint32_t bh0 = pack_bf16(ph[0], ph[1]), bh1 = pack_bf16(ph[2], ph[3]);
-        const uint32_t bl0 = pack_bf16(p[0] - ph[0], p[1] - ph[1]), bl1 = pack_bf16(p[2] - ph[2], p[3] - ph[3]);
-
-        // ---- rescale the running output when a maximum moved (columns of this lane: heads 2c, 2c+1)
-        if (__any_sync(0xffffffffu, corr != 1.0f)) {
-            const float ce = __shfl_sync(0xffffffffu, corr, (2 * c) * 4);
-            const float co = __shfl_sync(0xffffffffu, corr, (2 * c + 1) * 4);
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-                acc[mt][0] *= ce; acc[mt][1] *= co; acc[mt][2] *= ce; acc[mt][3] *= co;
-            }
-        }
-
-        // ---- O^T[d][head] += V^T P^T : row-tile mt covers d = 8*rho + mt, rho = lane group (+8)
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt) {
-            const int w = mt >> 1;
-            const uint32_t sel = (mt & 1) ? 0x7632u : 0x5410u;
-            const uint32_t a0 = __byte_perm(reg_of(v[0][0], w), reg_of(v[1][0], w), sel);
-            const uint32_t a1 = __byte_perm(reg_of(v[0][1], w), reg_of(v[1][1], w), sel);
-            const uint32_t a2 = __byte_perm(reg_of(v[2][0], w), reg_of(v[3][0], w), sel);
-            const uint32_t a3 = __byte_perm(reg_of(v[2][1], w), reg_of(v[3][1], w), sel);
-            mma_bf16_16816(acc[mt], a0, a1, a2, a3, bh0, bh1);
-            mma_bf16_16816(acc[mt], a0, a1, a2, a3, bl0, bl1);
-        }
-    }
-    if (bad) atomicOr(status, HA_DEV_BAD_INDEX);
-
-    // ---- merge the warps of this CTA through shared memory
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    if (c == 0) { s_m[warp][g] = m_run; s_l[warp][g] = l_run; }
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-        const int h = 2 * c + hh;
-        if (h < G) {
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-                s_acc[warp][h][8 * g + mt] = acc[mt][hh];
-                s_acc[warp][h][64 + 8 * g + mt] = acc[mt][2 + hh];
-            }
-        }
-    }
-    __syncthreads();
-    const int d = tid;   // kAttnThreads == kD
-    float Mj[G], Lj[G], Aj[G];
-#pragma unroll
-    for (int j = 0; j < G; ++j) {
-        float M = s_m[0][j];
-#pragma unroll
-        for (int w = 1; w < kAttnWarps; ++w) M = fmaxf(M, s_m[w][j]);
-        float L = 0.0f, A = 0.0f;
-        if (M > -CUDART_INF_F) {
-#pragma unroll
-            for (int w = 0; w < kAttnWarps; ++w) {
-                const float f = exp2f(s_m[w][j] - M);
-                L = fmaf(s_l[w][j], f, L);
-                A = fmaf(s_acc[w][j][d], f, A);
-            }
-        }
-        Mj[j] = M; Lj[j] = L; Aj[j] = A;
-    }
-
-    if (n_splits > 1) {
-        // publish this slice, take a ticket; the CTA that draws the last ticket merges all slices
-#pragma unroll
-        for (int j = 0; j < G; ++j) {
-            const long long pidx = (head0 + j) * kMaxSplits + split;
-            part_acc[pidx * kD + d] = Aj[j];
-            if (d == 0) { part_ml[pidx * 2] = Mj[j]; part_ml[pidx * 2 + 1] = Lj[j]; }
-        }
-        __threadfence();
+    // ---- this CTA's range [x, x_end) of the global block sequence
+    long long x, x_end, T;
+    int u;
+    if (a.balanced) {
+        for (int v = tid; v < a.n_units; v += kAttnThreads)
+            s_pref[v + 1] = (unit_count(v) + kBlockTokens - 1) / kBlockTokens;
+        if (tid == 0) s_pref[0] = 0;
         __syncthreads();
-        if (tid == 0) {
-            const int t = atomicAdd(&tickets[b * Hkv + kvh], 1);
-            s_last = (t == n_splits - 1);
-            if (s_last) tickets[b * Hkv + kvh] = 0;   // ready for the next call
+        if (warp == 0) {   // inclusive scan in place, one contiguous piece per lane
+            const int per = (a.n_units + 31) / 32;
+            const int lo = min(a.n_units, lane * per), hi = min(a.n_units, lo + per);
+            int sum = 0;
+            for (int v = lo; v < hi; ++v) sum += s_pref[v + 1];
+            int inc = sum;
+#pragma unroll
+            for (int dd = 1; dd < 32; dd <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, inc, dd);
+                if (lane >= dd) inc += o;
+            }
+            int run = inc - sum;
+            for (int v = lo; v < hi; ++v) { run += s_pref[v + 1]; s_pref[v + 1] = run; }
         }
         __syncthreads();
-        if (!s_last) return;
-        __threadfence();
+        T = s_pref[a.n_units];
+        for (int v = cta; v < a.n_units; v += P)
+            if (s_pref[v + 1] == s_pref[v]) write_empty(v);
+        if (T == 0) return;
+        x = (long long)cta * T / P;
+        x_end = (long long)(cta + 1) * T / P;
+        if (x >= x_end) return;
+        int lo = 0, hi = a.n_units;   // largest u with s_pref[u] <= x
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_pref[mid] <= x) lo = mid; else hi = mid;
+        }
+        u = lo;
+    } else {   // one CTA per unit
+        u = cta;
+        T = 0;
+        x = 0;
+        x_end = (unit_count(u) + kBlockTokens - 1) / kBlockTokens;
+        if (x_end == 0) { write_empty(u); return; }
+    }
+
+    while (x < x_end) {
+        // ---- segment: blocks [blk_lo, blk_hi) of unit u
+        long long u_lo = 0, u_hi = x_end;
+        int n_parts = 1, my_part = 0, slot0 = 0;
+        if (a.balanced) {
+            u_lo = s_pref[u];
+            u_hi = s_pref[u + 1];
+            const int c_first = (int)(((u_lo + 1) * P - 1) / T), c_last = (int)((u_hi * P - 1) / T);
+            n_parts = c_last - c_first + 1;
+            my_part = cta - c_first;
+            slot0 = c_first + u;   // slots of a unit are consecutive: CTA index + unit index
+        }
+        const long long seg_end = (x_end < u_hi) ? x_end : u_hi;
+        const int blk_lo = (int)(x - u_lo), blk_hi = (int)(seg_end - u_lo);
+        const int b = u / Hkv, kvh = u % Hkv;
+        const int n = a.seq_lens[b];
+        const int cnt = unit_count(u);
+        const long long head0 = (long long)b * Hq + (long long)kvh * G;
+        const int start = blk_lo * kBlockTokens, end = min(cnt, blk_hi * kBlockTokens);
+
+        const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (long long)b * a.K.sb + (long long)kvh * a.K.sh);
+        const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (long long)b * a.V.sb + (long long)kvh * a.V.sh);
+        const long long k_row = a.K.sn * 2, v_row = a.V.sn * 2;   // bytes
+        const int32_t *list = kGather ? a.idx + (long long)b * a.idx_sb + (long long)kvh * a.idx_sh : nullptr;
+
+        // raw list entry of position p for this lane; only the load is issued here, the value is first
+        // looked at when its block is started, one iteration later, so the warp never waits on it
+        auto fetch_raw = [&](int p) -> int { return (kGather && p < end) ? __ldg(list + p) : p; };
+        // token id from a raw entry (-1: past the slice, padding or outside the sequence)
+        auto token_of = [&](int p, int raw) -> int {
+            int t = (p < end) ? raw : -1;
+            if (t >= n) { bad = true; t = -1; }
+            return t;
+        };
+        // start the copies of one block (16 list entries) into ring stage `stg`: half-warp h copies row
+        // 2r+h, lane%16 picks the 16-byte chunk, so each row is one 256-byte burst
+        auto issue = [&](int stg, int my_t) {
+            const uint32_t valid = __ballot_sync(0xffffffffu, my_t >= 0) & 0xffffu;
+            if (lane == 0) s_mask[warp][stg] = valid;
+            const uint32_t kdst = ring_u32 + stg * kStageBytes + (lane >> 4) * kRowBytes + (lane & 15) * 16;
+            const uint32_t vdst = kdst + kTileBytes;
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                const int t = __shfl_sync(0xffffffffu, my_t, 2 * r + (lane >> 4));
+                const uint32_t nb = (t >= 0) ? 16u : 0u;
+                const long long tt = (t >= 0) ? t : 0;
+                cp_async16(kdst + r * 2 * kRowBytes, Kb + tt * k_row + (lane & 15) * 16, nb);
+                cp_async16(vdst + r * 2 * kRowBytes, Vb + tt * v_row + (lane & 15) * 16, nb);
+            }
+        };
+
+        // ---- software pipeline over this warp's blocks: block i lives at first + i * stride
+        const int stride = kAttnWarps * kBlockTokens;
+        const int first = start + warp * kBlockTokens;
+        const int nblk = (first < end) ? (end - first + stride - 1) / stride : 0;
+        int raw[kStages];
+#pragma unroll
+        for (int i = 0; i < kStages; ++i) raw[i] = fetch_raw(first + i * stride + (lane & 15));
+
+        // query A fragments: rows = heads (g), k = d; heads >= G are zero rows
+        uint32_t qa[8][2];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) { qa[s][0] = 0u; qa[s][1] = 0u; }
+        if (g < G) {
+            const uint32_t *qp = reinterpret_cast<const uint32_t *>(a.q + (head0 + g) * kD);
+#pragma unroll
+            for (int s = 0; s < 8; ++s) { qa[s][0] = __ldg(qp + 8 * s + c); qa[s][1] = __ldg(qp + 8 * s + c + 4); }
+        }
+        float acc[8][4];
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[mt][e] = 0.0f;
+        float m_run = -CUDART_INF_F, l_run = 0.0f;
+
+#pragma unroll
+        for (int i = 0; i < kStages - 1; ++i) {
+            if (i < nblk) issue(i, token_of(first + i * stride + (lane & 15), raw[i]));
+            cp_async_commit();
+        }
+        int next_raw = raw[kStages - 1];   // list entries of block kStages-1
+        int st = 0;
+        for (int i = 0; i < nblk; ++i) {
+            {   // refill the stage that block i-1 just released
+                const int j = i + kStages - 1;
+                const int pj = first + j * stride;
+                int stj = st + kStages - 1;
+                if (stj >= kStages) stj -= kStages;
+                if (j < nblk) issue(stj, token_of(pj + (lane & 15), next_raw));
+                cp_async_commit();
+                next_raw = fetch_raw(pj + stride + (lane & 15));   // one block ahead
+            }
+            cp_async_wait<kStages - 1>();
+            __syncwarp();
+            const uint32_t valid = s_mask[warp][st];
+            const uint32_t ks = ring_u32 + st * kStageBytes;
+            const uint32_t vs = ks + kTileBytes;
+            // ldmatrix lane address: matrix j = lane/8 -> tokens (j/2)*8 + lane%8, 16-byte column block j%2
+            const uint32_t lm_off = (((lane >> 4) << 3) + (lane & 7)) * kRowBytes + ((lane >> 3) & 1) * 16;
+
+            // ---- S[head g][tokens 2c, 2c+1, 8+2c, 8+2c+1] = Q K^T
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                uint32_t kb[4];
+                ldmatrix_x4(kb, ks + lm_off + s * 32);
+                mma_bf16_16816(s0, qa[s][0], 0u, qa[s][1], 0u, kb[0], kb[1]);
+                mma_bf16_16816(s1, qa[s][0], 0u, qa[s][1], 0u, kb[2], kb[3]);
+            }
+
+            // ---- online softmax for head g (log2 domain); masked entries contribute nothing
+            float sv[4];
+            sv[0] = ((valid >> (2 * c)) & 1u) ? s0[0] * a.scale_log2 : -CUDART_INF_F;
+            sv[1] = ((valid >> (2 * c + 1)) & 1u) ? s0[1] * a.scale_log2 : -CUDART_INF_F;
+            sv[2] = ((valid >> (2 * c + 8)) & 1u) ? s1[0] * a.scale_log2 : -CUDART_INF_F;
+            sv[3] = ((valid >> (2 * c + 9)) & 1u) ? s1[1] * a.scale_log2 : -CUDART_INF_F;
+            float bm = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
+            bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
+            const float m_new = fmaxf(m_run, bm);
+            const float m_use = (m_new == -CUDART_INF_F) ? 0.0f : m_new;
+            const float corr = exp2f(m_run - m_use);
+            float p[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) p[e] = exp2f(sv[e] - m_use);
+            l_run = fmaf(l_run, corr, (p[0] + p[1]) + (p[2] + p[3]));
+            m_run = m_new;
+            float ph[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) ph[e] = bf16_round(p[e]);
+            const uint32_t bh0 = pack_bf16(ph[0], ph[1]), bh1 = pack_bf16(ph[2], ph[3]);
+            const uint32_t bl0 = pack_bf16(p[0] - ph[0], p[1] - ph[1]), bl1 = pack_bf16(p[2] - ph[2], p[3] - ph[3]);
+
+            // ---- rescale the running output when a maximum moved (columns of this lane: heads 2c, 2c+1)
+            if (__any_sync(0xffffffffu, corr != 1.0f)) {
+                const float ce = __shfl_sync(0xffffffffu, corr, (2 * c) * 4);
+                const float co = __shfl_sync(0xffffffffu, corr, (2 * c + 1) * 4);
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    acc[mt][0] *= ce; acc[mt][1] *= co; acc[mt][2] *= ce; acc[mt][3] *= co;
+                }
+            }
+
+            // ---- O^T[d][head] += V^T P^T; the transposed ldmatrix pairs two tokens per register
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+                uint32_t va[4];
+                ldmatrix_x4_trans(va, vs + lm_off + mt * 32);
+                mma_bf16_16816(acc[mt], va[0], va[1], va[2], va[3], bh0, bh1);
+                mma_bf16_16816(acc[mt], va[0], va[1], va[2], va[3], bl0, bl1);
+            }
+            __syncwarp();   // every lane is done with this stage before it is refilled
+            if (++st == kStages) st = 0;
+        }
+        cp_async_wait<0>();
+
+        // ---- merge the warps of this CTA through shared memory (each warp reuses its own ring)
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        if (c == 0) { s_m[warp][g] = m_run; s_l[warp][g] = l_run; }
+        __syncwarp();
+        float *my_acc = reinterpret_cast<float *>(my_ring);   // [G][128]
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int h = 2 * c + hh;
+            if (h < G) {
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    my_acc[h * kD + 16 * mt + g] = acc[mt][hh];
+                    my_acc[h * kD + 16 * mt + 8 + g] = acc[mt][2 + hh];
+                }
+            }
+        }
+        __syncthreads();
+        const int d = tid;   // kAttnThreads == kD
+        float Mj[G], Lj[G], Aj[G];
 #pragma unroll
         for (int j = 0; j < G; ++j) {
-            const long long p0 = (head0 + j) * kMaxSplits;
-            float M = -CUDART_INF_F;
-            for (int s = 0; s < n_splits; ++s) M = fmaxf(M, __ldcg(part_ml + (p0 + s) * 2));
+            float M = s_m[0][j];
+#pragma unroll
+            for (int w = 1; w < kAttnWarps; ++w) M = fmaxf(M, s_m[w][j]);
             float L = 0.0f, A = 0.0f;
             if (M > -CUDART_INF_F) {
-                for (int s = 0; s < n_splits; ++s) {
-                    const float f = exp2f(__ldcg(part_ml + (p0 + s) * 2) - M);
-                    L = fmaf(__ldcg(part_ml + (p0 + s) * 2 + 1), f, L);
-                    A = fmaf(__ldcg(part_acc + (p0 + s) * kD + d), f, A);
+#pragma unroll
+                for (int w = 0; w < kAttnWarps; ++w) {
+                    const float f = exp2f(s_m[w][j] - M);
+                    L = fmaf(s_l[w][j], f, L);
+                    A = fmaf(reinterpret_cast<const float *>(ring + w * kWarpRingBytes)[j * kD + d], f, A);
                 }
             }
             Mj[j] = M; Lj[j] = L; Aj[j] = A;
         }
-    }
+
+        bool finalize = true;
+        if (n_parts > 1) {
+            // publish this part, take a ticket; the CTA that draws the last ticket merges all parts
+            const long long slot = (long long)(slot0 + my_part) * G;
 #pragma unroll
-    for (int j = 0; j < G; ++j) {
-        const float o = (Lj[j] > 0.0f) ? Aj[j] / Lj[j] : 0.0f;
-        const __nv_bfloat16 ob = __float2bfloat16_rn(o);
-        out[(head0 + j) * kD + d] = *reinterpret_cast<const uint16_t *>(&ob);
-        if (lse && d == 0) lse[head0 + j] = (Lj[j] > 0.0f) ? (Mj[j] * kLn2 + logf(Lj[j])) : -CUDART_INF_F;
+            for (int j = 0; j < G; ++j) {
+                a.part_acc[(slot + j) * kD + d] = Aj[j];
+                if (d == 0) { a.part_ml[(slot + j) * 2] = Mj[j]; a.part_ml[(slot + j) * 2 + 1] = Lj[j]; }
+            }
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) {
+                const int t = atomicAdd(&a.tickets[u], 1);
+                s_last = (t == n_parts - 1);
+                if (s_last) a.tickets[u] = 0;   // ready for the next call
+            }
+            __syncthreads();
+            finalize = (s_last != 0);
+            if (finalize) {
+                __threadfence();
+                // Merge of the parts: thread (dq, pg) owns dimensions 4dq..4dq+3 and the parts pg, pg+4, ...;
+                // a pass covers 16 (8 when G = 8) parts with every load issued before the first use (one L2 round trip),
+                // then the four part groups are folded through shared memory.
+                const int dq = tid & 31, pg = tid >> 5;
+                float Mt[G], Lt[G];
+                float4 At[G];
+#pragma unroll
+                for (int j = 0; j < G; ++j) { Mt[j] = -CUDART_INF_F; Lt[j] = 0.0f; At[j] = make_float4(0.f, 0.f, 0.f, 0.f); }
+                constexpr int kEB = (G >= 8) ? 2 : 4;   // loads in flight per head and thread
+                for (int part0 = 0; part0 < n_parts; part0 += 4 * kEB) {
+                    float4 av[G][kEB];
+                    float mv[G][kEB], lv[G][kEB];
+#pragma unroll
+                    for (int e = 0; e < kEB; ++e) {
+                        const int pp = part0 + 4 * e + pg;
+                        const bool ok = pp < n_parts;
+#pragma unroll
+                        for (int j = 0; j < G; ++j) {
+                            const long long sl = (long long)(slot0 + (ok ? pp : 0)) * G + j;
+                            const float2 ml = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + sl * 2));
+                            av[j][e] = __ldcg(reinterpret_cast<const float4 *>(a.part_acc + sl * kD) + dq);
+                            mv[j][e] = ok ? ml.x : -CUDART_INF_F;
+                            lv[j][e] = ok ? ml.y : 0.0f;
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < G; ++j) {
+                        float M = Mt[j];
+#pragma unroll
+                        for (int e = 0; e < kEB; ++e) M = fmaxf(M, mv[j][e]);
+                        if (M > -CUDART_INF_F) {
+                            const float f0 = exp2f(Mt[j] - M);
+                            float L = Lt[j] * f0;
+                            float4 A = make_float4(At[j].x * f0, At[j].y * f0, At[j].z * f0, At[j].w * f0);
+#pragma unroll
+                            for (int e = 0; e < kEB; ++e) {
+                                const float f = exp2f(mv[j][e] - M);   // 0 for absent parts
+                                L = fmaf(lv[j][e], f, L);
+                                A.x = fmaf(av[j][e].x, f, A.x); A.y = fmaf(av[j][e].y, f, A.y);
+                                A.z = fmaf(av[j][e].z, f, A.z); A.w = fmaf(av[j][e].w, f, A.w);
+                            }
+                            Mt[j] = M; Lt[j] = L; At[j] = A;
+                        }
+                    }
+                }
+                __syncthreads();   // the rings were last read by the warp merge above
+                float *red = reinterpret_cast<float *>(ring);   // [4 part groups][G][128] + [4][G][2]
+                float *red_ml = red + kAttnWarps * G * kD;
+#pragma unroll
+                for (int j = 0; j < G; ++j) {
+                    reinterpret_cast<float4 *>(red + (pg * G + j) * kD)[dq] = At[j];
+                    if (dq == 0) { red_ml[(pg * G + j) * 2] = Mt[j]; red_ml[(pg * G + j) * 2 + 1] = Lt[j]; }
+                }
+                __syncthreads();
+#pragma unroll
+                for (int j = 0; j < G; ++j) {
+                    float M = -CUDART_INF_F;
+#pragma unroll
+                    for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, red_ml[(w * G + j) * 2]);
+                    float L = 0.0f, A = 0.0f;
+                    if (M > -CUDART_INF_F) {
+#pragma unroll
+                        for (int w = 0; w < kAttnWarps; ++w) {
+                            const float f = exp2f(red_ml[(w * G + j) * 2] - M);
+                            L = fmaf(red_ml[(w * G + j) * 2 + 1], f, L);
+                            A = fmaf(red[(w * G + j) * kD + d], f, A);
+                        }
+                    }
+                    Mj[j] = M; Lj[j] = L; Aj[j] = A;
+                }
+            }
+        }
+        if (finalize) {
+#pragma unroll
+            for (int j = 0; j < G; ++j) {
+                const float o = (Lj[j] > 0.0f) ? Aj[j] / Lj[j] : 0.0f;
+                const __nv_bfloat16 ob = __float2bfloat16_rn(o);
+                a.out[(head0 + j) * kD + d] = *reinterpret_cast<const uint16_t *>(&ob);
+                if (a.lse && d == 0) a.lse[head0 + j] = (Lj[j] > 0.0f) ? (Mj[j] * kLn2 + logf(Lj[j])) : -CUDART_INF_F;
+            }
+        }
+
+        // ---- next unit of this CTA's range (units without blocks are skipped)
+        x = seg_end;
+        if (x < x_end) {
+            ++u;
+            while (s_pref[u + 1] == s_pref[u]) ++u;
+            __syncthreads();   // the rings are reused by the next segment
+        }
     }
+    if (bad) atomicOr(a.status, HA_DEV_BAD_INDEX);
 }
 
-int split_tokens_for(int n_units, int max_items) {
-    // About four waves of 3 CTAs per SM when there is that much work, never fewer than 64 list
-    // entries per CTA (one 16-entry block per warp), never more than kMaxSplits slices per unit.
-    const long long total = (long long)max(n_units, 1) * max(max_items, 1);
-    const long long target_ctas = 148LL * 3 * 4;
-    long long tokens = (total + target_ctas - 1) / target_ctas;
-    tokens = (tokens + kBlockTokens - 1) / kBlockTokens * kBlockTokens;
-    if (tokens < kAttnWarps * kBlockTokens) tokens = kAttnWarps * kBlockTokens;
-    while (((long long)max_items + tokens - 1) / tokens > kMaxSplits) tokens += kBlockTokens;
-    return (int)tokens;
+static int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+template <int G, bool kGather>
+static cudaError_t launch_attn_t(const AttnArgs &args, int grid, size_t smem, cudaStream_t st) {
+    static bool done[64] = {};   // opt in to the ring's shared memory once per device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(attn_kernel<G, kGather>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kAttnSmemBytes + (kMaxBalancedUnits + 1) * 4);
+        if (e != cudaSuccess) return e;
+        done[dev] = true;
+    }
+    attn_kernel<G, kGather><<<grid, kAttnThreads, smem, st>>>(args);
+    count_launch();
+    return cudaGetLastError();
 }
 
 template <int G>
-static cudaError_t launch_attn_g(bool gather, int B, int Hq, int Hkv, float sm_scale, const uint16_t *q,
-                                 TensorView K, TensorView V, const int32_t *seq_lens, const int32_t *idx,
-                                 long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
-                                 uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
-                                 uint32_t *status, cudaStream_t st) {
-    const int split_tokens = split_tokens_for(B * Hkv, max_items);
-    const int n_splits = max(1, (max_items + split_tokens - 1) / split_tokens);
-    dim3 grid(n_splits, Hkv, B);
-    const float scale_log2 = sm_scale * kLog2e;
-    if (gather)
-        attn_splitk_kernel<G, true><<<grid, kAttnThreads, 0, st>>>(q, K, V, seq_lens, idx, idx_sb, idx_sh, count,
-                                                                   max_items, Hq, Hkv, scale_log2, split_tokens,
-                                                                   part_ml, part_acc, tickets, status, out, lse);
-    else
-        attn_splitk_kernel<G, false><<<grid, kAttnThreads, 0, st>>>(q, K, V, seq_lens, idx, idx_sb, idx_sh, count,
-                                                                    max_items, Hq, Hkv, scale_log2, split_tokens,
-                                                                    part_ml, part_acc, tickets, status, out, lse);
-    count_launch();
-    return cudaGetLastError();
+static cudaError_t launch_attn_g(bool gather, const AttnArgs &args_in, cudaStream_t st) {
+    AttnArgs args = args_in;
+    const long long blocks_per_unit = (args.max_items + kBlockTokens - 1) / kBlockTokens;
+    const long long t_max = blocks_per_unit * args.n_units;
+    int grid;
+    size_t smem = kAttnSmemBytes;
+    if (args.n_units <= kMaxBalancedUnits) {
+        args.balanced = 1;
+        long long want = (t_max + kAttnWarps - 1) / kAttnWarps;   // at least one block per warp
+        const long long cap = (long long)min(2 * sm_count(), kMaxAttnCtas);
+        grid = (int)max(1LL, min(want, cap));
+        smem += (size_t)(args.n_units + 1) * 4;
+    } else {
+        args.balanced = 0;
+        grid = args.n_units;
+    }
+    return gather ? launch_attn_t<G, true>(args, grid, smem, st) : launch_attn_t<G, false>(args, grid, smem, st);
 }
 
 cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale, const uint16_t *q,
@@ -316,16 +512,18 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
                              uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
                              uint32_t *status, cudaStream_t st) {
-#define HA_ARGS gather, B, Hq, Hkv, sm_scale, q, K, V, seq_lens, idx, idx_sb, idx_sh, count, max_items, out, lse, \
-                part_ml, part_acc, tickets, status, st
+    AttnArgs a{};
+    a.q = q; a.K = K; a.V = V; a.seq_lens = seq_lens; a.idx = idx; a.count = count;
+    a.idx_sb = idx_sb; a.idx_sh = idx_sh; a.max_items = max_items; a.Hq = Hq; a.Hkv = Hkv;
+    a.n_units = B * Hkv; a.scale_log2 = sm_scale * kLog2e;
+    a.part_ml = part_ml; a.part_acc = part_acc; a.tickets = tickets; a.status = status; a.out = out; a.lse = lse;
     switch (Hq / Hkv) {
-        case 1: return launch_attn_g<1>(HA_ARGS);
-        case 2: return launch_attn_g<2>(HA_ARGS);
-        case 4: return launch_attn_g<4>(HA_ARGS);
-        case 8: return launch_attn_g<8>(HA_ARGS);
+        case 1: return launch_attn_g<1>(gather, a, st);
+        case 2: return launch_attn_g<2>(gather, a, st);
+        case 4: return launch_attn_g<4>(gather, a, st);
+        case 8: return launch_attn_g<8>(gather, a, st);
         default: return cudaErrorInvalidValue;
     }
-#undef HA_ARGS
 }
 
 // Writes this step's new K and V rows into the cache at slot seq_len-1 (host-driven entry only).

@@ -14,7 +14,8 @@ constexpr int kHid = 128;           // mapping hidden width
 constexpr int kBits = HA_N_BITS;    // signature width b
 constexpr int kBins = HA_HIST_BINS; // score levels 0..32
 constexpr int kMaxChunks = 128;     // chunks of the code scan per (sequence, KV head)
-constexpr int kMaxSplits = 64;      // split-K partials per query head
+constexpr int kMaxAttnCtas = 1024;  // persistent CTAs of the attention kernel (bounds the partial slots)
+constexpr int kMaxBalancedUnits = 1024;   // above this many (sequence, KV head) units: one CTA per unit
 constexpr int kMaxGroup = 8;        // query heads per KV head
 constexpr size_t kHeaderBytes = 256;   // device status word (+ padding)
 constexpr int kMaxUnits = 65536;       // (sequence, KV head) pairs: bounds the ticket region
@@ -24,8 +25,8 @@ constexpr int kMaxUnits = 65536;       // (sequence, KV head) pairs: bounds the 
 struct WorkspaceLayout {
     size_t off_tickets;   // i32 [B][Hkv]  arrival counters of the split-K merge; zero between calls
     size_t off_hist;      // i32 [B][Hkv][kMaxChunks][33]   per-chunk score histograms
-    size_t off_part_ml;   // f32 [B][Hq][kMaxSplits][2]     split-K running max (log2 domain) and sum
-    size_t off_part_acc;  // f32 [B][Hq][kMaxSplits][128]   split-K unnormalised outputs
+    size_t off_part_ml;   // f32 [slots][G][2]    split-K running max (log2 domain) and sum, slots = kMaxAttnCtas + B*Hkv
+    size_t off_part_acc;  // f32 [slots][G][128]  split-K unnormalised outputs
     size_t off_stage_q;   // bf16 [B][Hq][128]              host-entry staging
     size_t off_stage_k;   // bf16 [B][Hkv][128]
     size_t off_stage_v;   // bf16 [B][Hkv][128]
@@ -41,8 +42,9 @@ inline WorkspaceLayout make_layout(int B, int Hq, int Hkv) {
     size_t o = kHeaderBytes;
     L.off_tickets = o;   o = align_up(o + (size_t)B * Hkv * 4, 256);
     L.off_hist = o;      o = align_up(o + (size_t)B * Hkv * kMaxChunks * kBins * 4, 256);
-    L.off_part_ml = o;   o = align_up(o + (size_t)B * Hq * kMaxSplits * 2 * 4, 256);
-    L.off_part_acc = o;  o = align_up(o + (size_t)B * Hq * kMaxSplits * kD * 4, 256);
+    const size_t slots = (size_t)kMaxAttnCtas + (size_t)B * Hkv, G = (size_t)(Hq / (Hkv > 0 ? Hkv : 1));
+    L.off_part_ml = o;   o = align_up(o + slots * G * 2 * 4, 256);
+    L.off_part_acc = o;  o = align_up(o + slots * G * kD * 4, 256);
     L.off_stage_q = o;   o = align_up(o + (size_t)B * Hq * kD * 2, 256);
     L.off_stage_k = o;   o = align_up(o + (size_t)B * Hkv * kD * 2, 256);
     L.off_stage_v = o;   o = align_up(o + (size_t)B * Hkv * kD * 2, 256);
@@ -59,9 +61,6 @@ inline int chunk_tokens_for(int max_seq_len) {
     while ((max_seq_len + c - 1) / c > kMaxChunks) c *= 2;
     return (int)c;
 }
-
-// Tokens of the index list handled by one CTA of the attention kernel.
-int split_tokens_for(int n_units, int max_items);
 
 void count_launch(int n = 1);
 
