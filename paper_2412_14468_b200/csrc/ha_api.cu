@@ -93,16 +93,17 @@ int ha_encode(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, i
     if (!codes || batch < 0 || n_heads <= 0 || n_tokens < 0 || heads_per_kv <= 0) return HA_ERR_INVALID_ARG;
     if (n_heads % heads_per_kv != 0 || n_heads / heads_per_kv != map->n_kv_heads) return HA_ERR_INVALID_ARG;
     if (slot && n_tokens != 1) return HA_ERR_INVALID_ARG;
+    if (slot && heads_per_kv > 8) return HA_ERR_UNSUPPORTED;
     if (batch > 65535 || n_heads > 65535) return HA_ERR_UNSUPPORTED;
     if (batch == 0 || n_tokens == 0) return HA_OK;
     cudaStream_t st = (cudaStream_t)stream;
-    if (n_tokens == 1) {
+    if (n_tokens == 1 && heads_per_kv <= 8) {
         EncodeJob a{};
         a.x = reinterpret_cast<const uint16_t *>(x->ptr);
         a.x_sb = x->stride_b; a.x_sh = x->stride_h;
         a.codes = codes; a.c_sb = c_stride_b; a.c_sh = c_stride_h;
         a.slot = slot; a.slot_minus_one = 0;
-        a.n_heads = n_heads; a.heads_per_kv = heads_per_kv; a.n_vec = batch * n_heads;
+        a.n_heads = n_heads; a.heads_per_kv = heads_per_kv; a.n_cta = batch * (n_heads / heads_per_kv);
         a.map = view(map);
         EncodeJob none{};
         HA_CUDA(launch_encode_vectors(a, none, st));
@@ -202,14 +203,14 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
     jq.x = q; jq.x_sb = (long long)Hq * kD; jq.x_sh = kD;
     jq.codes = q_codes; jq.c_sb = Hq; jq.c_sh = 1;
     jq.slot = nullptr; jq.slot_minus_one = 0;
-    jq.n_heads = Hq; jq.heads_per_kv = Hq / Hkv; jq.n_vec = B * Hq;
+    jq.n_heads = Hq; jq.heads_per_kv = Hq / Hkv; jq.n_cta = B * Hkv;
     jq.map = view(map_q);
     EncodeJob jk{};
     if (k_new) {
         jk.x = k_new; jk.x_sb = (long long)Hkv * kD; jk.x_sh = kD;
         jk.codes = k_codes; jk.c_sb = kc_stride_b; jk.c_sh = kc_stride_h;
         jk.slot = seq_lens; jk.slot_minus_one = 1;
-        jk.n_heads = Hkv; jk.heads_per_kv = 1; jk.n_vec = B * Hkv;
+        jk.n_heads = Hkv; jk.heads_per_kv = 1; jk.n_cta = B * Hkv;
         jk.map = view(map_k);
     }
     HA_CUDA(launch_encode_vectors(jq, jk, st));

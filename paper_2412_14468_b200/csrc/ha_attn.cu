@@ -98,6 +98,10 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
     const uint32_t ring_u32 = smem_u32(my_ring);
     bool bad = false;
 
+    // everything below depends on the preceding kernels (count, idx, appended rows)
+    pdl_launch_dependents();
+    pdl_wait();
+
     auto unit_count = [&](int u) -> int {
         const int b = u / Hkv;
         return max(0, min(kGather ? a.count[u] : a.seq_lens[b], a.max_items));
@@ -482,7 +486,8 @@ static cudaError_t launch_attn_t(const AttnArgs &args, int grid, size_t smem, cu
         if (e != cudaSuccess) return e;
         done[dev] = true;
     }
-    attn_kernel<G, kGather><<<grid, kAttnThreads, smem, st>>>(args);
+    cudaError_t e = launch_pdl(attn_kernel<G, kGather>, dim3(grid), dim3(kAttnThreads), smem, st, args);
+    if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
 }

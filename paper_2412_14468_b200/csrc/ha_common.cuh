@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <cstdlib>
 
 #include "hashattn.h"
 
@@ -54,13 +55,41 @@ inline WorkspaceLayout make_layout(int B, int Hq, int Hkv) {
     return L;
 }
 
-// Tokens of the code cache scanned by one CTA: 2048, doubled until a sequence of max_seq_len
-// tokens needs at most kMaxChunks chunks.
-inline int chunk_tokens_for(int max_seq_len) {
-    long long c = 2048;
+// Tokens of the code cache scanned by one CTA: a power of two >= 1024 chosen so that the grid has
+// about four CTAs per SM when there is that much work, and so that a sequence of max_seq_len tokens
+// needs at most kMaxChunks chunks.
+inline int chunk_tokens_for(int n_units, int max_seq_len) {
+    const long long total = (long long)(n_units > 0 ? n_units : 1) * (max_seq_len > 0 ? max_seq_len : 1);
+    long long c = 1024;
+    if (const char *e = getenv("HA_CHUNK")) { c = atoi(e); while ((max_seq_len + c - 1) / c > kMaxChunks) c *= 2; return (int)c; }
+    while (c < 32768 && total / c > 148 * 4) c *= 2;
     while ((max_seq_len + c - 1) / c > kMaxChunks) c *= 2;
     return (int)c;
 }
+
+// ---- programmatic dependent launch: a kernel launched with launch_pdl may start while its
+// predecessor in the stream is still running; everything it reads from, or writes over, earlier
+// work must come after pdl_wait().
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = getenv("HA_NO_PDL") ? 0 : 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
 
 void count_launch(int n = 1);
 
@@ -74,7 +103,8 @@ struct MapView {
     const float *b1, *b2, *b3;
 };
 
-// One batch of vectors to encode: vector v = (b, h) with b = v / n_heads.
+// One batch of single vectors to encode (decode step): CTA i handles sequence i / n_nets and
+// network i % n_nets, i.e. the heads_per_kv (<= 8) heads that share that network.
 struct EncodeJob {
     const uint16_t *x;       // bf16, vector (b,h) at x + b*x_sb + h*x_sh
     long long x_sb, x_sh;
@@ -82,7 +112,7 @@ struct EncodeJob {
     long long c_sb, c_sh;
     const int32_t *slot;     // per-sequence slot (device) or NULL = 0
     int slot_minus_one;      // 1: slot[] holds sequence lengths, write at slot[b] - 1
-    int n_heads, heads_per_kv, n_vec;
+    int n_heads, heads_per_kv, n_cta;   // n_cta = batch * n_heads / heads_per_kv
     MapView map;
 };
 

@@ -10,59 +10,152 @@ namespace ha {
 
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t h) { return __uint_as_float(((uint32_t)h) << 16); }
 
-// ------------------------------------------------------------------ per-vector kernel
+// ------------------------------------------------------------------ decode-step kernel
+//
+// One CTA per (sequence, network): the G query vectors that share a network (or the one new key)
+// are encoded together, so the 72 KB of weights are fetched once per CTA.  All three weight
+// matrices are requested with cp.async at kernel entry (one HBM/L2 round trip instead of one per
+// unrolled batch of a dependent loop); each layer starts as soon as its matrix has landed.  Thread
+// o runs the fma chain of output o for every vector of the CTA (independent chains interleave).
 
-__device__ __forceinline__ float dense_chain_128(const float *h, const uint16_t *__restrict__ w, int ld,
-                                                 float z) {
-    // z += sum_k h[k] * w[k*ld], ascending k, one fmaf per term
-#pragma unroll 32
-    for (int k = 0; k < 128; ++k) z = __fmaf_rn(h[k], bf16_bits_to_float(__ldg(w + (size_t)k * ld)), z);
-    return z;
+constexpr int kVecThreads = 128;
+constexpr int kVecMax = 8;   // vectors per CTA
+constexpr size_t kVecSmem = (size_t)(kD * kHid + kHid * kHid + kHid * kBits) * 2 + (size_t)2 * kVecMax * kD * 4;
+
+__device__ __forceinline__ void cp_async16_enc(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 
-__global__ void __launch_bounds__(128) encode_vec_kernel(EncodeJob ja, EncodeJob jb) {
-    __shared__ float h0[kD];
-    __shared__ float h1[kHid];
-    int v = blockIdx.x;
-    const EncodeJob &J = (v < ja.n_vec) ? ja : jb;
-    if (v >= ja.n_vec) v -= ja.n_vec;
-    const int b = v / J.n_heads, h = v % J.n_heads;
-    const int net = h / J.heads_per_kv;
+template <int NV>
+__device__ __forceinline__ void vec_layer(const float *__restrict__ hin, const uint16_t *__restrict__ w, int ld,
+                                          int o, int nv, float (&z)[NV]) {
+    // z[v] += sum_k hin[v][k] * w[k][o], ascending k, one fmaf per term
+#pragma unroll 4
+    for (int k = 0; k < 128; k += 4) {
+        const float w0 = bf16_bits_to_float(w[(k + 0) * ld + o]);
+        const float w1 = bf16_bits_to_float(w[(k + 1) * ld + o]);
+        const float w2 = bf16_bits_to_float(w[(k + 2) * ld + o]);
+        const float w3 = bf16_bits_to_float(w[(k + 3) * ld + o]);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            if (v < nv) {
+                const float4 hv = *reinterpret_cast<const float4 *>(hin + v * kD + k);   // warp broadcast
+                z[v] = __fmaf_rn(hv.x, w0, z[v]);
+                z[v] = __fmaf_rn(hv.y, w1, z[v]);
+                z[v] = __fmaf_rn(hv.z, w2, z[v]);
+                z[v] = __fmaf_rn(hv.w, w3, z[v]);
+            }
+        }
+    }
+}
+
+template <int NV>
+__global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, EncodeJob jb) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    uint16_t *sw1 = reinterpret_cast<uint16_t *>(smem);
+    uint16_t *sw2 = sw1 + kD * kHid;
+    uint16_t *sw3 = sw2 + kHid * kHid;
+    float *actA = reinterpret_cast<float *>(sw3 + kHid * kBits);   // [NV][128]
+    float *actB = actA + kVecMax * kD;
+
+    int i = blockIdx.x;
+    const bool second = i >= ja.n_cta;
+    const EncodeJob &J = second ? jb : ja;
+    if (second) i -= ja.n_cta;
+    const int n_nets = J.n_heads / J.heads_per_kv;
+    const int b = i / n_nets, net = i % n_nets;
+    const int nv = J.heads_per_kv;   // <= NV
     const int o = threadIdx.x;
 
+    // ---- request all weights (three commit groups), then the inputs
+    {
+        const unsigned char *g1 = reinterpret_cast<const unsigned char *>(J.map.w1 + (size_t)net * kD * kHid);
+        const unsigned char *g2 = reinterpret_cast<const unsigned char *>(J.map.w2 + (size_t)net * kHid * kHid);
+        const unsigned char *g3 = reinterpret_cast<const unsigned char *>(J.map.w3 + (size_t)net * kHid * kBits);
+        const uint32_t s1 = (uint32_t)__cvta_generic_to_shared(sw1), s2 = (uint32_t)__cvta_generic_to_shared(sw2),
+                       s3 = (uint32_t)__cvta_generic_to_shared(sw3);
+        for (int c = o; c < kD * kHid / 8; c += kVecThreads) cp_async16_enc(s1 + c * 16, g1 + c * 16);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        for (int c = o; c < kHid * kHid / 8; c += kVecThreads) cp_async16_enc(s2 + c * 16, g2 + c * 16);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        for (int c = o; c < kHid * kBits / 8; c += kVecThreads) cp_async16_enc(s3 + c * 16, g3 + c * 16);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    const float bias1 = J.map.b1 ? __ldg(J.map.b1 + net * kHid + o) : 0.0f;
+    const float bias2 = J.map.b2 ? __ldg(J.map.b2 + net * kHid + o) : 0.0f;
+    const float bias3 = (J.map.b3 && o < kBits) ? __ldg(J.map.b3 + net * kBits + o) : 0.0f;
+    // the weights do not depend on earlier kernels of the stream; the vectors to encode may
+    pdl_launch_dependents();
+    pdl_wait();
+    for (int v = 0; v < nv; ++v) {
+        const uint16_t *x = J.x + (long long)b * J.x_sb + (long long)(net * J.heads_per_kv + v) * J.x_sh;
+        actA[v * kD + o] = bf16_bits_to_float(__ldg(x + o));
+    }
+
     int slot = 0;
-    if (J.slot) {
-        slot = J.slot[b] - J.slot_minus_one;
-        if (slot < 0) return;
+    if (J.slot) slot = J.slot[b] - J.slot_minus_one;   // a negative slot skips the sequence (no write below)
+
+    float z[NV];
+    // ---- layer 1
+    asm volatile("cp.async.wait_group 2;" ::: "memory");
+    __syncthreads();
+#pragma unroll
+    for (int v = 0; v < NV; ++v) z[v] = bias1;
+    vec_layer<NV>(actA, sw1, kHid, o, nv, z);
+#pragma unroll
+    for (int v = 0; v < NV; ++v)
+        if (v < nv) actB[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+    // ---- layer 2
+    asm volatile("cp.async.wait_group 1;" ::: "memory");
+    __syncthreads();
+#pragma unroll
+    for (int v = 0; v < NV; ++v) z[v] = bias2;
+    vec_layer<NV>(actB, sw2, kHid, o, nv, z);
+    // actA was last read in layer 1, which every thread left before the barrier above
+#pragma unroll
+    for (int v = 0; v < NV; ++v)
+        if (v < nv) actA[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+    // ---- layer 3: one output bit per lane of warp 0
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    if (o < kBits) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) z[v] = bias3;
+        vec_layer<NV>(actA, sw3, kBits, o, nv, z);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const uint32_t code = __ballot_sync(0xffffffffu, z[v] > 0.0f);
+            if (o == 0 && v < nv && slot >= 0)
+                J.codes[(long long)b * J.c_sb + (long long)(net * J.heads_per_kv + v) * J.c_sh + slot] = code;
+        }
     }
-    const uint16_t *x = J.x + (long long)b * J.x_sb + (long long)h * J.x_sh;
-    h0[o] = bf16_bits_to_float(x[o]);
-    __syncthreads();
+}
 
-    float z = J.map.b1 ? J.map.b1[net * kHid + o] : 0.0f;
-    z = dense_chain_128(h0, J.map.w1 + (size_t)net * kD * kHid + o, kHid, z);
-    h1[o] = (z > 0.0f) ? z : 0.0f;
-    __syncthreads();
-
-    z = J.map.b2 ? J.map.b2[net * kHid + o] : 0.0f;
-    z = dense_chain_128(h1, J.map.w2 + (size_t)net * kHid * kHid + o, kHid, z);
-    h0[o] = (z > 0.0f) ? z : 0.0f;
-    __syncthreads();
-
-    if (o < kBits) {   // warp 0: one output bit per lane
-        z = J.map.b3 ? J.map.b3[net * kBits + o] : 0.0f;
-        z = dense_chain_128(h0, J.map.w3 + (size_t)net * kHid * kBits + o, kBits, z);
-        const uint32_t code = __ballot_sync(0xffffffffu, z > 0.0f);
-        if (o == 0) J.codes[(long long)b * J.c_sb + (long long)h * J.c_sh + slot] = code;
+template <int NV>
+static cudaError_t launch_vec_t(const EncodeJob &a, const EncodeJob &b, cudaStream_t st) {
+    static bool done[64] = {};   // opt in to > 48 KB of shared memory once per device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(encode_vec_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kVecSmem);
+        if (e != cudaSuccess) return e;
+        done[dev] = true;
     }
+    cudaError_t e = launch_pdl(encode_vec_kernel<NV>, dim3(a.n_cta + b.n_cta), dim3(kVecThreads), kVecSmem, st, a, b);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    return cudaGetLastError();
 }
 
 cudaError_t launch_encode_vectors(const EncodeJob &a, const EncodeJob &b, cudaStream_t st) {
-    const int n = a.n_vec + b.n_vec;
-    if (n <= 0) return cudaSuccess;
-    encode_vec_kernel<<<n, 128, 0, st>>>(a, b);
-    count_launch();
-    return cudaGetLastError();
+    if (a.n_cta + b.n_cta <= 0) return cudaSuccess;
+    const int nv = max(a.n_cta > 0 ? a.heads_per_kv : 1, b.n_cta > 0 ? b.heads_per_kv : 1);
+    if (nv <= 1) return launch_vec_t<1>(a, b, st);
+    if (nv <= 2) return launch_vec_t<2>(a, b, st);
+    if (nv <= 4) return launch_vec_t<4>(a, b, st);
+    if (nv <= 8) return launch_vec_t<8>(a, b, st);
+    return cudaErrorInvalidValue;
 }
 
 // ------------------------------------------------------------------ token-tiled bulk kernel

@@ -4,17 +4,22 @@
 // score T and how many tokens r of score exactly T are still needed; the selection is every token
 // above T plus the first r tokens at T in index order, written in ascending token order.
 //
-// Kernel 1 (scan_hist): each CTA streams one chunk of the code cache with 16-byte loads and
-//   leaves the chunk's 33-bin histogram in the workspace.
+// Kernel 1 (scan_hist): each CTA streams one chunk of the code cache with 16-byte loads (all loads
+//   of a pass in flight before the first popc) and leaves the chunk's 33-bin histogram in the
+//   workspace.
 // Kernel 2 (select): each CTA sums the chunk histograms (total, and the part before its own
-//   chunk), derives T, r and its output offset, re-reads its chunk (an L2 hit) and compacts the
-//   selected token indices with warp-shuffle prefix sums.  No CTA waits on another.
+//   chunk), derives T, r and its output offset with warp shuffles, re-reads its chunk (an L2 hit)
+//   and compacts the selected token indices with shuffle prefix sums.  No CTA waits on another.
+// Both kernels request their first pass of codes before the programmatic-launch wait, so that the
+// fetch overlaps the tail of the preceding kernel; the one code that the preceding ENCODE may still
+// be writing (the appended token, slot n-1) is re-read after the wait.
 #include "ha_common.cuh"
 
 namespace ha {
 
 constexpr int kScanThreads = 256;
-constexpr int kScanTokensPerPass = kScanThreads * 4;   // one uint4 per thread
+constexpr int kPassTokens = kScanThreads * 16;   // four uint4 per thread
+constexpr int kHistGroups = 7;                   // 7 * 33 threads sum the chunk histograms
 
 template <int G>
 __device__ __forceinline__ int group_score(uint32_t code, const uint32_t (&qc)[G]) {
@@ -34,6 +39,15 @@ __device__ __forceinline__ uint4 load_codes4(const uint32_t *row, int base, int 
     return v;
 }
 
+// Re-read token `last` (coherently) if it lies in [base, base+4): it may have been written by the
+// kernel this one was launched behind.
+__device__ __forceinline__ void patch_token(uint4 &v, int base, int last, const uint32_t *row) {
+    const int e = last - base;
+    if (e < 0 || e > 3) return;
+    const uint32_t c = __ldcg(row + last);
+    if (e == 0) v.x = c; else if (e == 1) v.y = c; else if (e == 2) v.z = c; else v.w = c;
+}
+
 template <int G>
 __global__ void __launch_bounds__(kScanThreads) scan_hist_kernel(const uint32_t *__restrict__ q_codes,
                                                                 const uint32_t *__restrict__ k_codes,
@@ -49,22 +63,44 @@ __global__ void __launch_bounds__(kScanThreads) scan_hist_kernel(const uint32_t 
     const int start = chunk * chunk_tokens;
     if (start >= n) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    for (int i = tid; i < (kScanThreads / 32) * 4 * (kBins + 3); i += kScanThreads) (&hist[0][0][0])[i] = 0;
-    uint32_t qc[G];
-#pragma unroll
-    for (int j = 0; j < G; ++j) qc[j] = __ldg(q_codes + (long long)b * Hq + g * G + j);
-    __syncthreads();
-
     const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
     const int end = min(n, start + chunk_tokens);
+
+    // first pass of codes: sub-block j of 1024 tokens, one uint4 per thread (coalesced)
+    uint4 c[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int base = start + j * 1024 + tid * 4;
+        c[j] = (base < end) ? load_codes4(row, base, end) : make_uint4(0, 0, 0, 0);
+    }
+    for (int i = tid; i < (kScanThreads / 32) * 4 * (kBins + 3); i += kScanThreads) (&hist[0][0][0])[i] = 0;
+    pdl_launch_dependents();
+    pdl_wait();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) patch_token(c[j], start + j * 1024 + tid * 4, n - 1, row);
+    uint32_t qc[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
+    __syncthreads();
+
     int *my = hist[warp][lane & 3];
-    for (int base = start + tid * 4; base < end; base += kScanTokensPerPass) {
-        const uint4 c = load_codes4(row, base, end);
-        atomicAdd(&my[group_score<G>(c.x, qc)], 1);
-        if (base + 1 < end) atomicAdd(&my[group_score<G>(c.y, qc)], 1);
-        if (base + 2 < end) atomicAdd(&my[group_score<G>(c.z, qc)], 1);
-        if (base + 3 < end) atomicAdd(&my[group_score<G>(c.w, qc)], 1);
+    for (int pass = start; pass < end; pass += kPassTokens) {
+        if (pass > start) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int base = pass + j * 1024 + tid * 4;
+                c[j] = (base < end) ? load_codes4(row, base, end) : make_uint4(0, 0, 0, 0);
+                patch_token(c[j], base, n - 1, row);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int base = pass + j * 1024 + tid * 4;
+            if (base + 0 < end) atomicAdd(&my[group_score<G>(c[j].x, qc)], 1);
+            if (base + 1 < end) atomicAdd(&my[group_score<G>(c[j].y, qc)], 1);
+            if (base + 2 < end) atomicAdd(&my[group_score<G>(c[j].z, qc)], 1);
+            if (base + 3 < end) atomicAdd(&my[group_score<G>(c[j].w, qc)], 1);
+        }
     }
     __syncthreads();
     if (tid < kBins) {
@@ -89,7 +125,7 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
                                                              int32_t *__restrict__ idx, long long idx_sb,
                                                              long long idx_sh, int32_t *__restrict__ count,
                                                              int32_t *__restrict__ hist_out) {
-    __shared__ int tot[kBins], bef[kBins];
+    __shared__ int part_tot[kHistGroups][kBins], part_bef[kHistGroups][kBins];
     __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
     __shared__ int warp_tot[kScanThreads / 32];
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
@@ -101,69 +137,118 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
     const int n_chunks = (n + chunk_tokens - 1) / chunk_tokens;
     if (chunk > 0 && chunk >= n_chunks) return;
 
+    const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
+    const int start = chunk * chunk_tokens, end = min(n, start + chunk_tokens);
+    // first pass of codes: 16 consecutive tokens per thread (token order = thread order)
+    uint4 c[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int base = start + tid * 16 + j * 4;
+        c[j] = (base < end) ? load_codes4(row, base, end) : make_uint4(0, 0, 0, 0);
+    }
+    pdl_launch_dependents();
+    pdl_wait();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) patch_token(c[j], start + tid * 16 + j * 4, n - 1, row);
+
     // totals per score level, and the part contributed by the chunks before this one
-    if (tid < kBins) {
-        const int32_t *hb = ws_hist + ((long long)b * Hkv + g) * kMaxChunks * kBins + tid;
+    if (tid < kHistGroups * kBins) {
+        const int grp = tid / kBins, bin = tid % kBins;
+        const int32_t *hb = ws_hist + ((long long)b * Hkv + g) * kMaxChunks * kBins + bin;
         int t = 0, be = 0;
-        for (int c = 0; c < n_chunks; ++c) {
-            const int v = hb[c * kBins];
+#pragma unroll 4
+        for (int cc = grp; cc < n_chunks; cc += kHistGroups) {
+            const int v = __ldcg(hb + cc * kBins);
             t += v;
-            if (c < chunk) be += v;
+            if (cc < chunk) be += v;
         }
-        tot[tid] = t;
-        bef[tid] = be;
+        part_tot[grp][bin] = t;
+        part_bef[grp][bin] = be;
     }
     __syncthreads();
-    if (tid == 0) {
-        // T = largest level with #{S >= T} >= keep; r = keep - #{S > T}
-        int T = kBins, r = 0, cum = 0;
+    int my_tot = 0;
+    if (warp == 0) {
+        // lane l owns level l (0..31); level 32 is summed by every lane.  Suffix sums over the levels
+        // give #{S >= t}; T = largest level with #{S >= T} >= keep; r = keep - #{S > T}.
+        int tot = 0, bef = 0, tot32 = 0, bef32 = 0;
+#pragma unroll
+        for (int gi = 0; gi < kHistGroups; ++gi) {
+            tot += part_tot[gi][lane]; bef += part_bef[gi][lane];
+            tot32 += part_tot[gi][32]; bef32 += part_bef[gi][32];
+        }
+        my_tot = tot;
+        int st = tot, sb = bef;   // suffix sums over levels lane..31
+#pragma unroll
+        for (int dd = 1; dd < 32; dd <<= 1) {
+            const int vt = __shfl_down_sync(0xffffffffu, st, dd), vb = __shfl_down_sync(0xffffffffu, sb, dd);
+            if (lane + dd < 32) { st += vt; sb += vb; }
+        }
+        st += tot32;   // #{S >= lane}
+        sb += bef32;   // same, restricted to the chunks before this one
+        int T = kBins, r = 0, gt_before = 0, eq_before = 0;
         if (keep > 0) {
-            for (int t = kBins - 1; t >= 0; --t) {
-                if (cum + tot[t] >= keep) { T = t; r = keep - cum; break; }
-                cum += tot[t];
+            const unsigned ge = __ballot_sync(0xffffffffu, st >= keep);
+            if (tot32 >= keep) { T = 32; r = keep; gt_before = 0; eq_before = bef32; }
+            else {
+                T = 31 - __clz(ge);   // ge != 0 because #{S >= 0} = n >= keep
+                const int above = __shfl_sync(0xffffffffu, st, min(T + 1, 31));      // #{S >= T+1}
+                const int above_b = __shfl_sync(0xffffffffu, sb, min(T + 1, 31));
+                const int at_b = __shfl_sync(0xffffffffu, bef, T);
+                const int gt = (T == 31) ? tot32 : above;
+                r = keep - gt;
+                gt_before = (T == 31) ? bef32 : above_b;
+                eq_before = at_b;
             }
         }
-        int gb = 0;
-        for (int t = T + 1; t < kBins; ++t) gb += bef[t];
-        sh_T = T; sh_r = r; sh_gt_before = gb; sh_eq_before = (T < kBins) ? bef[T] : 0;
+        if (lane == 0) { sh_T = T; sh_r = r; sh_gt_before = gt_before; sh_eq_before = eq_before; }
+        if (chunk == 0 && hist_out) {
+            hist_out[((long long)b * Hkv + g) * kBins + lane] = tot;
+            if (lane == 0) hist_out[((long long)b * Hkv + g) * kBins + 32] = tot32;
+        }
     }
+    (void)my_tot;
     __syncthreads();
     const int T = sh_T, r = sh_r;
     int32_t *out = idx + (long long)b * idx_sb + (long long)g * idx_sh;
     if (chunk == 0) {
         if (tid == 0) count[b * Hkv + g] = keep;
-        if (hist_out && tid < kBins) hist_out[((long long)b * Hkv + g) * kBins + tid] = tot[tid];
         for (int i = keep + tid; i < k_max; i += kScanThreads) out[i] = -1;
     }
     if (chunk >= n_chunks || keep == 0) return;
 
     uint32_t qc[G];
 #pragma unroll
-    for (int j = 0; j < G; ++j) qc[j] = __ldg(q_codes + (long long)b * Hq + g * G + j);
-    const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
-    const int start = chunk * chunk_tokens, end = min(n, start + chunk_tokens);
+    for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
     int run_gt = sh_gt_before, run_eq = sh_eq_before;   // tokens before this pass with S > T / S == T
 
-    for (int pass = start; pass < end; pass += kScanTokensPerPass) {
-        const int base = pass + tid * 4;
-        int s[4] = {-1, -1, -1, -1};
-        if (base < end) {
-            const uint4 c = load_codes4(row, base, end);
-            s[0] = group_score<G>(c.x, qc);
-            if (base + 1 < end) s[1] = group_score<G>(c.y, qc);
-            if (base + 2 < end) s[2] = group_score<G>(c.z, qc);
-            if (base + 3 < end) s[3] = group_score<G>(c.w, qc);
+    for (int pass = start; pass < end; pass += kPassTokens) {
+        const int base = pass + tid * 16;
+        if (pass > start) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                c[j] = (base + j * 4 < end) ? load_codes4(row, base + j * 4, end) : make_uint4(0, 0, 0, 0);
+                patch_token(c[j], base + j * 4, n - 1, row);
+            }
+        }
+        int s[16];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int bj = base + j * 4;
+            s[4 * j + 0] = (bj + 0 < end) ? group_score<G>(c[j].x, qc) : -1;
+            s[4 * j + 1] = (bj + 1 < end) ? group_score<G>(c[j].y, qc) : -1;
+            s[4 * j + 2] = (bj + 2 < end) ? group_score<G>(c[j].z, qc) : -1;
+            s[4 * j + 3] = (bj + 3 < end) ? group_score<G>(c[j].w, qc) : -1;
         }
         int cg = 0, ce = 0;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) { cg += (s[e] > T); ce += (s[e] == T); }
-        // block-wide exclusive prefix of (cg, ce), packed as two 16-bit counters (pass <= 1024 tokens)
+        for (int e = 0; e < 16; ++e) { cg += (s[e] > T); ce += (s[e] == T); }
+        // block-wide exclusive prefix of (cg, ce), packed as two 16-bit counters (a pass has 4096 tokens)
         const int packed = cg | (ce << 16);
         int inc = packed;
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, inc, d);
-            if (lane >= d) inc += v;
+        for (int dd = 1; dd < 32; dd <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, inc, dd);
+            if (lane >= dd) inc += v;
         }
         if (lane == 31) warp_tot[warp] = inc;
         __syncthreads();
@@ -176,9 +261,9 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
         }
         const int excl = wpre + inc - packed;
         int gt_lt = run_gt + (excl & 0xffff);
-        int eq_lt = run_eq + (excl >> 16);
+        int eq_lt = run_eq + (int)((unsigned)excl >> 16);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < 16; ++e) {
             if (s[e] > T) {
                 out[gt_lt + min(eq_lt, r)] = base + e;
                 ++gt_lt;
@@ -188,9 +273,243 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
             }
         }
         run_gt += all & 0xffff;
-        run_eq += all >> 16;
+        run_eq += (int)((unsigned)all >> 16);
         __syncthreads();   // warp_tot is rewritten by the next pass
     }
+}
+
+// ------------------------------------------------------------------ fused single-kernel path
+//
+// For sequences of up to kClusterSize * 16384 tokens one thread-block cluster owns a
+// (sequence, KV head) unit: every CTA keeps its slice of the codes in registers, the CTAs exchange
+// their 33-bin histograms through distributed shared memory between two hardware cluster barriers,
+// and each CTA then compacts its own slice straight from registers.  The codes are read from HBM
+// once, there is no histogram round trip through global memory and no second launch.
+// Token order inside a CTA: warp w owns a contiguous range, pass p covers 128 tokens (one uint4 per
+// lane), so prefix sums need only warp shuffles plus one exchange of eight warp totals.
+
+constexpr int kClusterSize = 8;
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// read an int of CTA `rank`'s shared memory at the address that `local` has in this CTA
+__device__ __forceinline__ int ld_dsmem(const int *local, uint32_t rank) {
+    uint32_t a = (uint32_t)__cvta_generic_to_shared(local), ra;
+    int v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+    asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(ra) : "memory");
+    return v;
+}
+
+template <int G>
+__device__ __forceinline__ uint32_t scores4(const uint4 &c, const uint32_t (&qc)[G]) {
+    return (uint32_t)group_score<G>(c.x, qc) | ((uint32_t)group_score<G>(c.y, qc) << 8) |
+           ((uint32_t)group_score<G>(c.z, qc) << 16) | ((uint32_t)group_score<G>(c.w, qc) << 24);
+}
+
+template <int G, int L>
+__global__ void __launch_bounds__(kScanThreads) score_select_cluster_kernel(
+    const uint32_t *__restrict__ q_codes, const uint32_t *__restrict__ k_codes, long long kc_sb, long long kc_sh,
+    const int32_t *__restrict__ seq_lens, int max_seq_len, const int32_t *__restrict__ k_per_seq, int k_uniform,
+    int k_max, int Hq, int Hkv, int32_t *__restrict__ idx, long long idx_sb, long long idx_sh,
+    int32_t *__restrict__ count, int32_t *__restrict__ hist_out) {
+    __shared__ int w_hist[kScanThreads / 32][4][kBins + 3];
+    __shared__ int s_hist[kBins + 3];          // this CTA's histogram, read by the whole cluster
+    __shared__ int s_tot[kBins], s_bef[kBins];
+    __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
+    __shared__ int s_wcnt[kScanThreads / 32];
+    const uint32_t rank = cluster_rank();
+    const int g = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = max(min(seq_lens[b], max_seq_len), 0);
+    int k = k_per_seq ? k_per_seq[b] : k_uniform;
+    k = max(0, min(k, k_max));
+    const int keep = min(k, n);
+    const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
+    const int wbase = (int)rank * (L * 1024) + warp * (L * 128) + lane * 4;   // first token of this lane, pass 0
+
+    uint4 c[L];
+#pragma unroll
+    for (int p = 0; p < L; ++p) {
+        const int base = wbase + p * 128;
+        c[p] = (base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
+    }
+    for (int i = tid; i < (kScanThreads / 32) * 4 * (kBins + 3); i += kScanThreads) (&w_hist[0][0][0])[i] = 0;
+    pdl_launch_dependents();
+    pdl_wait();
+#pragma unroll
+    for (int p = 0; p < L; ++p) patch_token(c[p], wbase + p * 128, n - 1, row);
+    uint32_t qc[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
+    __syncthreads();
+
+    // ---- scores (kept as four bytes per register) and this CTA's histogram
+    uint32_t sc[L];
+    int *my = w_hist[warp][lane & 3];
+#pragma unroll
+    for (int p = 0; p < L; ++p) {
+        const int base = wbase + p * 128;
+        sc[p] = scores4<G>(c[p], qc);
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (base + e < n) atomicAdd(&my[(sc[p] >> (8 * e)) & 0xffu], 1);
+            else sc[p] |= 0xffu << (8 * e);   // 255 marks "no token": never equal to T, masked from ">"
+    }
+    __syncthreads();
+    if (tid < kBins) {
+        int s = 0;
+#pragma unroll
+        for (int w = 0; w < kScanThreads / 32; ++w)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) s += w_hist[w][r][tid];
+        s_hist[tid] = s;
+    }
+    cluster_sync_all();   // every CTA's histogram is complete and visible cluster-wide
+
+    if (tid < kBins) {
+        int tot = 0, bef = 0;
+#pragma unroll
+        for (uint32_t r = 0; r < (uint32_t)kClusterSize; ++r) {
+            const int v = ld_dsmem(&s_hist[tid], r);
+            tot += v;
+            if (r < rank) bef += v;
+        }
+        s_tot[tid] = tot;
+        s_bef[tid] = bef;
+    }
+    cluster_sync_all();   // all remote reads are done (a CTA may now exit) and s_tot/s_bef are visible
+    if (warp == 0) {
+        int tot = s_tot[lane], bef = s_bef[lane];
+        const int tot32 = s_tot[32], bef32 = s_bef[32];
+        int st = tot, sb = bef;   // suffix sums over levels lane..31
+#pragma unroll
+        for (int dd = 1; dd < 32; dd <<= 1) {
+            const int vt = __shfl_down_sync(0xffffffffu, st, dd), vb = __shfl_down_sync(0xffffffffu, sb, dd);
+            if (lane + dd < 32) { st += vt; sb += vb; }
+        }
+        st += tot32;
+        sb += bef32;
+        int T = kBins, r = 0, gt_before = 0, eq_before = 0;
+        if (keep > 0) {
+            const unsigned ge = __ballot_sync(0xffffffffu, st >= keep);
+            if (tot32 >= keep) { T = 32; r = keep; gt_before = 0; eq_before = bef32; }
+            else {
+                T = 31 - __clz(ge);
+                const int above = __shfl_sync(0xffffffffu, st, min(T + 1, 31));
+                const int above_b = __shfl_sync(0xffffffffu, sb, min(T + 1, 31));
+                const int at_b = __shfl_sync(0xffffffffu, bef, T);
+                const int gt = (T == 31) ? tot32 : above;
+                r = keep - gt;
+                gt_before = (T == 31) ? bef32 : above_b;
+                eq_before = at_b;
+            }
+        }
+        if (lane == 0) { sh_T = T; sh_r = r; sh_gt_before = gt_before; sh_eq_before = eq_before; }
+        if (rank == 0 && hist_out) {
+            hist_out[((long long)b * Hkv + g) * kBins + lane] = tot;
+            if (lane == 0) hist_out[((long long)b * Hkv + g) * kBins + 32] = tot32;
+        }
+    }
+    __syncthreads();
+    const int T = sh_T, r = sh_r;
+    int32_t *out = idx + (long long)b * idx_sb + (long long)g * idx_sh;
+    if (rank == 0) {
+        if (tid == 0) count[b * Hkv + g] = keep;
+        for (int i = keep + tid; i < k_max; i += kScanThreads) out[i] = -1;
+    }
+    if (keep == 0) return;
+
+    // ---- counts of (S > T, S == T) per thread and pass, packed in 16-bit halves
+    const uint32_t T4 = (uint32_t)T * 0x01010101u;
+    int tot_packed = 0;
+#pragma unroll
+    for (int p = 0; p < L; ++p) {
+        const uint32_t valid = __vcmpne4(sc[p], 0xffffffffu) & 0x01010101u;      // 1 per real token
+        const uint32_t gt = __vcmpgtu4(sc[p], T4) & valid;                        // bytes 0x01 where S > T
+        const uint32_t eq = __vcmpeq4(sc[p], T4) & 0x01010101u;
+        tot_packed += (int)(__vsadu4(gt, 0u) | (__vsadu4(eq, 0u) << 16));
+    }
+    int winc = tot_packed;   // inclusive scan over the lanes of the per-lane totals (all passes)
+#pragma unroll
+    for (int dd = 1; dd < 32; dd <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, winc, dd);
+        if (lane >= dd) winc += v;
+    }
+    if (lane == 31) s_wcnt[warp] = winc;
+    __syncthreads();
+    int run_gt = sh_gt_before, run_eq = sh_eq_before;   // tokens before this warp's range
+#pragma unroll
+    for (int w = 0; w < kScanThreads / 32; ++w) {
+        if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
+    }
+    // ---- positions, pass by pass (token order = pass, lane, element)
+#pragma unroll
+    for (int p = 0; p < L; ++p) {
+        const uint32_t valid = __vcmpne4(sc[p], 0xffffffffu) & 0x01010101u;
+        const uint32_t gt = __vcmpgtu4(sc[p], T4) & valid;
+        const uint32_t eq = __vcmpeq4(sc[p], T4) & 0x01010101u;
+        const int packed = (int)(__vsadu4(gt, 0u) | (__vsadu4(eq, 0u) << 16));
+        int inc = packed;
+#pragma unroll
+        for (int dd = 1; dd < 32; dd <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, inc, dd);
+            if (lane >= dd) inc += v;
+        }
+        const int all = __shfl_sync(0xffffffffu, inc, 31);
+        if (all != 0) {
+            const int excl = inc - packed;
+            int gt_lt = run_gt + (excl & 0xffff);
+            int eq_lt = run_eq + (int)((unsigned)excl >> 16);
+            const int base = wbase + p * 128;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if ((gt >> (8 * e)) & 1u) {
+                    out[gt_lt + min(eq_lt, r)] = base + e;
+                    ++gt_lt;
+                } else if ((eq >> (8 * e)) & 1u) {
+                    if (eq_lt < r) out[gt_lt + eq_lt] = base + e;
+                    ++eq_lt;
+                }
+            }
+        }
+        run_gt += all & 0xffff;
+        run_eq += (int)((unsigned)all >> 16);
+    }
+}
+
+template <int G, int L>
+static cudaError_t launch_cluster_t(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes,
+                                    long long kc_sb, long long kc_sh, const int32_t *seq_lens,
+                                    const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max, int32_t *idx,
+                                    long long idx_sb, long long idx_sh, int32_t *count, int32_t *hist_out,
+                                    cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kClusterSize, Hkv, B);
+    cfg.blockDim = dim3(kScanThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kClusterSize;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = getenv("HA_NO_PDL") ? 0 : 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, score_select_cluster_kernel<G, L>, q_codes, k_codes, kc_sb, kc_sh, seq_lens,
+                                       max_seq_len, k_per_seq, k_uniform, k_max, Hq, Hkv, idx, idx_sb, idx_sh, count,
+                                       hist_out);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    return cudaGetLastError();
 }
 
 template <int G>
@@ -199,14 +518,29 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
                             int k_uniform, int max_seq_len, int k_max, int32_t *idx, long long idx_sb,
                             long long idx_sh, int32_t *count, int32_t *hist_out, int32_t *ws_hist,
                             cudaStream_t st) {
-    const int chunk_tokens = chunk_tokens_for(max_seq_len);
+    if (max_seq_len <= kClusterSize * 16 * 1024 && !getenv("HA_NO_CLUSTER")) {
+        // fused path: one cluster per unit, L uint4 of codes per thread
+        const int per_cta = (max_seq_len + kClusterSize - 1) / kClusterSize;
+#define HA_CL(LL)                                                                                                   \
+    return launch_cluster_t<G, LL>(B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform,     \
+                                   max_seq_len, k_max, idx, idx_sb, idx_sh, count, hist_out, st)
+        if (per_cta <= 1024) HA_CL(1);
+        if (per_cta <= 2048) HA_CL(2);
+        if (per_cta <= 4096) HA_CL(4);
+        if (per_cta <= 8192) HA_CL(8);
+        HA_CL(16);
+#undef HA_CL
+    }
+    const int chunk_tokens = chunk_tokens_for(B * Hkv, max_seq_len);
     const int n_chunks = max(1, (max_seq_len + chunk_tokens - 1) / chunk_tokens);
     dim3 grid(n_chunks, Hkv, B);
-    scan_hist_kernel<G><<<grid, kScanThreads, 0, st>>>(q_codes, k_codes, kc_sb, kc_sh, seq_lens, max_seq_len,
-                                                      Hq, Hkv, chunk_tokens, ws_hist);
-    select_kernel<G><<<grid, kScanThreads, 0, st>>>(q_codes, k_codes, kc_sb, kc_sh, seq_lens, max_seq_len, k_per_seq,
-                                                   k_uniform, k_max, Hq, Hkv, chunk_tokens, ws_hist, idx, idx_sb, idx_sh,
-                                                   count, hist_out);
+    cudaError_t e = launch_pdl(scan_hist_kernel<G>, grid, dim3(kScanThreads), 0, st, q_codes, k_codes, kc_sb, kc_sh,
+                               seq_lens, max_seq_len, Hq, Hkv, chunk_tokens, ws_hist);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(select_kernel<G>, grid, dim3(kScanThreads), 0, st, q_codes, k_codes, kc_sb, kc_sh, seq_lens,
+                   max_seq_len, k_per_seq, k_uniform, k_max, Hq, Hkv, chunk_tokens, (const int32_t *)ws_hist, idx,
+                   idx_sb, idx_sh, count, hist_out);
+    if (e != cudaSuccess) return e;
     count_launch(2);
     return cudaGetLastError();
 }
