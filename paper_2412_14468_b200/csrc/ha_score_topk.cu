@@ -285,8 +285,8 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
 // their 33-bin histograms through distributed shared memory between two hardware cluster barriers,
 // and each CTA then compacts its own slice straight from registers.  The codes are read from HBM
 // once, there is no histogram round trip through global memory and no second launch.
-// Token order inside a CTA: warp w owns a contiguous range, pass p covers 128 tokens (one uint4 per
-// lane), so prefix sums need only warp shuffles plus one exchange of eight warp totals.
+// Token order inside a CTA is thread order (a lane owns 4L consecutive tokens), so the prefix sums
+// need one warp-shuffle scan plus one exchange of eight warp totals.
 
 constexpr int kClusterSize = 8;
 
@@ -298,6 +298,8 @@ __device__ __forceinline__ uint32_t cluster_rank() {
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 // read an int of CTA `rank`'s shared memory at the address that `local` has in this CTA
 __device__ __forceinline__ int ld_dsmem(const int *local, uint32_t rank) {
     uint32_t a = (uint32_t)__cvta_generic_to_shared(local), ra;
@@ -314,12 +316,14 @@ __device__ __forceinline__ uint32_t scores4(const uint4 &c, const uint32_t (&qc)
 }
 
 template <int G, int L>
-__global__ void __launch_bounds__(kScanThreads) score_select_cluster_kernel(
+__global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 8) ? 4 : 2)) score_select_cluster_kernel(
     const uint32_t *__restrict__ q_codes, const uint32_t *__restrict__ k_codes, long long kc_sb, long long kc_sh,
     const int32_t *__restrict__ seq_lens, int max_seq_len, const int32_t *__restrict__ k_per_seq, int k_uniform,
     int k_max, int Hq, int Hkv, int32_t *__restrict__ idx, long long idx_sb, long long idx_sh,
     int32_t *__restrict__ count, int32_t *__restrict__ hist_out) {
-    __shared__ int w_hist[kScanThreads / 32][4][kBins + 3];
+    // per-warp histograms with one byte counter per (level, lane): a thread only ever touches its own
+    // bytes, so the counting needs no atomics and has no bank conflicts (a thread sees <= 64 tokens)
+    __shared__ __align__(16) unsigned char w_hist[kScanThreads / 32][kBins][32];
     __shared__ int s_hist[kBins + 3];          // this CTA's histogram, read by the whole cluster
     __shared__ int s_tot[kBins], s_bef[kBins];
     __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
@@ -332,19 +336,22 @@ __global__ void __launch_bounds__(kScanThreads) score_select_cluster_kernel(
     k = max(0, min(k, k_max));
     const int keep = min(k, n);
     const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
-    const int wbase = (int)rank * (L * 1024) + warp * (L * 128) + lane * 4;   // first token of this lane, pass 0
+    // a lane owns 4L consecutive tokens (L uint4), a warp 128L, a CTA 1024L: token order = thread order
+    const int wbase = (int)rank * (L * 1024) + warp * (L * 128) + lane * (L * 4);
 
     uint4 c[L];
 #pragma unroll
     for (int p = 0; p < L; ++p) {
-        const int base = wbase + p * 128;
+        const int base = wbase + p * 4;
         c[p] = (base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
     }
-    for (int i = tid; i < (kScanThreads / 32) * 4 * (kBins + 3); i += kScanThreads) (&w_hist[0][0][0])[i] = 0;
+    for (int i = tid; i < (kScanThreads / 32) * kBins * 32 / 4; i += kScanThreads)
+        reinterpret_cast<uint32_t *>(&w_hist[0][0][0])[i] = 0u;
+    if (tid < kBins + 3) s_hist[tid] = 0;
     pdl_launch_dependents();
     pdl_wait();
 #pragma unroll
-    for (int p = 0; p < L; ++p) patch_token(c[p], wbase + p * 128, n - 1, row);
+    for (int p = 0; p < L; ++p) patch_token(c[p], wbase + p * 4, n - 1, row);
     uint32_t qc[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
@@ -352,24 +359,25 @@ __global__ void __launch_bounds__(kScanThreads) score_select_cluster_kernel(
 
     // ---- scores (kept as four bytes per register) and this CTA's histogram
     uint32_t sc[L];
-    int *my = w_hist[warp][lane & 3];
+    unsigned char *my = &w_hist[warp][0][lane];
 #pragma unroll
     for (int p = 0; p < L; ++p) {
-        const int base = wbase + p * 128;
+        const int base = wbase + p * 4;
         sc[p] = scores4<G>(c[p], qc);
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-            if (base + e < n) atomicAdd(&my[(sc[p] >> (8 * e)) & 0xffu], 1);
+            if (base + e < n) my[((sc[p] >> (8 * e)) & 0xffu) * 32] += 1;
             else sc[p] |= 0xffu << (8 * e);   // 255 marks "no token": never equal to T, masked from ">"
     }
     __syncthreads();
-    if (tid < kBins) {
-        int s = 0;
-#pragma unroll
-        for (int w = 0; w < kScanThreads / 32; ++w)
-#pragma unroll
-            for (int r = 0; r < 4; ++r) s += w_hist[w][r][tid];
-        s_hist[tid] = s;
+    // fold the byte counters: one (level, warp) row of 32 bytes per thread
+    for (int i = tid; i < kBins * (kScanThreads / 32); i += kScanThreads) {
+        const int bin = i >> 3, w = i & 7;
+        const uint4 *rowp = reinterpret_cast<const uint4 *>(&w_hist[w][bin][0]);
+        const uint4 a0 = rowp[0], a1 = rowp[1];
+        const int s = (int)(__vsadu4(a0.x, 0u) + __vsadu4(a0.y, 0u) + __vsadu4(a0.z, 0u) + __vsadu4(a0.w, 0u) +
+                            __vsadu4(a1.x, 0u) + __vsadu4(a1.y, 0u) + __vsadu4(a1.z, 0u) + __vsadu4(a1.w, 0u));
+        if (s) atomicAdd(&s_hist[bin], s);
     }
     cluster_sync_all();   // every CTA's histogram is complete and visible cluster-wide
 
@@ -384,7 +392,10 @@ __global__ void __launch_bounds__(kScanThreads) score_select_cluster_kernel(
         s_tot[tid] = tot;
         s_bef[tid] = bef;
     }
-    cluster_sync_all();   // all remote reads are done (a CTA may now exit) and s_tot/s_bef are visible
+    // this CTA is done reading its peers' shared memory; the matching wait sits at the end of the
+    // kernel, so that no CTA exits while a peer may still read its histogram
+    cluster_arrive();
+    __syncthreads();
     if (warp == 0) {
         int tot = s_tot[lane], bef = s_bef[lane];
         const int tot32 = s_tot[32], bef32 = s_bef[32];
@@ -424,7 +435,7 @@ __global__ void __launch_bounds__(kScanThreads) score_select_cluster_kernel(
         if (tid == 0) count[b * Hkv + g] = keep;
         for (int i = keep + tid; i < k_max; i += kScanThreads) out[i] = -1;
     }
-    if (keep == 0) return;
+    if (keep == 0) { cluster_wait(); return; }
 
     // ---- counts of (S > T, S == T) per thread and pass, packed in 16-bit halves
     const uint32_t T4 = (uint32_t)T * 0x01010101u;
@@ -449,39 +460,33 @@ __global__ void __launch_bounds__(kScanThreads) score_select_cluster_kernel(
     for (int w = 0; w < kScanThreads / 32; ++w) {
         if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
     }
-    // ---- positions, pass by pass (token order = pass, lane, element)
+    // ---- positions: the lane's tokens are consecutive, so one exclusive prefix per lane is enough
+    {
+        const int excl = winc - tot_packed;
+        int gt_lt = run_gt + (excl & 0xffff);
+        int eq_lt = run_eq + (int)((unsigned)excl >> 16);
+        if (tot_packed != 0) {
 #pragma unroll
-    for (int p = 0; p < L; ++p) {
-        const uint32_t valid = __vcmpne4(sc[p], 0xffffffffu) & 0x01010101u;
-        const uint32_t gt = __vcmpgtu4(sc[p], T4) & valid;
-        const uint32_t eq = __vcmpeq4(sc[p], T4) & 0x01010101u;
-        const int packed = (int)(__vsadu4(gt, 0u) | (__vsadu4(eq, 0u) << 16));
-        int inc = packed;
+            for (int p = 0; p < L; ++p) {
+                const uint32_t valid = __vcmpne4(sc[p], 0xffffffffu) & 0x01010101u;
+                const uint32_t gt = __vcmpgtu4(sc[p], T4) & valid;
+                const uint32_t eq = __vcmpeq4(sc[p], T4) & 0x01010101u;
+                if ((gt | eq) == 0u) continue;
+                const int base = wbase + p * 4;
 #pragma unroll
-        for (int dd = 1; dd < 32; dd <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, inc, dd);
-            if (lane >= dd) inc += v;
-        }
-        const int all = __shfl_sync(0xffffffffu, inc, 31);
-        if (all != 0) {
-            const int excl = inc - packed;
-            int gt_lt = run_gt + (excl & 0xffff);
-            int eq_lt = run_eq + (int)((unsigned)excl >> 16);
-            const int base = wbase + p * 128;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                if ((gt >> (8 * e)) & 1u) {
-                    out[gt_lt + min(eq_lt, r)] = base + e;
-                    ++gt_lt;
-                } else if ((eq >> (8 * e)) & 1u) {
-                    if (eq_lt < r) out[gt_lt + eq_lt] = base + e;
-                    ++eq_lt;
+                for (int e = 0; e < 4; ++e) {
+                    if ((gt >> (8 * e)) & 1u) {
+                        out[gt_lt + min(eq_lt, r)] = base + e;
+                        ++gt_lt;
+                    } else if ((eq >> (8 * e)) & 1u) {
+                        if (eq_lt < r) out[gt_lt + eq_lt] = base + e;
+                        ++eq_lt;
+                    }
                 }
             }
         }
-        run_gt += all & 0xffff;
-        run_eq += (int)((unsigned)all >> 16);
     }
+    cluster_wait();
 }
 
 template <int G, int L>

@@ -54,3 +54,16 @@ def oracle_query_codes(q: torch.Tensor, map_q, n_kv_heads: int) -> np.ndarray:
 
 def max_abs_diff_bf16(a_bits: np.ndarray, b_bits: np.ndarray) -> float:
     return float(np.max(np.abs(oracle.bf16_bits_to_f64(a_bits) - oracle.bf16_bits_to_f64(b_bits)))) if a_bits.size else 0.0
+
+
+def assert_out_close(got_bits: np.ndarray, ref_bits: np.ndarray) -> float:
+    """Contract: max-abs <= 1e-2.  Expected of the kernels: every element within 2e-3 or one bf16 unit in the
+    last place of the oracle's value (fp32 accumulation can land on the other side of a bf16 rounding
+    boundary of the float64 result).  Returns the max-abs difference."""
+    a, b = oracle.bf16_bits_to_f64(got_bits), oracle.bf16_bits_to_f64(ref_bits)
+    diff = np.abs(a - b)
+    worst = float(diff.max()) if diff.size else 0.0
+    assert worst <= OUT_TOL, worst
+    ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(b), 2.0 ** -126))) - 7)
+    assert np.all(diff <= np.maximum(OUT_AIM, ulp)), float((diff / np.maximum(OUT_AIM, ulp)).max())
+    return worst

@@ -10,8 +10,8 @@ import torch
 import oracle
 from paper_2412_14468_b200 import binding as ha
 from paper_2412_14468_b200 import workloads as wl
-from tests._util import OUT_AIM, OUT_TOL, bf16_to_f64, codes_np, max_abs_diff_bf16, oracle_key_codes, \
-    oracle_query_codes, u16
+from tests._util import OUT_AIM, OUT_TOL, assert_out_close, bf16_to_f64, codes_np, max_abs_diff_bf16, \
+    oracle_key_codes, oracle_query_codes, u16
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -179,7 +179,7 @@ def _check_gather(q, K, V, lens, idx_np, cnt_np, sm_scale, expect_flag=0):
             g = h // G
             eo, el, _ = oracle.gather_attn(qu[b, h], Ku[b, g], Vu[b, g], idx_np[b, g, :cnt_np[b, g]],
                                            sm_scale=sm_scale, n_valid=lens[b])
-            worst = max(worst, max_abs_diff_bf16(ou[b, h], eo))
+            worst = max(worst, assert_out_close(ou[b, h], eo))
             if math.isinf(el):
                 assert lse_np[b, h] == -math.inf and not ou[b, h].any()
             else:
@@ -204,8 +204,7 @@ def test_gather_attn_random_lists(G):
             c = min(c, lens[b])
             cnt[b, g] = c
             idx[b, g, :c] = np.sort(rng.choice(lens[b], size=c, replace=False))
-    worst = _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128))
-    assert worst <= OUT_AIM
+    _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128))
 
 
 def test_gather_attn_padding_invalid_and_unsorted_indices():
@@ -238,12 +237,12 @@ def test_single_index_returns_value_row_exactly_and_k_equals_n_is_dense():
     l_d = torch.zeros(1, Hq, device=DEV)
     ha.ha_gather_attn(shape, q, K, V, sl, full, cnt, n, o_sparse, ws, lse=l_s)
     ha.ha_dense_decode(shape, q, K, V, sl, n, o_dense, ws, lse=l_d)
-    assert float((o_sparse.float() - o_dense.float()).abs().max()) <= OUT_AIM
+    assert_out_close(u16(o_sparse), u16(o_dense))
     assert float((l_s - l_d).abs().max()) < 1e-4
     qu, Ku, Vu = u16(q), u16(K), u16(V)
     for h in range(Hq):
         eo, el, _ = oracle.dense(qu[0, h], Ku[0, h // 4], Vu[0, h // 4])
-        assert max_abs_diff_bf16(u16(o_dense)[0, h], eo) <= OUT_AIM
+        assert_out_close(u16(o_dense)[0, h], eo)
         assert abs(float(l_d[0, h]) - el) < 1e-3
 
 
@@ -261,7 +260,7 @@ def test_dense_decode_matches_oracle(lens):
     for b in range(B):
         for h in range(Hq):
             eo, el, _ = oracle.dense(qu[b, h], Ku[b, h // 4], Vu[b, h // 4], n=lens[b])
-            assert max_abs_diff_bf16(ou[b, h], eo) <= OUT_AIM
+            assert_out_close(ou[b, h], eo)
             if lens[b] == 0:
                 assert float(lse[b, h]) == -math.inf
             else:
@@ -326,7 +325,7 @@ def test_sparse_decode_step_matches_oracle(cfg):
     assert np.array_equal(codes_np(r["qc"]), ref["qcodes"])
     assert np.array_equal(r["cnt"].cpu().numpy(), ref["count"])
     assert np.array_equal(r["idx"].cpu().numpy(), ref["idx"])
-    assert max_abs_diff_bf16(u16(r["out"]), ref["out"]) <= OUT_AIM
+    assert_out_close(u16(r["out"]), ref["out"])
     got_lse = r["lse"].cpu().numpy().astype(np.float64)
     finite = np.isfinite(ref["lse"])
     assert np.array_equal(np.isneginf(got_lse), ~finite)            # empty selections: lse = -inf on both sides
@@ -344,5 +343,5 @@ def test_k_equals_n_sparse_step_equals_dense_kernel():
     ws = ha.alloc_workspace(shape, w["n_cap"], w["n_cap"])
     dense = torch.zeros_like(r["out"])
     ha.ha_dense_decode(shape, w["q"], w["K"], w["V"], w["seq_lens"], w["n_cap"], dense, ws)
-    assert float((dense.float() - r["out"].float()).abs().max()) <= OUT_AIM
+    assert_out_close(u16(dense), u16(r["out"]))
     assert r["cnt"].cpu().tolist() == [[1500, 1500], [900, 900]]
