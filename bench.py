@@ -130,7 +130,7 @@ class Bench:
         from paper_2412_14468_b200 import workloads as wl
         self.torch, self.ha, self.wl = torch, ha, wl
         self.device = device
-        cfg = wl.CONFIGS[cfg_name]
+        cfg = wl.CONFIGS[cfg_name] if isinstance(cfg_name, str) else cfg_name
         self.cfg = cfg
         base = (wl.BASE_SEED + cfg.index) if seed_base is None else seed_base
         self.reps = [Replica(cfg, base + 100003 * r, device, ha, wl, torch) for r in range(n_replicas)]
@@ -331,7 +331,7 @@ def main():
     g_us = parts["ha_gather_attn"]
     achieved = gather_bytes / (g_us * 1e-6) / 1e9
     roofline = {
-        "bound": "hbm", "kernel": "attn_partial_kernel (ha_gather_attn; includes its combine kernel)",
+        "bound": "hbm", "kernel": "attn_kernel<4,true> (the one kernel of ha_gather_attn)",
         "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
         "traffic": None, "algorithmic_bytes_per_launch": gather_bytes, "us_per_launch": g_us,
         "whole_step": {"algorithmic_bytes": alg_bytes, "achieved": alg_bytes / (us_per_step * 1e-6) / 1e9,
@@ -373,9 +373,12 @@ def main():
     if not args.no_supplementary and world == 1:
         del bench
         torch.cuda.empty_cache()
-        for name, reps_n, st in (("c3", 2, 400), ("c4", 2, 400)):
+        cases = [("c3", wl.CONFIGS["c3"], 2, 400), ("c4", wl.CONFIGS["c4"], 2, 400), ("c5", wl.CONFIGS["c5"], 2, 200)]
+        for bsz in (4, 16, 64):   # batch sweep at the headline shape: 32K context, 32x
+            cases.append((f"sweep_B{bsz}_32K_32x", wl.Config(f"sweep{bsz}", 10 + bsz, bsz, 32768, 1024, 0.01), 2 if bsz >= 16 else 8, 400))
+        for name, cfg_s, reps_n, st in cases:
             try:
-                b2 = Bench(name, reps_n, device)
+                b2 = Bench(cfg_s, reps_n, device)
                 l2, k2 = b2.reps[0].w["lens"], b2.reps[0].w["ks"]
                 ab = wl.algorithmic_bytes(l2, k2)
                 t_all, _ = b2.time_steps(b2.step, st, 20)
@@ -383,9 +386,11 @@ def main():
                 t_ga, _ = b2.time_steps(b2.gather, st, 20)
                 t_de, _ = b2.time_steps(b2.dense, 40, 4)
                 us = t_all * 1e3 / st
+                gb = sum(8 * 512 * min(kk, nn) + 32 * 512 for nn, kk in zip(l2, k2))
                 supplementary[name] = {
                     "us_per_layer_step": us, "algorithmic_bytes": ab, "achieved_gbs": ab / (us * 1e-6) / 1e9,
                     "frac": ab / (us * 1e-6) / 1e9 / peak, "score_topk_us": t_sc * 1e3 / st, "gather_attn_us": t_ga * 1e3 / st,
+                    "gather_attn_frac": gb / (t_ga * 1e3 / st * 1e-6) / 1e9 / peak,
                     "dense_us": t_de * 1e3 / 40, "dense_frac": wl.dense_bytes(l2) / (t_de * 1e3 / 40 * 1e-6) / 1e9 / peak,
                     "replicas": reps_n,
                 }
