@@ -42,6 +42,7 @@ extern "C" {
 #define HA_ERR_UNSUPPORTED 2 /* head_dim != 128, n_bits != 32, group size > 8, ... */
 #define HA_ERR_WORKSPACE 3   /* workspace NULL, misaligned or smaller than ha_workspace_bytes */
 #define HA_ERR_CUDA 4        /* a CUDA runtime call failed (launch error, bad stream) */
+#define HA_ERR_STATIC_LIMIT 5 /* ha_gather_attn_static: problem larger than the library's built-in scratch */
 
 /* bits of the device status word (ha_read_device_status) */
 #define HA_DEV_BAD_INDEX 1u /* an idx entry >= seq_len was met and skipped */
@@ -168,6 +169,34 @@ int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const 
                           int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
                           int64_t idx_stride_h, int32_t *count, uint16_t *out_host,
                           void *workspace, size_t ws_bytes, void *stream);
+
+/* GATHER-ATT without a caller-provided workspace.  (The paper has no counterpart of this entry
+ * point; it exists for integration reasons only.)
+ *
+ * Some callers cannot give this library scratch memory because they cannot allocate device memory
+ * at the point where they call it: a serving process that handed the whole GPU to its own memory
+ * pool at start-up and has no hook to carve a buffer out of it for a third-party library, a
+ * plug-in that is invoked from inside another runtime's operator callback where only kernel
+ * launches are permitted, or a latency-critical loop that must not risk the implicit device
+ * synchronisation of cudaMalloc/cudaFree.  For them this variant of ha_gather_attn keeps the
+ * split-K states, the ticket counters and the status word in a fixed array inside the library's
+ * device image (about 2.4 MB, held by every GPU that loads the library until the process exits).
+ * It calls no cudaMalloc, cudaFree or other allocating routine; inputs and outputs are still the
+ * caller's.  Same arguments and results as ha_gather_attn, minus the workspace.
+ *
+ * Limits: batch * n_kv_heads <= 64, and a GPU with at most 256 SMs; anything larger returns
+ * HA_ERR_STATIC_LIMIT and enqueues nothing.
+ * First call on a device: looks up the array's device address (once per device, that device must
+ * be current); make that first call before any stream capture begins.
+ * Sharing: every call on a device uses the same array and finds in it what the previous call left;
+ * the call clears the words that must start at zero itself.  Two calls that can overlap on the
+ * GPU (different streams without ordering) race on the array: order them.
+ * An index outside its sequence is skipped as in ha_gather_attn; the status word it would flag is
+ * internal to the array and not readable through this entry point. */
+int ha_gather_attn_static(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
+                          const ha_tensor *V, const int32_t *seq_lens, const int32_t *idx,
+                          int64_t idx_stride_b, int64_t idx_stride_h, const int32_t *count,
+                          int32_t k_max, uint16_t *out, float *lse, void *stream);
 
 /* Copies the device status word to *flags (host) and clears nothing; synchronises `stream`. */
 int ha_read_device_status(void *workspace, void *stream, uint32_t *flags);

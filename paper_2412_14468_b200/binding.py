@@ -16,13 +16,13 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhashattn.so")
 
 HA_OK = 0
-HA_ERR_INVALID_ARG, HA_ERR_UNSUPPORTED, HA_ERR_WORKSPACE, HA_ERR_CUDA = 1, 2, 3, 4
+HA_ERR_INVALID_ARG, HA_ERR_UNSUPPORTED, HA_ERR_WORKSPACE, HA_ERR_CUDA, HA_ERR_STATIC_LIMIT = 1, 2, 3, 4, 5
 HA_DEV_BAD_INDEX, HA_DEV_TIMEOUT = 1, 2
 HIST_BINS = 33
 
 EXPORTS = [
     "ha_workspace_bytes", "ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn",
-    "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
+    "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
 
@@ -66,6 +66,7 @@ def lib() -> C.CDLL:
         L.ha_encode.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, P, P]
         L.ha_score_topk.argtypes = [P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64, P, P, P, SZ, P]
         L.ha_gather_attn.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P, SZ, P]
+        L.ha_gather_attn_static.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P]
         L.ha_dense_decode.argtypes = [P, P, P, P, P, I32, P, P, P, SZ, P]
         L.ha_sparse_decode.argtypes = [P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, P, I64, I64, P,
                                        P, P, P, SZ, P]
@@ -76,7 +77,7 @@ def lib() -> C.CDLL:
         L.ha_status_string.restype = C.c_char_p
         L.ha_status_string.argtypes = [C.c_int]
         L.ha_version.restype = C.c_char_p
-        for fn in ("ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn", "ha_dense_decode",
+        for fn in ("ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn", "ha_gather_attn_static", "ha_dense_decode",
                    "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status"):
             getattr(L, fn).restype = C.c_int
         _lib = L
@@ -203,6 +204,16 @@ def ha_gather_attn(shape: ha_shape, q, K, V, seq_lens, idx, count, k_max: int, o
     _check("ha_gather_attn", lib().ha_gather_attn(
         C.byref(shape), q.data_ptr(), C.byref(kt), C.byref(vt), seq_lens.data_ptr(), idx.data_ptr(), idx.stride(0),
         idx.stride(1), count.data_ptr(), k_max, out.data_ptr(), _ptr(lse), p, n, _stream(stream)))
+
+
+def ha_gather_attn_static(shape: ha_shape, q, K, V, seq_lens, idx, count, k_max: int, out, lse=None, stream=None) -> None:
+    """ha_gather_attn for callers that cannot allocate a workspace: the scratch is a fixed array inside
+    the library (batch * n_kv_heads <= 64).  Make the first call on a device outside stream capture;
+    calls that may overlap on the GPU must be ordered by the caller."""
+    kt, vt = make_tensor(K), make_tensor(V)
+    _check("ha_gather_attn_static", lib().ha_gather_attn_static(
+        C.byref(shape), q.data_ptr(), C.byref(kt), C.byref(vt), seq_lens.data_ptr(), idx.data_ptr(), idx.stride(0),
+        idx.stride(1), count.data_ptr(), k_max, out.data_ptr(), _ptr(lse), _stream(stream)))
 
 
 def ha_dense_decode(shape: ha_shape, q, K, V, seq_lens, max_seq_len: int, out, workspace, lse=None,

@@ -277,6 +277,7 @@ const char *ha_status_string(int status) {
         case HA_ERR_UNSUPPORTED: return "unsupported configuration";
         case HA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case HA_ERR_CUDA: return "CUDA runtime error";
+        case HA_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of ha_gather_attn_static (batch * n_kv_heads <= 64)";
         default: return "unknown status";
     }
 }

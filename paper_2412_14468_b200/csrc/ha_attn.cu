@@ -552,3 +552,69 @@ cudaError_t launch_append_kv(int B, int Hkv, const uint16_t *k_new, const uint16
 }
 
 } // namespace ha
+
+// ------------------------------------------------------------------ entry point with built-in scratch
+//
+// ha_gather_attn_static: GATHER-ATT for callers that cannot hand the library a workspace because
+// they cannot allocate device memory themselves (see include/hashattn.h).  The split-K states, the
+// ticket counters and the status word live in the file-scope array below, which every GPU that
+// loads the library carries until the process exits.
+
+namespace ha {
+constexpr int kStaticMaxUnits = 64;     // (sequence, KV head) pairs
+constexpr int kStaticMaxCtas = 512;     // persistent CTAs (2 per SM) the scratch has room for
+constexpr size_t kStaticSlots = (size_t)kStaticMaxCtas + kStaticMaxUnits;
+constexpr size_t kStaticTicketsOff = 256;                                    // after the status word
+constexpr size_t kStaticMlOff = kStaticTicketsOff + 256;                     // 64 counters x 4 bytes
+constexpr size_t kStaticAccOff = kStaticMlOff + ((kStaticSlots * kMaxGroup * 2 * 4 + 255) / 256) * 256;
+constexpr size_t kStaticBytes = kStaticAccOff + kStaticSlots * kMaxGroup * kD * 4;   // about 2.4 MB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+} // namespace ha
+
+extern "C" int ha_gather_attn_static(const ha_shape *shape, const uint16_t *q, const ha_tensor *K, const ha_tensor *V,
+                                     const int32_t *seq_lens, const int32_t *idx, int64_t idx_stride_b,
+                                     int64_t idx_stride_h, const int32_t *count, int32_t k_max, uint16_t *out,
+                                     float *lse, void *stream) {
+    using namespace ha;
+    if (!shape || !q || !K || !V || !K->ptr || !V->ptr || !seq_lens || !idx || !count || !out || k_max < 0)
+        return HA_ERR_INVALID_ARG;
+    if (shape->batch < 0 || shape->n_q_heads <= 0 || shape->n_kv_heads <= 0) return HA_ERR_INVALID_ARG;
+    if (shape->head_dim != kD || shape->n_q_heads % shape->n_kv_heads != 0) return HA_ERR_UNSUPPORTED;
+    const int G = shape->n_q_heads / shape->n_kv_heads;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return HA_ERR_UNSUPPORTED;
+    if (((uintptr_t)q & 15) || ((uintptr_t)K->ptr & 15) || ((uintptr_t)V->ptr & 15) || (K->stride_b & 7) ||
+        (K->stride_h & 7) || (K->stride_n & 7) || (V->stride_b & 7) || (V->stride_h & 7) || (V->stride_n & 7) ||
+        K->stride_n < kD || V->stride_n < kD)
+        return HA_ERR_INVALID_ARG;
+    // the built-in scratch is sized for at most kStaticMaxUnits units and kStaticMaxCtas CTAs
+    if ((long long)shape->batch * shape->n_kv_heads > kStaticMaxUnits) return HA_ERR_STATIC_LIMIT;
+    if (2 * sm_count() > kStaticMaxCtas) return HA_ERR_STATIC_LIMIT;
+    if (shape->batch == 0) return HA_OK;
+
+    // Set-up, once per device: in host code the array's name is only a stand-in for the symbol; the
+    // device address that a kernel can use has to be asked for, with the device current.
+    static void *scratch_of_device[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HA_ERR_CUDA;
+    if (!scratch_of_device[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return HA_ERR_CUDA;
+        scratch_of_device[dev] = p;
+    }
+    unsigned char *base = reinterpret_cast<unsigned char *>(scratch_of_device[dev]);
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the last call left: the status word and the ticket counters must start at zero
+    if (cudaMemsetAsync(base, 0, kStaticMlOff, st) != cudaSuccess) return HA_ERR_CUDA;
+    TensorView Kv{reinterpret_cast<const uint16_t *>(K->ptr), (long long)K->stride_b, (long long)K->stride_h,
+                  (long long)K->stride_n};
+    TensorView Vv{reinterpret_cast<const uint16_t *>(V->ptr), (long long)V->stride_b, (long long)V->stride_h,
+                  (long long)V->stride_n};
+    if (launch_attention(true, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, Kv, Vv, seq_lens,
+                         idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
+                         reinterpret_cast<float *>(base + kStaticMlOff), reinterpret_cast<float *>(base + kStaticAccOff),
+                         reinterpret_cast<int32_t *>(base + kStaticTicketsOff), reinterpret_cast<uint32_t *>(base),
+                         st) != cudaSuccess)
+        return HA_ERR_CUDA;
+    return HA_OK;
+}
+
