@@ -13,50 +13,73 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t h) { return __uint_
 // ------------------------------------------------------------------ decode-step kernel
 //
 // One CTA per (sequence, network): the G query vectors that share a network (or the one new key)
-// are encoded together, so the 72 KB of weights are fetched once per CTA.  All three weight
-// matrices are requested with cp.async at kernel entry (one HBM/L2 round trip instead of one per
-// unrolled batch of a dependent loop); each layer starts as soon as its matrix has landed.  Thread
-// o runs the fma chain of output o for every vector of the CTA (independent chains interleave).
+// are encoded together, so the 72 KB of weights are fetched once per CTA.  One thread requests the
+// three weight matrices with bulk asynchronous copies (TMA, one mbarrier per matrix) at kernel
+// entry, before the programmatic-launch wait: the fetch overlaps the preceding kernels and costs no
+// issue slots; each layer starts as soon as its matrix has landed.  Thread (o, half) runs the fma
+// chain of output o for one half of the CTA's vectors; two warps per scheduler hide the
+// shared-memory latency of each other's chains.
 
-constexpr int kVecThreads = 128;
-constexpr int kVecMax = 8;   // vectors per CTA
-constexpr size_t kVecSmem = (size_t)(kD * kHid + kHid * kHid + kHid * kBits) * 2 + (size_t)2 * kVecMax * kD * 4;
+constexpr int kVecThreads = 256;
+constexpr size_t kVecWeightBytes = (size_t)(kD * kHid + kHid * kHid + kHid * kBits) * 2;
 
-__device__ __forceinline__ void cp_async16_enc(uint32_t dst, const void *src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Bounded wait for phase 0 of an mbarrier.  Returns false if the copy has not completed after the
+// limit (never seen; the caller then fetches the data with ordinary loads instead).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar) {
+    for (int it = 0; it < (1 << 20); ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(0u) : "memory");
+        if (done) return true;
+    }
+    return false;
 }
 
-template <int NV>
+// z[v] += sum_k hin[v][k] * w[k][o], ascending k, one fmaf per term; the VT chains are independent.
+template <int VT>
 __device__ __forceinline__ void vec_layer(const float *__restrict__ hin, const uint16_t *__restrict__ w, int ld,
-                                          int o, int nv, float (&z)[NV]) {
-    // z[v] += sum_k hin[v][k] * w[k][o], ascending k, one fmaf per term
-#pragma unroll 4
+                                          int o, float (&z)[VT]) {
+#pragma unroll 8
     for (int k = 0; k < 128; k += 4) {
         const float w0 = bf16_bits_to_float(w[(k + 0) * ld + o]);
         const float w1 = bf16_bits_to_float(w[(k + 1) * ld + o]);
         const float w2 = bf16_bits_to_float(w[(k + 2) * ld + o]);
         const float w3 = bf16_bits_to_float(w[(k + 3) * ld + o]);
+        float4 hv[VT];
 #pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            if (v < nv) {
-                const float4 hv = *reinterpret_cast<const float4 *>(hin + v * kD + k);   // warp broadcast
-                z[v] = __fmaf_rn(hv.x, w0, z[v]);
-                z[v] = __fmaf_rn(hv.y, w1, z[v]);
-                z[v] = __fmaf_rn(hv.z, w2, z[v]);
-                z[v] = __fmaf_rn(hv.w, w3, z[v]);
-            }
-        }
+        for (int v = 0; v < VT; ++v) hv[v] = *reinterpret_cast<const float4 *>(hin + v * kD + k);   // warp broadcast
+#pragma unroll
+        for (int v = 0; v < VT; ++v) z[v] = __fmaf_rn(hv[v].x, w0, z[v]);
+#pragma unroll
+        for (int v = 0; v < VT; ++v) z[v] = __fmaf_rn(hv[v].y, w1, z[v]);
+#pragma unroll
+        for (int v = 0; v < VT; ++v) z[v] = __fmaf_rn(hv[v].z, w2, z[v]);
+#pragma unroll
+        for (int v = 0; v < VT; ++v) z[v] = __fmaf_rn(hv[v].w, w3, z[v]);
     }
 }
 
 template <int NV>
 __global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, EncodeJob jb) {
-    extern __shared__ __align__(16) unsigned char smem[];
-    uint16_t *sw1 = reinterpret_cast<uint16_t *>(smem);
+    constexpr int VT = (NV + 1) / 2;   // vectors per thread: half h owns vectors h*VT .. h*VT+VT-1
+    constexpr int NS = 2 * VT;         // vector slots in shared memory (>= NV)
+    extern __shared__ __align__(128) unsigned char vec_smem[];
+    __shared__ __align__(8) unsigned long long s_bar[3];
+    uint16_t *sw1 = reinterpret_cast<uint16_t *>(vec_smem);
     uint16_t *sw2 = sw1 + kD * kHid;
     uint16_t *sw3 = sw2 + kHid * kHid;
-    float *actA = reinterpret_cast<float *>(sw3 + kHid * kBits);   // [NV][128]
-    float *actB = actA + kVecMax * kD;
+    float *actA = reinterpret_cast<float *>(sw3 + kHid * kBits);   // [NS][128]
+    float *actB = actA + NS * kD;
 
     int i = blockIdx.x;
     const bool second = i >= ja.n_cta;
@@ -65,67 +88,84 @@ __global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, E
     const int n_nets = J.n_heads / J.heads_per_kv;
     const int b = i / n_nets, net = i % n_nets;
     const int nv = J.heads_per_kv;   // <= NV
-    const int o = threadIdx.x;
+    const int tid = threadIdx.x, o = tid & 127, half = tid >> 7;
 
-    // ---- request all weights (three commit groups), then the inputs
-    {
-        const unsigned char *g1 = reinterpret_cast<const unsigned char *>(J.map.w1 + (size_t)net * kD * kHid);
-        const unsigned char *g2 = reinterpret_cast<const unsigned char *>(J.map.w2 + (size_t)net * kHid * kHid);
-        const unsigned char *g3 = reinterpret_cast<const unsigned char *>(J.map.w3 + (size_t)net * kHid * kBits);
-        const uint32_t s1 = (uint32_t)__cvta_generic_to_shared(sw1), s2 = (uint32_t)__cvta_generic_to_shared(sw2),
-                       s3 = (uint32_t)__cvta_generic_to_shared(sw3);
-        for (int c = o; c < kD * kHid / 8; c += kVecThreads) cp_async16_enc(s1 + c * 16, g1 + c * 16);
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        for (int c = o; c < kHid * kHid / 8; c += kVecThreads) cp_async16_enc(s2 + c * 16, g2 + c * 16);
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        for (int c = o; c < kHid * kBits / 8; c += kVecThreads) cp_async16_enc(s3 + c * 16, g3 + c * 16);
-        asm volatile("cp.async.commit_group;" ::: "memory");
+    const uint16_t *g1 = J.map.w1 + (size_t)net * kD * kHid;
+    const uint16_t *g2 = J.map.w2 + (size_t)net * kHid * kHid;
+    const uint16_t *g3 = J.map.w3 + (size_t)net * kHid * kBits;
+    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&s_bar[0]);
+    // ---- request all weights: three bulk copies, one mbarrier each
+    if (tid == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        mbar_init(bar0 + 16, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(bar0, kD * kHid * 2);
+        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw1), g1, kD * kHid * 2, bar0);
+        mbar_expect_tx(bar0 + 8, kHid * kHid * 2);
+        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw2), g2, kHid * kHid * 2, bar0 + 8);
+        mbar_expect_tx(bar0 + 16, kHid * kBits * 2);
+        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw3), g3, kHid * kBits * 2, bar0 + 16);
     }
     const float bias1 = J.map.b1 ? __ldg(J.map.b1 + net * kHid + o) : 0.0f;
     const float bias2 = J.map.b2 ? __ldg(J.map.b2 + net * kHid + o) : 0.0f;
-    const float bias3 = (J.map.b3 && o < kBits) ? __ldg(J.map.b3 + net * kBits + o) : 0.0f;
+    const float bias3 = J.map.b3 ? __ldg(J.map.b3 + net * kBits + (tid & (kBits - 1))) : 0.0f;
     // the weights do not depend on earlier kernels of the stream; the vectors to encode may
     pdl_launch_dependents();
     pdl_wait();
-    for (int v = 0; v < nv; ++v) {
-        const uint16_t *x = J.x + (long long)b * J.x_sb + (long long)(net * J.heads_per_kv + v) * J.x_sh;
-        actA[v * kD + o] = bf16_bits_to_float(__ldg(x + o));
+#pragma unroll
+    for (int vv = 0; vv < VT; ++vv) {
+        const int v = half * VT + vv;
+        float xv = 0.0f;   // unused slots are zero rows (their chains are computed and dropped)
+        if (v < nv) {
+            const uint16_t *x = J.x + (long long)b * J.x_sb + (long long)(net * J.heads_per_kv + v) * J.x_sh;
+            xv = bf16_bits_to_float(__ldg(x + o));
+        }
+        actA[v * kD + o] = xv;
     }
-
     int slot = 0;
     if (J.slot) slot = J.slot[b] - J.slot_minus_one;   // a negative slot skips the sequence (no write below)
+    __syncthreads();   // mbarrier inits and the inputs are visible to every thread
 
-    float z[NV];
+    // wait for one weight matrix; if the bulk copy never reports completion, load it the ordinary way
+    // (the decision is taken by the whole CTA together, so that the barrier below is never divergent)
+    auto weights_ready = [&](int which, uint16_t *dst, const uint16_t *src, int n_elems) {
+        const bool ok = mbar_wait_bounded(bar0 + 8 * which);
+        if (__syncthreads_or(!ok)) {
+            for (int c = tid; c < n_elems / 8; c += kVecThreads)
+                reinterpret_cast<uint4 *>(dst)[c] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
+            __syncthreads();
+        }
+    };
+
+    float z[VT];
+    const float *inA = actA + half * VT * kD, *inB = actB + half * VT * kD;
     // ---- layer 1
-    asm volatile("cp.async.wait_group 2;" ::: "memory");
+    weights_ready(0, sw1, g1, kD * kHid);
+#pragma unroll
+    for (int v = 0; v < VT; ++v) z[v] = bias1;
+    vec_layer<VT>(inA, sw1, kHid, o, z);
+#pragma unroll
+    for (int v = 0; v < VT; ++v) actB[(half * VT + v) * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
     __syncthreads();
-#pragma unroll
-    for (int v = 0; v < NV; ++v) z[v] = bias1;
-    vec_layer<NV>(actA, sw1, kHid, o, nv, z);
-#pragma unroll
-    for (int v = 0; v < NV; ++v)
-        if (v < nv) actB[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
     // ---- layer 2
-    asm volatile("cp.async.wait_group 1;" ::: "memory");
-    __syncthreads();
+    weights_ready(1, sw2, g2, kHid * kHid);
 #pragma unroll
-    for (int v = 0; v < NV; ++v) z[v] = bias2;
-    vec_layer<NV>(actB, sw2, kHid, o, nv, z);
+    for (int v = 0; v < VT; ++v) z[v] = bias2;
+    vec_layer<VT>(inB, sw2, kHid, o, z);
     // actA was last read in layer 1, which every thread left before the barrier above
 #pragma unroll
-    for (int v = 0; v < NV; ++v)
-        if (v < nv) actA[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
-    // ---- layer 3: one output bit per lane of warp 0
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    for (int v = 0; v < VT; ++v) actA[(half * VT + v) * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
     __syncthreads();
-    if (o < kBits) {
-#pragma unroll
-        for (int v = 0; v < NV; ++v) z[v] = bias3;
-        vec_layer<NV>(actA, sw3, kBits, o, nv, z);
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const uint32_t code = __ballot_sync(0xffffffffu, z[v] > 0.0f);
-            if (o == 0 && v < nv && slot >= 0)
+    // ---- layer 3: warp w encodes vector w, one output bit per lane
+    weights_ready(2, sw3, g3, kHid * kBits);
+    {
+        const int v = tid >> 5, lane = tid & 31;
+        if (v < NS) {   // warp-uniform
+            float z3[1] = {bias3};
+            vec_layer<1>(actA + v * kD, sw3, kBits, lane, z3);
+            const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
+            if (lane == 0 && v < nv && slot >= 0)
                 J.codes[(long long)b * J.c_sb + (long long)(net * J.heads_per_kv + v) * J.c_sh + slot] = code;
         }
     }
@@ -133,16 +173,16 @@ __global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, E
 
 template <int NV>
 static cudaError_t launch_vec_t(const EncodeJob &a, const EncodeJob &b, cudaStream_t st) {
+    constexpr size_t smem = kVecWeightBytes + (size_t)2 * (2 * ((NV + 1) / 2)) * kD * 4;
     static bool done[64] = {};   // opt in to > 48 KB of shared memory once per device
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(encode_vec_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kVecSmem);
+        cudaError_t e = cudaFuncSetAttribute(encode_vec_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         done[dev] = true;
     }
-    cudaError_t e = launch_pdl(encode_vec_kernel<NV>, dim3(a.n_cta + b.n_cta), dim3(kVecThreads), kVecSmem, st, a, b);
+    cudaError_t e = launch_pdl(encode_vec_kernel<NV>, dim3(a.n_cta + b.n_cta), dim3(kVecThreads), smem, st, a, b);
     if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
