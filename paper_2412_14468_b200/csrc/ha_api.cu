@@ -38,9 +38,10 @@ static int check_tensor(const ha_tensor *t) {
     return HA_OK;
 }
 
-static int check_workspace(const ha_shape *s, void *ws, size_t bytes, WorkspaceLayout *L) {
+// max_seq_len < 0: the call does not scan signatures and needs no score bytes
+static int check_workspace(const ha_shape *s, int max_seq_len, void *ws, size_t bytes, WorkspaceLayout *L) {
     if (!ws || ((uintptr_t)ws & 255)) return HA_ERR_WORKSPACE;
-    *L = make_layout(s->batch, s->n_q_heads, s->n_kv_heads);
+    *L = make_layout(s->batch, s->n_q_heads, s->n_kv_heads, max_seq_len < 0 ? 0 : max_seq_len);
     if (bytes < L->total) return HA_ERR_WORKSPACE;
     return HA_OK;
 }
@@ -73,7 +74,7 @@ extern "C" {
 
 size_t ha_workspace_bytes(const ha_shape *shape, int32_t max_seq_len, int32_t max_k) {
     if (check_shape(shape) != HA_OK || max_seq_len < 0 || max_k < 0) return 0;
-    return make_layout(shape->batch, shape->n_q_heads, shape->n_kv_heads).total;
+    return make_layout(shape->batch, shape->n_q_heads, shape->n_kv_heads, max_seq_len).total;
 }
 
 int ha_workspace_init(void *workspace, size_t ws_bytes, void *stream) {
@@ -132,12 +133,12 @@ int ha_score_topk(const ha_shape *shape, const uint32_t *q_codes, const uint32_t
     HA_TRY(check_score_args(shape, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_uniform, k_per_seq,
                             max_seq_len, k_max, idx, count));
     WorkspaceLayout L;
-    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    HA_TRY(check_workspace(shape, max_seq_len, workspace, ws_bytes, &L));
     if (shape->batch == 0) return HA_OK;
     HA_CUDA(launch_score_topk(shape->batch, shape->n_q_heads, shape->n_kv_heads, q_codes, k_codes, kc_stride_b,
                               kc_stride_h, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx, idx_stride_b,
                               idx_stride_h, count, hist_out, ws_ptr<int32_t>(workspace, L.off_hist),
-                              (cudaStream_t)stream));
+                              ws_ptr<unsigned char>(workspace, L.off_scores), (cudaStream_t)stream));
     return HA_OK;
 }
 
@@ -151,7 +152,7 @@ int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
     if (!q || !seq_lens || !idx || !count || !out || k_max < 0) return HA_ERR_INVALID_ARG;
     if ((uintptr_t)q & 15) return HA_ERR_INVALID_ARG;
     WorkspaceLayout L;
-    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    HA_TRY(check_workspace(shape, -1, workspace, ws_bytes, &L));
     if (shape->batch == 0) return HA_OK;
     HA_CUDA(launch_attention(true, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K),
                              view(V), seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
@@ -170,7 +171,7 @@ int ha_dense_decode(const ha_shape *shape, const uint16_t *q, const ha_tensor *K
     if (!q || !seq_lens || !out || max_seq_len < 0) return HA_ERR_INVALID_ARG;
     if ((uintptr_t)q & 15) return HA_ERR_INVALID_ARG;
     WorkspaceLayout L;
-    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    HA_TRY(check_workspace(shape, -1, workspace, ws_bytes, &L));
     if (shape->batch == 0) return HA_OK;
     HA_CUDA(launch_attention(false, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K),
                              view(V), seq_lens, nullptr, 0, 0, nullptr, max_seq_len, out, lse,
@@ -194,7 +195,7 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
     HA_TRY(check_tensor(V));
     if (!q || !out || ((uintptr_t)q & 15)) return HA_ERR_INVALID_ARG;
     WorkspaceLayout L;
-    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    HA_TRY(check_workspace(shape, max_seq_len, workspace, ws_bytes, &L));
     if (shape->batch == 0) return HA_OK;
     cudaStream_t st = (cudaStream_t)stream;
     const int B = shape->batch, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
@@ -216,7 +217,7 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
     HA_CUDA(launch_encode_vectors(jq, jk, st));
     HA_CUDA(launch_score_topk(B, Hq, Hkv, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
                               max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, nullptr,
-                              ws_ptr<int32_t>(workspace, L.off_hist), st));
+                              ws_ptr<int32_t>(workspace, L.off_hist), ws_ptr<unsigned char>(workspace, L.off_scores), st));
     HA_CUDA(launch_attention(true, B, Hq, Hkv, shape->sm_scale, q, view(K), view(V), seq_lens, idx, idx_stride_b,
                              idx_stride_h, count, k_max, out, lse, ws_ptr<float>(workspace, L.off_part_ml),
                              ws_ptr<float>(workspace, L.off_part_acc), ws_ptr<int32_t>(workspace, L.off_tickets),
@@ -238,7 +239,7 @@ int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const 
     HA_TRY(check_mapping(map_q, shape->n_kv_heads));
     HA_TRY(check_mapping(map_k, shape->n_kv_heads));
     WorkspaceLayout L;
-    HA_TRY(check_workspace(shape, workspace, ws_bytes, &L));
+    HA_TRY(check_workspace(shape, max_seq_len, workspace, ws_bytes, &L));
     HA_TRY(check_score_args(shape, ws_ptr<uint32_t>(workspace, L.off_qcodes), k_codes, kc_stride_b, kc_stride_h,
                             seq_lens, k_uniform, k_per_seq, max_seq_len, k_max, idx, count));
     if (shape->batch == 0) return HA_OK;

@@ -21,8 +21,11 @@ constexpr int kMaxGroup = 8;        // query heads per KV head
 constexpr size_t kHeaderBytes = 256;   // device status word (+ padding)
 constexpr int kMaxUnits = 65536;       // (sequence, KV head) pairs: bounds the ticket region
 
-// Where each scratch region lives inside the caller's workspace.  Sizes depend on the head counts
-// and the batch only, so a workspace sized once serves every smaller call.
+// Where each scratch region lives inside the caller's workspace.  All regions but the last depend
+// on the head counts and the batch only; the score bytes of the long-sequence scan come last and
+// grow with the maximum sequence length, so a workspace sized once serves every smaller call.
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
 struct WorkspaceLayout {
     size_t off_tickets;   // i32 [B][Hkv]  arrival counters of the split-K merge; zero between calls
     size_t off_hist;      // i32 [B][Hkv][kMaxChunks][33]   per-chunk score histograms
@@ -33,12 +36,13 @@ struct WorkspaceLayout {
     size_t off_stage_v;   // bf16 [B][Hkv][128]
     size_t off_stage_out; // bf16 [B][Hq][128]
     size_t off_qcodes;    // u32 [B][Hq]
+    size_t off_scores;    // u8 [B][Hkv][round_up(max_seq_len, 16)]  group scores (long-sequence path only)
     size_t total;
 };
 
-inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline size_t score_row_bytes(int max_seq_len) { return align_up((size_t)(max_seq_len > 0 ? max_seq_len : 0), 16); }
 
-inline WorkspaceLayout make_layout(int B, int Hq, int Hkv) {
+inline WorkspaceLayout make_layout(int B, int Hq, int Hkv, int max_seq_len) {
     WorkspaceLayout L;
     size_t o = kHeaderBytes;
     L.off_tickets = o;   o = align_up(o + (size_t)B * Hkv * 4, 256);
@@ -51,17 +55,18 @@ inline WorkspaceLayout make_layout(int B, int Hq, int Hkv) {
     L.off_stage_v = o;   o = align_up(o + (size_t)B * Hkv * kD * 2, 256);
     L.off_stage_out = o; o = align_up(o + (size_t)B * Hq * kD * 2, 256);
     L.off_qcodes = o;    o = align_up(o + (size_t)B * Hq * 4, 256);
+    L.off_scores = o;    o = align_up(o + (size_t)B * Hkv * score_row_bytes(max_seq_len), 256);
     L.total = o;
     return L;
 }
 
-// Tokens of the code cache scanned by one CTA: a power of two >= 1024 chosen so that the grid has
-// about four CTAs per SM when there is that much work, and so that a sequence of max_seq_len tokens
-// needs at most kMaxChunks chunks.
+// Tokens of the code cache scanned by one CTA of the long-sequence path: a power of two >= 4096
+// (one pass of 256 threads x 16 tokens) chosen so that the grid has about four CTAs per SM when
+// there is that much work, and so that a sequence of max_seq_len tokens needs at most kMaxChunks
+// chunks.
 inline int chunk_tokens_for(int n_units, int max_seq_len) {
     const long long total = (long long)(n_units > 0 ? n_units : 1) * (max_seq_len > 0 ? max_seq_len : 1);
-    long long c = 1024;
-    if (const char *e = getenv("HA_CHUNK")) { c = atoi(e); while ((max_seq_len + c - 1) / c > kMaxChunks) c *= 2; return (int)c; }
+    long long c = 4096;
     while (c < 32768 && total / c > 148 * 4) c *= 2;
     while ((max_seq_len + c - 1) / c > kMaxChunks) c *= 2;
     return (int)c;
@@ -125,7 +130,7 @@ cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, c
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens,
                               const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max,
                               int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
-                              int32_t *hist_out, int32_t *ws_hist, cudaStream_t st);
+                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st);
 
 cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale, const uint16_t *q,
                              TensorView K, TensorView V, const int32_t *seq_lens, const int32_t *idx,

@@ -4,22 +4,22 @@
 // score T and how many tokens r of score exactly T are still needed; the selection is every token
 // above T plus the first r tokens at T in index order, written in ascending token order.
 //
-// Kernel 1 (scan_hist): each CTA streams one chunk of the code cache with 16-byte loads (all loads
-//   of a pass in flight before the first popc) and leaves the chunk's 33-bin histogram in the
-//   workspace.
-// Kernel 2 (select): each CTA sums the chunk histograms (total, and the part before its own
-//   chunk), derives T, r and its output offset with warp shuffles, re-reads its chunk (an L2 hit)
-//   and compacts the selected token indices with shuffle prefix sums.  No CTA waits on another.
-// Both kernels request their first pass of codes before the programmatic-launch wait, so that the
-// fetch overlaps the tail of the preceding kernel; the one code that the preceding ENCODE may still
-// be writing (the appended token, slot n-1) is re-read after the wait.
+// Two implementations share the arithmetic:
+//  * sequences of up to 32768 tokens: ONE kernel, a thread-block cluster per (sequence, KV head)
+//    (score_select_cluster_kernel, second half of this file);
+//  * longer sequences: two kernels over chunks of the sequence, with the per-chunk histograms and
+//    one score byte per token passed through the workspace (scan_score_kernel, select_kernel).
+// No CTA ever spins on another: hand-offs are hardware cluster barriers or kernel boundaries.
+// The scanning kernels request their first signatures before the programmatic-launch wait, so that
+// the fetch overlaps the tail of the preceding kernel; the one signature that the preceding ENCODE
+// may still be writing (the appended token, slot n-1) is re-read after the wait.
 #include "ha_common.cuh"
 
 namespace ha {
 
 constexpr int kScanThreads = 256;
 constexpr int kPassTokens = kScanThreads * 16;   // four uint4 per thread
-constexpr int kHistGroups = 7;                   // 7 * 33 threads sum the chunk histograms
+constexpr int kClusterMaxSeq = 8 * 4 * 1024;     // longest sequence the fused cluster kernel takes (4 uint4 per thread)
 
 template <int G>
 __device__ __forceinline__ int group_score(uint32_t code, const uint32_t (&qc)[G]) {
@@ -49,83 +49,108 @@ __device__ __forceinline__ void patch_token(uint4 &v, int base, int last, const 
 }
 
 template <int G>
-__global__ void __launch_bounds__(kScanThreads) scan_hist_kernel(const uint32_t *__restrict__ q_codes,
-                                                                const uint32_t *__restrict__ k_codes,
-                                                                long long kc_sb, long long kc_sh,
-                                                                const int32_t *__restrict__ seq_lens,
-                                                                int max_seq_len, int Hq, int Hkv,
-                                                                int chunk_tokens,
-                                                                int32_t *__restrict__ ws_hist) {
-    // 4 sub-histograms per warp (by lane & 3) spread same-bin updates over several addresses
-    __shared__ int hist[kScanThreads / 32][4][kBins + 3];
+__device__ __forceinline__ uint32_t scores4(const uint4 &c, const uint32_t (&qc)[G]) {
+    return (uint32_t)group_score<G>(c.x, qc) | ((uint32_t)group_score<G>(c.y, qc) << 8) |
+           ((uint32_t)group_score<G>(c.z, qc) << 16) | ((uint32_t)group_score<G>(c.w, qc) << 24);
+}
+
+// ------------------------------------------------------------------ long-sequence path (two kernels)
+
+// Kernel 1: one chunk per CTA.  Streams the chunk's signatures (four uint4 per thread in flight, the
+// next pass requested before the current one is scored), leaves the group scores as one byte per
+// token in the workspace (so that kernel 2 needs neither the signatures nor popc again) and the
+// chunk's 33-bin histogram.  Counting uses one byte counter per (level, lane): no atomics.
+template <int G>
+__global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t *__restrict__ q_codes,
+                                                                 const uint32_t *__restrict__ k_codes,
+                                                                 long long kc_sb, long long kc_sh,
+                                                                 const int32_t *__restrict__ seq_lens,
+                                                                 int max_seq_len, int Hq, int Hkv,
+                                                                 int chunk_tokens, long long score_row,
+                                                                 unsigned char *__restrict__ ws_scores,
+                                                                 int32_t *__restrict__ ws_hist) {
+    __shared__ __align__(16) unsigned char w_hist[kScanThreads / 32][kBins][32];
+    __shared__ int s_hist[kBins + 3];
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int n = min(seq_lens[b], max_seq_len);
     const int start = chunk * chunk_tokens;
     if (start >= n) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
+    uint32_t *srow = reinterpret_cast<uint32_t *>(ws_scores + ((long long)b * Hkv + g) * score_row);
     const int end = min(n, start + chunk_tokens);
 
-    // first pass of codes: sub-block j of 1024 tokens, one uint4 per thread (coalesced)
-    uint4 c[4];
+    // pass = 4096 tokens: sub-block j of 1024 tokens, one uint4 per thread (coalesced)
+    auto load_pass = [&](uint4 (&c)[4], int pass) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int base = start + j * 1024 + tid * 4;
-        c[j] = (base < end) ? load_codes4(row, base, end) : make_uint4(0, 0, 0, 0);
-    }
-    for (int i = tid; i < (kScanThreads / 32) * 4 * (kBins + 3); i += kScanThreads) (&hist[0][0][0])[i] = 0;
+        for (int j = 0; j < 4; ++j) {
+            const int base = pass + j * 1024 + tid * 4;
+            c[j] = (base < end) ? load_codes4(row, base, end) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    uint4 cur[4], nxt[4];
+    load_pass(cur, start);
+    for (int i = tid; i < (kScanThreads / 32) * kBins * 32 / 4; i += kScanThreads)
+        reinterpret_cast<uint32_t *>(&w_hist[0][0][0])[i] = 0u;
+    if (tid < kBins + 3) s_hist[tid] = 0;
     pdl_launch_dependents();
     pdl_wait();
-#pragma unroll
-    for (int j = 0; j < 4; ++j) patch_token(c[j], start + j * 1024 + tid * 4, n - 1, row);
     uint32_t qc[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
     __syncthreads();
 
-    int *my = hist[warp][lane & 3];
+    unsigned char *my = &w_hist[warp][0][lane];
     for (int pass = start; pass < end; pass += kPassTokens) {
-        if (pass > start) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int base = pass + j * 1024 + tid * 4;
-                c[j] = (base < end) ? load_codes4(row, base, end) : make_uint4(0, 0, 0, 0);
-                patch_token(c[j], base, n - 1, row);
-            }
-        }
+        if (pass + kPassTokens < end) load_pass(nxt, pass + kPassTokens);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int base = pass + j * 1024 + tid * 4;
-            if (base + 0 < end) atomicAdd(&my[group_score<G>(c[j].x, qc)], 1);
-            if (base + 1 < end) atomicAdd(&my[group_score<G>(c[j].y, qc)], 1);
-            if (base + 2 < end) atomicAdd(&my[group_score<G>(c[j].z, qc)], 1);
-            if (base + 3 < end) atomicAdd(&my[group_score<G>(c[j].w, qc)], 1);
+            if (base < end) {
+                patch_token(cur[j], base, n - 1, row);   // the appended token may just have been written
+                uint32_t s4 = scores4<G>(cur[j], qc);
+                if (base + 3 < end) {                    // whole uint4 inside the chunk: no per-token checks
+                    my[(s4 & 0xffu) * 32] += 1;
+                    my[((s4 >> 8) & 0xffu) * 32] += 1;
+                    my[((s4 >> 16) & 0xffu) * 32] += 1;
+                    my[(s4 >> 24) * 32] += 1;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (base + e < end) my[((s4 >> (8 * e)) & 0xffu) * 32] += 1;
+                        else s4 |= 0xffu << (8 * e);      // 255 marks "no token"
+                }
+                srow[base >> 2] = s4;
+            }
         }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
     }
     __syncthreads();
-    if (tid < kBins) {
-        int s = 0;
-#pragma unroll
-        for (int w = 0; w < kScanThreads / 32; ++w)
-#pragma unroll
-            for (int r = 0; r < 4; ++r) s += hist[w][r][tid];
-        ws_hist[(((long long)b * Hkv + g) * kMaxChunks + chunk) * kBins + tid] = s;
+    for (int i = tid; i < kBins * (kScanThreads / 32); i += kScanThreads) {
+        const int bin = i >> 3, w = i & 7;
+        const uint4 *rowp = reinterpret_cast<const uint4 *>(&w_hist[w][bin][0]);
+        const uint4 a0 = rowp[0], a1 = rowp[1];
+        const int s = (int)(__vsadu4(a0.x, 0u) + __vsadu4(a0.y, 0u) + __vsadu4(a0.z, 0u) + __vsadu4(a0.w, 0u) +
+                            __vsadu4(a1.x, 0u) + __vsadu4(a1.y, 0u) + __vsadu4(a1.z, 0u) + __vsadu4(a1.w, 0u));
+        if (s) atomicAdd(&s_hist[bin], s);
     }
+    __syncthreads();
+    if (tid < kBins) ws_hist[(((long long)b * Hkv + g) * kMaxChunks + chunk) * kBins + tid] = s_hist[tid];
 }
 
-template <int G>
-__global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__restrict__ q_codes,
-                                                             const uint32_t *__restrict__ k_codes,
-                                                             long long kc_sb, long long kc_sh,
-                                                             const int32_t *__restrict__ seq_lens,
-                                                             int max_seq_len,
+// Kernel 2: one chunk per CTA.  Sums the chunk histograms (total, and the part before its own
+// chunk), derives T, r and its output offset, then walks its chunk's score bytes (16 consecutive
+// tokens per thread and pass) and writes the selected token indices in ascending order.
+__global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__restrict__ seq_lens, int max_seq_len,
                                                              const int32_t *__restrict__ k_per_seq, int k_uniform,
-                                                             int k_max, int Hq, int Hkv, int chunk_tokens,
+                                                             int k_max, int Hkv, int chunk_tokens, long long score_row,
+                                                             const unsigned char *__restrict__ ws_scores,
                                                              const int32_t *__restrict__ ws_hist,
                                                              int32_t *__restrict__ idx, long long idx_sb,
                                                              long long idx_sh, int32_t *__restrict__ count,
                                                              int32_t *__restrict__ hist_out) {
-    __shared__ int part_tot[kHistGroups][kBins], part_bef[kHistGroups][kBins];
+    __shared__ int s_tot[kBins + 3], s_bef[kBins + 3];
     __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
     __shared__ int warp_tot[kScanThreads / 32];
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
@@ -136,47 +161,43 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
     const int keep = min(k, n);
     const int n_chunks = (n + chunk_tokens - 1) / chunk_tokens;
     if (chunk > 0 && chunk >= n_chunks) return;
-
-    const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
-    const int start = chunk * chunk_tokens, end = min(n, start + chunk_tokens);
-    // first pass of codes: 16 consecutive tokens per thread (token order = thread order)
-    uint4 c[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int base = start + tid * 16 + j * 4;
-        c[j] = (base < end) ? load_codes4(row, base, end) : make_uint4(0, 0, 0, 0);
-    }
+    if (tid < kBins + 3) { s_tot[tid] = 0; s_bef[tid] = 0; }
     pdl_launch_dependents();
-    pdl_wait();
-#pragma unroll
-    for (int j = 0; j < 4; ++j) patch_token(c[j], start + tid * 16 + j * 4, n - 1, row);
+    pdl_wait();   // histograms and score bytes come from the preceding kernel
 
-    // totals per score level, and the part contributed by the chunks before this one
-    if (tid < kHistGroups * kBins) {
-        const int grp = tid / kBins, bin = tid % kBins;
-        const int32_t *hb = ws_hist + ((long long)b * Hkv + g) * kMaxChunks * kBins + bin;
-        int t = 0, be = 0;
-#pragma unroll 4
-        for (int cc = grp; cc < n_chunks; cc += kHistGroups) {
-            const int v = __ldcg(hb + cc * kBins);
-            t += v;
-            if (cc < chunk) be += v;
+    const uint4 *srow = reinterpret_cast<const uint4 *>(ws_scores + ((long long)b * Hkv + g) * score_row);
+    const int start = chunk * chunk_tokens, end = min(n, start + chunk_tokens);
+    // first pass of score bytes: requested now, used after the threshold is known
+    uint4 sv_next = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+    if (chunk < n_chunks && start + tid * 16 < end) sv_next = __ldcg(srow + ((start + tid * 16) >> 4));
+
+    // totals per score level, and the part contributed by the chunks before this one: every thread
+    // fetches its share of the n_chunks x 33 counters at once and adds them up in shared memory
+    __syncthreads();
+    {
+        const int32_t *hb = ws_hist + ((long long)b * Hkv + g) * kMaxChunks * kBins;
+        const int total = n_chunks * kBins;
+        int v[(kMaxChunks * kBins + kScanThreads - 1) / kScanThreads];
+#pragma unroll
+        for (int i = 0; i < (kMaxChunks * kBins + kScanThreads - 1) / kScanThreads; ++i) {
+            const int e = tid + i * kScanThreads;
+            v[i] = (e < total) ? __ldcg(hb + e) : 0;
         }
-        part_tot[grp][bin] = t;
-        part_bef[grp][bin] = be;
+#pragma unroll
+        for (int i = 0; i < (kMaxChunks * kBins + kScanThreads - 1) / kScanThreads; ++i) {
+            const int e = tid + i * kScanThreads;
+            if (e < total && v[i] != 0) {
+                const int cc = e / kBins, bin = e - cc * kBins;
+                atomicAdd(&s_tot[bin], v[i]);
+                if (cc < chunk) atomicAdd(&s_bef[bin], v[i]);
+            }
+        }
     }
     __syncthreads();
-    int my_tot = 0;
     if (warp == 0) {
-        // lane l owns level l (0..31); level 32 is summed by every lane.  Suffix sums over the levels
+        // lane l owns level l (0..31); level 32 is read by every lane.  Suffix sums over the levels
         // give #{S >= t}; T = largest level with #{S >= T} >= keep; r = keep - #{S > T}.
-        int tot = 0, bef = 0, tot32 = 0, bef32 = 0;
-#pragma unroll
-        for (int gi = 0; gi < kHistGroups; ++gi) {
-            tot += part_tot[gi][lane]; bef += part_bef[gi][lane];
-            tot32 += part_tot[gi][32]; bef32 += part_bef[gi][32];
-        }
-        my_tot = tot;
+        const int tot = s_tot[lane], bef = s_bef[lane], tot32 = s_tot[32], bef32 = s_bef[32];
         int st = tot, sb = bef;   // suffix sums over levels lane..31
 #pragma unroll
         for (int dd = 1; dd < 32; dd <<= 1) {
@@ -206,7 +227,6 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
             if (lane == 0) hist_out[((long long)b * Hkv + g) * kBins + 32] = tot32;
         }
     }
-    (void)my_tot;
     __syncthreads();
     const int T = sh_T, r = sh_r;
     int32_t *out = idx + (long long)b * idx_sb + (long long)g * idx_sh;
@@ -216,34 +236,25 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
     }
     if (chunk >= n_chunks || keep == 0) return;
 
-    uint32_t qc[G];
-#pragma unroll
-    for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
+    const uint32_t T4 = (uint32_t)T * 0x01010101u;
     int run_gt = sh_gt_before, run_eq = sh_eq_before;   // tokens before this pass with S > T / S == T
-
     for (int pass = start; pass < end; pass += kPassTokens) {
         const int base = pass + tid * 16;
-        if (pass > start) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                c[j] = (base + j * 4 < end) ? load_codes4(row, base + j * 4, end) : make_uint4(0, 0, 0, 0);
-                patch_token(c[j], base + j * 4, n - 1, row);
-            }
-        }
-        int s[16];
+        const uint4 sv = sv_next;
+        sv_next = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+        if (base + kPassTokens < end) sv_next = __ldcg(srow + ((base + kPassTokens) >> 4));   // next pass, in flight
+        const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
+        uint32_t gt[4], eq[4];
+        int packed = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int bj = base + j * 4;
-            s[4 * j + 0] = (bj + 0 < end) ? group_score<G>(c[j].x, qc) : -1;
-            s[4 * j + 1] = (bj + 1 < end) ? group_score<G>(c[j].y, qc) : -1;
-            s[4 * j + 2] = (bj + 2 < end) ? group_score<G>(c[j].z, qc) : -1;
-            s[4 * j + 3] = (bj + 3 < end) ? group_score<G>(c[j].w, qc) : -1;
+            const uint32_t in_chunk = (base + 4 * j < end) ? 0xffffffffu : 0u;   // end is a multiple of 4 or the sequence end
+            const uint32_t valid = __vcmpne4(sw[j], 0xffffffffu) & 0x01010101u & in_chunk;
+            gt[j] = __vcmpgtu4(sw[j], T4) & valid;
+            eq[j] = __vcmpeq4(sw[j], T4) & 0x01010101u & in_chunk;
+            packed += (int)(__vsadu4(gt[j], 0u) | (__vsadu4(eq[j], 0u) << 16));
         }
-        int cg = 0, ce = 0;
-#pragma unroll
-        for (int e = 0; e < 16; ++e) { cg += (s[e] > T); ce += (s[e] == T); }
-        // block-wide exclusive prefix of (cg, ce), packed as two 16-bit counters (a pass has 4096 tokens)
-        const int packed = cg | (ce << 16);
+        // block-wide exclusive prefix of the packed (gt, eq) counts (a pass has 4096 tokens: 16-bit halves suffice)
         int inc = packed;
 #pragma unroll
         for (int dd = 1; dd < 32; dd <<= 1) {
@@ -259,17 +270,23 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
             if (w < warp) wpre += v;
             all += v;
         }
-        const int excl = wpre + inc - packed;
-        int gt_lt = run_gt + (excl & 0xffff);
-        int eq_lt = run_eq + (int)((unsigned)excl >> 16);
+        if (packed != 0) {
+            const int excl = wpre + inc - packed;
+            int gt_lt = run_gt + (excl & 0xffff);
+            int eq_lt = run_eq + (int)((unsigned)excl >> 16);
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-            if (s[e] > T) {
-                out[gt_lt + min(eq_lt, r)] = base + e;
-                ++gt_lt;
-            } else if (s[e] == T) {
-                if (eq_lt < r) out[gt_lt + eq_lt] = base + e;
-                ++eq_lt;
+            for (int j = 0; j < 4; ++j) {
+                if ((gt[j] | eq[j]) == 0u) continue;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if ((gt[j] >> (8 * e)) & 1u) {
+                        out[gt_lt + min(eq_lt, r)] = base + 4 * j + e;
+                        ++gt_lt;
+                    } else if ((eq[j] >> (8 * e)) & 1u) {
+                        if (eq_lt < r) out[gt_lt + eq_lt] = base + 4 * j + e;
+                        ++eq_lt;
+                    }
+                }
             }
         }
         run_gt += all & 0xffff;
@@ -280,7 +297,7 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
 
 // ------------------------------------------------------------------ fused single-kernel path
 //
-// For sequences of up to kClusterSize * 16384 tokens one thread-block cluster owns a
+// For sequences of up to 32768 tokens one thread-block cluster of 8 CTAs owns a
 // (sequence, KV head) unit: every CTA keeps its slice of the codes in registers, the CTAs exchange
 // their 33-bin histograms through distributed shared memory between two hardware cluster barriers,
 // and each CTA then compacts its own slice straight from registers.  The codes are read from HBM
@@ -288,7 +305,6 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const uint32_t *__
 // Token order inside a CTA is thread order (a lane owns 4L consecutive tokens), so the prefix sums
 // need one warp-shuffle scan plus one exchange of eight warp totals.
 
-constexpr int kClusterSize = 8;
 
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
@@ -309,20 +325,14 @@ __device__ __forceinline__ int ld_dsmem(const int *local, uint32_t rank) {
     return v;
 }
 
-template <int G>
-__device__ __forceinline__ uint32_t scores4(const uint4 &c, const uint32_t (&qc)[G]) {
-    return (uint32_t)group_score<G>(c.x, qc) | ((uint32_t)group_score<G>(c.y, qc) << 8) |
-           ((uint32_t)group_score<G>(c.z, qc) << 16) | ((uint32_t)group_score<G>(c.w, qc) << 24);
-}
-
-template <int G, int L>
-__global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 8) ? 4 : 2)) score_select_cluster_kernel(
+template <int G, int L, int CS>
+__global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 16) ? 3 : 2)) score_select_cluster_kernel(
     const uint32_t *__restrict__ q_codes, const uint32_t *__restrict__ k_codes, long long kc_sb, long long kc_sh,
     const int32_t *__restrict__ seq_lens, int max_seq_len, const int32_t *__restrict__ k_per_seq, int k_uniform,
     int k_max, int Hq, int Hkv, int32_t *__restrict__ idx, long long idx_sb, long long idx_sh,
     int32_t *__restrict__ count, int32_t *__restrict__ hist_out) {
     // per-warp histograms with one byte counter per (level, lane): a thread only ever touches its own
-    // bytes, so the counting needs no atomics and has no bank conflicts (a thread sees <= 64 tokens)
+    // bytes, so the counting needs no atomics and has no bank conflicts (a thread sees <= 128 tokens)
     __shared__ __align__(16) unsigned char w_hist[kScanThreads / 32][kBins][32];
     __shared__ int s_hist[kBins + 3];          // this CTA's histogram, read by the whole cluster
     __shared__ int s_tot[kBins], s_bef[kBins];
@@ -336,14 +346,17 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 8) ? 4 : 2
     k = max(0, min(k, k_max));
     const int keep = min(k, n);
     const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
-    // a lane owns 4L consecutive tokens (L uint4), a warp 128L, a CTA 1024L: token order = thread order
-    const int wbase = (int)rank * (L * 1024) + warp * (L * 128) + lane * (L * 4);
+    // The sequence's own length is divided over the CS CTAs (ragged batches stay balanced): a lane owns
+    // 4*Lb consecutive tokens (Lb <= L uint4), a warp 128*Lb, a CTA 1024*Lb; token order = thread order.
+    const int Lb = (n + CS * 1024 - 1) / (CS * 1024);
+    const int wbase = ((int)rank * 1024 + warp * 128 + lane * 4) * Lb;
+    constexpr int kPre = (L < 4) ? L : 4;      // uint4 loads issued before the programmatic-launch wait
 
-    uint4 c[L];
+    uint4 c[kPre];
 #pragma unroll
-    for (int p = 0; p < L; ++p) {
+    for (int p = 0; p < kPre; ++p) {
         const int base = wbase + p * 4;
-        c[p] = (base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
+        c[p] = (p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
     }
     for (int i = tid; i < (kScanThreads / 32) * kBins * 32 / 4; i += kScanThreads)
         reinterpret_cast<uint32_t *>(&w_hist[0][0][0])[i] = 0u;
@@ -351,23 +364,42 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 8) ? 4 : 2
     pdl_launch_dependents();
     pdl_wait();
 #pragma unroll
-    for (int p = 0; p < L; ++p) patch_token(c[p], wbase + p * 4, n - 1, row);
+    for (int p = 0; p < kPre; ++p) patch_token(c[p], wbase + p * 4, n - 1, row);
     uint32_t qc[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
     __syncthreads();
 
-    // ---- scores (kept as four bytes per register) and this CTA's histogram
+    // ---- scores (kept as four bytes per register; 255 marks "no token") and this CTA's histogram
     uint32_t sc[L];
     unsigned char *my = &w_hist[warp][0][lane];
 #pragma unroll
-    for (int p = 0; p < L; ++p) {
-        const int base = wbase + p * 4;
-        sc[p] = scores4<G>(c[p], qc);
+    for (int p0 = 0; p0 < L; p0 += kPre) {
+        if (p0 > 0) {   // later batches of codes are streamed through the same registers
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-            if (base + e < n) my[((sc[p] >> (8 * e)) & 0xffu) * 32] += 1;
-            else sc[p] |= 0xffu << (8 * e);   // 255 marks "no token": never equal to T, masked from ">"
+            for (int p = 0; p < kPre; ++p) {
+                const int base = wbase + (p0 + p) * 4;
+                c[p] = (p0 + p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
+                patch_token(c[p], base, n - 1, row);
+            }
+        }
+#pragma unroll
+        for (int p = 0; p < kPre; ++p) {
+            const int base = wbase + (p0 + p) * 4;
+            uint32_t s4 = scores4<G>(c[p], qc);
+            if (p0 + p < Lb && base + 3 < n) {       // whole uint4 inside the sequence: no per-token checks
+                my[(s4 & 0xffu) * 32] += 1;
+                my[((s4 >> 8) & 0xffu) * 32] += 1;
+                my[((s4 >> 16) & 0xffu) * 32] += 1;
+                my[(s4 >> 24) * 32] += 1;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (p0 + p < Lb && base + e < n) my[((s4 >> (8 * e)) & 0xffu) * 32] += 1;
+                    else s4 |= 0xffu << (8 * e);
+            }
+            sc[p0 + p] = s4;
+        }
     }
     __syncthreads();
     // fold the byte counters: one (level, warp) row of 32 bytes per thread
@@ -384,7 +416,7 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 8) ? 4 : 2
     if (tid < kBins) {
         int tot = 0, bef = 0;
 #pragma unroll
-        for (uint32_t r = 0; r < (uint32_t)kClusterSize; ++r) {
+        for (uint32_t r = 0; r < (uint32_t)CS; ++r) {
             const int v = ld_dsmem(&s_hist[tid], r);
             tot += v;
             if (r < rank) bef += v;
@@ -437,7 +469,7 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 8) ? 4 : 2
     }
     if (keep == 0) { cluster_wait(); return; }
 
-    // ---- counts of (S > T, S == T) per thread and pass, packed in 16-bit halves
+    // ---- counts of (S > T, S == T) per thread, packed in 16-bit halves
     const uint32_t T4 = (uint32_t)T * 0x01010101u;
     int tot_packed = 0;
 #pragma unroll
@@ -447,7 +479,7 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 8) ? 4 : 2
         const uint32_t eq = __vcmpeq4(sc[p], T4) & 0x01010101u;
         tot_packed += (int)(__vsadu4(gt, 0u) | (__vsadu4(eq, 0u) << 16));
     }
-    int winc = tot_packed;   // inclusive scan over the lanes of the per-lane totals (all passes)
+    int winc = tot_packed;   // inclusive scan over the lanes of the per-lane totals
 #pragma unroll
     for (int dd = 1; dd < 32; dd <<= 1) {
         const int v = __shfl_up_sync(0xffffffffu, winc, dd);
@@ -489,29 +521,40 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 8) ? 4 : 2
     cluster_wait();
 }
 
-template <int G, int L>
+template <int G, int L, int CS>
 static cudaError_t launch_cluster_t(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes,
                                     long long kc_sb, long long kc_sh, const int32_t *seq_lens,
                                     const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max, int32_t *idx,
                                     long long idx_sb, long long idx_sh, int32_t *count, int32_t *hist_out,
                                     cudaStream_t st) {
+    if (CS > 8) {   // clusters of 16 CTAs need an opt-in, once per device
+        static bool done[64] = {};
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev >= 0 && dev < 64 && !done[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(score_select_cluster_kernel<G, L, CS>,
+                                                 cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            if (e != cudaSuccess) return e;
+            done[dev] = true;
+        }
+    }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kClusterSize, Hkv, B);
+    cfg.gridDim = dim3(CS, Hkv, B);
     cfg.blockDim = dim3(kScanThreads);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kClusterSize;
+    attr[0].val.clusterDim.x = CS;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = getenv("HA_NO_PDL") ? 0 : 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, score_select_cluster_kernel<G, L>, q_codes, k_codes, kc_sb, kc_sh, seq_lens,
-                                       max_seq_len, k_per_seq, k_uniform, k_max, Hq, Hkv, idx, idx_sb, idx_sh, count,
-                                       hist_out);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, score_select_cluster_kernel<G, L, CS>, q_codes, k_codes, kc_sb, kc_sh,
+                                       seq_lens, max_seq_len, k_per_seq, k_uniform, k_max, Hq, Hkv, idx, idx_sb, idx_sh,
+                                       count, hist_out);
     if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
@@ -522,29 +565,28 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
                             long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
                             int k_uniform, int max_seq_len, int k_max, int32_t *idx, long long idx_sb,
                             long long idx_sh, int32_t *count, int32_t *hist_out, int32_t *ws_hist,
-                            cudaStream_t st) {
-    if (max_seq_len <= kClusterSize * 16 * 1024 && !getenv("HA_NO_CLUSTER")) {
-        // fused path: one cluster per unit, L uint4 of codes per thread
-        const int per_cta = (max_seq_len + kClusterSize - 1) / kClusterSize;
-#define HA_CL(LL)                                                                                                   \
-    return launch_cluster_t<G, LL>(B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform,     \
-                                   max_seq_len, k_max, idx, idx_sb, idx_sh, count, hist_out, st)
-        if (per_cta <= 1024) HA_CL(1);
-        if (per_cta <= 2048) HA_CL(2);
-        if (per_cta <= 4096) HA_CL(4);
-        if (per_cta <= 8192) HA_CL(8);
-        HA_CL(16);
+                            unsigned char *ws_scores, cudaStream_t st) {
+    if (max_seq_len <= kClusterMaxSeq && !getenv("HA_NO_CLUSTER")) {
+        // fused path: one 8-CTA cluster per unit, up to 4 uint4 of signatures per thread
+#define HA_CL(LL, CSZ)                                                                                              \
+    return launch_cluster_t<G, LL, CSZ>(B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform, \
+                                        max_seq_len, k_max, idx, idx_sb, idx_sh, count, hist_out, st)
+        const int per8 = (max_seq_len + 8 * 1024 - 1) / (8 * 1024);     // uint4 per thread with 8 CTAs
+        if (per8 <= 1) HA_CL(1, 8);
+        if (per8 <= 2) HA_CL(2, 8);
+        HA_CL(4, 8);
 #undef HA_CL
     }
     const int chunk_tokens = chunk_tokens_for(B * Hkv, max_seq_len);
     const int n_chunks = max(1, (max_seq_len + chunk_tokens - 1) / chunk_tokens);
+    const long long score_row = (long long)score_row_bytes(max_seq_len);
     dim3 grid(n_chunks, Hkv, B);
-    cudaError_t e = launch_pdl(scan_hist_kernel<G>, grid, dim3(kScanThreads), 0, st, q_codes, k_codes, kc_sb, kc_sh,
-                               seq_lens, max_seq_len, Hq, Hkv, chunk_tokens, ws_hist);
+    cudaError_t e = launch_pdl(scan_score_kernel<G>, grid, dim3(kScanThreads), 0, st, q_codes, k_codes, kc_sb, kc_sh,
+                               seq_lens, max_seq_len, Hq, Hkv, chunk_tokens, score_row, ws_scores, ws_hist);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(select_kernel<G>, grid, dim3(kScanThreads), 0, st, q_codes, k_codes, kc_sb, kc_sh, seq_lens,
-                   max_seq_len, k_per_seq, k_uniform, k_max, Hq, Hkv, chunk_tokens, (const int32_t *)ws_hist, idx,
-                   idx_sb, idx_sh, count, hist_out);
+    e = launch_pdl(select_kernel, grid, dim3(kScanThreads), 0, st, seq_lens, max_seq_len, k_per_seq, k_uniform, k_max,
+                   Hkv, chunk_tokens, score_row, (const unsigned char *)ws_scores, (const int32_t *)ws_hist, idx, idx_sb,
+                   idx_sh, count, hist_out);
     if (e != cudaSuccess) return e;
     count_launch(2);
     return cudaGetLastError();
@@ -554,9 +596,9 @@ cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, c
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens,
                               const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max,
                               int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
-                              int32_t *hist_out, int32_t *ws_hist, cudaStream_t st) {
+                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st) {
 #define HA_ARGS B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx, \
-                idx_sb, idx_sh, count, hist_out, ws_hist, st
+                idx_sb, idx_sh, count, hist_out, ws_hist, ws_scores, st
     switch (Hq / Hkv) {
         case 1: return launch_g<1>(HA_ARGS);
         case 2: return launch_g<2>(HA_ARGS);
