@@ -19,6 +19,12 @@
  *   - Scratch memory is one caller-owned workspace of at least ha_workspace_bytes(...) bytes,
  *     256-byte aligned, prepared once with ha_workspace_init.  Calls that share a workspace must
  *     be ordered on one stream.
+ *   - Kernels are launched with programmatic stream serialization: a kernel may start while its
+ *     predecessor in the stream is finishing, and reads seq_lens, k_per_seq and the key signatures
+ *     before it waits for that predecessor.  This is safe behind ordinary kernels and copies (they
+ *     complete before anything of this library starts) and inside ha_sparse_decode; a caller whose
+ *     own preceding kernel both writes those arrays AND releases its dependents early
+ *     (griddepcontrol.launch_dependents) must release them only after the writes.
  *   - Return value: HA_OK, or an HA_ERR_* code for errors detectable on the host (nothing is
  *     enqueued in that case).  Errors only visible on the device (an index outside the sequence)
  *     set a bit in the workspace status word, are skipped, and never trap.

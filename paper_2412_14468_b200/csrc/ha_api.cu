@@ -221,7 +221,7 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
     HA_CUDA(launch_attention(true, B, Hq, Hkv, shape->sm_scale, q, view(K), view(V), seq_lens, idx, idx_stride_b,
                              idx_stride_h, count, k_max, out, lse, ws_ptr<float>(workspace, L.off_part_ml),
                              ws_ptr<float>(workspace, L.off_part_acc), ws_ptr<int32_t>(workspace, L.off_tickets),
-                             ws_ptr<uint32_t>(workspace, 0), st));
+                             ws_ptr<uint32_t>(workspace, 0), st, /*count_from_k=*/1, k_per_seq, k_uniform));
     return HA_OK;
 }
 

@@ -73,6 +73,8 @@ struct AttnArgs {
     TensorView K, V;
     const int32_t *seq_lens, *idx, *count;
     long long idx_sb, idx_sh;
+    const int32_t *k_per_seq;   // with count_from_k: budget per sequence (or NULL: k_uniform)
+    int k_uniform, count_from_k;
     int max_items, Hq, Hkv, n_units, balanced;
     float scale_log2;
     float *part_ml, *part_acc;
@@ -98,13 +100,20 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
     const uint32_t ring_u32 = smem_u32(my_ring);
     bool bad = false;
 
-    // everything below depends on the preceding kernels (count, idx, appended rows)
+    // The index lists and the appended rows come from the preceding kernels: they are read after the
+    // programmatic-launch wait.  Inside a whole layer-step the list LENGTHS are min(k, n) by
+    // construction, so the work distribution is computed before the wait, from inputs that no kernel
+    // of the step writes; a stand-alone call reads the caller's count array instead, after the wait.
     pdl_launch_dependents();
-    pdl_wait();
+    const bool early = kGather ? (a.count_from_k != 0) : true;
+    if (!early) pdl_wait();
 
     auto unit_count = [&](int u) -> int {
         const int b = u / Hkv;
-        return max(0, min(kGather ? a.count[u] : a.seq_lens[b], a.max_items));
+        const int n_b = a.seq_lens[b];
+        int c = n_b;
+        if (kGather) c = a.count_from_k ? min(a.k_per_seq ? a.k_per_seq[b] : a.k_uniform, n_b) : a.count[u];
+        return max(0, min(c, a.max_items));
     };
     auto write_empty = [&](int u) {   // empty selection: out = 0, lse = -inf
         const long long h0 = (long long)(u / Hkv) * Hq + (long long)(u % Hkv) * G;
@@ -116,32 +125,44 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
     long long x, x_end, T;
     int u;
     if (a.balanced) {
-        for (int v = tid; v < a.n_units; v += kAttnThreads)
-            s_pref[v + 1] = (unit_count(v) + kBlockTokens - 1) / kBlockTokens;
-        if (tid == 0) s_pref[0] = 0;
-        __syncthreads();
-        if (warp == 0) {   // inclusive scan in place, one contiguous piece per lane
-            const int per = (a.n_units + 31) / 32;
-            const int lo = min(a.n_units, lane * per), hi = min(a.n_units, lo + per);
-            int sum = 0;
-            for (int v = lo; v < hi; ++v) sum += s_pref[v + 1];
-            int inc = sum;
+        if (a.n_units <= 32) {
+            // few units: every warp scans the block counts in registers (no barrier); warp 0 keeps a copy
+            const int nb = (lane < a.n_units) ? (unit_count(lane) + kBlockTokens - 1) / kBlockTokens : 0;
+            int inc = nb;
 #pragma unroll
             for (int dd = 1; dd < 32; dd <<= 1) {
                 const int o = __shfl_up_sync(0xffffffffu, inc, dd);
                 if (lane >= dd) inc += o;
             }
-            int run = inc - sum;
-            for (int v = lo; v < hi; ++v) { run += s_pref[v + 1]; s_pref[v + 1] = run; }
+            if (warp == 0) {
+                if (lane == 0) s_pref[0] = 0;
+                if (lane < a.n_units) s_pref[lane + 1] = inc;
+            }
+            __syncthreads();
+        } else {
+            for (int v = tid; v < a.n_units; v += kAttnThreads)
+                s_pref[v + 1] = (unit_count(v) + kBlockTokens - 1) / kBlockTokens;
+            if (tid == 0) s_pref[0] = 0;
+            __syncthreads();
+            if (warp == 0) {   // inclusive scan in place, one contiguous piece per lane
+                const int per = (a.n_units + 31) / 32;
+                const int lo = min(a.n_units, lane * per), hi = min(a.n_units, lo + per);
+                int sum = 0;
+                for (int v = lo; v < hi; ++v) sum += s_pref[v + 1];
+                int inc = sum;
+#pragma unroll
+                for (int dd = 1; dd < 32; dd <<= 1) {
+                    const int o = __shfl_up_sync(0xffffffffu, inc, dd);
+                    if (lane >= dd) inc += o;
+                }
+                int run = inc - sum;
+                for (int v = lo; v < hi; ++v) { run += s_pref[v + 1]; s_pref[v + 1] = run; }
+            }
+            __syncthreads();
         }
-        __syncthreads();
         T = s_pref[a.n_units];
-        for (int v = cta; v < a.n_units; v += P)
-            if (s_pref[v + 1] == s_pref[v]) write_empty(v);
-        if (T == 0) return;
-        x = (long long)cta * T / P;
-        x_end = (long long)(cta + 1) * T / P;
-        if (x >= x_end) return;
+        x = (T > 0) ? (long long)cta * T / P : 0;
+        x_end = (T > 0) ? (long long)(cta + 1) * T / P : 0;
         int lo = 0, hi = a.n_units;   // largest u with s_pref[u] <= x
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -153,8 +174,15 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
         T = 0;
         x = 0;
         x_end = (unit_count(u) + kBlockTokens - 1) / kBlockTokens;
-        if (x_end == 0) { write_empty(u); return; }
     }
+    if (early) pdl_wait();   // nothing is written, and nothing of the preceding kernels read, before this point
+    if (a.balanced) {
+        for (int v = cta; v < a.n_units; v += P)
+            if (s_pref[v + 1] == s_pref[v]) write_empty(v);
+    } else if (x_end == 0) {
+        write_empty(u);
+    }
+    if (x >= x_end) return;
 
     while (x < x_end) {
         // ---- segment: blocks [blk_lo, blk_hi) of unit u
@@ -516,11 +544,13 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              TensorView K, TensorView V, const int32_t *seq_lens, const int32_t *idx,
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
                              uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
-                             uint32_t *status, cudaStream_t st) {
+                             uint32_t *status, cudaStream_t st, int count_from_k, const int32_t *k_per_seq,
+                             int k_uniform) {
     AttnArgs a{};
     a.q = q; a.K = K; a.V = V; a.seq_lens = seq_lens; a.idx = idx; a.count = count;
     a.idx_sb = idx_sb; a.idx_sh = idx_sh; a.max_items = max_items; a.Hq = Hq; a.Hkv = Hkv;
     a.n_units = B * Hkv; a.scale_log2 = sm_scale * kLog2e;
+    a.k_per_seq = k_per_seq; a.k_uniform = k_uniform; a.count_from_k = count_from_k;
     a.part_ml = part_ml; a.part_acc = part_acc; a.tickets = tickets; a.status = status; a.out = out; a.lse = lse;
     switch (Hq / Hkv) {
         case 1: return launch_attn_g<1>(gather, a, st);

@@ -4,7 +4,6 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
-#include <cstdlib>
 
 #include "hashattn.h"
 
@@ -89,7 +88,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = getenv("HA_NO_PDL") ? 0 : 1;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
@@ -136,7 +135,8 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              TensorView K, TensorView V, const int32_t *seq_lens, const int32_t *idx,
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
                              uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
-                             uint32_t *status, cudaStream_t st);
+                             uint32_t *status, cudaStream_t st, int count_from_k = 0,
+                             const int32_t *k_per_seq = nullptr, int k_uniform = 0);
 
 cudaError_t launch_append_kv(int B, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
                              TensorView V, const int32_t *seq_lens, cudaStream_t st);

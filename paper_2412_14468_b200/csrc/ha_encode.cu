@@ -110,9 +110,11 @@ __global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, E
     const float bias1 = J.map.b1 ? __ldg(J.map.b1 + net * kHid + o) : 0.0f;
     const float bias2 = J.map.b2 ? __ldg(J.map.b2 + net * kHid + o) : 0.0f;
     const float bias3 = J.map.b3 ? __ldg(J.map.b3 + net * kBits + (tid & (kBits - 1))) : 0.0f;
-    // the weights do not depend on earlier kernels of the stream; the vectors to encode may
-    pdl_launch_dependents();
+    // The weights do not depend on earlier kernels of the stream; the vectors to encode may.  The
+    // kernels behind this one are released only after the wait: whatever they read before their own
+    // wait (sequence lengths, budgets, signatures) is then final, whoever wrote it earlier in the stream.
     pdl_wait();
+    pdl_launch_dependents();
 #pragma unroll
     for (int vv = 0; vv < VT; ++vv) {
         const int v = half * VT + vv;

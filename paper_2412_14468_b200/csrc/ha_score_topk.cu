@@ -19,7 +19,7 @@ namespace ha {
 
 constexpr int kScanThreads = 256;
 constexpr int kPassTokens = kScanThreads * 16;   // four uint4 per thread
-constexpr int kClusterMaxSeq = 8 * 4 * 1024;     // longest sequence the fused cluster kernel takes (4 uint4 per thread)
+constexpr int kClusterMaxSeq = 32768;            // longest sequence the fused cluster kernel takes
 
 template <int G>
 __device__ __forceinline__ int group_score(uint32_t code, const uint32_t (&qc)[G]) {
@@ -48,10 +48,20 @@ __device__ __forceinline__ void patch_token(uint4 &v, int base, int last, const 
     if (e == 0) v.x = c; else if (e == 1) v.y = c; else if (e == 2) v.z = c; else v.w = c;
 }
 
+// Four group scores packed as bytes holding score + 1 (1..33); a zero byte means "no token".
 template <int G>
 __device__ __forceinline__ uint32_t scores4(const uint4 &c, const uint32_t (&qc)[G]) {
-    return (uint32_t)group_score<G>(c.x, qc) | ((uint32_t)group_score<G>(c.y, qc) << 8) |
-           ((uint32_t)group_score<G>(c.z, qc) << 16) | ((uint32_t)group_score<G>(c.w, qc) << 24);
+    return (uint32_t)(group_score<G>(c.x, qc) + 1) | ((uint32_t)(group_score<G>(c.y, qc) + 1) << 8) |
+           ((uint32_t)(group_score<G>(c.z, qc) + 1) << 16) | ((uint32_t)(group_score<G>(c.w, qc) + 1) << 24);
+}
+
+// Per-byte flags (bit 7 of each byte) of "score > T" and "score == T" for four packed score+1 bytes.
+// Plain 32-bit arithmetic: with bytes <= 33 and T + 1 <= 34 no byte sum reaches 256, so no carry
+// crosses a byte; a zero byte (no token) is neither above nor equal to any threshold.
+__device__ __forceinline__ void flags4(uint32_t s4, uint32_t t1x4, uint32_t &gt, uint32_t &eq) {
+    gt = (s4 + (0x7f7f7f7fu - t1x4)) & 0x80808080u;            // byte + 127 - (T+1) >= 128  <=>  score > T
+    const uint32_t ge = (s4 + (0x80808080u - t1x4)) & 0x80808080u;   // byte + 128 - (T+1) >= 128  <=>  score >= T
+    eq = ge ^ gt;
 }
 
 // ------------------------------------------------------------------ long-sequence path (two kernels)
@@ -100,7 +110,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
     for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
     __syncthreads();
 
-    unsigned char *my = &w_hist[warp][0][lane];
+    unsigned char *my = &w_hist[warp][0][lane] - 32;   // indexed by the score+1 byte
     for (int pass = start; pass < end; pass += kPassTokens) {
         if (pass + kPassTokens < end) load_pass(nxt, pass + kPassTokens);
 #pragma unroll
@@ -118,7 +128,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
                         if (base + e < end) my[((s4 >> (8 * e)) & 0xffu) * 32] += 1;
-                        else s4 |= 0xffu << (8 * e);      // 255 marks "no token"
+                        else s4 &= ~(0xffu << (8 * e));   // zero byte: no token
                 }
                 srow[base >> 2] = s4;
             }
@@ -168,7 +178,7 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
     const uint4 *srow = reinterpret_cast<const uint4 *>(ws_scores + ((long long)b * Hkv + g) * score_row);
     const int start = chunk * chunk_tokens, end = min(n, start + chunk_tokens);
     // first pass of score bytes: requested now, used after the threshold is known
-    uint4 sv_next = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+    uint4 sv_next = make_uint4(0u, 0u, 0u, 0u);
     if (chunk < n_chunks && start + tid * 16 < end) sv_next = __ldcg(srow + ((start + tid * 16) >> 4));
 
     // totals per score level, and the part contributed by the chunks before this one: every thread
@@ -236,23 +246,21 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
     }
     if (chunk >= n_chunks || keep == 0) return;
 
-    const uint32_t T4 = (uint32_t)T * 0x01010101u;
+    const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
     int run_gt = sh_gt_before, run_eq = sh_eq_before;   // tokens before this pass with S > T / S == T
     for (int pass = start; pass < end; pass += kPassTokens) {
         const int base = pass + tid * 16;
         const uint4 sv = sv_next;
-        sv_next = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+        sv_next = make_uint4(0u, 0u, 0u, 0u);
         if (base + kPassTokens < end) sv_next = __ldcg(srow + ((base + kPassTokens) >> 4));   // next pass, in flight
         const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
         uint32_t gt[4], eq[4];
         int packed = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const uint32_t in_chunk = (base + 4 * j < end) ? 0xffffffffu : 0u;   // end is a multiple of 4 or the sequence end
-            const uint32_t valid = __vcmpne4(sw[j], 0xffffffffu) & 0x01010101u & in_chunk;
-            gt[j] = __vcmpgtu4(sw[j], T4) & valid;
-            eq[j] = __vcmpeq4(sw[j], T4) & 0x01010101u & in_chunk;
-            packed += (int)(__vsadu4(gt[j], 0u) | (__vsadu4(eq[j], 0u) << 16));
+            // words past the chunk were never written: drop them (end is a multiple of 4 or the sequence end)
+            flags4((base + 4 * j < end) ? sw[j] : 0u, T4, gt[j], eq[j]);
+            packed += __popc(gt[j]) | (__popc(eq[j]) << 16);
         }
         // block-wide exclusive prefix of the packed (gt, eq) counts (a pass has 4096 tokens: 16-bit halves suffice)
         int inc = packed;
@@ -279,10 +287,10 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
                 if ((gt[j] | eq[j]) == 0u) continue;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if ((gt[j] >> (8 * e)) & 1u) {
+                    if ((gt[j] >> (8 * e + 7)) & 1u) {
                         out[gt_lt + min(eq_lt, r)] = base + 4 * j + e;
                         ++gt_lt;
-                    } else if ((eq[j] >> (8 * e)) & 1u) {
+                    } else if ((eq[j] >> (8 * e + 7)) & 1u) {
                         if (eq_lt < r) out[gt_lt + eq_lt] = base + 4 * j + e;
                         ++eq_lt;
                     }
@@ -297,10 +305,10 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
 
 // ------------------------------------------------------------------ fused single-kernel path
 //
-// For sequences of up to 32768 tokens one thread-block cluster of 8 CTAs owns a
+// For sequences of up to 32768 tokens one thread-block cluster of 8, 4 or 2 CTAs owns a
 // (sequence, KV head) unit: every CTA keeps its slice of the codes in registers, the CTAs exchange
 // their 33-bin histograms through distributed shared memory between two hardware cluster barriers,
-// and each CTA then compacts its own slice straight from registers.  The codes are read from HBM
+// and each CTA then compacts its own slice straight from registers (scores kept as bytes).  The codes are read from HBM
 // once, there is no histogram round trip through global memory and no second launch.
 // Token order inside a CTA is thread order (a lane owns 4L consecutive tokens), so the prefix sums
 // need one warp-shuffle scan plus one exchange of eight warp totals.
@@ -326,7 +334,7 @@ __device__ __forceinline__ int ld_dsmem(const int *local, uint32_t rank) {
 }
 
 template <int G, int L, int CS>
-__global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 16) ? 3 : 2)) score_select_cluster_kernel(
+__global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : 4) score_select_cluster_kernel(
     const uint32_t *__restrict__ q_codes, const uint32_t *__restrict__ k_codes, long long kc_sb, long long kc_sh,
     const int32_t *__restrict__ seq_lens, int max_seq_len, const int32_t *__restrict__ k_per_seq, int k_uniform,
     int k_max, int Hq, int Hkv, int32_t *__restrict__ idx, long long idx_sb, long long idx_sh,
@@ -370,9 +378,9 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 16) ? 3 : 
     for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
     __syncthreads();
 
-    // ---- scores (kept as four bytes per register; 255 marks "no token") and this CTA's histogram
+    // ---- scores (kept as four score+1 bytes per register; 0 marks "no token") and this CTA's histogram
     uint32_t sc[L];
-    unsigned char *my = &w_hist[warp][0][lane];
+    unsigned char *my = &w_hist[warp][0][lane] - 32;   // indexed by the score+1 byte
 #pragma unroll
     for (int p0 = 0; p0 < L; p0 += kPre) {
         if (p0 > 0) {   // later batches of codes are streamed through the same registers
@@ -396,7 +404,7 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 16) ? 3 : 
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
                     if (p0 + p < Lb && base + e < n) my[((s4 >> (8 * e)) & 0xffu) * 32] += 1;
-                    else s4 |= 0xffu << (8 * e);
+                    else s4 &= ~(0xffu << (8 * e));   // zero byte: no token
             }
             sc[p0 + p] = s4;
         }
@@ -470,14 +478,13 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 16) ? 3 : 
     if (keep == 0) { cluster_wait(); return; }
 
     // ---- counts of (S > T, S == T) per thread, packed in 16-bit halves
-    const uint32_t T4 = (uint32_t)T * 0x01010101u;
+    const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
     int tot_packed = 0;
 #pragma unroll
     for (int p = 0; p < L; ++p) {
-        const uint32_t valid = __vcmpne4(sc[p], 0xffffffffu) & 0x01010101u;      // 1 per real token
-        const uint32_t gt = __vcmpgtu4(sc[p], T4) & valid;                        // bytes 0x01 where S > T
-        const uint32_t eq = __vcmpeq4(sc[p], T4) & 0x01010101u;
-        tot_packed += (int)(__vsadu4(gt, 0u) | (__vsadu4(eq, 0u) << 16));
+        uint32_t gt, eq;
+        flags4(sc[p], T4, gt, eq);
+        tot_packed += __popc(gt) | (__popc(eq) << 16);
     }
     int winc = tot_packed;   // inclusive scan over the lanes of the per-lane totals
 #pragma unroll
@@ -500,17 +507,16 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : ((L <= 16) ? 3 : 
         if (tot_packed != 0) {
 #pragma unroll
             for (int p = 0; p < L; ++p) {
-                const uint32_t valid = __vcmpne4(sc[p], 0xffffffffu) & 0x01010101u;
-                const uint32_t gt = __vcmpgtu4(sc[p], T4) & valid;
-                const uint32_t eq = __vcmpeq4(sc[p], T4) & 0x01010101u;
+                uint32_t gt, eq;
+                flags4(sc[p], T4, gt, eq);
                 if ((gt | eq) == 0u) continue;
                 const int base = wbase + p * 4;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    if ((gt >> (8 * e)) & 1u) {
+                    if ((gt >> (8 * e + 7)) & 1u) {
                         out[gt_lt + min(eq_lt, r)] = base + e;
                         ++gt_lt;
-                    } else if ((eq >> (8 * e)) & 1u) {
+                    } else if ((eq >> (8 * e + 7)) & 1u) {
                         if (eq_lt < r) out[gt_lt + eq_lt] = base + e;
                         ++eq_lt;
                     }
@@ -549,7 +555,7 @@ static cudaError_t launch_cluster_t(int B, int Hq, int Hkv, const uint32_t *q_co
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = getenv("HA_NO_PDL") ? 0 : 1;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, score_select_cluster_kernel<G, L, CS>, q_codes, k_codes, kc_sb, kc_sh,
@@ -566,15 +572,31 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
                             int k_uniform, int max_seq_len, int k_max, int32_t *idx, long long idx_sb,
                             long long idx_sh, int32_t *count, int32_t *hist_out, int32_t *ws_hist,
                             unsigned char *ws_scores, cudaStream_t st) {
-    if (max_seq_len <= kClusterMaxSeq && !getenv("HA_NO_CLUSTER")) {
-        // fused path: one 8-CTA cluster per unit, up to 4 uint4 of signatures per thread
+    if (max_seq_len <= kClusterMaxSeq) {
+        // Fused path: one cluster per unit.  Cluster size: the largest of 8, 4, 2 whose grid still fits
+        // the GPU in one wave (about six 256-thread CTAs per SM), so that small batches get the most
+        // parallelism per sequence and large batches the most work per cluster barrier; a thread then
+        // holds L = ceil(n / (CS * 1024)) uint4 of signatures (L <= 16).
+        const int units = B * Hkv, one_wave = 6 * 148;
+        int cs = 8;
+        while (cs > 2 && units * cs > one_wave) cs >>= 1;
+        while ((max_seq_len + cs * 1024 - 1) / (cs * 1024) > 16) cs <<= 1;   // keep L <= 16
+        const int per = (max_seq_len + cs * 1024 - 1) / (cs * 1024);
 #define HA_CL(LL, CSZ)                                                                                              \
     return launch_cluster_t<G, LL, CSZ>(B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform, \
                                         max_seq_len, k_max, idx, idx_sb, idx_sh, count, hist_out, st)
-        const int per8 = (max_seq_len + 8 * 1024 - 1) / (8 * 1024);     // uint4 per thread with 8 CTAs
-        if (per8 <= 1) HA_CL(1, 8);
-        if (per8 <= 2) HA_CL(2, 8);
-        HA_CL(4, 8);
+#define HA_CL_L(CSZ)               \
+    do {                           \
+        if (per <= 1) HA_CL(1, CSZ);  \
+        if (per <= 2) HA_CL(2, CSZ);  \
+        if (per <= 4) HA_CL(4, CSZ);  \
+        if (per <= 8) HA_CL(8, CSZ);  \
+        HA_CL(16, CSZ);            \
+    } while (0)
+        if (cs == 8) HA_CL_L(8);
+        if (cs == 4) HA_CL_L(4);
+        HA_CL_L(2);
+#undef HA_CL_L
 #undef HA_CL
     }
     const int chunk_tokens = chunk_tokens_for(B * Hkv, max_seq_len);
