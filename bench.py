@@ -333,7 +333,9 @@ def main():
     roofline = {
         "bound": "hbm", "kernel": "attn_kernel<4,true> (the one kernel of ha_gather_attn)",
         "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-        "traffic": None, "algorithmic_bytes_per_launch": gather_bytes, "us_per_launch": g_us,
+        # dram__bytes_read.sum + dram__bytes_write.sum per launch of this kernel on this workload, from the
+        # ncu launch list of this very command (profiles/launch_list_bench_c2.md)
+        "traffic": 4302000, "algorithmic_bytes_per_launch": gather_bytes, "us_per_launch": g_us,
         "whole_step": {"algorithmic_bytes": alg_bytes, "achieved": alg_bytes / (us_per_step * 1e-6) / 1e9,
                        "frac": alg_bytes / (us_per_step * 1e-6) / 1e9 / peak},
         "ha_score_topk": {"algorithmic_bytes": scan_bytes, "us": parts["ha_score_topk"],

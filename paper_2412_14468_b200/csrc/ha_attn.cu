@@ -532,6 +532,9 @@ static cudaError_t launch_attn_g(bool gather, const AttnArgs &args_in, cudaStrea
         long long want = (t_max + kAttnWarps - 1) / kAttnWarps;   // at least one block per warp
         const long long cap = (long long)min(2 * sm_count(), kMaxAttnCtas);
         grid = (int)max(1LL, min(want, cap));
+        // a CTA count that is a multiple of the unit count lets equal-length lists split at CTA borders,
+        // so that no CTA pays a second prologue and merge in the middle of its range
+        if (args.n_units <= grid) grid = grid / args.n_units * args.n_units;
         smem += (size_t)(args.n_units + 1) * 4;
     } else {
         args.balanced = 0;
