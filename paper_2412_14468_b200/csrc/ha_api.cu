@@ -200,6 +200,14 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
     cudaStream_t st = (cudaStream_t)stream;
     const int B = shape->batch, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
 
+    if (fused_step_eligible(B, Hkv, max_seq_len)) {
+        // small batch: the whole step is one cluster kernel
+        HA_CUDA(launch_fused_step(B, Hq, Hkv, shape->sm_scale, view(map_q), k_new ? view(map_k) : MapView{}, q, k_new,
+                                  view(K), view(V), k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
+                                  max_seq_len, k_max, q_codes, idx, idx_stride_b, idx_stride_h, count, out, lse, st));
+        return HA_OK;
+    }
+
     EncodeJob jq{};
     jq.x = q; jq.x_sb = (long long)Hq * kD; jq.x_sh = kD;
     jq.codes = q_codes; jq.c_sb = Hq; jq.c_sh = 1;

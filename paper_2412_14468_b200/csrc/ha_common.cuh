@@ -138,6 +138,15 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              uint32_t *status, cudaStream_t st, int count_from_k = 0,
                              const int32_t *k_per_seq = nullptr, int k_uniform = 0);
 
+// The whole layer-step in one launch (one 8-CTA cluster per unit); only for small batches.
+bool fused_step_eligible(int B, int Hkv, int max_seq_len);
+cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapView &map_q, const MapView &map_k,
+                              const uint16_t *q, const uint16_t *k_new, TensorView K, TensorView V, uint32_t *k_codes,
+                              long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
+                              int k_uniform, int max_seq_len, int k_max, uint32_t *q_codes, int32_t *idx,
+                              long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
+                              cudaStream_t st);
+
 cudaError_t launch_append_kv(int B, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
                              TensorView V, const int32_t *seq_lens, cudaStream_t st);
 

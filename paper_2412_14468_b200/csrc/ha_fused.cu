@@ -1,0 +1,475 @@
+// The whole layer-step in ONE launch, for small batches (at most 18 (sequence, KV head) units and
+// sequences of up to 32768 tokens): ENCODE -> SCORE -> TOPK -> GATHER-ATT (Section 4 recipe,
+// Section 4.1 "Implementation") with one thread-block cluster of 8 CTAs per unit, so that a batch-1
+// decode step keeps 64 SMs busy without a single kernel boundary or global-memory hand-off on its
+// critical path:
+//
+//   P0  every CTA requests its slice of the signature cache; CTA 0 and CTA 1 of the cluster request
+//       the query-side / key-side mapping weights with bulk asynchronous copies (TMA, mbarriers);
+//       all of it before the programmatic-launch wait, i.e. behind the preceding kernel.
+//   P1  CTA 0 encodes the G query vectors, CTA 1 the appended key (fp32 fma chains, Eq. 2);
+//       cluster barrier; everybody reads the five signatures through distributed shared memory.
+//   P2  scores as bytes in registers, per-CTA histogram, cluster barrier, histogram exchange through
+//       distributed shared memory, threshold, compaction of the CTA's slice into the index list;
+//       cluster barrier (the list is now visible to the whole cluster).
+//   P3  each CTA takes an eighth of the list: rows fetched with 16-byte cp.async into per-warp
+//       shared-memory stages, QK^T and PV on the tensor cores, online softmax; the eight CTA states
+//       are written into CTA 0's shared memory (DSMEM stores), cluster barrier, CTA 0 merges,
+//       normalises and rounds once to bf16.
+// Every cross-CTA hand-off is a hardware cluster barrier (no flag, no spin).  Results are bit-identical
+// to the multi-kernel path for signatures, counts and index lists; attention outputs agree within
+// the usual fp32 reordering.
+#include "ha_attn_dev.cuh"
+#include "ha_encode_dev.cuh"
+#include "ha_score_dev.cuh"
+
+namespace ha {
+
+constexpr int kFusedCS = 8;
+constexpr int kFusedWarps = 8;
+constexpr int kFusedThreads = kFusedWarps * 32;
+constexpr int kFusedL = 4;                                   // uint4 of signatures per thread (n <= 32768)
+constexpr int kFusedStages = 2;                              // row blocks in flight per warp
+constexpr int kFusedRingBytes = kFusedWarps * kFusedStages * kStageBytes;
+constexpr int kFusedWeightBytes = (kD * kHid + kHid * kHid + kHid * kBits) * 2;
+constexpr int kFusedUnionBytes = (kFusedRingBytes > kFusedWeightBytes) ? kFusedRingBytes : kFusedWeightBytes;
+constexpr int kFusedActBytes = 2 * kMaxGroup * kD * 4;       // two activation buffers of up to 8 vectors
+constexpr int kFusedPartBytes = kFusedCS * kMaxGroup * (kD + 2) * 4;   // the eight CTA states, in CTA 0
+constexpr int kFusedSmemBytes = kFusedUnionBytes + kFusedActBytes + kFusedPartBytes;
+
+struct FusedArgs {
+    MapView map_q, map_k;
+    const uint16_t *q, *k_new;
+    TensorView K, V;
+    uint32_t *k_codes;
+    long long kc_sb, kc_sh;
+    const int32_t *seq_lens, *k_per_seq;
+    int k_uniform, max_seq_len, k_max, Hq, Hkv;
+    float scale_log2;
+    uint32_t *q_codes;
+    int32_t *idx;
+    long long idx_sb, idx_sh;
+    int32_t *count;
+    uint16_t *out;
+    float *lse;
+};
+
+__device__ __forceinline__ void st_dsmem_f32(float *local, uint32_t rank, float v) {
+    uint32_t a = (uint32_t)__cvta_generic_to_shared(local), ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
+}
+
+// ENCODE of NV vectors that share one network, by the whole CTA (256 threads: thread (o, half) runs
+// the chains of output o for half of the vectors).  Weights arrive in shared memory through three
+// mbarriers armed by the caller.  Signature v is returned in codes_out[v] (shared memory).
+template <int NV>
+__device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_stride, const MapView &map, int net,
+                                             uint16_t *sw1, uint16_t *sw2, uint16_t *sw3, uint32_t bar0, float *actA,
+                                             float *actB, uint32_t *codes_out) {
+    constexpr int VT = (NV + 1) / 2, NS = 2 * VT;
+    const int tid = threadIdx.x, o = tid & 127, half = tid >> 7;
+    const float bias1 = map.b1 ? __ldg(map.b1 + net * kHid + o) : 0.0f;
+    const float bias2 = map.b2 ? __ldg(map.b2 + net * kHid + o) : 0.0f;
+    const float bias3 = map.b3 ? __ldg(map.b3 + net * kBits + (tid & (kBits - 1))) : 0.0f;
+#pragma unroll
+    for (int vv = 0; vv < VT; ++vv) {
+        const int v = half * VT + vv;
+        actA[v * kD + o] = (v < NV) ? bf16_bits_to_float(__ldg(x0 + (long long)v * x_stride + o)) : 0.0f;
+    }
+    __syncthreads();
+    auto weights_ready = [&](int which, uint16_t *dst, const uint16_t *src, int n_elems) {
+        const bool ok = mbar_wait_bounded(bar0 + 8 * which);
+        if (__syncthreads_or(!ok)) {   // never seen: fetch the matrix with ordinary loads instead
+            for (int c = tid; c < n_elems / 8; c += kFusedThreads)
+                reinterpret_cast<uint4 *>(dst)[c] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
+            __syncthreads();
+        }
+    };
+    float z[VT];
+    weights_ready(0, sw1, map.w1 + (size_t)net * kD * kHid, kD * kHid);
+#pragma unroll
+    for (int v = 0; v < VT; ++v) z[v] = bias1;
+    vec_layer<VT>(actA + half * VT * kD, sw1, kHid, o, z);
+#pragma unroll
+    for (int v = 0; v < VT; ++v) actB[(half * VT + v) * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+    __syncthreads();
+    weights_ready(1, sw2, map.w2 + (size_t)net * kHid * kHid, kHid * kHid);
+#pragma unroll
+    for (int v = 0; v < VT; ++v) z[v] = bias2;
+    vec_layer<VT>(actB + half * VT * kD, sw2, kHid, o, z);
+#pragma unroll
+    for (int v = 0; v < VT; ++v) actA[(half * VT + v) * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+    __syncthreads();
+    weights_ready(2, sw3, map.w3 + (size_t)net * kHid * kBits, kHid * kBits);
+    {
+        const int v = tid >> 5, lane = tid & 31;   // warp v encodes vector v, one output bit per lane
+        if (v < NS) {
+            float z3[1] = {bias3};
+            vec_layer<1>(actA + v * kD, sw3, kBits, lane, z3);
+            const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
+            if (lane == 0 && v < NV) codes_out[v] = code;
+        }
+    }
+    __syncthreads();
+}
+
+template <int G>
+__global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const FusedArgs a) {
+    extern __shared__ __align__(128) unsigned char fsm[];
+    // dynamic: [weights | row ring] union, activations, the cluster's states (used in CTA 0)
+    uint16_t *sw1 = reinterpret_cast<uint16_t *>(fsm);
+    uint16_t *sw2 = sw1 + kD * kHid;
+    uint16_t *sw3 = sw2 + kHid * kHid;
+    unsigned char *ring = fsm;
+    float *actA = reinterpret_cast<float *>(fsm + kFusedUnionBytes);
+    float *actB = actA + kMaxGroup * kD;
+    float *part_ml = reinterpret_cast<float *>(fsm + kFusedUnionBytes + kFusedActBytes);   // [CS][G][2]
+    float *part_acc = part_ml + kFusedCS * kMaxGroup * 2;                                   // [CS][G][128]
+    __shared__ __align__(8) unsigned long long s_bar[3];
+    __shared__ uint32_t s_codes[kMaxGroup];   // signatures produced by this CTA (CTA 0: queries, CTA 1: new key)
+    __shared__ __align__(16) unsigned char w_hist[kFusedWarps][kBins][32];
+    __shared__ int s_hist[kBins + 3], s_tot[kBins], s_bef[kBins];
+    __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
+    __shared__ int s_wcnt[kFusedWarps];
+    __shared__ float s_m[kFusedWarps][8], s_l[kFusedWarps][8];
+    __shared__ uint32_t s_mask[kFusedWarps][kFusedStages];
+
+    const uint32_t rank = cluster_rank();
+    const int kvh = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int Hq = a.Hq, Hkv = a.Hkv;
+    const int n = max(min(a.seq_lens[b], a.max_seq_len), 0);
+    int k = a.k_per_seq ? a.k_per_seq[b] : a.k_uniform;
+    k = max(0, min(k, a.k_max));
+    const int keep = min(k, n);
+    const long long head0 = (long long)b * Hq + (long long)kvh * G;
+    uint32_t *row = a.k_codes + (long long)b * a.kc_sb + (long long)kvh * a.kc_sh;
+    const bool has_new_key = (a.k_new != nullptr) && n > 0;
+
+    // ---------------- P0: requests that do not depend on earlier kernels
+    const int Lb = (n + kFusedCS * 1024 - 1) / (kFusedCS * 1024);
+    const int wbase = ((int)rank * 1024 + warp * 128 + lane * 4) * Lb;
+    uint4 c[kFusedL];
+#pragma unroll
+    for (int p = 0; p < kFusedL; ++p) {
+        const int base = wbase + p * 4;
+        c[p] = (p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
+    }
+    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&s_bar[0]);
+    const bool encodes = (rank == 0) || (rank == 1 && has_new_key);
+    const MapView &map = (rank == 0) ? a.map_q : a.map_k;
+    if (encodes && tid == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        mbar_init(bar0 + 16, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(bar0, kD * kHid * 2);
+        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw1), map.w1 + (size_t)kvh * kD * kHid, kD * kHid * 2, bar0);
+        mbar_expect_tx(bar0 + 8, kHid * kHid * 2);
+        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw2), map.w2 + (size_t)kvh * kHid * kHid, kHid * kHid * 2, bar0 + 8);
+        mbar_expect_tx(bar0 + 16, kHid * kBits * 2);
+        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw3), map.w3 + (size_t)kvh * kHid * kBits, kHid * kBits * 2, bar0 + 16);
+    }
+    for (int i = tid; i < kFusedWarps * kBins * 32 / 4; i += kFusedThreads)
+        reinterpret_cast<uint32_t *>(&w_hist[0][0][0])[i] = 0u;
+    if (tid < kBins + 3) s_hist[tid] = 0;
+    pdl_wait();                  // q, k_new and everything older in the stream is final from here on
+    pdl_launch_dependents();
+
+    // ---------------- P1: ENCODE in CTA 0 (queries) and CTA 1 (appended key)
+    if (rank == 0) {
+        fused_encode<G>(a.q + head0 * kD, kD, a.map_q, kvh, sw1, sw2, sw3, bar0, actA, actB, s_codes);
+        if (tid < G) a.q_codes[head0 + tid] = s_codes[tid];
+    } else if (rank == 1 && has_new_key) {
+        fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, a.map_k, kvh, sw1, sw2, sw3, bar0, actA, actB,
+                        s_codes);
+        if (tid == 0) row[n - 1] = s_codes[0];
+    }
+    cluster_sync_all();   // #1: the signatures are in CTA 0's and CTA 1's shared memory
+    uint32_t qc[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) qc[j] = (uint32_t)ld_dsmem(reinterpret_cast<const int *>(&s_codes[j]), 0);
+    if (has_new_key) {   // the appended token's signature replaces whatever the early request saw
+        const uint32_t kc = (uint32_t)ld_dsmem(reinterpret_cast<const int *>(&s_codes[0]), 1);
+#pragma unroll
+        for (int p = 0; p < kFusedL; ++p) {
+            const int e = (n - 1) - (wbase + p * 4);
+            if (p < Lb && e >= 0 && e <= 3) {
+                if (e == 0) c[p].x = kc; else if (e == 1) c[p].y = kc; else if (e == 2) c[p].z = kc; else c[p].w = kc;
+            }
+        }
+    }
+    __syncthreads();   // w_hist / s_hist zeroing is visible
+
+    // ---------------- P2: SCORE, histogram, threshold, compaction
+    uint32_t sc[kFusedL];
+    {
+        unsigned char *my = &w_hist[warp][0][lane] - 32;   // indexed by the score+1 byte
+#pragma unroll
+        for (int p = 0; p < kFusedL; ++p) {
+            const int base = wbase + p * 4;
+            uint32_t s4 = scores4<G>(c[p], qc);
+            if (p < Lb && base + 3 < n) {
+                my[(s4 & 0xffu) * 32] += 1;
+                my[((s4 >> 8) & 0xffu) * 32] += 1;
+                my[((s4 >> 16) & 0xffu) * 32] += 1;
+                my[(s4 >> 24) * 32] += 1;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (p < Lb && base + e < n) my[((s4 >> (8 * e)) & 0xffu) * 32] += 1;
+                    else s4 &= ~(0xffu << (8 * e));   // zero byte: no token
+            }
+            sc[p] = s4;
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < kBins * kFusedWarps; i += kFusedThreads) {
+        const int bin = i >> 3, w = i & 7;
+        const uint4 *rowp = reinterpret_cast<const uint4 *>(&w_hist[w][bin][0]);
+        const uint4 a0 = rowp[0], a1 = rowp[1];
+        const int s = (int)(__vsadu4(a0.x, 0u) + __vsadu4(a0.y, 0u) + __vsadu4(a0.z, 0u) + __vsadu4(a0.w, 0u) +
+                            __vsadu4(a1.x, 0u) + __vsadu4(a1.y, 0u) + __vsadu4(a1.z, 0u) + __vsadu4(a1.w, 0u));
+        if (s) atomicAdd(&s_hist[bin], s);
+    }
+    cluster_sync_all();   // #2: every CTA's histogram is complete and visible cluster-wide
+    if (tid < kBins) {
+        int tot = 0, bef = 0;
+#pragma unroll
+        for (uint32_t r = 0; r < (uint32_t)kFusedCS; ++r) {
+            const int v = ld_dsmem(&s_hist[tid], r);
+            tot += v;
+            if (r < rank) bef += v;
+        }
+        s_tot[tid] = tot;
+        s_bef[tid] = bef;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int T, r, gt_before, eq_before;
+        find_threshold(s_tot[lane], s_bef[lane], s_tot[32], s_bef[32], keep, lane, T, r, gt_before, eq_before);
+        if (lane == 0) { sh_T = T; sh_r = r; sh_gt_before = gt_before; sh_eq_before = eq_before; }
+    }
+    __syncthreads();
+    int32_t *list = a.idx + (long long)b * a.idx_sb + (long long)kvh * a.idx_sh;
+    if (rank == 0) {
+        if (tid == 0) a.count[b * Hkv + kvh] = keep;
+        for (int i = keep + tid; i < a.k_max; i += kFusedThreads) list[i] = -1;
+    }
+    if (keep > 0) {
+        const int T = sh_T, r = sh_r;
+        const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
+        int tot_packed = 0;
+#pragma unroll
+        for (int p = 0; p < kFusedL; ++p) {
+            uint32_t gt, eq;
+            flags4(sc[p], T4, gt, eq);
+            tot_packed += __popc(gt) | (__popc(eq) << 16);
+        }
+        int winc = tot_packed;
+#pragma unroll
+        for (int dd = 1; dd < 32; dd <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, winc, dd);
+            if (lane >= dd) winc += v;
+        }
+        if (lane == 31) s_wcnt[warp] = winc;
+        __syncthreads();
+        int run_gt = sh_gt_before, run_eq = sh_eq_before;
+#pragma unroll
+        for (int w = 0; w < kFusedWarps; ++w)
+            if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
+        const int excl = winc - tot_packed;
+        int gt_lt = run_gt + (excl & 0xffff);
+        int eq_lt = run_eq + (int)((unsigned)excl >> 16);
+        if (tot_packed != 0) {
+#pragma unroll
+            for (int p = 0; p < kFusedL; ++p) {
+                uint32_t gt, eq;
+                flags4(sc[p], T4, gt, eq);
+                if ((gt | eq) == 0u) continue;
+                const int base = wbase + p * 4;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if ((gt >> (8 * e + 7)) & 1u) {
+                        list[gt_lt + min(eq_lt, r)] = base + e;
+                        ++gt_lt;
+                    } else if ((eq >> (8 * e + 7)) & 1u) {
+                        if (eq_lt < r) list[gt_lt + eq_lt] = base + e;
+                        ++eq_lt;
+                    }
+                }
+            }
+        }
+    }
+    cluster_sync_all();   // #3: the index list is complete and visible to the whole cluster; histograms are free
+
+    // ---------------- P3: GATHER-ATT over this CTA's eighth of the list
+    const int blocks_total = (keep + kBlockTokens - 1) / kBlockTokens;
+    const int bpc = (blocks_total + kFusedCS - 1) / kFusedCS;             // blocks per CTA
+    const int blk_lo = min(blocks_total, (int)rank * bpc), blk_hi = min(blocks_total, blk_lo + bpc);
+    const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (long long)b * a.K.sb + (long long)kvh * a.K.sh);
+    const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (long long)b * a.V.sb + (long long)kvh * a.V.sh);
+    const long long k_row = a.K.sn * 2, v_row = a.V.sn * 2;
+    unsigned char *my_ring = ring + warp * (kFusedStages * kStageBytes);
+    const uint32_t ring_u32 = smem_u32(my_ring);
+    const int g = lane >> 2, cc = lane & 3;
+
+    uint32_t qa[8][2];
+    attn_load_q<G>(qa, a.q + head0 * kD, lane);
+    float acc[8][4];
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[mt][e] = 0.0f;
+    float m_run = -CUDART_INF_F, l_run = 0.0f;
+    {
+        // this warp's blocks: blk_lo + warp, + 8, ...; list entries come from peer CTAs: read them from L2
+        const int nblk = (blk_lo + warp < blk_hi) ? (blk_hi - blk_lo - warp + kFusedWarps - 1) / kFusedWarps : 0;
+        auto token_of_block = [&](int i) -> int {
+            const int p = (blk_lo + warp + i * kFusedWarps) * kBlockTokens + (lane & 15);
+            return (i < nblk && p < keep) ? __ldcg(list + p) : -1;
+        };
+        auto issue = [&](int i, int stg) {
+            const uint32_t valid = attn_issue_block(ring_u32 + stg * kStageBytes, Kb, Vb, k_row, v_row, token_of_block(i), lane);
+            if (lane == 0) s_mask[warp][stg] = valid;
+        };
+        if (nblk > 0) issue(0, 0);
+        cp_async_commit();
+        for (int i = 0; i < nblk; ++i) {
+            const int stg = i & 1;
+            if (i + 1 < nblk) issue(i + 1, stg ^ 1);
+            cp_async_commit();
+            cp_async_wait<1>();
+            __syncwarp();
+            const uint32_t ks = ring_u32 + stg * kStageBytes;
+            attn_consume_block(ks, ks + kTileBytes, s_mask[warp][stg], qa, a.scale_log2, lane, acc, m_run, l_run);
+            __syncwarp();
+        }
+        cp_async_wait<0>();
+    }
+    // merge the warps of this CTA through shared memory (each warp reuses its own ring)
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (cc == 0) { s_m[warp][g] = m_run; s_l[warp][g] = l_run; }
+    __syncwarp();
+    {
+        float *my_acc = reinterpret_cast<float *>(my_ring);   // [G][128]
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int h = 2 * cc + hh;
+            if (h < G) {
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    my_acc[h * kD + 16 * mt + g] = acc[mt][hh];
+                    my_acc[h * kD + 16 * mt + 8 + g] = acc[mt][2 + hh];
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (tid < kD) {   // this CTA's state goes into slot `rank` of CTA 0's shared memory
+        const int d = tid;
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+            float M = s_m[0][j];
+#pragma unroll
+            for (int w = 1; w < kFusedWarps; ++w) M = fmaxf(M, s_m[w][j]);
+            float L = 0.0f, A = 0.0f;
+            if (M > -CUDART_INF_F) {
+#pragma unroll
+                for (int w = 0; w < kFusedWarps; ++w) {
+                    const float f = exp2f(s_m[w][j] - M);
+                    L = fmaf(s_l[w][j], f, L);
+                    A = fmaf(reinterpret_cast<const float *>(ring + w * (kFusedStages * kStageBytes))[j * kD + d], f, A);
+                }
+            }
+            st_dsmem_f32(part_acc + ((int)rank * G + j) * kD + d, 0, A);
+            if (d == 0) {
+                st_dsmem_f32(part_ml + ((int)rank * G + j) * 2, 0, M);
+                st_dsmem_f32(part_ml + ((int)rank * G + j) * 2 + 1, 0, L);
+            }
+        }
+    }
+    cluster_sync_all();   // #4: all eight states have landed in CTA 0
+    if (rank == 0 && tid < kD) {
+        const int d = tid;
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+            float M = -CUDART_INF_F;
+#pragma unroll
+            for (int r = 0; r < kFusedCS; ++r) M = fmaxf(M, part_ml[(r * G + j) * 2]);
+            float L = 0.0f, A = 0.0f;
+            if (M > -CUDART_INF_F) {
+#pragma unroll
+                for (int r = 0; r < kFusedCS; ++r) {
+                    const float f = exp2f(part_ml[(r * G + j) * 2] - M);
+                    L = fmaf(part_ml[(r * G + j) * 2 + 1], f, L);
+                    A = fmaf(part_acc[(r * G + j) * kD + d], f, A);
+                }
+            }
+            const float o = (L > 0.0f) ? A / L : 0.0f;
+            const __nv_bfloat16 ob = __float2bfloat16_rn(o);
+            a.out[(head0 + j) * kD + d] = *reinterpret_cast<const uint16_t *>(&ob);
+            if (a.lse && d == 0) a.lse[head0 + j] = (L > 0.0f) ? (M * kLn2 + logf(L)) : -CUDART_INF_F;
+        }
+    }
+}
+
+template <int G>
+static cudaError_t launch_fused_g(const FusedArgs &args, int B, cudaStream_t st) {
+    static bool done[64] = {};   // opt in to the large shared-memory carve-out once per device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(fused_step_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kFusedSmemBytes);
+        if (e != cudaSuccess) return e;
+        done[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kFusedCS, args.Hkv, B);
+    cfg.blockDim = dim3(kFusedThreads);
+    cfg.dynamicSmemBytes = kFusedSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kFusedCS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_step_kernel<G>, args);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    return cudaGetLastError();
+}
+
+bool fused_step_eligible(int B, int Hkv, int max_seq_len) {
+    return (long long)B * Hkv * kFusedCS <= 148 && max_seq_len <= kFusedCS * kFusedL * 1024;
+}
+
+cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapView &map_q, const MapView &map_k,
+                              const uint16_t *q, const uint16_t *k_new, TensorView K, TensorView V, uint32_t *k_codes,
+                              long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
+                              int k_uniform, int max_seq_len, int k_max, uint32_t *q_codes, int32_t *idx,
+                              long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
+                              cudaStream_t st) {
+    FusedArgs a{};
+    a.map_q = map_q; a.map_k = map_k; a.q = q; a.k_new = k_new; a.K = K; a.V = V;
+    a.k_codes = k_codes; a.kc_sb = kc_sb; a.kc_sh = kc_sh; a.seq_lens = seq_lens; a.k_per_seq = k_per_seq;
+    a.k_uniform = k_uniform; a.max_seq_len = max_seq_len; a.k_max = k_max; a.Hq = Hq; a.Hkv = Hkv;
+    a.scale_log2 = sm_scale * kLog2e; a.q_codes = q_codes; a.idx = idx; a.idx_sb = idx_sb; a.idx_sh = idx_sh;
+    a.count = count; a.out = out; a.lse = lse;
+    switch (Hq / Hkv) {
+        case 1: return launch_fused_g<1>(a, B, st);
+        case 2: return launch_fused_g<2>(a, B, st);
+        case 4: return launch_fused_g<4>(a, B, st);
+        case 8: return launch_fused_g<8>(a, B, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+} // namespace ha
