@@ -4,11 +4,12 @@
 // decode step keeps 64 SMs busy without a single kernel boundary or global-memory hand-off on its
 // critical path:
 //
-//   P0  every CTA requests its slice of the signature cache; CTA 0 and CTA 1 of the cluster request
+//   P0  every CTA requests its slice of the signature cache; the encoding CTAs of the cluster request
 //       the query-side / key-side mapping weights with bulk asynchronous copies (TMA, mbarriers);
 //       all of it before the programmatic-launch wait, i.e. behind the preceding kernel.
-//   P1  CTA 0 encodes the G query vectors, CTA 1 the appended key (fp32 fma chains, Eq. 2);
-//       cluster barrier; everybody reads the five signatures through distributed shared memory.
+//   P1  CTA r < ceil(G/2) encodes query vectors 2r, 2r+1, the next CTA the appended key (fp32 fma
+//       chains, Eq. 2, one chain per thread); cluster barrier; everybody reads the signatures
+//       through distributed shared memory.
 //   P2  scores as bytes in registers, per-CTA histogram, cluster barrier, histogram exchange through
 //       distributed shared memory, threshold, compaction of the CTA's slice into the index list;
 //       cluster barrier (the list is now visible to the whole cluster).
@@ -157,8 +158,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         c[p] = (p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
     }
     const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&s_bar[0]);
-    const bool encodes = (rank == 0) || (rank == 1 && has_new_key);
-    const MapView &map = (rank == 0) ? a.map_q : a.map_k;
+    // ENCODE roles: CTA r < kQCtas encodes query vectors 2r and 2r+1 (one fma chain per thread), CTA kQCtas
+    // encodes the appended key; the other CTAs only scan
+    constexpr int kQCtas = (G + 1) / 2;
+    constexpr int kQPer = (G >= 2) ? 2 : 1;
+    const bool enc_q = (int)rank < kQCtas, enc_k = ((int)rank == kQCtas) && has_new_key;
+    const bool encodes = enc_q || enc_k;
+    const MapView &map = enc_q ? a.map_q : a.map_k;
     if (encodes && tid == 0) {
         mbar_init(bar0, 1);
         mbar_init(bar0 + 8, 1);
@@ -178,20 +184,22 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     pdl_launch_dependents();
 
     // ---------------- P1: ENCODE in CTA 0 (queries) and CTA 1 (appended key)
-    if (rank == 0) {
-        fused_encode<G>(a.q + head0 * kD, kD, a.map_q, kvh, sw1, sw2, sw3, bar0, actA, actB, s_codes);
-        if (tid < G) a.q_codes[head0 + tid] = s_codes[tid];
-    } else if (rank == 1 && has_new_key) {
+    if (enc_q) {
+        fused_encode<kQPer>(a.q + (head0 + kQPer * (int)rank) * kD, kD, a.map_q, kvh, sw1, sw2, sw3, bar0, actA, actB,
+                            s_codes);
+        if (tid < kQPer) a.q_codes[head0 + kQPer * (int)rank + tid] = s_codes[tid];
+    } else if (enc_k) {
         fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, a.map_k, kvh, sw1, sw2, sw3, bar0, actA, actB,
                         s_codes);
         if (tid == 0) row[n - 1] = s_codes[0];
     }
-    cluster_sync_all();   // #1: the signatures are in CTA 0's and CTA 1's shared memory
+    cluster_sync_all();   // #1: the signatures are in the encoding CTAs' shared memory
     uint32_t qc[G];
 #pragma unroll
-    for (int j = 0; j < G; ++j) qc[j] = (uint32_t)ld_dsmem(reinterpret_cast<const int *>(&s_codes[j]), 0);
+    for (int j = 0; j < G; ++j)
+        qc[j] = (uint32_t)ld_dsmem(reinterpret_cast<const int *>(&s_codes[j % kQPer]), (uint32_t)(j / kQPer));
     if (has_new_key) {   // the appended token's signature replaces whatever the early request saw
-        const uint32_t kc = (uint32_t)ld_dsmem(reinterpret_cast<const int *>(&s_codes[0]), 1);
+        const uint32_t kc = (uint32_t)ld_dsmem(reinterpret_cast<const int *>(&s_codes[0]), (uint32_t)kQCtas);
 #pragma unroll
         for (int p = 0; p < kFusedL; ++p) {
             const int e = (n - 1) - (wbase + p * 4);
