@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     float *part_acc = part_ml + kFusedCS * kMaxGroup * 2;                                   // [CS][G][128]
     __shared__ __align__(8) unsigned long long s_bar[3];
     __shared__ uint32_t s_codes[kMaxGroup];   // signatures produced by this CTA (CTA 0: queries, CTA 1: new key)
-    __shared__ __align__(16) unsigned char w_hist[kFusedWarps][kBins][32];
+    __shared__ __align__(16) uint32_t w_hist[kFusedWarps][kBins][32];   // one counter per (warp, level, lane)
     __shared__ int s_hist[kBins + 3], s_tot[kBins], s_bef[kBins];
     __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
     __shared__ int s_wcnt[kFusedWarps];
@@ -177,8 +177,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         mbar_expect_tx(bar0 + 16, kHid * kBits * 2);
         bulk_g2s((uint32_t)__cvta_generic_to_shared(sw3), map.w3 + (size_t)kvh * kHid * kBits, kHid * kBits * 2, bar0 + 16);
     }
-    for (int i = tid; i < kFusedWarps * kBins * 32 / 4; i += kFusedThreads)
-        reinterpret_cast<uint32_t *>(&w_hist[0][0][0])[i] = 0u;
+    for (int i = tid; i < kFusedWarps * kBins * 32; i += kFusedThreads) (&w_hist[0][0][0])[i] = 0u;
     if (tid < kBins + 3) s_hist[tid] = 0;
     pdl_wait();                  // q, k_new and everything older in the stream is final from here on
     pdl_launch_dependents();
@@ -213,33 +212,35 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     // ---------------- P2: SCORE, histogram, threshold, compaction
     uint32_t sc[kFusedL];
     {
-        unsigned char *my = &w_hist[warp][0][lane] - 32;   // indexed by the score+1 byte
+        // counters are private to a lane, so the adds never conflict; they are issued without waiting
+        // for a result (reduction, not read-modify-write), 16 in a row
+        const uint32_t my = (uint32_t)__cvta_generic_to_shared(&w_hist[warp][0][lane]) - 32u * 4u;   // index: score+1
+        auto bump = [&](uint32_t byte) {
+            asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(my + byte * (32u * 4u)) : "memory");
+        };
 #pragma unroll
         for (int p = 0; p < kFusedL; ++p) {
             const int base = wbase + p * 4;
             uint32_t s4 = scores4<G>(c[p], qc);
             if (p < Lb && base + 3 < n) {
-                my[(s4 & 0xffu) * 32] += 1;
-                my[((s4 >> 8) & 0xffu) * 32] += 1;
-                my[((s4 >> 16) & 0xffu) * 32] += 1;
-                my[(s4 >> 24) * 32] += 1;
+                bump(s4 & 0xffu); bump((s4 >> 8) & 0xffu); bump((s4 >> 16) & 0xffu); bump(s4 >> 24);
             } else {
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (p < Lb && base + e < n) my[((s4 >> (8 * e)) & 0xffu) * 32] += 1;
+                    if (p < Lb && base + e < n) bump((s4 >> (8 * e)) & 0xffu);
                     else s4 &= ~(0xffu << (8 * e));   // zero byte: no token
             }
             sc[p] = s4;
         }
     }
     __syncthreads();
-    for (int i = tid; i < kBins * kFusedWarps; i += kFusedThreads) {
+    for (int i = tid; i < kBins * kFusedWarps; i += kFusedThreads) {   // one (level, warp) row of 32 counters per thread
         const int bin = i >> 3, w = i & 7;
         const uint4 *rowp = reinterpret_cast<const uint4 *>(&w_hist[w][bin][0]);
-        const uint4 a0 = rowp[0], a1 = rowp[1];
-        const int s = (int)(__vsadu4(a0.x, 0u) + __vsadu4(a0.y, 0u) + __vsadu4(a0.z, 0u) + __vsadu4(a0.w, 0u) +
-                            __vsadu4(a1.x, 0u) + __vsadu4(a1.y, 0u) + __vsadu4(a1.z, 0u) + __vsadu4(a1.w, 0u));
-        if (s) atomicAdd(&s_hist[bin], s);
+        uint32_t ssum = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) { const uint4 v = rowp[q]; ssum += (v.x + v.y) + (v.z + v.w); }
+        if (ssum) atomicAdd(&s_hist[bin], (int)ssum);
     }
     cluster_sync_all();   // #2: every CTA's histogram is complete and visible cluster-wide
     if (tid < kBins) {
@@ -268,13 +269,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     if (keep > 0) {
         const int T = sh_T, r = sh_r;
         const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
-        int tot_packed = 0;
+        uint32_t gt16 = 0, eq16 = 0;   // flags of this lane's 16 consecutive tokens
 #pragma unroll
         for (int p = 0; p < kFusedL; ++p) {
             uint32_t gt, eq;
             flags4(sc[p], T4, gt, eq);
-            tot_packed += __popc(gt) | (__popc(eq) << 16);
+            gt16 |= flags_to_nibble(gt) << (4 * p);
+            eq16 |= flags_to_nibble(eq) << (4 * p);
         }
+        const int tot_packed = __popc(gt16) | (__popc(eq16) << 16);
         int winc = tot_packed;
 #pragma unroll
         for (int dd = 1; dd < 32; dd <<= 1) {
@@ -288,27 +291,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         for (int w = 0; w < kFusedWarps; ++w)
             if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
         const int excl = winc - tot_packed;
-        int gt_lt = run_gt + (excl & 0xffff);
-        int eq_lt = run_eq + (int)((unsigned)excl >> 16);
-        if (tot_packed != 0) {
-#pragma unroll
-            for (int p = 0; p < kFusedL; ++p) {
-                uint32_t gt, eq;
-                flags4(sc[p], T4, gt, eq);
-                if ((gt | eq) == 0u) continue;
-                const int base = wbase + p * 4;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if ((gt >> (8 * e + 7)) & 1u) {
-                        list[gt_lt + min(eq_lt, r)] = base + e;
-                        ++gt_lt;
-                    } else if ((eq >> (8 * e + 7)) & 1u) {
-                        if (eq_lt < r) list[gt_lt + eq_lt] = base + e;
-                        ++eq_lt;
-                    }
-                }
-            }
-        }
+        write_selected16(list, wbase, gt16, eq16, run_gt + (excl & 0xffff), run_eq + (int)((unsigned)excl >> 16), r);
     }
     cluster_sync_all();   // #3: the index list is complete and visible to the whole cluster; histograms are free
 

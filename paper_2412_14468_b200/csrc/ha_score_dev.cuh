@@ -68,6 +68,28 @@ __device__ __forceinline__ int ld_dsmem(const int *local, uint32_t rank) {
 }
 
 
+// The four bit-7 flags of a word gathered into a nibble (bit e = flag of byte e).
+__device__ __forceinline__ uint32_t flags_to_nibble(uint32_t f) {
+    return ((((f >> 7) & 0x01010101u) * 0x01020408u) >> 24) & 0xfu;
+}
+
+// Writes the selected tokens among 16 consecutive tokens starting at `first`: gt16 / eq16 are the
+// per-token flags "score > T" / "score == T" (bit e = token first + e); gt_lt / eq_lt count the
+// tokens before `first` with those properties; r tokens of score T are still wanted overall.
+// Only the flagged tokens are visited; each position comes from popcounts, not from a running sum.
+__device__ __forceinline__ void write_selected16(int32_t *list, int first, uint32_t gt16, uint32_t eq16, int gt_lt,
+                                                 int eq_lt, int r) {
+    uint32_t m = gt16 | eq16;
+    while (m) {
+        const int e = __ffs((int)m) - 1;
+        m &= m - 1;
+        const uint32_t below = (1u << e) - 1u;
+        const int g = gt_lt + __popc(gt16 & below), q = eq_lt + __popc(eq16 & below);
+        if ((gt16 >> e) & 1u) list[g + min(q, r)] = first + e;
+        else if (q < r) list[g + q] = first + e;
+    }
+}
+
 // Warp-wide threshold search over the 33 score levels.  Lane l passes the count of level l (tot) and
 // the part of it that lies before the caller's own slice (bef); level 32 comes in tot32 / bef32.
 // Returns T = largest level with #{S >= T} >= keep, r = keep - #{S > T}, and the numbers of tokens
