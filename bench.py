@@ -27,6 +27,7 @@ if ROOT not in sys.path:
 
 METRIC = "sparse_decode_attn_us_per_layer_step"
 UNIT = "us"
+FUSED_KERNEL_TRAFFIC_C2 = 6519000   # dram__bytes_read.sum + write per launch, profiles/launch_list_bench_c2.md
 WORKLOAD = "c2: B=1, Hq=32, Hkv=8, d=128, ctx=32768, k=1024 (32x), 1% planted keys"
 
 
@@ -328,18 +329,30 @@ def main():
         parts[name] = t * 1e3 / sub_steps
     gather_bytes = sum(cfg.n_kv_heads * 512 * min(k, n) + cfg.n_q_heads * 512 for n, k in zip(lens, ks))
     scan_bytes = sum(cfg.n_kv_heads * 4 * n for n in lens)
+    launches_per_step = launches / steps
+    # At this batch size the whole layer-step is ONE kernel (fused_step_kernel: one 8-CTA cluster per
+    # (sequence, KV head)), so the timed region contains launches of that kernel only and its average
+    # launch duration is the step time itself.
+    achieved = alg_bytes / (us_per_step * 1e-6) / 1e9
     g_us = parts["ha_gather_attn"]
-    achieved = gather_bytes / (g_us * 1e-6) / 1e9
     roofline = {
-        "bound": "hbm", "kernel": "attn_kernel<4,true> (the one kernel of ha_gather_attn)",
+        "bound": "hbm",
+        "kernel": ("fused_step_kernel<4> (the one kernel of ha_sparse_decode at this batch size)"
+                   if launches_per_step < 1.5 else "kernels of ha_sparse_decode (multi-kernel path)"),
         "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
         # dram__bytes_read.sum + dram__bytes_write.sum per launch of this kernel on this workload, from the
         # ncu launch list of this very command (profiles/launch_list_bench_c2.md)
-        "traffic": 4302000, "algorithmic_bytes_per_launch": gather_bytes, "us_per_launch": g_us,
-        "whole_step": {"algorithmic_bytes": alg_bytes, "achieved": alg_bytes / (us_per_step * 1e-6) / 1e9,
-                       "frac": alg_bytes / (us_per_step * 1e-6) / 1e9 / peak},
-        "ha_score_topk": {"algorithmic_bytes": scan_bytes, "us": parts["ha_score_topk"],
-                          "achieved": scan_bytes / (parts["ha_score_topk"] * 1e-6) / 1e9},
+        "traffic": FUSED_KERNEL_TRAFFIC_C2 if launches_per_step < 1.5 else None,
+        "algorithmic_bytes_per_launch": alg_bytes, "us_per_launch": us_per_step,
+        "launches_per_step": launches_per_step,
+        "standalone_entry_points": {
+            "ha_gather_attn (attn_kernel<4,true>)": {"algorithmic_bytes": gather_bytes, "us": g_us,
+                                                      "achieved": gather_bytes / (g_us * 1e-6) / 1e9,
+                                                      "frac": gather_bytes / (g_us * 1e-6) / 1e9 / peak, "traffic": 4302000},
+            "ha_score_topk (score_select_cluster_kernel<4,4,8>)": {"algorithmic_bytes": scan_bytes, "us": parts["ha_score_topk"],
+                                                                    "achieved": scan_bytes / (parts["ha_score_topk"] * 1e-6) / 1e9},
+            "ha_encode[q] (encode_vec_kernel<4>)": {"us": parts["ha_encode[q]"]},
+        },
     }
 
     # ---- end to end through the host-buffer entry point (H2D of q/k_new/v_new, D2H of out, sync per step)
@@ -413,7 +426,7 @@ def main():
             "dtype": "bf16 in/out, fp32 accumulate; u32 signatures", "data": "synthetic",
             "config": {"workload": WORKLOAD, "replicas": R,
                        "l2": f"steps rotate over {R} layer replicas ({R * alg_bytes / 1e6:.0f} MB touched per rotation > 126 MB L2)",
-                       "launch": "CUDA graphs of ha_sparse_decode calls", "parallelism": f"replicas x{world}"},
+                       "launch": "CUDA graphs of ha_sparse_decode calls (one fused cluster kernel per step at this batch size)", "parallelism": f"replicas x{world}"},
             "clocks": sampler.summary(), "gpu_launches": launches, "e2e": e2e, "roofline": roofline,
             "cpu_baseline": cpu_baseline, "breakdown_us": parts, "dense_same_run": dense, "supplementary": supplementary,
             "paper_context": "A100: up to 4.3x (GPT-FAST) / 2.54x (FlashDecode) attention latency reduction at 32x",

@@ -258,14 +258,34 @@ int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const 
     uint16_t *dv = ws_ptr<uint16_t>(workspace, L.off_stage_v);
     uint16_t *dout = ws_ptr<uint16_t>(workspace, L.off_stage_out);
     uint32_t *dqc = ws_ptr<uint32_t>(workspace, L.off_qcodes);
-    HA_CUDA(cudaMemcpyAsync(dq, q_host, (size_t)B * Hq * kD * 2, cudaMemcpyHostToDevice, st));
-    HA_CUDA(cudaMemcpyAsync(dk, k_new_host, (size_t)B * Hkv * kD * 2, cudaMemcpyHostToDevice, st));
-    HA_CUDA(cudaMemcpyAsync(dv, v_new_host, (size_t)B * Hkv * kD * 2, cudaMemcpyHostToDevice, st));
-    HA_CUDA(launch_append_kv(B, Hkv, dk, dv, view(K), view(V), seq_lens, st));
-    HA_TRY(ha_sparse_decode(shape, map_q, map_k, dq, dk, K, V, k_codes, kc_stride_b, kc_stride_h, seq_lens,
-                            k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx, idx_stride_b, idx_stride_h, count,
-                            dout, nullptr, workspace, ws_bytes, stream));
-    HA_CUDA(cudaMemcpyAsync(out_host, dout, (size_t)B * Hq * kD * 2, cudaMemcpyDeviceToHost, st));
+    // Pinned host buffers that the device can address (cudaHostAlloc / cudaHostRegister under unified
+    // addressing) are read and written by the kernels themselves: one small kernel pulls q, k_new and
+    // v_new across the bus and the last kernel of the step writes `out` straight into host memory.
+    // Anything else goes through staged copies.
+    auto mapped = [](const void *p) -> void * {
+        cudaPointerAttributes at;
+        if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        return (at.type == cudaMemoryTypeHost) ? at.devicePointer : nullptr;
+    };
+    const uint16_t *mq = reinterpret_cast<const uint16_t *>(mapped(q_host));
+    const uint16_t *mkn = reinterpret_cast<const uint16_t *>(mapped(k_new_host));
+    const uint16_t *mvn = reinterpret_cast<const uint16_t *>(mapped(v_new_host));
+    uint16_t *mout = reinterpret_cast<uint16_t *>(mapped(out_host));
+    if (mq && mkn && mvn && mout) {
+        HA_CUDA(launch_append_kv(B, Hq, Hkv, mkn, mvn, view(K), view(V), seq_lens, mq, dq, dk, st));
+        HA_TRY(ha_sparse_decode(shape, map_q, map_k, dq, dk, K, V, k_codes, kc_stride_b, kc_stride_h, seq_lens,
+                                k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx, idx_stride_b, idx_stride_h, count,
+                                mout, nullptr, workspace, ws_bytes, stream));
+    } else {
+        HA_CUDA(cudaMemcpyAsync(dq, q_host, (size_t)B * Hq * kD * 2, cudaMemcpyHostToDevice, st));
+        HA_CUDA(cudaMemcpyAsync(dk, k_new_host, (size_t)B * Hkv * kD * 2, cudaMemcpyHostToDevice, st));
+        HA_CUDA(cudaMemcpyAsync(dv, v_new_host, (size_t)B * Hkv * kD * 2, cudaMemcpyHostToDevice, st));
+        HA_CUDA(launch_append_kv(B, Hq, Hkv, dk, dv, view(K), view(V), seq_lens, nullptr, nullptr, nullptr, st));
+        HA_TRY(ha_sparse_decode(shape, map_q, map_k, dq, dk, K, V, k_codes, kc_stride_b, kc_stride_h, seq_lens,
+                                k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx, idx_stride_b, idx_stride_h, count,
+                                dout, nullptr, workspace, ws_bytes, stream));
+        HA_CUDA(cudaMemcpyAsync(out_host, dout, (size_t)B * Hq * kD * 2, cudaMemcpyDeviceToHost, st));
+    }
     HA_CUDA(cudaStreamSynchronize(st));
     return HA_OK;
 }

@@ -451,22 +451,38 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
     }
 }
 
-// Writes this step's new K and V rows into the cache at slot seq_len-1 (host-driven entry only).
-__global__ void append_kv_kernel(int Hkv, const uint16_t *__restrict__ k_new, const uint16_t *__restrict__ v_new,
-                                 TensorView K, TensorView V, const int32_t *__restrict__ seq_lens) {
-    const int g = blockIdx.x, b = blockIdx.y, t = threadIdx.x;   // 32 threads x 8 bytes
+// Host-driven entry only: writes this step's new K and V rows into the cache at slot seq_len-1 and,
+// if q_src is given, copies the query vectors into the device staging buffer.  The sources may be
+// device memory or pinned host memory mapped into the device's address space (then this kernel IS
+// the host-to-device transfer: one launch instead of three copy operations).
+__global__ void append_kv_kernel(int Hq, int Hkv, const uint16_t *__restrict__ k_new,
+                                 const uint16_t *__restrict__ v_new, TensorView K, TensorView V,
+                                 const int32_t *__restrict__ seq_lens, const uint16_t *__restrict__ q_src,
+                                 uint16_t *__restrict__ q_dst, uint16_t *__restrict__ k_dst) {
+    const int g = blockIdx.x, b = blockIdx.y, t = threadIdx.x;   // 32 threads x 8 bytes per row
+    const long long src = ((long long)b * Hkv + g) * kD;
+    const uint2 kv = reinterpret_cast<const uint2 *>(k_new + src)[t];
+    const uint2 vv = reinterpret_cast<const uint2 *>(v_new + src)[t];
+    if (k_dst) reinterpret_cast<uint2 *>(k_dst + src)[t] = kv;   // device copy of k_new for ENCODE
+    if (q_src) {
+        const int G = Hq / Hkv;
+        for (int j = 0; j < G; ++j) {
+            const long long qo = ((long long)b * Hq + (long long)g * G + j) * kD;
+            reinterpret_cast<uint2 *>(q_dst + qo)[t] = reinterpret_cast<const uint2 *>(q_src + qo)[t];
+        }
+    }
     const int slot = seq_lens[b] - 1;
     if (slot < 0) return;
-    const long long src = ((long long)b * Hkv + g) * kD;
     uint16_t *kd = const_cast<uint16_t *>(K.ptr) + (long long)b * K.sb + (long long)g * K.sh + (long long)slot * K.sn;
     uint16_t *vd = const_cast<uint16_t *>(V.ptr) + (long long)b * V.sb + (long long)g * V.sh + (long long)slot * V.sn;
-    reinterpret_cast<uint2 *>(kd)[t] = reinterpret_cast<const uint2 *>(k_new + src)[t];
-    reinterpret_cast<uint2 *>(vd)[t] = reinterpret_cast<const uint2 *>(v_new + src)[t];
+    reinterpret_cast<uint2 *>(kd)[t] = kv;
+    reinterpret_cast<uint2 *>(vd)[t] = vv;
 }
 
-cudaError_t launch_append_kv(int B, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
-                             TensorView V, const int32_t *seq_lens, cudaStream_t st) {
-    append_kv_kernel<<<dim3(Hkv, B), 32, 0, st>>>(Hkv, k_new, v_new, K, V, seq_lens);
+cudaError_t launch_append_kv(int B, int Hq, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
+                             TensorView V, const int32_t *seq_lens, const uint16_t *q_src, uint16_t *q_dst,
+                             uint16_t *k_dst, cudaStream_t st) {
+    append_kv_kernel<<<dim3(Hkv, B), 32, 0, st>>>(Hq, Hkv, k_new, v_new, K, V, seq_lens, q_src, q_dst, k_dst);
     count_launch();
     return cudaGetLastError();
 }

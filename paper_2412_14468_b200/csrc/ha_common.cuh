@@ -147,7 +147,8 @@ cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapV
                               long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
                               cudaStream_t st);
 
-cudaError_t launch_append_kv(int B, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
-                             TensorView V, const int32_t *seq_lens, cudaStream_t st);
+cudaError_t launch_append_kv(int B, int Hq, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
+                             TensorView V, const int32_t *seq_lens, const uint16_t *q_src, uint16_t *q_dst,
+                             uint16_t *k_dst, cudaStream_t st);
 
 } // namespace ha

@@ -269,7 +269,7 @@ def test_dense_decode_matches_oracle(lens):
 
 # ---------------------------------------------------------------------------- whole step
 
-def _run_step(w, host=False):
+def _run_step(w, host=False, pinned=True):
     cfg = w["cfg"]
     B, Hq, Hkv = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads
     shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
@@ -291,8 +291,9 @@ def _run_step(w, host=False):
             if w["lens"][b] > 0:
                 K2[b, :, w["lens"][b] - 1] = 0
                 V2[b, :, w["lens"][b] - 1] = 0
-        hq, hk, hv = (w[x].cpu().pin_memory() for x in ("q", "k_new", "v_new"))
-        ho = torch.zeros(B, Hq, 128, dtype=torch.bfloat16).pin_memory()
+        pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)     # pageable buffers take the staged-copy route
+        hq, hk, hv = (pin(w[x].cpu()) for x in ("q", "k_new", "v_new"))
+        ho = pin(torch.zeros(B, Hq, 128, dtype=torch.bfloat16))
         ha.ha_sparse_decode_host(shape, mq, mk, hq, hk, hv, K2, V2, kc, w["seq_lens"], w["k_per_seq"], 0, w["n_cap"],
                                  w["k_max"], idx, cnt, ho, ws)
         assert torch.equal(K2, w["K"]) and torch.equal(V2, w["V"])   # the new rows were appended in place
@@ -331,8 +332,9 @@ def test_sparse_decode_step_matches_oracle(cfg):
     assert np.array_equal(np.isneginf(got_lse), ~finite)            # empty selections: lse = -inf on both sides
     assert np.max(np.abs(got_lse[finite] - ref["lse"][finite]), initial=0.0) < 1e-3
     # the host-buffer entry point gives the same result
-    rh = _run_step(w, host=True)
-    assert torch.equal(rh["idx"], r["idx"]) and torch.equal(rh["out"], r["out"])
+    for pinned in (True, False):
+        rh = _run_step(w, host=True, pinned=pinned)
+        assert torch.equal(rh["idx"], r["idx"]) and torch.equal(rh["out"], r["out"])
 
 
 def test_k_equals_n_sparse_step_equals_dense_kernel():
