@@ -347,3 +347,44 @@ def test_k_equals_n_sparse_step_equals_dense_kernel():
     ha.ha_dense_decode(shape, w["q"], w["K"], w["V"], w["seq_lens"], w["n_cap"], dense, ws)
     assert_out_close(u16(dense), u16(r["out"]))
     assert r["cnt"].cpu().tolist() == [[1500, 1500], [900, 900]]
+
+
+@pytest.mark.parametrize("reps", [1, 3])     # 8 units: single fused kernel; 24 units: three-kernel path
+def test_step_edge_cases_empty_sequence_budget_above_length_and_no_new_key(reps):
+    # one launch covers: an empty sequence, a one-token sequence, k > n, k = 0; then the same without a new key
+    cfg = wl.Config("edges", 53, 4 * reps, [0, 1, 37, 2500] * reps, 64, 0.0, n_q_heads=8, n_kv_heads=2)
+    w = wl.make_workload(cfg, DEV)
+    w["ks"] = [5, 9, 64, 0] * reps
+    w["k_per_seq"] = torch.tensor(w["ks"], dtype=torch.int32, device=DEV)
+    w["k_max"] = 64
+    B, Hq, Hkv = 4 * reps, 8, 2
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
+    ws = ha.alloc_workspace(shape, w["n_cap"], w["k_max"])
+    mq, mk = ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"])
+    Kc = oracle_key_codes(w["K"], w["map_k"], w["lens"])
+    for with_key in (True, False):
+        kc = torch.from_numpy(np.pad(Kc, ((0, 0), (0, 0), (0, (-Kc.shape[2]) % 4))).view(np.int32)).to(DEV)
+        if with_key:
+            for b in range(B):
+                if w["lens"][b] > 0:
+                    kc[b, :, w["lens"][b] - 1] = 0x0BADF00D
+        qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+        idx = torch.full((B, Hkv, 64), 7, dtype=torch.int32, device=DEV)
+        cnt = torch.full((B, Hkv), 7, dtype=torch.int32, device=DEV)
+        out = torch.full((B, Hq, 128), 3.0, dtype=torch.bfloat16, device=DEV)
+        lse = torch.zeros(B, Hq, device=DEV)
+        ha.ha_sparse_decode(shape, mq, mk if with_key else None, w["q"], w["k_new"] if with_key else None, w["K"], w["V"],
+                            kc, w["seq_lens"], w["k_per_seq"], 0, w["n_cap"], 64, qc, idx, cnt, out, ws, lse=lse)
+        torch.cuda.synchronize()
+        ref = oracle.decode_step(u16(w["q"]), u16(w["k_new"]) if with_key else None, u16(w["K"]), u16(w["V"]), Kc.copy(),
+                                 wl.mapping_numpy(w["map_q"]), wl.mapping_numpy(w["map_k"]), w["lens"], w["ks"],
+                                 sm_scale=w["sm_scale"])
+        assert np.array_equal(codes_np(kc)[:, :, :Kc.shape[2]], Kc)          # appended slots rewritten (or untouched)
+        assert np.array_equal(codes_np(qc), ref["qcodes"])
+        assert np.array_equal(cnt.cpu().numpy(), ref["count"]) and cnt.cpu().numpy().tolist() == [[0, 0], [1, 1], [37, 37], [0, 0]] * reps
+        assert np.array_equal(idx.cpu().numpy(), ref["idx"])
+        assert_out_close(u16(out), ref["out"])
+        got = lse.cpu().numpy().astype(np.float64)
+        fin = np.isfinite(ref["lse"])
+        assert np.array_equal(np.isneginf(got), ~fin) and np.max(np.abs(got[fin] - ref["lse"][fin]), initial=0.0) < 1e-3
+        assert not u16(out)[0::4].any() and not u16(out)[3::4].any()          # empty selections give zeros
