@@ -359,10 +359,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         }
     }
     __syncthreads();
-    if (tid < kD) {   // this CTA's state goes into slot `rank` of CTA 0's shared memory
-        const int d = tid;
+    {   // this CTA's state goes into slot `rank` of CTA 0's shared memory; the two thread halves share the heads
+        const int d = tid & (kD - 1), hsel = tid >> 7;
 #pragma unroll
         for (int j = 0; j < G; ++j) {
+            if (G > 1 && (j & 1) != hsel) continue;
+            if (G == 1 && hsel != 0) continue;
             float M = s_m[0][j];
 #pragma unroll
             for (int w = 1; w < kFusedWarps; ++w) M = fmaxf(M, s_m[w][j]);
@@ -383,10 +385,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         }
     }
     cluster_sync_all();   // #4: all eight states have landed in CTA 0
-    if (rank == 0 && tid < kD) {
-        const int d = tid;
+    if (rank == 0) {
+        const int d = tid & (kD - 1), hsel = tid >> 7;
 #pragma unroll
         for (int j = 0; j < G; ++j) {
+            if (G > 1 && (j & 1) != hsel) continue;
+            if (G == 1 && hsel != 0) continue;
             float M = -CUDART_INF_F;
 #pragma unroll
             for (int r = 0; r < kFusedCS; ++r) M = fmaxf(M, part_ml[(r * G + j) * 2]);
