@@ -377,19 +377,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
     if (bad) atomicOr(a.status, HA_DEV_BAD_INDEX);
 }
 
-static int sm_count() {
-    static int cached[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64) dev = 0;
-    if (!cached[dev]) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-        cached[dev] = n;
-    }
-    return cached[dev];
-}
-
 template <int G, bool kGather>
 static cudaError_t launch_attn_t(const AttnArgs &args, int grid, size_t smem, cudaStream_t st) {
     static bool done[64] = {};   // opt in to the ring's shared memory once per device

@@ -117,8 +117,23 @@ struct EncodeJob {
     const int32_t *slot;     // per-sequence slot (device) or NULL = 0
     int slot_minus_one;      // 1: slot[] holds sequence lengths, write at slot[b] - 1
     int n_heads, heads_per_kv, n_cta;   // n_cta = batch * n_heads / heads_per_kv
+    int batch, cta_per_net;  // filled in by the launcher: sequences, and CTAs that share one network's items
     MapView map;
 };
+
+// Number of SMs of the current device (cached per device).
+inline int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
 
 // ---- launchers (each enqueues kernels on `st` and returns the last CUDA error) ----
 cudaError_t launch_encode_vectors(const EncodeJob &a, const EncodeJob &b, cudaStream_t st);

@@ -1,8 +1,8 @@
 // ENCODE (Eq. 2): signature = packed sign bits of the Section 5.2 feed-forward net
 // 128 -> 128 -> 128 -> 32.  Every output is one fp32 fused-multiply-add chain over ascending
 // input index started from the bias, so the result does not depend on how outputs are spread
-// over threads.  Two kernels: one CTA per vector for the handful of vectors of a decode step
-// (latency-bound), and a token-tiled kernel with the weights held in shared memory for building
+// over threads.  Two kernels: one for the handful of vectors of a decode step (latency-bound), and a
+// token-tiled kernel with the weights held in shared memory for building
 // the signature cache of a whole prompt.
 #include "ha_encode_dev.cuh"
 
@@ -11,37 +11,41 @@ namespace ha {
 
 // ------------------------------------------------------------------ decode-step kernel
 //
-// One CTA per (sequence, network): the G query vectors that share a network (or the one new key)
-// are encoded together, so the 72 KB of weights are fetched once per CTA.  One thread requests the
-// three weight matrices with bulk asynchronous copies (TMA, one mbarrier per matrix) at kernel
-// entry, before the programmatic-launch wait: the fetch overlaps the preceding kernels and costs no
-// issue slots; each layer starts as soon as its matrix has landed.  Thread (o, half) runs the fma
-// chain of output o for one half of the CTA's vectors; two warps per scheduler hide the
-// shared-memory latency of each other's chains.
+// The vectors of one network (the queries of a KV head over the whole batch, or the appended keys)
+// are cut into items of NV vectors.  A CTA belongs to one network, fetches its 72 KB of weights
+// once and encodes the items part, part + P, ... of that network.  A step of few vectors uses
+// NV = 1 and one item per CTA (the chains of different vectors run on different SMs); a large batch
+// uses items of up to 8 vectors and, beyond two waves of CTAs, several items per CTA, so that the
+// weight traffic does not grow with the number of vectors.
+// One thread requests the three weight matrices with bulk asynchronous copies (TMA, one mbarrier
+// per matrix) at kernel entry, before the programmatic-launch wait: the fetch overlaps the
+// preceding kernels and costs no issue slots; each layer starts as soon as its matrix has landed.
+// Thread o runs the fma chains of output o for every vector of the item.  The layers are bound by
+// shared-memory bandwidth (one 2-byte weight per lane and term), so one warp per scheduler that
+// reuses each weight for all its vectors beats more warps that each re-read the matrix.
 
-constexpr int kVecThreads = 256;
+constexpr int kVecThreads = 128;
 constexpr size_t kVecWeightBytes = (size_t)(kD * kHid + kHid * kHid + kHid * kBits) * 2;
 
 template <int NV>
 __global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, EncodeJob jb) {
-    constexpr int VT = (NV + 1) / 2;   // vectors per thread: half h owns vectors h*VT .. h*VT+VT-1
-    constexpr int NS = 2 * VT;         // vector slots in shared memory (>= NV)
     extern __shared__ __align__(128) unsigned char vec_smem[];
     __shared__ __align__(8) unsigned long long s_bar[3];
     uint16_t *sw1 = reinterpret_cast<uint16_t *>(vec_smem);
     uint16_t *sw2 = sw1 + kD * kHid;
     uint16_t *sw3 = sw2 + kHid * kHid;
-    float *actA = reinterpret_cast<float *>(sw3 + kHid * kBits);   // [NS][128]
-    float *actB = actA + NS * kD;
+    float *actA = reinterpret_cast<float *>(sw3 + kHid * kBits);   // [NV][128]
+    float *actB = actA + NV * kD;
 
     int i = blockIdx.x;
     const bool second = i >= ja.n_cta;
     const EncodeJob &J = second ? jb : ja;
     if (second) i -= ja.n_cta;
-    const int n_nets = J.n_heads / J.heads_per_kv;
-    const int b = i / n_nets, net = i % n_nets;
-    const int nv = J.heads_per_kv;   // <= NV
-    const int tid = threadIdx.x, o = tid & 127, half = tid >> 7;
+    const int P = J.cta_per_net, net = i / P, part = i % P;
+    const int hpk = J.heads_per_kv;
+    const int n_vec = J.batch * hpk;                 // vectors of this network: t -> (b = t / hpk, head net*hpk + t % hpk)
+    const int n_items = (n_vec + NV - 1) / NV;
+    const int tid = threadIdx.x, o = tid;
 
     const uint16_t *g1 = J.map.w1 + (size_t)net * kD * kHid;
     const uint16_t *g2 = J.map.w2 + (size_t)net * kHid * kHid;
@@ -68,19 +72,6 @@ __global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, E
     // wait (sequence lengths, budgets, signatures) is then final, whoever wrote it earlier in the stream.
     pdl_wait();
     pdl_launch_dependents();
-#pragma unroll
-    for (int vv = 0; vv < VT; ++vv) {
-        const int v = half * VT + vv;
-        float xv = 0.0f;   // unused slots are zero rows (their chains are computed and dropped)
-        if (v < nv) {
-            const uint16_t *x = J.x + (long long)b * J.x_sb + (long long)(net * J.heads_per_kv + v) * J.x_sh;
-            xv = bf16_bits_to_float(__ldg(x + o));
-        }
-        actA[v * kD + o] = xv;
-    }
-    int slot = 0;
-    if (J.slot) slot = J.slot[b] - J.slot_minus_one;   // a negative slot skips the sequence (no write below)
-    __syncthreads();   // mbarrier inits and the inputs are visible to every thread
 
     // wait for one weight matrix; if the bulk copy never reports completion, load it the ordinary way
     // (the decision is taken by the whole CTA together, so that the barrier below is never divergent)
@@ -93,42 +84,66 @@ __global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, E
         }
     };
 
-    float z[VT];
-    const float *inA = actA + half * VT * kD, *inB = actB + half * VT * kD;
-    // ---- layer 1
-    weights_ready(0, sw1, g1, kD * kHid);
+    bool first = true;
+    for (int item = part; item < n_items; item += P) {   // CTA-uniform
+        const int t0 = item * NV, nv = min(NV, n_vec - t0);
 #pragma unroll
-    for (int v = 0; v < VT; ++v) z[v] = bias1;
-    vec_layer<VT>(inA, sw1, kHid, o, z);
-#pragma unroll
-    for (int v = 0; v < VT; ++v) actB[(half * VT + v) * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
-    __syncthreads();
-    // ---- layer 2
-    weights_ready(1, sw2, g2, kHid * kHid);
-#pragma unroll
-    for (int v = 0; v < VT; ++v) z[v] = bias2;
-    vec_layer<VT>(inB, sw2, kHid, o, z);
-    // actA was last read in layer 1, which every thread left before the barrier above
-#pragma unroll
-    for (int v = 0; v < VT; ++v) actA[(half * VT + v) * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
-    __syncthreads();
-    // ---- layer 3: warp w encodes vector w, one output bit per lane
-    weights_ready(2, sw3, g3, kHid * kBits);
-    {
-        const int v = tid >> 5, lane = tid & 31;
-        if (v < NS) {   // warp-uniform
-            float z3[1] = {bias3};
-            vec_layer<1>(actA + v * kD, sw3, kBits, lane, z3);
-            const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
-            if (lane == 0 && v < nv && slot >= 0)
-                J.codes[(long long)b * J.c_sb + (long long)(net * J.heads_per_kv + v) * J.c_sh + slot] = code;
+        for (int v = 0; v < NV; ++v) {
+            float xv = 0.0f;   // unused slots are zero rows (their chains are computed and dropped)
+            if (v < nv) {
+                const int t = t0 + v;
+                const uint16_t *x = J.x + (long long)(t / hpk) * J.x_sb + (long long)(net * hpk + t % hpk) * J.x_sh;
+                xv = bf16_bits_to_float(__ldg(x + o));
+            }
+            actA[v * kD + o] = xv;
         }
+        __syncthreads();   // mbarrier inits and the inputs are visible to every thread
+
+        float z[NV];
+        // ---- layer 1
+        if (first) weights_ready(0, sw1, g1, kD * kHid);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) z[v] = bias1;
+        vec_layer<NV>(actA, sw1, kHid, o, z);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) actB[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+        __syncthreads();
+        // ---- layer 2
+        if (first) weights_ready(1, sw2, g2, kHid * kHid);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) z[v] = bias2;
+        vec_layer<NV>(actB, sw2, kHid, o, z);
+        // actA was last read in layer 1, which every thread left before the barrier above
+#pragma unroll
+        for (int v = 0; v < NV; ++v) actA[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+        __syncthreads();
+        // ---- layer 3: one warp per vector, one output bit per lane
+        if (first) weights_ready(2, sw3, g3, kHid * kBits);
+        first = false;
+        {
+            const int warp = tid >> 5, lane = tid & 31;
+#pragma unroll
+            for (int v0 = 0; v0 < NV; v0 += kVecThreads / 32) {
+                const int v = v0 + warp;
+                if (v < nv) {   // warp-uniform
+                    float z3[1] = {bias3};
+                    vec_layer<1>(actA + v * kD, sw3, kBits, lane, z3);
+                    const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
+                    const int t = t0 + v, b = t / hpk;
+                    int slot = 0;
+                    if (J.slot) slot = J.slot[b] - J.slot_minus_one;   // a negative slot skips the sequence
+                    if (lane == 0 && slot >= 0)
+                        J.codes[(long long)b * J.c_sb + (long long)(net * hpk + t % hpk) * J.c_sh + slot] = code;
+                }
+            }
+        }
+        __syncthreads();   // layer 3 has read actA before the next item overwrites it
     }
 }
 
 template <int NV>
 static cudaError_t launch_vec_t(const EncodeJob &a, const EncodeJob &b, cudaStream_t st) {
-    constexpr size_t smem = kVecWeightBytes + (size_t)2 * (2 * ((NV + 1) / 2)) * kD * 4;
+    constexpr size_t smem = kVecWeightBytes + (size_t)2 * NV * kD * 4;
     static bool done[64] = {};   // opt in to > 48 KB of shared memory once per device
     int dev = 0;
     cudaGetDevice(&dev);
@@ -143,14 +158,39 @@ static cudaError_t launch_vec_t(const EncodeJob &a, const EncodeJob &b, cudaStre
     return cudaGetLastError();
 }
 
-cudaError_t launch_encode_vectors(const EncodeJob &a, const EncodeJob &b, cudaStream_t st) {
-    if (a.n_cta + b.n_cta <= 0) return cudaSuccess;
-    const int nv = max(a.n_cta > 0 ? a.heads_per_kv : 1, b.n_cta > 0 ? b.heads_per_kv : 1);
-    if (nv <= 1) return launch_vec_t<1>(a, b, st);
-    if (nv <= 2) return launch_vec_t<2>(a, b, st);
-    if (nv <= 4) return launch_vec_t<4>(a, b, st);
-    if (nv <= 8) return launch_vec_t<8>(a, b, st);
-    return cudaErrorInvalidValue;
+// `a` and `b` arrive with n_cta = the number of (sequence, network) pairs (0 = no such job); the item
+// width and the CTAs per network are chosen here.
+cudaError_t launch_encode_vectors(const EncodeJob &a_in, const EncodeJob &b_in, cudaStream_t st) {
+    if (a_in.n_cta + b_in.n_cta <= 0) return cudaSuccess;
+    EncodeJob job[2] = {a_in, b_in};
+    int nets[2], vec_per_net[2];
+    long long vectors = 0;
+    for (int j = 0; j < 2; ++j) {
+        EncodeJob &J = job[j];
+        nets[j] = (J.n_cta > 0) ? J.n_heads / J.heads_per_kv : 0;
+        J.batch = (J.n_cta > 0) ? J.n_cta / nets[j] : 0;
+        vec_per_net[j] = J.batch * J.heads_per_kv;
+        vectors += (long long)nets[j] * vec_per_net[j];
+    }
+    const long long room = 2LL * sm_count();   // two CTAs (76 KB of shared memory each) fit one SM
+    int nv = 1;
+    auto items = [&](int width) {
+        long long n = 0;
+        for (int j = 0; j < 2; ++j) n += (long long)nets[j] * ((vec_per_net[j] + width - 1) / width);
+        return n;
+    };
+    while (nv < 8 && items(nv) > room) nv *= 2;
+    const long long rounds = (items(nv) + 2 * room - 1) / (2 * room);   // up to two waves of one-item CTAs
+    for (int j = 0; j < 2; ++j) {
+        EncodeJob &J = job[j];
+        const long long it = (vec_per_net[j] + nv - 1) / nv;
+        J.cta_per_net = (int)((it + rounds - 1) / rounds);
+        J.n_cta = nets[j] * J.cta_per_net;
+    }
+    if (nv == 1) return launch_vec_t<1>(job[0], job[1], st);
+    if (nv == 2) return launch_vec_t<2>(job[0], job[1], st);
+    if (nv == 4) return launch_vec_t<4>(job[0], job[1], st);
+    return launch_vec_t<8>(job[0], job[1], st);
 }
 
 // ------------------------------------------------------------------ token-tiled bulk kernel

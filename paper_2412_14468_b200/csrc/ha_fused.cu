@@ -61,22 +61,23 @@ __device__ __forceinline__ void st_dsmem_f32(float *local, uint32_t rank, float 
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
 }
 
-// ENCODE of NV vectors that share one network, by the whole CTA (256 threads: thread (o, half) runs
-// the chains of output o for half of the vectors).  Weights arrive in shared memory through three
-// mbarriers armed by the caller.  Signature v is returned in codes_out[v] (shared memory).
+// ENCODE of NV vectors that share one network by the first 128 threads of the CTA: thread o runs the
+// chains of output o for every vector.  The layers are bound by shared-memory bandwidth, so a second
+// warp per scheduler would only compete for it without shortening any chain.  Weights arrive in
+// shared memory through three mbarriers armed by the caller.  Signature v is returned in codes_out[v]
+// (shared memory).
 template <int NV>
 __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_stride, const MapView &map, int net,
                                              uint16_t *sw1, uint16_t *sw2, uint16_t *sw3, uint32_t bar0, float *actA,
                                              float *actB, uint32_t *codes_out) {
-    constexpr int VT = (NV + 1) / 2, NS = 2 * VT;
-    const int tid = threadIdx.x, o = tid & 127, half = tid >> 7;
+    const int tid = threadIdx.x, o = tid & 127;
+    const bool active = tid < 128;
     const float bias1 = map.b1 ? __ldg(map.b1 + net * kHid + o) : 0.0f;
     const float bias2 = map.b2 ? __ldg(map.b2 + net * kHid + o) : 0.0f;
     const float bias3 = map.b3 ? __ldg(map.b3 + net * kBits + (tid & (kBits - 1))) : 0.0f;
+    if (active) {
 #pragma unroll
-    for (int vv = 0; vv < VT; ++vv) {
-        const int v = half * VT + vv;
-        actA[v * kD + o] = (v < NV) ? bf16_bits_to_float(__ldg(x0 + (long long)v * x_stride + o)) : 0.0f;
+        for (int v = 0; v < NV; ++v) actA[v * kD + o] = bf16_bits_to_float(__ldg(x0 + (long long)v * x_stride + o));
     }
     __syncthreads();
     auto weights_ready = [&](int which, uint16_t *dst, const uint16_t *src, int n_elems) {
@@ -87,29 +88,33 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
             __syncthreads();
         }
     };
-    float z[VT];
+    float z[NV];
     weights_ready(0, sw1, map.w1 + (size_t)net * kD * kHid, kD * kHid);
+    if (active) {
 #pragma unroll
-    for (int v = 0; v < VT; ++v) z[v] = bias1;
-    vec_layer<VT>(actA + half * VT * kD, sw1, kHid, o, z);
+        for (int v = 0; v < NV; ++v) z[v] = bias1;
+        vec_layer<NV>(actA, sw1, kHid, o, z);
 #pragma unroll
-    for (int v = 0; v < VT; ++v) actB[(half * VT + v) * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+        for (int v = 0; v < NV; ++v) actB[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+    }
     __syncthreads();
     weights_ready(1, sw2, map.w2 + (size_t)net * kHid * kHid, kHid * kHid);
+    if (active) {
 #pragma unroll
-    for (int v = 0; v < VT; ++v) z[v] = bias2;
-    vec_layer<VT>(actB + half * VT * kD, sw2, kHid, o, z);
+        for (int v = 0; v < NV; ++v) z[v] = bias2;
+        vec_layer<NV>(actB, sw2, kHid, o, z);
 #pragma unroll
-    for (int v = 0; v < VT; ++v) actA[(half * VT + v) * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+        for (int v = 0; v < NV; ++v) actA[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
+    }
     __syncthreads();
     weights_ready(2, sw3, map.w3 + (size_t)net * kHid * kBits, kHid * kBits);
     {
         const int v = tid >> 5, lane = tid & 31;   // warp v encodes vector v, one output bit per lane
-        if (v < NS) {
+        if (v < NV) {
             float z3[1] = {bias3};
             vec_layer<1>(actA + v * kD, sw3, kBits, lane, z3);
             const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
-            if (lane == 0 && v < NV) codes_out[v] = code;
+            if (lane == 0) codes_out[v] = code;
         }
     }
     __syncthreads();
@@ -158,10 +163,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         c[p] = (p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
     }
     const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&s_bar[0]);
-    // ENCODE roles: CTA r < kQCtas encodes query vectors 2r and 2r+1 (one fma chain per thread), CTA kQCtas
-    // encodes the appended key; the other CTAs only scan
-    constexpr int kQCtas = (G + 1) / 2;
-    constexpr int kQPer = (G >= 2) ? 2 : 1;
+    // ENCODE roles: CTA r < kQCtas encodes kQPer query vectors (one per CTA while the cluster has room),
+    // CTA kQCtas encodes the appended key; the other CTAs only scan
+    constexpr int kQPer = (G < kFusedCS) ? 1 : 2;
+    constexpr int kQCtas = (G + kQPer - 1) / kQPer;
+    static_assert(kQCtas < kFusedCS, "the cluster needs one more CTA for the appended key");
     const bool enc_q = (int)rank < kQCtas, enc_k = ((int)rank == kQCtas) && has_new_key;
     const bool encodes = enc_q || enc_k;
     const MapView &map = enc_q ? a.map_q : a.map_k;

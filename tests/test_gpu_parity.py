@@ -63,6 +63,25 @@ def test_encode_query_side_group_sharing_and_append_slot():
     assert np.all(got == 0x55)
 
 
+@pytest.mark.parametrize("B,Hq,Hkv", [(1, 8, 2), (19, 8, 2), (50, 8, 2), (101, 8, 2), (300, 32, 8), (37, 16, 2), (333, 3, 3)])
+def test_encode_single_token_batches_cover_every_item_width(B, Hq, Hkv):
+    """One vector per head and sequence: small batches run one vector per CTA, larger ones items of 2, 4 or
+    8 vectors (ragged last item), and the largest several items per CTA; all bit-exact."""
+    mp = _mapping(Hkv, 1000 + B)
+    g = torch.Generator(DEV).manual_seed(B)
+    q = torch.randn(B, Hq, 128, device=DEV, generator=g).to(torch.bfloat16)
+    qc = torch.full((B, Hq, 2), 0x33, dtype=torch.int32, device=DEV)
+    slot = torch.ones(B, dtype=torch.int32, device=DEV)
+    slot[B // 2] = -1                                    # this sequence is skipped
+    ha.ha_encode(ha.Mapping(mp), Hq // Hkv, q, qc, slot=slot)
+    got = codes_np(qc)
+    exp = oracle_query_codes(q, mp, Hkv)
+    keep = np.ones(B, bool)
+    keep[B // 2] = False
+    assert np.array_equal(got[keep, :, 1], exp[keep])
+    assert np.all(got[:, :, 0] == 0x33) and np.all(got[~keep] == 0x33)
+
+
 def test_encode_without_biases_and_strided_input():
     H, T = 2, 70
     mp = _mapping(H, 9)
