@@ -13,6 +13,7 @@
 // The scanning kernels request their first signatures before the programmatic-launch wait, so that
 // the fetch overlaps the tail of the preceding kernel; the one signature that the preceding ENCODE
 // may still be writing (the appended token, slot n-1) is re-read after the wait.
+#include <cstdlib>
 #include "ha_score_dev.cuh"
 
 namespace ha {
@@ -241,24 +242,55 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
 
 // ------------------------------------------------------------------ fused single-kernel path
 //
-// For sequences of up to 32768 tokens one thread-block cluster of 8, 4 or 2 CTAs owns a
-// (sequence, KV head) unit: every CTA keeps its slice of the codes in registers, the CTAs exchange
-// their 33-bin histograms through distributed shared memory between two hardware cluster barriers,
-// and each CTA then compacts its own slice straight from registers (scores kept as bytes).  The codes are read from HBM
-// once, there is no histogram round trip through global memory and no second launch.
-// Token order inside a CTA is thread order (a lane owns 4L consecutive tokens), so the prefix sums
-// need one warp-shuffle scan plus one exchange of eight warp totals.
+// For sequences of up to CS * 16384 tokens one thread-block cluster of CS = 8, 4 or 2 CTAs owns a
+// (sequence, KV head) unit: every CTA leaves the scores of its slice in shared memory (one byte per
+// token), the CTAs exchange their 33-bin histograms through distributed shared memory between two
+// hardware cluster barriers, and each CTA then compacts its own slice from those bytes.  The
+// signatures are read from HBM once, there is no histogram round trip through global memory and no
+// second launch.
+// Reading: a warp owns 256*Rb consecutive tokens and reads them in rows of 256 tokens, a lane 8
+// consecutive tokens (one 32-byte sector) per row, so that every request of a warp covers 1 KB of
+// contiguous memory.  Few registers are live (no per-thread score array), so six CTAs share an SM
+// and hide each other's barriers and the latency of the population-count unit, which is the
+// scarce resource here (one quarter-rate instruction per query head and token).
+// Counting: one 32-bit counter per (level, lane), shared by the eight warps and bumped with
+// shared-memory reductions: a lane only meets its own column, so an instruction never conflicts
+// with itself, and nothing waits for a result.
+// Writing: lane l owns the 8*Rb consecutive tokens l*8*Rb .. of its warp's range, so the prefix sums
+// need one warp-shuffle scan plus one exchange of eight warp totals; only flagged tokens are
+// visited, with plain integer arithmetic (the selection never queues behind the scoring for the
+// population-count unit).
 
+// Index of the single set bit of `one_hot`.
+__device__ __forceinline__ int one_hot_index(uint32_t one_hot) {
+    return ((one_hot & 0xaaaaaaaau) ? 1 : 0) | ((one_hot & 0xccccccccu) ? 2 : 0) | ((one_hot & 0xf0f0f0f0u) ? 4 : 0) |
+           ((one_hot & 0xff00ff00u) ? 8 : 0) | ((one_hot & 0xffff0000u) ? 16 : 0);
+}
 
-template <int G, int L, int CS>
-__global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : 4) score_select_cluster_kernel(
+// Visits the flagged tokens among 32 consecutive tokens from `first` on in ascending order; g_run / q_run
+// count the tokens with S > T / S == T seen so far in the whole sequence; r tokens of score T are wanted.
+__device__ __forceinline__ void write_selected32(int32_t *list, int first, uint32_t gt, uint32_t eq, int &g_run,
+                                                 int &q_run, int r) {
+    uint32_t m = gt | eq;
+    while (m) {
+        const uint32_t lb = m & (0u - m);
+        m ^= lb;
+        const int t = first + one_hot_index(lb);
+        if (gt & lb) { list[g_run + min(q_run, r)] = t; ++g_run; }
+        else { if (q_run < r) list[g_run + q_run] = t; ++q_run; }
+    }
+}
+
+constexpr int kClusterMaxRows = 8;   // rows of 8 tokens per lane: a lane's flags fit one 64-bit word each
+
+template <int G, int CS>
+__global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
     const uint32_t *__restrict__ q_codes, const uint32_t *__restrict__ k_codes, long long kc_sb, long long kc_sh,
     const int32_t *__restrict__ seq_lens, int max_seq_len, const int32_t *__restrict__ k_per_seq, int k_uniform,
     int k_max, int Hq, int Hkv, int32_t *__restrict__ idx, long long idx_sb, long long idx_sh,
     int32_t *__restrict__ count, int32_t *__restrict__ hist_out) {
-    // per-warp histograms with one byte counter per (level, lane): a thread only ever touches its own
-    // bytes, so the counting needs no atomics and has no bank conflicts (a thread sees <= 128 tokens)
-    __shared__ __align__(16) unsigned char w_hist[kScanThreads / 32][kBins][32];
+    extern __shared__ __align__(16) unsigned char s_sc[];      // score + 1 of this CTA's tokens (0 = no token)
+    __shared__ __align__(16) uint32_t c_hist[kBins][32];       // counters [level][lane]
     __shared__ int s_hist[kBins + 3];          // this CTA's histogram, read by the whole cluster
     __shared__ int s_tot[kBins], s_bef[kBins];
     __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
@@ -271,70 +303,94 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : 4) score_select_c
     k = max(0, min(k, k_max));
     const int keep = min(k, n);
     const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
-    // The sequence's own length is divided over the CS CTAs (ragged batches stay balanced): a lane owns
-    // 4*Lb consecutive tokens (Lb <= L uint4), a warp 128*Lb, a CTA 1024*Lb; token order = thread order.
-    const int Lb = (n + CS * 1024 - 1) / (CS * 1024);
-    const int wbase = ((int)rank * 1024 + warp * 128 + lane * 4) * Lb;
-    constexpr int kPre = (L < 4) ? L : 4;      // uint4 loads issued before the programmatic-launch wait
+    // The sequence's own length is divided over the CS CTAs (ragged batches stay balanced): Rb rows per
+    // lane, a warp owns the 256*Rb tokens from wb on, a CTA 2048*Rb; row p of a lane is
+    // wb + 256 p + 8 lane .. + 7.
+    const int Rb = (n + CS * 2048 - 1) / (CS * 2048);
+    const int wl = warp * 256 * Rb;                    // the warp's first token inside the CTA's slice
+    const int wb = (int)rank * 2048 * Rb + wl;
 
-    uint4 c[kPre];
-#pragma unroll
-    for (int p = 0; p < kPre; ++p) {
-        const int base = wbase + p * 4;
-        c[p] = (p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
-    }
-    for (int i = tid; i < (kScanThreads / 32) * kBins * 32 / 4; i += kScanThreads)
-        reinterpret_cast<uint32_t *>(&w_hist[0][0][0])[i] = 0u;
+    auto load_row = [&](int p, uint4 &lo, uint4 &hi, bool early) {
+        const int t = wb + p * 256 + lane * 8;
+        if (p < Rb && t + 8 <= n) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(row + t);
+            if (early) { lo = __ldg(src); hi = __ldg(src + 1); }
+            else { lo = __ldcg(src); hi = __ldcg(src + 1); }
+        } else {
+            lo = (p < Rb && t < n) ? load_codes4(row, t, n) : make_uint4(0, 0, 0, 0);
+            hi = (p < Rb && t + 4 < n) ? load_codes4(row, t + 4, n) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    uint4 c[4];   // two rows
+    load_row(0, c[0], c[1], true);
+    load_row(1, c[2], c[3], true);
+    for (int i = tid; i < kBins * 32 / 4; i += kScanThreads)
+        reinterpret_cast<uint4 *>(&c_hist[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
     if (tid < kBins + 3) s_hist[tid] = 0;
     pdl_launch_dependents();
     pdl_wait();
+    {   // the signature that the preceding ENCODE may just have written: re-read by the one lane that holds it
+        const int e_last = (n - 1) - wb;
+        if (e_last >= 0 && e_last < 512 && e_last < 256 * Rb && ((e_last & 255) >> 3) == lane) {
 #pragma unroll
-    for (int p = 0; p < kPre; ++p) patch_token(c[p], wbase + p * 4, n - 1, row);
+            for (int j = 0; j < 2; ++j) {
+                patch_token(c[2 * j], wb + j * 256 + lane * 8, n - 1, row);
+                patch_token(c[2 * j + 1], wb + j * 256 + lane * 8 + 4, n - 1, row);
+            }
+        }
+    }
     uint32_t qc[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
     __syncthreads();
 
-    // ---- scores (kept as four score+1 bytes per register; 0 marks "no token") and this CTA's histogram
-    uint32_t sc[L];
-    unsigned char *my = &w_hist[warp][0][lane] - 32;   // indexed by the score+1 byte
+    // ---- scores (four score+1 bytes per word) and this CTA's histogram.  The counter of score s sits
+    // (32 - s) rows below the lane's counter of level 32, so the address comes straight from the
+    // Hamming distance 32 - s.
+    const uint32_t top = (uint32_t)__cvta_generic_to_shared(&c_hist[kBins - 1][lane]);
+    auto bump = [&](int ham) { asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(top - (uint32_t)ham * 128u) : "memory"); };
+    auto hamming = [&](uint32_t code) {
+        int h = __popc(code ^ qc[0]);
 #pragma unroll
-    for (int p0 = 0; p0 < L; p0 += kPre) {
-        if (p0 > 0) {   // later batches of codes are streamed through the same registers
-#pragma unroll
-            for (int p = 0; p < kPre; ++p) {
-                const int base = wbase + (p0 + p) * 4;
-                c[p] = (p0 + p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
-                patch_token(c[p], base, n - 1, row);
-            }
+        for (int j = 1; j < G; ++j) h = min(h, __popc(code ^ qc[j]));
+        return h;
+    };
+    auto score_word = [&](const uint4 &cw, int t) -> uint32_t {
+        const int h0 = hamming(cw.x), h1 = hamming(cw.y), h2 = hamming(cw.z), h3 = hamming(cw.w);
+        // bytes 33 - h = score + 1; no byte borrows because h <= 32
+        uint32_t s4 = 0x21212121u - ((uint32_t)h0 | ((uint32_t)h1 << 8) | ((uint32_t)h2 << 16) | ((uint32_t)h3 << 24));
+        if (t + 4 <= n) {
+            bump(h0); bump(h1); bump(h2); bump(h3);
+        } else {
+            if (t + 0 < n) bump(h0); else s4 &= 0xffffff00u;   // zero byte: no token
+            if (t + 1 < n) bump(h1); else s4 &= 0xffff00ffu;
+            if (t + 2 < n) bump(h2); else s4 &= 0xff00ffffu;
+            if (t + 3 < n) bump(h3); else s4 &= 0x00ffffffu;
+        }
+        return s4;
+    };
+    for (int p0 = 0; p0 < Rb; p0 += 2) {   // CTA-uniform
+        if (p0 > 0) {
+            load_row(p0, c[0], c[1], false);
+            load_row(p0 + 1, c[2], c[3], false);
         }
 #pragma unroll
-        for (int p = 0; p < kPre; ++p) {
-            const int base = wbase + (p0 + p) * 4;
-            uint32_t s4 = scores4<G>(c[p], qc);
-            if (p0 + p < Lb && base + 3 < n) {       // whole uint4 inside the sequence: no per-token checks
-                my[(s4 & 0xffu) * 32] += 1;
-                my[((s4 >> 8) & 0xffu) * 32] += 1;
-                my[((s4 >> 16) & 0xffu) * 32] += 1;
-                my[(s4 >> 24) * 32] += 1;
-            } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (p0 + p < Lb && base + e < n) my[((s4 >> (8 * e)) & 0xffu) * 32] += 1;
-                    else s4 &= ~(0xffu << (8 * e));   // zero byte: no token
+        for (int j = 0; j < 2; ++j) {
+            const int p = p0 + j, t = wb + p * 256 + lane * 8;
+            if (p < Rb) {
+                uint2 w;
+                w.x = score_word(c[2 * j], t);
+                w.y = score_word(c[2 * j + 1], t + 4);
+                *reinterpret_cast<uint2 *>(s_sc + wl + p * 256 + lane * 8) = w;
             }
-            sc[p0 + p] = s4;
         }
     }
     __syncthreads();
-    // fold the byte counters: one (level, warp) row of 32 bytes per thread
-    for (int i = tid; i < kBins * (kScanThreads / 32); i += kScanThreads) {
-        const int bin = i >> 3, w = i & 7;
-        const uint4 *rowp = reinterpret_cast<const uint4 *>(&w_hist[w][bin][0]);
-        const uint4 a0 = rowp[0], a1 = rowp[1];
-        const int s = (int)(__vsadu4(a0.x, 0u) + __vsadu4(a0.y, 0u) + __vsadu4(a0.z, 0u) + __vsadu4(a0.w, 0u) +
-                            __vsadu4(a1.x, 0u) + __vsadu4(a1.y, 0u) + __vsadu4(a1.z, 0u) + __vsadu4(a1.w, 0u));
-        if (s) atomicAdd(&s_hist[bin], s);
+    // fold the counters: eight threads per level, four counters each
+    for (int i = tid; i < kBins * 8; i += kScanThreads) {
+        const uint4 v = reinterpret_cast<const uint4 *>(&c_hist[i >> 3][0])[i & 7];
+        const uint32_t ssum = (v.x + v.y) + (v.z + v.w);
+        if (ssum) atomicAdd(&s_hist[i >> 3], (int)ssum);
     }
     cluster_sync_all();   // every CTA's histogram is complete and visible cluster-wide
 
@@ -373,15 +429,24 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : 4) score_select_c
     }
     if (keep == 0) { cluster_wait(); return; }
 
-    // ---- counts of (S > T, S == T) per thread, packed in 16-bit halves
+    // ---- flags "S > T" / "S == T" of the lane's 8*Rb consecutive tokens (bit i = token first + i)
     const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
-    int tot_packed = 0;
+    const int first_l = wl + 8 * Rb * lane;
+    uint32_t gt_lo = 0u, gt_hi = 0u, eq_lo = 0u, eq_hi = 0u;
 #pragma unroll
-    for (int p = 0; p < L; ++p) {
-        uint32_t gt, eq;
-        flags4(sc[p], T4, gt, eq);
-        tot_packed += __popc(gt) | (__popc(eq) << 16);
+    for (int j = 0; j < kClusterMaxRows; ++j) {
+        if (j < Rb) {
+            const uint2 w = *reinterpret_cast<const uint2 *>(s_sc + first_l + 8 * j);
+            uint32_t gt0, eq0, gt1, eq1;
+            flags4(w.x, T4, gt0, eq0);
+            flags4(w.y, T4, gt1, eq1);
+            const uint32_t gb = flags_to_nibble(gt0) | (flags_to_nibble(gt1) << 4);
+            const uint32_t eb = flags_to_nibble(eq0) | (flags_to_nibble(eq1) << 4);
+            if (j < 4) { gt_lo |= gb << (8 * j); eq_lo |= eb << (8 * j); }
+            else { gt_hi |= gb << (8 * (j - 4)); eq_hi |= eb << (8 * (j - 4)); }
+        }
     }
+    const int tot_packed = (__popc(gt_lo) + __popc(gt_hi)) | ((__popc(eq_lo) + __popc(eq_hi)) << 16);
     int winc = tot_packed;   // inclusive scan over the lanes of the per-lane totals
 #pragma unroll
     for (int dd = 1; dd < 32; dd <<= 1) {
@@ -395,55 +460,27 @@ __global__ void __launch_bounds__(kScanThreads, (L <= 4) ? 6 : 4) score_select_c
     for (int w = 0; w < kScanThreads / 32; ++w) {
         if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
     }
-    // ---- positions: the lane's tokens are consecutive, so one exclusive prefix per lane is enough
-    {
+    if (tot_packed != 0) {
         const int excl = winc - tot_packed;
-        int gt_lt = run_gt + (excl & 0xffff);
-        int eq_lt = run_eq + (int)((unsigned)excl >> 16);
-        if (tot_packed != 0) {
-#pragma unroll
-            for (int p = 0; p < L; ++p) {
-                uint32_t gt, eq;
-                flags4(sc[p], T4, gt, eq);
-                if ((gt | eq) == 0u) continue;
-                const int base = wbase + p * 4;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if ((gt >> (8 * e + 7)) & 1u) {
-                        out[gt_lt + min(eq_lt, r)] = base + e;
-                        ++gt_lt;
-                    } else if ((eq >> (8 * e + 7)) & 1u) {
-                        if (eq_lt < r) out[gt_lt + eq_lt] = base + e;
-                        ++eq_lt;
-                    }
-                }
-            }
-        }
+        int g_run = run_gt + (excl & 0xffff);
+        int q_run = run_eq + (int)((unsigned)excl >> 16);
+        const int first = (int)rank * 2048 * Rb + first_l;
+        write_selected32(out, first, gt_lo, eq_lo, g_run, q_run, r);
+        write_selected32(out, first + 32, gt_hi, eq_hi, g_run, q_run, r);
     }
     cluster_wait();
 }
 
-template <int G, int L, int CS>
-static cudaError_t launch_cluster_t(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes,
+template <int G, int CS>
+static cudaError_t launch_cluster_t(int rows, int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes,
                                     long long kc_sb, long long kc_sh, const int32_t *seq_lens,
                                     const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max, int32_t *idx,
                                     long long idx_sb, long long idx_sh, int32_t *count, int32_t *hist_out,
                                     cudaStream_t st) {
-    if (CS > 8) {   // clusters of 16 CTAs need an opt-in, once per device
-        static bool done[64] = {};
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (dev >= 0 && dev < 64 && !done[dev]) {
-            cudaError_t e = cudaFuncSetAttribute(score_select_cluster_kernel<G, L, CS>,
-                                                 cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-            if (e != cudaSuccess) return e;
-            done[dev] = true;
-        }
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CS, Hkv, B);
     cfg.blockDim = dim3(kScanThreads);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = (size_t)rows * 2048;   // one score byte per token of the CTA's slice (<= 16 KB)
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -454,7 +491,7 @@ static cudaError_t launch_cluster_t(int B, int Hq, int Hkv, const uint32_t *q_co
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, score_select_cluster_kernel<G, L, CS>, q_codes, k_codes, kc_sb, kc_sh,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, score_select_cluster_kernel<G, CS>, q_codes, k_codes, kc_sb, kc_sh,
                                        seq_lens, max_seq_len, k_per_seq, k_uniform, k_max, Hq, Hkv, idx, idx_sb, idx_sh,
                                        count, hist_out);
     if (e != cudaSuccess) return e;
@@ -471,28 +508,19 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
     if (max_seq_len <= kClusterMaxSeq) {
         // Fused path: one cluster per unit.  Cluster size: the largest of 8, 4, 2 whose grid still fits
         // the GPU in one wave (about six 256-thread CTAs per SM), so that small batches get the most
-        // parallelism per sequence and large batches the most work per cluster barrier; a thread then
-        // holds L = ceil(n / (CS * 1024)) uint4 of signatures (L <= 16).
-        const int units = B * Hkv, one_wave = 6 * 148;
+        // parallelism per sequence and large batches the most work per cluster barrier; a lane then
+        // holds R = ceil(n / (CS * 2048)) rows of 8 tokens (R <= 8).
+        const int units = B * Hkv, one_wave = 6 * sm_count();
         int cs = 8;
         while (cs > 2 && units * cs > one_wave) cs >>= 1;
-        while ((max_seq_len + cs * 1024 - 1) / (cs * 1024) > 16) cs <<= 1;   // keep L <= 16
-        const int per = (max_seq_len + cs * 1024 - 1) / (cs * 1024);
-#define HA_CL(LL, CSZ)                                                                                              \
-    return launch_cluster_t<G, LL, CSZ>(B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform, \
-                                        max_seq_len, k_max, idx, idx_sb, idx_sh, count, hist_out, st)
-#define HA_CL_L(CSZ)               \
-    do {                           \
-        if (per <= 1) HA_CL(1, CSZ);  \
-        if (per <= 2) HA_CL(2, CSZ);  \
-        if (per <= 4) HA_CL(4, CSZ);  \
-        if (per <= 8) HA_CL(8, CSZ);  \
-        HA_CL(16, CSZ);            \
-    } while (0)
-        if (cs == 8) HA_CL_L(8);
-        if (cs == 4) HA_CL_L(4);
-        HA_CL_L(2);
-#undef HA_CL_L
+        while ((max_seq_len + cs * 2048 - 1) / (cs * 2048) > kClusterMaxRows) cs <<= 1;
+        const int rows = max(1, (max_seq_len + cs * 2048 - 1) / (cs * 2048));
+#define HA_CL(CSZ)                                                                                                    \
+    return launch_cluster_t<G, CSZ>(rows, B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform, \
+                                    max_seq_len, k_max, idx, idx_sb, idx_sh, count, hist_out, st)
+        if (cs == 8) HA_CL(8);
+        if (cs == 4) HA_CL(4);
+        HA_CL(2);
 #undef HA_CL
     }
     const int chunk_tokens = chunk_tokens_for(B * Hkv, max_seq_len);

@@ -15,13 +15,46 @@ from . import binding as ha
 from . import workloads as wl
 
 
+def score_only(args):
+    cfg = wl.CONFIGS[args.config]
+    B = args.batch if args.batch is not None else cfg.batch
+    n, k = cfg.n, cfg.k
+    assert n is not None, "score-only runs need a config with one fixed length"
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    Hq, Hkv = cfg.n_q_heads, cfg.n_kv_heads
+    g = torch.Generator(dev).manual_seed(wl.BASE_SEED + 77)
+    kc = torch.randint(-2**31, 2**31 - 1, (B, Hkv, n), dtype=torch.int32, device=dev, generator=g)
+    qc = torch.randint(-2**31, 2**31 - 1, (B, Hq), dtype=torch.int32, device=dev, generator=g)
+    shape = ha.make_shape(B, Hq, Hkv, 1.0)
+    ws = ha.alloc_workspace(shape, n, k, device=dev)
+    lens = torch.full((B,), n, dtype=torch.int32, device=dev)
+    idx = torch.zeros(B, Hkv, k, dtype=torch.int32, device=dev)
+    cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+    for s in range(args.steps):
+        _ = int(flush.sum())
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ha.ha_score_topk(shape, qc, kc, lens, None, k, n, k, idx, cnt, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        print(f"step {s}: {e0.elapsed_time(e1) * 1e3:.1f} us (plain launch, L2 flushed)")
+    print("signature bytes per step:", B * Hkv * n * 4)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="c3")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--dense", action="store_true", help="also run the dense comparator each step")
+    ap.add_argument("--score-only", action="store_true",
+                    help="SCORE + TOPK alone on random signatures (no K/V allocated: large batches stay small)")
     args = ap.parse_args()
+    if args.score_only:
+        return score_only(args)
     cfg = wl.CONFIGS[args.config]
     if args.batch is not None:
         cfg = dataclasses.replace(cfg, batch=args.batch)
