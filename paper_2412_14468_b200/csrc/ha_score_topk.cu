@@ -261,6 +261,12 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
 // visited, with plain integer arithmetic (the selection never queues behind the scoring for the
 // population-count unit).
 
+// Bits 7, 15, 23, 31 of x gathered into a nibble (bit e = bit 7 of byte e).  The four partial products
+// land on distinct bit positions, so the multiplication carries nothing into bits 28..31.
+__device__ __forceinline__ uint32_t high_bits_to_nibble(uint32_t x) {
+    return ((x & 0x80808080u) * 0x00204081u) >> 28;
+}
+
 // Index of the single set bit of `one_hot`.
 __device__ __forceinline__ int one_hot_index(uint32_t one_hot) {
     return ((one_hot & 0xaaaaaaaau) ? 1 : 0) | ((one_hot & 0xccccccccu) ? 2 : 0) | ((one_hot & 0xf0f0f0f0u) ? 4 : 0) |
@@ -355,11 +361,11 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
         for (int j = 1; j < G; ++j) h = min(h, __popc(code ^ qc[j]));
         return h;
     };
-    auto score_word = [&](const uint4 &cw, int t) -> uint32_t {
+    auto score_word = [&](const uint4 &cw, int t, bool whole_row) -> uint32_t {
         const int h0 = hamming(cw.x), h1 = hamming(cw.y), h2 = hamming(cw.z), h3 = hamming(cw.w);
         // bytes 33 - h = score + 1; no byte borrows because h <= 32
         uint32_t s4 = 0x21212121u - ((uint32_t)h0 | ((uint32_t)h1 << 8) | ((uint32_t)h2 << 16) | ((uint32_t)h3 << 24));
-        if (t + 4 <= n) {
+        if (whole_row) {
             bump(h0); bump(h1); bump(h2); bump(h3);
         } else {
             if (t + 0 < n) bump(h0); else s4 &= 0xffffff00u;   // zero byte: no token
@@ -378,9 +384,10 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
         for (int j = 0; j < 2; ++j) {
             const int p = p0 + j, t = wb + p * 256 + lane * 8;
             if (p < Rb) {
+                const bool whole_row = t + 8 <= n;
                 uint2 w;
-                w.x = score_word(c[2 * j], t);
-                w.y = score_word(c[2 * j + 1], t + 4);
+                w.x = score_word(c[2 * j], t, whole_row);
+                w.y = score_word(c[2 * j + 1], t + 4, whole_row);
                 *reinterpret_cast<uint2 *>(s_sc + wl + p * 256 + lane * 8) = w;
             }
         }
@@ -430,22 +437,23 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
     if (keep == 0) { cluster_wait(); return; }
 
     // ---- flags "S > T" / "S == T" of the lane's 8*Rb consecutive tokens (bit i = token first + i)
+    // Per byte b = score + 1 (0 = no token): b + 127 - (T+1) sets bit 7 iff score > T, b + 128 - (T+1) iff
+    // score >= T (no byte sum reaches 256); high_bits_to_nibble gathers the four bit-7 flags of a word.
     const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
+    const uint32_t c_gt = 0x7f7f7f7fu - T4, c_ge = 0x80808080u - T4;
     const int first_l = wl + 8 * Rb * lane;
-    uint32_t gt_lo = 0u, gt_hi = 0u, eq_lo = 0u, eq_hi = 0u;
+    uint32_t gt_lo = 0u, gt_hi = 0u, ge_lo = 0u, ge_hi = 0u;
 #pragma unroll
     for (int j = 0; j < kClusterMaxRows; ++j) {
         if (j < Rb) {
             const uint2 w = *reinterpret_cast<const uint2 *>(s_sc + first_l + 8 * j);
-            uint32_t gt0, eq0, gt1, eq1;
-            flags4(w.x, T4, gt0, eq0);
-            flags4(w.y, T4, gt1, eq1);
-            const uint32_t gb = flags_to_nibble(gt0) | (flags_to_nibble(gt1) << 4);
-            const uint32_t eb = flags_to_nibble(eq0) | (flags_to_nibble(eq1) << 4);
-            if (j < 4) { gt_lo |= gb << (8 * j); eq_lo |= eb << (8 * j); }
-            else { gt_hi |= gb << (8 * (j - 4)); eq_hi |= eb << (8 * (j - 4)); }
+            const uint32_t gb = high_bits_to_nibble(w.x + c_gt) | (high_bits_to_nibble(w.y + c_gt) << 4);
+            const uint32_t eb = high_bits_to_nibble(w.x + c_ge) | (high_bits_to_nibble(w.y + c_ge) << 4);
+            if (j < 4) { gt_lo |= gb << (8 * j); ge_lo |= eb << (8 * j); }
+            else { gt_hi |= gb << (8 * (j - 4)); ge_hi |= eb << (8 * (j - 4)); }
         }
     }
+    const uint32_t eq_lo = ge_lo ^ gt_lo, eq_hi = ge_hi ^ gt_hi;   // score > T implies score >= T
     const int tot_packed = (__popc(gt_lo) + __popc(gt_hi)) | ((__popc(eq_lo) + __popc(eq_hi)) << 16);
     int winc = tot_packed;   // inclusive scan over the lanes of the per-lane totals
 #pragma unroll
