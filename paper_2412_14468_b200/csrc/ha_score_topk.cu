@@ -5,7 +5,7 @@
 // above T plus the first r tokens at T in index order, written in ascending token order.
 //
 // Two implementations share the arithmetic:
-//  * sequences of up to 32768 tokens: ONE kernel, a thread-block cluster per (sequence, KV head)
+//  * sequences of up to 131072 tokens: ONE kernel, a thread-block cluster per (sequence, KV head)
 //    (score_select_cluster_kernel, second half of this file);
 //  * longer sequences: two kernels over chunks of the sequence, with the per-chunk histograms and
 //    one score byte per token passed through the workspace (scan_score_kernel, select_kernel).
@@ -20,7 +20,7 @@ namespace ha {
 
 constexpr int kScanThreads = 256;
 constexpr int kPassTokens = kScanThreads * 16;   // four uint4 per thread
-constexpr int kClusterMaxSeq = 32768;            // longest sequence the fused cluster kernel takes
+constexpr int kClusterMaxSeq = 8 * 8 * 2048;     // longest sequence the cluster kernel takes (8 CTAs x 8 rows x 2048 tokens)
 
 // ------------------------------------------------------------------ long-sequence path (two kernels)
 
