@@ -349,7 +349,7 @@ def main():
             "ha_gather_attn (attn_kernel<4,true>)": {"algorithmic_bytes": gather_bytes, "us": g_us,
                                                       "achieved": gather_bytes / (g_us * 1e-6) / 1e9,
                                                       "frac": gather_bytes / (g_us * 1e-6) / 1e9 / peak, "traffic": 4302000},
-            "ha_score_topk (score_select_cluster_kernel<4,4,8>)": {"algorithmic_bytes": scan_bytes, "us": parts["ha_score_topk"],
+            "ha_score_topk (score_select_cluster_kernel<4,8>)": {"algorithmic_bytes": scan_bytes, "us": parts["ha_score_topk"],
                                                                     "achieved": scan_bytes / (parts["ha_score_topk"] * 1e-6) / 1e9},
             "ha_encode[q] (encode_vec_kernel<4>)": {"us": parts["ha_encode[q]"]},
         },
