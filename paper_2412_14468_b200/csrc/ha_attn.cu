@@ -409,6 +409,12 @@ static cudaError_t launch_attn_g(bool gather, const AttnArgs &args_in, cudaStrea
         // a CTA count that is a multiple of the unit count lets equal-length lists split at CTA borders,
         // so that no CTA pays a second prologue and merge in the middle of its range
         if (args.n_units <= grid) grid = grid / args.n_units * args.n_units;
+        else {
+            // more units than CTAs: m whole units per CTA (no unit is split, so nothing is published and
+            // merged through global memory) when that still fills most of the CTA slots
+            const int m = (args.n_units + grid - 1) / grid;
+            if (args.n_units % m == 0 && (long long)(args.n_units / m) * 5 >= (long long)grid * 4) grid = args.n_units / m;
+        }
         smem += (size_t)(args.n_units + 1) * 4;
     } else {
         args.balanced = 0;
