@@ -125,11 +125,13 @@ def test_full_size_config_matches_oracle(cfg_name):
             assert max_abs_diff_bf16(u16(dense)[0, h], eo) <= OUT_TOL
 
 
-def test_many_units_take_the_one_cta_per_unit_path():
-    # more than 1024 (sequence, KV head) units: the attention kernel maps one CTA to each unit
-    cfg = wl.Config("many", 60, 130, [200 + 3 * i for i in range(130)], None, 0.02, n_q_heads=16, n_kv_heads=8, sparsity=4)
+@pytest.mark.parametrize("B", [130, 74, 50])
+def test_many_units(B):
+    # 130 sequences: more than 1024 (sequence, KV head) units, the attention kernel maps one CTA to each unit;
+    # 74: twice as many units as CTA slots, whole units per CTA; 50: more units than CTAs, units split over CTAs
+    cfg = wl.Config("many", 60 + B, B, [200 + 3 * i for i in range(B)], None, 0.02, n_q_heads=16, n_kv_heads=8, sparsity=4)
     w = wl.make_workload(cfg, DEV)
-    B, Hq, Hkv = 130, 16, 8
+    Hq, Hkv = 16, 8
     shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
     ws = ha.alloc_workspace(shape, w["n_cap"], w["k_max"])
     mq, mk = ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"])
