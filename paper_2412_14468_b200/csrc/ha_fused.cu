@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     float *part_acc = part_ml + kFusedCS * kMaxGroup * 2;                                   // [CS][G][128]
     __shared__ __align__(8) unsigned long long s_bar[3];
     __shared__ uint32_t s_codes[kMaxGroup];   // signatures produced by this CTA (CTA 0: queries, CTA 1: new key)
-    __shared__ __align__(16) uint32_t w_hist[kFusedWarps][kBins][32];   // one counter per (warp, level, lane)
+    __shared__ __align__(16) uint32_t c_hist[kBins][32];   // one counter per (level, lane), shared by the warps
     __shared__ int s_hist[kBins + 3], s_tot[kBins], s_bef[kBins];
     __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
     __shared__ int s_wcnt[kFusedWarps];
@@ -183,7 +183,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         mbar_expect_tx(bar0 + 16, kHid * kBits * 2);
         bulk_g2s((uint32_t)__cvta_generic_to_shared(sw3), map.w3 + (size_t)kvh * kHid * kBits, kHid * kBits * 2, bar0 + 16);
     }
-    for (int i = tid; i < kFusedWarps * kBins * 32; i += kFusedThreads) (&w_hist[0][0][0])[i] = 0u;
+    for (int i = tid; i < kBins * 32 / 4; i += kFusedThreads)
+        reinterpret_cast<uint4 *>(&c_hist[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
     if (tid < kBins + 3) s_hist[tid] = 0;
     pdl_wait();                  // q, k_new and everything older in the stream is final from here on
     pdl_launch_dependents();
@@ -213,40 +214,44 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
             }
         }
     }
-    __syncthreads();   // w_hist / s_hist zeroing is visible
+    __syncthreads();   // c_hist / s_hist zeroing is visible
 
     // ---------------- P2: SCORE, histogram, threshold, compaction
     uint32_t sc[kFusedL];
     {
-        // counters are private to a lane, so the adds never conflict; they are issued without waiting
-        // for a result (reduction, not read-modify-write), 16 in a row
-        const uint32_t my = (uint32_t)__cvta_generic_to_shared(&w_hist[warp][0][lane]) - 32u * 4u;   // index: score+1
-        auto bump = [&](uint32_t byte) {
-            asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(my + byte * (32u * 4u)) : "memory");
+        // a lane only meets its own column of counters, so an instruction never conflicts with itself; the
+        // adds are reductions that never wait for a result.  The counter of score s sits (32 - s) rows
+        // below the lane's counter of level 32: the address comes straight from the Hamming distance.
+        const uint32_t top = (uint32_t)__cvta_generic_to_shared(&c_hist[kBins - 1][lane]);
+        auto bump = [&](int ham) { asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(top - (uint32_t)ham * 128u) : "memory"); };
+        auto hamming = [&](uint32_t code) {
+            int h = __popc(code ^ qc[0]);
+#pragma unroll
+            for (int j = 1; j < G; ++j) h = min(h, __popc(code ^ qc[j]));
+            return h;
         };
 #pragma unroll
         for (int p = 0; p < kFusedL; ++p) {
             const int base = wbase + p * 4;
-            uint32_t s4 = scores4<G>(c[p], qc);
+            const int h0 = hamming(c[p].x), h1 = hamming(c[p].y), h2 = hamming(c[p].z), h3 = hamming(c[p].w);
+            // bytes 33 - h = score + 1 (0 marks "no token"); no byte borrows because h <= 32
+            uint32_t s4 = 0x21212121u - ((uint32_t)h0 | ((uint32_t)h1 << 8) | ((uint32_t)h2 << 16) | ((uint32_t)h3 << 24));
             if (p < Lb && base + 3 < n) {
-                bump(s4 & 0xffu); bump((s4 >> 8) & 0xffu); bump((s4 >> 16) & 0xffu); bump(s4 >> 24);
+                bump(h0); bump(h1); bump(h2); bump(h3);
             } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (p < Lb && base + e < n) bump((s4 >> (8 * e)) & 0xffu);
-                    else s4 &= ~(0xffu << (8 * e));   // zero byte: no token
+                if (p < Lb && base + 0 < n) bump(h0); else s4 &= 0xffffff00u;
+                if (p < Lb && base + 1 < n) bump(h1); else s4 &= 0xffff00ffu;
+                if (p < Lb && base + 2 < n) bump(h2); else s4 &= 0xff00ffffu;
+                if (p < Lb && base + 3 < n) bump(h3); else s4 &= 0x00ffffffu;
             }
             sc[p] = s4;
         }
     }
     __syncthreads();
-    for (int i = tid; i < kBins * kFusedWarps; i += kFusedThreads) {   // one (level, warp) row of 32 counters per thread
-        const int bin = i >> 3, w = i & 7;
-        const uint4 *rowp = reinterpret_cast<const uint4 *>(&w_hist[w][bin][0]);
-        uint32_t ssum = 0;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) { const uint4 v = rowp[q]; ssum += (v.x + v.y) + (v.z + v.w); }
-        if (ssum) atomicAdd(&s_hist[bin], (int)ssum);
+    for (int i = tid; i < kBins * 8; i += kFusedThreads) {   // eight threads per level, four counters each
+        const uint4 v = reinterpret_cast<const uint4 *>(&c_hist[i >> 3][0])[i & 7];
+        const uint32_t ssum = (v.x + v.y) + (v.z + v.w);
+        if (ssum) atomicAdd(&s_hist[i >> 3], (int)ssum);
     }
     cluster_sync_all();   // #2: every CTA's histogram is complete and visible cluster-wide
     if (tid < kBins) {
