@@ -143,16 +143,15 @@ def test_score_topk_sizes_ragged_tail_and_budgets(G):
         _check_score_topk(qc, kc, lens, ks, Hq, Hkv)
 
 
-def test_score_topk_beyond_the_cluster_kernel_uses_the_two_kernel_path():
+@pytest.mark.parametrize("lens,n_cap", [([140001, 131073, 9], 140004), ([600001, 524289, 9], 600004)])
+def test_score_topk_long_sequences(lens, n_cap):
     """Sequences longer than 131072 tokens take the chunked scan + select kernels; shorter ones in the same
     batch ride along."""
     rng = np.random.default_rng(77)
     Hkv, Hq = 1, 4
-    lens = [140001, 131073, 9]
-    n_cap = 140004
     kc = rng.integers(0, 2 ** 32, size=(len(lens), Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
     qc = rng.integers(0, 2 ** 32, size=(len(lens), Hq), dtype=np.uint64).astype(np.uint32)
-    for ks in ([n // 32 for n in lens], [3, 131073, 20]):
+    for ks in ([n // 32 for n in lens], [3, lens[1], 20]):
         _check_score_topk(qc, kc, lens, ks, Hq, Hkv)
 
 
