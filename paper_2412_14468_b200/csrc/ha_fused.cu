@@ -279,15 +279,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     }
     if (keep > 0) {
         const int T = sh_T, r = sh_r;
+        // Per byte b = score + 1 (0 = no token): b + 127 - (T+1) sets bit 7 iff score > T, b + 128 - (T+1) iff
+        // score >= T (no byte sum reaches 256).
         const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
-        uint32_t gt16 = 0, eq16 = 0;   // flags of this lane's 16 consecutive tokens
+        const uint32_t c_gt = 0x7f7f7f7fu - T4, c_ge = 0x80808080u - T4;
+        uint32_t gt16 = 0, ge16 = 0;   // flags of this lane's 16 consecutive tokens
 #pragma unroll
         for (int p = 0; p < kFusedL; ++p) {
-            uint32_t gt, eq;
-            flags4(sc[p], T4, gt, eq);
-            gt16 |= flags_to_nibble(gt) << (4 * p);
-            eq16 |= flags_to_nibble(eq) << (4 * p);
+            gt16 |= high_bits_to_nibble(sc[p] + c_gt) << (4 * p);
+            ge16 |= high_bits_to_nibble(sc[p] + c_ge) << (4 * p);
         }
+        const uint32_t eq16 = ge16 ^ gt16;   // score > T implies score >= T
         const int tot_packed = __popc(gt16) | (__popc(eq16) << 16);
         int winc = tot_packed;
 #pragma unroll
@@ -302,7 +304,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         for (int w = 0; w < kFusedWarps; ++w)
             if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
         const int excl = winc - tot_packed;
-        write_selected16(list, wbase, gt16, eq16, run_gt + (excl & 0xffff), run_eq + (int)((unsigned)excl >> 16), r);
+        int g_run = run_gt + (excl & 0xffff), q_run = run_eq + (int)((unsigned)excl >> 16);
+        write_selected32(list, wbase, gt16, eq16, g_run, q_run, r);
     }
     cluster_sync_all();   // #3: the index list is complete and visible to the whole cluster; histograms are free
 

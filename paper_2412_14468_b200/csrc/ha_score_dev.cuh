@@ -5,14 +5,6 @@
 
 namespace ha {
 
-template <int G>
-__device__ __forceinline__ int group_score(uint32_t code, const uint32_t (&qc)[G]) {
-    int h = __popc(code ^ qc[0]);
-#pragma unroll
-    for (int j = 1; j < G; ++j) h = min(h, __popc(code ^ qc[j]));
-    return kBits - h;
-}
-
 __device__ __forceinline__ uint4 load_codes4(const uint32_t *row, int base, int n) {
     // tokens base..base+3 of a 16-byte aligned row; tokens >= n come back as don't-care zeros
     if (base + 3 < n) return __ldg(reinterpret_cast<const uint4 *>(row + base));
@@ -30,22 +22,6 @@ __device__ __forceinline__ void patch_token(uint4 &v, int base, int last, const 
     if (e < 0 || e > 3) return;
     const uint32_t c = __ldcg(row + last);
     if (e == 0) v.x = c; else if (e == 1) v.y = c; else if (e == 2) v.z = c; else v.w = c;
-}
-
-// Four group scores packed as bytes holding score + 1 (1..33); a zero byte means "no token".
-template <int G>
-__device__ __forceinline__ uint32_t scores4(const uint4 &c, const uint32_t (&qc)[G]) {
-    return (uint32_t)(group_score<G>(c.x, qc) + 1) | ((uint32_t)(group_score<G>(c.y, qc) + 1) << 8) |
-           ((uint32_t)(group_score<G>(c.z, qc) + 1) << 16) | ((uint32_t)(group_score<G>(c.w, qc) + 1) << 24);
-}
-
-// Per-byte flags (bit 7 of each byte) of "score > T" and "score == T" for four packed score+1 bytes.
-// Plain 32-bit arithmetic: with bytes <= 33 and T + 1 <= 34 no byte sum reaches 256, so no carry
-// crosses a byte; a zero byte (no token) is neither above nor equal to any threshold.
-__device__ __forceinline__ void flags4(uint32_t s4, uint32_t t1x4, uint32_t &gt, uint32_t &eq) {
-    gt = (s4 + (0x7f7f7f7fu - t1x4)) & 0x80808080u;            // byte + 127 - (T+1) >= 128  <=>  score > T
-    const uint32_t ge = (s4 + (0x80808080u - t1x4)) & 0x80808080u;   // byte + 128 - (T+1) >= 128  <=>  score >= T
-    eq = ge ^ gt;
 }
 
 __device__ __forceinline__ uint32_t cluster_rank() {
@@ -68,25 +44,29 @@ __device__ __forceinline__ int ld_dsmem(const int *local, uint32_t rank) {
 }
 
 
-// The four bit-7 flags of a word gathered into a nibble (bit e = flag of byte e).
-__device__ __forceinline__ uint32_t flags_to_nibble(uint32_t f) {
-    return ((((f >> 7) & 0x01010101u) * 0x01020408u) >> 24) & 0xfu;
+// Bits 7, 15, 23, 31 of x gathered into a nibble (bit e = bit 7 of byte e).  The four partial products
+// land on distinct bit positions, so the multiplication carries nothing into bits 28..31.
+__device__ __forceinline__ uint32_t high_bits_to_nibble(uint32_t x) {
+    return ((x & 0x80808080u) * 0x00204081u) >> 28;
 }
 
-// Writes the selected tokens among 16 consecutive tokens starting at `first`: gt16 / eq16 are the
-// per-token flags "score > T" / "score == T" (bit e = token first + e); gt_lt / eq_lt count the
-// tokens before `first` with those properties; r tokens of score T are still wanted overall.
-// Only the flagged tokens are visited; each position comes from popcounts, not from a running sum.
-__device__ __forceinline__ void write_selected16(int32_t *list, int first, uint32_t gt16, uint32_t eq16, int gt_lt,
-                                                 int eq_lt, int r) {
-    uint32_t m = gt16 | eq16;
+// Index of the single set bit of `one_hot`.
+__device__ __forceinline__ int one_hot_index(uint32_t one_hot) {
+    return ((one_hot & 0xaaaaaaaau) ? 1 : 0) | ((one_hot & 0xccccccccu) ? 2 : 0) | ((one_hot & 0xf0f0f0f0u) ? 4 : 0) |
+           ((one_hot & 0xff00ff00u) ? 8 : 0) | ((one_hot & 0xffff0000u) ? 16 : 0);
+}
+
+// Visits the flagged tokens among 32 consecutive tokens from `first` on in ascending order; g_run / q_run
+// count the tokens with S > T / S == T seen so far in the whole sequence; r tokens of score T are wanted.
+__device__ __forceinline__ void write_selected32(int32_t *list, int first, uint32_t gt, uint32_t eq, int &g_run,
+                                                 int &q_run, int r) {
+    uint32_t m = gt | eq;
     while (m) {
-        const int e = __ffs((int)m) - 1;
-        m &= m - 1;
-        const uint32_t below = (1u << e) - 1u;
-        const int g = gt_lt + __popc(gt16 & below), q = eq_lt + __popc(eq16 & below);
-        if ((gt16 >> e) & 1u) list[g + min(q, r)] = first + e;
-        else if (q < r) list[g + q] = first + e;
+        const uint32_t lb = m & (0u - m);
+        m ^= lb;
+        const int t = first + one_hot_index(lb);
+        if (gt & lb) { list[g_run + min(q_run, r)] = t; ++g_run; }
+        else { if (q_run < r) list[g_run + q_run] = t; ++q_run; }
     }
 }
 

@@ -27,7 +27,8 @@ constexpr int kClusterMaxSeq = 8 * 8 * 2048;     // longest sequence the cluster
 // Kernel 1: one chunk per CTA.  Streams the chunk's signatures (four uint4 per thread in flight, the
 // next pass requested before the current one is scored), leaves the group scores as one byte per
 // token in the workspace (so that kernel 2 needs neither the signatures nor popc again) and the
-// chunk's 33-bin histogram.  Counting uses one byte counter per (level, lane): no atomics.
+// chunk's 33-bin histogram.  Counting: one 32-bit counter per (level, lane), shared by the warps and
+// bumped with shared-memory reductions (a lane only meets its own column; nothing waits for a result).
 template <int G>
 __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t *__restrict__ q_codes,
                                                                  const uint32_t *__restrict__ k_codes,
@@ -37,13 +38,13 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
                                                                  int chunk_tokens, long long score_row,
                                                                  unsigned char *__restrict__ ws_scores,
                                                                  int32_t *__restrict__ ws_hist) {
-    __shared__ __align__(16) unsigned char w_hist[kScanThreads / 32][kBins][32];
+    __shared__ __align__(16) uint32_t c_hist[kBins][32];
     __shared__ int s_hist[kBins + 3];
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int n = min(seq_lens[b], max_seq_len);
     const int start = chunk * chunk_tokens;
     if (start >= n) return;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
     const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
     uint32_t *srow = reinterpret_cast<uint32_t *>(ws_scores + ((long long)b * Hkv + g) * score_row);
     const int end = min(n, start + chunk_tokens);
@@ -58,8 +59,8 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
     };
     uint4 cur[4], nxt[4];
     load_pass(cur, start);
-    for (int i = tid; i < (kScanThreads / 32) * kBins * 32 / 4; i += kScanThreads)
-        reinterpret_cast<uint32_t *>(&w_hist[0][0][0])[i] = 0u;
+    for (int i = tid; i < kBins * 32 / 4; i += kScanThreads)
+        reinterpret_cast<uint4 *>(&c_hist[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
     if (tid < kBins + 3) s_hist[tid] = 0;
     pdl_launch_dependents();
     pdl_wait();
@@ -68,7 +69,15 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
     for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
     __syncthreads();
 
-    unsigned char *my = &w_hist[warp][0][lane] - 32;   // indexed by the score+1 byte
+    // the counter of score s sits (32 - s) rows below the lane's counter of level 32
+    const uint32_t top = (uint32_t)__cvta_generic_to_shared(&c_hist[kBins - 1][lane]);
+    auto bump = [&](int ham) { asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(top - (uint32_t)ham * 128u) : "memory"); };
+    auto hamming = [&](uint32_t code) {
+        int h = __popc(code ^ qc[0]);
+#pragma unroll
+        for (int j = 1; j < G; ++j) h = min(h, __popc(code ^ qc[j]));
+        return h;
+    };
     for (int pass = start; pass < end; pass += kPassTokens) {
         if (pass + kPassTokens < end) load_pass(nxt, pass + kPassTokens);
 #pragma unroll
@@ -76,17 +85,16 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
             const int base = pass + j * 1024 + tid * 4;
             if (base < end) {
                 patch_token(cur[j], base, n - 1, row);   // the appended token may just have been written
-                uint32_t s4 = scores4<G>(cur[j], qc);
+                const int h0 = hamming(cur[j].x), h1 = hamming(cur[j].y), h2 = hamming(cur[j].z), h3 = hamming(cur[j].w);
+                // bytes 33 - h = score + 1 (0 = no token); no byte borrows because h <= 32
+                uint32_t s4 = 0x21212121u - ((uint32_t)h0 | ((uint32_t)h1 << 8) | ((uint32_t)h2 << 16) | ((uint32_t)h3 << 24));
                 if (base + 3 < end) {                    // whole uint4 inside the chunk: no per-token checks
-                    my[(s4 & 0xffu) * 32] += 1;
-                    my[((s4 >> 8) & 0xffu) * 32] += 1;
-                    my[((s4 >> 16) & 0xffu) * 32] += 1;
-                    my[(s4 >> 24) * 32] += 1;
+                    bump(h0); bump(h1); bump(h2); bump(h3);
                 } else {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (base + e < end) my[((s4 >> (8 * e)) & 0xffu) * 32] += 1;
-                        else s4 &= ~(0xffu << (8 * e));   // zero byte: no token
+                    if (base + 0 < end) bump(h0); else s4 &= 0xffffff00u;
+                    if (base + 1 < end) bump(h1); else s4 &= 0xffff00ffu;
+                    if (base + 2 < end) bump(h2); else s4 &= 0xff00ffffu;
+                    if (base + 3 < end) bump(h3); else s4 &= 0x00ffffffu;
                 }
                 srow[base >> 2] = s4;
             }
@@ -95,13 +103,10 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
         for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
     }
     __syncthreads();
-    for (int i = tid; i < kBins * (kScanThreads / 32); i += kScanThreads) {
-        const int bin = i >> 3, w = i & 7;
-        const uint4 *rowp = reinterpret_cast<const uint4 *>(&w_hist[w][bin][0]);
-        const uint4 a0 = rowp[0], a1 = rowp[1];
-        const int s = (int)(__vsadu4(a0.x, 0u) + __vsadu4(a0.y, 0u) + __vsadu4(a0.z, 0u) + __vsadu4(a0.w, 0u) +
-                            __vsadu4(a1.x, 0u) + __vsadu4(a1.y, 0u) + __vsadu4(a1.z, 0u) + __vsadu4(a1.w, 0u));
-        if (s) atomicAdd(&s_hist[bin], s);
+    for (int i = tid; i < kBins * 8; i += kScanThreads) {   // eight threads per level, four counters each
+        const uint4 v = reinterpret_cast<const uint4 *>(&c_hist[i >> 3][0])[i & 7];
+        const uint32_t ssum = (v.x + v.y) + (v.z + v.w);
+        if (ssum) atomicAdd(&s_hist[i >> 3], (int)ssum);
     }
     __syncthreads();
     if (tid < kBins) ws_hist[(((long long)b * Hkv + g) * kMaxChunks + chunk) * kBins + tid] = s_hist[tid];
@@ -183,7 +188,10 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
     }
     if (chunk >= n_chunks || keep == 0) return;
 
+    // Per byte b = score + 1 (0 = no token): b + 127 - (T+1) sets bit 7 iff score > T, b + 128 - (T+1) iff
+    // score >= T (no byte sum reaches 256).
     const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
+    const uint32_t c_gt = 0x7f7f7f7fu - T4, c_ge = 0x80808080u - T4;
     int run_gt = sh_gt_before, run_eq = sh_eq_before;   // tokens before this pass with S > T / S == T
     for (int pass = start; pass < end; pass += kPassTokens) {
         const int base = pass + tid * 16;
@@ -191,14 +199,16 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
         sv_next = make_uint4(0u, 0u, 0u, 0u);
         if (base + kPassTokens < end) sv_next = __ldcg(srow + ((base + kPassTokens) >> 4));   // next pass, in flight
         const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
-        uint32_t gt[4], eq[4];
-        int packed = 0;
+        uint32_t gt16 = 0u, ge16 = 0u;   // bit i = token base + i
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             // words past the chunk were never written: drop them (end is a multiple of 4 or the sequence end)
-            flags4((base + 4 * j < end) ? sw[j] : 0u, T4, gt[j], eq[j]);
-            packed += __popc(gt[j]) | (__popc(eq[j]) << 16);
+            const uint32_t w = (base + 4 * j < end) ? sw[j] : 0u;
+            gt16 |= high_bits_to_nibble(w + c_gt) << (4 * j);
+            ge16 |= high_bits_to_nibble(w + c_ge) << (4 * j);
         }
+        const uint32_t eq16 = ge16 ^ gt16;   // score > T implies score >= T
+        const int packed = __popc(gt16) | (__popc(eq16) << 16);
         // block-wide exclusive prefix of the packed (gt, eq) counts (a pass has 4096 tokens: 16-bit halves suffice)
         int inc = packed;
 #pragma unroll
@@ -217,22 +227,9 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
         }
         if (packed != 0) {
             const int excl = wpre + inc - packed;
-            int gt_lt = run_gt + (excl & 0xffff);
-            int eq_lt = run_eq + (int)((unsigned)excl >> 16);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if ((gt[j] | eq[j]) == 0u) continue;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if ((gt[j] >> (8 * e + 7)) & 1u) {
-                        out[gt_lt + min(eq_lt, r)] = base + 4 * j + e;
-                        ++gt_lt;
-                    } else if ((eq[j] >> (8 * e + 7)) & 1u) {
-                        if (eq_lt < r) out[gt_lt + eq_lt] = base + 4 * j + e;
-                        ++eq_lt;
-                    }
-                }
-            }
+            int g_run = run_gt + (excl & 0xffff);
+            int q_run = run_eq + (int)((unsigned)excl >> 16);
+            write_selected32(out, base, gt16, eq16, g_run, q_run, r);
         }
         run_gt += all & 0xffff;
         run_eq += (int)((unsigned)all >> 16);
@@ -260,32 +257,6 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
 // need one warp-shuffle scan plus one exchange of eight warp totals; only flagged tokens are
 // visited, with plain integer arithmetic (the selection never queues behind the scoring for the
 // population-count unit).
-
-// Bits 7, 15, 23, 31 of x gathered into a nibble (bit e = bit 7 of byte e).  The four partial products
-// land on distinct bit positions, so the multiplication carries nothing into bits 28..31.
-__device__ __forceinline__ uint32_t high_bits_to_nibble(uint32_t x) {
-    return ((x & 0x80808080u) * 0x00204081u) >> 28;
-}
-
-// Index of the single set bit of `one_hot`.
-__device__ __forceinline__ int one_hot_index(uint32_t one_hot) {
-    return ((one_hot & 0xaaaaaaaau) ? 1 : 0) | ((one_hot & 0xccccccccu) ? 2 : 0) | ((one_hot & 0xf0f0f0f0u) ? 4 : 0) |
-           ((one_hot & 0xff00ff00u) ? 8 : 0) | ((one_hot & 0xffff0000u) ? 16 : 0);
-}
-
-// Visits the flagged tokens among 32 consecutive tokens from `first` on in ascending order; g_run / q_run
-// count the tokens with S > T / S == T seen so far in the whole sequence; r tokens of score T are wanted.
-__device__ __forceinline__ void write_selected32(int32_t *list, int first, uint32_t gt, uint32_t eq, int &g_run,
-                                                 int &q_run, int r) {
-    uint32_t m = gt | eq;
-    while (m) {
-        const uint32_t lb = m & (0u - m);
-        m ^= lb;
-        const int t = first + one_hot_index(lb);
-        if (gt & lb) { list[g_run + min(q_run, r)] = t; ++g_run; }
-        else { if (q_run < r) list[g_run + q_run] = t; ++q_run; }
-    }
-}
 
 constexpr int kClusterMaxRows = 8;   // rows of 8 tokens per lane: a lane's flags fit one 64-bit word each
 
