@@ -25,6 +25,7 @@ def lib():
     if _lib is None:
         _lib = C.CDLL(_build())
         _lib.ora_topk.restype = C.c_int64
+        _lib.ora_topk_windows.restype = C.c_int64
         _lib.ora_f64_to_bf16.restype = C.c_uint16
         _lib.ora_f64_to_bf16.argtypes = [C.c_double]
         _lib.ora_max_threads.restype = C.c_int32
@@ -83,6 +84,16 @@ def topk(scores, k: int) -> np.ndarray:
     return out[:cnt].copy()
 
 
+def topk_windows(scores, k: int, n_sink: int, n_local: int) -> np.ndarray:
+    """The first n_sink and the last n_local tokens always, plus the top k of the others (Section 5,
+    paragraph on baselines); indices returned ascending."""
+    scores = np.ascontiguousarray(scores, dtype=np.int32).reshape(-1)
+    n = scores.shape[0]
+    out = np.full(max(n, 1), -1, dtype=np.int32)
+    cnt = lib().ora_topk_windows(_p(scores), C.c_int64(n), C.c_int64(k), C.c_int64(n_sink), C.c_int64(n_local), _p(out))
+    return out[:cnt].copy()
+
+
 def gather_attn(q, K, V, idx, sm_scale=None, n_valid=None):
     """GATHER-ATT for one query head.  q: uint16 [128]; K, V: uint16 [n,128]; idx: int32 list or None.
     Returns (out uint16 [128], lse float, out float64 [128])."""
@@ -115,12 +126,14 @@ def max_threads() -> int:
     return int(lib().ora_max_threads())
 
 
-def decode_step(q, k_new, K, V, kcodes, map_q, map_k, seq_lens, k_per_seq, sm_scale=None, n_threads=1):
+def decode_step(q, k_new, K, V, kcodes, map_q, map_k, seq_lens, k_per_seq, sm_scale=None, n_threads=1,
+                n_sink=0, n_local=0):
     """One layer-step: ENCODE -> SCORE -> TOPK -> GATHER-ATT for the batch.
 
     q uint16 [B,Hq,128]; k_new uint16 [B,Hkv,128] or None; K, V uint16 [B,Hkv,n_cap,128];
     kcodes uint32 [B,Hkv,n_cap] (slot n_b-1 is overwritten when k_new is given);
     map_q / map_k: dict with w1,w2,w3 (uint16 [Hkv,...]) and b1,b2,b3 (float32 [Hkv,out] or None).
+    n_sink / n_local: tokens always kept in addition to the budget (0, 0 = plain top-k).
     Returns dict(qcodes, idx, count, out, lse)."""
     q = _u16(q)
     B, Hq, _ = q.shape
@@ -129,7 +142,7 @@ def decode_step(q, k_new, K, V, kcodes, map_q, map_k, seq_lens, k_per_seq, sm_sc
     assert kcodes.dtype == np.uint32 and kcodes.flags.c_contiguous and kcodes.shape == (B, Hkv, n_cap)
     seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
     k_per_seq = np.ascontiguousarray(k_per_seq, dtype=np.int32)
-    k_max = max(int(k_per_seq.max()), 1)
+    k_max = max(int(k_per_seq.max()) + int(n_sink) + int(n_local), 1)
     if sm_scale is None:
         sm_scale = 1.0 / math.sqrt(D)
 
@@ -152,5 +165,5 @@ def decode_step(q, k_new, K, V, kcodes, map_q, map_k, seq_lens, k_per_seq, sm_sc
         _p(wq[0]), _p(wq[1]), _p(wq[2]), _p(bq[0]), _p(bq[1]), _p(bq[2]),
         _p(wk[0]), _p(wk[1]), _p(wk[2]), _p(bk[0]), _p(bk[1]), _p(bk[2]),
         _p(seq_lens), _p(k_per_seq), C.c_double(sm_scale),
-        _p(qcodes), _p(idx), _p(count), _p(out), _p(lse), C.c_int32(n_threads))
+        _p(qcodes), _p(idx), _p(count), _p(out), _p(lse), C.c_int32(n_threads), C.c_int32(n_sink), C.c_int32(n_local))
     return dict(qcodes=qcodes, idx=idx, count=count, out=out, lse=lse)

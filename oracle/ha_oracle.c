@@ -19,6 +19,10 @@
  *                    share the KV head (reduces to Eq. 1 when the group has one head).
  *   ora_topk         "the standard top-k on these scores" (Section 4): sort by
  *                    (score descending, token index ascending), keep min(k, n).
+ *   ora_topk_windows the selection used for every method in the experiments (Section 5,
+ *                    paragraph on baselines): the first n_sink and the most recent n_local
+ *                    tokens are always in context, the token budget k counts the heavy
+ *                    tokens retrieved in addition, by the same order, among the others.
  *   ora_gather_attn  the GATHER-ATT formula of Section 4 (softmax restricted to the index
  *                    set), with the 1/sqrt(d) factor of the SDPA definition (Section 3.1)
  *                    passed in as sm_scale.
@@ -184,6 +188,29 @@ int64_t ora_topk(const int32_t *scores, int64_t n, int64_t k, int32_t *idx_out) 
     return keep;
 }
 
+/* Always keep tokens [0, n_sink) and [n - n_local, n); among the other tokens keep the first
+ * min(k, how many there are) of the order (score desc, index asc); emit everything ascending.
+ * Returns the number of indices written (at most n).  n_sink = n_local = 0 is ora_topk. */
+int64_t ora_topk_windows(const int32_t *scores, int64_t n, int64_t k, int64_t n_sink, int64_t n_local,
+                         int32_t *idx_out) {
+    if (n <= 0) return 0;
+    if (n_sink < 0) n_sink = 0;
+    if (n_local < 0) n_local = 0;
+    int64_t written = 0, n_rest = 0;
+    int32_t *rest = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);
+    int32_t *tmp = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);
+    for (int64_t i = 0; i < n; ++i) {
+        if (i < n_sink || i >= n - n_local) idx_out[written++] = (int32_t)i;   /* always in context */
+        else rest[n_rest++] = (int32_t)i;
+    }
+    int64_t keep = k < 0 ? 0 : (k < n_rest ? k : n_rest);
+    merge_sort_desc(rest, tmp, 0, n_rest, scores);
+    for (int64_t i = 0; i < keep; ++i) idx_out[written++] = rest[i];
+    qsort(idx_out, (size_t)written, sizeof(int32_t), cmp_i32);
+    free(rest); free(tmp);
+    return written;
+}
+
 /* ---------------------------------------------------------------- GATHER-ATT / SDPA */
 
 /* One query head over an index list.
@@ -246,6 +273,8 @@ uint16_t ora_f64_to_bf16(double x) { return f64_to_bf16(x); }
  *   wq*, wk*: per-KV-head mappings, w1/w2 [Hkv][128][128], w3 [Hkv][128][32], biases [Hkv][out] or NULL
  *   seq_lens [B], k_per_seq [B]
  *   qcodes out [B][Hq]; idx out [B][Hkv][k_max] (ascending, -1 padded); count out [B][Hkv]
+ *   n_sink, n_local: tokens always kept in addition to the budget (0, 0 = plain top-k); k_max must
+ *   hold the windows plus the budget
  *   out bf16 [B][Hq][128]; lse double [B][Hq]
  * One OpenMP loop over (b, g) when compiled with -fopenmp and n_threads > 1. */
 void ora_decode_step(int32_t B, int32_t Hq, int32_t Hkv, int64_t n_cap, int64_t k_max,
@@ -257,7 +286,7 @@ void ora_decode_step(int32_t B, int32_t Hq, int32_t Hkv, int64_t n_cap, int64_t 
                      const float *bk1, const float *bk2, const float *bk3,
                      const int32_t *seq_lens, const int32_t *k_per_seq, double sm_scale,
                      uint32_t *qcodes, int32_t *idx, int32_t *count,
-                     uint16_t *out, double *lse, int32_t n_threads) {
+                     uint16_t *out, double *lse, int32_t n_threads, int32_t n_sink, int32_t n_local) {
     const int32_t G = Hq / Hkv;
     const int64_t units = (int64_t)B * Hkv;
     (void)n_threads;
@@ -291,7 +320,8 @@ void ora_decode_step(int32_t B, int32_t Hq, int32_t Hkv, int64_t n_cap, int64_t 
         /* SCORE -> TOPK */
         int32_t *scores = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n > 0 ? n : 1));
         ora_score(qc, G, codes, n, scores);
-        int64_t cnt = ora_topk(scores, n, k, idx_u);
+        int64_t cnt = (n_sink > 0 || n_local > 0) ? ora_topk_windows(scores, n, k, n_sink, n_local, idx_u)
+                                                  : ora_topk(scores, n, k, idx_u);
         count[u] = (int32_t)cnt;
         free(scores);
 

@@ -69,6 +69,50 @@ def test_golden_topk_cases():
         assert got.tolist() == [int(v) for v in sel.split()], ln
 
 
+def test_golden_topk_window_cases():
+    for ln in _lines("topk_window_cases.txt"):
+        k, n_sink, n_local, scores, sel = [p.strip() for p in ln.split("|")]
+        got = oracle.topk_windows([int(v) for v in scores.split()], int(k), int(n_sink), int(n_local))
+        assert got.tolist() == [int(v) for v in sel.split()], ln
+
+
+def _window_definition(scores, k, n_sink, n_local):
+    """Written from the sentence, not from the code: always-kept tokens, then rank among the others."""
+    n = len(scores)
+    forced = [i for i in range(n) if i < n_sink or i >= n - n_local]
+    others = [i for i in range(n) if i not in forced]
+    heavy = []
+    for i in others:
+        better = sum(1 for j in others if scores[j] > scores[i] or (scores[j] == scores[i] and j < i))
+        if better < k:
+            heavy.append(i)
+    return sorted(forced + heavy)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_topk_windows_matches_its_definition_and_reduces_to_plain_topk(seed):
+    rng = np.random.default_rng(300 + seed)
+    for n in (1, 2, 7, 33, 64):
+        scores = rng.integers(12, 22, size=n)           # narrow range -> heavy ties
+        for k in (0, 1, n // 2, n):
+            assert oracle.topk_windows(scores, k, 0, 0).tolist() == oracle.topk(scores, k).tolist()
+            for n_sink, n_local in ((1, 0), (0, 1), (2, 3), (n // 2, n // 2), (n, 0), (n + 2, n + 2), (5, 40)):
+                got = oracle.topk_windows(scores, k, n_sink, n_local).tolist()
+                assert got == _window_definition(scores.tolist(), k, n_sink, n_local), (n, k, n_sink, n_local)
+
+
+def test_topk_windows_properties_on_large_input():
+    rng = np.random.default_rng(9)
+    n, k, n_sink, n_local = 50000, 1500, 128, 128
+    scores = rng.integers(14, 24, size=n)
+    sel = oracle.topk_windows(scores, k, n_sink, n_local)
+    assert len(sel) == n_sink + n_local + k and np.all(np.diff(sel) > 0)
+    assert set(range(n_sink)) <= set(sel.tolist()) and set(range(n - n_local, n)) <= set(sel.tolist())
+    heavy = np.array(sorted(set(sel.tolist()) - set(range(n_sink)) - set(range(n - n_local, n))))
+    middle = scores[n_sink:n - n_local]
+    assert np.array_equal(heavy - n_sink, oracle.topk(middle, k))   # plain top-k of the tokens in between
+
+
 def _rank_definition(scores, k):
     n = len(scores)
     sel = []
