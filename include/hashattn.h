@@ -59,13 +59,19 @@ extern "C" {
 #define HA_HIST_BINS 33 /* scores 0..32 */
 
 /* Problem shape of one layer-step. sm_scale multiplies the logits (1/sqrt(d) in the SDPA
- * definition, Section 3.1). */
+ * definition, Section 3.1).
+ * n_sink / n_local: the first n_sink and the most recent n_local tokens of every sequence are always
+ * in context, and the budget k counts the heavy tokens retrieved in addition among the others
+ * (Section 5, paragraph on baselines, where both are 128).  0 / 0 is the plain top-k of Section 4.
+ * Only SCORE + TOPK (ha_score_topk, ha_sparse_decode, ha_sparse_decode_host) looks at them. */
 typedef struct ha_shape {
     int32_t batch;
     int32_t n_q_heads;
     int32_t n_kv_heads;
     int32_t head_dim; /* must be 128 */
     float sm_scale;
+    int32_t n_sink;   /* >= 0 */
+    int32_t n_local;  /* >= 0 */
 } ha_shape;
 
 /* One side's mapping networks (phi_q or phi_kv of Eq. 2), one network per KV head.
@@ -124,7 +130,11 @@ int ha_encode(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, i
  *              entries count..k_max-1 set to -1; k_max = max budget = the k passed to
  *              ha_workspace_bytes or less
  *   count      out i32 [batch][n_kv_heads] = min(k_b, seq_len_b)
- *   hist_out   optional out i32 [batch][n_kv_heads][33]: histogram of the group scores */
+ *   hist_out   optional out i32 [batch][n_kv_heads][33]: histogram of the group scores
+ * With shape->n_sink or shape->n_local > 0: tokens [0, n_sink) and [seq_len - n_local, seq_len) are
+ * always selected, k_b more come from the others by the same order; count = windows + min(k_b, others);
+ * hist_out covers the others only; k_max must be >= n_sink + n_local (else HA_ERR_INVALID_ARG) and
+ * should be >= n_sink + n_local + max k_b, since the budget is cut to what fits in k_max. */
 int ha_score_topk(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes,
                   int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens,
                   const int32_t *k_per_seq, int32_t k_uniform, int32_t max_seq_len, int32_t k_max,

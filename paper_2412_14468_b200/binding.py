@@ -29,7 +29,7 @@ EXPORTS = [
 
 class ha_shape(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
-                ("head_dim", C.c_int32), ("sm_scale", C.c_float)]
+                ("head_dim", C.c_int32), ("sm_scale", C.c_float), ("n_sink", C.c_int32), ("n_local", C.c_int32)]
 
 
 class ha_mapping(C.Structure):
@@ -117,8 +117,10 @@ def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
     return t
 
 
-def make_shape(batch: int, n_q_heads: int, n_kv_heads: int, sm_scale: float, head_dim: int = 128) -> ha_shape:
-    return ha_shape(batch, n_q_heads, n_kv_heads, head_dim, float(sm_scale))
+def make_shape(batch: int, n_q_heads: int, n_kv_heads: int, sm_scale: float, head_dim: int = 128,
+               n_sink: int = 0, n_local: int = 0) -> ha_shape:
+    """n_sink / n_local: tokens always in context in addition to the budget (SCORE + TOPK only)."""
+    return ha_shape(batch, n_q_heads, n_kv_heads, head_dim, float(sm_scale), n_sink, n_local)
 
 
 def make_tensor(t: torch.Tensor) -> ha_tensor:

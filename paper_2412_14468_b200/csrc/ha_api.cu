@@ -19,6 +19,7 @@ static int check_shape(const ha_shape *s) {
     if (s->n_kv_heads > 65535 || s->batch > 65535) return HA_ERR_UNSUPPORTED;
     if ((long long)s->n_kv_heads * s->batch > kMaxUnits) return HA_ERR_UNSUPPORTED;
     if (!(s->sm_scale == s->sm_scale)) return HA_ERR_INVALID_ARG;
+    if (s->n_sink < 0 || s->n_local < 0) return HA_ERR_INVALID_ARG;
     return HA_OK;
 }
 
@@ -123,6 +124,7 @@ static int check_score_args(const ha_shape *shape, const uint32_t *q_codes, cons
     if (!q_codes || !k_codes || !seq_lens || !idx || !count) return HA_ERR_INVALID_ARG;
     if (max_seq_len < 0 || k_max < 0 || (!k_per_seq && k_uniform < 0)) return HA_ERR_INVALID_ARG;
     if (((uintptr_t)k_codes & 15) || (kc_stride_b & 3) || (kc_stride_h & 3)) return HA_ERR_INVALID_ARG;
+    if ((long long)shape->n_sink + shape->n_local > k_max) return HA_ERR_INVALID_ARG;   // idx rows must hold the windows
     return HA_OK;
 }
 
@@ -138,7 +140,8 @@ int ha_score_topk(const ha_shape *shape, const uint32_t *q_codes, const uint32_t
     HA_CUDA(launch_score_topk(shape->batch, shape->n_q_heads, shape->n_kv_heads, q_codes, k_codes, kc_stride_b,
                               kc_stride_h, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx, idx_stride_b,
                               idx_stride_h, count, hist_out, ws_ptr<int32_t>(workspace, L.off_hist),
-                              ws_ptr<unsigned char>(workspace, L.off_scores), (cudaStream_t)stream));
+                              ws_ptr<unsigned char>(workspace, L.off_scores), (cudaStream_t)stream,
+                              Windows{shape->n_sink, shape->n_local}));
     return HA_OK;
 }
 
@@ -204,7 +207,8 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
         // small batch: the whole step is one cluster kernel
         HA_CUDA(launch_fused_step(B, Hq, Hkv, shape->sm_scale, view(map_q), k_new ? view(map_k) : MapView{}, q, k_new,
                                   view(K), view(V), k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
-                                  max_seq_len, k_max, q_codes, idx, idx_stride_b, idx_stride_h, count, out, lse, st));
+                                  max_seq_len, k_max, q_codes, idx, idx_stride_b, idx_stride_h, count, out, lse, st,
+                                  Windows{shape->n_sink, shape->n_local}));
         return HA_OK;
     }
 
@@ -225,11 +229,13 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
     HA_CUDA(launch_encode_vectors(jq, jk, st));
     HA_CUDA(launch_score_topk(B, Hq, Hkv, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
                               max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, nullptr,
-                              ws_ptr<int32_t>(workspace, L.off_hist), ws_ptr<unsigned char>(workspace, L.off_scores), st));
+                              ws_ptr<int32_t>(workspace, L.off_hist), ws_ptr<unsigned char>(workspace, L.off_scores), st,
+                              Windows{shape->n_sink, shape->n_local}));
     HA_CUDA(launch_attention(true, B, Hq, Hkv, shape->sm_scale, q, view(K), view(V), seq_lens, idx, idx_stride_b,
                              idx_stride_h, count, k_max, out, lse, ws_ptr<float>(workspace, L.off_part_ml),
                              ws_ptr<float>(workspace, L.off_part_acc), ws_ptr<int32_t>(workspace, L.off_tickets),
-                             ws_ptr<uint32_t>(workspace, 0), st, /*count_from_k=*/1, k_per_seq, k_uniform));
+                             ws_ptr<uint32_t>(workspace, 0), st, /*count_from_k=*/1, k_per_seq, k_uniform,
+                             Windows{shape->n_sink, shape->n_local}));
     return HA_OK;
 }
 

@@ -34,6 +34,7 @@ struct AttnArgs {
     long long idx_sb, idx_sh;
     const int32_t *k_per_seq;   // with count_from_k: budget per sequence (or NULL: k_uniform)
     int k_uniform, count_from_k;
+    Windows win;                // with count_from_k: tokens always kept in addition to the budget
     int max_items, Hq, Hkv, n_units, balanced;
     float scale_log2;
     float *part_ml, *part_acc;
@@ -71,7 +72,15 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
         const int b = u / Hkv;
         const int n_b = a.seq_lens[b];
         int c = n_b;
-        if (kGather) c = a.count_from_k ? min(a.k_per_seq ? a.k_per_seq[b] : a.k_uniform, n_b) : a.count[u];
+        if (kGather) {
+            if (a.count_from_k) {   // what SCORE + TOPK is about to report: windows plus the budget among the others
+                const int nf = forced_before(window_bounds(a.win, max(n_b, 0)), max(n_b, 0));
+                const int kb = a.k_per_seq ? a.k_per_seq[b] : a.k_uniform;
+                c = nf + max(0, min(min(kb, a.max_items - nf), n_b - nf));
+            } else {
+                c = a.count[u];
+            }
+        }
         return max(0, min(c, a.max_items));
     };
     auto write_empty = [&](int u) {   // empty selection: out = 0, lse = -inf
@@ -428,8 +437,9 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
                              uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
                              uint32_t *status, cudaStream_t st, int count_from_k, const int32_t *k_per_seq,
-                             int k_uniform) {
+                             int k_uniform, Windows win) {
     AttnArgs a{};
+    a.win = win;
     a.q = q; a.K = K; a.V = V; a.seq_lens = seq_lens; a.idx = idx; a.count = count;
     a.idx_sb = idx_sb; a.idx_sh = idx_sh; a.max_items = max_items; a.Hq = Hq; a.Hkv = Hkv;
     a.n_units = B * Hkv; a.scale_log2 = sm_scale * kLog2e;

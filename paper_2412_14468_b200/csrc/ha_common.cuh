@@ -107,6 +107,33 @@ struct MapView {
     const float *b1, *b2, *b3;
 };
 
+// Tokens that are always in context (Section 5, paragraph on baselines): the first n_sink and the most
+// recent n_local of a sequence; the budget k counts the heavy tokens retrieved in addition.
+struct Windows {
+    int n_sink, n_local;
+};
+// For a sequence of n tokens: token t is forced iff t < sink_end or t >= local_begin.
+struct WindowBounds {
+    int sink_end, local_begin;   // sink_end <= local_begin <= n (touching or overlapping windows: equal)
+};
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline WindowBounds window_bounds(Windows w, int n) {
+    WindowBounds r;
+    r.sink_end = w.n_sink < n ? w.n_sink : n;
+    const int lb = n - w.n_local;
+    r.local_begin = lb > r.sink_end ? lb : r.sink_end;
+    return r;
+}
+// number of forced tokens with index < p (0 <= p <= n)
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+inline int forced_before(WindowBounds w, int p) {
+    return (p < w.sink_end ? p : w.sink_end) + (p > w.local_begin ? p - w.local_begin : 0);
+}
+
 // One batch of single vectors to encode (decode step): CTA i handles sequence i / n_nets and
 // network i % n_nets, i.e. the heads_per_kv (<= 8) heads that share that network.
 struct EncodeJob {
@@ -144,14 +171,14 @@ cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, c
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens,
                               const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max,
                               int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
-                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st);
+                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st, Windows win = Windows{0, 0});
 
 cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale, const uint16_t *q,
                              TensorView K, TensorView V, const int32_t *seq_lens, const int32_t *idx,
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
                              uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
                              uint32_t *status, cudaStream_t st, int count_from_k = 0,
-                             const int32_t *k_per_seq = nullptr, int k_uniform = 0);
+                             const int32_t *k_per_seq = nullptr, int k_uniform = 0, Windows win = Windows{0, 0});
 
 // The whole layer-step in one launch (one 8-CTA cluster per unit); only for small batches.
 bool fused_step_eligible(int B, int Hkv, int max_seq_len);
@@ -160,7 +187,7 @@ cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapV
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
                               int k_uniform, int max_seq_len, int k_max, uint32_t *q_codes, int32_t *idx,
                               long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
-                              cudaStream_t st);
+                              cudaStream_t st, Windows win = Windows{0, 0});
 
 cudaError_t launch_append_kv(int B, int Hq, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
                              TensorView V, const int32_t *seq_lens, const uint16_t *q_src, uint16_t *q_dst,

@@ -46,6 +46,7 @@ struct FusedArgs {
     long long kc_sb, kc_sh;
     const int32_t *seq_lens, *k_per_seq;
     int k_uniform, max_seq_len, k_max, Hq, Hkv;
+    Windows win;
     float scale_log2;
     uint32_t *q_codes;
     int32_t *idx;
@@ -147,8 +148,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     const int Hq = a.Hq, Hkv = a.Hkv;
     const int n = max(min(a.seq_lens[b], a.max_seq_len), 0);
     int k = a.k_per_seq ? a.k_per_seq[b] : a.k_uniform;
-    k = max(0, min(k, a.k_max));
-    const int keep = min(k, n);
+    const WindowBounds wbd = window_bounds(a.win, n);   // always-kept tokens: byte kForcedByte, not counted
+    const int n_forced = forced_before(wbd, n);
+    const int keep_rest = max(0, min(min(k, a.k_max - n_forced), n - n_forced));   // heavy tokens among the others
+    const int keep = n_forced + keep_rest;
     const long long head0 = (long long)b * Hq + (long long)kvh * G;
     uint32_t *row = a.k_codes + (long long)b * a.kc_sb + (long long)kvh * a.kc_sh;
     const bool has_new_key = (a.k_new != nullptr) && n > 0;
@@ -236,13 +239,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
             const int h0 = hamming(c[p].x), h1 = hamming(c[p].y), h2 = hamming(c[p].z), h3 = hamming(c[p].w);
             // bytes 33 - h = score + 1 (0 marks "no token"); no byte borrows because h <= 32
             uint32_t s4 = 0x21212121u - ((uint32_t)h0 | ((uint32_t)h1 << 8) | ((uint32_t)h2 << 16) | ((uint32_t)h3 << 24));
-            if (p < Lb && base + 3 < n) {
+            if (p < Lb && base + 3 < n && base >= wbd.sink_end && base + 4 <= wbd.local_begin) {
                 bump(h0); bump(h1); bump(h2); bump(h3);
             } else {
-                if (p < Lb && base + 0 < n) bump(h0); else s4 &= 0xffffff00u;
-                if (p < Lb && base + 1 < n) bump(h1); else s4 &= 0xffff00ffu;
-                if (p < Lb && base + 2 < n) bump(h2); else s4 &= 0xff00ffffu;
-                if (p < Lb && base + 3 < n) bump(h3); else s4 &= 0x00ffffffu;
+                const int hh[4] = {h0, h1, h2, h3};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int t = base + e;
+                    if (p >= Lb || t >= n) s4 &= ~(0xffu << (8 * e));                      // zero byte: no token
+                    else if (t < wbd.sink_end || t >= wbd.local_begin) s4 = (s4 & ~(0xffu << (8 * e))) | (kForcedByte << (8 * e));
+                    else bump(hh[e]);
+                }
             }
             sc[p] = s4;
         }
@@ -268,7 +275,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     __syncthreads();
     if (warp == 0) {
         int T, r, gt_before, eq_before;
-        find_threshold(s_tot[lane], s_bef[lane], s_tot[32], s_bef[32], keep, lane, T, r, gt_before, eq_before);
+        find_threshold(s_tot[lane], s_bef[lane], s_tot[32], s_bef[32], keep_rest, lane, T, r, gt_before, eq_before);
         if (lane == 0) { sh_T = T; sh_r = r; sh_gt_before = gt_before; sh_eq_before = eq_before; }
     }
     __syncthreads();
@@ -299,7 +306,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         }
         if (lane == 31) s_wcnt[warp] = winc;
         __syncthreads();
-        int run_gt = sh_gt_before, run_eq = sh_eq_before;
+        // tokens before this warp's range with S > T (always-kept tokens count as such) / S == T
+        int run_gt = sh_gt_before + forced_before(wbd, min((int)rank * 1024 * Lb, n)), run_eq = sh_eq_before;
 #pragma unroll
         for (int w = 0; w < kFusedWarps; ++w)
             if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
@@ -465,8 +473,9 @@ cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapV
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
                               int k_uniform, int max_seq_len, int k_max, uint32_t *q_codes, int32_t *idx,
                               long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
-                              cudaStream_t st) {
+                              cudaStream_t st, Windows win) {
     FusedArgs a{};
+    a.win = win;
     a.map_q = map_q; a.map_k = map_k; a.q = q; a.k_new = k_new; a.K = K; a.V = V;
     a.k_codes = k_codes; a.kc_sb = kc_sb; a.kc_sh = kc_sh; a.seq_lens = seq_lens; a.k_per_seq = k_per_seq;
     a.k_uniform = k_uniform; a.max_seq_len = max_seq_len; a.k_max = k_max; a.Hq = Hq; a.Hkv = Hkv;

@@ -44,6 +44,10 @@ __device__ __forceinline__ int ld_dsmem(const int *local, uint32_t rank) {
 }
 
 
+// Score byte of a token that is always in context (Windows): above every real score + 1 (<= 33), so the
+// flag arithmetic below sees "score > T" for every threshold, and small enough that no byte sum reaches 256.
+constexpr uint32_t kForcedByte = 63u;
+
 // Bits 7, 15, 23, 31 of x gathered into a nibble (bit e = bit 7 of byte e).  The four partial products
 // land on distinct bit positions, so the multiplication carries nothing into bits 28..31.
 __device__ __forceinline__ uint32_t high_bits_to_nibble(uint32_t x) {

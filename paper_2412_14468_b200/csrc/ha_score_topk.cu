@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
                                                                  int max_seq_len, int Hq, int Hkv,
                                                                  int chunk_tokens, long long score_row,
                                                                  unsigned char *__restrict__ ws_scores,
-                                                                 int32_t *__restrict__ ws_hist) {
+                                                                 int32_t *__restrict__ ws_hist, Windows win) {
     __shared__ __align__(16) uint32_t c_hist[kBins][32];
     __shared__ int s_hist[kBins + 3];
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
@@ -48,6 +48,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
     const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
     uint32_t *srow = reinterpret_cast<uint32_t *>(ws_scores + ((long long)b * Hkv + g) * score_row);
     const int end = min(n, start + chunk_tokens);
+    const WindowBounds wbd = window_bounds(win, n);   // always-kept tokens: byte kForcedByte, not counted
 
     // pass = 4096 tokens: sub-block j of 1024 tokens, one uint4 per thread (coalesced)
     auto load_pass = [&](uint4 (&c)[4], int pass) {
@@ -88,13 +89,17 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
                 const int h0 = hamming(cur[j].x), h1 = hamming(cur[j].y), h2 = hamming(cur[j].z), h3 = hamming(cur[j].w);
                 // bytes 33 - h = score + 1 (0 = no token); no byte borrows because h <= 32
                 uint32_t s4 = 0x21212121u - ((uint32_t)h0 | ((uint32_t)h1 << 8) | ((uint32_t)h2 << 16) | ((uint32_t)h3 << 24));
-                if (base + 3 < end) {                    // whole uint4 inside the chunk: no per-token checks
-                    bump(h0); bump(h1); bump(h2); bump(h3);
+                if (base + 3 < end && base >= wbd.sink_end && base + 4 <= wbd.local_begin) {
+                    bump(h0); bump(h1); bump(h2); bump(h3);   // whole uint4 inside the chunk, outside the windows
                 } else {
-                    if (base + 0 < end) bump(h0); else s4 &= 0xffffff00u;
-                    if (base + 1 < end) bump(h1); else s4 &= 0xffff00ffu;
-                    if (base + 2 < end) bump(h2); else s4 &= 0xff00ffffu;
-                    if (base + 3 < end) bump(h3); else s4 &= 0x00ffffffu;
+                    const int hh[4] = {h0, h1, h2, h3};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int t = base + e;
+                        if (t >= end) s4 &= ~(0xffu << (8 * e));                           // zero byte: no token
+                        else if (t < wbd.sink_end || t >= wbd.local_begin) s4 = (s4 & ~(0xffu << (8 * e))) | (kForcedByte << (8 * e));
+                        else bump(hh[e]);
+                    }
                 }
                 srow[base >> 2] = s4;
             }
@@ -122,7 +127,7 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
                                                              const int32_t *__restrict__ ws_hist,
                                                              int32_t *__restrict__ idx, long long idx_sb,
                                                              long long idx_sh, int32_t *__restrict__ count,
-                                                             int32_t *__restrict__ hist_out) {
+                                                             int32_t *__restrict__ hist_out, Windows win) {
     __shared__ int s_tot[kBins + 3], s_bef[kBins + 3];
     __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
     __shared__ int warp_tot[kScanThreads / 32];
@@ -130,8 +135,10 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = max(min(seq_lens[b], max_seq_len), 0);
     int k = k_per_seq ? k_per_seq[b] : k_uniform;
-    k = max(0, min(k, k_max));
-    const int keep = min(k, n);
+    const WindowBounds wbd = window_bounds(win, n);
+    const int n_forced = forced_before(wbd, n);
+    const int keep_rest = max(0, min(min(k, k_max - n_forced), n - n_forced));   // heavy tokens among the others
+    const int keep = n_forced + keep_rest;
     const int n_chunks = (n + chunk_tokens - 1) / chunk_tokens;
     if (chunk > 0 && chunk >= n_chunks) return;
     if (tid < kBins + 3) { s_tot[tid] = 0; s_bef[tid] = 0; }
@@ -172,7 +179,7 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
         // give #{S >= t}; T = largest level with #{S >= T} >= keep; r = keep - #{S > T}.
         const int tot = s_tot[lane], bef = s_bef[lane], tot32 = s_tot[32], bef32 = s_bef[32];
         int T, r, gt_before, eq_before;
-        find_threshold(tot, bef, tot32, bef32, keep, lane, T, r, gt_before, eq_before);
+        find_threshold(tot, bef, tot32, bef32, keep_rest, lane, T, r, gt_before, eq_before);
         if (lane == 0) { sh_T = T; sh_r = r; sh_gt_before = gt_before; sh_eq_before = eq_before; }
         if (chunk == 0 && hist_out) {
             hist_out[((long long)b * Hkv + g) * kBins + lane] = tot;
@@ -192,7 +199,8 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
     // score >= T (no byte sum reaches 256).
     const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
     const uint32_t c_gt = 0x7f7f7f7fu - T4, c_ge = 0x80808080u - T4;
-    int run_gt = sh_gt_before, run_eq = sh_eq_before;   // tokens before this pass with S > T / S == T
+    // tokens before this pass with S > T (always-kept tokens count as such) / S == T
+    int run_gt = sh_gt_before + forced_before(wbd, start), run_eq = sh_eq_before;
     for (int pass = start; pass < end; pass += kPassTokens) {
         const int base = pass + tid * 16;
         const uint4 sv = sv_next;
@@ -265,7 +273,7 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
     const uint32_t *__restrict__ q_codes, const uint32_t *__restrict__ k_codes, long long kc_sb, long long kc_sh,
     const int32_t *__restrict__ seq_lens, int max_seq_len, const int32_t *__restrict__ k_per_seq, int k_uniform,
     int k_max, int Hq, int Hkv, int32_t *__restrict__ idx, long long idx_sb, long long idx_sh,
-    int32_t *__restrict__ count, int32_t *__restrict__ hist_out) {
+    int32_t *__restrict__ count, int32_t *__restrict__ hist_out, Windows win) {
     extern __shared__ __align__(16) unsigned char s_sc[];      // score + 1 of this CTA's tokens (0 = no token)
     __shared__ __align__(16) uint32_t c_hist[kBins][32];       // counters [level][lane]
     __shared__ int s_hist[kBins + 3];          // this CTA's histogram, read by the whole cluster
@@ -277,8 +285,10 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = max(min(seq_lens[b], max_seq_len), 0);
     int k = k_per_seq ? k_per_seq[b] : k_uniform;
-    k = max(0, min(k, k_max));
-    const int keep = min(k, n);
+    const WindowBounds wbd = window_bounds(win, n);   // always-kept tokens: byte kForcedByte, not counted
+    const int n_forced = forced_before(wbd, n);
+    const int keep_rest = max(0, min(min(k, k_max - n_forced), n - n_forced));   // heavy tokens among the others
+    const int keep = n_forced + keep_rest;
     const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
     // The sequence's own length is divided over the CS CTAs (ragged batches stay balanced): Rb rows per
     // lane, a warp owns the 256*Rb tokens from wb on, a CTA 2048*Rb; row p of a lane is
@@ -339,10 +349,14 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
         if (whole_row) {
             bump(h0); bump(h1); bump(h2); bump(h3);
         } else {
-            if (t + 0 < n) bump(h0); else s4 &= 0xffffff00u;   // zero byte: no token
-            if (t + 1 < n) bump(h1); else s4 &= 0xffff00ffu;
-            if (t + 2 < n) bump(h2); else s4 &= 0xff00ffffu;
-            if (t + 3 < n) bump(h3); else s4 &= 0x00ffffffu;
+            const int hh[4] = {h0, h1, h2, h3};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int tt = t + e;
+                if (tt >= n) s4 &= ~(0xffu << (8 * e));                                // zero byte: no token
+                else if (tt < wbd.sink_end || tt >= wbd.local_begin) s4 = (s4 & ~(0xffu << (8 * e))) | (kForcedByte << (8 * e));
+                else bump(hh[e]);
+            }
         }
         return s4;
     };
@@ -355,7 +369,7 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
         for (int j = 0; j < 2; ++j) {
             const int p = p0 + j, t = wb + p * 256 + lane * 8;
             if (p < Rb) {
-                const bool whole_row = t + 8 <= n;
+                const bool whole_row = t + 8 <= n && t >= wbd.sink_end && t + 8 <= wbd.local_begin;
                 uint2 w;
                 w.x = score_word(c[2 * j], t, whole_row);
                 w.y = score_word(c[2 * j + 1], t + 4, whole_row);
@@ -391,7 +405,7 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
         int tot = s_tot[lane], bef = s_bef[lane];
         const int tot32 = s_tot[32], bef32 = s_bef[32];
         int T, r, gt_before, eq_before;
-        find_threshold(tot, bef, tot32, bef32, keep, lane, T, r, gt_before, eq_before);
+        find_threshold(tot, bef, tot32, bef32, keep_rest, lane, T, r, gt_before, eq_before);
         if (lane == 0) { sh_T = T; sh_r = r; sh_gt_before = gt_before; sh_eq_before = eq_before; }
         if (rank == 0 && hist_out) {
             hist_out[((long long)b * Hkv + g) * kBins + lane] = tot;
@@ -434,7 +448,8 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
     }
     if (lane == 31) s_wcnt[warp] = winc;
     __syncthreads();
-    int run_gt = sh_gt_before, run_eq = sh_eq_before;   // tokens before this warp's range
+    // tokens before this warp's range with S > T (always-kept tokens count as such) / S == T
+    int run_gt = sh_gt_before + forced_before(wbd, min((int)rank * 2048 * Rb, n)), run_eq = sh_eq_before;
 #pragma unroll
     for (int w = 0; w < kScanThreads / 32; ++w) {
         if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
@@ -455,7 +470,7 @@ static cudaError_t launch_cluster_t(int rows, int B, int Hq, int Hkv, const uint
                                     long long kc_sb, long long kc_sh, const int32_t *seq_lens,
                                     const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max, int32_t *idx,
                                     long long idx_sb, long long idx_sh, int32_t *count, int32_t *hist_out,
-                                    cudaStream_t st) {
+                                    cudaStream_t st, Windows win) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CS, Hkv, B);
     cfg.blockDim = dim3(kScanThreads);
@@ -472,7 +487,7 @@ static cudaError_t launch_cluster_t(int rows, int B, int Hq, int Hkv, const uint
     cfg.numAttrs = 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, score_select_cluster_kernel<G, CS>, q_codes, k_codes, kc_sb, kc_sh,
                                        seq_lens, max_seq_len, k_per_seq, k_uniform, k_max, Hq, Hkv, idx, idx_sb, idx_sh,
-                                       count, hist_out);
+                                       count, hist_out, win);
     if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
@@ -483,7 +498,7 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
                             long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
                             int k_uniform, int max_seq_len, int k_max, int32_t *idx, long long idx_sb,
                             long long idx_sh, int32_t *count, int32_t *hist_out, int32_t *ws_hist,
-                            unsigned char *ws_scores, cudaStream_t st) {
+                            unsigned char *ws_scores, cudaStream_t st, Windows win) {
     if (max_seq_len <= kClusterMaxSeq) {
         // Fused path: one cluster per unit.  Cluster size: the largest of 8, 4, 2 whose grid still fits
         // the GPU in one wave (about six 256-thread CTAs per SM), so that small batches get the most
@@ -496,7 +511,7 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
         const int rows = max(1, (max_seq_len + cs * 2048 - 1) / (cs * 2048));
 #define HA_CL(CSZ)                                                                                                    \
     return launch_cluster_t<G, CSZ>(rows, B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform, \
-                                    max_seq_len, k_max, idx, idx_sb, idx_sh, count, hist_out, st)
+                                    max_seq_len, k_max, idx, idx_sb, idx_sh, count, hist_out, st, win)
         if (cs == 8) HA_CL(8);
         if (cs == 4) HA_CL(4);
         HA_CL(2);
@@ -507,11 +522,11 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
     const long long score_row = (long long)score_row_bytes(max_seq_len);
     dim3 grid(n_chunks, Hkv, B);
     cudaError_t e = launch_pdl(scan_score_kernel<G>, grid, dim3(kScanThreads), 0, st, q_codes, k_codes, kc_sb, kc_sh,
-                               seq_lens, max_seq_len, Hq, Hkv, chunk_tokens, score_row, ws_scores, ws_hist);
+                               seq_lens, max_seq_len, Hq, Hkv, chunk_tokens, score_row, ws_scores, ws_hist, win);
     if (e != cudaSuccess) return e;
     e = launch_pdl(select_kernel, grid, dim3(kScanThreads), 0, st, seq_lens, max_seq_len, k_per_seq, k_uniform, k_max,
                    Hkv, chunk_tokens, score_row, (const unsigned char *)ws_scores, (const int32_t *)ws_hist, idx, idx_sb,
-                   idx_sh, count, hist_out);
+                   idx_sh, count, hist_out, win);
     if (e != cudaSuccess) return e;
     count_launch(2);
     return cudaGetLastError();
@@ -521,9 +536,9 @@ cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, c
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens,
                               const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max,
                               int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
-                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st) {
+                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st, Windows win) {
 #define HA_ARGS B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx, \
-                idx_sb, idx_sh, count, hist_out, ws_hist, ws_scores, st
+                idx_sb, idx_sh, count, hist_out, ws_hist, ws_scores, st, win
     switch (Hq / Hkv) {
         case 1: return launch_g<1>(HA_ARGS);
         case 2: return launch_g<2>(HA_ARGS);

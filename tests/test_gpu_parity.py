@@ -98,11 +98,11 @@ def test_encode_without_biases_and_strided_input():
 
 # ---------------------------------------------------------------------------- SCORE + TOPK
 
-def _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, k_uniform=None):
+def _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, k_uniform=None, n_sink=0, n_local=0):
     B = len(lens)
     n_cap = kc_np.shape[2]
-    k_max = max(max(ks), 1)
-    shape = ha.make_shape(B, Hq, Hkv, 1.0)
+    k_max = max(max(ks) + n_sink + n_local, 1)
+    shape = ha.make_shape(B, Hq, Hkv, 1.0, n_sink=n_sink, n_local=n_local)
     ws = ha.alloc_workspace(shape, n_cap, k_max)
     qc = torch.from_numpy(qc_np.view(np.int32)).to(DEV)
     kc = torch.from_numpy(kc_np.view(np.int32)).to(DEV)
@@ -117,17 +117,26 @@ def _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, k_uniform=None):
     return idx.cpu().numpy(), cnt.cpu().numpy(), hist.cpu().numpy()
 
 
-def _check_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, **kw):
-    idx, cnt, hist = _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, **kw)
+def _check_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, n_sink=0, n_local=0, **kw):
+    idx, cnt, hist = _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, n_sink=n_sink, n_local=n_local, **kw)
     G = Hq // Hkv
     for b, (n, k) in enumerate(zip(lens, ks)):
         for g in range(Hkv):
             s = oracle.score(qc_np[b, g * G:(g + 1) * G], kc_np[b, g, :n])
-            exp = oracle.topk(s, k)
-            assert cnt[b, g] == len(exp) == min(k, n)
-            assert np.array_equal(idx[b, g, :len(exp)], exp), (b, g, n, k)
+            if n_sink == 0 and n_local == 0:
+                exp = oracle.topk(s, k)
+                assert cnt[b, g] == len(exp) == min(k, n)
+                others = s
+            else:
+                exp = oracle.topk_windows(s, k, n_sink, n_local)
+                forced = np.zeros(n, bool)
+                forced[:n_sink] = True
+                forced[max(n - n_local, 0):] = True
+                assert cnt[b, g] == len(exp) == forced.sum() + min(k, n - forced.sum())
+                others = s[~forced]
+            assert np.array_equal(idx[b, g, :len(exp)], exp), (b, g, n, k, n_sink, n_local)
             assert np.all(idx[b, g, len(exp):] == -1)
-            assert np.array_equal(hist[b, g], np.bincount(s, minlength=33))
+            assert np.array_equal(hist[b, g], np.bincount(others, minlength=33))
 
 
 @pytest.mark.parametrize("G", [1, 4])
@@ -153,6 +162,40 @@ def test_score_topk_long_sequences(lens, n_cap):
     qc = rng.integers(0, 2 ** 32, size=(len(lens), Hq), dtype=np.uint64).astype(np.uint32)
     for ks in ([n // 32 for n in lens], [3, lens[1], 20]):
         _check_score_topk(qc, kc, lens, ks, Hq, Hkv)
+
+
+@pytest.mark.parametrize("n_sink,n_local", [(128, 128), (1, 0), (0, 3), (5000, 7), (300, 70000)])
+def test_score_topk_with_always_kept_windows(n_sink, n_local):
+    """First n_sink and most recent n_local tokens always selected, the budget on top (Section 5, baselines):
+    sequences shorter than a window, windows that overlap, the cluster kernel at every cluster size and the
+    two-kernel path."""
+    rng = np.random.default_rng(21 + n_sink)
+    Hkv, Hq = 2, 8
+    lens = [0, 1, 5, 100, 255, 256, 257, 2049, 5000, 70001, 140001]
+    n_cap = 140004
+    kc = rng.integers(0, 2 ** 32, size=(len(lens), Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    qc = rng.integers(0, 2 ** 32, size=(len(lens), Hq), dtype=np.uint64).astype(np.uint32)
+    for ks in ([n // 16 for n in lens], [0] * len(lens), [n for n in lens]):
+        _check_score_topk(qc, kc, lens, ks, Hq, Hkv, n_sink=n_sink, n_local=n_local)
+    short = [n for n in lens if n <= 5000]          # shorter batch: the cluster kernel with clusters of 8 and 4
+    _check_score_topk(qc[:len(short)], kc[:len(short), :, :5000].copy(), short, [n // 8 for n in short], Hq, Hkv,
+                      n_sink=n_sink, n_local=n_local)
+
+
+def test_score_topk_windows_with_heavy_ties_and_small_k_max():
+    rng = np.random.default_rng(12)
+    Hq, Hkv, n = 8, 2, 9000
+    pool = rng.integers(0, 2 ** 32, size=4, dtype=np.uint64).astype(np.uint32)
+    kc = pool[rng.integers(0, 4, size=(2, Hkv, n))]
+    qc = rng.integers(0, 2 ** 32, size=(2, Hq), dtype=np.uint64).astype(np.uint32)
+    for k in (1, 100, 4500):
+        _check_score_topk(qc, kc, [n, n - 13], [k, k], Hq, Hkv, k_uniform=k, n_sink=128, n_local=128)
+    # windows that do not fit the index rows are refused on the host
+    shape = ha.make_shape(2, Hq, Hkv, 1.0, n_sink=128, n_local=128)
+    ws = ha.alloc_workspace(shape, n, 256)
+    t = lambda *s_: torch.zeros(*s_, dtype=torch.int32, device=DEV)
+    with pytest.raises(RuntimeError):
+        ha.ha_score_topk(shape, t(2, Hq), t(2, Hkv, n), t(2), None, 10, n, 200, t(2, Hkv, 200), t(2, Hkv), ws)
 
 
 def test_score_topk_heavy_ties():
@@ -300,10 +343,12 @@ def test_dense_decode_matches_oracle(lens):
 
 # ---------------------------------------------------------------------------- whole step
 
-def _run_step(w, host=False, pinned=True):
+def _run_step(w, host=False, pinned=True, n_sink=0, n_local=0):
     cfg = w["cfg"]
     B, Hq, Hkv = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads
-    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"], n_sink=n_sink, n_local=n_local)
+    if n_sink or n_local:
+        w = dict(w, k_max=w["k_max"] + n_sink + n_local)             # the index rows hold the windows too
     ws = ha.alloc_workspace(shape, w["n_cap"], w["k_max"])
     mq, mk = ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"])
     kc = torch.zeros(B, Hkv, (w["n_cap"] + 3) // 4 * 4, dtype=torch.int32, device=DEV)
@@ -366,6 +411,31 @@ def test_sparse_decode_step_matches_oracle(cfg):
     for pinned in (True, False):
         rh = _run_step(w, host=True, pinned=pinned)
         assert torch.equal(rh["idx"], r["idx"]) and torch.equal(rh["out"], r["out"])
+
+
+@pytest.mark.parametrize("cfg", [
+    wl.Config("win-ragged", 55, 3, [300, 2049, 1], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8),     # one fused launch
+    wl.Config("win-batch", 56, 24, [900 + 37 * i for i in range(24)], None, 0.02, n_q_heads=8, n_kv_heads=2,
+              sparsity=8),                                                                                  # three kernels
+    wl.CONFIGS["c1"],
+])
+@pytest.mark.parametrize("n_sink,n_local", [(128, 128), (4, 500)])
+def test_sparse_decode_step_with_always_kept_windows(cfg, n_sink, n_local):
+    w = wl.make_workload(cfg, DEV)
+    r = _run_step(w, n_sink=n_sink, n_local=n_local)
+    Kc = oracle_key_codes(w["K"], w["map_k"], w["lens"])
+    ref = oracle.decode_step(u16(w["q"]), u16(w["k_new"]), u16(w["K"]), u16(w["V"]), Kc.copy(),
+                             wl.mapping_numpy(w["map_q"]), wl.mapping_numpy(w["map_k"]), w["lens"], w["ks"],
+                             sm_scale=w["sm_scale"], n_threads=4, n_sink=n_sink, n_local=n_local)
+    assert np.array_equal(r["cnt"].cpu().numpy(), ref["count"])
+    assert np.array_equal(r["idx"].cpu().numpy(), ref["idx"])
+    for b, n in enumerate(w["lens"]):                                # the windows really are in every list
+        for g in range(cfg.n_kv_heads):
+            got = set(r["idx"][b, g, :int(r["cnt"][b, g])].tolist())
+            assert set(range(min(n_sink, n))) <= got and set(range(max(n - n_local, 0), n)) <= got
+    assert_out_close(u16(r["out"]), ref["out"])
+    rh = _run_step(w, host=True, n_sink=n_sink, n_local=n_local)
+    assert torch.equal(rh["idx"], r["idx"]) and torch.equal(rh["out"], r["out"])
 
 
 def test_k_equals_n_sparse_step_equals_dense_kernel():
