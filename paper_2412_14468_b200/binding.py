@@ -21,7 +21,7 @@ HA_DEV_BAD_INDEX, HA_DEV_TIMEOUT = 1, 2
 HIST_BINS = 33
 
 EXPORTS = [
-    "ha_workspace_bytes", "ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn",
+    "ha_workspace_bytes", "ha_workspace_init", "ha_encode", "ha_encode_prefill", "ha_score_topk", "ha_gather_attn",
     "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
@@ -64,6 +64,7 @@ def lib() -> C.CDLL:
         L.ha_workspace_bytes.argtypes = [P, I32, I32]
         L.ha_workspace_init.argtypes = [P, SZ, P]
         L.ha_encode.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, P, P]
+        L.ha_encode_prefill.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, P]
         L.ha_score_topk.argtypes = [P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64, P, P, P, SZ, P]
         L.ha_gather_attn.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P, SZ, P]
         L.ha_gather_attn_static.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P]
@@ -187,6 +188,17 @@ def ha_encode(mapping: Mapping, heads_per_kv: int, x: torch.Tensor, codes: torch
     assert codes.dim() == 3 and codes.stride(2) == 1
     _check("ha_encode", lib().ha_encode(mapping.ref, heads_per_kv, C.byref(xt), B, H, T, codes.data_ptr(),
                                         codes.stride(0), codes.stride(1), _ptr(slot), _stream(stream)))
+
+
+def ha_encode_prefill(mapping: Mapping, heads_per_kv: int, x: torch.Tensor, codes: torch.Tensor, stream=None) -> None:
+    """Tensor-core ENCODE of whole prompts; x: bf16 [B,H,T,128]; codes: int32 [B,H,>=T] (last dim contiguous)."""
+    xt = make_tensor(x)
+    B, H = x.shape[0], x.shape[1]
+    T = 1 if x.dim() == 3 else x.shape[2]
+    _dev(codes, torch.int32, "codes")
+    assert codes.dim() == 3 and codes.stride(2) == 1
+    _check("ha_encode_prefill", lib().ha_encode_prefill(mapping.ref, heads_per_kv, C.byref(xt), B, H, T, codes.data_ptr(),
+                                                        codes.stride(0), codes.stride(1), _stream(stream)))
 
 
 def ha_score_topk(shape: ha_shape, q_codes, k_codes, seq_lens, k_per_seq, k_uniform: int, max_seq_len: int,

@@ -116,6 +116,18 @@ int ha_encode(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, i
     return HA_OK;
 }
 
+int ha_encode_prefill(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, int32_t batch, int32_t n_heads,
+                      int32_t n_tokens, uint32_t *codes, int64_t c_stride_b, int64_t c_stride_h, void *stream) {
+    HA_TRY(check_mapping(map, 0));
+    HA_TRY(check_tensor(x));
+    if (!codes || batch < 0 || n_heads <= 0 || n_tokens < 0 || heads_per_kv <= 0) return HA_ERR_INVALID_ARG;
+    if (n_heads % heads_per_kv != 0 || n_heads / heads_per_kv != map->n_kv_heads) return HA_ERR_INVALID_ARG;
+    if (batch == 0 || n_tokens == 0) return HA_OK;
+    HA_CUDA(launch_encode_tc(view(map), heads_per_kv, view(x), batch, n_heads, n_tokens, codes, c_stride_b, c_stride_h,
+                             (cudaStream_t)stream));
+    return HA_OK;
+}
+
 static int check_score_args(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes,
                             int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens, int32_t k_uniform,
                             const int32_t *k_per_seq, int32_t max_seq_len, int32_t k_max, int32_t *idx,
