@@ -122,14 +122,21 @@ int ha_encode(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, i
 /* ENCODE of whole prompts on the tensor cores — the signature cache of n_tokens tokens per head at
  * once (Section 4.1 "Implementation": signatures are computed and cached along with the KV cache;
  * Section 5.2 names these matrix multiplications as the latency bottleneck at short contexts).
- * Same arguments as ha_encode without `slot`.  The three layers run as bf16 tensor-core GEMMs with
- * fp32 accumulation; hidden activations enter the next layer as a bf16 pair hi + lo.  The sums are
+ * Arguments as ha_encode without `slot`.  The three layers run as bf16 tensor-core GEMMs with fp32
+ * accumulation; hidden activations enter the next layer as a bf16 pair hi + lo.  The sums are
  * therefore NOT the fused-multiply-add chain of ha_encode: a signature bit may differ from
  * ha_encode's where the exact last-layer output lies within about 1e-5 of zero, and is identical
- * everywhere else.  Use ha_encode where bit-exact agreement with the decode step matters. */
+ * everywhere else.  Use ha_encode where bit-exact agreement with the decode step matters.
+ *   path       HA_PREFILL_TCGEN05: tcgen05.mma with the accumulators and the hidden activations in
+ *              tensor memory; HA_PREFILL_MMA_SYNC: warp-level mma.sync with the activations chained
+ *              through registers (the earlier tensor-core generation's path, kept for comparison)
+ *   workspace  optional (may be NULL): a workspace from ha_workspace_bytes; if the tcgen05 kernel
+ *              gives up waiting for its tensor cores it raises HA_DEV_TIMEOUT in its status word */
+#define HA_PREFILL_TCGEN05 0
+#define HA_PREFILL_MMA_SYNC 1
 int ha_encode_prefill(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, int32_t batch,
                       int32_t n_heads, int32_t n_tokens, uint32_t *codes, int64_t c_stride_b,
-                      int64_t c_stride_h, void *stream);
+                      int64_t c_stride_h, int32_t path, void *workspace, void *stream);
 
 /* SCORE + TOPK — Eq. 1 as s = 32 - bitcount(k_code xor q_code) (Section 4.1), group score =
  * max over the G query heads of the KV head, then the standard top-k (Section 4) with ties

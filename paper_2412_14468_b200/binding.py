@@ -64,7 +64,7 @@ def lib() -> C.CDLL:
         L.ha_workspace_bytes.argtypes = [P, I32, I32]
         L.ha_workspace_init.argtypes = [P, SZ, P]
         L.ha_encode.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, P, P]
-        L.ha_encode_prefill.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, P]
+        L.ha_encode_prefill.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, I32, P, P]
         L.ha_score_topk.argtypes = [P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64, P, P, P, SZ, P]
         L.ha_gather_attn.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P, SZ, P]
         L.ha_gather_attn_static.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P]
@@ -190,7 +190,11 @@ def ha_encode(mapping: Mapping, heads_per_kv: int, x: torch.Tensor, codes: torch
                                         codes.stride(0), codes.stride(1), _ptr(slot), _stream(stream)))
 
 
-def ha_encode_prefill(mapping: Mapping, heads_per_kv: int, x: torch.Tensor, codes: torch.Tensor, stream=None) -> None:
+HA_PREFILL_TCGEN05, HA_PREFILL_MMA_SYNC = 0, 1
+
+
+def ha_encode_prefill(mapping: Mapping, heads_per_kv: int, x: torch.Tensor, codes: torch.Tensor,
+                      path: int = HA_PREFILL_TCGEN05, workspace: Optional[torch.Tensor] = None, stream=None) -> None:
     """Tensor-core ENCODE of whole prompts; x: bf16 [B,H,T,128]; codes: int32 [B,H,>=T] (last dim contiguous)."""
     xt = make_tensor(x)
     B, H = x.shape[0], x.shape[1]
@@ -198,7 +202,8 @@ def ha_encode_prefill(mapping: Mapping, heads_per_kv: int, x: torch.Tensor, code
     _dev(codes, torch.int32, "codes")
     assert codes.dim() == 3 and codes.stride(2) == 1
     _check("ha_encode_prefill", lib().ha_encode_prefill(mapping.ref, heads_per_kv, C.byref(xt), B, H, T, codes.data_ptr(),
-                                                        codes.stride(0), codes.stride(1), _stream(stream)))
+                                                        codes.stride(0), codes.stride(1), path, _ptr(workspace),
+                                                        _stream(stream)))
 
 
 def ha_score_topk(shape: ha_shape, q_codes, k_codes, seq_lens, k_per_seq, k_uniform: int, max_seq_len: int,

@@ -117,14 +117,21 @@ int ha_encode(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, i
 }
 
 int ha_encode_prefill(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, int32_t batch, int32_t n_heads,
-                      int32_t n_tokens, uint32_t *codes, int64_t c_stride_b, int64_t c_stride_h, void *stream) {
+                      int32_t n_tokens, uint32_t *codes, int64_t c_stride_b, int64_t c_stride_h, int32_t path,
+                      void *workspace, void *stream) {
     HA_TRY(check_mapping(map, 0));
     HA_TRY(check_tensor(x));
     if (!codes || batch < 0 || n_heads <= 0 || n_tokens < 0 || heads_per_kv <= 0) return HA_ERR_INVALID_ARG;
     if (n_heads % heads_per_kv != 0 || n_heads / heads_per_kv != map->n_kv_heads) return HA_ERR_INVALID_ARG;
+    if (path != HA_PREFILL_TCGEN05 && path != HA_PREFILL_MMA_SYNC) return HA_ERR_INVALID_ARG;
+    if (workspace && ((uintptr_t)workspace & 255)) return HA_ERR_WORKSPACE;
     if (batch == 0 || n_tokens == 0) return HA_OK;
-    HA_CUDA(launch_encode_tc(view(map), heads_per_kv, view(x), batch, n_heads, n_tokens, codes, c_stride_b, c_stride_h,
-                             (cudaStream_t)stream));
+    if (path == HA_PREFILL_MMA_SYNC)
+        HA_CUDA(launch_encode_tc(view(map), heads_per_kv, view(x), batch, n_heads, n_tokens, codes, c_stride_b, c_stride_h,
+                                 (cudaStream_t)stream));
+    else
+        HA_CUDA(launch_encode_umma(view(map), heads_per_kv, view(x), batch, n_heads, n_tokens, codes, c_stride_b,
+                                   c_stride_h, reinterpret_cast<uint32_t *>(workspace), (cudaStream_t)stream));
     return HA_OK;
 }
 

@@ -168,6 +168,8 @@ cudaError_t launch_encode_bulk(const MapView &map, int heads_per_kv, TensorView 
                                uint32_t *codes, long long c_sb, long long c_sh, cudaStream_t st);
 cudaError_t launch_encode_tc(const MapView &map, int heads_per_kv, TensorView x, int B, int H, int T, uint32_t *codes,
                              long long c_sb, long long c_sh, cudaStream_t st);
+cudaError_t launch_encode_umma(const MapView &map, int heads_per_kv, TensorView x, int B, int H, int T, uint32_t *codes,
+                               long long c_sb, long long c_sh, uint32_t *status, cudaStream_t st);
 
 cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes,
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens,

@@ -213,4 +213,301 @@ cudaError_t launch_encode_tc(const MapView &map, int heads_per_kv, TensorView x,
     return cudaGetLastError();
 }
 
+
+// ------------------------------------------------------------------ tcgen05 version
+//
+// The same chain of three GEMMs on the fifth-generation tensor cores.  One CTA of 128 threads
+// owns a tile of 128 tokens: M = 128 rows = the 128 lanes of tensor memory, thread r owns row r.
+//   layer 1  D1[128 x 128] = X W1      A = token tile in shared memory (K-major core matrices),
+//                                      B = W1 in shared memory (N-major core matrices), 8 x K16
+//   epilogue threads read their row of D1 (tcgen05.ld), add the bias, apply ReLU, split into a bf16
+//            pair hi + lo and write both back to tensor memory as the next A operand (tcgen05.st)
+//   layer 2  D2 = A_hi W2 + A_lo W2    A from tensor memory, 16 x K16
+//   layer 3  D3[128 x 32] likewise; the epilogue packs the 32 sign bits of a row into its code.
+// Activations never leave tensor memory and registers.  Tensor memory use: 128 columns D1 / D3,
+// 128 columns A (64 hi + 64 lo), 128 columns D2 = 384 of the 512 allocated; two CTAs cannot share an
+// SM (shared memory), so the whole allocation is free to take.
+// MMAs are issued by thread 0 and tracked by one mbarrier (tcgen05.commit); every wait on it is
+// bounded: on a timeout the CTA raises HA_DEV_TIMEOUT in the status word, stops issuing work,
+// frees its tensor memory and returns.
+
+constexpr int kU_Threads = 128;
+constexpr int kU_WBytes = kD * kHid * 2;          // 32768: W1 or W2 as 16 k-groups x 16 n-blocks x (8 x 16 B)
+constexpr int kU_W3Bytes = kHid * kBits * 2;      // 8192
+constexpr int kU_XBytes = kTcTile * kD * 2;       // 32768: 16 k-chunks x 16 row-groups x (8 x 16 B)
+constexpr int kU_Smem = 2 * kU_WBytes + kU_W3Bytes + 2 * kU_XBytes + 1024;
+constexpr uint32_t kU_TmemCols = 512;
+constexpr uint32_t kU_ColD1 = 0, kU_ColA = 128, kU_ColD2 = 256;   // column offsets inside the allocation
+
+// 64-bit shared-memory matrix descriptor, no swizzle: start address, leading and stride byte offsets
+// in 16-byte units, descriptor version 1 (bits 46-47), layout type 0 (bits 61-63).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((smem_addr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | (1ull << 46);
+}
+// 32-bit instruction descriptor of kind::f16: fp32 accumulate (bits 4-5 = 1), A and B bf16 (bits 7-9 and
+// 10-12 = 1), A K-major (bit 15 = 0), B N-major (bit 16 = 1), N / 8 in bits 17-22, M / 16 in bits 24-28.
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// 32 consecutive 32-bit columns of this thread's lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+                   "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+                   "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+                   "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
+                 ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+                   "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
+                   "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
+                   "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ bool mbar_wait_parity_bounded(uint32_t bar, uint32_t parity) {
+    for (int it = 0; it < (1 << 22); ++it) {   // non-blocking probes: a few tenths of a second at most
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+__global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map, int heads_per_kv, TensorView x, int B,
+                                                                   int H, int T, uint32_t *__restrict__ codes,
+                                                                   long long c_sb, long long c_sh,
+                                                                   uint32_t *__restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char usm[];
+    unsigned char *sW1 = usm, *sW2 = sW1 + kU_WBytes, *sW3 = sW2 + kU_WBytes, *sX = sW3 + kU_W3Bytes;
+    __shared__ __align__(8) unsigned long long s_mbar;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_fail;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tiles_per_row = (T + kTcTile - 1) / kTcTile;
+    const long long n_work = (long long)H * B * tiles_per_row;   // head-major order: a CTA keeps its weights
+    const long long w_lo = n_work * blockIdx.x / gridDim.x, w_hi = n_work * (blockIdx.x + 1) / gridDim.x;
+    if (w_lo >= w_hi) return;
+    const uint32_t bar = smem_u32(&s_mbar);
+
+    if (tid == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s_fail = 0;
+    }
+    if (warp == 0) {   // one warp allocates the tensor memory and passes the allocation right on
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)), "r"(kU_TmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base;
+    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
+
+    auto decode = [&](long long w, int &h, int &b, int &t0) {
+        const long long per_head = (long long)B * tiles_per_row;
+        h = (int)(w / per_head);
+        const long long r = w - (long long)h * per_head;
+        b = (int)(r / tiles_per_row);
+        t0 = (int)(r - (long long)b * tiles_per_row) * kTcTile;
+    };
+    // token tile, K-major core matrices: element (row r, k) at (k/8) * 2048 + (r/8) * 128 + (r%8) * 16 + (k%8) * 2
+    auto load_x = [&](long long w, int buf) {
+        int h, b, t0;
+        decode(w, h, b, t0);
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(x.ptr + (long long)b * x.sb + (long long)h * x.sh);
+        const uint32_t dst = smem_u32(sX + buf * kU_XBytes);
+#pragma unroll
+        for (int i = 0; i < kTcTile * 16 / kU_Threads; ++i) {
+            const int e = tid + i * kU_Threads, row = e >> 4, ch = e & 15;
+            const bool ok = t0 + row < T;
+            cp_async16(dst + ch * 2048 + (row >> 3) * 128 + (row & 7) * 16,
+                       src + (long long)(ok ? t0 + row : 0) * x.sn * 2 + ch * 16, ok ? 16u : 0u);
+        }
+    };
+    // weights [k][n], N-major core matrices: element (k, n) at (k/8) * LBO + (n/8) * 128 + (k%8) * 16 + (n%8) * 2
+    auto load_weights = [&](int net) {
+        const unsigned char *g1 = reinterpret_cast<const unsigned char *>(map.w1 + (size_t)net * kD * kHid);
+        const unsigned char *g2 = reinterpret_cast<const unsigned char *>(map.w2 + (size_t)net * kHid * kHid);
+        const unsigned char *g3 = reinterpret_cast<const unsigned char *>(map.w3 + (size_t)net * kHid * kBits);
+        for (int e = tid; e < kD * 16; e += kU_Threads) {   // 16 chunks of 8 outputs per row k
+            const int k = e >> 4, nb = e & 15;
+            const uint32_t off = (k >> 3) * 2048 + nb * 128 + (k & 7) * 16;
+            cp_async16(smem_u32(sW1) + off, g1 + (size_t)e * 16, 16u);
+            cp_async16(smem_u32(sW2) + off, g2 + (size_t)e * 16, 16u);
+        }
+        for (int e = tid; e < kHid * 4; e += kU_Threads) {  // 4 chunks per row k
+            const int k = e >> 2, nb = e & 3;
+            cp_async16(smem_u32(sW3) + (k >> 3) * 512 + nb * 128 + (k & 7) * 16, g3 + (size_t)e * 16, 16u);
+        }
+    };
+
+    constexpr uint32_t kIdesc128 = umma_idesc(128, 128), kIdesc32 = umma_idesc(128, 32);
+    uint32_t phase = 0;
+    bool failed = false;
+    // wait for the MMAs committed last; CTA-uniform result
+    auto wait_mma = [&]() -> bool {
+        const bool ok = mbar_wait_parity_bounded(bar, phase);
+        phase ^= 1u;
+        if (!ok) s_fail = 1;
+        tc_fence_after();
+        __syncthreads();
+        return s_fail == 0;
+    };
+    // this thread's row of a 128-column accumulator -> bias, ReLU, hi / lo -> the A operand columns
+    auto epilogue_hidden = [&](uint32_t col_d, const float *bias) {
+        uint32_t hi[64], lo[64];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint32_t v[32];
+            tmem_ld32(lane_base + col_d + q * 32, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int o = q * 32 + 2 * i;
+                const float z0 = __uint_as_float(v[2 * i]) + (bias ? __ldg(bias + o) : 0.0f);
+                const float z1 = __uint_as_float(v[2 * i + 1]) + (bias ? __ldg(bias + o + 1) : 0.0f);
+                split_relu(z0, z1, hi[q * 16 + i], lo[q * 16 + i]);
+            }
+        }
+        {
+            uint32_t t[32];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) t[i] = hi[q * 32 + i];
+                tmem_st32(lane_base + kU_ColA + q * 32, t);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) t[i] = lo[q * 32 + i];
+                tmem_st32(lane_base + kU_ColA + 64 + q * 32, t);
+            }
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        __syncthreads();
+    };
+
+    int cur_net = -1;
+    load_x(w_lo, 0);
+    cp_async_commit();
+    int buf = 0;
+    for (long long w = w_lo; w < w_hi && !failed; ++w, buf ^= 1) {
+        int h, b, t0;
+        decode(w, h, b, t0);
+        const int net = h / heads_per_kv;
+        if (net != cur_net) {
+            load_weights(net);
+            cur_net = net;
+        }
+        cp_async_commit();      // group of the weights (empty when they stay)
+        if (w + 1 < w_hi) load_x(w + 1, buf ^ 1);
+        cp_async_commit();      // group of the next tile (empty after the last one)
+        cp_async_wait<1>();     // this tile and the weights have landed
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ordinary writes -> visible to the tensor cores
+        __syncthreads();
+
+        const float *bias1 = map.b1 ? map.b1 + net * kHid : nullptr;
+        const float *bias2 = map.b2 ? map.b2 + net * kHid : nullptr;
+        const float *bias3 = map.b3 ? map.b3 + net * kBits : nullptr;
+
+        // ---- layer 1: D1 = X W1 (both operands from shared memory), one MMA per 16 values of k
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t xa = smem_u32(sX + buf * kU_XBytes), wa = smem_u32(sW1);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                umma_ss(tmem + kU_ColD1, umma_desc(xa + ks * 4096, 2048, 128), umma_desc(wa + ks * 4096, 2048, 128),
+                        kIdesc128, ks > 0 ? 1u : 0u);
+            umma_commit(bar);
+        }
+        if (!wait_mma()) { failed = true; break; }
+        epilogue_hidden(kU_ColD1, bias1);
+
+        // ---- layer 2: D2 = A_hi W2 + A_lo W2, A from tensor memory (8 columns per 16 values of k)
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t wa = smem_u32(sW2);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                umma_ts(tmem + kU_ColD2, tmem + kU_ColA + ks * 8, umma_desc(wa + ks * 4096, 2048, 128), kIdesc128, ks > 0 ? 1u : 0u);
+                umma_ts(tmem + kU_ColD2, tmem + kU_ColA + 64 + ks * 8, umma_desc(wa + ks * 4096, 2048, 128), kIdesc128, 1u);
+            }
+            umma_commit(bar);
+        }
+        if (!wait_mma()) { failed = true; break; }
+        epilogue_hidden(kU_ColD2, bias2);
+
+        // ---- layer 3: D3[128 x 32] into the columns of D1
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t wa = smem_u32(sW3);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                umma_ts(tmem + kU_ColD1, tmem + kU_ColA + ks * 8, umma_desc(wa + ks * 1024, 512, 128), kIdesc32, ks > 0 ? 1u : 0u);
+                umma_ts(tmem + kU_ColD1, tmem + kU_ColA + 64 + ks * 8, umma_desc(wa + ks * 1024, 512, 128), kIdesc32, 1u);
+            }
+            umma_commit(bar);
+        }
+        if (!wait_mma()) { failed = true; break; }
+        {
+            uint32_t v[32];
+            tmem_ld32(lane_base + kU_ColD1, v);
+            tmem_wait_ld();
+            uint32_t code = 0u;
+#pragma unroll
+            for (int o = 0; o < 32; ++o) {
+                const float z = __uint_as_float(v[o]) + (bias3 ? __ldg(bias3 + o) : 0.0f);
+                code |= (z > 0.0f ? 1u : 0u) << o;
+            }
+            if (t0 + tid < T) codes[(long long)b * c_sb + (long long)h * c_sh + t0 + tid] = code;
+        }
+        tc_fence_before();
+        __syncthreads();   // every thread is done with this token buffer, these weights and D1 before they are reused
+    }
+    if (failed && tid == 0 && status) atomicOr(status, HA_DEV_TIMEOUT);
+    cp_async_wait<0>();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kU_TmemCols) : "memory");
+    }
+}
+
+cudaError_t launch_encode_umma(const MapView &map, int heads_per_kv, TensorView x, int B, int H, int T, uint32_t *codes,
+                               long long c_sb, long long c_sh, uint32_t *status, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(encode_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kU_Smem);
+    if (e != cudaSuccess) return e;
+    const long long n_work = (long long)H * B * ((T + kTcTile - 1) / kTcTile);
+    if (n_work <= 0) return cudaSuccess;
+    const int grid = (int)((n_work < sm_count()) ? n_work : sm_count());
+    encode_umma_kernel<<<grid, kU_Threads, kU_Smem, st>>>(map, heads_per_kv, x, B, H, T, codes, c_sb, c_sh, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
 } // namespace ha

@@ -96,8 +96,9 @@ def test_encode_without_biases_and_strided_input():
         assert np.array_equal(codes_np(codes)[0, h], oracle.encode(xu[0, h], m["w1"][h], m["w2"][h], m["w3"][h]))
 
 
+@pytest.mark.parametrize("path", [ha.HA_PREFILL_TCGEN05, ha.HA_PREFILL_MMA_SYNC])
 @pytest.mark.parametrize("T,strided", [(1, False), (77, False), (300, True), (4099, False)])
-def test_encode_prefill_on_tensor_cores_matches_the_chain_up_to_its_margin(T, strided):
+def test_encode_prefill_on_tensor_cores_matches_the_chain_up_to_its_margin(T, strided, path):
     """The tensor-core prompt encoder sums in another order and feeds 16-bit activations to the next layer:
     its signature bits must equal the chain-exact ones wherever the exact last-layer output is not within
     1e-3 of zero (the stated accuracy is ~1e-5), and only a tiny share of bits may differ at all."""
@@ -110,7 +111,10 @@ def test_encode_prefill_on_tensor_cores_matches_the_chain_up_to_its_margin(T, st
     else:
         x = torch.randn(B, H, T, 128, device=DEV, generator=g).to(torch.bfloat16)
     codes = torch.full((B, H, T + 5), 0x33, dtype=torch.int32, device=DEV)
-    ha.ha_encode_prefill(ha.Mapping(mp), heads_per_kv, x, codes)
+    shape = ha.make_shape(B, H, H // heads_per_kv, 1.0)
+    ws = ha.alloc_workspace(shape, 16, 16)
+    ha.ha_encode_prefill(ha.Mapping(mp), heads_per_kv, x, codes, path=path, workspace=ws)
+    assert ha.ha_read_device_status(ws) == 0          # no wait on the tensor cores ran out
     exact = torch.zeros(B, H, T, dtype=torch.int32, device=DEV)
     ha.ha_encode(ha.Mapping(mp), heads_per_kv, x, exact)
     torch.cuda.synchronize()
