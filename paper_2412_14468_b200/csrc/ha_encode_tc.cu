@@ -216,28 +216,34 @@ cudaError_t launch_encode_tc(const MapView &map, int heads_per_kv, TensorView x,
 
 // ------------------------------------------------------------------ tcgen05 version
 //
-// The same chain of three GEMMs on the fifth-generation tensor cores.  One CTA of 128 threads
-// owns a tile of 128 tokens: M = 128 rows = the 128 lanes of tensor memory, thread r owns row r.
-//   layer 1  D1[128 x 128] = X W1      A = token tile in shared memory (K-major core matrices),
-//                                      B = W1 in shared memory (N-major core matrices), 8 x K16
-//   epilogue threads read their row of D1 (tcgen05.ld), add the bias, apply ReLU, split into a bf16
-//            pair hi + lo and write both back to tensor memory as the next A operand (tcgen05.st)
-//   layer 2  D2 = A_hi W2 + A_lo W2    A from tensor memory, 16 x K16
-//   layer 3  D3[128 x 32] likewise; the epilogue packs the 32 sign bits of a row into its code.
-// Activations never leave tensor memory and registers.  Tensor memory use: 128 columns D1 / D3,
-// 128 columns A (64 hi + 64 lo), 128 columns D2 = 384 of the 512 allocated; two CTAs cannot share an
-// SM (shared memory), so the whole allocation is free to take.
-// MMAs are issued by thread 0 and tracked by one mbarrier (tcgen05.commit); every wait on it is
-// bounded: on a timeout the CTA raises HA_DEV_TIMEOUT in the status word, stops issuing work,
-// frees its tensor memory and returns.
+// The same chain of three GEMMs on the fifth-generation tensor cores.  A tile of 128 tokens is
+// M = 128 rows = the 128 lanes of tensor memory; thread r of a group of 128 threads owns row r.
+//   layer 1  D[128 x 128] = X W1 + b1   A = token tile in shared memory (K-major core matrices),
+//                                       B = W1 in shared memory (N-major core matrices), 8 x K16;
+//                                       the bias is one more K16 step: A = a constant tile whose
+//                                       rows are (1, 1, 0, ...), B = two rows holding b1 as a bf16
+//                                       pair hi + lo
+//   epilogue threads read their row of D (tcgen05.ld), apply ReLU, split into a bf16 pair hi + lo
+//            (cvt.rn.bf16x2) and write both to tensor memory as the next A operand (tcgen05.st)
+//   layer 2  D = A_hi W2 + A_lo W2 + b2  A from tensor memory, 16 x K16 + the bias step
+//   layer 3  D[128 x 32] likewise; the epilogue packs the 32 sign bits of a row into its code.
+// Activations never leave tensor memory and registers.
+// Two groups of 128 threads work on alternate tiles with their own token buffers, their own half of
+// tensor memory (D 128 + A_hi 64 + A_lo 64 columns) and their own mbarrier, so that one group's
+// tensor-core work runs under the other group's epilogue.  A CTA stays with one network: its
+// weights are loaded once.  MMAs are issued by the first thread of a group and tracked with
+// tcgen05.commit; every wait is bounded: on a timeout the group raises HA_DEV_TIMEOUT in the status
+// word and stops, and the CTA frees its tensor memory and returns.
 
-constexpr int kU_Threads = 128;
-constexpr int kU_WBytes = kD * kHid * 2;          // 32768: W1 or W2 as 16 k-groups x 16 n-blocks x (8 x 16 B)
-constexpr int kU_W3Bytes = kHid * kBits * 2;      // 8192
+constexpr int kU_Threads = 256;                   // two groups of 128
+constexpr int kU_KG = kD / 8 + 2;                 // k-groups of 8 rows per weight matrix: 16 + 2 for the bias step
+constexpr int kU_WBytes = kU_KG * 2048;           // 36864: W1 or W2 as k-groups x 16 n-blocks x (8 x 16 B)
+constexpr int kU_W3Bytes = kU_KG * 512;           // 9216
+constexpr int kU_OnesBytes = 4096;                // [128 rows x 16 k] tile of (1, 1, 0, ...) rows
 constexpr int kU_XBytes = kTcTile * kD * 2;       // 32768: 16 k-chunks x 16 row-groups x (8 x 16 B)
-constexpr int kU_Smem = 2 * kU_WBytes + kU_W3Bytes + 2 * kU_XBytes + 1024;
+constexpr int kU_Smem = 2 * kU_WBytes + kU_W3Bytes + kU_OnesBytes + 4 * kU_XBytes;   // 218112
 constexpr uint32_t kU_TmemCols = 512;
-constexpr uint32_t kU_ColD1 = 0, kU_ColA = 128, kU_ColD2 = 256;   // column offsets inside the allocation
+constexpr uint32_t kU_SlotCols = 256, kU_ColD = 0, kU_ColAhi = 128, kU_ColAlo = 192;   // per group
 
 // 64-bit shared-memory matrix descriptor, no swizzle: start address, leading and stride byte offsets
 // in 16-byte units, descriptor version 1 (bits 46-47), layout type 0 (bits 61-63).
@@ -275,82 +281,71 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
                    "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
-                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
+// 16 consecutive 32-bit columns of this thread's lane
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
                  ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-                   "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
-                   "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
-                   "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
+                   "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(taddr)
                  : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void group_sync(int group) { asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory"); }
 
+// try_wait parks the warp for a bounded time instead of spinning, so a waiting group leaves the issue
+// slots to the group that is converting; the number of attempts is bounded as well.
 __device__ __forceinline__ bool mbar_wait_parity_bounded(uint32_t bar, uint32_t parity) {
-    for (int it = 0; it < (1 << 22); ++it) {   // non-blocking probes: a few tenths of a second at most
+    for (int it = 0; it < (1 << 18); ++it) {
         uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
         if (done) return true;
     }
     return false;
 }
 
+// ReLU + split of two fp32 values into packed bf16 pairs: hi = round(max(v, 0)), lo = round(max(v, 0) - hi);
+// the remainder keeps its sign (hi may have been rounded up).  Low half = first value.
+__device__ __forceinline__ void relu_split_pair(float v0, float v1, uint32_t &hi, uint32_t &lo) {
+    v0 = fmaxf(v0, 0.0f);
+    v1 = fmaxf(v1, 0.0f);
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi) : "f"(v1), "f"(v0));
+    const float r0 = v0 - __uint_as_float(hi << 16), r1 = v1 - __uint_as_float(hi & 0xffff0000u);
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo) : "f"(r1), "f"(r0));
+}
+
 __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map, int heads_per_kv, TensorView x, int B,
-                                                                   int H, int T, uint32_t *__restrict__ codes,
-                                                                   long long c_sb, long long c_sh,
-                                                                   uint32_t *__restrict__ status) {
+                                                                   int H, int T, int ctas_per_net,
+                                                                   uint32_t *__restrict__ codes, long long c_sb,
+                                                                   long long c_sh, uint32_t *__restrict__ status) {
     extern __shared__ __align__(1024) unsigned char usm[];
-    unsigned char *sW1 = usm, *sW2 = sW1 + kU_WBytes, *sW3 = sW2 + kU_WBytes, *sX = sW3 + kU_W3Bytes;
-    __shared__ __align__(8) unsigned long long s_mbar;
+    unsigned char *sW1 = usm, *sW2 = sW1 + kU_WBytes, *sW3 = sW2 + kU_WBytes, *sOnes = sW3 + kU_W3Bytes,
+                  *sX = sOnes + kU_OnesBytes;
+    __shared__ __align__(8) unsigned long long s_mbar[2];
     __shared__ uint32_t s_tmem_base;
-    __shared__ int s_fail;
-    const int tid = threadIdx.x, warp = tid >> 5;
+    __shared__ int s_fail[2];
+    const int tid = threadIdx.x, warp = tid >> 5, group = tid >> 7, gt = tid & 127;
     const int tiles_per_row = (T + kTcTile - 1) / kTcTile;
-    const long long n_work = (long long)H * B * tiles_per_row;   // head-major order: a CTA keeps its weights
-    const long long w_lo = n_work * blockIdx.x / gridDim.x, w_hi = n_work * (blockIdx.x + 1) / gridDim.x;
+    const int net = blockIdx.x / ctas_per_net, part = blockIdx.x % ctas_per_net;
+    // tiles of this network in the order (head of the network, sequence, tile); this CTA takes a contiguous share
+    const long long n_net = (long long)heads_per_kv * B * tiles_per_row;
+    const long long w_lo = n_net * part / ctas_per_net, w_hi = n_net * (part + 1) / ctas_per_net;
     if (w_lo >= w_hi) return;
-    const uint32_t bar = smem_u32(&s_mbar);
 
     if (tid == 0) {
-        mbar_init(bar, 1);
+        mbar_init(smem_u32(&s_mbar[0]), 1);
+        mbar_init(smem_u32(&s_mbar[1]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        s_fail = 0;
+        s_fail[0] = 0;
+        s_fail[1] = 0;
     }
     if (warp == 0) {   // one warp allocates the tensor memory and passes the allocation right on
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)), "r"(kU_TmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = s_tmem_base;
-    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
-
-    auto decode = [&](long long w, int &h, int &b, int &t0) {
-        const long long per_head = (long long)B * tiles_per_row;
-        h = (int)(w / per_head);
-        const long long r = w - (long long)h * per_head;
-        b = (int)(r / tiles_per_row);
-        t0 = (int)(r - (long long)b * tiles_per_row) * kTcTile;
-    };
-    // token tile, K-major core matrices: element (row r, k) at (k/8) * 2048 + (r/8) * 128 + (r%8) * 16 + (k%8) * 2
-    auto load_x = [&](long long w, int buf) {
-        int h, b, t0;
-        decode(w, h, b, t0);
-        const unsigned char *src = reinterpret_cast<const unsigned char *>(x.ptr + (long long)b * x.sb + (long long)h * x.sh);
-        const uint32_t dst = smem_u32(sX + buf * kU_XBytes);
-#pragma unroll
-        for (int i = 0; i < kTcTile * 16 / kU_Threads; ++i) {
-            const int e = tid + i * kU_Threads, row = e >> 4, ch = e & 15;
-            const bool ok = t0 + row < T;
-            cp_async16(dst + ch * 2048 + (row >> 3) * 128 + (row & 7) * 16,
-                       src + (long long)(ok ? t0 + row : 0) * x.sn * 2 + ch * 16, ok ? 16u : 0u);
-        }
-    };
-    // weights [k][n], N-major core matrices: element (k, n) at (k/8) * LBO + (n/8) * 128 + (k%8) * 16 + (n%8) * 2
-    auto load_weights = [&](int net) {
+    // ---- weights (N-major core matrices: element (k, n) at (k/8) * LBO + (n/8) * 128 + (k%8) * 16 + (n%8) * 2),
+    // the bias rows k = 128 (hi) and 129 (lo) behind them, and the constant tile of ones
+    {
         const unsigned char *g1 = reinterpret_cast<const unsigned char *>(map.w1 + (size_t)net * kD * kHid);
         const unsigned char *g2 = reinterpret_cast<const unsigned char *>(map.w2 + (size_t)net * kHid * kHid);
         const unsigned char *g3 = reinterpret_cast<const unsigned char *>(map.w3 + (size_t)net * kHid * kBits);
@@ -364,137 +359,173 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map,
             const int k = e >> 2, nb = e & 3;
             cp_async16(smem_u32(sW3) + (k >> 3) * 512 + nb * 128 + (k & 7) * 16, g3 + (size_t)e * 16, 16u);
         }
+        cp_async_commit();
+        // k-groups 16 and 17: zero, then the bias pair in rows 0 and 1 of k-group 16
+        for (int i = tid; i < 4096 / 16; i += kU_Threads) {
+            reinterpret_cast<uint4 *>(sW1 + 16 * 2048)[i] = make_uint4(0u, 0u, 0u, 0u);
+            reinterpret_cast<uint4 *>(sW2 + 16 * 2048)[i] = make_uint4(0u, 0u, 0u, 0u);
+            reinterpret_cast<uint4 *>(sOnes)[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        for (int i = tid; i < 1024 / 16; i += kU_Threads) reinterpret_cast<uint4 *>(sW3 + 16 * 512)[i] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();
+        auto put_bias = [&](unsigned char *base, const float *bias, int n) {
+            const float v = bias ? __ldg(bias + n) : 0.0f;
+            const float h = bf16_round(v);
+            const __nv_bfloat16 bh = __float2bfloat16_rn(h), bl = __float2bfloat16_rn(v - h);
+            unsigned char *p = base + (n >> 3) * 128 + (n & 7) * 2;
+            *reinterpret_cast<uint16_t *>(p) = *reinterpret_cast<const uint16_t *>(&bh);        // row k = 128
+            *reinterpret_cast<uint16_t *>(p + 16) = *reinterpret_cast<const uint16_t *>(&bl);   // row k = 129
+        };
+        if (tid < kHid) {
+            put_bias(sW1 + 16 * 2048, map.b1 ? map.b1 + net * kHid : nullptr, tid);
+            put_bias(sW2 + 16 * 2048, map.b2 ? map.b2 + net * kHid : nullptr, tid);
+            // ones tile, K-major: row r at (r/8) * 128 + (r%8) * 16 of k-chunk 0 holds (1, 1, 0, 0, 0, 0, 0, 0)
+            *reinterpret_cast<uint32_t *>(sOnes + (tid >> 3) * 128 + (tid & 7) * 16) = 0x3f803f80u;
+        }
+        if (tid < kBits) put_bias(sW3 + 16 * 512, map.b3 ? map.b3 + net * kBits : nullptr, tid);
+    }
+    cp_async_wait<0>();
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ordinary writes -> visible to the tensor cores
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base + group * kU_SlotCols;                 // this group's half
+    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 lanes
+    const uint32_t bar = smem_u32(&s_mbar[group]);
+    unsigned char *gX = sX + group * 2 * kU_XBytes;
+
+    auto decode = [&](long long w, int &h, int &b, int &t0) {
+        const long long per_head = (long long)B * tiles_per_row;
+        const int hh = (int)(w / per_head);
+        const long long r = w - (long long)hh * per_head;
+        h = net * heads_per_kv + hh;
+        b = (int)(r / tiles_per_row);
+        t0 = (int)(r - (long long)b * tiles_per_row) * kTcTile;
+    };
+    // token tile, K-major core matrices: element (row r, k) at (k/8) * 2048 + (r/8) * 128 + (r%8) * 16 + (k%8) * 2.
+    // A lane pair copies one 32-byte sector of a row, 16 consecutive rows per warp: whole sectors on the
+    // global side, consecutive 16-byte slots (two-way bank conflicts at most) on the shared side.
+    auto load_x = [&](long long w, int buf) {
+        int h, b, t0;
+        decode(w, h, b, t0);
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(x.ptr + (long long)b * x.sb + (long long)h * x.sh);
+        const uint32_t dst = smem_u32(gX + buf * kU_XBytes);
+#pragma unroll
+        for (int i = 0; i < kTcTile * 16 / 128; ++i) {
+            const int e = gt + i * 128, row = (e >> 1) & 127, ch = 2 * (e >> 8) + (e & 1);
+            const bool ok = t0 + row < T;
+            cp_async16(dst + ch * 2048 + (row >> 3) * 128 + (row & 7) * 16,
+                       src + (long long)(ok ? t0 + row : 0) * x.sn * 2 + ch * 16, ok ? 16u : 0u);
+        }
     };
 
     constexpr uint32_t kIdesc128 = umma_idesc(128, 128), kIdesc32 = umma_idesc(128, 32);
+    const uint64_t ones_desc = umma_desc(smem_u32(sOnes), 2048, 128);
     uint32_t phase = 0;
-    bool failed = false;
-    // wait for the MMAs committed last; CTA-uniform result
+    // wait for the MMAs committed last; group-uniform result
     auto wait_mma = [&]() -> bool {
         const bool ok = mbar_wait_parity_bounded(bar, phase);
         phase ^= 1u;
-        if (!ok) s_fail = 1;
+        if (!ok) s_fail[group] = 1;
         tc_fence_after();
-        __syncthreads();
-        return s_fail == 0;
+        group_sync(group);
+        return s_fail[group] == 0;
     };
-    // this thread's row of a 128-column accumulator -> bias, ReLU, hi / lo -> the A operand columns
-    auto epilogue_hidden = [&](uint32_t col_d, const float *bias) {
-        uint32_t hi[64], lo[64];
+    // this thread's row of the 128-column accumulator -> ReLU, hi / lo -> the A operand columns
+    auto epilogue_hidden = [&]() {
+        uint32_t v[4][32];   // the whole row is requested at once: one tensor-memory round trip, not four
+#pragma unroll
+        for (int q = 0; q < 4; ++q) tmem_ld32(lane_base + kU_ColD + q * 32, v[q]);
+        tmem_wait_ld();
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            uint32_t v[32];
-            tmem_ld32(lane_base + col_d + q * 32, v);
-            tmem_wait_ld();
+            uint32_t hi[16], lo[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int o = q * 32 + 2 * i;
-                const float z0 = __uint_as_float(v[2 * i]) + (bias ? __ldg(bias + o) : 0.0f);
-                const float z1 = __uint_as_float(v[2 * i + 1]) + (bias ? __ldg(bias + o + 1) : 0.0f);
-                split_relu(z0, z1, hi[q * 16 + i], lo[q * 16 + i]);
-            }
-        }
-        {
-            uint32_t t[32];
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) t[i] = hi[q * 32 + i];
-                tmem_st32(lane_base + kU_ColA + q * 32, t);
-#pragma unroll
-                for (int i = 0; i < 32; ++i) t[i] = lo[q * 32 + i];
-                tmem_st32(lane_base + kU_ColA + 64 + q * 32, t);
-            }
+            for (int i = 0; i < 16; ++i)
+                relu_split_pair(__uint_as_float(v[q][2 * i]), __uint_as_float(v[q][2 * i + 1]), hi[i], lo[i]);
+            tmem_st16(lane_base + kU_ColAhi + q * 16, hi);
+            tmem_st16(lane_base + kU_ColAlo + q * 16, lo);
         }
         tmem_wait_st();
         tc_fence_before();
-        __syncthreads();
+        group_sync(group);
     };
 
-    int cur_net = -1;
-    load_x(w_lo, 0);
+    bool failed = false;
+    long long w = w_lo + group;
+    if (w < w_hi) load_x(w, 0);
     cp_async_commit();
     int buf = 0;
-    for (long long w = w_lo; w < w_hi && !failed; ++w, buf ^= 1) {
+    for (; w < w_hi; w += 2, buf ^= 1) {
         int h, b, t0;
         decode(w, h, b, t0);
-        const int net = h / heads_per_kv;
-        if (net != cur_net) {
-            load_weights(net);
-            cur_net = net;
-        }
-        cp_async_commit();      // group of the weights (empty when they stay)
-        if (w + 1 < w_hi) load_x(w + 1, buf ^ 1);
+        if (w + 2 < w_hi) load_x(w + 2, buf ^ 1);
         cp_async_commit();      // group of the next tile (empty after the last one)
-        cp_async_wait<1>();     // this tile and the weights have landed
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ordinary writes -> visible to the tensor cores
-        __syncthreads();
+        cp_async_wait<1>();     // this tile has landed
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        group_sync(group);
 
-        const float *bias1 = map.b1 ? map.b1 + net * kHid : nullptr;
-        const float *bias2 = map.b2 ? map.b2 + net * kHid : nullptr;
-        const float *bias3 = map.b3 ? map.b3 + net * kBits : nullptr;
-
-        // ---- layer 1: D1 = X W1 (both operands from shared memory), one MMA per 16 values of k
-        if (tid == 0) {
+        // ---- layer 1: D = X W1 + b1 (operands from shared memory), one MMA per 16 values of k
+        if (gt == 0) {
             tc_fence_after();
-            const uint32_t xa = smem_u32(sX + buf * kU_XBytes), wa = smem_u32(sW1);
+            const uint32_t xa = smem_u32(gX + buf * kU_XBytes), wa = smem_u32(sW1);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-                umma_ss(tmem + kU_ColD1, umma_desc(xa + ks * 4096, 2048, 128), umma_desc(wa + ks * 4096, 2048, 128),
+                umma_ss(tmem + kU_ColD, umma_desc(xa + ks * 4096, 2048, 128), umma_desc(wa + ks * 4096, 2048, 128),
                         kIdesc128, ks > 0 ? 1u : 0u);
+            umma_ss(tmem + kU_ColD, ones_desc, umma_desc(wa + 8 * 4096, 2048, 128), kIdesc128, 1u);
             umma_commit(bar);
         }
         if (!wait_mma()) { failed = true; break; }
-        epilogue_hidden(kU_ColD1, bias1);
+        epilogue_hidden();
 
-        // ---- layer 2: D2 = A_hi W2 + A_lo W2, A from tensor memory (8 columns per 16 values of k)
-        if (tid == 0) {
+        // ---- layer 2: D = A_hi W2 + A_lo W2 + b2, A from tensor memory (8 columns per 16 values of k)
+        if (gt == 0) {
             tc_fence_after();
             const uint32_t wa = smem_u32(sW2);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-                umma_ts(tmem + kU_ColD2, tmem + kU_ColA + ks * 8, umma_desc(wa + ks * 4096, 2048, 128), kIdesc128, ks > 0 ? 1u : 0u);
-                umma_ts(tmem + kU_ColD2, tmem + kU_ColA + 64 + ks * 8, umma_desc(wa + ks * 4096, 2048, 128), kIdesc128, 1u);
+                umma_ts(tmem + kU_ColD, tmem + kU_ColAhi + ks * 8, umma_desc(wa + ks * 4096, 2048, 128), kIdesc128, ks > 0 ? 1u : 0u);
+                umma_ts(tmem + kU_ColD, tmem + kU_ColAlo + ks * 8, umma_desc(wa + ks * 4096, 2048, 128), kIdesc128, 1u);
             }
+            umma_ss(tmem + kU_ColD, ones_desc, umma_desc(wa + 8 * 4096, 2048, 128), kIdesc128, 1u);
             umma_commit(bar);
         }
         if (!wait_mma()) { failed = true; break; }
-        epilogue_hidden(kU_ColD2, bias2);
+        epilogue_hidden();
 
-        // ---- layer 3: D3[128 x 32] into the columns of D1
-        if (tid == 0) {
+        // ---- layer 3: D[128 x 32]
+        if (gt == 0) {
             tc_fence_after();
             const uint32_t wa = smem_u32(sW3);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-                umma_ts(tmem + kU_ColD1, tmem + kU_ColA + ks * 8, umma_desc(wa + ks * 1024, 512, 128), kIdesc32, ks > 0 ? 1u : 0u);
-                umma_ts(tmem + kU_ColD1, tmem + kU_ColA + 64 + ks * 8, umma_desc(wa + ks * 1024, 512, 128), kIdesc32, 1u);
+                umma_ts(tmem + kU_ColD, tmem + kU_ColAhi + ks * 8, umma_desc(wa + ks * 1024, 512, 128), kIdesc32, ks > 0 ? 1u : 0u);
+                umma_ts(tmem + kU_ColD, tmem + kU_ColAlo + ks * 8, umma_desc(wa + ks * 1024, 512, 128), kIdesc32, 1u);
             }
+            umma_ss(tmem + kU_ColD, ones_desc, umma_desc(wa + 8 * 1024, 512, 128), kIdesc32, 1u);
             umma_commit(bar);
         }
         if (!wait_mma()) { failed = true; break; }
         {
             uint32_t v[32];
-            tmem_ld32(lane_base + kU_ColD1, v);
+            tmem_ld32(lane_base + kU_ColD, v);
             tmem_wait_ld();
             uint32_t code = 0u;
 #pragma unroll
-            for (int o = 0; o < 32; ++o) {
-                const float z = __uint_as_float(v[o]) + (bias3 ? __ldg(bias3 + o) : 0.0f);
-                code |= (z > 0.0f ? 1u : 0u) << o;
-            }
-            if (t0 + tid < T) codes[(long long)b * c_sb + (long long)h * c_sh + t0 + tid] = code;
+            for (int o = 0; o < 32; ++o) code |= (__uint_as_float(v[o]) > 0.0f ? 1u : 0u) << o;
+            if (t0 + gt < T) codes[(long long)b * c_sb + (long long)h * c_sh + t0 + gt] = code;
         }
         tc_fence_before();
-        __syncthreads();   // every thread is done with this token buffer, these weights and D1 before they are reused
+        group_sync(group);   // the group is done with this token buffer and with D before they are reused
     }
-    if (failed && tid == 0 && status) atomicOr(status, HA_DEV_TIMEOUT);
+    if (failed && gt == 0 && status) atomicOr(status, HA_DEV_TIMEOUT);
     cp_async_wait<0>();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kU_TmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(s_tmem_base), "r"(kU_TmemCols) : "memory");
     }
 }
 
@@ -502,10 +533,15 @@ cudaError_t launch_encode_umma(const MapView &map, int heads_per_kv, TensorView 
                                long long c_sb, long long c_sh, uint32_t *status, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(encode_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kU_Smem);
     if (e != cudaSuccess) return e;
-    const long long n_work = (long long)H * B * ((T + kTcTile - 1) / kTcTile);
-    if (n_work <= 0) return cudaSuccess;
-    const int grid = (int)((n_work < sm_count()) ? n_work : sm_count());
-    encode_umma_kernel<<<grid, kU_Threads, kU_Smem, st>>>(map, heads_per_kv, x, B, H, T, codes, c_sb, c_sh, status);
+    const int n_nets = H / heads_per_kv;
+    const long long n_net = (long long)heads_per_kv * B * ((T + kTcTile - 1) / kTcTile);   // tiles per network
+    if (n_net <= 0 || n_nets <= 0) return cudaSuccess;
+    long long per = sm_count() / n_nets;                 // CTAs per network: a CTA never changes its weights
+    if (per < 1) per = 1;
+    if (per > (n_net + 1) / 2) per = (n_net + 1) / 2;    // at least two tiles (one per group) for a CTA to be worth it
+    if (per < 1) per = 1;
+    encode_umma_kernel<<<(int)(n_nets * per), kU_Threads, kU_Smem, st>>>(map, heads_per_kv, x, B, H, T, (int)per, codes,
+                                                                        c_sb, c_sh, status);
     count_launch();
     return cudaGetLastError();
 }

@@ -101,7 +101,8 @@ def test_encode_without_biases_and_strided_input():
 def test_encode_prefill_on_tensor_cores_matches_the_chain_up_to_its_margin(T, strided, path):
     """The tensor-core prompt encoder sums in another order and feeds 16-bit activations to the next layer:
     its signature bits must equal the chain-exact ones wherever the exact last-layer output is not within
-    1e-3 of zero (the stated accuracy is ~1e-5), and only a tiny share of bits may differ at all."""
+    1e-3 of zero (the stated accuracy is ~1e-5), and at most one bit in 100000 may differ at all (a
+    16-bit split that loses the sign of its remainder already fails this)."""
     B, H, heads_per_kv = 2, 4, 2
     mp = _mapping(H // heads_per_kv, 500 + T)
     g = torch.Generator(DEV).manual_seed(T)
@@ -135,7 +136,7 @@ def test_encode_prefill_on_tensor_cores_matches_the_chain_up_to_its_margin(T, st
                     if (int(diff[t]) >> o) & 1:
                         n_diff += 1
                         assert abs(float(z3[t, o])) < 1e-3, (b, h, t, o, float(z3[t, o]))
-    assert n_diff <= max(2, B * H * T * 32 // 2000)
+    assert n_diff <= max(2, B * H * T * 32 // 100000)
 
 
 # ---------------------------------------------------------------------------- SCORE + TOPK
