@@ -240,8 +240,10 @@ constexpr int kU_KG = kD / 8 + 2;                 // k-groups of 8 rows per weig
 constexpr int kU_WBytes = kU_KG * 2048;           // 36864: W1 or W2 as k-groups x 16 n-blocks x (8 x 16 B)
 constexpr int kU_W3Bytes = kU_KG * 512;           // 9216
 constexpr int kU_OnesBytes = 4096;                // [128 rows x 16 k] tile of (1, 1, 0, ...) rows
-constexpr int kU_XBytes = kTcTile * kD * 2;       // 32768: 16 k-chunks x 16 row-groups x (8 x 16 B)
-constexpr int kU_Smem = 2 * kU_WBytes + kU_W3Bytes + kU_OnesBytes + 4 * kU_XBytes;   // 218112
+constexpr int kU_XLbo = 2048 + 16;                // bytes between the k-chunks of a token tile: 16 row-groups x 128 B, plus one
+                                                  // 16-byte slot so that the 16 chunks of a row fall into different banks
+constexpr int kU_XBytes = 16 * kU_XLbo;           // 33024
+constexpr int kU_Smem = 2 * kU_WBytes + kU_W3Bytes + kU_OnesBytes + 4 * kU_XBytes;   // 219136
 constexpr uint32_t kU_TmemCols = 512;
 constexpr uint32_t kU_SlotCols = 256, kU_ColD = 0, kU_ColAhi = 128, kU_ColAlo = 192;   // per group
 
@@ -402,9 +404,8 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map,
         b = (int)(r / tiles_per_row);
         t0 = (int)(r - (long long)b * tiles_per_row) * kTcTile;
     };
-    // token tile, K-major core matrices: element (row r, k) at (k/8) * 2048 + (r/8) * 128 + (r%8) * 16 + (k%8) * 2.
-    // A lane pair copies one 32-byte sector of a row, 16 consecutive rows per warp: whole sectors on the
-    // global side, consecutive 16-byte slots (two-way bank conflicts at most) on the shared side.
+    // token tile, K-major core matrices: element (row r, k) at (k/8) * kU_XLbo + (r/8) * 128 + (r%8) * 16 + (k%8) * 2.
+    // A half-warp copies one 256-byte row: whole lines on the global side, 16 different banks on the shared side.
     auto load_x = [&](long long w, int buf) {
         int h, b, t0;
         decode(w, h, b, t0);
@@ -412,9 +413,9 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map,
         const uint32_t dst = smem_u32(gX + buf * kU_XBytes);
 #pragma unroll
         for (int i = 0; i < kTcTile * 16 / 128; ++i) {
-            const int e = gt + i * 128, row = (e >> 1) & 127, ch = 2 * (e >> 8) + (e & 1);
+            const int e = gt + i * 128, row = e >> 4, ch = e & 15;
             const bool ok = t0 + row < T;
-            cp_async16(dst + ch * 2048 + (row >> 3) * 128 + (row & 7) * 16,
+            cp_async16(dst + ch * kU_XLbo + (row >> 3) * 128 + (row & 7) * 16,
                        src + (long long)(ok ? t0 + row : 0) * x.sn * 2 + ch * 16, ok ? 16u : 0u);
         }
     };
@@ -471,7 +472,7 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map,
             const uint32_t xa = smem_u32(gX + buf * kU_XBytes), wa = smem_u32(sW1);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-                umma_ss(tmem + kU_ColD, umma_desc(xa + ks * 4096, 2048, 128), umma_desc(wa + ks * 4096, 2048, 128),
+                umma_ss(tmem + kU_ColD, umma_desc(xa + ks * 2 * kU_XLbo, kU_XLbo, 128), umma_desc(wa + ks * 4096, 2048, 128),
                         kIdesc128, ks > 0 ? 1u : 0u);
             umma_ss(tmem + kU_ColD, ones_desc, umma_desc(wa + 8 * 4096, 2048, 128), kIdesc128, 1u);
             umma_commit(bar);
