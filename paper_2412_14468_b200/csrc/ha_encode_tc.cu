@@ -18,6 +18,9 @@
 #include "ha_attn_dev.cuh"
 #include "ha_encode_dev.cuh"
 
+#include <cstring>
+#include <cuda.h>   // CUtensorMap (types only; the encoder is fetched through the runtime)
+
 namespace ha {
 
 constexpr int kTcTile = 128;                       // tokens per tile
@@ -240,9 +243,9 @@ constexpr int kU_KG = kD / 8 + 2;                 // k-groups of 8 rows per weig
 constexpr int kU_WBytes = kU_KG * 2048;           // 36864: W1 or W2 as k-groups x 16 n-blocks x (8 x 16 B)
 constexpr int kU_W3Bytes = kU_KG * 512;           // 9216
 constexpr int kU_OnesBytes = 4096;                // [128 rows x 16 k] tile of (1, 1, 0, ...) rows
-constexpr int kU_XLbo = 2048 + 16;                // bytes between the k-chunks of a token tile: 16 row-groups x 128 B, plus one
-                                                  // 16-byte slot so that the 16 chunks of a row fall into different banks
-constexpr int kU_XBytes = 16 * kU_XLbo;           // 33024
+constexpr int kU_XLboPad = 2048 + 16;             // bytes between the k-chunks of a token tile copied by the threads: 16 row-groups
+                                                  // x 128 B, plus one 16-byte slot so that the 16 chunks of a row fall into different banks
+constexpr int kU_XBytes = 16 * kU_XLboPad;        // 33024 (a tile copied by TMA uses 16 x 2048 of it)
 constexpr int kU_Smem = 2 * kU_WBytes + kU_W3Bytes + kU_OnesBytes + 4 * kU_XBytes;   // 219136
 constexpr uint32_t kU_TmemCols = 512;
 constexpr uint32_t kU_SlotCols = 256, kU_ColD = 0, kU_ColAhi = 128, kU_ColAlo = 192;   // per group
@@ -316,14 +319,27 @@ __device__ __forceinline__ void relu_split_pair(float v0, float v1, uint32_t &hi
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo) : "f"(r1), "f"(r0));
 }
 
-__global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map, int heads_per_kv, TensorView x, int B,
-                                                                   int H, int T, int ctas_per_net,
-                                                                   uint32_t *__restrict__ codes, long long c_sb,
-                                                                   long long c_sh, uint32_t *__restrict__ status) {
+// One k-chunk of a token tile (8 values of k x 128 tokens) through the tensor map of x [B][H][T][128]: the
+// box lands as 128 consecutive 16-byte rows, which is the core-matrix layout the MMA descriptor names.
+__device__ __forceinline__ void tma_load_chunk(uint32_t dst, const CUtensorMap *tmap, int k0, int t0, int h, int b, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(dst), "l"(tmap), "r"(k0), "r"(t0), "r"(h), "r"(b), "r"(bar) : "memory");
+}
+
+// kTma: token tiles arrive through TMA (one thread per group issues 16 box copies and the tile's mbarrier
+// counts the bytes); otherwise every thread copies 16-byte pieces with cp.async.
+template <bool kTma>
+__global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid_constant__ CUtensorMap tmap, MapView map,
+                                                                   int heads_per_kv, TensorView x, int B, int H, int T,
+                                                                   int ctas_per_net, uint32_t *__restrict__ codes,
+                                                                   long long c_sb, long long c_sh,
+                                                                   uint32_t *__restrict__ status) {
+    constexpr int kU_XLbo = kTma ? 2048 : kU_XLboPad;
     extern __shared__ __align__(1024) unsigned char usm[];
     unsigned char *sW1 = usm, *sW2 = sW1 + kU_WBytes, *sW3 = sW2 + kU_WBytes, *sOnes = sW3 + kU_W3Bytes,
                   *sX = sOnes + kU_OnesBytes;
     __shared__ __align__(8) unsigned long long s_mbar[2];
+    __shared__ __align__(8) unsigned long long s_xbar[2][2];   // [group][buffer]: arrival of a token tile (TMA)
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_fail[2];
     const int tid = threadIdx.x, warp = tid >> 5, group = tid >> 7, gt = tid & 127;
@@ -337,6 +353,7 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map,
     if (tid == 0) {
         mbar_init(smem_u32(&s_mbar[0]), 1);
         mbar_init(smem_u32(&s_mbar[1]), 1);
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&s_xbar[0][0]) + 8 * i, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s_fail[0] = 0;
         s_fail[1] = 0;
@@ -405,18 +422,29 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map,
         t0 = (int)(r - (long long)b * tiles_per_row) * kTcTile;
     };
     // token tile, K-major core matrices: element (row r, k) at (k/8) * kU_XLbo + (r/8) * 128 + (r%8) * 16 + (k%8) * 2.
-    // A half-warp copies one 256-byte row: whole lines on the global side, 16 different banks on the shared side.
+    // TMA: 16 box copies of 8 x 128 elements; rows past T are filled with zeros by the tensor map.
+    // Threads: a half-warp copies one 256-byte row (whole lines on the global side, 16 different banks on the
+    // shared side thanks to the padded chunk stride).
     auto load_x = [&](long long w, int buf) {
         int h, b, t0;
         decode(w, h, b, t0);
-        const unsigned char *src = reinterpret_cast<const unsigned char *>(x.ptr + (long long)b * x.sb + (long long)h * x.sh);
         const uint32_t dst = smem_u32(gX + buf * kU_XBytes);
+        if (kTma) {
+            if (gt == 0) {
+                const uint32_t xb = smem_u32(&s_xbar[group][buf]);
+                mbar_expect_tx(xb, kTcTile * kD * 2);
 #pragma unroll
-        for (int i = 0; i < kTcTile * 16 / 128; ++i) {
-            const int e = gt + i * 128, row = e >> 4, ch = e & 15;
-            const bool ok = t0 + row < T;
-            cp_async16(dst + ch * kU_XLbo + (row >> 3) * 128 + (row & 7) * 16,
-                       src + (long long)(ok ? t0 + row : 0) * x.sn * 2 + ch * 16, ok ? 16u : 0u);
+                for (int ch = 0; ch < 16; ++ch) tma_load_chunk(dst + ch * kU_XLbo, &tmap, 8 * ch, t0, h, b, xb);
+            }
+        } else {
+            const unsigned char *src = reinterpret_cast<const unsigned char *>(x.ptr + (long long)b * x.sb + (long long)h * x.sh);
+#pragma unroll
+            for (int i = 0; i < kTcTile * 16 / 128; ++i) {
+                const int e = gt + i * 128, row = e >> 4, ch = e & 15;
+                const bool ok = t0 + row < T;
+                cp_async16(dst + ch * kU_XLbo + (row >> 3) * 128 + (row & 7) * 16,
+                           src + (long long)(ok ? t0 + row : 0) * x.sn * 2 + ch * 16, ok ? 16u : 0u);
+            }
         }
     };
 
@@ -457,14 +485,22 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map,
     if (w < w_hi) load_x(w, 0);
     cp_async_commit();
     int buf = 0;
+    uint32_t xphase[2] = {0u, 0u};
     for (; w < w_hi; w += 2, buf ^= 1) {
         int h, b, t0;
         decode(w, h, b, t0);
         if (w + 2 < w_hi) load_x(w + 2, buf ^ 1);
-        cp_async_commit();      // group of the next tile (empty after the last one)
-        cp_async_wait<1>();     // this tile has landed
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        group_sync(group);
+        if (kTma) {             // this tile has landed when its mbarrier has counted all its bytes
+            if (!mbar_wait_parity_bounded(smem_u32(&s_xbar[group][buf]), xphase[buf])) s_fail[group] = 1;
+            xphase[buf] ^= 1u;
+            group_sync(group);
+            if (s_fail[group]) { failed = true; break; }
+        } else {
+            cp_async_commit();      // group of the next tile (empty after the last one)
+            cp_async_wait<1>();     // this tile has landed
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            group_sync(group);
+        }
 
         // ---- layer 1: D = X W1 + b1 (operands from shared memory), one MMA per 16 values of k
         if (gt == 0) {
@@ -530,10 +566,37 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(MapView map,
     }
 }
 
+// Tensor map of x [B][H][T][128] (bf16, strides in elements) with boxes of 8 x 128 elements; false if the
+// driver entry point is missing or the strides do not fit a tensor map.
+static bool make_x_tensor_map(CUtensorMap *tm, TensorView x, int B, int H, int T) {
+    typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                 const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn fn = nullptr;
+    static bool looked = false;
+    if (!looked) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+        else
+            cudaGetLastError();
+        looked = true;
+    }
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)T, (cuuint64_t)H, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)x.sn * 2, (cuuint64_t)x.sh * 2, (cuuint64_t)x.sb * 2};   // bytes
+    const cuuint32_t box[4] = {8u, (cuuint32_t)kTcTile, 1u, 1u}, estr[4] = {1u, 1u, 1u, 1u};
+    for (int i = 0; i < 3; ++i)
+        if (strides[i] == 0 || (strides[i] & 15)) return false;
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<uint16_t *>(x.ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 cudaError_t launch_encode_umma(const MapView &map, int heads_per_kv, TensorView x, int B, int H, int T, uint32_t *codes,
                                long long c_sb, long long c_sh, uint32_t *status, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(encode_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kU_Smem);
-    if (e != cudaSuccess) return e;
     const int n_nets = H / heads_per_kv;
     const long long n_net = (long long)heads_per_kv * B * ((T + kTcTile - 1) / kTcTile);   // tiles per network
     if (n_net <= 0 || n_nets <= 0) return cudaSuccess;
@@ -541,8 +604,18 @@ cudaError_t launch_encode_umma(const MapView &map, int heads_per_kv, TensorView 
     if (per < 1) per = 1;
     if (per > (n_net + 1) / 2) per = (n_net + 1) / 2;    // at least two tiles (one per group) for a CTA to be worth it
     if (per < 1) per = 1;
-    encode_umma_kernel<<<(int)(n_nets * per), kU_Threads, kU_Smem, st>>>(map, heads_per_kv, x, B, H, T, (int)per, codes,
-                                                                        c_sb, c_sh, status);
+    CUtensorMap tm;
+    memset(&tm, 0, sizeof(tm));
+    const bool tma = make_x_tensor_map(&tm, x, B, H, T);
+    cudaError_t e = tma ? cudaFuncSetAttribute(encode_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kU_Smem)
+                        : cudaFuncSetAttribute(encode_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kU_Smem);
+    if (e != cudaSuccess) return e;
+    if (tma)
+        encode_umma_kernel<true><<<(int)(n_nets * per), kU_Threads, kU_Smem, st>>>(tm, map, heads_per_kv, x, B, H, T, (int)per,
+                                                                                  codes, c_sb, c_sh, status);
+    else
+        encode_umma_kernel<false><<<(int)(n_nets * per), kU_Threads, kU_Smem, st>>>(tm, map, heads_per_kv, x, B, H, T, (int)per,
+                                                                                   codes, c_sb, c_sh, status);
     count_launch();
     return cudaGetLastError();
 }
