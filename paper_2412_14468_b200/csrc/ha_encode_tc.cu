@@ -319,14 +319,15 @@ __device__ __forceinline__ void relu_split_pair(float v0, float v1, uint32_t &hi
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo) : "f"(r1), "f"(r0));
 }
 
-// One k-chunk of a token tile (8 values of k x 128 tokens) through the tensor map of x [B][H][T][128]: the
-// box lands as 128 consecutive 16-byte rows, which is the core-matrix layout the MMA descriptor names.
-__device__ __forceinline__ void tma_load_chunk(uint32_t dst, const CUtensorMap *tmap, int k0, int t0, int h, int b, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-                 ::"r"(dst), "l"(tmap), "r"(k0), "r"(t0), "r"(h), "r"(b), "r"(bar) : "memory");
+// A whole token tile through the tensor map of x seen as [B][H][16 k-chunks][T][8]: the box of 8 x 128 x 16
+// elements lands chunk after chunk, each as 128 consecutive 16-byte rows, which is the core-matrix layout
+// the MMA descriptor names (k-chunk stride 2048 bytes).  One instruction per tile.
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap *tmap, int t0, int h, int b, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                 ::"r"(dst), "l"(tmap), "r"(0), "r"(t0), "r"(0), "r"(h), "r"(b), "r"(bar) : "memory");
 }
 
-// kTma: token tiles arrive through TMA (one thread per group issues 16 box copies and the tile's mbarrier
+// kTma: token tiles arrive through TMA (one thread per group issues one box copy and the tile's mbarrier
 // counts the bytes); otherwise every thread copies 16-byte pieces with cp.async.
 template <bool kTma>
 __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid_constant__ CUtensorMap tmap, MapView map,
@@ -422,7 +423,7 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid
         t0 = (int)(r - (long long)b * tiles_per_row) * kTcTile;
     };
     // token tile, K-major core matrices: element (row r, k) at (k/8) * kU_XLbo + (r/8) * 128 + (r%8) * 16 + (k%8) * 2.
-    // TMA: 16 box copies of 8 x 128 elements; rows past T are filled with zeros by the tensor map.
+    // TMA: one box copy per tile; rows past T are filled with zeros by the tensor map.
     // Threads: a half-warp copies one 256-byte row (whole lines on the global side, 16 different banks on the
     // shared side thanks to the padded chunk stride).
     auto load_x = [&](long long w, int buf) {
@@ -433,8 +434,7 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid
             if (gt == 0) {
                 const uint32_t xb = smem_u32(&s_xbar[group][buf]);
                 mbar_expect_tx(xb, kTcTile * kD * 2);
-#pragma unroll
-                for (int ch = 0; ch < 16; ++ch) tma_load_chunk(dst + ch * kU_XLbo, &tmap, 8 * ch, t0, h, b, xb);
+                tma_load_tile(dst, &tmap, t0, h, b, xb);
             }
         } else {
             const unsigned char *src = reinterpret_cast<const unsigned char *>(x.ptr + (long long)b * x.sb + (long long)h * x.sh);
@@ -566,8 +566,8 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid
     }
 }
 
-// Tensor map of x [B][H][T][128] (bf16, strides in elements) with boxes of 8 x 128 elements; false if the
-// driver entry point is missing or the strides do not fit a tensor map.
+// Tensor map of x [B][H][T][128] (bf16, strides in elements) seen as [B][H][16][T][8], with boxes of
+// 8 x 128 x 16 elements; false if the driver entry point is missing or the strides do not fit a tensor map.
 static bool make_x_tensor_map(CUtensorMap *tm, TensorView x, int B, int H, int T) {
     typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -585,12 +585,12 @@ static bool make_x_tensor_map(CUtensorMap *tm, TensorView x, int B, int H, int T
         looked = true;
     }
     if (!fn) return false;
-    const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)T, (cuuint64_t)H, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)x.sn * 2, (cuuint64_t)x.sh * 2, (cuuint64_t)x.sb * 2};   // bytes
-    const cuuint32_t box[4] = {8u, (cuuint32_t)kTcTile, 1u, 1u}, estr[4] = {1u, 1u, 1u, 1u};
-    for (int i = 0; i < 3; ++i)
+    const cuuint64_t dims[5] = {8u, (cuuint64_t)T, (cuuint64_t)(kD / 8), (cuuint64_t)H, (cuuint64_t)B};
+    const cuuint64_t strides[4] = {(cuuint64_t)x.sn * 2, 16u, (cuuint64_t)x.sh * 2, (cuuint64_t)x.sb * 2};   // bytes
+    const cuuint32_t box[5] = {8u, (cuuint32_t)kTcTile, (cuuint32_t)(kD / 8), 1u, 1u}, estr[5] = {1u, 1u, 1u, 1u, 1u};
+    for (int i = 0; i < 4; ++i)
         if (strides[i] == 0 || (strides[i] & 15)) return false;
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<uint16_t *>(x.ptr), dims, strides, box, estr,
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<uint16_t *>(x.ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
