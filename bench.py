@@ -421,7 +421,8 @@ def main():
             xk = torch.randn(1, 8, 32768, 128, device=device, generator=gq).to(torch.bfloat16)
             ck = torch.zeros(1, 8, 32768, dtype=torch.int32, device=device)
             res = {}
-            for nm, fn in (("chain_exact_us", ha.ha_encode), ("tensor_core_us", ha.ha_encode_prefill)):
+            f_sync = lambda m_, h_, x_, o_: ha.ha_encode_prefill(m_, h_, x_, o_, path=ha.HA_PREFILL_MMA_SYNC)
+            for nm, fn in (("chain_exact_us", ha.ha_encode), ("mma_sync_us", f_sync), ("tcgen05_us", ha.ha_encode_prefill)):
                 for _ in range(3):
                     fn(mm, 1, xk, ck)
                 torch.cuda.synchronize()
@@ -432,7 +433,8 @@ def main():
                 e1.record()
                 torch.cuda.synchronize()
                 res[nm] = e0.elapsed_time(e1) * 100.0
-            res["algorithmic_tflops_tensor_core"] = 8 * 32768 * 2 * (128 * 128 * 2 + 128 * 32) / res["tensor_core_us"] / 1e6
+            res["algorithmic_tflops_tcgen05"] = 8 * 32768 * 2 * (128 * 128 * 2 + 128 * 32) / res["tcgen05_us"] / 1e6
+            res["input_gbs_tcgen05"] = 8 * 32768 * 256 / res["tcgen05_us"] / 1e3
             supplementary["prefill_encode_32K_tokens_8_heads"] = res
             del xk, ck
             torch.cuda.empty_cache()
