@@ -15,6 +15,30 @@ from . import binding as ha
 from . import workloads as wl
 
 
+def prefill(args):
+    cfg = wl.CONFIGS[args.config]
+    B = args.batch if args.batch is not None else cfg.batch
+    T = cfg.n
+    assert T is not None, "prefill runs need a config with one fixed length"
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    Hkv = cfg.n_kv_heads
+    g = torch.Generator(dev).manual_seed(wl.BASE_SEED + 78)
+    mp = ha.Mapping(wl.make_mapping(Hkv, g, dev))
+    x = torch.randn(B, Hkv, T, 128, device=dev, generator=g).to(torch.bfloat16)
+    codes = torch.zeros(B, Hkv, T, dtype=torch.int32, device=dev)
+    torch.cuda.synchronize()
+    for s in range(args.steps):
+        for name, path in (("tcgen05", ha.HA_PREFILL_TCGEN05), ("mma.sync", ha.HA_PREFILL_MMA_SYNC)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ha.ha_encode_prefill(mp, 1, x, codes, path=path)
+            e1.record()
+            torch.cuda.synchronize()
+            print(f"step {s} {name}: {e0.elapsed_time(e1) * 1e3:.1f} us")
+    print("key bytes per call:", B * Hkv * T * 256, " algorithmic flop per call:", B * Hkv * T * 2 * (128 * 128 * 2 + 128 * 32))
+
+
 def score_only(args):
     cfg = wl.CONFIGS[args.config]
     B = args.batch if args.batch is not None else cfg.batch
@@ -50,11 +74,15 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--dense", action="store_true", help="also run the dense comparator each step")
+    ap.add_argument("--prefill", action="store_true",
+                    help="prompt ENCODE alone (tcgen05 and mma.sync kernels) on --batch sequences of the config's length")
     ap.add_argument("--score-only", action="store_true",
                     help="SCORE + TOPK alone on random signatures (no K/V allocated: large batches stay small)")
     args = ap.parse_args()
     if args.score_only:
         return score_only(args)
+    if args.prefill:
+        return prefill(args)
     cfg = wl.CONFIGS[args.config]
     if args.batch is not None:
         cfg = dataclasses.replace(cfg, batch=args.batch)
