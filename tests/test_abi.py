@@ -98,6 +98,27 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.ha_dense_decode(C.byref(s0), fake, C.byref(t), C.byref(t), fake, 16, fake, None, fake, 1 << 30, None) == ha.HA_OK
 
 
+def test_windows_and_prefill_arguments_are_checked_on_the_host(lib):
+    fake = 0x1000
+    # always-kept windows: negative sizes, and windows that do not fit the index rows
+    neg = ha.make_shape(1, 32, 8, 0.088, n_sink=-1)
+    assert lib.ha_score_topk(C.byref(neg), fake, fake, 16, 16, fake, None, 4, 16, 4, fake, 0, 0, fake, None, fake, 1 << 30, None) \
+        == ha.HA_ERR_INVALID_ARG
+    wide = ha.make_shape(1, 32, 8, 0.088, n_sink=128, n_local=128)
+    assert lib.ha_score_topk(C.byref(wide), fake, fake, 16, 16, fake, None, 4, 4096, 255, fake, 0, 0, fake, None, fake, 1 << 30, None) \
+        == ha.HA_ERR_INVALID_ARG
+    assert ha.ha_workspace_bytes(wide, 32768, 1280) == ha.ha_workspace_bytes(ha.make_shape(1, 32, 8, 0.088), 32768, 1280)
+    # prompt encoder: unknown path, misaligned workspace, mismatching head counts; an empty call succeeds
+    m = ha.ha_mapping(8, 128, 128, 32, fake, fake, fake, None, None, None)
+    t = ha.ha_tensor(fake, 1 << 20, 1 << 16, 128)
+    assert lib.ha_encode_prefill(C.byref(m), 1, C.byref(t), 1, 8, 64, fake, 64, 64, 7, None, None) == ha.HA_ERR_INVALID_ARG
+    assert lib.ha_encode_prefill(C.byref(m), 1, C.byref(t), 1, 8, 64, fake, 64, 64, ha.HA_PREFILL_TCGEN05, fake + 8, None) \
+        == ha.HA_ERR_WORKSPACE
+    assert lib.ha_encode_prefill(C.byref(m), 4, C.byref(t), 1, 8, 64, fake, 64, 64, ha.HA_PREFILL_MMA_SYNC, None, None) \
+        == ha.HA_ERR_INVALID_ARG
+    assert lib.ha_encode_prefill(C.byref(m), 1, C.byref(t), 1, 8, 0, fake, 64, 64, ha.HA_PREFILL_TCGEN05, None, None) == ha.HA_OK
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(ha, "_lib", None)
     monkeypatch.setattr(ha, "LIB_PATH", str(tmp_path / "nope.so"))
