@@ -220,7 +220,7 @@ cudaError_t launch_encode_tc(const MapView &map, int heads_per_kv, TensorView x,
 // ------------------------------------------------------------------ tcgen05 version
 //
 // The same chain of three GEMMs on the fifth-generation tensor cores.  A tile of 128 tokens is
-// M = 128 rows = the 128 lanes of tensor memory; thread r of a group of 128 threads owns row r.
+// M = 128 rows = the 128 lanes of tensor memory; threads r and r + 128 of a group own row r.
 //   layer 1  D[128 x 128] = X W1 + b1   A = token tile in shared memory (K-major core matrices),
 //                                       B = W1 in shared memory (N-major core matrices), 8 x K16;
 //                                       the bias is one more K16 step: A = a constant tile whose
@@ -231,14 +231,15 @@ cudaError_t launch_encode_tc(const MapView &map, int heads_per_kv, TensorView x,
 //   layer 2  D = A_hi W2 + A_lo W2 + b2  A from tensor memory, 16 x K16 + the bias step
 //   layer 3  D[128 x 32] likewise; the epilogue packs the 32 sign bits of a row into its code.
 // Activations never leave tensor memory and registers.
-// Two groups of 128 threads work on alternate tiles with their own token buffers, their own half of
+// Two groups of 256 threads (two per token row, each converting half of the columns) work on alternate tiles with their own token buffers, their own half of
 // tensor memory (D 128 + A_hi 64 + A_lo 64 columns) and their own mbarrier, so that one group's
 // tensor-core work runs under the other group's epilogue.  A CTA stays with one network: its
 // weights are loaded once.  MMAs are issued by the first thread of a group and tracked with
 // tcgen05.commit; every wait is bounded: on a timeout the group raises HA_DEV_TIMEOUT in the status
 // word and stops, and the CTA frees its tensor memory and returns.
 
-constexpr int kU_Threads = 256;                   // two groups of 128
+constexpr int kU_GroupThreads = 256;              // two threads per token row: each converts half of the columns
+constexpr int kU_Threads = 2 * kU_GroupThreads;   // two groups
 constexpr int kU_KG = kD / 8 + 2;                 // k-groups of 8 rows per weight matrix: 16 + 2 for the bias step
 constexpr int kU_WBytes = kU_KG * 2048;           // 36864: W1 or W2 as k-groups x 16 n-blocks x (8 x 16 B)
 constexpr int kU_W3Bytes = kU_KG * 512;           // 9216
@@ -295,7 +296,7 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void group_sync(int group) { asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory"); }
+__device__ __forceinline__ void group_sync(int group) { asm volatile("bar.sync %0, 256;" ::"r"(group + 1) : "memory"); }
 
 // try_wait parks the warp for a bounded time instead of spinning, so a waiting group leaves the issue
 // slots to the group that is converting; the number of attempts is bounded as well.
@@ -343,7 +344,8 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid
     __shared__ __align__(8) unsigned long long s_xbar[2][2];   // [group][buffer]: arrival of a token tile (TMA)
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_fail[2];
-    const int tid = threadIdx.x, warp = tid >> 5, group = tid >> 7, gt = tid & 127;
+    const int tid = threadIdx.x, warp = tid >> 5, group = tid >> 8, gt = tid & 255;
+    const int row = gt & 127, half = gt >> 7;   // thread (row, half) converts columns 64 half .. 64 half + 63 of its row
     const int tiles_per_row = (T + kTcTile - 1) / kTcTile;
     const int net = blockIdx.x / ctas_per_net, part = blockIdx.x % ctas_per_net;
     // tiles of this network in the order (head of the network, sequence, tile); this CTA takes a contiguous share
@@ -410,7 +412,7 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem_base + group * kU_SlotCols;                 // this group's half
-    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 lanes
+    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 lanes (warps w and w + 4 share them)
     const uint32_t bar = smem_u32(&s_mbar[group]);
     unsigned char *gX = sX + group * 2 * kU_XBytes;
 
@@ -439,11 +441,11 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid
         } else {
             const unsigned char *src = reinterpret_cast<const unsigned char *>(x.ptr + (long long)b * x.sb + (long long)h * x.sh);
 #pragma unroll
-            for (int i = 0; i < kTcTile * 16 / 128; ++i) {
-                const int e = gt + i * 128, row = e >> 4, ch = e & 15;
-                const bool ok = t0 + row < T;
-                cp_async16(dst + ch * kU_XLbo + (row >> 3) * 128 + (row & 7) * 16,
-                           src + (long long)(ok ? t0 + row : 0) * x.sn * 2 + ch * 16, ok ? 16u : 0u);
+            for (int i = 0; i < kTcTile * 16 / kU_GroupThreads; ++i) {
+                const int e = gt + i * kU_GroupThreads, r = e >> 4, ch = e & 15;
+                const bool ok = t0 + r < T;
+                cp_async16(dst + ch * kU_XLbo + (r >> 3) * 128 + (r & 7) * 16,
+                           src + (long long)(ok ? t0 + r : 0) * x.sn * 2 + ch * 16, ok ? 16u : 0u);
             }
         }
     };
@@ -460,20 +462,20 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid
         group_sync(group);
         return s_fail[group] == 0;
     };
-    // this thread's row of the 128-column accumulator -> ReLU, hi / lo -> the A operand columns
+    // this thread's half row of the 128-column accumulator -> ReLU, hi / lo -> the A operand columns
     auto epilogue_hidden = [&]() {
-        uint32_t v[4][32];   // the whole row is requested at once: one tensor-memory round trip, not four
+        uint32_t v[2][32];   // both pieces are requested at once: one tensor-memory round trip
 #pragma unroll
-        for (int q = 0; q < 4; ++q) tmem_ld32(lane_base + kU_ColD + q * 32, v[q]);
+        for (int q = 0; q < 2; ++q) tmem_ld32(lane_base + kU_ColD + (2 * half + q) * 32, v[q]);
         tmem_wait_ld();
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < 2; ++q) {
             uint32_t hi[16], lo[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i)
                 relu_split_pair(__uint_as_float(v[q][2 * i]), __uint_as_float(v[q][2 * i + 1]), hi[i], lo[i]);
-            tmem_st16(lane_base + kU_ColAhi + q * 16, hi);
-            tmem_st16(lane_base + kU_ColAlo + q * 16, lo);
+            tmem_st16(lane_base + kU_ColAhi + (2 * half + q) * 16, hi);
+            tmem_st16(lane_base + kU_ColAlo + (2 * half + q) * 16, lo);
         }
         tmem_wait_st();
         tc_fence_before();
@@ -544,14 +546,14 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid
             umma_commit(bar);
         }
         if (!wait_mma()) { failed = true; break; }
-        {
+        if (half == 0) {   // warp-uniform
             uint32_t v[32];
             tmem_ld32(lane_base + kU_ColD, v);
             tmem_wait_ld();
             uint32_t code = 0u;
 #pragma unroll
             for (int o = 0; o < 32; ++o) code |= (__uint_as_float(v[o]) > 0.0f ? 1u : 0u) << o;
-            if (t0 + gt < T) codes[(long long)b * c_sb + (long long)h * c_sh + t0 + gt] = code;
+            if (t0 + row < T) codes[(long long)b * c_sb + (long long)h * c_sh + t0 + row] = code;
         }
         tc_fence_before();
         group_sync(group);   // the group is done with this token buffer and with D before they are reused
