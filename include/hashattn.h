@@ -171,6 +171,23 @@ int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
                    int64_t idx_stride_b, int64_t idx_stride_h, const int32_t *count, int32_t k_max,
                    uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream);
 
+/* GATHER-ATT over a paged K/V cache (Section 4.4: K/V rows are read in place through the indices; the
+ * paper's vLLM integration keeps K/V in pages addressed through a block table).  Same computation and
+ * arguments as ha_gather_attn, except that token t of sequence b is found in page
+ * block_table[b * bt_stride_b + t / page_size] at slot t % page_size:
+ *   K_pool, V_pool  bf16 rows [n_pages][n_kv_heads][page_size][128] described by (stride_b = page stride,
+ *                   stride_h = head stride, stride_n = slot stride), elements; both pools must have the same
+ *                   number of rows per page stride (stride_b / stride_n, an integer)
+ *   block_table     i32 [batch][>= ceil(seq_len / page_size)] page numbers (device)
+ *   page_size       power of two (1 = every token its own page)
+ * The index lists hold logical token numbers, exactly as ha_score_topk writes them (the signature cache
+ * stays one contiguous array per sequence and KV head: 4 bytes per token). */
+int ha_gather_attn_paged(const ha_shape *shape, const uint16_t *q, const ha_tensor *K_pool,
+                         const ha_tensor *V_pool, const int32_t *block_table, int64_t bt_stride_b,
+                         int32_t page_size, const int32_t *seq_lens, const int32_t *idx,
+                         int64_t idx_stride_b, int64_t idx_stride_h, const int32_t *count, int32_t k_max,
+                         uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream);
+
 /* Dense decode attention — single-query SDPA over all seq_len tokens (Section 3.1): the
  * computation the sparse path replaces, provided as the same-run comparator. */
 int ha_dense_decode(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,

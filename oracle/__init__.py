@@ -117,6 +117,17 @@ def gather_attn(q, K, V, idx, sm_scale=None, n_valid=None):
     return out, lse.value, out64
 
 
+def unpage_rows(pool, block_table_row, page_size: int, head: int, n: int) -> np.ndarray:
+    """Rows 0..n-1 of one sequence and KV head out of a paged cache (Section 4.4: K/V are read in place; the
+    vLLM integration keeps them in pages): pool is [n_pages, Hkv, page_size, 128]; token t lives in page
+    block_table_row[t // page_size] at slot t % page_size.  Paging is storage only: GATHER-ATT over a paged
+    cache is gather_attn over these rows."""
+    pool = _u16(pool)
+    t = np.arange(n)
+    pages = np.asarray(block_table_row, dtype=np.int64)[t // page_size]
+    return np.ascontiguousarray(pool[pages, head, t % page_size, :])
+
+
 def dense(q, K, V, n=None, sm_scale=None):
     """SDPA for one query over tokens 0..n-1."""
     return gather_attn(q, K, V, None, sm_scale=sm_scale, n_valid=n)

@@ -22,6 +22,7 @@ HIST_BINS = 33
 
 EXPORTS = [
     "ha_workspace_bytes", "ha_workspace_init", "ha_encode", "ha_encode_prefill", "ha_score_topk", "ha_gather_attn",
+    "ha_gather_attn_paged",
     "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
@@ -67,6 +68,7 @@ def lib() -> C.CDLL:
         L.ha_encode_prefill.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, I32, P, P]
         L.ha_score_topk.argtypes = [P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64, P, P, P, SZ, P]
         L.ha_gather_attn.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P, SZ, P]
+        L.ha_gather_attn_paged.argtypes = [P, P, P, P, P, I64, I32, P, P, I64, I64, P, I32, P, P, P, SZ, P]
         L.ha_gather_attn_static.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P]
         L.ha_dense_decode.argtypes = [P, P, P, P, P, I32, P, P, P, SZ, P]
         L.ha_sparse_decode.argtypes = [P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, P, I64, I64, P,
@@ -223,6 +225,17 @@ def ha_gather_attn(shape: ha_shape, q, K, V, seq_lens, idx, count, k_max: int, o
     _check("ha_gather_attn", lib().ha_gather_attn(
         C.byref(shape), q.data_ptr(), C.byref(kt), C.byref(vt), seq_lens.data_ptr(), idx.data_ptr(), idx.stride(0),
         idx.stride(1), count.data_ptr(), k_max, out.data_ptr(), _ptr(lse), p, n, _stream(stream)))
+
+
+def ha_gather_attn_paged(shape: ha_shape, q, K_pool, V_pool, block_table, page_size: int, seq_lens, idx, count, k_max: int,
+                         out, workspace, lse=None, stream=None) -> None:
+    """K_pool, V_pool: bf16 [n_pages, Hkv, page_size, 128]; block_table: int32 [B, pages per sequence]."""
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K_pool), make_tensor(V_pool)
+    _check("ha_gather_attn_paged", lib().ha_gather_attn_paged(
+        C.byref(shape), q.data_ptr(), C.byref(kt), C.byref(vt), block_table.data_ptr(), block_table.stride(0), page_size,
+        seq_lens.data_ptr(), idx.data_ptr(), idx.stride(0), idx.stride(1), count.data_ptr(), k_max, out.data_ptr(),
+        _ptr(lse), p, n, _stream(stream)))
 
 
 def ha_gather_attn_static(shape: ha_shape, q, K, V, seq_lens, idx, count, k_max: int, out, lse=None, stream=None) -> None:

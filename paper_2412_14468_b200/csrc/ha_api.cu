@@ -184,6 +184,33 @@ int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
     return HA_OK;
 }
 
+int ha_gather_attn_paged(const ha_shape *shape, const uint16_t *q, const ha_tensor *K_pool, const ha_tensor *V_pool,
+                         const int32_t *block_table, int64_t bt_stride_b, int32_t page_size, const int32_t *seq_lens,
+                         const int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, const int32_t *count,
+                         int32_t k_max, uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream) {
+    HA_TRY(check_shape(shape));
+    HA_TRY(check_tensor(K_pool));
+    HA_TRY(check_tensor(V_pool));
+    if (!q || !block_table || !seq_lens || !idx || !count || !out || k_max < 0) return HA_ERR_INVALID_ARG;
+    if ((uintptr_t)q & 15) return HA_ERR_INVALID_ARG;
+    if (page_size <= 0 || (page_size & (page_size - 1)) || page_size > 65536) return HA_ERR_INVALID_ARG;
+    // a page is page_size consecutive slots: both pools must step through pages in whole rows, the same way
+    if (K_pool->stride_b % K_pool->stride_n != 0 || V_pool->stride_b % V_pool->stride_n != 0 ||
+        K_pool->stride_b / K_pool->stride_n != V_pool->stride_b / V_pool->stride_n)
+        return HA_ERR_INVALID_ARG;
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(shape, -1, workspace, ws_bytes, &L));
+    if (shape->batch == 0) return HA_OK;
+    int shift = 0;
+    while ((1 << shift) < page_size) ++shift;
+    HA_CUDA(launch_attention(true, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K_pool),
+                             view(V_pool), seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
+                             ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),
+                             ws_ptr<int32_t>(workspace, L.off_tickets), ws_ptr<uint32_t>(workspace, 0),
+                             (cudaStream_t)stream, 0, nullptr, 0, Windows{0, 0}, block_table, bt_stride_b, shift));
+    return HA_OK;
+}
+
 int ha_dense_decode(const ha_shape *shape, const uint16_t *q, const ha_tensor *K, const ha_tensor *V,
                     const int32_t *seq_lens, int32_t max_seq_len, uint16_t *out, float *lse, void *workspace,
                     size_t ws_bytes, void *stream) {

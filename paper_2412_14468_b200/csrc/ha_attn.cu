@@ -35,6 +35,11 @@ struct AttnArgs {
     const int32_t *k_per_seq;   // with count_from_k: budget per sequence (or NULL: k_uniform)
     int k_uniform, count_from_k;
     Windows win;                // with count_from_k: tokens always kept in addition to the budget
+    // paged K/V (block_table != NULL): token t of sequence b lives in page block_table[b*bt_sb + (t >> page_shift)],
+    // slot t & (2^page_shift - 1); K.sb / V.sb are then the page strides and page_rows = K.sb / K.sn
+    const int32_t *block_table;
+    long long bt_sb;
+    int page_shift, page_rows;
     int max_items, Hq, Hkv, n_units, balanced;
     float scale_log2;
     float *part_ml, *part_acc;
@@ -172,8 +177,10 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
         const long long head0 = (long long)b * Hq + (long long)kvh * G;
         const int start = blk_lo * kBlockTokens, end = min(cnt, blk_hi * kBlockTokens);
 
-        const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (long long)b * a.K.sb + (long long)kvh * a.K.sh);
-        const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (long long)b * a.V.sb + (long long)kvh * a.V.sh);
+        const bool paged = kGather && a.block_table != nullptr;   // rows are then addressed from the pool's base
+        const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (paged ? 0LL : (long long)b * a.K.sb) + (long long)kvh * a.K.sh);
+        const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (paged ? 0LL : (long long)b * a.V.sb) + (long long)kvh * a.V.sh);
+        const int32_t *pages = paged ? a.block_table + (long long)b * a.bt_sb : nullptr;
         const long long k_row = a.K.sn * 2, v_row = a.V.sn * 2;   // bytes
         const int32_t *list = kGather ? a.idx + (long long)b * a.idx_sb + (long long)kvh * a.idx_sh : nullptr;
 
@@ -184,6 +191,8 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
         auto token_of = [&](int p, int raw) -> int {
             int t = (p < end) ? raw : -1;
             if (t >= n) { bad = true; t = -1; }
+            // paged: logical token -> row of the pool (page * rows per page + slot)
+            if (paged && t >= 0) t = __ldg(pages + (t >> a.page_shift)) * a.page_rows + (t & ((1 << a.page_shift) - 1));
             return t;
         };
         auto issue = [&](int stg, int my_t) {
@@ -437,9 +446,11 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
                              uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
                              uint32_t *status, cudaStream_t st, int count_from_k, const int32_t *k_per_seq,
-                             int k_uniform, Windows win) {
+                             int k_uniform, Windows win, const int32_t *block_table, long long bt_sb, int page_shift) {
     AttnArgs a{};
     a.win = win;
+    a.block_table = block_table; a.bt_sb = bt_sb; a.page_shift = page_shift;
+    a.page_rows = (block_table && K.sn > 0) ? (int)(K.sb / K.sn) : 0;
     a.q = q; a.K = K; a.V = V; a.seq_lens = seq_lens; a.idx = idx; a.count = count;
     a.idx_sb = idx_sb; a.idx_sh = idx_sh; a.max_items = max_items; a.Hq = Hq; a.Hkv = Hkv;
     a.n_units = B * Hkv; a.scale_log2 = sm_scale * kLog2e;

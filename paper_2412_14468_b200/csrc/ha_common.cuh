@@ -182,7 +182,8 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
                              uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
                              uint32_t *status, cudaStream_t st, int count_from_k = 0,
-                             const int32_t *k_per_seq = nullptr, int k_uniform = 0, Windows win = Windows{0, 0});
+                             const int32_t *k_per_seq = nullptr, int k_uniform = 0, Windows win = Windows{0, 0},
+                             const int32_t *block_table = nullptr, long long bt_sb = 0, int page_shift = 0);
 
 // The whole layer-step in one launch (one 8-CTA cluster per unit); only for small batches.
 bool fused_step_eligible(int B, int Hkv, int max_seq_len);

@@ -384,6 +384,48 @@ def test_dense_decode_matches_oracle(lens):
                 assert abs(float(lse[b, h]) - el) < 1e-3
 
 
+@pytest.mark.parametrize("page_size", [1, 16, 64])
+def test_gather_attn_over_a_paged_cache(page_size):
+    """K/V rows live in pages scattered over a pool and are found through a block table (page sizes 1 and 16
+    of the vLLM integration, and a larger one); results equal the oracle over the un-paged rows."""
+    rng = np.random.default_rng(40 + page_size)
+    B, Hq, Hkv = 3, 8, 2
+    lens = [300, 2049, 17]
+    n_cap = max(lens)
+    g = torch.Generator(DEV).manual_seed(page_size)
+    q = torch.randn(B, Hq, 128, device=DEV, generator=g).to(torch.bfloat16)
+    pages_per_seq = (n_cap + page_size - 1) // page_size
+    n_pages = B * pages_per_seq + 5
+    K_pool = torch.randn(n_pages, Hkv, page_size, 128, device=DEV, generator=g).to(torch.bfloat16)
+    V_pool = torch.randn(n_pages, Hkv, page_size, 128, device=DEV, generator=g).to(torch.bfloat16)
+    table = torch.from_numpy(rng.permutation(n_pages)[:B * pages_per_seq].reshape(B, pages_per_seq).astype(np.int32)).to(DEV)
+    k_max = 256
+    idx_np = np.full((B, Hkv, k_max), -1, np.int32)
+    cnt_np = np.zeros((B, Hkv), np.int32)
+    for b, n in enumerate(lens):
+        for h in range(Hkv):
+            c = min(n, int(rng.integers(1, k_max + 1)))
+            idx_np[b, h, :c] = np.sort(rng.choice(n, size=c, replace=False))
+            cnt_np[b, h] = c
+    shape = ha.make_shape(B, Hq, Hkv, 1.0 / np.sqrt(128))
+    ws = ha.alloc_workspace(shape, n_cap, k_max)
+    out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(B, Hq, device=DEV)
+    ha.ha_gather_attn_paged(shape, q, K_pool, V_pool, table, page_size, torch.tensor(lens, dtype=torch.int32, device=DEV),
+                            torch.from_numpy(idx_np).to(DEV), torch.from_numpy(cnt_np).to(DEV), k_max, out, ws, lse=lse)
+    torch.cuda.synchronize()
+    assert ha.ha_read_device_status(ws) == 0
+    G = Hq // Hkv
+    qu, Kp, Vp, tb = u16(q), u16(K_pool), u16(V_pool), table.cpu().numpy()
+    for b, n in enumerate(lens):
+        for h in range(Hkv):
+            Kr, Vr = oracle.unpage_rows(Kp, tb[b], page_size, h, n), oracle.unpage_rows(Vp, tb[b], page_size, h, n)
+            for j in range(G):
+                eo, el, _ = oracle.gather_attn(qu[b, h * G + j], Kr, Vr, idx_np[b, h, :cnt_np[b, h]], sm_scale=1.0 / np.sqrt(128))
+                assert_out_close(u16(out[b, h * G + j]), eo)
+                assert abs(float(lse[b, h * G + j]) - el) < 1e-3
+
+
 # ---------------------------------------------------------------------------- whole step
 
 def _run_step(w, host=False, pinned=True, n_sink=0, n_local=0):

@@ -173,3 +173,19 @@ def test_decode_step_is_the_composition_and_k_equals_n_is_dense():
         for h in range(Hq):
             out, lse, _ = oracle.dense(q[b, h], K[b, h // G], V[b, h // G], n=w["lens"][b])
             assert np.array_equal(full["out"][b, h], out) and abs(full["lse"][b, h] - lse) < 1e-12
+
+
+def test_unpaging_is_storage_only():
+    """A paged cache read back through its block table gives the rows that were put in, whatever the page
+    order and page size; attention over them equals attention over the contiguous rows."""
+    rng = np.random.default_rng(5)
+    n, Hkv = 70, 2
+    K = rng.integers(0, 2 ** 16, size=(Hkv, n, 128), dtype=np.uint64).astype(np.uint16) & 0xBFFF   # finite bf16 patterns
+    for ps in (1, 16, 64):
+        n_pages = (n + ps - 1) // ps
+        perm = rng.permutation(n_pages + 3)[:n_pages]                 # pages scattered over a larger pool
+        pool = np.zeros((n_pages + 3, Hkv, ps, 128), np.uint16)
+        for t in range(n):
+            pool[perm[t // ps], :, t % ps] = K[:, t]
+        for h in range(Hkv):
+            assert np.array_equal(oracle.unpage_rows(pool, perm, ps, h, n), K[h])
