@@ -414,6 +414,28 @@ def main():
                     "dense_us": t_de * 1e3 / 40, "dense_frac": wl.dense_bytes(l2) / (t_de * 1e3 / 40 * 1e-6) / 1e9 / peak,
                     "replicas": reps_n,
                 }
+                if name == "c3":   # the same lists over a paged copy of K/V (pages of 16 tokens scattered over a pool)
+                    ps, pools = 16, []
+                    for r in b2.reps:
+                        K, V = r.w["K"], r.w["V"]
+                        Bn, Hk, N, _ = K.shape
+                        pps = (N + ps - 1) // ps
+                        perm = torch.randperm(Bn * pps, device=device).to(torch.int32).reshape(Bn, pps)
+                        pool = []
+                        for X in (K, V):
+                            Xp = torch.zeros(Bn * pps, Hk, ps, 128, dtype=X.dtype, device=device)
+                            Xp[perm.reshape(-1).long(), :, :, :] = torch.nn.functional.pad(X, (0, 0, 0, pps * ps - N)) \
+                                .reshape(Bn, Hk, pps, ps, 128).permute(0, 2, 1, 3, 4).reshape(Bn * pps, Hk, ps, 128)
+                            pool.append(Xp)
+                        pools.append((pool[0], pool[1], perm))
+
+                    def gather_paged(r):
+                        Kp, Vp, perm = pools[b2.reps.index(r)]
+                        ha.ha_gather_attn_paged(r.shape, r.w["q"], Kp, Vp, perm, ps, r.w["seq_lens"], r.idx, r.cnt, r.w["k_max"],
+                                                r.out, b2.ws)
+                    t_pg, _ = b2.time_steps(gather_paged, st, 20)
+                    supplementary[name]["gather_attn_paged16_us"] = t_pg * 1e3 / st
+                    del pools
                 del b2
                 torch.cuda.empty_cache()
             except Exception as ex:   # supplementary numbers never take the headline down
