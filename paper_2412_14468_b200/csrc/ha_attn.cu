@@ -187,11 +187,12 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
         // raw list entry of position p for this lane; only the load is issued here, the value is first
         // looked at when its block is started, one iteration later, so the warp never waits on it
         auto fetch_raw = [&](int p) -> int { return (kGather && p < end) ? __ldg(list + p) : p; };
-        // token id from a raw entry (-1: past the slice, padding or outside the sequence)
-        auto token_of = [&](int p, int raw) -> int {
+        // row to fetch for a raw entry (-1: past the slice, padding or outside the sequence).  Contiguous cache:
+        // the token id itself; paged cache: page * rows per page stride + slot, which costs one more load,
+        // so rows are resolved one block before they are requested and list entries one block before that.
+        auto row_of = [&](int p, int raw) -> int {
             int t = (p < end) ? raw : -1;
             if (t >= n) { bad = true; t = -1; }
-            // paged: logical token -> row of the pool (page * rows per page + slot)
             if (paged && t >= 0) t = __ldg(pages + (t >> a.page_shift)) * a.page_rows + (t & ((1 << a.page_shift) - 1));
             return t;
         };
@@ -204,9 +205,9 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
         const int stride = kAttnWarps * kBlockTokens;
         const int first = start + warp * kBlockTokens;
         const int nblk = (first < end) ? (end - first + stride - 1) / stride : 0;
-        int raw[kStages];
+        int raw[kStages + 1];
 #pragma unroll
-        for (int i = 0; i < kStages; ++i) raw[i] = fetch_raw(first + i * stride + (lane & 15));
+        for (int i = 0; i < kStages + 1; ++i) raw[i] = fetch_raw(first + i * stride + (lane & 15));
 
         uint32_t qa[8][2];
         attn_load_q<G>(qa, a.q + head0 * kD, lane);
@@ -219,10 +220,11 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
 
 #pragma unroll
         for (int i = 0; i < kStages - 1; ++i) {
-            if (i < nblk) issue(i, token_of(first + i * stride + (lane & 15), raw[i]));
+            if (i < nblk) issue(i, row_of(first + i * stride + (lane & 15), raw[i]));
             cp_async_commit();
         }
-        int next_raw = raw[kStages - 1];   // list entries of block kStages-1
+        int next_row = row_of(first + (kStages - 1) * stride + (lane & 15), raw[kStages - 1]);   // row of block kStages-1
+        int after_raw = raw[kStages];                                                            // list entry of the block after it
         int st = 0;
         for (int i = 0; i < nblk; ++i) {
             {   // refill the stage that block i-1 just released
@@ -230,9 +232,10 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
                 const int pj = first + j * stride;
                 int stj = st + kStages - 1;
                 if (stj >= kStages) stj -= kStages;
-                if (j < nblk) issue(stj, token_of(pj + (lane & 15), next_raw));
+                if (j < nblk) issue(stj, next_row);
                 cp_async_commit();
-                next_raw = fetch_raw(pj + stride + (lane & 15));   // one block ahead
+                next_row = row_of(pj + stride + (lane & 15), after_raw);      // one block ahead
+                after_raw = fetch_raw(pj + 2 * stride + (lane & 15));         // two blocks ahead
             }
             cp_async_wait<kStages - 1>();
             __syncwarp();
