@@ -207,6 +207,17 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
                      int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
                      uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream);
 
+/* One whole layer-step over a paged K/V cache: ha_sparse_decode with K/V addressed as in
+ * ha_gather_attn_paged (pools + block table + page_size); the signature cache k_codes stays contiguous. */
+int ha_sparse_decode_paged(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
+                           const uint16_t *q, const uint16_t *k_new, const ha_tensor *K_pool,
+                           const ha_tensor *V_pool, const int32_t *block_table, int64_t bt_stride_b,
+                           int32_t page_size, uint32_t *k_codes, int64_t kc_stride_b, int64_t kc_stride_h,
+                           const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                           int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx,
+                           int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, uint16_t *out,
+                           float *lse, void *workspace, size_t ws_bytes, void *stream);
+
 /* The same layer-step driven from HOST buffers (the per-step inputs of a decoder: the new
  * query, key and value vectors; Section 4.1): copies q_host, k_new_host, v_new_host to the device
  * (staging inside the workspace), writes the new K/V rows into the resident cache at slot

@@ -22,7 +22,7 @@ HIST_BINS = 33
 
 EXPORTS = [
     "ha_workspace_bytes", "ha_workspace_init", "ha_encode", "ha_encode_prefill", "ha_score_topk", "ha_gather_attn",
-    "ha_gather_attn_paged",
+    "ha_gather_attn_paged", "ha_sparse_decode_paged",
     "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
@@ -73,6 +73,8 @@ def lib() -> C.CDLL:
         L.ha_dense_decode.argtypes = [P, P, P, P, P, I32, P, P, P, SZ, P]
         L.ha_sparse_decode.argtypes = [P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, P, I64, I64, P,
                                        P, P, P, SZ, P]
+        L.ha_sparse_decode_paged.argtypes = [P, P, P, P, P, P, P, P, I64, I32, P, I64, I64, P, P, I32, I32, I32, P, P, I64, I64,
+                                             P, P, P, P, SZ, P]
         L.ha_sparse_decode_host.argtypes = [P, P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64,
                                             P, P, P, SZ, P]
         L.ha_read_device_status.argtypes = [P, P, P]
@@ -267,6 +269,19 @@ def ha_sparse_decode(shape: ha_shape, map_q: Mapping, map_k: Optional[Mapping], 
         C.byref(vt), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1), seq_lens.data_ptr(), _ptr(k_per_seq),
         k_uniform, max_seq_len, k_max, q_codes.data_ptr(), idx.data_ptr(), idx.stride(0), idx.stride(1),
         count.data_ptr(), out.data_ptr(), _ptr(lse), p, n, _stream(stream)))
+
+
+def ha_sparse_decode_paged(shape: ha_shape, map_q: Mapping, map_k: Optional[Mapping], q, k_new, K_pool, V_pool, block_table,
+                           page_size: int, k_codes, seq_lens, k_per_seq, k_uniform: int, max_seq_len: int, k_max: int,
+                           q_codes, idx, count, out, workspace, lse=None, stream=None) -> None:
+    """The whole step over a paged K/V cache: pools bf16 [n_pages, Hkv, page_size, 128], block_table int32 [B, pages]."""
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K_pool), make_tensor(V_pool)
+    _check("ha_sparse_decode_paged", lib().ha_sparse_decode_paged(
+        C.byref(shape), map_q.ref, None if map_k is None else map_k.ref, q.data_ptr(), _ptr(k_new), C.byref(kt),
+        C.byref(vt), block_table.data_ptr(), block_table.stride(0), page_size, k_codes.data_ptr(), k_codes.stride(0),
+        k_codes.stride(1), seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform, max_seq_len, k_max, q_codes.data_ptr(),
+        idx.data_ptr(), idx.stride(0), idx.stride(1), count.data_ptr(), out.data_ptr(), _ptr(lse), p, n, _stream(stream)))
 
 
 def ha_sparse_decode_host(shape: ha_shape, map_q: Mapping, map_k: Mapping, q_host, k_new_host, v_new_host, K, V,

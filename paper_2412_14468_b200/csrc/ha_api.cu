@@ -230,12 +230,13 @@ int ha_dense_decode(const ha_shape *shape, const uint16_t *q, const ha_tensor *K
     return HA_OK;
 }
 
-int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k, const uint16_t *q,
-                     const uint16_t *k_new, const ha_tensor *K, const ha_tensor *V, uint32_t *k_codes,
-                     int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
-                     int32_t k_uniform, int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx,
-                     int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse,
-                     void *workspace, size_t ws_bytes, void *stream) {
+static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k, const uint16_t *q,
+                              const uint16_t *k_new, const ha_tensor *K, const ha_tensor *V, const int32_t *block_table,
+                              int64_t bt_stride_b, int page_shift, uint32_t *k_codes, int64_t kc_stride_b,
+                              int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                              int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx, int64_t idx_stride_b,
+                              int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse, void *workspace,
+                              size_t ws_bytes, void *stream) {
     HA_TRY(check_score_args(shape, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_uniform, k_per_seq,
                             max_seq_len, k_max, idx, count));
     HA_TRY(check_mapping(map_q, shape->n_kv_heads));
@@ -254,7 +255,7 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
         HA_CUDA(launch_fused_step(B, Hq, Hkv, shape->sm_scale, view(map_q), k_new ? view(map_k) : MapView{}, q, k_new,
                                   view(K), view(V), k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
                                   max_seq_len, k_max, q_codes, idx, idx_stride_b, idx_stride_h, count, out, lse, st,
-                                  Windows{shape->n_sink, shape->n_local}));
+                                  Windows{shape->n_sink, shape->n_local}, block_table, bt_stride_b, page_shift));
         return HA_OK;
     }
 
@@ -281,8 +282,38 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
                              idx_stride_h, count, k_max, out, lse, ws_ptr<float>(workspace, L.off_part_ml),
                              ws_ptr<float>(workspace, L.off_part_acc), ws_ptr<int32_t>(workspace, L.off_tickets),
                              ws_ptr<uint32_t>(workspace, 0), st, /*count_from_k=*/1, k_per_seq, k_uniform,
-                             Windows{shape->n_sink, shape->n_local}));
+                             Windows{shape->n_sink, shape->n_local}, block_table, bt_stride_b, page_shift));
     return HA_OK;
+}
+
+int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k, const uint16_t *q,
+                     const uint16_t *k_new, const ha_tensor *K, const ha_tensor *V, uint32_t *k_codes,
+                     int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
+                     int32_t k_uniform, int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx,
+                     int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse,
+                     void *workspace, size_t ws_bytes, void *stream) {
+    return sparse_decode_impl(shape, map_q, map_k, q, k_new, K, V, nullptr, 0, 0, k_codes, kc_stride_b, kc_stride_h, seq_lens,
+                              k_per_seq, k_uniform, max_seq_len, k_max, q_codes, idx, idx_stride_b, idx_stride_h, count, out,
+                              lse, workspace, ws_bytes, stream);
+}
+
+int ha_sparse_decode_paged(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k, const uint16_t *q,
+                           const uint16_t *k_new, const ha_tensor *K_pool, const ha_tensor *V_pool,
+                           const int32_t *block_table, int64_t bt_stride_b, int32_t page_size, uint32_t *k_codes,
+                           int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
+                           int32_t k_uniform, int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx,
+                           int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse,
+                           void *workspace, size_t ws_bytes, void *stream) {
+    if (!block_table || !K_pool || !V_pool) return HA_ERR_INVALID_ARG;
+    if (page_size <= 0 || (page_size & (page_size - 1)) || page_size > 65536) return HA_ERR_INVALID_ARG;
+    if (K_pool->stride_n <= 0 || V_pool->stride_n <= 0 || K_pool->stride_b % K_pool->stride_n != 0 ||
+        V_pool->stride_b % V_pool->stride_n != 0 || K_pool->stride_b / K_pool->stride_n != V_pool->stride_b / V_pool->stride_n)
+        return HA_ERR_INVALID_ARG;
+    int shift = 0;
+    while ((1 << shift) < page_size) ++shift;
+    return sparse_decode_impl(shape, map_q, map_k, q, k_new, K_pool, V_pool, block_table, bt_stride_b, shift, k_codes,
+                              kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, q_codes, idx,
+                              idx_stride_b, idx_stride_h, count, out, lse, workspace, ws_bytes, stream);
 }
 
 int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,

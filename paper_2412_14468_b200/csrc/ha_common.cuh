@@ -192,7 +192,8 @@ cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapV
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
                               int k_uniform, int max_seq_len, int k_max, uint32_t *q_codes, int32_t *idx,
                               long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
-                              cudaStream_t st, Windows win = Windows{0, 0});
+                              cudaStream_t st, Windows win = Windows{0, 0}, const int32_t *block_table = nullptr,
+                              long long bt_sb = 0, int page_shift = 0);
 
 cudaError_t launch_append_kv(int B, int Hq, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
                              TensorView V, const int32_t *seq_lens, const uint16_t *q_src, uint16_t *q_dst,

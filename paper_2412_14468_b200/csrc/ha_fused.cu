@@ -54,6 +54,11 @@ struct FusedArgs {
     int32_t *count;
     uint16_t *out;
     float *lse;
+    // paged K/V (block_table != NULL): token t of sequence b lives in page block_table[b*bt_sb + (t >> page_shift)],
+    // slot t & (2^page_shift - 1); K.sb / V.sb are then the page strides and page_rows = K.sb / K.sn
+    const int32_t *block_table;
+    long long bt_sb;
+    int page_shift, page_rows;
 };
 
 __device__ __forceinline__ void st_dsmem_f32(float *local, uint32_t rank, float v) {
@@ -321,8 +326,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     const int blocks_total = (keep + kBlockTokens - 1) / kBlockTokens;
     const int bpc = (blocks_total + kFusedCS - 1) / kFusedCS;             // blocks per CTA
     const int blk_lo = min(blocks_total, (int)rank * bpc), blk_hi = min(blocks_total, blk_lo + bpc);
-    const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (long long)b * a.K.sb + (long long)kvh * a.K.sh);
-    const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (long long)b * a.V.sb + (long long)kvh * a.V.sh);
+    const bool paged = a.block_table != nullptr;   // rows are then addressed from the pool's base
+    const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (paged ? 0LL : (long long)b * a.K.sb) + (long long)kvh * a.K.sh);
+    const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (paged ? 0LL : (long long)b * a.V.sb) + (long long)kvh * a.V.sh);
+    const int32_t *pages = paged ? a.block_table + (long long)b * a.bt_sb : nullptr;
     const long long k_row = a.K.sn * 2, v_row = a.V.sn * 2;
     unsigned char *my_ring = ring + warp * (kFusedStages * kStageBytes);
     const uint32_t ring_u32 = smem_u32(my_ring);
@@ -341,7 +348,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         const int nblk = (blk_lo + warp < blk_hi) ? (blk_hi - blk_lo - warp + kFusedWarps - 1) / kFusedWarps : 0;
         auto token_of_block = [&](int i) -> int {
             const int p = (blk_lo + warp + i * kFusedWarps) * kBlockTokens + (lane & 15);
-            return (i < nblk && p < keep) ? __ldcg(list + p) : -1;
+            int t = (i < nblk && p < keep) ? __ldcg(list + p) : -1;
+            // paged: logical token -> row of the pool (page * rows per page stride + slot)
+            if (paged && t >= 0) t = __ldg(pages + (t >> a.page_shift)) * a.page_rows + (t & ((1 << a.page_shift) - 1));
+            return t;
         };
         auto issue = [&](int i, int stg) {
             const uint32_t valid = attn_issue_block(ring_u32 + stg * kStageBytes, Kb, Vb, k_row, v_row, token_of_block(i), lane);
@@ -473,9 +483,11 @@ cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapV
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
                               int k_uniform, int max_seq_len, int k_max, uint32_t *q_codes, int32_t *idx,
                               long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
-                              cudaStream_t st, Windows win) {
+                              cudaStream_t st, Windows win, const int32_t *block_table, long long bt_sb, int page_shift) {
     FusedArgs a{};
     a.win = win;
+    a.block_table = block_table; a.bt_sb = bt_sb; a.page_shift = page_shift;
+    a.page_rows = (block_table && K.sn > 0) ? (int)(K.sb / K.sn) : 0;
     a.map_q = map_q; a.map_k = map_k; a.q = q; a.k_new = k_new; a.K = K; a.V = V;
     a.k_codes = k_codes; a.kc_sb = kc_sb; a.kc_sh = kc_sh; a.seq_lens = seq_lens; a.k_per_seq = k_per_seq;
     a.k_uniform = k_uniform; a.max_seq_len = max_seq_len; a.k_max = k_max; a.Hq = Hq; a.Hkv = Hkv;

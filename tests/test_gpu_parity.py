@@ -523,6 +523,44 @@ def test_sparse_decode_step_with_always_kept_windows(cfg, n_sink, n_local):
     assert torch.equal(rh["idx"], r["idx"]) and torch.equal(rh["out"], r["out"])
 
 
+@pytest.mark.parametrize("cfg", [
+    wl.Config("paged-small", 57, 2, [1500, 333], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8),        # one fused launch
+    wl.Config("paged-batch", 58, 20, [700 + 53 * i for i in range(20)], None, 0.02, n_q_heads=8, n_kv_heads=2,
+              sparsity=8),                                                                                   # three kernels
+])
+@pytest.mark.parametrize("page_size", [1, 16])
+def test_sparse_decode_step_over_a_paged_cache(cfg, page_size):
+    """The whole step with K/V in pages scattered over a pool gives exactly what it gives on the contiguous
+    cache (same lists, same outputs), with and without always-kept windows."""
+    w = wl.make_workload(cfg, DEV)
+    B, Hq, Hkv, N = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, w["n_cap"]
+    pps = (N + page_size - 1) // page_size
+    g = torch.Generator(DEV).manual_seed(page_size)
+    perm = torch.randperm(B * pps + 7, device=DEV, generator=g)[:B * pps].to(torch.int32).reshape(B, pps)
+    pools = []
+    for X in (w["K"], w["V"]):
+        Xp = torch.zeros(B * pps + 7, Hkv, page_size, 128, dtype=X.dtype, device=DEV)
+        Xp[perm.reshape(-1).long()] = torch.nn.functional.pad(X, (0, 0, 0, pps * page_size - N)) \
+            .reshape(B, Hkv, pps, page_size, 128).permute(0, 2, 1, 3, 4).reshape(B * pps, Hkv, page_size, 128)
+        pools.append(Xp)
+    for n_sink, n_local in ((0, 0), (16, 48)):
+        ref = _run_step(w, n_sink=n_sink, n_local=n_local)            # contiguous cache (itself checked against the oracle)
+        k_max = w["k_max"] + n_sink + n_local
+        shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"], n_sink=n_sink, n_local=n_local)
+        ws = ha.alloc_workspace(shape, N, k_max)
+        kc = ref["kc"].clone()
+        qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+        idx = torch.zeros(B, Hkv, k_max, dtype=torch.int32, device=DEV)
+        cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=DEV)
+        out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=DEV)
+        ha.ha_sparse_decode_paged(shape, ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"]), w["q"], w["k_new"], pools[0], pools[1],
+                                  perm, page_size, kc, w["seq_lens"], w["k_per_seq"], 0, N, k_max, qc, idx, cnt, out, ws)
+        torch.cuda.synchronize()
+        assert ha.ha_read_device_status(ws) == 0
+        assert torch.equal(idx, ref["idx"]) and torch.equal(cnt, ref["cnt"]) and torch.equal(qc, ref["qc"])
+        assert torch.equal(out, ref["out"])
+
+
 def test_k_equals_n_sparse_step_equals_dense_kernel():
     cfg = wl.Config("k=n", 52, 2, [1500, 900], None, 0.0, n_q_heads=8, n_kv_heads=2, sparsity=1)
     w = wl.make_workload(cfg, DEV)
