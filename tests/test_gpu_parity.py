@@ -241,6 +241,27 @@ def test_score_topk_windows_with_heavy_ties_and_small_k_max():
         ha.ha_score_topk(shape, t(2, Hq), t(2, Hkv, n), t(2), None, 10, n, 200, t(2, Hkv, 200), t(2, Hkv), ws)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_score_topk_random_shapes_budgets_and_windows(seed):
+    """Seeded sweep: batch, heads, group size, ragged lengths, budgets (0 .. beyond n) and window sizes drawn at
+    random; few distinct signatures in some cases (long tie blocks).  Index sets, counts and histograms exact."""
+    rng = np.random.default_rng(9000 + seed)
+    B = int(rng.integers(1, 7))
+    Hkv = int(rng.choice([1, 2, 4]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    lens = [int(v) for v in rng.integers(0, int(rng.choice([40, 3000, 20000])), size=B)]
+    n_cap = (max(max(lens), 4) + 3) // 4 * 4
+    if seed % 3 == 0:
+        pool = rng.integers(0, 2 ** 32, size=5, dtype=np.uint64).astype(np.uint32)
+        kc = pool[rng.integers(0, 5, size=(B, Hkv, n_cap))]
+    else:
+        kc = rng.integers(0, 2 ** 32, size=(B, Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    qc = rng.integers(0, 2 ** 32, size=(B, Hkv * G), dtype=np.uint64).astype(np.uint32)
+    ks = [int(rng.integers(0, n + 10)) for n in lens]
+    n_sink, n_local = (0, 0) if seed % 2 == 0 else (int(rng.integers(0, 200)), int(rng.integers(0, 200)))
+    _check_score_topk(qc, kc, lens, ks, Hkv * G, Hkv, n_sink=n_sink, n_local=n_local)
+
+
 def test_score_topk_heavy_ties():
     rng = np.random.default_rng(11)
     Hq, Hkv, n = 8, 2, 9000
@@ -559,6 +580,30 @@ def test_sparse_decode_step_over_a_paged_cache(cfg, page_size):
         assert ha.ha_read_device_status(ws) == 0
         assert torch.equal(idx, ref["idx"]) and torch.equal(cnt, ref["cnt"]) and torch.equal(qc, ref["qc"])
         assert torch.equal(out, ref["out"])
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_sparse_decode_step_random_configs(seed):
+    """Seeded sweep over batch (both the fused launch and the three-kernel path), KV heads, group size, ragged
+    lengths, sparsity and window sizes; everything the step returns is checked against the oracle."""
+    rng = np.random.default_rng(7000 + seed)
+    B = int(rng.integers(1, 13))
+    Hkv = int(rng.choice([1, 2]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    lens = [int(v) for v in rng.integers(1, 3000, size=B)]
+    cfg = wl.Config(f"rand{seed}", 70 + seed, B, lens, None, 0.02, n_q_heads=Hkv * G, n_kv_heads=Hkv,
+                    sparsity=int(rng.choice([2, 8, 16])))
+    n_sink, n_local = (0, 0) if seed % 2 == 0 else (int(rng.integers(0, 100)), int(rng.integers(0, 100)))
+    w = wl.make_workload(cfg, DEV)
+    r = _run_step(w, n_sink=n_sink, n_local=n_local)
+    Kc = oracle_key_codes(w["K"], w["map_k"], w["lens"])
+    ref = oracle.decode_step(u16(w["q"]), u16(w["k_new"]), u16(w["K"]), u16(w["V"]), Kc.copy(),
+                             wl.mapping_numpy(w["map_q"]), wl.mapping_numpy(w["map_k"]), w["lens"], w["ks"],
+                             sm_scale=w["sm_scale"], n_threads=4, n_sink=n_sink, n_local=n_local)
+    assert np.array_equal(codes_np(r["qc"]), ref["qcodes"])
+    assert np.array_equal(r["cnt"].cpu().numpy(), ref["count"])
+    assert np.array_equal(r["idx"].cpu().numpy(), ref["idx"])
+    assert_out_close(u16(r["out"]), ref["out"])
 
 
 def test_k_equals_n_sparse_step_equals_dense_kernel():
