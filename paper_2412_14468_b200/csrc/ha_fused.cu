@@ -75,12 +75,9 @@ __device__ __forceinline__ void st_dsmem_f32(float *local, uint32_t rank, float 
 template <int NV>
 __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_stride, const MapView &map, int net,
                                              uint16_t *sw1, uint16_t *sw2, uint16_t *sw3, uint32_t bar0, float *actA,
-                                             float *actB, uint32_t *codes_out) {
+                                             float *actB, uint32_t *codes_out, float bias1, float bias2, float bias3) {
     const int tid = threadIdx.x, o = tid & 127;
     const bool active = tid < 128;
-    const float bias1 = map.b1 ? __ldg(map.b1 + net * kHid + o) : 0.0f;
-    const float bias2 = map.b2 ? __ldg(map.b2 + net * kHid + o) : 0.0f;
-    const float bias3 = map.b3 ? __ldg(map.b3 + net * kBits + (tid & (kBits - 1))) : 0.0f;
     if (active) {
 #pragma unroll
         for (int v = 0; v < NV; ++v) actA[v * kD + o] = bf16_bits_to_float(__ldg(x0 + (long long)v * x_stride + o));
@@ -191,6 +188,21 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         mbar_expect_tx(bar0 + 16, kHid * kBits * 2);
         bulk_g2s((uint32_t)__cvta_generic_to_shared(sw3), map.w3 + (size_t)kvh * kHid * kBits, kHid * kBits * 2, bar0 + 16);
     }
+    // biases are weights: they are fetched before the wait, like the matrices.  The vector to encode may
+    // still be written by the kernel in front of this one, so it is only pulled into L2 here (a hint: the
+    // writer's store updates the same L2 line) and read after the wait.
+    float bias1 = 0.0f, bias2 = 0.0f, bias3 = 0.0f;
+    if (encodes) {
+        const int o = tid & 127;
+        if (map.b1) bias1 = __ldg(map.b1 + kvh * kHid + o);
+        if (map.b2) bias2 = __ldg(map.b2 + kvh * kHid + o);
+        if (map.b3) bias3 = __ldg(map.b3 + kvh * kBits + (tid & (kBits - 1)));
+        if (tid < 2) {
+            const uint16_t *xv = enc_q ? a.q + (head0 + kQPer * (int)rank) * kD : a.k_new + ((long long)b * Hkv + kvh) * kD;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(xv) + 128 * tid));
+            if (enc_q && kQPer > 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(xv) + 256 + 128 * tid));
+        }
+    }
     for (int i = tid; i < kBins * 32 / 4; i += kFusedThreads)
         reinterpret_cast<uint4 *>(&c_hist[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
     if (tid < kBins + 3) s_hist[tid] = 0;
@@ -200,11 +212,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     // ---------------- P1: ENCODE in CTA 0 (queries) and CTA 1 (appended key)
     if (enc_q) {
         fused_encode<kQPer>(a.q + (head0 + kQPer * (int)rank) * kD, kD, a.map_q, kvh, sw1, sw2, sw3, bar0, actA, actB,
-                            s_codes);
+                            s_codes, bias1, bias2, bias3);
         if (tid < kQPer) a.q_codes[head0 + kQPer * (int)rank + tid] = s_codes[tid];
     } else if (enc_k) {
         fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, a.map_k, kvh, sw1, sw2, sw3, bar0, actA, actB,
-                        s_codes);
+                        s_codes, bias1, bias2, bias3);
         if (tid == 0) row[n - 1] = s_codes[0];
     }
     cluster_sync_all();   // #1: the signatures are in the encoding CTAs' shared memory
