@@ -82,17 +82,20 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
 #pragma unroll
         for (int v = 0; v < NV; ++v) actA[v * kD + o] = bf16_bits_to_float(__ldg(x0 + (long long)v * x_stride + o));
     }
-    __syncthreads();
-    auto weights_ready = [&](int which, uint16_t *dst, const uint16_t *src, int n_elems) {
+    // Each matrix was requested at kernel entry (a whole step ahead in steady state).  The wait for a
+    // matrix is folded into the barrier that publishes the layer's input, so a layer costs one barrier.
+    // If a copy never reports completion (never seen) the CTA fetches the matrix with ordinary loads
+    // instead; the decision is taken by the whole CTA together.
+    auto publish_and_await = [&](int which, uint16_t *dst, const uint16_t *src, int n_elems) {
         const bool ok = mbar_wait_bounded(bar0 + 8 * which);
-        if (__syncthreads_or(!ok)) {   // never seen: fetch the matrix with ordinary loads instead
+        if (__syncthreads_or(!ok)) {
             for (int c = tid; c < n_elems / 8; c += kFusedThreads)
                 reinterpret_cast<uint4 *>(dst)[c] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
             __syncthreads();
         }
     };
     float z[NV];
-    weights_ready(0, sw1, map.w1 + (size_t)net * kD * kHid, kD * kHid);
+    publish_and_await(0, sw1, map.w1 + (size_t)net * kD * kHid, kD * kHid);
     if (active) {
 #pragma unroll
         for (int v = 0; v < NV; ++v) z[v] = bias1;
@@ -100,8 +103,7 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
 #pragma unroll
         for (int v = 0; v < NV; ++v) actB[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
     }
-    __syncthreads();
-    weights_ready(1, sw2, map.w2 + (size_t)net * kHid * kHid, kHid * kHid);
+    publish_and_await(1, sw2, map.w2 + (size_t)net * kHid * kHid, kHid * kHid);
     if (active) {
 #pragma unroll
         for (int v = 0; v < NV; ++v) z[v] = bias2;
@@ -109,8 +111,7 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
 #pragma unroll
         for (int v = 0; v < NV; ++v) actA[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
     }
-    __syncthreads();
-    weights_ready(2, sw3, map.w3 + (size_t)net * kHid * kBits, kHid * kBits);
+    publish_and_await(2, sw3, map.w3 + (size_t)net * kHid * kBits, kHid * kBits);
     {
         const int v = tid >> 5, lane = tid & 31;   // warp v encodes vector v, one output bit per lane
         if (v < NV) {
