@@ -250,7 +250,7 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
     cudaStream_t st = (cudaStream_t)stream;
     const int B = shape->batch, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
 
-    if (fused_step_eligible(B, Hkv, max_seq_len)) {
+    if (fused_step_eligible(B, Hq, Hkv, max_seq_len, k_max)) {
         // small batch: the whole step is one cluster kernel
         HA_CUDA(launch_fused_step(B, Hq, Hkv, shape->sm_scale, view(map_q), k_new ? view(map_k) : MapView{}, q, k_new,
                                   view(K), view(V), k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,

@@ -186,7 +186,7 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              const int32_t *block_table = nullptr, long long bt_sb = 0, int page_shift = 0);
 
 // The whole layer-step in one launch (one 8-CTA cluster per unit); only for small batches.
-bool fused_step_eligible(int B, int Hkv, int max_seq_len);
+bool fused_step_eligible(int B, int Hq, int Hkv, int max_seq_len, int k_max);
 cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapView &map_q, const MapView &map_k,
                               const uint16_t *q, const uint16_t *k_new, TensorView K, TensorView V, uint32_t *k_codes,
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,

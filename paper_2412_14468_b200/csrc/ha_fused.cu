@@ -1,14 +1,14 @@
-// The whole layer-step in ONE launch, for small batches (at most 18 (sequence, KV head) units and
-// sequences of up to 32768 tokens): ENCODE -> SCORE -> TOPK -> GATHER-ATT (Section 4 recipe,
-// Section 4.1 "Implementation") with one thread-block cluster of 8 CTAs per unit, so that a batch-1
-// decode step keeps 64 SMs busy without a single kernel boundary or global-memory hand-off on its
-// critical path:
+// The whole layer-step in ONE launch, for small batches (as many (sequence, KV head) units as clusters
+// are resident at once: 33 when the budget is at most 1024 rows, 15 beyond, on a 148-SM device) and
+// sequences of up to 32768 tokens: ENCODE -> SCORE -> TOPK -> GATHER-ATT (Section 4 recipe,
+// Section 4.1 "Implementation") with one thread-block cluster of 8 CTAs per unit, so that a small-batch
+// decode step has no kernel boundary or global-memory hand-off on its critical path:
 //
-//   P0  every CTA requests its slice of the signature cache; the encoding CTAs of the cluster request
-//       the query-side / key-side mapping weights with bulk asynchronous copies (TMA, mbarriers);
-//       all of it before the programmatic-launch wait, i.e. behind the preceding kernel.
-//   P1  CTA r < ceil(G/2) encodes query vectors 2r, 2r+1, the next CTA the appended key (fp32 fma
-//       chains, Eq. 2, one chain per thread); cluster barrier; everybody reads the signatures
+//   P0  every CTA requests its slice of the signature cache; the encoding CTAs of the cluster fetch the
+//       query-side / key-side mapping weights and store them transposed in shared memory; all of it
+//       before the programmatic-launch wait, i.e. behind the preceding kernel.
+//   P1  CTA r < G (r < G/2 for G = 8) encodes one (two) query vectors, the next CTA the appended key
+//       (fp32 fma chains, Eq. 2, one chain per thread); cluster barrier; everybody reads the signatures
 //       through distributed shared memory.
 //   P2  scores as bytes in registers, per-CTA histogram, cluster barrier, histogram exchange through
 //       distributed shared memory, threshold, compaction of the CTA's slice into the index list;
@@ -30,13 +30,17 @@ constexpr int kFusedCS = 8;
 constexpr int kFusedWarps = 8;
 constexpr int kFusedThreads = kFusedWarps * 32;
 constexpr int kFusedL = 4;                                   // uint4 of signatures per thread (n <= 32768)
-constexpr int kFusedStages = 2;                              // row blocks in flight per warp
-constexpr int kFusedRingBytes = kFusedWarps * kFusedStages * kStageBytes;
+constexpr int kFusedMaxStages = 2;                           // row blocks in flight per warp (template parameter S)
 constexpr int kFusedWeightBytes = (kD * kHid + kHid * kHid + kHid * kBits) * 2;
-constexpr int kFusedUnionBytes = (kFusedRingBytes > kFusedWeightBytes) ? kFusedRingBytes : kFusedWeightBytes;
-constexpr int kFusedActBytes = 2 * kMaxGroup * kD * 4;       // two activation buffers of up to 8 vectors
-constexpr int kFusedPartBytes = kFusedCS * kMaxGroup * (kD + 2) * 4;   // the eight CTA states, in CTA 0
-constexpr int kFusedSmemBytes = kFusedUnionBytes + kFusedActBytes + kFusedPartBytes;
+constexpr int kFusedActBytes = 2 * 2 * kD * 4;               // two activation buffers of up to 2 vectors
+// Dynamic shared memory of a CTA: [weights | S row stages per warp] union, activations, the eight CTA states
+// of the G heads (used in CTA 0).  With S = 1 two CTAs fit one SM (and the kernel is compiled for 128
+// registers): two consecutive steps are then resident together, each cluster of the later one already
+// parked at its launch wait, whereas only 15 clusters of eight one-CTA SMs exist on the device.
+__host__ __device__ constexpr int fused_ring_bytes(int S) { return kFusedWarps * S * kStageBytes; }
+__host__ __device__ constexpr int fused_union_bytes(int S) { return fused_ring_bytes(S) > kFusedWeightBytes ? fused_ring_bytes(S) : kFusedWeightBytes; }
+__host__ __device__ constexpr int fused_part_bytes(int G) { return kFusedCS * G * (kD + 2) * 4; }
+__host__ __device__ constexpr int fused_smem_bytes(int G, int S) { return fused_union_bytes(S) + kFusedActBytes + fused_part_bytes(G); }
 
 struct FusedArgs {
     MapView map_q, map_k;
@@ -68,55 +72,43 @@ __device__ __forceinline__ void st_dsmem_f32(float *local, uint32_t rank, float 
 }
 
 // ENCODE of NV vectors that share one network by the first 128 threads of the CTA: thread o runs the
-// chains of output o for every vector.  The layers are bound by shared-memory bandwidth, so a second
-// warp per scheduler would only compete for it without shortening any chain.  Weights arrive in
-// shared memory through three mbarriers armed by the caller.  Signature v is returned in codes_out[v]
-// (shared memory).
+// chains of output o for every vector.  A second warp per scheduler would not shorten any chain.  The
+// caller has put the three matrices into shared memory, transposed (TransposedFetch), before the
+// call; the barrier that publishes the input vectors also publishes them.  Signature v is returned in
+// codes_out[v] (shared memory).
 template <int NV>
-__device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_stride, const MapView &map, int net,
-                                             uint16_t *sw1, uint16_t *sw2, uint16_t *sw3, uint32_t bar0, float *actA,
-                                             float *actB, uint32_t *codes_out, float bias1, float bias2, float bias3) {
+__device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_stride, const uint16_t *sw1,
+                                             const uint16_t *sw2, const uint16_t *sw3, float *actA, float *actB,
+                                             uint32_t *codes_out, float bias1, float bias2, float bias3) {
     const int tid = threadIdx.x, o = tid & 127;
     const bool active = tid < 128;
     if (active) {
 #pragma unroll
         for (int v = 0; v < NV; ++v) actA[v * kD + o] = bf16_bits_to_float(__ldg(x0 + (long long)v * x_stride + o));
     }
-    // Each matrix was requested at kernel entry (a whole step ahead in steady state).  The wait for a
-    // matrix is folded into the barrier that publishes the layer's input, so a layer costs one barrier.
-    // If a copy never reports completion (never seen) the CTA fetches the matrix with ordinary loads
-    // instead; the decision is taken by the whole CTA together.
-    auto publish_and_await = [&](int which, uint16_t *dst, const uint16_t *src, int n_elems) {
-        const bool ok = mbar_wait_bounded(bar0 + 8 * which);
-        if (__syncthreads_or(!ok)) {
-            for (int c = tid; c < n_elems / 8; c += kFusedThreads)
-                reinterpret_cast<uint4 *>(dst)[c] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
-            __syncthreads();
-        }
-    };
+    __syncthreads();
     float z[NV];
-    publish_and_await(0, sw1, map.w1 + (size_t)net * kD * kHid, kD * kHid);
     if (active) {
 #pragma unroll
         for (int v = 0; v < NV; ++v) z[v] = bias1;
-        vec_layer<NV>(actA, sw1, kHid, o, z);
+        vec_layer_t<NV>(actA, sw1, o, z);
 #pragma unroll
         for (int v = 0; v < NV; ++v) actB[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
     }
-    publish_and_await(1, sw2, map.w2 + (size_t)net * kHid * kHid, kHid * kHid);
+    __syncthreads();
     if (active) {
 #pragma unroll
         for (int v = 0; v < NV; ++v) z[v] = bias2;
-        vec_layer<NV>(actB, sw2, kHid, o, z);
+        vec_layer_t<NV>(actB, sw2, o, z);
 #pragma unroll
         for (int v = 0; v < NV; ++v) actA[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
     }
-    publish_and_await(2, sw3, map.w3 + (size_t)net * kHid * kBits, kHid * kBits);
+    __syncthreads();
     {
         const int v = tid >> 5, lane = tid & 31;   // warp v encodes vector v, one output bit per lane
         if (v < NV) {
             float z3[1] = {bias3};
-            vec_layer<1>(actA + v * kD, sw3, kBits, lane, z3);
+            vec_layer_t<1>(actA + v * kD, sw3, lane, z3);
             const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
             if (lane == 0) codes_out[v] = code;
         }
@@ -124,8 +116,9 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
     __syncthreads();
 }
 
-template <int G>
-__global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const FusedArgs a) {
+template <int G, int S>
+__global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kernel(const FusedArgs a) {
+    constexpr int kFusedUnionBytes = fused_union_bytes(S);
     extern __shared__ __align__(128) unsigned char fsm[];
     // dynamic: [weights | row ring] union, activations, the cluster's states (used in CTA 0)
     uint16_t *sw1 = reinterpret_cast<uint16_t *>(fsm);
@@ -133,17 +126,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     uint16_t *sw3 = sw2 + kHid * kHid;
     unsigned char *ring = fsm;
     float *actA = reinterpret_cast<float *>(fsm + kFusedUnionBytes);
-    float *actB = actA + kMaxGroup * kD;
+    float *actB = actA + 2 * kD;
     float *part_ml = reinterpret_cast<float *>(fsm + kFusedUnionBytes + kFusedActBytes);   // [CS][G][2]
-    float *part_acc = part_ml + kFusedCS * kMaxGroup * 2;                                   // [CS][G][128]
-    __shared__ __align__(8) unsigned long long s_bar[3];
+    float *part_acc = part_ml + kFusedCS * G * 2;                                   // [CS][G][128]
     __shared__ uint32_t s_codes[kMaxGroup];   // signatures produced by this CTA (CTA 0: queries, CTA 1: new key)
     __shared__ __align__(16) uint32_t c_hist[kBins][32];   // one counter per (level, lane), shared by the warps
     __shared__ int s_hist[kBins + 3], s_tot[kBins], s_bef[kBins];
     __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
     __shared__ int s_wcnt[kFusedWarps];
     __shared__ float s_m[kFusedWarps][8], s_l[kFusedWarps][8];
-    __shared__ uint32_t s_mask[kFusedWarps][kFusedStages];
+    __shared__ uint32_t s_mask[kFusedWarps][kFusedMaxStages];
 
     const uint32_t rank = cluster_rank();
     const int kvh = blockIdx.y, b = blockIdx.z;
@@ -168,7 +160,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         const int base = wbase + p * 4;
         c[p] = (p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
     }
-    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&s_bar[0]);
     // ENCODE roles: CTA r < kQCtas encodes kQPer query vectors (one per CTA while the cluster has room),
     // CTA kQCtas encodes the appended key; the other CTAs only scan
     constexpr int kQPer = (G < kFusedCS) ? 1 : 2;
@@ -177,17 +168,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     const bool enc_q = (int)rank < kQCtas, enc_k = ((int)rank == kQCtas) && has_new_key;
     const bool encodes = enc_q || enc_k;
     const MapView &map = enc_q ? a.map_q : a.map_k;
-    if (encodes && tid == 0) {
-        mbar_init(bar0, 1);
-        mbar_init(bar0 + 8, 1);
-        mbar_init(bar0 + 16, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        mbar_expect_tx(bar0, kD * kHid * 2);
-        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw1), map.w1 + (size_t)kvh * kD * kHid, kD * kHid * 2, bar0);
-        mbar_expect_tx(bar0 + 8, kHid * kHid * 2);
-        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw2), map.w2 + (size_t)kvh * kHid * kHid, kHid * kHid * 2, bar0 + 8);
-        mbar_expect_tx(bar0 + 16, kHid * kBits * 2);
-        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw3), map.w3 + (size_t)kvh * kHid * kBits, kHid * kBits * 2, bar0 + 16);
+    if (encodes) {   // the mapping's matrices do not depend on earlier kernels: fetched, transposed, behind them
+        TransposedFetch<kFusedThreads, kHid> f1, f2;
+        TransposedFetch<kFusedThreads, kBits> f3;
+        f1.load(map.w1 + (size_t)kvh * kD * kHid, tid);   // all loads in flight before the first store
+        f2.load(map.w2 + (size_t)kvh * kHid * kHid, tid);
+        f3.load(map.w3 + (size_t)kvh * kHid * kBits, tid);
+        f1.store(sw1, tid);
+        f2.store(sw2, tid);
+        f3.store(sw3, tid);
     }
     // biases are weights: they are fetched before the wait, like the matrices.  The vector to encode may
     // still be written by the kernel in front of this one, so it is only pulled into L2 here (a hint: the
@@ -212,12 +201,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
 
     // ---------------- P1: ENCODE in CTA 0 (queries) and CTA 1 (appended key)
     if (enc_q) {
-        fused_encode<kQPer>(a.q + (head0 + kQPer * (int)rank) * kD, kD, a.map_q, kvh, sw1, sw2, sw3, bar0, actA, actB,
-                            s_codes, bias1, bias2, bias3);
+        fused_encode<kQPer>(a.q + (head0 + kQPer * (int)rank) * kD, kD, sw1, sw2, sw3, actA, actB, s_codes, bias1,
+                            bias2, bias3);
         if (tid < kQPer) a.q_codes[head0 + kQPer * (int)rank + tid] = s_codes[tid];
     } else if (enc_k) {
-        fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, a.map_k, kvh, sw1, sw2, sw3, bar0, actA, actB,
-                        s_codes, bias1, bias2, bias3);
+        fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, sw1, sw2, sw3, actA, actB, s_codes, bias1, bias2,
+                        bias3);
         if (tid == 0) row[n - 1] = s_codes[0];
     }
     cluster_sync_all();   // #1: the signatures are in the encoding CTAs' shared memory
@@ -344,7 +333,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (paged ? 0LL : (long long)b * a.V.sb) + (long long)kvh * a.V.sh);
     const int32_t *pages = paged ? a.block_table + (long long)b * a.bt_sb : nullptr;
     const long long k_row = a.K.sn * 2, v_row = a.V.sn * 2;
-    unsigned char *my_ring = ring + warp * (kFusedStages * kStageBytes);
+    unsigned char *my_ring = ring + warp * (S * kStageBytes);
     const uint32_t ring_u32 = smem_u32(my_ring);
     const int g = lane >> 2, cc = lane & 3;
 
@@ -373,14 +362,22 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
         if (nblk > 0) issue(0, 0);
         cp_async_commit();
         for (int i = 0; i < nblk; ++i) {
-            const int stg = i & 1;
-            if (i + 1 < nblk) issue(i + 1, stg ^ 1);
-            cp_async_commit();
-            cp_async_wait<1>();
+            const int stg = (S > 1) ? (i & 1) : 0;
+            if (S > 1) {   // the next block travels while this one is consumed
+                if (i + 1 < nblk) issue(i + 1, stg ^ 1);
+                cp_async_commit();
+                cp_async_wait<1>();
+            } else {
+                cp_async_wait<0>();
+            }
             __syncwarp();
             const uint32_t ks = ring_u32 + stg * kStageBytes;
             attn_consume_block(ks, ks + kTileBytes, s_mask[warp][stg], qa, a.scale_log2, lane, acc, m_run, l_run);
             __syncwarp();
+            if (S == 1) {   // one stage: the next block is requested once this one has been read
+                if (i + 1 < nblk) issue(i + 1, 0);
+                cp_async_commit();
+            }
         }
         cp_async_wait<0>();
     }
@@ -419,7 +416,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
                 for (int w = 0; w < kFusedWarps; ++w) {
                     const float f = exp2f(s_m[w][j] - M);
                     L = fmaf(s_l[w][j], f, L);
-                    A = fmaf(reinterpret_cast<const float *>(ring + w * (kFusedStages * kStageBytes))[j * kD + d], f, A);
+                    A = fmaf(reinterpret_cast<const float *>(ring + w * (S * kStageBytes))[j * kD + d], f, A);
                 }
             }
             st_dsmem_f32(part_acc + ((int)rank * G + j) * kD + d, 0, A);
@@ -456,23 +453,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     }
 }
 
-template <int G>
-static cudaError_t launch_fused_g(const FusedArgs &args, int B, cudaStream_t st) {
-    static bool done[64] = {};   // opt in to the large shared-memory carve-out once per device
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(fused_step_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kFusedSmemBytes);
-        if (e != cudaSuccess) return e;
-        done[dev] = true;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kFusedCS, args.Hkv, B);
+template <int G, int S>
+static void fused_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute (&attr)[2], int Hkv, int B, cudaStream_t st) {
+    cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = dim3(kFusedCS, Hkv, B);
     cfg.blockDim = dim3(kFusedThreads);
-    cfg.dynamicSmemBytes = kFusedSmemBytes;
+    cfg.dynamicSmemBytes = fused_smem_bytes(G, S);
     cfg.stream = st;
-    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = kFusedCS;
     attr[0].val.clusterDim.y = 1;
@@ -481,14 +468,70 @@ static cudaError_t launch_fused_g(const FusedArgs &args, int B, cudaStream_t st)
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_step_kernel<G>, args);
+}
+
+// Opt in to the shared-memory carve-out (once per device) and return how many clusters of this variant the
+// device holds at once (0 on error).
+template <int G, int S>
+static int fused_prepare() {
+    static int clusters[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (!clusters[dev]) {
+        if (cudaFuncSetAttribute(fused_step_kernel<G, S>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 fused_smem_bytes(G, S)) != cudaSuccess)
+            return 0;
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attr[2];
+        fused_config<G, S>(cfg, attr, 1, 64, nullptr);
+        cfg.numAttrs = 1;   // the cluster shape is all the occupancy query looks at
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, fused_step_kernel<G, S>, &cfg) != cudaSuccess || n <= 0) return 0;
+        clusters[dev] = n;
+    }
+    return clusters[dev];
+}
+
+template <int G, int S>
+static cudaError_t launch_fused_gs(const FusedArgs &args, int B, cudaStream_t st) {
+    if (fused_prepare<G, S>() <= 0) return cudaErrorInvalidConfiguration;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    fused_config<G, S>(cfg, attr, args.Hkv, B, st);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_step_kernel<G, S>, args);
     if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
 }
 
-bool fused_step_eligible(int B, int Hkv, int max_seq_len) {
-    return (long long)B * Hkv * kFusedCS <= 148 && max_seq_len <= kFusedCS * kFusedL * 1024;
+// One stage per warp (two CTAs per SM) when no warp meets more than one block of the list, i.e. up to
+// 8 CTAs x 8 warps x 16 selected rows; two stages (one CTA per SM) beyond.
+static bool fused_one_stage(int k_max) { return k_max <= kFusedCS * kFusedWarps * kBlockTokens; }
+
+template <int G>
+static int fused_cluster_limit(int k_max) {
+    return fused_one_stage(k_max) ? fused_prepare<G, 1>() : fused_prepare<G, 2>();
+}
+
+// The fused step is used while every cluster of the step is resident at once (a cluster that has to wait
+// for another one to finish would double the latency) and a CTA's eighth of a sequence fits its registers.
+bool fused_step_eligible(int B, int Hq, int Hkv, int max_seq_len, int k_max) {
+    if (max_seq_len > kFusedCS * kFusedL * 1024 || Hkv <= 0) return false;
+    int limit = 0;
+    switch (Hq / Hkv) {
+        case 1: limit = fused_cluster_limit<1>(k_max); break;
+        case 2: limit = fused_cluster_limit<2>(k_max); break;
+        case 4: limit = fused_cluster_limit<4>(k_max); break;
+        case 8: limit = fused_cluster_limit<8>(k_max); break;
+        default: return false;
+    }
+    return (long long)B * Hkv <= limit;
+}
+
+template <int G>
+static cudaError_t launch_fused_g(const FusedArgs &args, int B, cudaStream_t st) {
+    return fused_one_stage(args.k_max) ? launch_fused_gs<G, 1>(args, B, st) : launch_fused_gs<G, 2>(args, B, st);
 }
 
 cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapView &map_q, const MapView &map_k,

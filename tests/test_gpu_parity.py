@@ -606,6 +606,38 @@ def test_sparse_decode_step_random_configs(seed):
     assert_out_close(u16(r["out"]), ref["out"])
 
 
+@pytest.mark.parametrize("cfg,launches", [
+    # 32 units, small budgets: one fused launch of the one-stage variant (two CTAs per SM)
+    (wl.Config("fused-32-units", 80, 16, [1000 + 61 * i for i in range(16)], None, 0.02, n_q_heads=8, n_kv_heads=2,
+               sparsity=8), 1),
+    # 6 units, budgets above 1024 rows: one fused launch of the two-stage variant, several blocks per warp
+    (wl.Config("fused-large-k", 81, 3, [9000, 5000, 12001], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=4), 1),
+    # 20 units with budgets above 1024 rows: more clusters than the two-stage variant holds at once
+    (wl.Config("split-large-k", 82, 10, [6000 + 7 * i for i in range(10)], None, 0.02, n_q_heads=8, n_kv_heads=2,
+               sparsity=4), 3),
+    # 34 units: more clusters than the device holds at once
+    (wl.Config("split-34-units", 83, 17, [800 + 29 * i for i in range(17)], None, 0.02, n_q_heads=4, n_kv_heads=2,
+               sparsity=8), 3),
+])
+def test_sparse_decode_step_every_launch_variant(cfg, launches):
+    """The step picks the fused cluster kernel (one or two row stages per warp) or the three-kernel path from
+    the number of units and the budget; each choice gives the oracle's result."""
+    w = wl.make_workload(cfg, DEV)
+    _run_step(w)                                   # first call: attributes, occupancy query
+    before = ha.ha_kernel_launches()
+    r = _run_step(w)
+    # _run_step also builds the prompt's signature cache with one ha_encode launch
+    assert ha.ha_kernel_launches() - before == launches + 1
+    Kc = oracle_key_codes(w["K"], w["map_k"], w["lens"])
+    ref = oracle.decode_step(u16(w["q"]), u16(w["k_new"]), u16(w["K"]), u16(w["V"]), Kc.copy(),
+                             wl.mapping_numpy(w["map_q"]), wl.mapping_numpy(w["map_k"]), w["lens"], w["ks"],
+                             sm_scale=w["sm_scale"], n_threads=4)
+    assert np.array_equal(codes_np(r["qc"]), ref["qcodes"])
+    assert np.array_equal(r["cnt"].cpu().numpy(), ref["count"])
+    assert np.array_equal(r["idx"].cpu().numpy(), ref["idx"])
+    assert_out_close(u16(r["out"]), ref["out"])
+
+
 def test_k_equals_n_sparse_step_equals_dense_kernel():
     cfg = wl.Config("k=n", 52, 2, [1500, 900], None, 0.0, n_q_heads=8, n_kv_heads=2, sparsity=1)
     w = wl.make_workload(cfg, DEV)
@@ -618,7 +650,7 @@ def test_k_equals_n_sparse_step_equals_dense_kernel():
     assert r["cnt"].cpu().tolist() == [[1500, 1500], [900, 900]]
 
 
-@pytest.mark.parametrize("reps", [1, 3])     # 8 units: single fused kernel; 24 units: three-kernel path
+@pytest.mark.parametrize("reps", [1, 5])     # 8 units: single fused kernel; 40 units: three-kernel path
 def test_step_edge_cases_empty_sequence_budget_above_length_and_no_new_key(reps):
     # one launch covers: an empty sequence, a one-token sequence, k > n, k = 0; then the same without a new key
     cfg = wl.Config("edges", 53, 4 * reps, [0, 1, 37, 2500] * reps, 64, 0.0, n_q_heads=8, n_kv_heads=2)
