@@ -117,23 +117,28 @@ __global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, E
 #pragma unroll
         for (int v = 0; v < NV; ++v) actA[v * kD + o] = (z[v] > 0.0f) ? z[v] : 0.0f;
         __syncthreads();
-        // ---- layer 3: one warp per vector, one output bit per lane
+        // ---- layer 3: one output bit per lane; warp w takes vectors w, w + 4 (their chains interleaved)
         if (first) weights_ready(2, sw3, g3, kHid * kBits);
         first = false;
         {
+            constexpr int kWarps = kVecThreads / 32, VT3 = (NV + kWarps - 1) / kWarps;
             const int warp = tid >> 5, lane = tid & 31;
+            if (warp < nv) {   // warp-uniform; chains of slots >= nv read rows of the activation buffers and are dropped
+                float z3[VT3];
 #pragma unroll
-            for (int v0 = 0; v0 < NV; v0 += kVecThreads / 32) {
-                const int v = v0 + warp;
-                if (v < nv) {   // warp-uniform
-                    float z3[1] = {bias3};
-                    vec_layer<1>(actA + v * kD, sw3, kBits, lane, z3);
-                    const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
-                    const int t = t0 + v, b = t / hpk;
-                    int slot = 0;
-                    if (J.slot) slot = J.slot[b] - J.slot_minus_one;   // a negative slot skips the sequence
-                    if (lane == 0 && slot >= 0)
-                        J.codes[(long long)b * J.c_sb + (long long)(net * hpk + t % hpk) * J.c_sh + slot] = code;
+                for (int i = 0; i < VT3; ++i) z3[i] = bias3;
+                vec_layer<VT3>(actA + warp * kD, sw3, kBits, lane, z3, kWarps * kD);
+#pragma unroll
+                for (int i = 0; i < VT3; ++i) {
+                    const int v = warp + i * kWarps;
+                    const uint32_t code = __ballot_sync(0xffffffffu, z3[i] > 0.0f);
+                    if (v < nv) {
+                        const int t = t0 + v, b = t / hpk;
+                        int slot = 0;
+                        if (J.slot) slot = J.slot[b] - J.slot_minus_one;   // a negative slot skips the sequence
+                        if (lane == 0 && slot >= 0)
+                            J.codes[(long long)b * J.c_sb + (long long)(net * hpk + t % hpk) * J.c_sh + slot] = code;
+                    }
                 }
             }
         }
@@ -159,38 +164,45 @@ static cudaError_t launch_vec_t(const EncodeJob &a, const EncodeJob &b, cudaStre
 }
 
 // `a` and `b` arrive with n_cta = the number of (sequence, network) pairs (0 = no such job); the item
-// width and the CTAs per network are chosen here.
+// width and the CTAs per network are chosen here: the smallest number m of vectors per CTA for which
+// all CTAs are resident at once (two CTAs of 76 KB fit one SM; a second wave would double the latency),
+// each network getting CTAs in proportion to its vectors, and a CTA's m vectors cut into the fewest
+// items of at most 8 vectors, equal in width.
 cudaError_t launch_encode_vectors(const EncodeJob &a_in, const EncodeJob &b_in, cudaStream_t st) {
     if (a_in.n_cta + b_in.n_cta <= 0) return cudaSuccess;
     EncodeJob job[2] = {a_in, b_in};
     int nets[2], vec_per_net[2];
-    long long vectors = 0;
     for (int j = 0; j < 2; ++j) {
         EncodeJob &J = job[j];
         nets[j] = (J.n_cta > 0) ? J.n_heads / J.heads_per_kv : 0;
         J.batch = (J.n_cta > 0) ? J.n_cta / nets[j] : 0;
         vec_per_net[j] = J.batch * J.heads_per_kv;
-        vectors += (long long)nets[j] * vec_per_net[j];
     }
-    const long long room = 2LL * sm_count();   // two CTAs (76 KB of shared memory each) fit one SM
-    int nv = 1;
-    auto items = [&](int width) {
+    const long long room = 2LL * sm_count();
+    auto ctas = [&](int m) {
         long long n = 0;
-        for (int j = 0; j < 2; ++j) n += (long long)nets[j] * ((vec_per_net[j] + width - 1) / width);
+        for (int j = 0; j < 2; ++j) n += (long long)nets[j] * ((vec_per_net[j] + m - 1) / m);
         return n;
     };
-    while (nv < 8 && items(nv) > room) nv *= 2;
-    const long long rounds = (items(nv) + 2 * room - 1) / (2 * room);   // up to two waves of one-item CTAs
+    const int m_max = vec_per_net[0] > vec_per_net[1] ? vec_per_net[0] : vec_per_net[1];   // one CTA per network
+    int m = 1;
+    while (m < m_max && ctas(m) > room) ++m;   // more networks than CTA slots: several waves, nothing to balance
+    const int items_per_cta = (m + 7) / 8, nv = (m + items_per_cta - 1) / items_per_cta;
     for (int j = 0; j < 2; ++j) {
         EncodeJob &J = job[j];
-        const long long it = (vec_per_net[j] + nv - 1) / nv;
-        J.cta_per_net = (int)((it + rounds - 1) / rounds);
+        J.cta_per_net = (vec_per_net[j] + m - 1) / m;
         J.n_cta = nets[j] * J.cta_per_net;
     }
-    if (nv == 1) return launch_vec_t<1>(job[0], job[1], st);
-    if (nv == 2) return launch_vec_t<2>(job[0], job[1], st);
-    if (nv == 4) return launch_vec_t<4>(job[0], job[1], st);
-    return launch_vec_t<8>(job[0], job[1], st);
+    switch (nv) {
+        case 1: return launch_vec_t<1>(job[0], job[1], st);
+        case 2: return launch_vec_t<2>(job[0], job[1], st);
+        case 3: return launch_vec_t<3>(job[0], job[1], st);
+        case 4: return launch_vec_t<4>(job[0], job[1], st);
+        case 5: return launch_vec_t<5>(job[0], job[1], st);
+        case 6: return launch_vec_t<6>(job[0], job[1], st);
+        case 7: return launch_vec_t<7>(job[0], job[1], st);
+        default: return launch_vec_t<8>(job[0], job[1], st);
+    }
 }
 
 // ------------------------------------------------------------------ token-tiled bulk kernel

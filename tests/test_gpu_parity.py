@@ -63,10 +63,11 @@ def test_encode_query_side_group_sharing_and_append_slot():
     assert np.all(got == 0x55)
 
 
-@pytest.mark.parametrize("B,Hq,Hkv", [(1, 8, 2), (19, 8, 2), (50, 8, 2), (101, 8, 2), (300, 32, 8), (37, 16, 2), (333, 3, 3)])
+@pytest.mark.parametrize("B,Hq,Hkv", [(1, 8, 2), (19, 8, 2), (50, 8, 2), (101, 8, 2), (300, 32, 8), (37, 16, 2), (333, 3, 3),
+                                      (1300, 1, 1), (1600, 1, 1), (2200, 1, 1), (2500, 1, 1)])   # item widths 5, 6, 8, 2 x 5
 def test_encode_single_token_batches_cover_every_item_width(B, Hq, Hkv):
-    """One vector per head and sequence: small batches run one vector per CTA, larger ones items of 2, 4 or
-    8 vectors (ragged last item), and the largest several items per CTA; all bit-exact."""
+    """One vector per head and sequence: small batches run one vector per CTA, larger ones items of 2 to 8
+    vectors (ragged last item), and the largest several items per CTA; all bit-exact."""
     mp = _mapping(Hkv, 1000 + B)
     g = torch.Generator(DEV).manual_seed(B)
     q = torch.randn(B, Hq, 128, device=DEV, generator=g).to(torch.bfloat16)
