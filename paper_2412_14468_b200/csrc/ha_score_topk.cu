@@ -40,6 +40,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
                                                                  int32_t *__restrict__ ws_hist, Windows win) {
     __shared__ __align__(16) uint32_t c_hist[kBins][32];
     __shared__ int s_hist[kBins + 3];
+    __shared__ uint32_t s_qc[G];
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int n = min(seq_lens[b], max_seq_len);
     const int start = chunk * chunk_tokens;
@@ -65,10 +66,13 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
     if (tid < kBins + 3) s_hist[tid] = 0;
     pdl_launch_dependents();
     pdl_wait();
+    // The query signatures were written by the kernel in front of this one and must come from L2; the many
+    // CTAs of a long sequence all want the same few words, so one thread per word fetches them for the CTA.
+    if (tid < G) s_qc[tid] = __ldcg(q_codes + (long long)b * Hq + g * G + tid);
+    __syncthreads();
     uint32_t qc[G];
 #pragma unroll
-    for (int j = 0; j < G; ++j) qc[j] = __ldcg(q_codes + (long long)b * Hq + g * G + j);
-    __syncthreads();
+    for (int j = 0; j < G; ++j) qc[j] = s_qc[j];
 
     // the counter of score s sits (32 - s) rows below the lane's counter of level 32
     const uint32_t top = (uint32_t)__cvta_generic_to_shared(&c_hist[kBins - 1][lane]);
@@ -129,6 +133,7 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
                                                              long long idx_sh, int32_t *__restrict__ count,
                                                              int32_t *__restrict__ hist_out, Windows win) {
     __shared__ int s_tot[kBins + 3], s_bef[kBins + 3];
+    __shared__ int s_wtot[kScanThreads / 32][kBins + 3], s_wbef[kScanThreads / 32][kBins + 3];
     __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
     __shared__ int warp_tot[kScanThreads / 32];
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
@@ -151,27 +156,39 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
     uint4 sv_next = make_uint4(0u, 0u, 0u, 0u);
     if (chunk < n_chunks && start + tid * 16 < end) sv_next = __ldcg(srow + ((start + tid * 16) >> 4));
 
-    // totals per score level, and the part contributed by the chunks before this one: every thread
-    // fetches its share of the n_chunks x 33 counters at once and adds them up in shared memory
-    __syncthreads();
+    // totals per score level, and the part contributed by the chunks before this one.  Lane l of warp w sums
+    // level l over the chunks w, w + 8, ... (coalesced rows of the counter table, every load issued before
+    // the first use), lane 0 also level 32; the eight warps' sums meet in shared memory.  No atomics: a
+    // hundred adds queued on one shared-memory word would stall the loads that follow them.
     {
         const int32_t *hb = ws_hist + ((long long)b * Hkv + g) * kMaxChunks * kBins;
-        const int total = n_chunks * kBins;
-        int v[(kMaxChunks * kBins + kScanThreads - 1) / kScanThreads];
+        constexpr int kWarps = kScanThreads / 32, kPer = kMaxChunks / kWarps;
+        int v[kPer], v32[kPer];
 #pragma unroll
-        for (int i = 0; i < (kMaxChunks * kBins + kScanThreads - 1) / kScanThreads; ++i) {
-            const int e = tid + i * kScanThreads;
-            v[i] = (e < total) ? __ldcg(hb + e) : 0;
+        for (int i = 0; i < kPer; ++i) {
+            const int cc = warp + i * kWarps;
+            v[i] = (cc < n_chunks) ? __ldcg(hb + cc * kBins + lane) : 0;
+            v32[i] = (cc < n_chunks && lane == 0) ? __ldcg(hb + cc * kBins + 32) : 0;
         }
+        int tot = 0, bef = 0, tot32 = 0, bef32 = 0;
 #pragma unroll
-        for (int i = 0; i < (kMaxChunks * kBins + kScanThreads - 1) / kScanThreads; ++i) {
-            const int e = tid + i * kScanThreads;
-            if (e < total && v[i] != 0) {
-                const int cc = e / kBins, bin = e - cc * kBins;
-                atomicAdd(&s_tot[bin], v[i]);
-                if (cc < chunk) atomicAdd(&s_bef[bin], v[i]);
-            }
+        for (int i = 0; i < kPer; ++i) {
+            const int cc = warp + i * kWarps;
+            tot += v[i];
+            tot32 += v32[i];
+            if (cc < chunk) { bef += v[i]; bef32 += v32[i]; }
         }
+        s_wtot[warp][lane] = tot;
+        s_wbef[warp][lane] = bef;
+        if (lane == 0) { s_wtot[warp][32] = tot32; s_wbef[warp][32] = bef32; }
+    }
+    __syncthreads();
+    if (tid < kBins) {
+        int tot = 0, bef = 0;
+#pragma unroll
+        for (int w = 0; w < kScanThreads / 32; ++w) { tot += s_wtot[w][tid]; bef += s_wbef[w][tid]; }
+        s_tot[tid] = tot;
+        s_bef[tid] = bef;
     }
     __syncthreads();
     if (warp == 0) {
