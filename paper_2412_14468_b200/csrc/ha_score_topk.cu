@@ -132,9 +132,7 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
                                                              int32_t *__restrict__ idx, long long idx_sb,
                                                              long long idx_sh, int32_t *__restrict__ count,
                                                              int32_t *__restrict__ hist_out, Windows win) {
-    __shared__ int s_tot[kBins + 3], s_bef[kBins + 3];
     __shared__ int s_wtot[kScanThreads / 32][kBins + 3], s_wbef[kScanThreads / 32][kBins + 3];
-    __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
     __shared__ int warp_tot[kScanThreads / 32];
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -146,7 +144,6 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
     const int keep = n_forced + keep_rest;
     const int n_chunks = (n + chunk_tokens - 1) / chunk_tokens;
     if (chunk > 0 && chunk >= n_chunks) return;
-    if (tid < kBins + 3) { s_tot[tid] = 0; s_bef[tid] = 0; }
     pdl_launch_dependents();
     pdl_wait();   // histograms and score bytes come from the preceding kernel
 
@@ -183,28 +180,25 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
         if (lane == 0) { s_wtot[warp][32] = tot32; s_wbef[warp][32] = bef32; }
     }
     __syncthreads();
-    if (tid < kBins) {
-        int tot = 0, bef = 0;
+    // Every warp folds the eight partial sums and derives the threshold for itself (lane l owns level l,
+    // level 32 is read by every lane): no broadcast, no further barrier.  Suffix sums over the levels give
+    // #{S >= t}; T = largest level with #{S >= T} >= keep; r = keep - #{S > T}.
+    int T, r, gt_before, eq_before;
+    {
+        int tot = 0, bef = 0, tot32 = 0, bef32 = 0;
 #pragma unroll
-        for (int w = 0; w < kScanThreads / 32; ++w) { tot += s_wtot[w][tid]; bef += s_wbef[w][tid]; }
-        s_tot[tid] = tot;
-        s_bef[tid] = bef;
-    }
-    __syncthreads();
-    if (warp == 0) {
-        // lane l owns level l (0..31); level 32 is read by every lane.  Suffix sums over the levels
-        // give #{S >= t}; T = largest level with #{S >= T} >= keep; r = keep - #{S > T}.
-        const int tot = s_tot[lane], bef = s_bef[lane], tot32 = s_tot[32], bef32 = s_bef[32];
-        int T, r, gt_before, eq_before;
+        for (int w = 0; w < kScanThreads / 32; ++w) {
+            tot += s_wtot[w][lane];
+            bef += s_wbef[w][lane];
+            tot32 += s_wtot[w][32];
+            bef32 += s_wbef[w][32];
+        }
         find_threshold(tot, bef, tot32, bef32, keep_rest, lane, T, r, gt_before, eq_before);
-        if (lane == 0) { sh_T = T; sh_r = r; sh_gt_before = gt_before; sh_eq_before = eq_before; }
-        if (chunk == 0 && hist_out) {
+        if (warp == 0 && chunk == 0 && hist_out) {
             hist_out[((long long)b * Hkv + g) * kBins + lane] = tot;
             if (lane == 0) hist_out[((long long)b * Hkv + g) * kBins + 32] = tot32;
         }
     }
-    __syncthreads();
-    const int T = sh_T, r = sh_r;
     int32_t *out = idx + (long long)b * idx_sb + (long long)g * idx_sh;
     if (chunk == 0) {
         if (tid == 0) count[b * Hkv + g] = keep;
@@ -217,7 +211,7 @@ __global__ void __launch_bounds__(kScanThreads) select_kernel(const int32_t *__r
     const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
     const uint32_t c_gt = 0x7f7f7f7fu - T4, c_ge = 0x80808080u - T4;
     // tokens before this pass with S > T (always-kept tokens count as such) / S == T
-    int run_gt = sh_gt_before + forced_before(wbd, start), run_eq = sh_eq_before;
+    int run_gt = gt_before + forced_before(wbd, start), run_eq = eq_before;
     for (int pass = start; pass < end; pass += kPassTokens) {
         const int base = pass + tid * 16;
         const uint4 sv = sv_next;
