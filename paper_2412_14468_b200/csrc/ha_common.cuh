@@ -59,16 +59,21 @@ inline WorkspaceLayout make_layout(int B, int Hq, int Hkv, int max_seq_len) {
     return L;
 }
 
-// Tokens of the code cache scanned by one CTA of the long-sequence path: a power of two >= 4096
-// (one pass of 256 threads x 16 tokens) chosen so that the grid has about four CTAs per SM when
-// there is that much work, and so that a sequence of max_seq_len tokens needs at most kMaxChunks
-// chunks.
-inline int chunk_tokens_for(int n_units, int max_seq_len) {
-    const long long total = (long long)(n_units > 0 ? n_units : 1) * (max_seq_len > 0 ? max_seq_len : 1);
-    long long c = 4096;
-    while (c < 32768 && total / c > 148 * 4) c *= 2;
-    while ((max_seq_len + c - 1) / c > kMaxChunks) c *= 2;
-    return (int)c;
+// Tokens of the code cache scanned by one CTA of the long-sequence path: the sequence is cut into equal
+// chunks (a multiple of 16 tokens, at least one pass of 256 threads x 16 tokens) so that the grid has
+// about three and a half CTAs per SM when there is that much work (four stay resident of either kernel;
+// filling every slot made the whole step slower, because the CTAs of the kernel behind could not become
+// resident early), and so that a sequence of max_seq_len tokens needs at most kMaxChunks chunks.
+inline int chunk_tokens_for(int n_units, int max_seq_len, int n_sm) {
+    const long long units = n_units > 0 ? n_units : 1, n = max_seq_len > 0 ? max_seq_len : 1;
+    long long per_unit = 7LL * (n_sm > 0 ? n_sm : 148) / 2 / units;
+    if (per_unit < 1) per_unit = 1;
+    if (per_unit > kMaxChunks) per_unit = kMaxChunks;
+    long long c = (n + per_unit - 1) / per_unit;
+    if (c < 4096) c = 4096;
+    const long long c_min = (n + kMaxChunks - 1) / kMaxChunks;
+    if (c < c_min) c = c_min;
+    return (int)((c + 15) / 16 * 16);
 }
 
 // ---- programmatic dependent launch: a kernel launched with launch_pdl may start while its

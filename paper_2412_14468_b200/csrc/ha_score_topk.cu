@@ -528,7 +528,7 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
         HA_CL(2);
 #undef HA_CL
     }
-    const int chunk_tokens = chunk_tokens_for(B * Hkv, max_seq_len);
+    const int chunk_tokens = chunk_tokens_for(B * Hkv, max_seq_len, sm_count());
     const int n_chunks = max(1, (max_seq_len + chunk_tokens - 1) / chunk_tokens);
     const long long score_row = (long long)score_row_bytes(max_seq_len);
     dim3 grid(n_chunks, Hkv, B);
