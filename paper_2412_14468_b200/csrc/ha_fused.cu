@@ -65,6 +65,11 @@ struct FusedArgs {
     int page_shift, page_rows;
 };
 
+__device__ __forceinline__ void st_dsmem_u32(uint32_t *local, uint32_t rank, uint32_t v) {
+    uint32_t a = (uint32_t)__cvta_generic_to_shared(local), ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(ra), "r"(v) : "memory");
+}
 __device__ __forceinline__ void st_dsmem_f32(float *local, uint32_t rank, float v) {
     uint32_t a = (uint32_t)__cvta_generic_to_shared(local), ra;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
@@ -74,12 +79,13 @@ __device__ __forceinline__ void st_dsmem_f32(float *local, uint32_t rank, float 
 // ENCODE of NV vectors that share one network by the first 128 threads of the CTA: thread o runs the
 // chains of output o for every vector.  A second warp per scheduler would not shorten any chain.  The
 // caller has put the three matrices into shared memory, transposed (TransposedFetch), before the
-// call; the barrier that publishes the input vectors also publishes them.  Signature v is returned in
-// codes_out[v] (shared memory).
+// call; the barrier that publishes the input vectors also publishes them.  Signature v is written to
+// word v of `dst` in the shared memory of EVERY CTA of the cluster (lanes 0..7 of the warp that holds it
+// store to CTAs 0..7; the cluster barrier that follows makes the stores visible) and to global_dst[v].
 template <int NV>
 __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_stride, const uint16_t *sw1,
                                              const uint16_t *sw2, const uint16_t *sw3, float *actA, float *actB,
-                                             uint32_t *codes_out, float bias1, float bias2, float bias3) {
+                                             uint32_t *dst, uint32_t *global_dst, float bias1, float bias2, float bias3) {
     const int tid = threadIdx.x, o = tid & 127;
     const bool active = tid < 128;
     if (active) {
@@ -110,10 +116,10 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
             float z3[1] = {bias3};
             vec_layer_t<1>(actA + v * kD, sw3, lane, z3);
             const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
-            if (lane == 0) codes_out[v] = code;
+            if (lane < kFusedCS) st_dsmem_u32(dst + v, (uint32_t)lane, code);
+            if (lane == kFusedCS) global_dst[v] = code;
         }
     }
-    __syncthreads();
 }
 
 template <int G, int S>
@@ -129,14 +135,15 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     float *actB = actA + 2 * kD;
     float *part_ml = reinterpret_cast<float *>(fsm + kFusedUnionBytes + kFusedActBytes);   // [CS][G][2]
     float *part_acc = part_ml + kFusedCS * G * 2;                                   // [CS][G][128]
-    __shared__ uint32_t s_codes[kMaxGroup];   // signatures produced by this CTA (CTA 0: queries, CTA 1: new key)
+    __shared__ uint32_t s_codes[kMaxGroup + 1];   // the G query signatures and the appended key's, pushed by the encoding CTAs
+    __shared__ uint32_t s_hist[kBins + 3];   // this CTA's histogram
+    __shared__ int s_all[kFusedCS][kBins + 3];   // the eight CTAs' histograms, each pushed by its owner
     __shared__ __align__(16) uint32_t c_hist[kBins][32];   // one counter per (level, lane), shared by the warps
-    __shared__ int s_hist[kBins + 3], s_tot[kBins], s_bef[kBins];
-    __shared__ int sh_T, sh_r, sh_gt_before, sh_eq_before;
     __shared__ int s_wcnt[kFusedWarps];
     __shared__ float s_m[kFusedWarps][8], s_l[kFusedWarps][8];
     __shared__ uint32_t s_mask[kFusedWarps][kFusedMaxStages];
 
+    cluster_arrive();   // completed below, before the first store into a peer's shared memory: every CTA has started
     const uint32_t rank = cluster_rank();
     const int kvh = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -195,27 +202,24 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     }
     for (int i = tid; i < kBins * 32 / 4; i += kFusedThreads)
         reinterpret_cast<uint4 *>(&c_hist[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (tid < kBins + 3) s_hist[tid] = 0;
     pdl_wait();                  // q, k_new and everything older in the stream is final from here on
     pdl_launch_dependents();
+    cluster_wait();              // #0: all eight CTAs are running (their shared memory may be written)
 
     // ---------------- P1: ENCODE in CTA 0 (queries) and CTA 1 (appended key)
     if (enc_q) {
-        fused_encode<kQPer>(a.q + (head0 + kQPer * (int)rank) * kD, kD, sw1, sw2, sw3, actA, actB, s_codes, bias1,
-                            bias2, bias3);
-        if (tid < kQPer) a.q_codes[head0 + kQPer * (int)rank + tid] = s_codes[tid];
+        fused_encode<kQPer>(a.q + (head0 + kQPer * (int)rank) * kD, kD, sw1, sw2, sw3, actA, actB,
+                            s_codes + kQPer * (int)rank, a.q_codes + head0 + kQPer * (int)rank, bias1, bias2, bias3);
     } else if (enc_k) {
-        fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, sw1, sw2, sw3, actA, actB, s_codes, bias1, bias2,
-                        bias3);
-        if (tid == 0) row[n - 1] = s_codes[0];
+        fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, sw1, sw2, sw3, actA, actB, s_codes + G,
+                        row + (n - 1), bias1, bias2, bias3);
     }
-    cluster_sync_all();   // #1: the signatures are in the encoding CTAs' shared memory
+    cluster_sync_all();   // #1: every CTA holds all signatures (and its counters are zeroed)
     uint32_t qc[G];
 #pragma unroll
-    for (int j = 0; j < G; ++j)
-        qc[j] = (uint32_t)ld_dsmem(reinterpret_cast<const int *>(&s_codes[j % kQPer]), (uint32_t)(j / kQPer));
+    for (int j = 0; j < G; ++j) qc[j] = s_codes[j];
     if (has_new_key) {   // the appended token's signature replaces whatever the early request saw
-        const uint32_t kc = (uint32_t)ld_dsmem(reinterpret_cast<const int *>(&s_codes[0]), (uint32_t)kQCtas);
+        const uint32_t kc = s_codes[G];
 #pragma unroll
         for (int p = 0; p < kFusedL; ++p) {
             const int e = (n - 1) - (wbase + p * 4);
@@ -224,7 +228,6 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
             }
         }
     }
-    __syncthreads();   // c_hist / s_hist zeroing is visible
 
     // ---------------- P2: SCORE, histogram, threshold, compaction
     uint32_t sc[kFusedL];
@@ -262,37 +265,41 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         }
     }
     __syncthreads();
-    for (int i = tid; i < kBins * 8; i += kFusedThreads) {   // eight threads per level, four counters each
+    // Fold and exchange: eight threads per level add four counters each and a shuffle tree completes the
+    // level; then warp w stores the 33 counts into row `rank` of CTA w's table (one destination per warp, so
+    // that a store instruction travels as one packet).
+    for (int i = tid; i < kBins * 8; i += kFusedThreads) {   // 264 = 33 aligned groups of eight lanes
         const uint4 v = reinterpret_cast<const uint4 *>(&c_hist[i >> 3][0])[i & 7];
-        const uint32_t ssum = (v.x + v.y) + (v.z + v.w);
-        if (ssum) atomicAdd(&s_hist[i >> 3], (int)ssum);
+        uint32_t ssum = (v.x + v.y) + (v.z + v.w);
+        const unsigned grp = 0xffu << (lane & 24);
+        ssum += __shfl_xor_sync(grp, ssum, 1);
+        ssum += __shfl_xor_sync(grp, ssum, 2);
+        ssum += __shfl_xor_sync(grp, ssum, 4);
+        if ((i & 7) == 0) s_hist[i >> 3] = ssum;
     }
-    cluster_sync_all();   // #2: every CTA's histogram is complete and visible cluster-wide
-    if (tid < kBins) {
-        int tot = 0, bef = 0;
+    __syncthreads();
+    st_dsmem_u32(reinterpret_cast<uint32_t *>(&s_all[rank][lane]), (uint32_t)warp, s_hist[lane]);
+    if (lane == 0) st_dsmem_u32(reinterpret_cast<uint32_t *>(&s_all[rank][32]), (uint32_t)warp, s_hist[32]);
+    cluster_sync_all();   // #2: every CTA holds all eight histograms
+    // every warp derives the threshold for itself (lane l owns level l, level 32 is read by every lane)
+    int T, r, gt_before, eq_before;
+    {
+        int tot = 0, bef = 0, tot32 = 0, bef32 = 0;
 #pragma unroll
-        for (uint32_t r = 0; r < (uint32_t)kFusedCS; ++r) {
-            const int v = ld_dsmem(&s_hist[tid], r);
+        for (int rr = 0; rr < kFusedCS; ++rr) {
+            const int v = s_all[rr][lane], v32 = s_all[rr][32];
             tot += v;
-            if (r < rank) bef += v;
+            tot32 += v32;
+            if (rr < (int)rank) { bef += v; bef32 += v32; }
         }
-        s_tot[tid] = tot;
-        s_bef[tid] = bef;
+        find_threshold(tot, bef, tot32, bef32, keep_rest, lane, T, r, gt_before, eq_before);
     }
-    __syncthreads();
-    if (warp == 0) {
-        int T, r, gt_before, eq_before;
-        find_threshold(s_tot[lane], s_bef[lane], s_tot[32], s_bef[32], keep_rest, lane, T, r, gt_before, eq_before);
-        if (lane == 0) { sh_T = T; sh_r = r; sh_gt_before = gt_before; sh_eq_before = eq_before; }
-    }
-    __syncthreads();
     int32_t *list = a.idx + (long long)b * a.idx_sb + (long long)kvh * a.idx_sh;
     if (rank == 0) {
         if (tid == 0) a.count[b * Hkv + kvh] = keep;
         for (int i = keep + tid; i < a.k_max; i += kFusedThreads) list[i] = -1;
     }
     if (keep > 0) {
-        const int T = sh_T, r = sh_r;
         // Per byte b = score + 1 (0 = no token): b + 127 - (T+1) sets bit 7 iff score > T, b + 128 - (T+1) iff
         // score >= T (no byte sum reaches 256).
         const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
@@ -314,7 +321,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         if (lane == 31) s_wcnt[warp] = winc;
         __syncthreads();
         // tokens before this warp's range with S > T (always-kept tokens count as such) / S == T
-        int run_gt = sh_gt_before + forced_before(wbd, min((int)rank * 1024 * Lb, n)), run_eq = sh_eq_before;
+        int run_gt = gt_before + forced_before(wbd, min((int)rank * 1024 * Lb, n)), run_eq = eq_before;
 #pragma unroll
         for (int w = 0; w < kFusedWarps; ++w)
             if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
