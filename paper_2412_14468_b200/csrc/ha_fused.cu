@@ -81,11 +81,11 @@ __device__ __forceinline__ void st_dsmem_f32(float *local, uint32_t rank, float 
 // caller has put the three matrices into shared memory, transposed (TransposedFetch), before the
 // call; the barrier that publishes the input vectors also publishes them.  Signature v is written to
 // word v of `dst` in the shared memory of EVERY CTA of the cluster (lanes 0..7 of the warp that holds it
-// store to CTAs 0..7; the cluster barrier that follows makes the stores visible) and to global_dst[v].
+// store to CTAs 0..7; the cluster barrier that follows makes the stores visible).
 template <int NV>
 __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_stride, const uint16_t *sw1,
                                              const uint16_t *sw2, const uint16_t *sw3, float *actA, float *actB,
-                                             uint32_t *dst, uint32_t *global_dst, float bias1, float bias2, float bias3) {
+                                             uint32_t *dst, float bias1, float bias2, float bias3) {
     const int tid = threadIdx.x, o = tid & 127;
     const bool active = tid < 128;
     if (active) {
@@ -117,7 +117,6 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
             vec_layer_t<1>(actA + v * kD, sw3, lane, z3);
             const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
             if (lane < kFusedCS) st_dsmem_u32(dst + v, (uint32_t)lane, code);
-            if (lane == kFusedCS) global_dst[v] = code;
         }
     }
 }
@@ -209,12 +208,16 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     // ---------------- P1: ENCODE in CTA 0 (queries) and CTA 1 (appended key)
     if (enc_q) {
         fused_encode<kQPer>(a.q + (head0 + kQPer * (int)rank) * kD, kD, sw1, sw2, sw3, actA, actB,
-                            s_codes + kQPer * (int)rank, a.q_codes + head0 + kQPer * (int)rank, bias1, bias2, bias3);
+                            s_codes + kQPer * (int)rank, bias1, bias2, bias3);
     } else if (enc_k) {
-        fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, sw1, sw2, sw3, actA, actB, s_codes + G,
-                        row + (n - 1), bias1, bias2, bias3);
+        fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, sw1, sw2, sw3, actA, actB, s_codes + G, bias1,
+                        bias2, bias3);
     }
     cluster_sync_all();   // #1: every CTA holds all signatures (and its counters are zeroed)
+    // the signatures also go to global memory (outputs of the step; nobody in this kernel reads them there):
+    // stored after the barrier, so that its release had nothing but shared-memory stores to wait for
+    if (enc_q && tid < kQPer) a.q_codes[head0 + kQPer * (int)rank + tid] = s_codes[kQPer * (int)rank + tid];
+    if (enc_k && tid == 0) row[n - 1] = s_codes[G];
     uint32_t qc[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) qc[j] = s_codes[j];
