@@ -136,6 +136,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     float *part_acc = part_ml + kFusedCS * G * 2;                                   // [CS][G][128]
     __shared__ uint32_t s_codes[kMaxGroup + 1];   // the G query signatures and the appended key's, pushed by the encoding CTAs
     __shared__ uint32_t s_hist[kBins + 3];   // this CTA's histogram
+    __shared__ int32_t s_list[kFusedWarps * kBlockTokens];   // one-stage variant: this CTA's part of the index list
     __shared__ int s_all[kFusedCS][kBins + 3];   // the eight CTAs' histograms, each pushed by its owner
     __shared__ __align__(16) uint32_t c_hist[kBins][32];   // one counter per (level, lane), shared by the warps
     __shared__ int s_wcnt[kFusedWarps];
@@ -298,7 +299,18 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         find_threshold(tot, bef, tot32, bef32, keep_rest, lane, T, r, gt_before, eq_before);
     }
     int32_t *list = a.idx + (long long)b * a.idx_sb + (long long)kvh * a.idx_sh;
-    if (rank == 0) {
+    // GATHER-ATT shares: CTA c attends to blocks [c * bpc, (c + 1) * bpc) of the list (16 entries each)
+    const int blocks_total = (keep + kBlockTokens - 1) / kBlockTokens;
+    const int bpc = (blocks_total + kFusedCS - 1) / kFusedCS;             // blocks per CTA
+    const int blk_lo = min(blocks_total, (int)rank * bpc), blk_hi = min(blocks_total, blk_lo + bpc);
+    // One-stage variant (at most 1024 entries): the selected tokens of this CTA's slice, which are a run of
+    // consecutive list positions, are compacted in shared memory and sent, coalesced, into the shared memory
+    // of the CTAs that will attend to them; each CTA writes its own part of the list to global memory after
+    // the barrier.  Nothing but shared-memory stores is pending at the barrier and nobody reads the list from L2.
+    constexpr bool kLocalList = (S == 1);
+    int32_t *s_sel = reinterpret_cast<int32_t *>(&c_hist[0][0]);   // the counters are dead by now
+    static_assert(sizeof(uint32_t) * kBins * 32 >= sizeof(int32_t) * kFusedCS * kFusedWarps * kBlockTokens, "s_sel fits c_hist");
+    if (!kLocalList && rank == 0) {
         if (tid == 0) a.count[b * Hkv + kvh] = keep;
         for (int i = keep + tid; i < a.k_max; i += kFusedThreads) list[i] = -1;
     }
@@ -324,20 +336,41 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         if (lane == 31) s_wcnt[warp] = winc;
         __syncthreads();
         // tokens before this warp's range with S > T (always-kept tokens count as such) / S == T
-        int run_gt = gt_before + forced_before(wbd, min((int)rank * 1024 * Lb, n)), run_eq = eq_before;
+        const int cta_gt = gt_before + forced_before(wbd, min((int)rank * 1024 * Lb, n)), cta_eq = eq_before;
+        int run_gt = cta_gt, run_eq = cta_eq, all_gt = cta_gt, all_eq = cta_eq;
 #pragma unroll
-        for (int w = 0; w < kFusedWarps; ++w)
-            if (w < warp) { run_gt += s_wcnt[w] & 0xffff; run_eq += (int)((unsigned)s_wcnt[w] >> 16); }
+        for (int w = 0; w < kFusedWarps; ++w) {
+            const int wg = s_wcnt[w] & 0xffff, wq = (int)((unsigned)s_wcnt[w] >> 16);
+            if (w < warp) { run_gt += wg; run_eq += wq; }
+            all_gt += wg;
+            all_eq += wq;
+        }
         const int excl = winc - tot_packed;
         int g_run = run_gt + (excl & 0xffff), q_run = run_eq + (int)((unsigned)excl >> 16);
-        write_selected32(list, wbase, gt16, eq16, g_run, q_run, r);
+        if (kLocalList) {
+            const int pos0 = cta_gt + min(cta_eq, r), cnt = all_gt + min(all_eq, r) - pos0;   // this CTA's run of positions
+            visit_selected32(wbase, gt16, eq16, g_run, q_run, r, [&](int pos, int t) { s_sel[pos - pos0] = t; });
+            __syncthreads();
+            const int per_cta = bpc * kBlockTokens;
+            for (int i = tid; i < cnt; i += kFusedThreads) {
+                const int pos = pos0 + i, owner = pos / per_cta;
+                st_dsmem_u32(reinterpret_cast<uint32_t *>(&s_list[pos - owner * per_cta]), (uint32_t)owner, (uint32_t)s_sel[i]);
+            }
+        } else {
+            write_selected32(list, wbase, gt16, eq16, g_run, q_run, r);
+        }
     }
-    cluster_sync_all();   // #3: the index list is complete and visible to the whole cluster; histograms are free
+    cluster_sync_all();   // #3: the index list is complete and visible to the whole cluster
+    if (kLocalList) {
+        const int my_lo = blk_lo * kBlockTokens, my_n = min(keep, blk_hi * kBlockTokens) - my_lo;
+        if (tid < my_n) list[my_lo + tid] = s_list[tid];
+        if (rank == 0) {
+            if (tid == 0) a.count[b * Hkv + kvh] = keep;
+            for (int i = keep + tid; i < a.k_max; i += kFusedThreads) list[i] = -1;
+        }
+    }
 
     // ---------------- P3: GATHER-ATT over this CTA's eighth of the list
-    const int blocks_total = (keep + kBlockTokens - 1) / kBlockTokens;
-    const int bpc = (blocks_total + kFusedCS - 1) / kFusedCS;             // blocks per CTA
-    const int blk_lo = min(blocks_total, (int)rank * bpc), blk_hi = min(blocks_total, blk_lo + bpc);
     const bool paged = a.block_table != nullptr;   // rows are then addressed from the pool's base
     const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (paged ? 0LL : (long long)b * a.K.sb) + (long long)kvh * a.K.sh);
     const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (paged ? 0LL : (long long)b * a.V.sb) + (long long)kvh * a.V.sh);
@@ -360,7 +393,8 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         const int nblk = (blk_lo + warp < blk_hi) ? (blk_hi - blk_lo - warp + kFusedWarps - 1) / kFusedWarps : 0;
         auto token_of_block = [&](int i) -> int {
             const int p = (blk_lo + warp + i * kFusedWarps) * kBlockTokens + (lane & 15);
-            int t = (i < nblk && p < keep) ? __ldcg(list + p) : -1;
+            int t = -1;
+            if (i < nblk && p < keep) t = kLocalList ? s_list[p - blk_lo * kBlockTokens] : __ldcg(list + p);
             // paged: logical token -> row of the pool (page * rows per page stride + slot)
             if (paged && t >= 0) t = __ldg(pages + (t >> a.page_shift)) * a.page_rows + (t & ((1 << a.page_shift) - 1));
             return t;

@@ -62,16 +62,22 @@ __device__ __forceinline__ int one_hot_index(uint32_t one_hot) {
 
 // Visits the flagged tokens among 32 consecutive tokens from `first` on in ascending order; g_run / q_run
 // count the tokens with S > T / S == T seen so far in the whole sequence; r tokens of score T are wanted.
-__device__ __forceinline__ void write_selected32(int32_t *list, int first, uint32_t gt, uint32_t eq, int &g_run,
-                                                 int &q_run, int r) {
+// sink(position in the index list, token) is called for every selected token.
+template <typename Sink>
+__device__ __forceinline__ void visit_selected32(int first, uint32_t gt, uint32_t eq, int &g_run, int &q_run, int r,
+                                                 Sink &&sink) {
     uint32_t m = gt | eq;
     while (m) {
         const uint32_t lb = m & (0u - m);
         m ^= lb;
         const int t = first + one_hot_index(lb);
-        if (gt & lb) { list[g_run + min(q_run, r)] = t; ++g_run; }
-        else { if (q_run < r) list[g_run + q_run] = t; ++q_run; }
+        if (gt & lb) { sink(g_run + min(q_run, r), t); ++g_run; }
+        else { if (q_run < r) sink(g_run + q_run, t); ++q_run; }
     }
+}
+__device__ __forceinline__ void write_selected32(int32_t *list, int first, uint32_t gt, uint32_t eq, int &g_run,
+                                                 int &q_run, int r) {
+    visit_selected32(first, gt, eq, g_run, q_run, r, [&](int pos, int t) { list[pos] = t; });
 }
 
 // Warp-wide threshold search over the 33 score levels.  Lane l passes the count of level l (tot) and
