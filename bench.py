@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 
 METRIC = "sparse_decode_attn_us_per_layer_step"
 UNIT = "us"
-FUSED_KERNEL_TRAFFIC_C2 = 6519000   # dram__bytes_read.sum + write per launch, profiles/launch_list_bench_c2.md
+FUSED_KERNEL_TRAFFIC_C2 = 6543000   # dram__bytes_read.sum + write per launch, profiles/launch_list_bench_c2.md
 WORKLOAD = "c2: B=1, Hq=32, Hkv=8, d=128, ctx=32768, k=1024 (32x), 1% planted keys"
 
 
@@ -342,7 +342,7 @@ def main():
     g_us = parts["ha_gather_attn"]
     roofline = {
         "bound": "hbm",
-        "kernel": ("fused_step_kernel<4> (the one kernel of ha_sparse_decode at this batch size)"
+        "kernel": ("fused_step_kernel<4,1> (the one kernel of ha_sparse_decode at this batch size)"
                    if launches_per_step < 1.5 else "kernels of ha_sparse_decode (multi-kernel path)"),
         "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
         # dram__bytes_read.sum + dram__bytes_write.sum per launch of this kernel on this workload, from the
