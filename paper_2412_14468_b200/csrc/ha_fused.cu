@@ -26,21 +26,30 @@
 
 namespace ha {
 
-constexpr int kFusedCS = 8;
+constexpr int kFusedMaxCS = 8;                               // CTAs per cluster (template parameter CS: 8 or 4; 2 is supported, unused)
 constexpr int kFusedWarps = 8;
 constexpr int kFusedThreads = kFusedWarps * 32;
-constexpr int kFusedL = 4;                                   // uint4 of signatures per thread (n <= 32768)
+constexpr int kFusedMaxSeq = 32768;                          // 32 uint4 of signatures per thread position, shared by the cluster
 constexpr int kFusedMaxStages = 2;                           // row blocks in flight per warp (template parameter S)
 constexpr int kFusedWeightBytes = (kD * kHid + kHid * kHid + kHid * kBits) * 2;
-constexpr int kFusedActBytes = 2 * 2 * kD * 4;               // two activation buffers of up to 2 vectors
+constexpr int kFusedOneStageMaxK = 2048;                     // one-stage variant: longest index list
+constexpr int kFusedListOffset = kFusedWarps * kStageBytes;  // one-stage variant: this CTA's part of the list sits behind the ring
+// query vectors per encoding CTA: the smallest divisor of G that leaves the cluster one CTA for the appended key
+__host__ __device__ constexpr int fused_q_per_cta(int G, int CS) {
+    return (G <= CS - 1) ? 1 : (G / 2 <= CS - 1) ? 2 : (G / 4 <= CS - 1) ? 4 : 8;
+}
 // Dynamic shared memory of a CTA: [weights | S row stages per warp] union, activations, the eight CTA states
 // of the G heads (used in CTA 0).  With S = 1 two CTAs fit one SM (and the kernel is compiled for 128
 // registers): two consecutive steps are then resident together, each cluster of the later one already
 // parked at its launch wait, whereas only 15 clusters of eight one-CTA SMs exist on the device.
 __host__ __device__ constexpr int fused_ring_bytes(int S) { return kFusedWarps * S * kStageBytes; }
 __host__ __device__ constexpr int fused_union_bytes(int S) { return fused_ring_bytes(S) > kFusedWeightBytes ? fused_ring_bytes(S) : kFusedWeightBytes; }
-__host__ __device__ constexpr int fused_part_bytes(int G) { return kFusedCS * G * (kD + 2) * 4; }
-__host__ __device__ constexpr int fused_smem_bytes(int G, int S) { return fused_union_bytes(S) + kFusedActBytes + fused_part_bytes(G); }
+__host__ __device__ constexpr int fused_act_bytes(int G, int CS) { return 2 * fused_q_per_cta(G, CS) * kD * 4; }   // two activation buffers
+__host__ __device__ constexpr int fused_part_bytes(int G, int CS) { return CS * G * (kD + 2) * 4; }
+__host__ __device__ constexpr int fused_smem_bytes(int G, int S, int CS) {
+    return fused_union_bytes(S) + fused_act_bytes(G, CS) + fused_part_bytes(G, CS);
+}
+static_assert(kFusedListOffset + kFusedOneStageMaxK / 2 * 4 <= kFusedWeightBytes, "the list part fits behind the one-stage ring");
 
 struct FusedArgs {
     MapView map_q, map_k;
@@ -80,9 +89,9 @@ __device__ __forceinline__ void st_dsmem_f32(float *local, uint32_t rank, float 
 // chains of output o for every vector.  A second warp per scheduler would not shorten any chain.  The
 // caller has put the three matrices into shared memory, transposed (TransposedFetch), before the
 // call; the barrier that publishes the input vectors also publishes them.  Signature v is written to
-// word v of `dst` in the shared memory of EVERY CTA of the cluster (lanes 0..7 of the warp that holds it
-// store to CTAs 0..7; the cluster barrier that follows makes the stores visible).
-template <int NV>
+// word v of `dst` in the shared memory of EVERY CTA of the cluster (lanes 0..CS-1 of the warp that holds it
+// store to CTAs 0..CS-1; the cluster barrier that follows makes the stores visible).
+template <int NV, int CS>
 __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_stride, const uint16_t *sw1,
                                              const uint16_t *sw2, const uint16_t *sw3, float *actA, float *actB,
                                              uint32_t *dst, float bias1, float bias2, float bias3) {
@@ -116,14 +125,21 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
             float z3[1] = {bias3};
             vec_layer_t<1>(actA + v * kD, sw3, lane, z3);
             const uint32_t code = __ballot_sync(0xffffffffu, z3[0] > 0.0f);
-            if (lane < kFusedCS) st_dsmem_u32(dst + v, (uint32_t)lane, code);
+            if (lane < CS) st_dsmem_u32(dst + v, (uint32_t)lane, code);
         }
     }
 }
 
-template <int G, int S>
+template <int G, int S, int CS>
 __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kernel(const FusedArgs a) {
     constexpr int kFusedUnionBytes = fused_union_bytes(S);
+    constexpr int kFusedActBytes = fused_act_bytes(G, CS);
+    constexpr int kL = kFusedMaxSeq / (CS * 4096) * 4;   // uint4 of signatures per thread: 4, 8 or 16
+    constexpr int kFlagWords = (kL + 7) / 8;             // 32 tokens' flags per word
+    constexpr int kQPer = fused_q_per_cta(G, CS);
+    constexpr int kQCtas = G / kQPer;
+    static_assert(kQCtas * kQPer == G && kQCtas < CS, "the cluster needs one more CTA for the appended key");
+    constexpr bool kPreload = (CS > 2);   // signatures requested before the launch wait (16 uint4 would not fit the registers)
     extern __shared__ __align__(128) unsigned char fsm[];
     // dynamic: [weights | row ring] union, activations, the cluster's states (used in CTA 0)
     uint16_t *sw1 = reinterpret_cast<uint16_t *>(fsm);
@@ -131,13 +147,12 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     uint16_t *sw3 = sw2 + kHid * kHid;
     unsigned char *ring = fsm;
     float *actA = reinterpret_cast<float *>(fsm + kFusedUnionBytes);
-    float *actB = actA + 2 * kD;
+    float *actB = actA + kQPer * kD;
     float *part_ml = reinterpret_cast<float *>(fsm + kFusedUnionBytes + kFusedActBytes);   // [CS][G][2]
-    float *part_acc = part_ml + kFusedCS * G * 2;                                   // [CS][G][128]
+    float *part_acc = part_ml + CS * G * 2;                                   // [CS][G][128]
     __shared__ uint32_t s_codes[kMaxGroup + 1];   // the G query signatures and the appended key's, pushed by the encoding CTAs
     __shared__ uint32_t s_hist[kBins + 3];   // this CTA's histogram
-    __shared__ int32_t s_list[kFusedWarps * kBlockTokens];   // one-stage variant: this CTA's part of the index list
-    __shared__ int s_all[kFusedCS][kBins + 3];   // the eight CTAs' histograms, each pushed by its owner
+    __shared__ int s_all[kFusedMaxCS][kBins + 3];   // the eight CTAs' histograms, each pushed by its owner
     __shared__ __align__(16) uint32_t c_hist[kBins][32];   // one counter per (level, lane), shared by the warps
     __shared__ int s_wcnt[kFusedWarps];
     __shared__ float s_m[kFusedWarps][8], s_l[kFusedWarps][8];
@@ -159,19 +174,19 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     const bool has_new_key = (a.k_new != nullptr) && n > 0;
 
     // ---------------- P0: requests that do not depend on earlier kernels
-    const int Lb = (n + kFusedCS * 1024 - 1) / (kFusedCS * 1024);
+    const int Lb = (n + CS * 1024 - 1) / (CS * 1024);
     const int wbase = ((int)rank * 1024 + warp * 128 + lane * 4) * Lb;
-    uint4 c[kFusedL];
+    uint4 c[kL];
+    auto load_signatures = [&]() {
 #pragma unroll
-    for (int p = 0; p < kFusedL; ++p) {
-        const int base = wbase + p * 4;
-        c[p] = (p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
-    }
+        for (int p = 0; p < kL; ++p) {
+            const int base = wbase + p * 4;
+            c[p] = (p < Lb && base < n) ? load_codes4(row, base, n) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    if (kPreload) load_signatures();
     // ENCODE roles: CTA r < kQCtas encodes kQPer query vectors (one per CTA while the cluster has room),
     // CTA kQCtas encodes the appended key; the other CTAs only scan
-    constexpr int kQPer = (G < kFusedCS) ? 1 : 2;
-    constexpr int kQCtas = (G + kQPer - 1) / kQPer;
-    static_assert(kQCtas < kFusedCS, "the cluster needs one more CTA for the appended key");
     const bool enc_q = (int)rank < kQCtas, enc_k = ((int)rank == kQCtas) && has_new_key;
     const bool encodes = enc_q || enc_k;
     const MapView &map = enc_q ? a.map_q : a.map_k;
@@ -194,24 +209,23 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         if (map.b1) bias1 = __ldg(map.b1 + kvh * kHid + o);
         if (map.b2) bias2 = __ldg(map.b2 + kvh * kHid + o);
         if (map.b3) bias3 = __ldg(map.b3 + kvh * kBits + (tid & (kBits - 1)));
-        if (tid < 2) {
+        if (tid < 2 * (enc_q ? kQPer : 1)) {   // 256 bytes per vector
             const uint16_t *xv = enc_q ? a.q + (head0 + kQPer * (int)rank) * kD : a.k_new + ((long long)b * Hkv + kvh) * kD;
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(xv) + 128 * tid));
-            if (enc_q && kQPer > 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(xv) + 256 + 128 * tid));
         }
     }
     for (int i = tid; i < kBins * 32 / 4; i += kFusedThreads)
         reinterpret_cast<uint4 *>(&c_hist[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
     pdl_wait();                  // q, k_new and everything older in the stream is final from here on
     pdl_launch_dependents();
-    cluster_wait();              // #0: all eight CTAs are running (their shared memory may be written)
+    cluster_wait();              // #0: all CTAs of the cluster are running (their shared memory may be written)
 
     // ---------------- P1: ENCODE in CTA 0 (queries) and CTA 1 (appended key)
     if (enc_q) {
-        fused_encode<kQPer>(a.q + (head0 + kQPer * (int)rank) * kD, kD, sw1, sw2, sw3, actA, actB,
+        fused_encode<kQPer, CS>(a.q + (head0 + kQPer * (int)rank) * kD, kD, sw1, sw2, sw3, actA, actB,
                             s_codes + kQPer * (int)rank, bias1, bias2, bias3);
     } else if (enc_k) {
-        fused_encode<1>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, sw1, sw2, sw3, actA, actB, s_codes + G, bias1,
+        fused_encode<1, CS>(a.k_new + ((long long)b * Hkv + kvh) * kD, kD, sw1, sw2, sw3, actA, actB, s_codes + G, bias1,
                         bias2, bias3);
     }
     cluster_sync_all();   // #1: every CTA holds all signatures (and its counters are zeroed)
@@ -222,10 +236,11 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     uint32_t qc[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) qc[j] = s_codes[j];
+    if (!kPreload) load_signatures();
     if (has_new_key) {   // the appended token's signature replaces whatever the early request saw
         const uint32_t kc = s_codes[G];
 #pragma unroll
-        for (int p = 0; p < kFusedL; ++p) {
+        for (int p = 0; p < kL; ++p) {
             const int e = (n - 1) - (wbase + p * 4);
             if (p < Lb && e >= 0 && e <= 3) {
                 if (e == 0) c[p].x = kc; else if (e == 1) c[p].y = kc; else if (e == 2) c[p].z = kc; else c[p].w = kc;
@@ -234,7 +249,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     }
 
     // ---------------- P2: SCORE, histogram, threshold, compaction
-    uint32_t sc[kFusedL];
+    uint32_t sc[kL];
     {
         // a lane only meets its own column of counters, so an instruction never conflicts with itself; the
         // adds are reductions that never wait for a result.  The counter of score s sits (32 - s) rows
@@ -248,7 +263,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
             return h;
         };
 #pragma unroll
-        for (int p = 0; p < kFusedL; ++p) {
+        for (int p = 0; p < kL; ++p) {
             const int base = wbase + p * 4;
             const int h0 = hamming(c[p].x), h1 = hamming(c[p].y), h2 = hamming(c[p].z), h3 = hamming(c[p].w);
             // bytes 33 - h = score + 1 (0 marks "no token"); no byte borrows because h <= 32
@@ -282,15 +297,17 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         if ((i & 7) == 0) s_hist[i >> 3] = ssum;
     }
     __syncthreads();
-    st_dsmem_u32(reinterpret_cast<uint32_t *>(&s_all[rank][lane]), (uint32_t)warp, s_hist[lane]);
-    if (lane == 0) st_dsmem_u32(reinterpret_cast<uint32_t *>(&s_all[rank][32]), (uint32_t)warp, s_hist[32]);
-    cluster_sync_all();   // #2: every CTA holds all eight histograms
+    if (warp < CS) {
+        st_dsmem_u32(reinterpret_cast<uint32_t *>(&s_all[rank][lane]), (uint32_t)warp, s_hist[lane]);
+        if (lane == 0) st_dsmem_u32(reinterpret_cast<uint32_t *>(&s_all[rank][32]), (uint32_t)warp, s_hist[32]);
+    }
+    cluster_sync_all();   // #2: every CTA holds all histograms of the cluster
     // every warp derives the threshold for itself (lane l owns level l, level 32 is read by every lane)
     int T, r, gt_before, eq_before;
     {
         int tot = 0, bef = 0, tot32 = 0, bef32 = 0;
 #pragma unroll
-        for (int rr = 0; rr < kFusedCS; ++rr) {
+        for (int rr = 0; rr < CS; ++rr) {
             const int v = s_all[rr][lane], v32 = s_all[rr][32];
             tot += v;
             tot32 += v32;
@@ -301,15 +318,15 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     int32_t *list = a.idx + (long long)b * a.idx_sb + (long long)kvh * a.idx_sh;
     // GATHER-ATT shares: CTA c attends to blocks [c * bpc, (c + 1) * bpc) of the list (16 entries each)
     const int blocks_total = (keep + kBlockTokens - 1) / kBlockTokens;
-    const int bpc = (blocks_total + kFusedCS - 1) / kFusedCS;             // blocks per CTA
+    const int bpc = (blocks_total + CS - 1) / CS;                         // blocks per CTA
     const int blk_lo = min(blocks_total, (int)rank * bpc), blk_hi = min(blocks_total, blk_lo + bpc);
-    // One-stage variant (at most 1024 entries): the selected tokens of this CTA's slice, which are a run of
+    // One-stage variant (at most kFusedOneStageMaxK entries): the selected tokens of this CTA's slice, which are a run of
     // consecutive list positions, are compacted in shared memory and sent, coalesced, into the shared memory
     // of the CTAs that will attend to them; each CTA writes its own part of the list to global memory after
     // the barrier.  Nothing but shared-memory stores is pending at the barrier and nobody reads the list from L2.
     constexpr bool kLocalList = (S == 1);
-    int32_t *s_sel = reinterpret_cast<int32_t *>(&c_hist[0][0]);   // the counters are dead by now
-    static_assert(sizeof(uint32_t) * kBins * 32 >= sizeof(int32_t) * kFusedCS * kFusedWarps * kBlockTokens, "s_sel fits c_hist");
+    int32_t *s_sel = reinterpret_cast<int32_t *>(fsm);                       // weights are dead, the ring not yet in use
+    int32_t *s_list = reinterpret_cast<int32_t *>(fsm + kFusedListOffset);   // this CTA's part of the list, behind the ring
     if (!kLocalList && rank == 0) {
         if (tid == 0) a.count[b * Hkv + kvh] = keep;
         for (int i = keep + tid; i < a.k_max; i += kFusedThreads) list[i] = -1;
@@ -319,14 +336,20 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         // score >= T (no byte sum reaches 256).
         const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
         const uint32_t c_gt = 0x7f7f7f7fu - T4, c_ge = 0x80808080u - T4;
-        uint32_t gt16 = 0, ge16 = 0;   // flags of this lane's 16 consecutive tokens
+        uint32_t gtw[kFlagWords], eqw[kFlagWords];   // flags of this lane's 4 kL consecutive tokens, 32 per word
 #pragma unroll
-        for (int p = 0; p < kFusedL; ++p) {
-            gt16 |= high_bits_to_nibble(sc[p] + c_gt) << (4 * p);
-            ge16 |= high_bits_to_nibble(sc[p] + c_ge) << (4 * p);
+        for (int w = 0; w < kFlagWords; ++w) { gtw[w] = 0u; eqw[w] = 0u; }
+#pragma unroll
+        for (int p = 0; p < kL; ++p) {
+            gtw[p / 8] |= high_bits_to_nibble(sc[p] + c_gt) << (4 * (p % 8));
+            eqw[p / 8] |= high_bits_to_nibble(sc[p] + c_ge) << (4 * (p % 8));
         }
-        const uint32_t eq16 = ge16 ^ gt16;   // score > T implies score >= T
-        const int tot_packed = __popc(gt16) | (__popc(eq16) << 16);
+        int tot_packed = 0;
+#pragma unroll
+        for (int w = 0; w < kFlagWords; ++w) {
+            eqw[w] ^= gtw[w];   // score > T implies score >= T
+            tot_packed += __popc(gtw[w]) | (__popc(eqw[w]) << 16);
+        }
         int winc = tot_packed;
 #pragma unroll
         for (int dd = 1; dd < 32; dd <<= 1) {
@@ -349,7 +372,9 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         int g_run = run_gt + (excl & 0xffff), q_run = run_eq + (int)((unsigned)excl >> 16);
         if (kLocalList) {
             const int pos0 = cta_gt + min(cta_eq, r), cnt = all_gt + min(all_eq, r) - pos0;   // this CTA's run of positions
-            visit_selected32(wbase, gt16, eq16, g_run, q_run, r, [&](int pos, int t) { s_sel[pos - pos0] = t; });
+#pragma unroll
+            for (int w = 0; w < kFlagWords; ++w)
+                visit_selected32(wbase + 32 * w, gtw[w], eqw[w], g_run, q_run, r, [&](int pos, int t) { s_sel[pos - pos0] = t; });
             __syncthreads();
             const int per_cta = bpc * kBlockTokens;
             for (int i = tid; i < cnt; i += kFusedThreads) {
@@ -357,13 +382,14 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
                 st_dsmem_u32(reinterpret_cast<uint32_t *>(&s_list[pos - owner * per_cta]), (uint32_t)owner, (uint32_t)s_sel[i]);
             }
         } else {
-            write_selected32(list, wbase, gt16, eq16, g_run, q_run, r);
+#pragma unroll
+            for (int w = 0; w < kFlagWords; ++w) write_selected32(list, wbase + 32 * w, gtw[w], eqw[w], g_run, q_run, r);
         }
     }
     cluster_sync_all();   // #3: the index list is complete and visible to the whole cluster
     if (kLocalList) {
         const int my_lo = blk_lo * kBlockTokens, my_n = min(keep, blk_hi * kBlockTokens) - my_lo;
-        if (tid < my_n) list[my_lo + tid] = s_list[tid];
+        for (int i = tid; i < my_n; i += kFusedThreads) list[my_lo + i] = s_list[i];
         if (rank == 0) {
             if (tid == 0) a.count[b * Hkv + kvh] = keep;
             for (int i = keep + tid; i < a.k_max; i += kFusedThreads) list[i] = -1;
@@ -470,7 +496,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
             }
         }
     }
-    cluster_sync_all();   // #4: all eight states have landed in CTA 0
+    cluster_sync_all();   // #4: the states of all CTAs have landed in CTA 0
     if (rank == 0) {
         const int d = tid & (kD - 1), hsel = tid >> 7;
 #pragma unroll
@@ -479,11 +505,11 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
             if (G == 1 && hsel != 0) continue;
             float M = -CUDART_INF_F;
 #pragma unroll
-            for (int r = 0; r < kFusedCS; ++r) M = fmaxf(M, part_ml[(r * G + j) * 2]);
+            for (int r = 0; r < CS; ++r) M = fmaxf(M, part_ml[(r * G + j) * 2]);
             float L = 0.0f, A = 0.0f;
             if (M > -CUDART_INF_F) {
 #pragma unroll
-                for (int r = 0; r < kFusedCS; ++r) {
+                for (int r = 0; r < CS; ++r) {
                     const float f = exp2f(part_ml[(r * G + j) * 2] - M);
                     L = fmaf(part_ml[(r * G + j) * 2 + 1], f, L);
                     A = fmaf(part_acc[(r * G + j) * kD + d], f, A);
@@ -497,15 +523,15 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     }
 }
 
-template <int G, int S>
+template <int G, int S, int CS>
 static void fused_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute (&attr)[2], int Hkv, int B, cudaStream_t st) {
     cfg = cudaLaunchConfig_t{};
-    cfg.gridDim = dim3(kFusedCS, Hkv, B);
+    cfg.gridDim = dim3(CS, Hkv, B);
     cfg.blockDim = dim3(kFusedThreads);
-    cfg.dynamicSmemBytes = fused_smem_bytes(G, S);
+    cfg.dynamicSmemBytes = fused_smem_bytes(G, S, CS);
     cfg.stream = st;
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kFusedCS;
+    attr[0].val.clusterDim.x = CS;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -516,66 +542,79 @@ static void fused_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute (&attr)[2]
 
 // Opt in to the shared-memory carve-out (once per device) and return how many clusters of this variant the
 // device holds at once (0 on error).
-template <int G, int S>
+template <int G, int S, int CS>
 static int fused_prepare() {
     static int clusters[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
     if (!clusters[dev]) {
-        if (cudaFuncSetAttribute(fused_step_kernel<G, S>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 fused_smem_bytes(G, S)) != cudaSuccess)
+        if (cudaFuncSetAttribute(fused_step_kernel<G, S, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 fused_smem_bytes(G, S, CS)) != cudaSuccess)
             return 0;
         cudaLaunchConfig_t cfg;
         cudaLaunchAttribute attr[2];
-        fused_config<G, S>(cfg, attr, 1, 64, nullptr);
+        fused_config<G, S, CS>(cfg, attr, 1, 64, nullptr);
         cfg.numAttrs = 1;   // the cluster shape is all the occupancy query looks at
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, fused_step_kernel<G, S>, &cfg) != cudaSuccess || n <= 0) return 0;
+        if (cudaOccupancyMaxActiveClusters(&n, fused_step_kernel<G, S, CS>, &cfg) != cudaSuccess || n <= 0) return 0;
         clusters[dev] = n;
     }
     return clusters[dev];
 }
 
-template <int G, int S>
-static cudaError_t launch_fused_gs(const FusedArgs &args, int B, cudaStream_t st) {
-    if (fused_prepare<G, S>() <= 0) return cudaErrorInvalidConfiguration;
+template <int G, int S, int CS>
+static cudaError_t launch_fused_gsc(const FusedArgs &args, int B, cudaStream_t st) {
+    if (fused_prepare<G, S, CS>() <= 0) return cudaErrorInvalidConfiguration;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
-    fused_config<G, S>(cfg, attr, args.Hkv, B, st);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_step_kernel<G, S>, args);
+    fused_config<G, S, CS>(cfg, attr, args.Hkv, B, st);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_step_kernel<G, S, CS>, args);
     if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
 }
 
-// One stage per warp (two CTAs per SM) when no warp meets more than one block of the list, i.e. up to
-// 8 CTAs x 8 warps x 16 selected rows; two stages (one CTA per SM) beyond.
-static bool fused_one_stage(int k_max) { return k_max <= kFusedCS * kFusedWarps * kBlockTokens; }
-
+// Variant for a step of `units` (sequence, KV head) pairs with index lists of up to k_max entries.
+// Lists of up to kFusedOneStageMaxK entries take the one-stage kernel (two CTAs per SM) with the larger
+// cluster, 8 or 4 CTAs per unit, of which `units` are resident at once; longer lists the two-stage kernel
+// with clusters of 8.  Returns the cluster size, 0 if the step does not fit (a cluster that had to wait
+// for another one to finish would double the latency).  Clusters of 2 work as well (the kernel is
+// written for them) but lose to the three-kernel path at the batch sizes they would serve (45.7 against
+// 41.3 us at 128 units), so they are not offered.
 template <int G>
-static int fused_cluster_limit(int k_max) {
-    return fused_one_stage(k_max) ? fused_prepare<G, 1>() : fused_prepare<G, 2>();
+static int fused_variant(long long units, int k_max, int *stages) {
+    if (k_max <= kFusedOneStageMaxK) {
+        *stages = 1;
+        if (units <= fused_prepare<G, 1, 8>()) return 8;
+        if (units <= fused_prepare<G, 1, 4>()) return 4;
+        return 0;
+    }
+    *stages = 2;
+    return units <= fused_prepare<G, 2, 8>() ? 8 : 0;
 }
 
-// The fused step is used while every cluster of the step is resident at once (a cluster that has to wait
-// for another one to finish would double the latency) and a CTA's eighth of a sequence fits its registers.
 bool fused_step_eligible(int B, int Hq, int Hkv, int max_seq_len, int k_max) {
-    if (max_seq_len > kFusedCS * kFusedL * 1024 || Hkv <= 0) return false;
-    int limit = 0;
+    if (max_seq_len > kFusedMaxSeq || Hkv <= 0) return false;
+    const long long units = (long long)B * Hkv;
+    int stages = 0;
     switch (Hq / Hkv) {
-        case 1: limit = fused_cluster_limit<1>(k_max); break;
-        case 2: limit = fused_cluster_limit<2>(k_max); break;
-        case 4: limit = fused_cluster_limit<4>(k_max); break;
-        case 8: limit = fused_cluster_limit<8>(k_max); break;
+        case 1: return fused_variant<1>(units, k_max, &stages) > 0;
+        case 2: return fused_variant<2>(units, k_max, &stages) > 0;
+        case 4: return fused_variant<4>(units, k_max, &stages) > 0;
+        case 8: return fused_variant<8>(units, k_max, &stages) > 0;
         default: return false;
     }
-    return (long long)B * Hkv <= limit;
 }
 
 template <int G>
 static cudaError_t launch_fused_g(const FusedArgs &args, int B, cudaStream_t st) {
-    return fused_one_stage(args.k_max) ? launch_fused_gs<G, 1>(args, B, st) : launch_fused_gs<G, 2>(args, B, st);
+    int stages = 0;
+    const int cs = fused_variant<G>((long long)B * args.Hkv, args.k_max, &stages);
+    if (stages == 2 && cs == 8) return launch_fused_gsc<G, 2, 8>(args, B, st);
+    if (cs == 8) return launch_fused_gsc<G, 1, 8>(args, B, st);
+    if (cs == 4) return launch_fused_gsc<G, 1, 4>(args, B, st);
+    return cudaErrorInvalidConfiguration;
 }
 
 cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapView &map_q, const MapView &map_k,

@@ -523,6 +523,8 @@ def test_sparse_decode_step_matches_oracle(cfg):
 @pytest.mark.parametrize("cfg", [
     wl.Config("win-ragged", 55, 3, [300, 2049, 1], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8),     # one fused launch
     wl.Config("win-batch", 56, 24, [900 + 37 * i for i in range(24)], None, 0.02, n_q_heads=8, n_kv_heads=2,
+              sparsity=8),                                                             # one fused launch, clusters of 4
+    wl.Config("win-large-batch", 59, 90, [500 + 11 * i for i in range(90)], None, 0.02, n_q_heads=8, n_kv_heads=2,
               sparsity=8),                                                                                  # three kernels
     wl.CONFIGS["c1"],
 ])
@@ -548,6 +550,8 @@ def test_sparse_decode_step_with_always_kept_windows(cfg, n_sink, n_local):
 @pytest.mark.parametrize("cfg", [
     wl.Config("paged-small", 57, 2, [1500, 333], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8),        # one fused launch
     wl.Config("paged-batch", 58, 20, [700 + 53 * i for i in range(20)], None, 0.02, n_q_heads=8, n_kv_heads=2,
+              sparsity=8),                                                              # one fused launch, clusters of 4
+    wl.Config("paged-large-batch", 60, 85, [300 + 13 * i for i in range(85)], None, 0.02, n_q_heads=8, n_kv_heads=2,
               sparsity=8),                                                                                   # three kernels
 ])
 @pytest.mark.parametrize("page_size", [1, 16])
@@ -583,12 +587,12 @@ def test_sparse_decode_step_over_a_paged_cache(cfg, page_size):
         assert torch.equal(out, ref["out"])
 
 
-@pytest.mark.parametrize("seed", range(8))
+@pytest.mark.parametrize("seed", range(14))
 def test_sparse_decode_step_random_configs(seed):
     """Seeded sweep over batch (both the fused launch and the three-kernel path), KV heads, group size, ragged
     lengths, sparsity and window sizes; everything the step returns is checked against the oracle."""
     rng = np.random.default_rng(7000 + seed)
-    B = int(rng.integers(1, 13))
+    B = int(rng.integers(1, 13)) if seed < 8 else int(rng.integers(13, 110))   # up to 24 units / up to 220 units
     Hkv = int(rng.choice([1, 2]))
     G = int(rng.choice([1, 2, 4, 8]))
     lens = [int(v) for v in rng.integers(1, 3000, size=B)]
@@ -608,17 +612,20 @@ def test_sparse_decode_step_random_configs(seed):
 
 
 @pytest.mark.parametrize("cfg,launches", [
-    # 32 units, small budgets: one fused launch of the one-stage variant (two CTAs per SM)
+    # 32 units, small budgets: one fused launch of the one-stage variant (two CTAs per SM), clusters of 8
     (wl.Config("fused-32-units", 80, 16, [1000 + 61 * i for i in range(16)], None, 0.02, n_q_heads=8, n_kv_heads=2,
                sparsity=8), 1),
-    # 6 units, budgets above 1024 rows: one fused launch of the two-stage variant, several blocks per warp
-    (wl.Config("fused-large-k", 81, 3, [9000, 5000, 12001], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=4), 1),
-    # 20 units with budgets above 1024 rows: more clusters than the two-stage variant holds at once
+    # 60 units: clusters of 4 (two query vectors per encoding CTA, 32 tokens per thread)
+    (wl.Config("fused-60-units", 84, 30, [1500 + 97 * i for i in range(30)], None, 0.02, n_q_heads=8, n_kv_heads=2,
+               sparsity=8), 1),
+    # 100 units: more clusters of four than the device holds at once
+    (wl.Config("split-100-units", 85, 50, [2500 + 301 * i for i in range(50)], None, 0.02, n_q_heads=16, n_kv_heads=2,
+               sparsity=16), 3),
+    # 6 units, budgets above 2048 rows: one fused launch of the two-stage variant, several blocks per warp
+    (wl.Config("fused-large-k", 81, 3, [9000, 5000, 12001], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=2), 1),
+    # 20 units with budgets above 2048 rows: more clusters than the two-stage variant holds at once
     (wl.Config("split-large-k", 82, 10, [6000 + 7 * i for i in range(10)], None, 0.02, n_q_heads=8, n_kv_heads=2,
-               sparsity=4), 3),
-    # 34 units: more clusters than the device holds at once
-    (wl.Config("split-34-units", 83, 17, [800 + 29 * i for i in range(17)], None, 0.02, n_q_heads=4, n_kv_heads=2,
-               sparsity=8), 3),
+               sparsity=2), 3),
 ])
 def test_sparse_decode_step_every_launch_variant(cfg, launches):
     """The step picks the fused cluster kernel (one or two row stages per warp) or the three-kernel path from
@@ -651,7 +658,7 @@ def test_k_equals_n_sparse_step_equals_dense_kernel():
     assert r["cnt"].cpu().tolist() == [[1500, 1500], [900, 900]]
 
 
-@pytest.mark.parametrize("reps", [1, 5])     # 8 units: single fused kernel; 40 units: three-kernel path
+@pytest.mark.parametrize("reps", [1, 5, 12, 40])     # 8 / 40 units: fused kernel, clusters of 8 / 4; 96 and 320 units: three-kernel path
 def test_step_edge_cases_empty_sequence_budget_above_length_and_no_new_key(reps):
     # one launch covers: an empty sequence, a one-token sequence, k > n, k = 0; then the same without a new key
     cfg = wl.Config("edges", 53, 4 * reps, [0, 1, 37, 2500] * reps, 64, 0.0, n_q_heads=8, n_kv_heads=2)
