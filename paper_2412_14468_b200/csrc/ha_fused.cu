@@ -575,23 +575,28 @@ static cudaError_t launch_fused_gsc(const FusedArgs &args, int B, cudaStream_t s
     return cudaGetLastError();
 }
 
-// Variant for a step of `units` (sequence, KV head) pairs with index lists of up to k_max entries.
-// Lists of up to kFusedOneStageMaxK entries take the one-stage kernel (two CTAs per SM) with the larger
-// cluster, 8 or 4 CTAs per unit, of which `units` are resident at once; longer lists the two-stage kernel
-// with clusters of 8.  Returns the cluster size, 0 if the step does not fit (a cluster that had to wait
-// for another one to finish would double the latency).  Clusters of 2 work as well (the kernel is
-// written for them) but lose to the three-kernel path at the batch sizes they would serve (45.7 against
-// 41.3 us at 128 units), so they are not offered.
+// Variant for a step of `units` (sequence, KV head) pairs with index lists of up to k_max entries: the number
+// of row stages per warp in *stages, the cluster size as the result, 0 if the step does not fit (a
+// cluster that had to wait for another one to finish would double the latency).
+//  * lists of up to 1024 entries (one block per warp with clusters of 8): the one-stage kernel, two CTAs per
+//    SM, with the larger cluster, 8 or 4 CTAs per unit, of which `units` are resident at once;
+//  * longer lists: the two-stage kernel (one CTA per SM, clusters of 8) while `units` of its clusters are
+//    resident at once, else, up to kFusedOneStageMaxK entries, the one-stage kernel as above (its warps then
+//    take their blocks one after the other).
+// Clusters of 2 work as well (the kernel is written for them) but lose to the three-kernel path at the batch
+// sizes they would serve (45.7 against 41.3 us at 128 units), so they are not offered.
 template <int G>
 static int fused_variant(long long units, int k_max, int *stages) {
-    if (k_max <= kFusedOneStageMaxK) {
-        *stages = 1;
-        if (units <= fused_prepare<G, 1, 8>()) return 8;
-        if (units <= fused_prepare<G, 1, 4>()) return 4;
-        return 0;
+    const bool one_block_per_warp = k_max <= kFusedMaxCS * kFusedWarps * kBlockTokens;
+    if (!one_block_per_warp && units <= fused_prepare<G, 2, 8>()) {
+        *stages = 2;
+        return 8;
     }
-    *stages = 2;
-    return units <= fused_prepare<G, 2, 8>() ? 8 : 0;
+    *stages = 1;
+    if (k_max > kFusedOneStageMaxK) return 0;
+    if (units <= fused_prepare<G, 1, 8>()) return 8;
+    if (units <= fused_prepare<G, 1, 4>()) return 4;
+    return 0;
 }
 
 bool fused_step_eligible(int B, int Hq, int Hkv, int max_seq_len, int k_max) {

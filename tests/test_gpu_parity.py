@@ -623,7 +623,11 @@ def test_sparse_decode_step_random_configs(seed):
                sparsity=16), 3),
     # 6 units, budgets above 2048 rows: one fused launch of the two-stage variant, several blocks per warp
     (wl.Config("fused-large-k", 81, 3, [9000, 5000, 12001], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=2), 1),
-    # 20 units with budgets above 2048 rows: more clusters than the two-stage variant holds at once
+    # 20 units with budgets of 1500 rows: more clusters than the two-stage variant holds at once, so the
+    # one-stage variant takes them, two blocks per warp one after the other
+    (wl.Config("fused-20-units-1500", 86, 10, [6000 + 7 * i for i in range(10)], None, 0.02, n_q_heads=8, n_kv_heads=2,
+               sparsity=4), 1),
+    # 20 units with budgets above 2048 rows: three kernels
     (wl.Config("split-large-k", 82, 10, [6000 + 7 * i for i in range(10)], None, 0.02, n_q_heads=8, n_kv_heads=2,
                sparsity=2), 3),
 ])
