@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 
 METRIC = "sparse_decode_attn_us_per_layer_step"
 UNIT = "us"
-FUSED_KERNEL_TRAFFIC_C2 = 6543000   # dram__bytes_read.sum + write per launch, profiles/launch_list_bench_c2.md
+FUSED_KERNEL_TRAFFIC_C2 = 6552000   # dram__bytes_read.sum + write per launch, profiles/launch_list_bench_c2.md
 WORKLOAD = "c2: B=1, Hq=32, Hkv=8, d=128, ctx=32768, k=1024 (32x), 1% planted keys"
 
 
