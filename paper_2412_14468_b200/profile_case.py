@@ -56,6 +56,7 @@ def score_only(args):
     idx = torch.zeros(B, Hkv, k, dtype=torch.int32, device=dev)
     cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
     flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    last_slot = (w["seq_lens"] - 1).to(torch.int32)   # where the appended key's signature goes
     torch.cuda.synchronize()
     for s in range(args.steps):
         _ = int(flush.sum())
@@ -76,6 +77,9 @@ def main():
     ap.add_argument("--dense", action="store_true", help="also run the dense comparator each step")
     ap.add_argument("--prefill", action="store_true",
                     help="prompt ENCODE alone (tcgen05 and mma.sync kernels) on --batch sequences of the config's length")
+    ap.add_argument("--entry-points", action="store_true",
+                    help="run the step as its separate entry points (ha_encode, ha_score_topk, ha_gather_attn), i.e. the "
+                         "kernels of the three-kernel path, also at batch sizes where ha_sparse_decode is one fused launch")
     ap.add_argument("--score-only", action="store_true",
                     help="SCORE + TOPK alone on random signatures (no K/V allocated: large batches stay small)")
     args = ap.parse_args()
@@ -100,13 +104,20 @@ def main():
     cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
     out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=dev)
     flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    last_slot = (w["seq_lens"] - 1).to(torch.int32)   # where the appended key's signature goes
     torch.cuda.synchronize()
     for s in range(args.steps):
         _ = int(flush.sum())                       # read 256 MB: evicts L2 and leaves only clean lines
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
-                            w["n_cap"], w["k_max"], qc, idx, cnt, out, ws)
+        if args.entry_points:
+            ha.ha_encode(mq, Hq // Hkv, w["q"], qc.view(B, Hq, 1))
+            ha.ha_encode(mk, 1, w["k_new"], kc, slot=last_slot)
+            ha.ha_score_topk(shape, qc, kc, w["seq_lens"], w["k_per_seq"], 0, w["n_cap"], w["k_max"], idx, cnt, ws)
+            ha.ha_gather_attn(shape, w["q"], w["K"], w["V"], w["seq_lens"], idx, cnt, w["k_max"], out, ws)
+        else:
+            ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
+                                w["n_cap"], w["k_max"], qc, idx, cnt, out, ws)
         e1.record()
         if args.dense:
             ha.ha_dense_decode(shape, w["q"], w["K"], w["V"], w["seq_lens"], w["n_cap"], out, ws)
