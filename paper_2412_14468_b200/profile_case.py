@@ -56,7 +56,6 @@ def score_only(args):
     idx = torch.zeros(B, Hkv, k, dtype=torch.int32, device=dev)
     cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
     flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
-    last_slot = (w["seq_lens"] - 1).to(torch.int32)   # where the appended key's signature goes
     torch.cuda.synchronize()
     for s in range(args.steps):
         _ = int(flush.sum())
