@@ -1,25 +1,27 @@
 // The whole layer-step in ONE launch, for small batches (as many (sequence, KV head) units as clusters
-// are resident at once: 33 when the budget is at most 1024 rows, 15 beyond, on a 148-SM device) and
-// sequences of up to 32768 tokens: ENCODE -> SCORE -> TOPK -> GATHER-ATT (Section 4 recipe,
-// Section 4.1 "Implementation") with one thread-block cluster of 8 CTAs per unit, so that a small-batch
-// decode step has no kernel boundary or global-memory hand-off on its critical path:
+// are resident at once: on a 148-SM device 33 clusters of 8 CTAs or 71 of 4 with index lists of up to 1024
+// entries, 15 clusters of 8 with longer lists) and sequences of up to 32768 tokens: ENCODE -> SCORE -> TOPK
+// -> GATHER-ATT (Section 4 recipe, Section 4.1 "Implementation") with one thread-block cluster of CS
+// CTAs per unit, so that a small-batch decode step has no kernel boundary or global-memory hand-off on
+// its critical path:
 //
 //   P0  every CTA requests its slice of the signature cache; the encoding CTAs of the cluster fetch the
 //       query-side / key-side mapping weights and store them transposed in shared memory; all of it
 //       before the programmatic-launch wait, i.e. behind the preceding kernel.
-//   P1  CTA r < G (r < G/2 for G = 8) encodes one (two) query vectors, the next CTA the appended key
-//       (fp32 fma chains, Eq. 2, one chain per thread); cluster barrier; everybody reads the signatures
-//       through distributed shared memory.
-//   P2  scores as bytes in registers, per-CTA histogram, cluster barrier, histogram exchange through
-//       distributed shared memory, threshold, compaction of the CTA's slice into the index list;
-//       cluster barrier (the list is now visible to the whole cluster).
-//   P3  each CTA takes an eighth of the list: rows fetched with 16-byte cp.async into per-warp
-//       shared-memory stages, QK^T and PV on the tensor cores, online softmax; the eight CTA states
+//   P1  the first CTAs of the cluster encode the G query vectors (one per CTA when the cluster has room,
+//       else 2 or 4), the next CTA the appended key (fp32 fma chains, Eq. 2, one chain per thread); the
+//       signatures are stored into every CTA's shared memory (DSMEM); cluster barrier.
+//   P2  scores as bytes in registers, per-CTA histogram stored into every CTA's table, cluster barrier,
+//       threshold (every warp for itself), compaction of the CTA's slice; the parts of the index list
+//       are stored into the shared memory of the CTAs that will attend to them (one-stage variant) or
+//       into global memory; cluster barrier.
+//   P3  each CTA takes a 1/CS of the list: rows fetched with 16-byte cp.async into per-warp
+//       shared-memory stages, QK^T and PV on the tensor cores, online softmax; the CTA states
 //       are written into CTA 0's shared memory (DSMEM stores), cluster barrier, CTA 0 merges,
 //       normalises and rounds once to bf16.
-// Every cross-CTA hand-off is a hardware cluster barrier (no flag, no spin).  Results are bit-identical
-// to the multi-kernel path for signatures, counts and index lists; attention outputs agree within
-// the usual fp32 reordering.
+// Every cross-CTA hand-off is a push followed by a hardware cluster barrier (no flag, no spin, no remote
+// read).  Results are bit-identical to the multi-kernel path for signatures, counts and index lists;
+// attention outputs agree within the usual fp32 reordering.
 #include "ha_attn_dev.cuh"
 #include "ha_encode_dev.cuh"
 #include "ha_score_dev.cuh"
@@ -38,7 +40,7 @@ constexpr int kFusedListOffset = kFusedWarps * kStageBytes;  // one-stage varian
 __host__ __device__ constexpr int fused_q_per_cta(int G, int CS) {
     return (G <= CS - 1) ? 1 : (G / 2 <= CS - 1) ? 2 : (G / 4 <= CS - 1) ? 4 : 8;
 }
-// Dynamic shared memory of a CTA: [weights | S row stages per warp] union, activations, the eight CTA states
+// Dynamic shared memory of a CTA: [weights | S row stages per warp] union, activations, the CS CTA states
 // of the G heads (used in CTA 0).  With S = 1 two CTAs fit one SM (and the kernel is compiled for 128
 // registers): two consecutive steps are then resident together, each cluster of the later one already
 // parked at its launch wait, whereas only 15 clusters of eight one-CTA SMs exist on the device.
@@ -152,7 +154,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     float *part_acc = part_ml + CS * G * 2;                                   // [CS][G][128]
     __shared__ uint32_t s_codes[kMaxGroup + 1];   // the G query signatures and the appended key's, pushed by the encoding CTAs
     __shared__ uint32_t s_hist[kBins + 3];   // this CTA's histogram
-    __shared__ int s_all[kFusedMaxCS][kBins + 3];   // the eight CTAs' histograms, each pushed by its owner
+    __shared__ int s_all[kFusedMaxCS][kBins + 3];   // the histograms of the cluster's CTAs, each pushed by its owner
     __shared__ __align__(16) uint32_t c_hist[kBins][32];   // one counter per (level, lane), shared by the warps
     __shared__ int s_wcnt[kFusedWarps];
     __shared__ float s_m[kFusedWarps][8], s_l[kFusedWarps][8];
@@ -220,7 +222,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     pdl_launch_dependents();
     cluster_wait();              // #0: all CTAs of the cluster are running (their shared memory may be written)
 
-    // ---------------- P1: ENCODE in CTA 0 (queries) and CTA 1 (appended key)
+    // ---------------- P1: ENCODE in the first kQCtas CTAs (queries) and the next one (appended key)
     if (enc_q) {
         fused_encode<kQPer, CS>(a.q + (head0 + kQPer * (int)rank) * kD, kD, sw1, sw2, sw3, actA, actB,
                             s_codes + kQPer * (int)rank, bias1, bias2, bias3);
@@ -396,7 +398,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         }
     }
 
-    // ---------------- P3: GATHER-ATT over this CTA's eighth of the list
+    // ---------------- P3: GATHER-ATT over this CTA's share of the list
     const bool paged = a.block_table != nullptr;   // rows are then addressed from the pool's base
     const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (paged ? 0LL : (long long)b * a.K.sb) + (long long)kvh * a.K.sh);
     const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (paged ? 0LL : (long long)b * a.V.sb) + (long long)kvh * a.V.sh);
@@ -415,7 +417,8 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         for (int e = 0; e < 4; ++e) acc[mt][e] = 0.0f;
     float m_run = -CUDART_INF_F, l_run = 0.0f;
     {
-        // this warp's blocks: blk_lo + warp, + 8, ...; list entries come from peer CTAs: read them from L2
+        // this warp's blocks: blk_lo + warp, + 8, ...; list entries were selected by peer CTAs: they sit in this
+        // CTA's shared memory (one-stage variant) or are read from L2
         const int nblk = (blk_lo + warp < blk_hi) ? (blk_hi - blk_lo - warp + kFusedWarps - 1) / kFusedWarps : 0;
         auto token_of_block = [&](int i) -> int {
             const int p = (blk_lo + warp + i * kFusedWarps) * kBlockTokens + (lane & 15);
