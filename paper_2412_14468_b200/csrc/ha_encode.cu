@@ -14,9 +14,9 @@ namespace ha {
 // The vectors of one network (the queries of a KV head over the whole batch, or the appended keys)
 // are cut into items of NV vectors.  A CTA belongs to one network, fetches its 72 KB of weights
 // once and encodes the items part, part + P, ... of that network.  A step of few vectors uses
-// NV = 1 and one item per CTA (the chains of different vectors run on different SMs); a large batch
-// uses items of up to 8 vectors and, beyond two waves of CTAs, several items per CTA, so that the
-// weight traffic does not grow with the number of vectors.
+// NV = 1 and one item per CTA (the chains of different vectors run on different SMs); a larger one
+// as many vectors per CTA as it takes for all CTAs to be resident at once, in items of up to 8
+// vectors (launch_encode_vectors), so that neither a second wave nor the weight traffic grows the latency.
 // One thread requests the three weight matrices with bulk asynchronous copies (TMA, one mbarrier
 // per matrix) at kernel entry, before the programmatic-launch wait: the fetch overlaps the
 // preceding kernels and costs no issue slots; each layer starts as soon as its matrix has landed.
