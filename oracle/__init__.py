@@ -75,6 +75,26 @@ def score(qcodes, kcodes) -> np.ndarray:
     return out
 
 
+def score_wide(qcode, kcodes) -> np.ndarray:
+    """Score of the SCORE-latency table: b - Hamming for signatures of b = 64 * W bits, kcodes uint64 [n, W]."""
+    qcode = np.ascontiguousarray(qcode, dtype=np.uint64).reshape(-1)
+    kcodes = np.ascontiguousarray(kcodes, dtype=np.uint64)
+    assert kcodes.ndim == 2 and kcodes.shape[1] == qcode.shape[0]
+    out = np.zeros(kcodes.shape[0], dtype=np.int32)
+    lib().ora_score_wide(_p(qcode), _p(kcodes), C.c_int64(kcodes.shape[0]), C.c_int32(qcode.shape[0]), _p(out))
+    return out
+
+
+def inner_products(q, K) -> np.ndarray:
+    """<q, K_i> for bf16 bit patterns q [128], K [n, 128]; float64 accumulation."""
+    q = _u16(q).reshape(-1)
+    K = _u16(K)
+    assert q.shape[0] == D and K.ndim == 2 and K.shape[1] == D
+    out = np.zeros(K.shape[0], dtype=np.float64)
+    lib().ora_inner_products(_p(q), _p(K), C.c_int64(K.shape[0]), C.c_int64(D), _p(out))
+    return out
+
+
 def topk(scores, k: int) -> np.ndarray:
     """Standard top-k with ties to the lowest token index; indices returned ascending."""
     scores = np.ascontiguousarray(scores, dtype=np.int32).reshape(-1)

@@ -17,6 +17,12 @@
  *                    (Section 4.1), reported as 32 - Hamming distance; for grouped-query
  *                    attention the group score is the maximum over the query heads that
  *                    share the KV head (reduces to Eq. 1 when the group has one head).
+ *   ora_score_wide   the same score for a signature of b = 64 .. 512 bits kept as b/64 packed
+ *                    64-bit integers (the setting of the SCORE-latency table, "Latency of
+ *                    SCORE computation"): b - Hamming distance, one query signature against n
+ *                    key signatures, counted bit by bit.
+ *   ora_inner_products  the comparator column of that table: the inner product of one query
+ *                    with each of n keys of 128 16-bit floats (bf16 here), in float64.
  *   ora_topk         "the standard top-k on these scores" (Section 4): sort by
  *                    (score descending, token index ascending), keep min(k, n).
  *   ora_topk_windows the selection used for every method in the experiments (Section 5,
@@ -32,7 +38,8 @@
  *
  * Pins (tests/test_oracle_*.py): closed forms (identity / zero weights, single token,
  * zero query), hand-derived fixtures in tests/golden/, an O(n^2) rank definition of
- * top-k, bit-level brute force for the score, float64 numpy for the mapping net, and
+ * top-k, bit-level brute force for the score, the +-1 inner-product identity and the 32-bit
+ * score for the wide score, float64 numpy for the mapping net and the inner products, and
  * torch's scaled_dot_product_attention in float64 for the attention.
  * The fp32 accumulation ORDER inside ora_encode is a definition of this build, not of
  * the paper: it is pinned only up to the float64 margin test ("parity unpinned" for
@@ -147,6 +154,28 @@ void ora_score(const uint32_t *qcodes, int32_t group, const uint32_t *kcodes, in
             if (s > best) best = s;
         }
         scores[i] = best;
+    }
+}
+
+/* scores[i] = n_bits - Hamming(k_i, q) for signatures of n_words packed 64-bit integers
+ * (n_bits = 64 n_words; bit j of the signature is bit j % 64 of word j / 64).  Counted one
+ * bit at a time: a score is the number of positions in which the two signatures agree. */
+void ora_score_wide(const uint64_t *qcode, const uint64_t *kcodes, int64_t n, int32_t n_words, int32_t *scores) {
+    for (int64_t i = 0; i < n; ++i) {
+        int agree = 0;
+        for (int w = 0; w < n_words; ++w)
+            for (int bit = 0; bit < 64; ++bit)
+                agree += (int)(((kcodes[i * n_words + w] >> bit) & 1u) == ((qcode[w] >> bit) & 1u));
+        scores[i] = agree;
+    }
+}
+
+/* dots[i] = <q, K_i> over 128 bf16 components, accumulated in float64 (the comparator of the table). */
+void ora_inner_products(const uint16_t *q, const uint16_t *K, int64_t n, int64_t row_stride, double *dots) {
+    for (int64_t i = 0; i < n; ++i) {
+        double acc = 0.0;
+        for (int d = 0; d < HA_D; ++d) acc += (double)bf16_to_f32(q[d]) * (double)bf16_to_f32(K[i * row_stride + d]);
+        dots[i] = acc;
     }
 }
 
