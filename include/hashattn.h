@@ -261,6 +261,29 @@ int ha_gather_attn_static(const ha_shape *shape, const uint16_t *q, const ha_ten
                           int64_t idx_stride_b, int64_t idx_stride_h, const int32_t *count,
                           int32_t k_max, uint16_t *out, float *lse, void *stream);
 
+/* SCORE for wide signatures (Section "Latency of SCORE computation" and its table: Hamming distance on
+ * packed 64-bit integers, 64 to 512 bits per token; Eq. 1 with the bitcount identity of Section 4.1 at
+ * b bits).  scores[i] = n_bits - popcount(k_codes[i] xor q_code), 0 <= i < n.
+ *   q_code   device, n_bits / 64 words; bit j of a signature is bit j % 64 of word j / 64.
+ *   k_codes  device, [n][n_bits / 64] words, contiguous, 16-byte aligned.
+ *   scores   device, n 16-bit values, 4-byte aligned; written by the call, owned by the caller.
+ * n_bits must be 64, 128, 256 or 512 (HA_ERR_UNSUPPORTED otherwise); n = 0 returns HA_OK without a
+ * launch; null or misaligned pointers and n < 0 give HA_ERR_INVALID_ARG.  One query, no group
+ * reduction, no selection: this is the stand-alone scoring pass that the paper times against the
+ * inner product, not a step of ha_sparse_decode (whose signatures have 32 bits). */
+int ha_score_wide(const uint64_t *q_code, const uint64_t *k_codes, int64_t n, int32_t n_bits,
+                  uint16_t *scores, void *stream);
+
+/* The comparator column of the same table: dots[i] = <q, K[i]> for one query and n keys of 128 bf16
+ * components ("128 x 16Float"), fp32 accumulation.
+ *   q     device, 128 bf16 values, 16-byte aligned.
+ *   K     device, row i at K + i * row_stride (elements); row_stride >= 128 and a multiple of 8,
+ *         base 16-byte aligned.
+ *   dots  device, n fp32 values.
+ * Errors as for ha_score_wide. */
+int ha_inner_products(const uint16_t *q, const uint16_t *K, int64_t n, int64_t row_stride, float *dots,
+                      void *stream);
+
 /* Copies the device status word to *flags (host) and clears nothing; synchronises `stream`. */
 int ha_read_device_status(void *workspace, void *stream, uint32_t *flags);
 

@@ -24,6 +24,7 @@ EXPORTS = [
     "ha_workspace_bytes", "ha_workspace_init", "ha_encode", "ha_encode_prefill", "ha_score_topk", "ha_gather_attn",
     "ha_gather_attn_paged", "ha_sparse_decode_paged",
     "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
+    "ha_score_wide", "ha_inner_products",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
 
@@ -78,12 +79,15 @@ def lib() -> C.CDLL:
         L.ha_sparse_decode_host.argtypes = [P, P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64,
                                             P, P, P, SZ, P]
         L.ha_read_device_status.argtypes = [P, P, P]
+        L.ha_score_wide.argtypes = [P, P, I64, I32, P, P]
+        L.ha_inner_products.argtypes = [P, P, I64, I64, P, P]
         L.ha_kernel_launches.restype = C.c_uint64
         L.ha_status_string.restype = C.c_char_p
         L.ha_status_string.argtypes = [C.c_int]
         L.ha_version.restype = C.c_char_p
         for fn in ("ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn", "ha_gather_attn_static", "ha_dense_decode",
-                   "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status"):
+                   "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status", "ha_score_wide",
+                   "ha_inner_products"):
             getattr(L, fn).restype = C.c_int
         _lib = L
     return _lib
@@ -95,6 +99,24 @@ def status_string(status: int) -> str:
 
 def ha_version() -> str:
     return lib().ha_version().decode()
+
+
+def ha_score_wide(q_code: torch.Tensor, k_codes: torch.Tensor, n_bits: int, scores: torch.Tensor, stream=None) -> None:
+    """q_code int64 [n_bits/64]; k_codes int64 [n, n_bits/64] (the 64-bit words of the signatures); scores int16 [n]."""
+    _dev(q_code, torch.int64, "q_code"); _dev(k_codes, torch.int64, "k_codes"); _dev(scores, torch.int16, "scores")
+    assert k_codes.is_contiguous() and q_code.is_contiguous() and scores.is_contiguous()
+    n = k_codes.shape[0]
+    assert k_codes.dim() == 2 and k_codes.shape[1] * 64 == n_bits == q_code.numel() * 64 and scores.numel() == n
+    _check("ha_score_wide", lib().ha_score_wide(q_code.data_ptr(), k_codes.data_ptr(), n, n_bits, scores.data_ptr(),
+                                                _stream(stream)))
+
+
+def ha_inner_products(q: torch.Tensor, K: torch.Tensor, dots: torch.Tensor, stream=None) -> None:
+    """q bf16 [128]; K bf16 [n, 128] (row stride a multiple of 8 elements); dots fp32 [n]."""
+    _dev(q, torch.bfloat16, "q"); _dev(K, torch.bfloat16, "K"); _dev(dots, torch.float32, "dots")
+    assert K.dim() == 2 and K.shape[1] == 128 and K.stride(1) == 1 and q.numel() == 128 and dots.numel() == K.shape[0]
+    _check("ha_inner_products", lib().ha_inner_products(q.data_ptr(), K.data_ptr(), K.shape[0], K.stride(0), dots.data_ptr(),
+                                                        _stream(stream)))
 
 
 def ha_kernel_launches() -> int:

@@ -373,6 +373,25 @@ int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const 
     return HA_OK;
 }
 
+int ha_score_wide(const uint64_t *q_code, const uint64_t *k_codes, int64_t n, int32_t n_bits, uint16_t *scores,
+                  void *stream) {
+    if (n < 0 || !q_code || (n > 0 && (!k_codes || !scores))) return HA_ERR_INVALID_ARG;
+    if (n_bits != 64 && n_bits != 128 && n_bits != 256 && n_bits != 512) return HA_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(k_codes) & 15) || (reinterpret_cast<uintptr_t>(scores) & 3) ||
+        (reinterpret_cast<uintptr_t>(q_code) & 7))
+        return HA_ERR_INVALID_ARG;
+    HA_CUDA(launch_score_wide(q_code, k_codes, n, n_bits / 64, scores, (cudaStream_t)stream));
+    return HA_OK;
+}
+
+int ha_inner_products(const uint16_t *q, const uint16_t *K, int64_t n, int64_t row_stride, float *dots, void *stream) {
+    if (n < 0 || !q || (n > 0 && (!K || !dots)) || row_stride < kD || (row_stride & 7)) return HA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(K) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(dots) & 3))
+        return HA_ERR_INVALID_ARG;
+    HA_CUDA(launch_inner_products(q, K, n, row_stride, dots, (cudaStream_t)stream));
+    return HA_OK;
+}
+
 int ha_read_device_status(void *workspace, void *stream, uint32_t *flags) {
     if (!workspace || !flags) return HA_ERR_INVALID_ARG;
     HA_CUDA(cudaMemcpyAsync(flags, workspace, sizeof(uint32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream));

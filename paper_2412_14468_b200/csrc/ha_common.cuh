@@ -200,6 +200,11 @@ cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapV
                               cudaStream_t st, Windows win = Windows{0, 0}, const int32_t *block_table = nullptr,
                               long long bt_sb = 0, int page_shift = 0);
 
+cudaError_t launch_score_wide(const uint64_t *q_code, const uint64_t *k_codes, long long n, int n_words, uint16_t *scores,
+                              cudaStream_t st);
+cudaError_t launch_inner_products(const uint16_t *q, const uint16_t *K, long long n, long long row_stride, float *dots,
+                                  cudaStream_t st);
+
 cudaError_t launch_append_kv(int B, int Hq, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
                              TensorView V, const int32_t *seq_lens, const uint16_t *q_src, uint16_t *q_dst,
                              uint16_t *k_dst, cudaStream_t st);

@@ -119,6 +119,20 @@ def test_windows_and_prefill_arguments_are_checked_on_the_host(lib):
     assert lib.ha_encode_prefill(C.byref(m), 1, C.byref(t), 1, 8, 0, fake, 64, 64, ha.HA_PREFILL_TCGEN05, None, None) == ha.HA_OK
 
 
+def test_wide_score_and_inner_product_arguments_are_checked_on_the_host(lib):
+    fake = 0x1000
+    assert lib.ha_score_wide(fake, fake, 100, 96, fake, None) == ha.HA_ERR_UNSUPPORTED        # width not 64/128/256/512
+    assert lib.ha_score_wide(fake, fake, -1, 64, fake, None) == ha.HA_ERR_INVALID_ARG
+    assert lib.ha_score_wide(fake, fake + 8, 100, 128, fake, None) == ha.HA_ERR_INVALID_ARG   # signatures not 16-byte aligned
+    assert lib.ha_score_wide(fake, fake, 100, 64, fake + 2, None) == ha.HA_ERR_INVALID_ARG    # scores not 4-byte aligned
+    assert lib.ha_score_wide(None, fake, 100, 64, fake, None) == ha.HA_ERR_INVALID_ARG
+    assert lib.ha_score_wide(fake, None, 0, 512, None, None) == ha.HA_OK                      # empty: no launch
+    assert lib.ha_inner_products(fake, fake, 10, 100, fake, None) == ha.HA_ERR_INVALID_ARG    # rows shorter than 128
+    assert lib.ha_inner_products(fake, fake, 10, 132, fake, None) == ha.HA_ERR_INVALID_ARG    # row stride not a multiple of 8
+    assert lib.ha_inner_products(fake, fake + 4, 10, 128, fake, None) == ha.HA_ERR_INVALID_ARG
+    assert lib.ha_inner_products(fake, None, 0, 128, None, None) == ha.HA_OK
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(ha, "_lib", None)
     monkeypatch.setattr(ha, "LIB_PATH", str(tmp_path / "nope.so"))

@@ -701,3 +701,47 @@ def test_step_edge_cases_empty_sequence_budget_above_length_and_no_new_key(reps)
         fin = np.isfinite(ref["lse"])
         assert np.array_equal(np.isneginf(got), ~fin) and np.max(np.abs(got[fin] - ref["lse"][fin]), initial=0.0) < 1e-3
         assert not u16(out)[0::4].any() and not u16(out)[3::4].any()          # empty selections give zeros
+
+
+# ---------------------------------------------------------------- wide signatures (SCORE-latency table)
+
+def _wide_codes(rng, n, W):
+    return rng.integers(0, 2**63, size=(n, W), dtype=np.uint64) * np.uint64(2) + rng.integers(0, 2, size=(n, W), dtype=np.uint64)
+
+
+@pytest.mark.parametrize("n_bits", [64, 128, 256, 512])
+@pytest.mark.parametrize("n", [1, 2, 3, 1000, 100003, 1 << 20])
+def test_score_wide_is_bit_exact(n_bits, n):
+    """Every score of the stand-alone wide-signature pass equals the oracle's bit-by-bit count: single tokens,
+    odd counts (the 64-bit case packs two tokens per load), several CTA iterations and a ragged tail."""
+    W = n_bits // 64
+    rng = np.random.default_rng(9000 + n_bits + n % 97)
+    q, k = _wide_codes(rng, 1, W)[0], _wide_codes(rng, n, W)
+    if n >= 3:
+        k[0] = q          # a full match and a complement among the tokens
+        k[2] = ~q
+    dq = torch.from_numpy(q.view(np.int64)).to(DEV)
+    dk = torch.from_numpy(k.view(np.int64)).to(DEV)
+    out = torch.full((n + 3,), -7, dtype=torch.int16, device=DEV)
+    ha.ha_score_wide(dq, dk, n_bits, out[:n])
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    assert np.array_equal(got[:n].astype(np.int32), oracle.score_wide(q, k))
+    assert np.all(got[n:] == -7)                       # nothing written past the last token
+    if n >= 3:
+        assert got[0] == n_bits and got[2] == 0
+
+
+@pytest.mark.parametrize("n,stride", [(1, 128), (77, 128), (5000, 136), (200003, 128)])
+def test_inner_products_match_the_oracle(n, stride):
+    g = torch.Generator(DEV).manual_seed(n)
+    K = torch.randn(n, stride, device=DEV, generator=g).to(torch.bfloat16)[:, :128]
+    q = torch.randn(128, device=DEV, generator=g).to(torch.bfloat16)
+    dots = torch.full((n + 1,), 123.0, device=DEV)
+    ha.ha_inner_products(q, K, dots[:n])
+    torch.cuda.synchronize()
+    ref = oracle.inner_products(u16(q), u16(K.contiguous()))
+    got = dots.cpu().numpy().astype(np.float64)
+    # 128 products of magnitude ~1 accumulated in fp32: error far below 1e-3
+    assert np.max(np.abs(got[:n] - ref)) < 1e-3
+    assert got[n] == 123.0
