@@ -480,6 +480,55 @@ def main():
         except Exception as ex:
             supplementary["c2_sink128_local128"] = {"error": repr(ex)[:200]}
 
+        try:   # the paper's table "Latency of SCORE computation": one query against n tokens, signatures of 64 .. 512 bits
+            #      (packed 64-bit words) against the inner product with keys of 128 16-bit floats; every timed launch is
+            #      L2-cold (a 256 MB buffer is rewritten in front of it)
+            paper_ms = {262144: (0.13, 0.085, 0.084, 0.087, 0.112), 2097152: (1.698, 0.144, 0.247, 0.445, 0.85),
+                        33554432: (16.61, 2.188, 3.817, 7.005, 13.48)}   # inner product, 64, 128, 256, 512 bit (hardware not stated)
+            flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+
+            def cold_us(fn, iters=7):
+                ts = []
+                for _ in range(iters + 2):
+                    flush.fill_(1)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    fn()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ts.append(e0.elapsed_time(e1) * 1e3)
+                return float(sorted(ts[2:])[len(ts[2:]) // 2])
+
+            table = {}
+            gs = torch.Generator(device).manual_seed(wl.BASE_SEED + 77)
+            for n_tok, pm in paper_ms.items():
+                row = {}
+                Kd = torch.randn(n_tok, 128, device=device, generator=gs, dtype=torch.float32).to(torch.bfloat16) \
+                    if n_tok <= (1 << 21) else torch.empty(n_tok, 128, device=device, dtype=torch.bfloat16).normal_(generator=gs)
+                qd = torch.randn(128, device=device, generator=gs).to(torch.bfloat16)
+                dots = torch.empty(n_tok, device=device)
+                us = cold_us(lambda: ha.ha_inner_products(qd, Kd, dots))
+                row["inner_product_128xbf16"] = {"us": us, "gbs": n_tok * 260 / us / 1e3, "frac": n_tok * 260 / us / 1e3 / peak,
+                                                 "paper_ms": pm[0]}
+                del Kd, dots
+                for j, bits in enumerate((64, 128, 256, 512)):
+                    W = bits // 64
+                    kc = torch.randint(-2**63, 2**63 - 1, (n_tok, W), dtype=torch.int64, device=device, generator=gs)
+                    qc = torch.randint(-2**63, 2**63 - 1, (W,), dtype=torch.int64, device=device, generator=gs)
+                    sc = torch.empty(n_tok, dtype=torch.int16, device=device)
+                    us = cold_us(lambda: ha.ha_score_wide(qc, kc, bits, sc))
+                    nbytes = n_tok * (8 * W + 2)
+                    row[f"hamming_{bits}bit"] = {"us": us, "gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak,
+                                                 "paper_ms": pm[1 + j]}
+                    del kc, sc
+                table[f"{n_tok}_tokens"] = row
+                torch.cuda.empty_cache()
+            supplementary["score_latency_table"] = table
+            del flush
+            torch.cuda.empty_cache()
+        except Exception as ex:
+            supplementary["score_latency_table"] = {"error": repr(ex)[:200]}
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         us, threads, sample = oracle_time("c2", 200, budget_s=15.0)

@@ -16,7 +16,7 @@ constexpr int kWideLoads = 4;   // 16-byte loads in flight per thread
 
 // W = 64-bit words per signature (1, 2, 4, 8).  n16 = number of whole 16-byte pieces of the key array.
 template <int W>
-__global__ void __launch_bounds__(kWideThreads) score_wide_kernel(const uint64_t *__restrict__ q_code,
+__global__ void __launch_bounds__(kWideThreads, (W == 2 || W == 4) ? 8 : 1) score_wide_kernel(const uint64_t *__restrict__ q_code,
                                                                  const uint64_t *__restrict__ k_codes, long long n,
                                                                  uint16_t *__restrict__ scores) {
     constexpr int kLanesPerToken = (W >= 2) ? W / 2 : 1;   // 16-byte pieces per token
@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(kWideThreads) score_wide_kernel(const uint64_t
 }
 
 // dots[i] = <q, K_i>, 128 bf16 components, fp32 accumulation: 16 lanes per row (eight components each).
-__global__ void __launch_bounds__(kWideThreads) inner_product_kernel(const uint16_t *__restrict__ q,
+__global__ void __launch_bounds__(kWideThreads, 8) inner_product_kernel(const uint16_t *__restrict__ q,
                                                                     const uint16_t *__restrict__ K, long long n,
                                                                     long long row_stride, float *__restrict__ dots) {
     const int lane = threadIdx.x & 31, part = lane & 15;

@@ -68,6 +68,38 @@ def score_only(args):
     print("signature bytes per step:", B * Hkv * n * 4)
 
 
+def score_wide(args):
+    """The stand-alone wide-signature SCORE pass and its inner-product comparator on --tokens tokens."""
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    n = args.tokens
+    g = torch.Generator(dev).manual_seed(wl.BASE_SEED + 5)
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    K = torch.empty(n, 128, device=dev, dtype=torch.bfloat16).normal_(generator=g)
+    q = torch.randn(128, device=dev, generator=g).to(torch.bfloat16)
+    dots = torch.empty(n, device=dev)
+    cases = [("inner product", lambda: ha.ha_inner_products(q, K, dots), n * 260)]
+    keep = []
+    for bits in (64, 128, 256, 512):
+        W = bits // 64
+        kc = torch.randint(-2**63, 2**63 - 1, (n, W), dtype=torch.int64, device=dev, generator=g)
+        qc = torch.randint(-2**63, 2**63 - 1, (W,), dtype=torch.int64, device=dev, generator=g)
+        sc = torch.empty(n, dtype=torch.int16, device=dev)
+        keep.append((kc, qc, sc))
+        cases.append((f"{bits} bit", (lambda kc=kc, qc=qc, sc=sc, bits=bits: ha.ha_score_wide(qc, kc, bits, sc)), n * (8 * W + 2)))
+    torch.cuda.synchronize()
+    for s in range(args.steps):
+        for name, fn, nbytes in cases:
+            _ = int(flush.sum())
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3
+            print(f"step {s} {name:14s}: {us:9.1f} us  {nbytes / us / 1e3:8.1f} GB/s (plain launch, L2 flushed)")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="c3")
@@ -81,7 +113,12 @@ def main():
                          "kernels of the three-kernel path, also at batch sizes where ha_sparse_decode is one fused launch")
     ap.add_argument("--score-only", action="store_true",
                     help="SCORE + TOPK alone on random signatures (no K/V allocated: large batches stay small)")
+    ap.add_argument("--score-wide", action="store_true",
+                    help="stand-alone SCORE on signatures of 64..512 bits and the inner-product comparator on --tokens tokens")
+    ap.add_argument("--tokens", type=int, default=1 << 23)
     args = ap.parse_args()
+    if args.score_wide:
+        return score_wide(args)
     if args.score_only:
         return score_only(args)
     if args.prefill:
