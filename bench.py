@@ -11,7 +11,8 @@ enqueue kernels) so that host launch overhead does not hide the kernels.
 Prints ONE JSON line: `value` = microseconds per layer-step with the inputs resident in HBM, `e2e` the same
 step driven from pinned host buffers, `roofline` (algorithmic bytes of the step over its time, against the
 measured HBM peak), `breakdown_us` of the stand-alone entry points, `dense_same_run`, `supplementary`
-(larger batches, longer and ragged contexts, always-kept windows, the prompt encoders) and `cpu_baseline`
+(larger batches, longer and ragged contexts, always-kept windows, the prompt encoders, the SCORE latency
+against the signature width) and `cpu_baseline`
 (the oracle on the host cores).  `--impl reference` times the CPU oracle instead (the only reference this
 method has here).
 """
