@@ -123,11 +123,13 @@ class Replica:
         self.cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=device)
         self.out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=device)
         self.host = None
+        self.host_step = None
 
     def pin_host(self, torch):
         w = self.w
         self.host = tuple(w[x].cpu().pin_memory() for x in ("q", "k_new", "v_new")) + \
             (torch.zeros(tuple(self.out.shape), dtype=torch.bfloat16).pin_memory(),)
+        self.host_step = None
 
 
 class Bench:
@@ -153,10 +155,14 @@ class Bench:
                             0, w["n_cap"], w["k_max"], r.qc, r.idx, r.cnt, r.out, self.ws)
 
     def step_host(self, r):
-        ha, w = self.ha, r.w
-        hq, hk, hv, ho = r.host
-        ha.ha_sparse_decode_host(r.shape, r.mq, r.mk, hq, hk, hv, w["K"], w["V"], r.kc, w["seq_lens"], w["k_per_seq"],
-                                 0, w["n_cap"], w["k_max"], r.idx, r.cnt, ho, self.ws)
+        """One layer-step from pinned host buffers: a prepared ha_sparse_decode_host call (arguments marshalled
+        once per replica, as a decode loop that reuses its staging buffers would)."""
+        if r.host_step is None:
+            ha, w = self.ha, r.w
+            hq, hk, hv, ho = r.host
+            r.host_step = ha.SparseDecodeHostStep(r.shape, r.mq, r.mk, hq, hk, hv, w["K"], w["V"], r.kc, w["seq_lens"],
+                                                  w["k_per_seq"], 0, w["n_cap"], w["k_max"], r.idx, r.cnt, ho, self.ws)
+        r.host_step()
 
     def encode(self, r):
         ha, w = self.ha, r.w

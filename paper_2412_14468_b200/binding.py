@@ -322,6 +322,34 @@ def ha_sparse_decode_host(shape: ha_shape, map_q: Mapping, map_k: Mapping, q_hos
         count.data_ptr(), out_host.data_ptr(), p, n, _stream(stream)))
 
 
+class SparseDecodeHostStep:
+    """ha_sparse_decode_host with its arguments marshalled once: for a decode loop that reuses the same pinned
+    host buffers, device caches and workspace every step, calling the object costs one foreign call instead
+    of ~12 us of Python argument handling.  The tensors are kept alive by the object; their addresses, shapes
+    and strides must not change (write new q / k_new / v_new values INTO the host buffers)."""
+
+    def __init__(self, shape: ha_shape, map_q: Mapping, map_k: Mapping, q_host, k_new_host, v_new_host, K, V,
+                 k_codes, seq_lens, k_per_seq, k_uniform: int, max_seq_len: int, k_max: int, idx, count, out_host,
+                 workspace, stream=None):
+        for t in (q_host, k_new_host, v_new_host, out_host):
+            if t.is_cuda or not t.is_contiguous():
+                raise TypeError("host buffers must be contiguous CPU tensors")
+        p, n = _ws(workspace)
+        self._kt, self._vt = make_tensor(K), make_tensor(V)
+        self._keep = (shape, map_q, map_k, q_host, k_new_host, v_new_host, K, V, k_codes, seq_lens, k_per_seq, idx, count,
+                      out_host, workspace)
+        self._fn = lib().ha_sparse_decode_host
+        self._args = (C.byref(shape), map_q.ref, map_k.ref, q_host.data_ptr(), k_new_host.data_ptr(), v_new_host.data_ptr(),
+                      C.byref(self._kt), C.byref(self._vt), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1),
+                      seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform, max_seq_len, k_max, idx.data_ptr(), idx.stride(0),
+                      idx.stride(1), count.data_ptr(), out_host.data_ptr(), p, n, _stream(stream))
+
+    def __call__(self) -> None:
+        status = self._fn(*self._args)
+        if status != HA_OK:
+            raise HashAttnError("ha_sparse_decode_host", status)
+
+
 def ha_read_device_status(workspace, stream=None) -> int:
     flags = C.c_uint32(0)
     _check("ha_read_device_status", lib().ha_read_device_status(workspace.data_ptr(), _stream(stream), C.byref(flags)))

@@ -450,7 +450,7 @@ def test_gather_attn_over_a_paged_cache(page_size):
 
 # ---------------------------------------------------------------------------- whole step
 
-def _run_step(w, host=False, pinned=True, n_sink=0, n_local=0):
+def _run_step(w, host=False, pinned=True, n_sink=0, n_local=0, prepared=False):
     cfg = w["cfg"]
     B, Hq, Hkv = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads
     shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"], n_sink=n_sink, n_local=n_local)
@@ -477,8 +477,15 @@ def _run_step(w, host=False, pinned=True, n_sink=0, n_local=0):
         pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)     # pageable buffers take the staged-copy route
         hq, hk, hv = (pin(w[x].cpu()) for x in ("q", "k_new", "v_new"))
         ho = pin(torch.zeros(B, Hq, 128, dtype=torch.bfloat16))
-        ha.ha_sparse_decode_host(shape, mq, mk, hq, hk, hv, K2, V2, kc, w["seq_lens"], w["k_per_seq"], 0, w["n_cap"],
-                                 w["k_max"], idx, cnt, ho, ws)
+        if prepared:
+            step = ha.SparseDecodeHostStep(shape, mq, mk, hq, hk, hv, K2, V2, kc, w["seq_lens"], w["k_per_seq"], 0,
+                                           w["n_cap"], w["k_max"], idx, cnt, ho, ws)
+            step()
+            ho.zero_()
+            step()                                                   # the second call sees the same inputs
+        else:
+            ha.ha_sparse_decode_host(shape, mq, mk, hq, hk, hv, K2, V2, kc, w["seq_lens"], w["k_per_seq"], 0, w["n_cap"],
+                                     w["k_max"], idx, cnt, ho, ws)
         assert torch.equal(K2, w["K"]) and torch.equal(V2, w["V"])   # the new rows were appended in place
         out = ho.to(DEV)
         lse = None
@@ -518,6 +525,9 @@ def test_sparse_decode_step_matches_oracle(cfg):
     for pinned in (True, False):
         rh = _run_step(w, host=True, pinned=pinned)
         assert torch.equal(rh["idx"], r["idx"]) and torch.equal(rh["out"], r["out"])
+    # ... and so does the same call with its arguments marshalled once (SparseDecodeHostStep), run twice
+    rp = _run_step(w, host=True, pinned=True, prepared=True)
+    assert torch.equal(rp["idx"], r["idx"]) and torch.equal(rp["out"], r["out"])
 
 
 @pytest.mark.parametrize("cfg", [
