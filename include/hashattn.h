@@ -222,8 +222,12 @@ int ha_sparse_decode_paged(const ha_shape *shape, const ha_mapping *map_q, const
  * query, key and value vectors; Section 4.1): copies q_host, k_new_host, v_new_host to the device
  * (staging inside the workspace), writes the new K/V rows into the resident cache at slot
  * seq_len-1, runs ha_sparse_decode, copies `out` back to out_host and SYNCHRONISES the stream.
- * Host buffers should be pinned.  K, V, k_codes, seq_lens, k_per_seq, idx, count stay device
- * pointers (resident state).  K and V must be writable. */
+ * Host buffers should be pinned: buffers that the device can address (cudaHostAlloc / cudaHostRegister
+ * under unified addressing) are read and written by the kernels themselves, without staged copies, and
+ * when the step is one fused launch with lists of up to 2048 entries that kernel also appends the new
+ * rows; any other buffer goes through staged cudaMemcpyAsync calls.  The result is the same in every case.
+ * K, V, k_codes, seq_lens, k_per_seq, idx, count stay device pointers (resident state).  K and V must
+ * be writable. */
 int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
                           const uint16_t *q_host, const uint16_t *k_new_host,
                           const uint16_t *v_new_host, const ha_tensor *K, const ha_tensor *V,

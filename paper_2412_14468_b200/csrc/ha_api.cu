@@ -236,7 +236,7 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
                               int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
                               int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx, int64_t idx_stride_b,
                               int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse, void *workspace,
-                              size_t ws_bytes, void *stream) {
+                              size_t ws_bytes, void *stream, const uint16_t *v_new_host = nullptr) {
     HA_TRY(check_score_args(shape, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_uniform, k_per_seq,
                             max_seq_len, k_max, idx, count));
     HA_TRY(check_mapping(map_q, shape->n_kv_heads));
@@ -255,9 +255,10 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
         HA_CUDA(launch_fused_step(B, Hq, Hkv, shape->sm_scale, view(map_q), k_new ? view(map_k) : MapView{}, q, k_new,
                                   view(K), view(V), k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
                                   max_seq_len, k_max, q_codes, idx, idx_stride_b, idx_stride_h, count, out, lse, st,
-                                  Windows{shape->n_sink, shape->n_local}, block_table, bt_stride_b, page_shift));
+                                  Windows{shape->n_sink, shape->n_local}, block_table, bt_stride_b, page_shift, v_new_host));
         return HA_OK;
     }
+    if (v_new_host) return HA_ERR_INVALID_ARG;   // only the fused kernel appends by itself
 
     EncodeJob jq{};
     jq.x = q; jq.x_sb = (long long)Hq * kD; jq.x_sh = kD;
@@ -354,7 +355,12 @@ int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const 
     const uint16_t *mkn = reinterpret_cast<const uint16_t *>(mapped(k_new_host));
     const uint16_t *mvn = reinterpret_cast<const uint16_t *>(mapped(v_new_host));
     uint16_t *mout = reinterpret_cast<uint16_t *>(mapped(out_host));
-    if (mq && mkn && mvn && mout) {
+    if (mq && mkn && mvn && mout && fused_step_from_host_eligible(B, Hq, Hkv, max_seq_len, k_max)) {
+        // one launch: the fused kernel reads q / k_new / v_new across the bus, appends the new rows and writes `out`
+        HA_TRY(sparse_decode_impl(shape, map_q, map_k, mq, mkn, K, V, nullptr, 0, 0, k_codes, kc_stride_b, kc_stride_h,
+                                  seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx, idx_stride_b, idx_stride_h,
+                                  count, mout, nullptr, workspace, ws_bytes, stream, mvn));
+    } else if (mq && mkn && mvn && mout) {
         HA_CUDA(launch_append_kv(B, Hq, Hkv, mkn, mvn, view(K), view(V), seq_lens, mq, dq, dk, st));
         HA_TRY(ha_sparse_decode(shape, map_q, map_k, dq, dk, K, V, k_codes, kc_stride_b, kc_stride_h, seq_lens,
                                 k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx, idx_stride_b, idx_stride_h, count,

@@ -69,7 +69,7 @@ __device__ __forceinline__ uint32_t attn_issue_block(uint32_t stage_u32, const u
 }
 
 // Query A fragments of head g = lane/4 (rows = heads, k = d); heads >= G are zero rows.
-template <int G>
+template <int G, bool kShared = false>
 __device__ __forceinline__ void attn_load_q(uint32_t (&qa)[8][2], const uint16_t *q_group, int lane) {
     const int g = lane >> 2, c = lane & 3;
 #pragma unroll
@@ -77,7 +77,10 @@ __device__ __forceinline__ void attn_load_q(uint32_t (&qa)[8][2], const uint16_t
     if (g < G) {
         const uint32_t *qp = reinterpret_cast<const uint32_t *>(q_group + (long long)g * kD);
 #pragma unroll
-        for (int s = 0; s < 8; ++s) { qa[s][0] = __ldg(qp + 8 * s + c); qa[s][1] = __ldg(qp + 8 * s + c + 4); }
+        for (int s = 0; s < 8; ++s) {
+            if (kShared) { qa[s][0] = qp[8 * s + c]; qa[s][1] = qp[8 * s + c + 4]; }   // a copy in shared memory
+            else { qa[s][0] = __ldg(qp + 8 * s + c); qa[s][1] = __ldg(qp + 8 * s + c + 4); }
+        }
     }
 }
 

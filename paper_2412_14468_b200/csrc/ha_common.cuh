@@ -190,15 +190,17 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              const int32_t *k_per_seq = nullptr, int k_uniform = 0, Windows win = Windows{0, 0},
                              const int32_t *block_table = nullptr, long long bt_sb = 0, int page_shift = 0);
 
-// The whole layer-step in one launch (one 8-CTA cluster per unit); only for small batches.
+// The whole layer-step in one launch (one cluster per unit); only for small batches.  v_new_host != NULL: q,
+// k_new and v_new are mapped host memory and the kernel appends the new K/V rows itself (host-buffer entry).
 bool fused_step_eligible(int B, int Hq, int Hkv, int max_seq_len, int k_max);
+bool fused_step_from_host_eligible(int B, int Hq, int Hkv, int max_seq_len, int k_max);   // ... with mapped host inputs
 cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapView &map_q, const MapView &map_k,
                               const uint16_t *q, const uint16_t *k_new, TensorView K, TensorView V, uint32_t *k_codes,
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
                               int k_uniform, int max_seq_len, int k_max, uint32_t *q_codes, int32_t *idx,
                               long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
                               cudaStream_t st, Windows win = Windows{0, 0}, const int32_t *block_table = nullptr,
-                              long long bt_sb = 0, int page_shift = 0);
+                              long long bt_sb = 0, int page_shift = 0, const uint16_t *v_new_host = nullptr);
 
 cudaError_t launch_score_wide(const uint64_t *q_code, const uint64_t *k_codes, long long n, int n_words, uint16_t *scores,
                               cudaStream_t st);

@@ -74,6 +74,10 @@ struct FusedArgs {
     const int32_t *block_table;
     long long bt_sb;
     int page_shift, page_rows;
+    // host-buffer entry: q, k_new and v_new are mapped host memory.  The kernel then appends the new K and V
+    // rows itself (slot n - 1) and keeps a copy of the unit's queries in shared memory, so that each of them
+    // crosses the bus once per CTA and never on the critical path of the attention phase.
+    const uint16_t *v_new;
 };
 
 __device__ __forceinline__ void st_dsmem_u32(uint32_t *local, uint32_t rank, uint32_t v) {
@@ -132,7 +136,7 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
     }
 }
 
-template <int G, int S, int CS>
+template <int G, int S, int CS, bool kHost>
 __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kernel(const FusedArgs a) {
     constexpr int kFusedUnionBytes = fused_union_bytes(S);
     constexpr int kFusedActBytes = fused_act_bytes(G, CS);
@@ -211,7 +215,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         if (map.b1) bias1 = __ldg(map.b1 + kvh * kHid + o);
         if (map.b2) bias2 = __ldg(map.b2 + kvh * kHid + o);
         if (map.b3) bias3 = __ldg(map.b3 + kvh * kBits + (tid & (kBits - 1)));
-        if (tid < 2 * (enc_q ? kQPer : 1)) {   // 256 bytes per vector
+        if (!kHost && tid < 2 * (enc_q ? kQPer : 1)) {   // 256 bytes per vector
             const uint16_t *xv = enc_q ? a.q + (head0 + kQPer * (int)rank) * kD : a.k_new + ((long long)b * Hkv + kvh) * kD;
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(xv) + 128 * tid));
         }
@@ -221,6 +225,20 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     pdl_wait();                  // q, k_new and everything older in the stream is final from here on
     pdl_launch_dependents();
     cluster_wait();              // #0: all CTAs of the cluster are running (their shared memory may be written)
+    uint4 q_stage = make_uint4(0u, 0u, 0u, 0u);
+    if (kHost) {
+        // the unit's G query vectors (16 bytes per thread) start their way across the bus now and are parked in
+        // shared memory once the encoders are done with it
+        if (tid < G * 16) q_stage = __ldg(reinterpret_cast<const uint4 *>(a.q + head0 * kD) + tid);
+        if (enc_k && a.v_new && tid < 64) {   // the appended rows: 32 threads x 8 bytes for K, 32 for V (contiguous cache only)
+            const int t = tid & 31;
+            const long long src = ((long long)b * Hkv + kvh) * kD;
+            const TensorView &X = (tid < 32) ? a.K : a.V;
+            const uint2 v = __ldg(reinterpret_cast<const uint2 *>(((tid < 32) ? a.k_new : a.v_new) + src) + t);
+            uint16_t *dst = const_cast<uint16_t *>(X.ptr) + (long long)b * X.sb + (long long)kvh * X.sh + (long long)(n - 1) * X.sn;
+            reinterpret_cast<uint2 *>(dst)[t] = v;
+        }
+    }
 
     // ---------------- P1: ENCODE in the first kQCtas CTAs (queries) and the next one (appended key)
     if (enc_q) {
@@ -235,6 +253,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     // stored after the barrier, so that its release had nothing but shared-memory stores to wait for
     if (enc_q && tid < kQPer) a.q_codes[head0 + kQPer * (int)rank + tid] = s_codes[kQPer * (int)rank + tid];
     if (enc_k && tid == 0) row[n - 1] = s_codes[G];
+    if (kHost && tid < G * 16) reinterpret_cast<uint4 *>(actA)[tid] = q_stage;   // the activations are dead
     uint32_t qc[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) qc[j] = s_codes[j];
@@ -409,7 +428,8 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     const int g = lane >> 2, cc = lane & 3;
 
     uint32_t qa[8][2];
-    attn_load_q<G>(qa, a.q + head0 * kD, lane);
+    if (kHost) attn_load_q<G, true>(qa, reinterpret_cast<const uint16_t *>(actA), lane);
+    else attn_load_q<G>(qa, a.q + head0 * kD, lane);
     float acc[8][4];
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt)
@@ -545,14 +565,14 @@ static void fused_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute (&attr)[2]
 
 // Opt in to the shared-memory carve-out (once per device) and return how many clusters of this variant the
 // device holds at once (0 on error).
-template <int G, int S, int CS>
+template <int G, int S, int CS, bool kHost = false>
 static int fused_prepare() {
     static int clusters[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
     if (!clusters[dev]) {
-        if (cudaFuncSetAttribute(fused_step_kernel<G, S, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(fused_step_kernel<G, S, CS, kHost>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  fused_smem_bytes(G, S, CS)) != cudaSuccess)
             return 0;
         cudaLaunchConfig_t cfg;
@@ -560,19 +580,19 @@ static int fused_prepare() {
         fused_config<G, S, CS>(cfg, attr, 1, 64, nullptr);
         cfg.numAttrs = 1;   // the cluster shape is all the occupancy query looks at
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, fused_step_kernel<G, S, CS>, &cfg) != cudaSuccess || n <= 0) return 0;
+        if (cudaOccupancyMaxActiveClusters(&n, fused_step_kernel<G, S, CS, kHost>, &cfg) != cudaSuccess || n <= 0) return 0;
         clusters[dev] = n;
     }
     return clusters[dev];
 }
 
-template <int G, int S, int CS>
+template <int G, int S, int CS, bool kHost = false>
 static cudaError_t launch_fused_gsc(const FusedArgs &args, int B, cudaStream_t st) {
-    if (fused_prepare<G, S, CS>() <= 0) return cudaErrorInvalidConfiguration;
+    if (fused_prepare<G, S, CS, kHost>() <= 0) return cudaErrorInvalidConfiguration;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
     fused_config<G, S, CS>(cfg, attr, args.Hkv, B, st);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_step_kernel<G, S, CS>, args);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_step_kernel<G, S, CS, kHost>, args);
     if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
@@ -615,10 +635,29 @@ bool fused_step_eligible(int B, int Hq, int Hkv, int max_seq_len, int k_max) {
     }
 }
 
+bool fused_step_from_host_eligible(int B, int Hq, int Hkv, int max_seq_len, int k_max) {
+    if (max_seq_len > kFusedMaxSeq || Hkv <= 0) return false;
+    const long long units = (long long)B * Hkv;
+    int stages = 0, cs = 0;
+    switch (Hq / Hkv) {
+        case 1: cs = fused_variant<1>(units, k_max, &stages); break;
+        case 2: cs = fused_variant<2>(units, k_max, &stages); break;
+        case 4: cs = fused_variant<4>(units, k_max, &stages); break;
+        case 8: cs = fused_variant<8>(units, k_max, &stages); break;
+        default: return false;
+    }
+    return cs > 0 && stages == 1;
+}
+
 template <int G>
 static cudaError_t launch_fused_g(const FusedArgs &args, int B, cudaStream_t st) {
     int stages = 0;
     const int cs = fused_variant<G>((long long)B * args.Hkv, args.k_max, &stages);
+    if (args.v_new) {   // host-buffer entry: only the one-stage variants read their inputs across the bus
+        if (stages == 1 && cs == 8) return launch_fused_gsc<G, 1, 8, true>(args, B, st);
+        if (stages == 1 && cs == 4) return launch_fused_gsc<G, 1, 4, true>(args, B, st);
+        return cudaErrorInvalidConfiguration;
+    }
     if (stages == 2 && cs == 8) return launch_fused_gsc<G, 2, 8>(args, B, st);
     if (cs == 8) return launch_fused_gsc<G, 1, 8>(args, B, st);
     if (cs == 4) return launch_fused_gsc<G, 1, 4>(args, B, st);
@@ -630,8 +669,10 @@ cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapV
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
                               int k_uniform, int max_seq_len, int k_max, uint32_t *q_codes, int32_t *idx,
                               long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
-                              cudaStream_t st, Windows win, const int32_t *block_table, long long bt_sb, int page_shift) {
+                              cudaStream_t st, Windows win, const int32_t *block_table, long long bt_sb, int page_shift,
+                              const uint16_t *v_new_host) {
     FusedArgs a{};
+    a.v_new = v_new_host;
     a.win = win;
     a.block_table = block_table; a.bt_sb = bt_sb; a.page_shift = page_shift;
     a.page_rows = (block_table && K.sn > 0) ? (int)(K.sb / K.sn) : 0;

@@ -658,6 +658,14 @@ def test_sparse_decode_step_every_launch_variant(cfg, launches):
     assert np.array_equal(r["cnt"].cpu().numpy(), ref["count"])
     assert np.array_equal(r["idx"].cpu().numpy(), ref["idx"])
     assert_out_close(u16(r["out"]), ref["out"])
+    # The host-buffer entry takes the same variant.  The one-stage fused kernel reads q / k_new / v_new from the
+    # pinned buffers and appends the new rows itself (one launch); every other variant is preceded by the small
+    # kernel that pulls the inputs across the bus and appends (one launch more).
+    before = ha.ha_kernel_launches()
+    rh = _run_step(w, host=True)                   # checks that the new K/V rows were appended in place
+    one_stage_fused = launches == 1 and w["k_max"] <= 2048 and cfg.name != "fused-large-k"
+    assert ha.ha_kernel_launches() - before == (1 if one_stage_fused else launches + 1) + 1
+    assert torch.equal(rh["idx"], r["idx"]) and torch.equal(rh["out"], r["out"])
 
 
 def test_k_equals_n_sparse_step_equals_dense_kernel():
