@@ -20,8 +20,12 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
+# the bench's batch sweep at the headline shape: one fused launch with clusters of 8 (32 units) and of 4 (64 units)
+SWEEP = {f"sweep_B{bsz}_32K_32x": wl.Config(f"sweep{bsz}", 10 + bsz, bsz, 32768, 1024, 0.01) for bsz in (4, 8)}
+
+
 def _run(cfg_name):
-    w = wl.make_workload(cfg_name, DEV)
+    w = wl.make_workload(SWEEP.get(cfg_name, cfg_name), DEV)
     cfg = w["cfg"]
     B, Hq, Hkv = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads
     shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
@@ -48,7 +52,7 @@ def _run(cfg_name):
     return w, dict(kc=kc, qc=qc, idx=idx, cnt=cnt, out=out, lse=lse, hist=hist, shape=shape, ws=ws)
 
 
-@pytest.mark.parametrize("cfg_name", ["c2", "c3", "c4", "c5"])
+@pytest.mark.parametrize("cfg_name", ["c2", "c3", "c4", "c5", "sweep_B4_32K_32x", "sweep_B8_32K_32x"])
 def test_full_size_config_matches_oracle(cfg_name):
     import time
     t_start = time.time()
