@@ -136,6 +136,146 @@ __device__ __forceinline__ void fused_encode(const uint16_t *x0, long long x_str
     }
 }
 
+// GATHER-ATT over this CTA's share of a unit's index list, blocks [blk_lo, blk_hi) of 16 entries, and the merge
+// of the cluster's CTA states in CTA 0, which writes the unit's outputs.  Shared by the fused step and the
+// stand-alone cluster gather.  kLocalList: the CTA's part of the list sits in its shared memory (s_list), else
+// in global memory (list).  kQShared: q_src is a copy of the unit's queries in shared memory.  kCheck: entries
+// >= n_rows are skipped and reported through `bad` (lists that the caller wrote).
+template <int G, int S, int CS, bool kLocalList, bool kQShared, bool kCheck>
+__device__ __forceinline__ void fused_attention(const FusedArgs &a, uint32_t rank, int b, int kvh, long long head0, int keep,
+                                                int n_rows, int blk_lo, int blk_hi, const int32_t *list,
+                                                const int32_t *s_list, const uint16_t *q_src, unsigned char *ring,
+                                                float *part_ml, float *part_acc, float (*s_m)[8], float (*s_l)[8],
+                                                uint32_t (*s_mask)[kFusedMaxStages], bool &bad) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool paged = a.block_table != nullptr;   // rows are then addressed from the pool's base
+    const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (paged ? 0LL : (long long)b * a.K.sb) + (long long)kvh * a.K.sh);
+    const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (paged ? 0LL : (long long)b * a.V.sb) + (long long)kvh * a.V.sh);
+    const int32_t *pages = paged ? a.block_table + (long long)b * a.bt_sb : nullptr;
+    const long long k_row = a.K.sn * 2, v_row = a.V.sn * 2;
+    unsigned char *my_ring = ring + warp * (S * kStageBytes);
+    const uint32_t ring_u32 = smem_u32(my_ring);
+    const int g = lane >> 2, cc = lane & 3;
+
+    uint32_t qa[8][2];
+    attn_load_q<G, kQShared>(qa, q_src, lane);
+    float acc[8][4];
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[mt][e] = 0.0f;
+    float m_run = -CUDART_INF_F, l_run = 0.0f;
+    {
+        // this warp's blocks: blk_lo + warp, + 8, ...; list entries were selected by peer CTAs: they sit in this
+        // CTA's shared memory (one-stage variant) or are read from L2
+        const int nblk = (blk_lo + warp < blk_hi) ? (blk_hi - blk_lo - warp + kFusedWarps - 1) / kFusedWarps : 0;
+        auto token_of_block = [&](int i) -> int {
+            const int p = (blk_lo + warp + i * kFusedWarps) * kBlockTokens + (lane & 15);
+            int t = -1;
+            if (i < nblk && p < keep) t = kLocalList ? s_list[p - blk_lo * kBlockTokens] : __ldcg(list + p);
+            if (kCheck && t >= n_rows) { bad = true; t = -1; }   // a caller's list may point outside the sequence
+            // paged: logical token -> row of the pool (page * rows per page stride + slot)
+            if (paged && t >= 0) t = __ldg(pages + (t >> a.page_shift)) * a.page_rows + (t & ((1 << a.page_shift) - 1));
+            return t;
+        };
+        auto issue = [&](int i, int stg) {
+            const uint32_t valid = attn_issue_block(ring_u32 + stg * kStageBytes, Kb, Vb, k_row, v_row, token_of_block(i), lane);
+            if (lane == 0) s_mask[warp][stg] = valid;
+        };
+        if (nblk > 0) issue(0, 0);
+        cp_async_commit();
+        for (int i = 0; i < nblk; ++i) {
+            const int stg = (S > 1) ? (i & 1) : 0;
+            if (S > 1) {   // the next block travels while this one is consumed
+                if (i + 1 < nblk) issue(i + 1, stg ^ 1);
+                cp_async_commit();
+                cp_async_wait<1>();
+            } else {
+                cp_async_wait<0>();
+            }
+            __syncwarp();
+            const uint32_t ks = ring_u32 + stg * kStageBytes;
+            attn_consume_block(ks, ks + kTileBytes, s_mask[warp][stg], qa, a.scale_log2, lane, acc, m_run, l_run);
+            __syncwarp();
+            if (S == 1) {   // one stage: the next block is requested once this one has been read
+                if (i + 1 < nblk) issue(i + 1, 0);
+                cp_async_commit();
+            }
+        }
+        cp_async_wait<0>();
+    }
+    // merge the warps of this CTA through shared memory (each warp reuses its own ring)
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (cc == 0) { s_m[warp][g] = m_run; s_l[warp][g] = l_run; }
+    __syncwarp();
+    {
+        float *my_acc = reinterpret_cast<float *>(my_ring);   // [G][128]
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int h = 2 * cc + hh;
+            if (h < G) {
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    my_acc[h * kD + 16 * mt + g] = acc[mt][hh];
+                    my_acc[h * kD + 16 * mt + 8 + g] = acc[mt][2 + hh];
+                }
+            }
+        }
+    }
+    __syncthreads();
+    {   // this CTA's state goes into slot `rank` of CTA 0's shared memory; the two thread halves share the heads
+        const int d = tid & (kD - 1), hsel = tid >> 7;
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+            if (G > 1 && (j & 1) != hsel) continue;
+            if (G == 1 && hsel != 0) continue;
+            float M = s_m[0][j];
+#pragma unroll
+            for (int w = 1; w < kFusedWarps; ++w) M = fmaxf(M, s_m[w][j]);
+            float L = 0.0f, A = 0.0f;
+            if (M > -CUDART_INF_F) {
+#pragma unroll
+                for (int w = 0; w < kFusedWarps; ++w) {
+                    const float f = exp2f(s_m[w][j] - M);
+                    L = fmaf(s_l[w][j], f, L);
+                    A = fmaf(reinterpret_cast<const float *>(ring + w * (S * kStageBytes))[j * kD + d], f, A);
+                }
+            }
+            st_dsmem_f32(part_acc + ((int)rank * G + j) * kD + d, 0, A);
+            if (d == 0) {
+                st_dsmem_f32(part_ml + ((int)rank * G + j) * 2, 0, M);
+                st_dsmem_f32(part_ml + ((int)rank * G + j) * 2 + 1, 0, L);
+            }
+        }
+    }
+    cluster_sync_all();   // #4: the states of all CTAs have landed in CTA 0
+    if (rank == 0) {
+        const int d = tid & (kD - 1), hsel = tid >> 7;
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+            if (G > 1 && (j & 1) != hsel) continue;
+            if (G == 1 && hsel != 0) continue;
+            float M = -CUDART_INF_F;
+#pragma unroll
+            for (int r = 0; r < CS; ++r) M = fmaxf(M, part_ml[(r * G + j) * 2]);
+            float L = 0.0f, A = 0.0f;
+            if (M > -CUDART_INF_F) {
+#pragma unroll
+                for (int r = 0; r < CS; ++r) {
+                    const float f = exp2f(part_ml[(r * G + j) * 2] - M);
+                    L = fmaf(part_ml[(r * G + j) * 2 + 1], f, L);
+                    A = fmaf(part_acc[(r * G + j) * kD + d], f, A);
+                }
+            }
+            const float o = (L > 0.0f) ? A / L : 0.0f;
+            const __nv_bfloat16 ob = __float2bfloat16_rn(o);
+            a.out[(head0 + j) * kD + d] = *reinterpret_cast<const uint16_t *>(&ob);
+            if (a.lse && d == 0) a.lse[head0 + j] = (L > 0.0f) ? (M * kLn2 + logf(L)) : -CUDART_INF_F;
+        }
+    }
+}
+
 template <int G, int S, int CS, bool kHost>
 __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kernel(const FusedArgs a) {
     constexpr int kFusedUnionBytes = fused_union_bytes(S);
@@ -235,7 +375,8 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
             const long long src = ((long long)b * Hkv + kvh) * kD;
             const TensorView &X = (tid < 32) ? a.K : a.V;
             const uint2 v = __ldg(reinterpret_cast<const uint2 *>(((tid < 32) ? a.k_new : a.v_new) + src) + t);
-            uint16_t *dst = const_cast<uint16_t *>(X.ptr) + (long long)b * X.sb + (long long)kvh * X.sh + (long long)(n - 1) * X.sn;
+            // slot seq_len - 1 as the stand-alone append kernel takes it (n is the length clamped to max_seq_len)
+            uint16_t *dst = const_cast<uint16_t *>(X.ptr) + (long long)b * X.sb + (long long)kvh * X.sh + (long long)(a.seq_lens[b] - 1) * X.sn;
             reinterpret_cast<uint2 *>(dst)[t] = v;
         }
     }
@@ -417,133 +558,11 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
         }
     }
 
-    // ---------------- P3: GATHER-ATT over this CTA's share of the list
-    const bool paged = a.block_table != nullptr;   // rows are then addressed from the pool's base
-    const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (paged ? 0LL : (long long)b * a.K.sb) + (long long)kvh * a.K.sh);
-    const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (paged ? 0LL : (long long)b * a.V.sb) + (long long)kvh * a.V.sh);
-    const int32_t *pages = paged ? a.block_table + (long long)b * a.bt_sb : nullptr;
-    const long long k_row = a.K.sn * 2, v_row = a.V.sn * 2;
-    unsigned char *my_ring = ring + warp * (S * kStageBytes);
-    const uint32_t ring_u32 = smem_u32(my_ring);
-    const int g = lane >> 2, cc = lane & 3;
-
-    uint32_t qa[8][2];
-    if (kHost) attn_load_q<G, true>(qa, reinterpret_cast<const uint16_t *>(actA), lane);
-    else attn_load_q<G>(qa, a.q + head0 * kD, lane);
-    float acc[8][4];
-#pragma unroll
-    for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[mt][e] = 0.0f;
-    float m_run = -CUDART_INF_F, l_run = 0.0f;
-    {
-        // this warp's blocks: blk_lo + warp, + 8, ...; list entries were selected by peer CTAs: they sit in this
-        // CTA's shared memory (one-stage variant) or are read from L2
-        const int nblk = (blk_lo + warp < blk_hi) ? (blk_hi - blk_lo - warp + kFusedWarps - 1) / kFusedWarps : 0;
-        auto token_of_block = [&](int i) -> int {
-            const int p = (blk_lo + warp + i * kFusedWarps) * kBlockTokens + (lane & 15);
-            int t = -1;
-            if (i < nblk && p < keep) t = kLocalList ? s_list[p - blk_lo * kBlockTokens] : __ldcg(list + p);
-            // paged: logical token -> row of the pool (page * rows per page stride + slot)
-            if (paged && t >= 0) t = __ldg(pages + (t >> a.page_shift)) * a.page_rows + (t & ((1 << a.page_shift) - 1));
-            return t;
-        };
-        auto issue = [&](int i, int stg) {
-            const uint32_t valid = attn_issue_block(ring_u32 + stg * kStageBytes, Kb, Vb, k_row, v_row, token_of_block(i), lane);
-            if (lane == 0) s_mask[warp][stg] = valid;
-        };
-        if (nblk > 0) issue(0, 0);
-        cp_async_commit();
-        for (int i = 0; i < nblk; ++i) {
-            const int stg = (S > 1) ? (i & 1) : 0;
-            if (S > 1) {   // the next block travels while this one is consumed
-                if (i + 1 < nblk) issue(i + 1, stg ^ 1);
-                cp_async_commit();
-                cp_async_wait<1>();
-            } else {
-                cp_async_wait<0>();
-            }
-            __syncwarp();
-            const uint32_t ks = ring_u32 + stg * kStageBytes;
-            attn_consume_block(ks, ks + kTileBytes, s_mask[warp][stg], qa, a.scale_log2, lane, acc, m_run, l_run);
-            __syncwarp();
-            if (S == 1) {   // one stage: the next block is requested once this one has been read
-                if (i + 1 < nblk) issue(i + 1, 0);
-                cp_async_commit();
-            }
-        }
-        cp_async_wait<0>();
-    }
-    // merge the warps of this CTA through shared memory (each warp reuses its own ring)
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    if (cc == 0) { s_m[warp][g] = m_run; s_l[warp][g] = l_run; }
-    __syncwarp();
-    {
-        float *my_acc = reinterpret_cast<float *>(my_ring);   // [G][128]
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-            const int h = 2 * cc + hh;
-            if (h < G) {
-#pragma unroll
-                for (int mt = 0; mt < 8; ++mt) {
-                    my_acc[h * kD + 16 * mt + g] = acc[mt][hh];
-                    my_acc[h * kD + 16 * mt + 8 + g] = acc[mt][2 + hh];
-                }
-            }
-        }
-    }
-    __syncthreads();
-    {   // this CTA's state goes into slot `rank` of CTA 0's shared memory; the two thread halves share the heads
-        const int d = tid & (kD - 1), hsel = tid >> 7;
-#pragma unroll
-        for (int j = 0; j < G; ++j) {
-            if (G > 1 && (j & 1) != hsel) continue;
-            if (G == 1 && hsel != 0) continue;
-            float M = s_m[0][j];
-#pragma unroll
-            for (int w = 1; w < kFusedWarps; ++w) M = fmaxf(M, s_m[w][j]);
-            float L = 0.0f, A = 0.0f;
-            if (M > -CUDART_INF_F) {
-#pragma unroll
-                for (int w = 0; w < kFusedWarps; ++w) {
-                    const float f = exp2f(s_m[w][j] - M);
-                    L = fmaf(s_l[w][j], f, L);
-                    A = fmaf(reinterpret_cast<const float *>(ring + w * (S * kStageBytes))[j * kD + d], f, A);
-                }
-            }
-            st_dsmem_f32(part_acc + ((int)rank * G + j) * kD + d, 0, A);
-            if (d == 0) {
-                st_dsmem_f32(part_ml + ((int)rank * G + j) * 2, 0, M);
-                st_dsmem_f32(part_ml + ((int)rank * G + j) * 2 + 1, 0, L);
-            }
-        }
-    }
-    cluster_sync_all();   // #4: the states of all CTAs have landed in CTA 0
-    if (rank == 0) {
-        const int d = tid & (kD - 1), hsel = tid >> 7;
-#pragma unroll
-        for (int j = 0; j < G; ++j) {
-            if (G > 1 && (j & 1) != hsel) continue;
-            if (G == 1 && hsel != 0) continue;
-            float M = -CUDART_INF_F;
-#pragma unroll
-            for (int r = 0; r < CS; ++r) M = fmaxf(M, part_ml[(r * G + j) * 2]);
-            float L = 0.0f, A = 0.0f;
-            if (M > -CUDART_INF_F) {
-#pragma unroll
-                for (int r = 0; r < CS; ++r) {
-                    const float f = exp2f(part_ml[(r * G + j) * 2] - M);
-                    L = fmaf(part_ml[(r * G + j) * 2 + 1], f, L);
-                    A = fmaf(part_acc[(r * G + j) * kD + d], f, A);
-                }
-            }
-            const float o = (L > 0.0f) ? A / L : 0.0f;
-            const __nv_bfloat16 ob = __float2bfloat16_rn(o);
-            a.out[(head0 + j) * kD + d] = *reinterpret_cast<const uint16_t *>(&ob);
-            if (a.lse && d == 0) a.lse[head0 + j] = (L > 0.0f) ? (M * kLn2 + logf(L)) : -CUDART_INF_F;
-        }
-    }
+    // ---------------- P3: GATHER-ATT over this CTA's share of the list, merge, output
+    bool bad = false;
+    fused_attention<G, S, CS, kLocalList, kHost, false>(a, rank, b, kvh, head0, keep, n, blk_lo, blk_hi, list, s_list,
+                                                        kHost ? reinterpret_cast<const uint16_t *>(actA) : a.q + head0 * kD,
+                                                        ring, part_ml, part_acc, s_m, s_l, s_mask, bad);
 }
 
 template <int G, int S, int CS>
