@@ -176,6 +176,13 @@ int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
     WorkspaceLayout L;
     HA_TRY(check_workspace(shape, -1, workspace, ws_bytes, &L));
     if (shape->batch == 0) return HA_OK;
+    if (gather_cluster_eligible(shape->batch, shape->n_q_heads, shape->n_kv_heads, k_max)) {
+        // few units, short lists: one cluster per unit, merged through distributed shared memory
+        HA_CUDA(launch_gather_cluster(shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K), view(V),
+                                      seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
+                                      ws_ptr<uint32_t>(workspace, 0), (cudaStream_t)stream));
+        return HA_OK;
+    }
     HA_CUDA(launch_attention(true, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K),
                              view(V), seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
                              ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),
@@ -203,6 +210,12 @@ int ha_gather_attn_paged(const ha_shape *shape, const uint16_t *q, const ha_tens
     if (shape->batch == 0) return HA_OK;
     int shift = 0;
     while ((1 << shift) < page_size) ++shift;
+    if (gather_cluster_eligible(shape->batch, shape->n_q_heads, shape->n_kv_heads, k_max)) {
+        HA_CUDA(launch_gather_cluster(shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K_pool),
+                                      view(V_pool), seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
+                                      ws_ptr<uint32_t>(workspace, 0), (cudaStream_t)stream, block_table, bt_stride_b, shift));
+        return HA_OK;
+    }
     HA_CUDA(launch_attention(true, shape->batch, shape->n_q_heads, shape->n_kv_heads, shape->sm_scale, q, view(K_pool),
                              view(V_pool), seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
                              ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),

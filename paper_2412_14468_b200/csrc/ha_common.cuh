@@ -202,6 +202,14 @@ cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapV
                               cudaStream_t st, Windows win = Windows{0, 0}, const int32_t *block_table = nullptr,
                               long long bt_sb = 0, int page_shift = 0, const uint16_t *v_new_host = nullptr);
 
+// Stand-alone GATHER-ATT with one 8-CTA cluster per unit (few units, short lists).
+bool gather_cluster_eligible(int B, int Hq, int Hkv, int k_max);
+cudaError_t launch_gather_cluster(int B, int Hq, int Hkv, float sm_scale, const uint16_t *q, TensorView K, TensorView V,
+                                  const int32_t *seq_lens, const int32_t *idx, long long idx_sb, long long idx_sh,
+                                  const int32_t *count, int k_max, uint16_t *out, float *lse, uint32_t *status,
+                                  cudaStream_t st, const int32_t *block_table = nullptr, long long bt_sb = 0,
+                                  int page_shift = 0);
+
 cudaError_t launch_score_wide(const uint64_t *q_code, const uint64_t *k_codes, long long n, int n_words, uint16_t *scores,
                               cudaStream_t st);
 cudaError_t launch_inner_products(const uint16_t *q, const uint16_t *K, long long n, long long row_stride, float *dots,

@@ -78,6 +78,7 @@ struct FusedArgs {
     // rows itself (slot n - 1) and keeps a copy of the unit's queries in shared memory, so that each of them
     // crosses the bus once per CTA and never on the critical path of the attention phase.
     const uint16_t *v_new;
+    uint32_t *status;   // stand-alone cluster gather: device status word (HA_DEV_BAD_INDEX)
 };
 
 __device__ __forceinline__ void st_dsmem_u32(uint32_t *local, uint32_t rank, uint32_t v) {
@@ -563,6 +564,124 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
     fused_attention<G, S, CS, kLocalList, kHost, false>(a, rank, b, kvh, head0, keep, n, blk_lo, blk_hi, list, s_list,
                                                         kHost ? reinterpret_cast<const uint16_t *>(actA) : a.q + head0 * kD,
                                                         ring, part_ml, part_acc, s_m, s_l, s_mask, bad);
+}
+
+// ------------------------------------------------------------------ stand-alone GATHER-ATT with clusters
+//
+// ha_gather_attn for few units and short lists: the attention phase of the fused step on a list that the caller
+// provides (one cluster of 8 CTAs per (sequence, KV head), each CTA an eighth of the list, states merged in
+// CTA 0's shared memory), instead of the persistent split-K kernel whose work split and global-memory merge cost
+// more than the attention itself at this size.
+__host__ __device__ constexpr int gather_cluster_smem_bytes(int G, int CS) { return fused_ring_bytes(1) + fused_part_bytes(G, CS); }
+
+template <int G, int CS>
+__global__ void __launch_bounds__(kFusedThreads, 2) gather_cluster_kernel(const FusedArgs a) {
+    extern __shared__ __align__(128) unsigned char gsm[];
+    unsigned char *ring = gsm;
+    float *part_ml = reinterpret_cast<float *>(gsm + fused_ring_bytes(1));   // [CS][G][2]
+    float *part_acc = part_ml + CS * G * 2;                                  // [CS][G][128]
+    __shared__ float s_m[kFusedWarps][8], s_l[kFusedWarps][8];
+    __shared__ uint32_t s_mask[kFusedWarps][kFusedMaxStages];
+    cluster_arrive();   // completed before the first store into CTA 0's shared memory: every CTA has started
+    const uint32_t rank = cluster_rank();
+    const int kvh = blockIdx.y, b = blockIdx.z;
+    const long long head0 = (long long)b * a.Hq + (long long)kvh * G;
+    pdl_launch_dependents();
+    pdl_wait();   // the list, its length and the rows may come from the kernels in front
+    cluster_wait();
+    const int n = a.seq_lens[b];
+    const int keep = max(0, min(a.count[b * a.Hkv + kvh], a.k_max));
+    const int blocks_total = (keep + kBlockTokens - 1) / kBlockTokens;
+    const int bpc = (blocks_total + CS - 1) / CS;
+    const int blk_lo = min(blocks_total, (int)rank * bpc), blk_hi = min(blocks_total, blk_lo + bpc);
+    const int32_t *list = a.idx + (long long)b * a.idx_sb + (long long)kvh * a.idx_sh;
+    bool bad = false;
+    fused_attention<G, 1, CS, false, false, true>(a, rank, b, kvh, head0, keep, n, blk_lo, blk_hi, list, nullptr,
+                                                  a.q + head0 * kD, ring, part_ml, part_acc, s_m, s_l, s_mask, bad);
+    if (bad) atomicOr(a.status, HA_DEV_BAD_INDEX);
+}
+
+template <int G>
+static int gather_cluster_prepare() {
+    static int clusters[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (!clusters[dev]) {
+        constexpr int smem = gather_cluster_smem_bytes(G, 8);
+        if (cudaFuncSetAttribute(gather_cluster_kernel<G, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+            return 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(8, 1, 64);
+        cfg.blockDim = dim3(kFusedThreads);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 8;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gather_cluster_kernel<G, 8>, &cfg) != cudaSuccess || n <= 0) return 0;
+        clusters[dev] = n;
+    }
+    return clusters[dev];
+}
+
+// Lists of up to 2048 entries (at most two blocks per warp) and as many units as clusters are resident at once.
+bool gather_cluster_eligible(int B, int Hq, int Hkv, int k_max) {
+    if (Hkv <= 0 || k_max > kFusedOneStageMaxK) return false;
+    const long long units = (long long)B * Hkv;
+    switch (Hq / Hkv) {
+        case 1: return units <= gather_cluster_prepare<1>();
+        case 2: return units <= gather_cluster_prepare<2>();
+        case 4: return units <= gather_cluster_prepare<4>();
+        case 8: return units <= gather_cluster_prepare<8>();
+        default: return false;
+    }
+}
+
+template <int G>
+static cudaError_t launch_gather_cluster_g(const FusedArgs &args, int B, cudaStream_t st) {
+    if (gather_cluster_prepare<G>() <= 0) return cudaErrorInvalidConfiguration;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(8, args.Hkv, B);
+    cfg.blockDim = dim3(kFusedThreads);
+    cfg.dynamicSmemBytes = gather_cluster_smem_bytes(G, 8);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 8;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gather_cluster_kernel<G, 8>, args);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather_cluster(int B, int Hq, int Hkv, float sm_scale, const uint16_t *q, TensorView K, TensorView V,
+                                  const int32_t *seq_lens, const int32_t *idx, long long idx_sb, long long idx_sh,
+                                  const int32_t *count, int k_max, uint16_t *out, float *lse, uint32_t *status,
+                                  cudaStream_t st, const int32_t *block_table, long long bt_sb, int page_shift) {
+    FusedArgs a{};
+    a.block_table = block_table; a.bt_sb = bt_sb; a.page_shift = page_shift;
+    a.page_rows = (block_table && K.sn > 0) ? (int)(K.sb / K.sn) : 0;
+    a.q = q; a.K = K; a.V = V; a.seq_lens = seq_lens; a.k_max = k_max; a.Hq = Hq; a.Hkv = Hkv;
+    a.scale_log2 = sm_scale * kLog2e; a.idx = const_cast<int32_t *>(idx); a.idx_sb = idx_sb; a.idx_sh = idx_sh;
+    a.count = const_cast<int32_t *>(count); a.out = out; a.lse = lse; a.status = status;
+    switch (Hq / Hkv) {
+        case 1: return launch_gather_cluster_g<1>(a, B, st);
+        case 2: return launch_gather_cluster_g<2>(a, B, st);
+        case 4: return launch_gather_cluster_g<4>(a, B, st);
+        case 8: return launch_gather_cluster_g<8>(a, B, st);
+        default: return cudaErrorInvalidValue;
+    }
 }
 
 template <int G, int S, int CS>
