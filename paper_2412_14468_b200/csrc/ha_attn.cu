@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
     };
 
     // ---- this CTA's range [x, x_end) of the global block sequence
-    long long x, x_end, T;
+    long long x, x_end, T, Pe = P;   // Pe: CTAs that take part in the split
     int u;
     if (a.balanced) {
         if (a.n_units <= 32) {
@@ -134,8 +134,12 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
             __syncthreads();
         }
         T = s_pref[a.n_units];
-        x = (T > 0) ? (long long)cta * T / P : 0;
-        x_end = (T > 0) ? (long long)(cta + 1) * T / P : 0;
+        // Fewer blocks than CTAs (lists much shorter than the rows that hold them): only the first T CTAs take a
+        // range, one block each.  With the full grid in the formulas some CTAs of a unit's range would be empty
+        // and leave without a ticket, and the unit would never be finalised.
+        if (T > 0 && T < Pe) Pe = T;
+        x = (T > 0 && cta < Pe) ? (long long)cta * T / Pe : 0;
+        x_end = (T > 0 && cta < Pe) ? (long long)(cta + 1) * T / Pe : 0;
         int lo = 0, hi = a.n_units;   // largest u with s_pref[u] <= x
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -164,7 +168,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
         if (a.balanced) {
             u_lo = s_pref[u];
             u_hi = s_pref[u + 1];
-            const int c_first = (int)(((u_lo + 1) * P - 1) / T), c_last = (int)((u_hi * P - 1) / T);
+            const int c_first = (int)(((u_lo + 1) * Pe - 1) / T), c_last = (int)((u_hi * Pe - 1) / T);
             n_parts = c_last - c_first + 1;
             my_part = cta - c_first;
             slot0 = c_first + u;   // slots of a unit are consecutive: CTA index + unit index

@@ -327,14 +327,14 @@ def _check_gather(q, K, V, lens, idx_np, cnt_np, sm_scale, expect_flag=0):
     return worst
 
 
+@pytest.mark.parametrize("k_max", [700, 2100])   # index rows of up to 2048 entries: one cluster per unit; wider: split-K kernel
 @pytest.mark.parametrize("G", [1, 4, 8])
-def test_gather_attn_random_lists(G):
+def test_gather_attn_random_lists(G, k_max):
     Hkv, Hq, n_cap = 2, 2 * G, 3000
     B = 3
     lens = [3000, 1777, 64]
     q, K, V = _attn_inputs(B, Hq, Hkv, n_cap, 40 + G)
     rng = np.random.default_rng(41)
-    k_max = 700
     idx = np.full((B, Hkv, k_max), -1, np.int32)
     cnt = np.zeros((B, Hkv), np.int32)
     for b in range(B):
@@ -346,10 +346,11 @@ def test_gather_attn_random_lists(G):
     _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128))
 
 
-def test_gather_attn_padding_invalid_and_unsorted_indices():
+@pytest.mark.parametrize("width", [64, 2100])   # both stand-alone gather kernels (see test_gather_attn_random_lists)
+def test_gather_attn_padding_invalid_and_unsorted_indices(width):
     Hq, Hkv, n_cap = 8, 2, 500
     q, K, V = _attn_inputs(1, Hq, Hkv, n_cap, 50, scale=2.0)
-    idx = np.full((1, Hkv, 64), -1, np.int32)
+    idx = np.full((1, Hkv, width), -1, np.int32)
     idx[0, 0, :10] = [499, 3, 3, -1, 250, 7, -1, 0, 42, 499]       # padding inside, duplicates, unsorted
     idx[0, 1, :6] = [5, 400, 450, 10, 399, 1]                       # 400, 450 are beyond seq_len = 400
     cnt = np.array([[10, 6]], np.int32)
