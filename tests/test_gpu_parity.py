@@ -386,10 +386,11 @@ def test_single_index_returns_value_row_exactly_and_k_equals_n_is_dense():
         assert abs(float(l_d[0, h]) - el) < 1e-3
 
 
-@pytest.mark.parametrize("lens", [[1], [33, 4097], [20000, 1, 0]])
-def test_dense_decode_matches_oracle(lens):
+@pytest.mark.parametrize("lens,cap", [([1], None), ([33, 4097], None), ([20000, 1, 0], None),
+                                      ([100, 1], 30000)])   # a cache far longer than its sequences: fewer blocks than CTAs
+def test_dense_decode_matches_oracle(lens, cap):
     Hq, Hkv = 8, 2
-    B, n_cap = len(lens), max(max(lens), 1)
+    B, n_cap = len(lens), cap or max(max(lens), 1)
     q, K, V = _attn_inputs(B, Hq, Hkv, n_cap, 70 + len(lens))
     shape = ha.make_shape(B, Hq, Hkv, 1.0 / math.sqrt(128))
     ws = ha.alloc_workspace(shape, n_cap, n_cap)
