@@ -358,7 +358,7 @@ def main():
         "algorithmic_bytes_per_launch": alg_bytes, "us_per_launch": us_per_step,
         "launches_per_step": launches_per_step,
         "standalone_entry_points": {
-            "ha_gather_attn (attn_kernel<4,true>)": {"algorithmic_bytes": gather_bytes, "us": g_us,
+            "ha_gather_attn (gather_cluster_kernel<4,8>)": {"algorithmic_bytes": gather_bytes, "us": g_us,
                                                       "achieved": gather_bytes / (g_us * 1e-6) / 1e9,
                                                       "frac": gather_bytes / (g_us * 1e-6) / 1e9 / peak, "traffic": 4302000},
             "ha_score_topk (score_select_cluster_kernel<4,8>)": {"algorithmic_bytes": scan_bytes, "us": parts["ha_score_topk"],
