@@ -360,7 +360,7 @@ def main():
         "standalone_entry_points": {
             "ha_gather_attn (gather_cluster_kernel<4,8>)": {"algorithmic_bytes": gather_bytes, "us": g_us,
                                                       "achieved": gather_bytes / (g_us * 1e-6) / 1e9,
-                                                      "frac": gather_bytes / (g_us * 1e-6) / 1e9 / peak, "traffic": 4302000},
+                                                      "frac": gather_bytes / (g_us * 1e-6) / 1e9 / peak, "traffic": 4275000},
             "ha_score_topk (score_select_cluster_kernel<4,8>)": {"algorithmic_bytes": scan_bytes, "us": parts["ha_score_topk"],
                                                                     "achieved": scan_bytes / (parts["ha_score_topk"] * 1e-6) / 1e9},
             "ha_encode[q] (encode_vec_kernel<1>)": {"us": parts["ha_encode[q]"]},
