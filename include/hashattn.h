@@ -237,6 +237,19 @@ int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const 
                           int64_t idx_stride_h, int32_t *count, uint16_t *out_host,
                           void *workspace, size_t ws_bytes, void *stream);
 
+/* ha_sparse_decode_host over a paged K/V cache (pools + block table + page_size as in ha_gather_attn_paged): the
+ * new K/V rows of sequence b go to slot (seq_len - 1) % page_size of page block_table[b][(seq_len - 1) / page_size],
+ * which the caller must have allocated; everything else as ha_sparse_decode_host. */
+int ha_sparse_decode_paged_host(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
+                                const uint16_t *q_host, const uint16_t *k_new_host,
+                                const uint16_t *v_new_host, const ha_tensor *K_pool,
+                                const ha_tensor *V_pool, const int32_t *block_table, int64_t bt_stride_b,
+                                int32_t page_size, uint32_t *k_codes, int64_t kc_stride_b,
+                                int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
+                                int32_t k_uniform, int32_t max_seq_len, int32_t k_max, int32_t *idx,
+                                int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
+                                uint16_t *out_host, void *workspace, size_t ws_bytes, void *stream);
+
 /* GATHER-ATT without a caller-provided workspace.  (The paper has no counterpart of this entry
  * point; it exists for integration reasons only.)
  *

@@ -24,7 +24,7 @@ EXPORTS = [
     "ha_workspace_bytes", "ha_workspace_init", "ha_encode", "ha_encode_prefill", "ha_score_topk", "ha_gather_attn",
     "ha_gather_attn_paged", "ha_sparse_decode_paged",
     "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
-    "ha_score_wide", "ha_inner_products",
+    "ha_score_wide", "ha_inner_products", "ha_sparse_decode_paged_host",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
 
@@ -79,6 +79,8 @@ def lib() -> C.CDLL:
         L.ha_sparse_decode_host.argtypes = [P, P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64,
                                             P, P, P, SZ, P]
         L.ha_read_device_status.argtypes = [P, P, P]
+        L.ha_sparse_decode_paged_host.argtypes = [P, P, P, P, P, P, P, P, P, I64, I32, P, I64, I64, P, P, I32, I32, I32, P,
+                                                  I64, I64, P, P, P, SZ, P]
         L.ha_score_wide.argtypes = [P, P, I64, I32, P, P]
         L.ha_inner_products.argtypes = [P, P, I64, I64, P, P]
         L.ha_kernel_launches.restype = C.c_uint64
@@ -87,7 +89,8 @@ def lib() -> C.CDLL:
         L.ha_version.restype = C.c_char_p
         for fn in ("ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn", "ha_gather_attn_static", "ha_dense_decode",
                    "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status", "ha_score_wide",
-                   "ha_inner_products"):
+                   "ha_inner_products", "ha_sparse_decode_paged_host", "ha_sparse_decode_paged", "ha_gather_attn_paged",
+                   "ha_encode_prefill"):
             getattr(L, fn).restype = C.c_int
         _lib = L
     return _lib
@@ -320,6 +323,22 @@ def ha_sparse_decode_host(shape: ha_shape, map_q: Mapping, map_k: Mapping, q_hos
         C.byref(kt), C.byref(vt), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1), seq_lens.data_ptr(),
         _ptr(k_per_seq), k_uniform, max_seq_len, k_max, idx.data_ptr(), idx.stride(0), idx.stride(1),
         count.data_ptr(), out_host.data_ptr(), p, n, _stream(stream)))
+
+
+def ha_sparse_decode_paged_host(shape: ha_shape, map_q: Mapping, map_k: Mapping, q_host, k_new_host, v_new_host, K_pool,
+                                V_pool, block_table, page_size: int, k_codes, seq_lens, k_per_seq, k_uniform: int,
+                                max_seq_len: int, k_max: int, idx, count, out_host, workspace, stream=None) -> None:
+    """ha_sparse_decode_host over a paged K/V cache (pools bf16 [n_pages, Hkv, page_size, 128], block_table int32 [B, pages])."""
+    for t in (q_host, k_new_host, v_new_host, out_host):
+        if t.is_cuda or not t.is_contiguous():
+            raise TypeError("host buffers must be contiguous CPU tensors")
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K_pool), make_tensor(V_pool)
+    _check("ha_sparse_decode_paged_host", lib().ha_sparse_decode_paged_host(
+        C.byref(shape), map_q.ref, map_k.ref, q_host.data_ptr(), k_new_host.data_ptr(), v_new_host.data_ptr(),
+        C.byref(kt), C.byref(vt), block_table.data_ptr(), block_table.stride(0), page_size, k_codes.data_ptr(),
+        k_codes.stride(0), k_codes.stride(1), seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform, max_seq_len, k_max,
+        idx.data_ptr(), idx.stride(0), idx.stride(1), count.data_ptr(), out_host.data_ptr(), p, n, _stream(stream)))
 
 
 class SparseDecodeHostStep:

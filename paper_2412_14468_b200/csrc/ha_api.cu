@@ -330,13 +330,16 @@ int ha_sparse_decode_paged(const ha_shape *shape, const ha_mapping *map_q, const
                               idx_stride_b, idx_stride_h, count, out, lse, workspace, ws_bytes, stream);
 }
 
-int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
-                          const uint16_t *q_host, const uint16_t *k_new_host, const uint16_t *v_new_host,
-                          const ha_tensor *K, const ha_tensor *V, uint32_t *k_codes, int64_t kc_stride_b,
-                          int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
-                          int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
-                          int64_t idx_stride_h, int32_t *count, uint16_t *out_host, void *workspace, size_t ws_bytes,
-                          void *stream) {
+// Both host-buffer entries: block_table == NULL is the contiguous cache, else K / V are pools (page_shift = log2 of
+// the page size).
+static int sparse_decode_host_impl(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
+                                   const uint16_t *q_host, const uint16_t *k_new_host, const uint16_t *v_new_host,
+                                   const ha_tensor *K, const ha_tensor *V, const int32_t *block_table, int64_t bt_stride_b,
+                                   int page_shift, uint32_t *k_codes, int64_t kc_stride_b, int64_t kc_stride_h,
+                                   const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                                   int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
+                                   int64_t idx_stride_h, int32_t *count, uint16_t *out_host, void *workspace,
+                                   size_t ws_bytes, void *stream) {
     HA_TRY(check_shape(shape));
     if (!q_host || !k_new_host || !v_new_host || !out_host) return HA_ERR_INVALID_ARG;
     HA_TRY(check_tensor(K));
@@ -368,28 +371,63 @@ int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const 
     const uint16_t *mkn = reinterpret_cast<const uint16_t *>(mapped(k_new_host));
     const uint16_t *mvn = reinterpret_cast<const uint16_t *>(mapped(v_new_host));
     uint16_t *mout = reinterpret_cast<uint16_t *>(mapped(out_host));
-    if (mq && mkn && mvn && mout && fused_step_from_host_eligible(B, Hq, Hkv, max_seq_len, k_max)) {
+    if (!block_table && mq && mkn && mvn && mout && fused_step_from_host_eligible(B, Hq, Hkv, max_seq_len, k_max)) {
         // one launch: the fused kernel reads q / k_new / v_new across the bus, appends the new rows and writes `out`
         HA_TRY(sparse_decode_impl(shape, map_q, map_k, mq, mkn, K, V, nullptr, 0, 0, k_codes, kc_stride_b, kc_stride_h,
                                   seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx, idx_stride_b, idx_stride_h,
                                   count, mout, nullptr, workspace, ws_bytes, stream, mvn));
     } else if (mq && mkn && mvn && mout) {
-        HA_CUDA(launch_append_kv(B, Hq, Hkv, mkn, mvn, view(K), view(V), seq_lens, mq, dq, dk, st));
-        HA_TRY(ha_sparse_decode(shape, map_q, map_k, dq, dk, K, V, k_codes, kc_stride_b, kc_stride_h, seq_lens,
-                                k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx, idx_stride_b, idx_stride_h, count,
-                                mout, nullptr, workspace, ws_bytes, stream));
+        HA_CUDA(launch_append_kv(B, Hq, Hkv, mkn, mvn, view(K), view(V), seq_lens, mq, dq, dk, st, block_table, bt_stride_b,
+                                 page_shift));
+        HA_TRY(sparse_decode_impl(shape, map_q, map_k, dq, dk, K, V, block_table, bt_stride_b, page_shift, k_codes,
+                                  kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx,
+                                  idx_stride_b, idx_stride_h, count, mout, nullptr, workspace, ws_bytes, stream));
     } else {
         HA_CUDA(cudaMemcpyAsync(dq, q_host, (size_t)B * Hq * kD * 2, cudaMemcpyHostToDevice, st));
         HA_CUDA(cudaMemcpyAsync(dk, k_new_host, (size_t)B * Hkv * kD * 2, cudaMemcpyHostToDevice, st));
         HA_CUDA(cudaMemcpyAsync(dv, v_new_host, (size_t)B * Hkv * kD * 2, cudaMemcpyHostToDevice, st));
-        HA_CUDA(launch_append_kv(B, Hq, Hkv, dk, dv, view(K), view(V), seq_lens, nullptr, nullptr, nullptr, st));
-        HA_TRY(ha_sparse_decode(shape, map_q, map_k, dq, dk, K, V, k_codes, kc_stride_b, kc_stride_h, seq_lens,
-                                k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx, idx_stride_b, idx_stride_h, count,
-                                dout, nullptr, workspace, ws_bytes, stream));
+        HA_CUDA(launch_append_kv(B, Hq, Hkv, dk, dv, view(K), view(V), seq_lens, nullptr, nullptr, nullptr, st, block_table,
+                                 bt_stride_b, page_shift));
+        HA_TRY(sparse_decode_impl(shape, map_q, map_k, dq, dk, K, V, block_table, bt_stride_b, page_shift, k_codes,
+                                  kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, dqc, idx,
+                                  idx_stride_b, idx_stride_h, count, dout, nullptr, workspace, ws_bytes, stream));
         HA_CUDA(cudaMemcpyAsync(out_host, dout, (size_t)B * Hq * kD * 2, cudaMemcpyDeviceToHost, st));
     }
     HA_CUDA(cudaStreamSynchronize(st));
     return HA_OK;
+}
+
+int ha_sparse_decode_host(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
+                          const uint16_t *q_host, const uint16_t *k_new_host, const uint16_t *v_new_host,
+                          const ha_tensor *K, const ha_tensor *V, uint32_t *k_codes, int64_t kc_stride_b,
+                          int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                          int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
+                          int64_t idx_stride_h, int32_t *count, uint16_t *out_host, void *workspace, size_t ws_bytes,
+                          void *stream) {
+    return sparse_decode_host_impl(shape, map_q, map_k, q_host, k_new_host, v_new_host, K, V, nullptr, 0, 0, k_codes,
+                                   kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx,
+                                   idx_stride_b, idx_stride_h, count, out_host, workspace, ws_bytes, stream);
+}
+
+int ha_sparse_decode_paged_host(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
+                                const uint16_t *q_host, const uint16_t *k_new_host, const uint16_t *v_new_host,
+                                const ha_tensor *K_pool, const ha_tensor *V_pool, const int32_t *block_table,
+                                int64_t bt_stride_b, int32_t page_size, uint32_t *k_codes, int64_t kc_stride_b,
+                                int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
+                                int32_t k_uniform, int32_t max_seq_len, int32_t k_max, int32_t *idx,
+                                int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, uint16_t *out_host,
+                                void *workspace, size_t ws_bytes, void *stream) {
+    if (!block_table || !K_pool || !V_pool) return HA_ERR_INVALID_ARG;
+    if (page_size <= 0 || (page_size & (page_size - 1)) || page_size > 65536) return HA_ERR_INVALID_ARG;
+    if (K_pool->stride_n <= 0 || V_pool->stride_n <= 0 || K_pool->stride_b % K_pool->stride_n != 0 ||
+        V_pool->stride_b % V_pool->stride_n != 0 || K_pool->stride_b / K_pool->stride_n != V_pool->stride_b / V_pool->stride_n)
+        return HA_ERR_INVALID_ARG;
+    int shift = 0;
+    while ((1 << shift) < page_size) ++shift;
+    return sparse_decode_host_impl(shape, map_q, map_k, q_host, k_new_host, v_new_host, K_pool, V_pool, block_table,
+                                   bt_stride_b, shift, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
+                                   max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, out_host, workspace,
+                                   ws_bytes, stream);
 }
 
 int ha_score_wide(const uint64_t *q_code, const uint64_t *k_codes, int64_t n, int32_t n_bits, uint16_t *scores,

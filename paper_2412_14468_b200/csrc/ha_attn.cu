@@ -479,7 +479,8 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
 __global__ void append_kv_kernel(int Hq, int Hkv, const uint16_t *__restrict__ k_new,
                                  const uint16_t *__restrict__ v_new, TensorView K, TensorView V,
                                  const int32_t *__restrict__ seq_lens, const uint16_t *__restrict__ q_src,
-                                 uint16_t *__restrict__ q_dst, uint16_t *__restrict__ k_dst) {
+                                 uint16_t *__restrict__ q_dst, uint16_t *__restrict__ k_dst,
+                                 const int32_t *__restrict__ block_table, long long bt_sb, int page_shift, int page_rows) {
     const int g = blockIdx.x, b = blockIdx.y, t = threadIdx.x;   // 32 threads x 8 bytes per row
     const long long src = ((long long)b * Hkv + g) * kD;
     const uint2 kv = reinterpret_cast<const uint2 *>(k_new + src)[t];
@@ -494,16 +495,24 @@ __global__ void append_kv_kernel(int Hq, int Hkv, const uint16_t *__restrict__ k
     }
     const int slot = seq_lens[b] - 1;
     if (slot < 0) return;
-    uint16_t *kd = const_cast<uint16_t *>(K.ptr) + (long long)b * K.sb + (long long)g * K.sh + (long long)slot * K.sn;
-    uint16_t *vd = const_cast<uint16_t *>(V.ptr) + (long long)b * V.sb + (long long)g * V.sh + (long long)slot * V.sn;
+    // contiguous cache: row `slot` of sequence b; paged cache: the row of the pool that the block table names
+    long long base_b = b, row = slot;
+    if (block_table) {
+        base_b = 0;
+        row = (long long)block_table[(long long)b * bt_sb + (slot >> page_shift)] * page_rows + (slot & ((1 << page_shift) - 1));
+    }
+    uint16_t *kd = const_cast<uint16_t *>(K.ptr) + base_b * K.sb + (long long)g * K.sh + row * K.sn;
+    uint16_t *vd = const_cast<uint16_t *>(V.ptr) + base_b * V.sb + (long long)g * V.sh + row * V.sn;
     reinterpret_cast<uint2 *>(kd)[t] = kv;
     reinterpret_cast<uint2 *>(vd)[t] = vv;
 }
 
 cudaError_t launch_append_kv(int B, int Hq, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
                              TensorView V, const int32_t *seq_lens, const uint16_t *q_src, uint16_t *q_dst,
-                             uint16_t *k_dst, cudaStream_t st) {
-    append_kv_kernel<<<dim3(Hkv, B), 32, 0, st>>>(Hq, Hkv, k_new, v_new, K, V, seq_lens, q_src, q_dst, k_dst);
+                             uint16_t *k_dst, cudaStream_t st, const int32_t *block_table, long long bt_sb, int page_shift) {
+    const int page_rows = (block_table && K.sn > 0) ? (int)(K.sb / K.sn) : 0;
+    append_kv_kernel<<<dim3(Hkv, B), 32, 0, st>>>(Hq, Hkv, k_new, v_new, K, V, seq_lens, q_src, q_dst, k_dst, block_table,
+                                                  bt_sb, page_shift, page_rows);
     count_launch();
     return cudaGetLastError();
 }

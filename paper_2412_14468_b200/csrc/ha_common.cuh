@@ -217,6 +217,7 @@ cudaError_t launch_inner_products(const uint16_t *q, const uint16_t *K, long lon
 
 cudaError_t launch_append_kv(int B, int Hq, int Hkv, const uint16_t *k_new, const uint16_t *v_new, TensorView K,
                              TensorView V, const int32_t *seq_lens, const uint16_t *q_src, uint16_t *q_dst,
-                             uint16_t *k_dst, cudaStream_t st);
+                             uint16_t *k_dst, cudaStream_t st, const int32_t *block_table = nullptr, long long bt_sb = 0,
+                             int page_shift = 0);
 
 } // namespace ha

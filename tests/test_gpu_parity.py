@@ -597,6 +597,23 @@ def test_sparse_decode_step_over_a_paged_cache(cfg, page_size):
         assert ha.ha_read_device_status(ws) == 0
         assert torch.equal(idx, ref["idx"]) and torch.equal(cnt, ref["cnt"]) and torch.equal(qc, ref["qc"])
         assert torch.equal(out, ref["out"])
+        # The host-buffer entry over the same pools: the rows of the appended token are wiped first, the call has to
+        # put them back (into the right page and slot) and to give the same lists and outputs, from pinned and from
+        # pageable host buffers.
+        last = [(b, int(perm[b, (w["lens"][b] - 1) // page_size]), (w["lens"][b] - 1) % page_size) for b in range(B) if w["lens"][b] > 0]
+        for pinned in (True, False):
+            pk, pv = pools[0].clone(), pools[1].clone()
+            for (b, page, slot) in last:
+                pk[page, :, slot] = 0
+                pv[page, :, slot] = 0
+            pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+            hq, hk, hv = (pin(w[x].cpu()) for x in ("q", "k_new", "v_new"))
+            ho = pin(torch.zeros(B, Hq, 128, dtype=torch.bfloat16))
+            kc2, idx2, cnt2 = ref["kc"].clone(), torch.zeros_like(idx), torch.zeros_like(cnt)
+            ha.ha_sparse_decode_paged_host(shape, ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"]), hq, hk, hv, pk, pv, perm,
+                                           page_size, kc2, w["seq_lens"], w["k_per_seq"], 0, N, k_max, idx2, cnt2, ho, ws)
+            assert torch.equal(pk, pools[0]) and torch.equal(pv, pools[1])
+            assert torch.equal(idx2, ref["idx"]) and torch.equal(cnt2, ref["cnt"]) and torch.equal(ho.to(DEV), ref["out"])
 
 
 @pytest.mark.parametrize("seed", range(14))
