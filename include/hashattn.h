@@ -15,7 +15,7 @@
  *     as uint16_t bit patterns.  `stream` is a cudaStream_t passed as void* (NULL = legacy
  *     default stream).
  *   - Calls only enqueue work on `stream`: no host synchronisation and no allocation, except
- *     where stated (ha_read_device_status, ha_sparse_decode_host).
+ *     where stated (ha_read_device_status, ha_sparse_decode_host, ha_sparse_decode_paged_host).
  *   - Scratch memory is one caller-owned workspace of at least ha_workspace_bytes(...) bytes,
  *     256-byte aligned, prepared once with ha_workspace_init.  Calls that share a workspace must
  *     be ordered on one stream.
