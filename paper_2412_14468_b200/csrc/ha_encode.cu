@@ -207,38 +207,62 @@ cudaError_t launch_encode_vectors(const EncodeJob &a_in, const EncodeJob &b_in, 
 
 // ------------------------------------------------------------------ token-tiled bulk kernel
 
-constexpr int kTile = 64;             // tokens per CTA
-constexpr int kBulkThreads = 256;
+constexpr int kTile = 128;            // tokens per CTA
+constexpr int kBulkThreads = 512;
 constexpr int kActLd = kD + 4;        // padded row of the activation tile (floats)
 constexpr size_t kBulkSmem = (size_t)(kD * kHid + kHid * kHid + kHid * kBits) * 2   // bf16 weights
                              + (size_t)2 * kTile * kActLd * 4;                    // two activation tiles
 
-// One hidden layer for a 64-token tile: thread (o, half) owns output o of 32 tokens.
+// One hidden layer for a 64-token tile: thread (oq, tg) owns the four outputs 4 oq .. 4 oq + 3 of the eight tokens
+// 8 tg .. 8 tg + 7 (32 independent chains).  Per four terms a thread reads four 8-byte weight groups and eight
+// 16-byte activation groups (a warp = the 32 output groups of one token group: the activations are broadcasts)
+// for 128 fmas, which leaves the layer bound by the fp32 pipe, not by shared memory.
 __device__ __forceinline__ void bulk_hidden_layer(const float *__restrict__ in, float *__restrict__ out,
-                                                  const uint16_t *__restrict__ w, const float *bias, int o,
-                                                  int half) {
-    float z[32];
-    const float b = bias ? bias[o] : 0.0f;
+                                                  const uint16_t *__restrict__ w, const float *bias, int oq, int tg) {
+    float z[8][4];
+    {
+        float b4[4];
 #pragma unroll
-    for (int t = 0; t < 32; ++t) z[t] = b;
-    const float *hin = in + (size_t)half * 32 * kActLd;
+        for (int j = 0; j < 4; ++j) b4[j] = bias ? bias[4 * oq + j] : 0.0f;
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) z[t][j] = b4[j];
+    }
+    const float *hin = in + (size_t)tg * 8 * kActLd;
+#pragma unroll 4
     for (int k = 0; k < 128; k += 4) {
-        const float w0 = bf16_bits_to_float(w[(k + 0) * kHid + o]);
-        const float w1 = bf16_bits_to_float(w[(k + 1) * kHid + o]);
-        const float w2 = bf16_bits_to_float(w[(k + 2) * kHid + o]);
-        const float w3 = bf16_bits_to_float(w[(k + 3) * kHid + o]);
+        float wf[4][4];   // [term][output]
 #pragma unroll
-        for (int t = 0; t < 32; ++t) {
+        for (int i = 0; i < 4; ++i) {
+            const uint2 wv = *reinterpret_cast<const uint2 *>(w + (k + i) * kHid + 4 * oq);
+            wf[i][0] = __uint_as_float(wv.x << 16);
+            wf[i][1] = __uint_as_float(wv.x & 0xffff0000u);
+            wf[i][2] = __uint_as_float(wv.y << 16);
+            wf[i][3] = __uint_as_float(wv.y & 0xffff0000u);
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
             const float4 hv = *reinterpret_cast<const float4 *>(hin + t * kActLd + k);   // warp broadcast
-            z[t] = __fmaf_rn(hv.x, w0, z[t]);
-            z[t] = __fmaf_rn(hv.y, w1, z[t]);
-            z[t] = __fmaf_rn(hv.z, w2, z[t]);
-            z[t] = __fmaf_rn(hv.w, w3, z[t]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {   // ascending term index within every chain
+                z[t][j] = __fmaf_rn(hv.x, wf[0][j], z[t][j]);
+                z[t][j] = __fmaf_rn(hv.y, wf[1][j], z[t][j]);
+                z[t][j] = __fmaf_rn(hv.z, wf[2][j], z[t][j]);
+                z[t][j] = __fmaf_rn(hv.w, wf[3][j], z[t][j]);
+            }
         }
     }
-    float *hout = out + (size_t)half * 32 * kActLd;
+    float *hout = out + (size_t)tg * 8 * kActLd + 4 * oq;
 #pragma unroll
-    for (int t = 0; t < 32; ++t) hout[t * kActLd + o] = (z[t] > 0.0f) ? z[t] : 0.0f;
+    for (int t = 0; t < 8; ++t) {
+        float4 r;
+        r.x = (z[t][0] > 0.0f) ? z[t][0] : 0.0f;
+        r.y = (z[t][1] > 0.0f) ? z[t][1] : 0.0f;
+        r.z = (z[t][2] > 0.0f) ? z[t][2] : 0.0f;
+        r.w = (z[t][3] > 0.0f) ? z[t][3] : 0.0f;
+        *reinterpret_cast<float4 *>(hout + t * kActLd) = r;
+    }
 }
 
 __global__ void __launch_bounds__(kBulkThreads) encode_bulk_kernel(MapView map, int heads_per_kv, TensorView x,
@@ -283,39 +307,57 @@ __global__ void __launch_bounds__(kBulkThreads) encode_bulk_kernel(MapView map, 
     }
     __syncthreads();
 
-    const int o = tid & 127, half = tid >> 7;
-    bulk_hidden_layer(actA, actB, sw1, map.b1 ? map.b1 + net * kHid : nullptr, o, half);
+    const int oq = tid & 31, tg = tid >> 5;   // a warp: the 32 groups of four outputs, for one group of eight tokens
+    bulk_hidden_layer(actA, actB, sw1, map.b1 ? map.b1 + net * kHid : nullptr, oq, tg);
     __syncthreads();
-    bulk_hidden_layer(actB, actA, sw2, map.b2 ? map.b2 + net * kHid : nullptr, o, half);
+    bulk_hidden_layer(actB, actA, sw2, map.b2 ? map.b2 + net * kHid : nullptr, oq, tg);
     __syncthreads();
 
-    // last layer: lane = output bit, warp w owns tokens 8w .. 8w+7
+    // last layer: thread (op, tq) owns outputs 2 op, 2 op + 1 of the four tokens 4 tq .. 4 tq + 3; a half-warp
+    // holds the 16 output pairs of one token group, so two ballots per token collect its 32 sign bits
     {
-        const int lane = tid & 31, w = tid >> 5;
-        float z[8];
-        const float bb = map.b3 ? map.b3[net * kBits + lane] : 0.0f;
+        const int lane = tid & 31, op = tid & 15, tq = tid >> 4;
+        float z[4][2];
+        const float b0 = map.b3 ? map.b3[net * kBits + 2 * op] : 0.0f, b1 = map.b3 ? map.b3[net * kBits + 2 * op + 1] : 0.0f;
 #pragma unroll
-        for (int t = 0; t < 8; ++t) z[t] = bb;
-        const float *hin = actA + (size_t)w * 8 * kActLd;
+        for (int t = 0; t < 4; ++t) { z[t][0] = b0; z[t][1] = b1; }
+        const float *hin = actA + (size_t)tq * 4 * kActLd;
+#pragma unroll 4
         for (int k = 0; k < 128; k += 4) {
-            const float w0 = bf16_bits_to_float(sw3[(k + 0) * kBits + lane]);
-            const float w1 = bf16_bits_to_float(sw3[(k + 1) * kBits + lane]);
-            const float w2 = bf16_bits_to_float(sw3[(k + 2) * kBits + lane]);
-            const float w3 = bf16_bits_to_float(sw3[(k + 3) * kBits + lane]);
+            float wf[4][2];
 #pragma unroll
-            for (int t = 0; t < 8; ++t) {
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t wv = *reinterpret_cast<const uint32_t *>(sw3 + (k + i) * kBits + 2 * op);
+                wf[i][0] = __uint_as_float(wv << 16);
+                wf[i][1] = __uint_as_float(wv & 0xffff0000u);
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
                 const float4 hv = *reinterpret_cast<const float4 *>(hin + t * kActLd + k);
-                z[t] = __fmaf_rn(hv.x, w0, z[t]);
-                z[t] = __fmaf_rn(hv.y, w1, z[t]);
-                z[t] = __fmaf_rn(hv.z, w2, z[t]);
-                z[t] = __fmaf_rn(hv.w, w3, z[t]);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    z[t][j] = __fmaf_rn(hv.x, wf[0][j], z[t][j]);
+                    z[t][j] = __fmaf_rn(hv.y, wf[1][j], z[t][j]);
+                    z[t][j] = __fmaf_rn(hv.z, wf[2][j], z[t][j]);
+                    z[t][j] = __fmaf_rn(hv.w, wf[3][j], z[t][j]);
+                }
             }
         }
         uint32_t *cb = codes + (long long)b * c_sb + (long long)h * c_sh + t0;
+        auto spread16 = [](uint32_t v) {   // bit i -> bit 2 i
+            v = (v | (v << 8)) & 0x00ff00ffu;
+            v = (v | (v << 4)) & 0x0f0f0f0fu;
+            v = (v | (v << 2)) & 0x33333333u;
+            v = (v | (v << 1)) & 0x55555555u;
+            return v;
+        };
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const uint32_t code = __ballot_sync(0xffffffffu, z[t] > 0.0f);
-            if (lane == 0 && w * 8 + t < nt) cb[w * 8 + t] = code;
+        for (int t = 0; t < 4; ++t) {
+            const uint32_t even = __ballot_sync(0xffffffffu, z[t][0] > 0.0f), odd = __ballot_sync(0xffffffffu, z[t][1] > 0.0f);
+            const int shift = lane & 16;   // this half-warp's 16 bits of either ballot
+            const uint32_t code = spread16((even >> shift) & 0xffffu) | (spread16((odd >> shift) & 0xffffu) << 1);
+            const int tok = tq * 4 + t;
+            if (op == 0 && tok < nt) cb[tok] = code;
         }
     }
 }
