@@ -29,10 +29,13 @@ def prefill(args):
     codes = torch.zeros(B, Hkv, T, dtype=torch.int32, device=dev)
     torch.cuda.synchronize()
     for s in range(args.steps):
-        for name, path in (("tcgen05", ha.HA_PREFILL_TCGEN05), ("mma.sync", ha.HA_PREFILL_MMA_SYNC)):
+        for name, path in (("tcgen05", ha.HA_PREFILL_TCGEN05), ("mma.sync", ha.HA_PREFILL_MMA_SYNC), ("chain-exact fp32", None)):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            ha.ha_encode_prefill(mp, 1, x, codes, path=path)
+            if path is None:
+                ha.ha_encode(mp, 1, x, codes)             # encode_bulk_kernel: the fma chain of the decode step
+            else:
+                ha.ha_encode_prefill(mp, 1, x, codes, path=path)
             e1.record()
             torch.cuda.synchronize()
             print(f"step {s} {name}: {e0.elapsed_time(e1) * 1e3:.1f} us")
