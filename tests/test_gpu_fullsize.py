@@ -24,11 +24,13 @@ DEV = "cuda"
 SWEEP = {f"sweep_B{bsz}_32K_32x": wl.Config(f"sweep{bsz}", 10 + bsz, bsz, 32768, 1024, 0.01) for bsz in (4, 8)}
 
 
-def _run(cfg_name):
+def _run(cfg_name, n_sink=0, n_local=0):
     w = wl.make_workload(SWEEP.get(cfg_name, cfg_name), DEV)
+    if n_sink or n_local:
+        w = dict(w, k_max=w["k_max"] + n_sink + n_local)      # the index rows hold the always-kept tokens too
     cfg = w["cfg"]
     B, Hq, Hkv = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads
-    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"], n_sink=n_sink, n_local=n_local)
     ws = ha.alloc_workspace(shape, w["n_cap"], w["k_max"])
     mq, mk = ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"])
     kc = torch.zeros(B, Hkv, (w["n_cap"] + 3) // 4 * 4, dtype=torch.int32, device=DEV)
@@ -52,11 +54,13 @@ def _run(cfg_name):
     return w, dict(kc=kc, qc=qc, idx=idx, cnt=cnt, out=out, lse=lse, hist=hist, shape=shape, ws=ws)
 
 
-@pytest.mark.parametrize("cfg_name", ["c2", "c3", "c4", "c5", "sweep_B4_32K_32x", "sweep_B8_32K_32x"])
+@pytest.mark.parametrize("cfg_name", ["c2", "c3", "c4", "c5", "sweep_B4_32K_32x", "sweep_B8_32K_32x", "c2+sink128+local128"])
 def test_full_size_config_matches_oracle(cfg_name):
     import time
     t_start = time.time()
-    w, r = _run(cfg_name)
+    n_sink, n_local = (128, 128) if cfg_name.endswith("+sink128+local128") else (0, 0)   # the bench's window line
+    cfg_name = cfg_name.split("+")[0]
+    w, r = _run(cfg_name, n_sink, n_local)
     t_gpu = time.time() - t_start
     cfg = w["cfg"]
     B, Hq, Hkv = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads
@@ -81,9 +85,12 @@ def test_full_size_config_matches_oracle(cfg_name):
         n, k = w["lens"][b], w["ks"][b]
         for g in range(Hkv):
             s = oracle.score(qc_np[b, g * G:(g + 1) * G], kc_np[b, g, :n])
-            assert np.array_equal(hist_np[b, g], np.bincount(s, minlength=33)), (b, g)
-            exp = oracle.topk(s, k)
-            assert cnt_np[b, g] == len(exp) == min(k, n)
+            counted = s[n_sink:max(n - n_local, n_sink)]               # always-kept tokens are not counted
+            assert np.array_equal(hist_np[b, g], np.bincount(counted, minlength=33)), (b, g)
+            exp = oracle.topk_windows(s, k, n_sink, n_local) if (n_sink or n_local) else oracle.topk(s, k)
+            assert cnt_np[b, g] == len(exp)
+            if not (n_sink or n_local):
+                assert len(exp) == min(k, n)
             assert np.array_equal(idx_np[b, g, :len(exp)], exp), (b, g)
             assert np.all(idx_np[b, g, len(exp):] == -1)
 
