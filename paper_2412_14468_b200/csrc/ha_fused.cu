@@ -569,7 +569,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
 // ------------------------------------------------------------------ stand-alone GATHER-ATT with clusters
 //
 // ha_gather_attn for few units and short lists: the attention phase of the fused step on a list that the caller
-// provides (one cluster of 8 CTAs per (sequence, KV head), each CTA an eighth of the list, states merged in
+// provides (one cluster of 8 or 4 CTAs per (sequence, KV head), each CTA its share of the list, states merged in
 // CTA 0's shared memory), instead of the persistent split-K kernel whose work split and global-memory merge cost
 // more than the attention itself at this size.
 __host__ __device__ constexpr int gather_cluster_smem_bytes(int G, int CS) { return fused_ring_bytes(1) + fused_part_bytes(G, CS); }
@@ -601,68 +601,83 @@ __global__ void __launch_bounds__(kFusedThreads, 2) gather_cluster_kernel(const 
     if (bad) atomicOr(a.status, HA_DEV_BAD_INDEX);
 }
 
-template <int G>
-static int gather_cluster_prepare() {
-    static int clusters[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64) dev = 0;
-    if (!clusters[dev]) {
-        constexpr int smem = gather_cluster_smem_bytes(G, 8);
-        if (cudaFuncSetAttribute(gather_cluster_kernel<G, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-            return 0;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(8, 1, 64);
-        cfg.blockDim = dim3(kFusedThreads);
-        cfg.dynamicSmemBytes = smem;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 8;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, gather_cluster_kernel<G, 8>, &cfg) != cudaSuccess || n <= 0) return 0;
-        clusters[dev] = n;
-    }
-    return clusters[dev];
-}
-
-// Lists of up to 2048 entries (at most two blocks per warp) and as many units as clusters are resident at once.
-bool gather_cluster_eligible(int B, int Hq, int Hkv, int k_max) {
-    if (Hkv <= 0 || k_max > kFusedOneStageMaxK) return false;
-    const long long units = (long long)B * Hkv;
-    switch (Hq / Hkv) {
-        case 1: return units <= gather_cluster_prepare<1>();
-        case 2: return units <= gather_cluster_prepare<2>();
-        case 4: return units <= gather_cluster_prepare<4>();
-        case 8: return units <= gather_cluster_prepare<8>();
-        default: return false;
-    }
-}
-
-template <int G>
-static cudaError_t launch_gather_cluster_g(const FusedArgs &args, int B, cudaStream_t st) {
-    if (gather_cluster_prepare<G>() <= 0) return cudaErrorInvalidConfiguration;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(8, args.Hkv, B);
+template <int G, int CS>
+static void gather_cluster_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute (&attr)[2], int Hkv, int B, cudaStream_t st) {
+    cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = dim3(CS, Hkv, B);
     cfg.blockDim = dim3(kFusedThreads);
-    cfg.dynamicSmemBytes = gather_cluster_smem_bytes(G, 8);
+    cfg.dynamicSmemBytes = gather_cluster_smem_bytes(G, CS);
     cfg.stream = st;
-    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 8;
+    attr[0].val.clusterDim.x = CS;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gather_cluster_kernel<G, 8>, args);
+}
+
+// Opt in to the shared-memory carve-out (once per device); returns how many clusters the device holds at once.
+template <int G, int CS>
+static int gather_cluster_prepare() {
+    static int clusters[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) dev = 0;
+    if (!clusters[dev]) {
+        if (cudaFuncSetAttribute(gather_cluster_kernel<G, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 gather_cluster_smem_bytes(G, CS)) != cudaSuccess)
+            return 0;
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attr[2];
+        gather_cluster_config<G, CS>(cfg, attr, 1, 64, nullptr);
+        cfg.numAttrs = 1;   // the cluster shape is all the occupancy query looks at
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gather_cluster_kernel<G, CS>, &cfg) != cudaSuccess || n <= 0) return 0;
+        clusters[dev] = n;
+    }
+    return clusters[dev];
+}
+
+// Cluster size for `units` units: 8 while that many clusters are resident at once, else 4, else 0 (not eligible).
+template <int G>
+static int gather_cluster_size(long long units) {
+    if (units <= gather_cluster_prepare<G, 8>()) return 8;
+    if (units <= gather_cluster_prepare<G, 4>()) return 4;
+    return 0;
+}
+
+// Lists of up to 2048 entries (a few blocks per warp) and as many units as clusters are resident at once.
+bool gather_cluster_eligible(int B, int Hq, int Hkv, int k_max) {
+    if (Hkv <= 0 || k_max > kFusedOneStageMaxK) return false;
+    const long long units = (long long)B * Hkv;
+    switch (Hq / Hkv) {
+        case 1: return gather_cluster_size<1>(units) > 0;
+        case 2: return gather_cluster_size<2>(units) > 0;
+        case 4: return gather_cluster_size<4>(units) > 0;
+        case 8: return gather_cluster_size<8>(units) > 0;
+        default: return false;
+    }
+}
+
+template <int G, int CS>
+static cudaError_t launch_gather_cluster_gc(const FusedArgs &args, int B, cudaStream_t st) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    gather_cluster_config<G, CS>(cfg, attr, args.Hkv, B, st);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gather_cluster_kernel<G, CS>, args);
     if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
+}
+
+template <int G>
+static cudaError_t launch_gather_cluster_g(const FusedArgs &args, int B, cudaStream_t st) {
+    const int cs = gather_cluster_size<G>((long long)B * args.Hkv);
+    if (cs == 8) return launch_gather_cluster_gc<G, 8>(args, B, st);
+    if (cs == 4) return launch_gather_cluster_gc<G, 4>(args, B, st);
+    return cudaErrorInvalidConfiguration;
 }
 
 cudaError_t launch_gather_cluster(int B, int Hq, int Hkv, float sm_scale, const uint16_t *q, TensorView K, TensorView V,

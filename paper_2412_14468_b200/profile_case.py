@@ -114,6 +114,9 @@ def main():
     ap.add_argument("--entry-points", action="store_true",
                     help="run the step as its separate entry points (ha_encode, ha_score_topk, ha_gather_attn), i.e. the "
                          "kernels of the three-kernel path, also at batch sizes where ha_sparse_decode is one fused launch")
+    ap.add_argument("--wide-index-rows", action="store_true",
+                    help="with --entry-points: index rows one entry wider than the budget, which makes ha_gather_attn take "
+                         "its split-K kernel also where few units with short rows would get the cluster kernel")
     ap.add_argument("--score-only", action="store_true",
                     help="SCORE + TOPK alone on random signatures (no K/V allocated: large batches stay small)")
     ap.add_argument("--score-wide", action="store_true",
@@ -139,7 +142,8 @@ def main():
     kc = torch.zeros(B, Hkv, (w["n_cap"] + 3) // 4 * 4, dtype=torch.int32, device=dev)
     ha.ha_encode(mk, 1, w["K"], kc)
     qc = torch.zeros(B, Hq, dtype=torch.int32, device=dev)
-    idx = torch.zeros(B, Hkv, w["k_max"], dtype=torch.int32, device=dev)
+    row_width = w["k_max"] + (2049 - w["k_max"] if args.wide_index_rows and w["k_max"] <= 2048 else 0)
+    idx = torch.zeros(B, Hkv, row_width, dtype=torch.int32, device=dev)
     cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
     out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=dev)
     flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
@@ -153,7 +157,7 @@ def main():
             ha.ha_encode(mq, Hq // Hkv, w["q"], qc.view(B, Hq, 1))
             ha.ha_encode(mk, 1, w["k_new"], kc, slot=last_slot)
             ha.ha_score_topk(shape, qc, kc, w["seq_lens"], w["k_per_seq"], 0, w["n_cap"], w["k_max"], idx, cnt, ws)
-            ha.ha_gather_attn(shape, w["q"], w["K"], w["V"], w["seq_lens"], idx, cnt, w["k_max"], out, ws)
+            ha.ha_gather_attn(shape, w["q"], w["K"], w["V"], w["seq_lens"], idx, cnt, row_width, out, ws)
         else:
             ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
                                 w["n_cap"], w["k_max"], qc, idx, cnt, out, ws)

@@ -346,6 +346,30 @@ def test_gather_attn_random_lists(G, k_max):
     _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128))
 
 
+def test_gather_attn_forty_units_take_clusters_of_four():
+    """34 to 71 units with short lists: the stand-alone gather runs one cluster of 4 CTAs per unit (several blocks per
+    warp, one after the other); random lists with padding inside, duplicates, and one index outside its sequence."""
+    B, Hkv, G, n_cap, k_max = 20, 2, 4, 2500, 900
+    Hq = Hkv * G
+    rng = np.random.default_rng(77)
+    lens = [int(v) for v in rng.integers(1, n_cap + 1, size=B)]
+    q, K, V = _attn_inputs(B, Hq, Hkv, n_cap, 78)
+    idx = np.full((B, Hkv, k_max), -1, np.int32)
+    cnt = np.zeros((B, Hkv), np.int32)
+    for b in range(B):
+        for g in range(Hkv):
+            c = int(rng.integers(0, k_max + 1))
+            cnt[b, g] = c
+            idx[b, g, :c] = rng.integers(0, lens[b], size=c)
+            idx[b, g, :c][rng.random(c) < 0.05] = -1
+    before = ha.ha_kernel_launches()
+    _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128))
+    assert ha.ha_kernel_launches() - before == 1
+    idx[7, 1, 0] = lens[7]                       # one entry past the end of its sequence: skipped and flagged
+    cnt[7, 1] = max(cnt[7, 1], 1)
+    _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128), expect_flag=ha.HA_DEV_BAD_INDEX)
+
+
 @pytest.mark.parametrize("width", [64, 2100])   # both stand-alone gather kernels (see test_gather_attn_random_lists)
 def test_gather_attn_padding_invalid_and_unsorted_indices(width):
     Hq, Hkv, n_cap = 8, 2, 500
