@@ -292,6 +292,13 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
                               max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, nullptr,
                               ws_ptr<int32_t>(workspace, L.off_hist), ws_ptr<unsigned char>(workspace, L.off_scores), st,
                               Windows{shape->n_sink, shape->n_local}));
+    if (gather_cluster_eligible(B, Hq, Hkv, k_max)) {
+        // up to a cluster per unit resident at once and short lists: GATHER-ATT with the states merged in shared memory
+        HA_CUDA(launch_gather_cluster(B, Hq, Hkv, shape->sm_scale, q, view(K), view(V), seq_lens, idx, idx_stride_b,
+                                      idx_stride_h, count, k_max, out, lse, ws_ptr<uint32_t>(workspace, 0), st, block_table,
+                                      bt_stride_b, page_shift));
+        return HA_OK;
+    }
     HA_CUDA(launch_attention(true, B, Hq, Hkv, shape->sm_scale, q, view(K), view(V), seq_lens, idx, idx_stride_b,
                              idx_stride_h, count, k_max, out, lse, ws_ptr<float>(workspace, L.off_part_ml),
                              ws_ptr<float>(workspace, L.off_part_acc), ws_ptr<int32_t>(workspace, L.off_tickets),

@@ -569,7 +569,7 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
 // ------------------------------------------------------------------ stand-alone GATHER-ATT with clusters
 //
 // ha_gather_attn for few units and short lists: the attention phase of the fused step on a list that the caller
-// provides (one cluster of 8 or 4 CTAs per (sequence, KV head), each CTA its share of the list, states merged in
+// provides (one cluster of 8, 4 or 2 CTAs per (sequence, KV head), each CTA its share of the list, states merged in
 // CTA 0's shared memory), instead of the persistent split-K kernel whose work split and global-memory merge cost
 // more than the attention itself at this size.
 __host__ __device__ constexpr int gather_cluster_smem_bytes(int G, int CS) { return fused_ring_bytes(1) + fused_part_bytes(G, CS); }
@@ -640,11 +640,14 @@ static int gather_cluster_prepare() {
     return clusters[dev];
 }
 
-// Cluster size for `units` units: 8 while that many clusters are resident at once, else 4, else 0 (not eligible).
+// Cluster size for `units` units: 8 while that many clusters are resident at once, else 4, else 2, else 0 (not
+// eligible).  Unlike the fused step, whose clusters of 2 lose to the three-kernel path, the attention phase alone
+// beats the split-K kernel at every cluster size (c3: 27.7 against 32.0 us with 128 clusters of 2).
 template <int G>
 static int gather_cluster_size(long long units) {
     if (units <= gather_cluster_prepare<G, 8>()) return 8;
     if (units <= gather_cluster_prepare<G, 4>()) return 4;
+    if (units <= gather_cluster_prepare<G, 2>()) return 2;
     return 0;
 }
 
@@ -677,6 +680,7 @@ static cudaError_t launch_gather_cluster_g(const FusedArgs &args, int B, cudaStr
     const int cs = gather_cluster_size<G>((long long)B * args.Hkv);
     if (cs == 8) return launch_gather_cluster_gc<G, 8>(args, B, st);
     if (cs == 4) return launch_gather_cluster_gc<G, 4>(args, B, st);
+    if (cs == 2) return launch_gather_cluster_gc<G, 2>(args, B, st);
     return cudaErrorInvalidConfiguration;
 }
 

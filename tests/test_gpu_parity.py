@@ -346,10 +346,12 @@ def test_gather_attn_random_lists(G, k_max):
     _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128))
 
 
-def test_gather_attn_forty_units_take_clusters_of_four():
-    """34 to 71 units with short lists: the stand-alone gather runs one cluster of 4 CTAs per unit (several blocks per
-    warp, one after the other); random lists with padding inside, duplicates, and one index outside its sequence."""
-    B, Hkv, G, n_cap, k_max = 20, 2, 4, 2500, 900
+@pytest.mark.parametrize("B", [20, 50])
+def test_gather_attn_with_smaller_clusters(B):
+    """34 to 71 units with short lists: the stand-alone gather runs one cluster of 4 CTAs per unit, up to 148 units one
+    of 2 (several blocks per warp, one after the other); random lists with padding inside, duplicates, and one index
+    outside its sequence."""
+    Hkv, G, n_cap, k_max = 2, 4, 2500, 900
     Hq = Hkv * G
     rng = np.random.default_rng(77)
     lens = [int(v) for v in rng.integers(1, n_cap + 1, size=B)]
