@@ -75,6 +75,15 @@ def score(qcodes, kcodes) -> np.ndarray:
     return out
 
 
+def score_sum(qcodes, kcodes) -> np.ndarray:
+    """Eq. 1 per query code, summed over the query codes of one GQA group (range 0 .. 32 * group)."""
+    qcodes = np.ascontiguousarray(qcodes, dtype=np.uint32).reshape(-1)
+    kcodes = np.ascontiguousarray(kcodes, dtype=np.uint32).reshape(-1)
+    out = np.zeros(kcodes.shape[0], dtype=np.int32)
+    lib().ora_score_sum(_p(qcodes), C.c_int32(qcodes.shape[0]), _p(kcodes), C.c_int64(kcodes.shape[0]), _p(out))
+    return out
+
+
 def score_wide(qcode, kcodes) -> np.ndarray:
     """Score of the SCORE-latency table: b - Hamming for signatures of b = 64 * W bits, kcodes uint64 [n, W]."""
     qcode = np.ascontiguousarray(qcode, dtype=np.uint64).reshape(-1)

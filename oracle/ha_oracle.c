@@ -17,6 +17,9 @@
  *                    (Section 4.1), reported as 32 - Hamming distance; for grouped-query
  *                    attention the group score is the maximum over the query heads that
  *                    share the KV head (reduces to Eq. 1 when the group has one head).
+ *   ora_score_sum    the other way to reduce Eq. 1 over a group (an option of ha_score_topk_grouped,
+ *                    not of the layer-step): the per-head scores added up, 0 .. 32 G; the score
+ *                    of the G query signatures concatenated against the key signature repeated.
  *   ora_score_wide   the same score for a signature of b = 64 .. 512 bits kept as b/64 packed
  *                    64-bit integers (the setting of the SCORE-latency table, "Latency of
  *                    SCORE computation"): b - Hamming distance, one query signature against n
@@ -39,7 +42,7 @@
  * Pins (tests/test_oracle_*.py): closed forms (identity / zero weights, single token,
  * zero query), hand-derived fixtures in tests/golden/, an O(n^2) rank definition of
  * top-k, bit-level brute force for the score, the +-1 inner-product identity and the 32-bit
- * score for the wide score, float64 numpy for the mapping net and the inner products, and
+ * score for the wide score, concatenated signatures and the +-1 identity for the summed score, float64 numpy for the mapping net and the inner products, and
  * torch's scaled_dot_product_attention in float64 for the attention.
  * The fp32 accumulation ORDER inside ora_encode is a definition of this build, not of
  * the paper: it is pinned only up to the float64 margin test ("parity unpinned" for
@@ -154,6 +157,18 @@ void ora_score(const uint32_t *qcodes, int32_t group, const uint32_t *kcodes, in
             if (s > best) best = s;
         }
         scores[i] = best;
+    }
+}
+
+/* Alternative reduction over a GQA group: scores[i] = sum over the group's query codes of
+ * (32 - Hamming(kcodes[i], qcodes[j])), i.e. Eq. 1 per query head added up; range 0 .. 32 * group.
+ * The paper defines the score for one query head only; with group = 1 this is Eq. 1 itself. */
+void ora_score_sum(const uint32_t *qcodes, int32_t group, const uint32_t *kcodes, int64_t n,
+                   int32_t *scores) {
+    for (int64_t i = 0; i < n; ++i) {
+        int total = 0;
+        for (int j = 0; j < group; ++j) total += HA_BITS - hamming32(kcodes[i], qcodes[j]);
+        scores[i] = total;
     }
 }
 
