@@ -160,6 +160,21 @@ int ha_score_topk(const ha_shape *shape, const uint32_t *q_codes, const uint32_t
                   int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
                   int32_t *hist_out, void *workspace, size_t ws_bytes, void *stream);
 
+/* SCORE + TOPK with the other reduction over a GQA group: the per-head scores of Eq. 1 (as 32 - bitcount(k_code
+ * xor q_code), Section 4.1) ADDED over the G query heads of the KV head, range 0 .. 32 G, then the standard top-k
+ * of Section 4 with ties towards the lowest token index.  The paper defines the score for one query head; the
+ * layer-step (ha_sparse_decode, ha_score_topk) takes the maximum over the group, this entry is the stand-alone
+ * alternative and equals ha_score_topk when G = 1.  Arguments, layouts, windows (shape->n_sink / n_local) and
+ * the idx / count outputs as in ha_score_topk; no workspace and no maximum sequence length are needed (any
+ * seq_len >= 0), and
+ *   hist_out   optional out i32 [batch][n_kv_heads][32 G + 1]: histogram of the summed scores (windows excluded).
+ * The index lists feed ha_gather_attn unchanged. */
+int ha_score_topk_sum(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes,
+                      int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens,
+                      const int32_t *k_per_seq, int32_t k_uniform, int32_t k_max, int32_t *idx,
+                      int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, int32_t *hist_out,
+                      void *stream);
+
 /* GATHER-ATT — Section 4: out_j = sum_{i in I} softmax_I(sm_scale <q_j, k_i>) v_i for every
  * query head j, I = idx[b][j / G][0..count).  K/V rows are read in place through the indices
  * (Section 4.4).  fp32 accumulation, one rounding to bf16.

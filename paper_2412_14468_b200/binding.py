@@ -24,7 +24,7 @@ EXPORTS = [
     "ha_workspace_bytes", "ha_workspace_init", "ha_encode", "ha_encode_prefill", "ha_score_topk", "ha_gather_attn",
     "ha_gather_attn_paged", "ha_sparse_decode_paged",
     "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
-    "ha_score_wide", "ha_inner_products", "ha_sparse_decode_paged_host",
+    "ha_score_wide", "ha_inner_products", "ha_sparse_decode_paged_host", "ha_score_topk_sum",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
 
@@ -68,6 +68,7 @@ def lib() -> C.CDLL:
         L.ha_encode.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, P, P]
         L.ha_encode_prefill.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, I32, P, P]
         L.ha_score_topk.argtypes = [P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64, P, P, P, SZ, P]
+        L.ha_score_topk_sum.argtypes = [P, P, P, I64, I64, P, P, I32, I32, P, I64, I64, P, P, P]
         L.ha_gather_attn.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P, SZ, P]
         L.ha_gather_attn_paged.argtypes = [P, P, P, P, P, I64, I32, P, P, I64, I64, P, I32, P, P, P, SZ, P]
         L.ha_gather_attn_static.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P]
@@ -90,7 +91,7 @@ def lib() -> C.CDLL:
         for fn in ("ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn", "ha_gather_attn_static", "ha_dense_decode",
                    "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status", "ha_score_wide",
                    "ha_inner_products", "ha_sparse_decode_paged_host", "ha_sparse_decode_paged", "ha_gather_attn_paged",
-                   "ha_encode_prefill"):
+                   "ha_encode_prefill", "ha_score_topk_sum"):
             getattr(L, fn).restype = C.c_int
         _lib = L
     return _lib
@@ -243,6 +244,15 @@ def ha_score_topk(shape: ha_shape, q_codes, k_codes, seq_lens, k_per_seq, k_unif
         C.byref(shape), q_codes.data_ptr(), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1),
         seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform, max_seq_len, k_max, idx.data_ptr(), idx.stride(0),
         idx.stride(1), count.data_ptr(), _ptr(hist_out), p, n, _stream(stream)))
+
+
+def ha_score_topk_sum(shape: ha_shape, q_codes, k_codes, seq_lens, k_per_seq, k_uniform: int, k_max: int, idx, count,
+                      hist_out=None, stream=None) -> None:
+    """ha_score_topk with the per-head scores of a group added up (0 .. 32 G); hist_out int32 [B,Hkv,32 G + 1]."""
+    _check("ha_score_topk_sum", lib().ha_score_topk_sum(
+        C.byref(shape), q_codes.data_ptr(), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1),
+        seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform, k_max, idx.data_ptr(), idx.stride(0), idx.stride(1),
+        count.data_ptr(), _ptr(hist_out), _stream(stream)))
 
 
 def ha_gather_attn(shape: ha_shape, q, K, V, seq_lens, idx, count, k_max: int, out, workspace, lse=None,

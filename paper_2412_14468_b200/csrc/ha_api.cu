@@ -164,6 +164,19 @@ int ha_score_topk(const ha_shape *shape, const uint32_t *q_codes, const uint32_t
     return HA_OK;
 }
 
+int ha_score_topk_sum(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes, int64_t kc_stride_b,
+                      int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                      int32_t k_max, int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
+                      int32_t *hist_out, void *stream) {
+    HA_TRY(check_score_args(shape, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_uniform, k_per_seq, 0, k_max,
+                            idx, count));
+    if (shape->batch == 0) return HA_OK;
+    HA_CUDA(launch_score_topk_sum(shape->batch, shape->n_q_heads, shape->n_kv_heads, q_codes, k_codes, kc_stride_b,
+                                  kc_stride_h, seq_lens, k_per_seq, k_uniform, k_max, idx, idx_stride_b, idx_stride_h,
+                                  count, hist_out, (cudaStream_t)stream, Windows{shape->n_sink, shape->n_local}));
+    return HA_OK;
+}
+
 int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K, const ha_tensor *V,
                    const int32_t *seq_lens, const int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h,
                    const int32_t *count, int32_t k_max, uint16_t *out, float *lse, void *workspace, size_t ws_bytes,

@@ -182,6 +182,12 @@ cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, c
                               int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
                               int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st, Windows win = Windows{0, 0});
 
+// SCORE + TOPK with the group's per-head scores added instead of maximised (one cluster per unit, no scratch).
+cudaError_t launch_score_topk_sum(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes, long long kc_sb,
+                                  long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq, int k_uniform,
+                                  int k_max, int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
+                                  int32_t *hist_out, cudaStream_t st, Windows win = Windows{0, 0});
+
 cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale, const uint16_t *q,
                              TensorView K, TensorView V, const int32_t *seq_lens, const int32_t *idx,
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,

@@ -1,0 +1,277 @@
+// SCORE + TOPK with the per-head scores of a GQA group ADDED instead of maximised: S(i) = sum over the G query
+// heads of (32 - popc(k_i xor q_j)) (Eq. 1 with the bitcount identity of Section 4.1, per head), 0 .. 32 G, then the
+// standard top-k of Section 4 with ties towards the lowest token index.  The paper defines the score for one query
+// head; the layer-step reduces a group with the maximum (33 levels), this is the stand-alone alternative with
+// 32 G + 1 levels.
+//
+// One thread-block cluster per (sequence, KV head): the CTAs cut the signature row into equal contiguous slices.
+//   pass 1  every CTA streams its slice (16-byte loads, the next tile requested before the current one is counted)
+//           into per-warp histograms in shared memory;
+//   merge   the CTA histograms meet through distributed shared memory: every CTA reads all of them and derives the
+//           same threshold T (largest level with #{S >= T} >= k), r = k - #{S > T}, and how many tokens with
+//           S > T / S == T lie before its slice;
+//   pass 2  the slice is scored again (the signatures now come from L2; a slice of one tile keeps its scores in
+//           registers) and the selected tokens are written at their final positions: position = #{selected tokens
+//           with a smaller index}, from a prefix sum over lanes, loads and warps.
+// Nothing is kept in global scratch.  Tokens that are always in context (first n_sink, most recent n_local) are
+// written without being scored, exactly as in the maximum variant.
+#include "ha_score_dev.cuh"
+
+namespace ha {
+
+constexpr int kSumThreads = 256;
+constexpr int kSumWarps = kSumThreads / 32;
+constexpr int kSumLoads = 4;                                    // 16-byte loads per lane and tile
+constexpr int kSumWarpTokens = 32 * 4 * kSumLoads;              // 512 tokens per warp and tile
+constexpr int kSumTileTokens = kSumWarps * kSumWarpTokens;      // 4096 tokens per CTA and tile
+constexpr int kSumForced = -2, kSumAbsent = -1;                 // score stand-ins: always in context / outside the slice
+
+struct SumArgs {
+    const uint32_t *q_codes, *k_codes;
+    long long kc_sb, kc_sh;
+    const int32_t *seq_lens, *k_per_seq;
+    int k_uniform, k_max, Hq, Hkv;
+    int32_t *idx;
+    long long idx_sb, idx_sh;
+    int32_t *count, *hist_out;
+    Windows win;
+};
+
+// Scores of the 16 tokens this lane owns in tile `it` of the slice [lo, hi): load j covers tokens
+// tile_base + j * 128 + 4 * lane .. + 3.
+template <int G>
+__device__ __forceinline__ void sum_scores_of(const uint4 (&v)[kSumLoads], int tile_base, int lane, int hi, WindowBounds wb,
+                                              const uint32_t (&q)[G], int (&sc)[4 * kSumLoads]) {
+#pragma unroll
+    for (int j = 0; j < kSumLoads; ++j) {
+        const uint32_t c[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int t = tile_base + j * 128 + 4 * lane + e;
+            int h = 0;
+#pragma unroll
+            for (int g = 0; g < G; ++g) h += __popc(c[e] ^ q[g]);
+            int s = 32 * G - h;
+            if (t < wb.sink_end || t >= wb.local_begin) s = kSumForced;
+            if (t >= hi) s = kSumAbsent;
+            sc[4 * j + e] = s;
+        }
+    }
+}
+
+__device__ __forceinline__ void sum_load_tile(const uint32_t *row, int tile_base, int lane, int hi, uint4 (&v)[kSumLoads]) {
+#pragma unroll
+    for (int j = 0; j < kSumLoads; ++j) {
+        const int t = tile_base + j * 128 + 4 * lane;
+        v[j] = (t < hi) ? load_codes4(row, t, hi) : make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
+template <int G, int CS>
+__global__ void __launch_bounds__(kSumThreads) score_sum_select_kernel(const SumArgs a) {
+    constexpr int NB = 32 * G + 1;                      // score levels
+    constexpr int kPer = (NB + 31) / 32;                // levels per lane in the threshold search
+    __shared__ int w_hist[kSumWarps][NB];               // pass 1: one histogram per warp
+    __shared__ int s_hist[NB];                          // this CTA's histogram, read by the whole cluster
+    __shared__ int s_tot[NB], s_bef[NB];                // whole sequence / slices before this one
+    __shared__ int s_wsum[2][kSumWarps];                // pass 2: packed (S > T, S == T) counts per warp, double buffered
+    __shared__ int s_T, s_r, s_gtb, s_eqb;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rank = cluster_rank();
+    const int g = blockIdx.y, b = blockIdx.z;
+    const int n = max(a.seq_lens[b], 0);
+    const WindowBounds wb = window_bounds(a.win, n);
+    const int nf = forced_before(wb, n);
+    const int kb = a.k_per_seq ? a.k_per_seq[b] : a.k_uniform;
+    const int keep = max(0, min(min(kb, a.k_max - nf), n - nf));     // heavy tokens retrieved among the others
+    const uint32_t *row = a.k_codes + (long long)b * a.kc_sb + (long long)g * a.kc_sh;
+    int32_t *list = a.idx + (long long)b * a.idx_sb + (long long)g * a.idx_sh;
+
+    uint32_t q[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) q[j] = __ldg(a.q_codes + (long long)b * a.Hq + (long long)g * G + j);
+
+    // slice of this CTA: a multiple of four tokens, so that every 16-byte load stays inside it
+    const int per = ((n + 3) / 4 + CS - 1) / CS * 4;
+    const int lo = min(n, (int)rank * per), hi = min(n, lo + per);
+    const int n_tiles = (hi - lo + kSumTileTokens - 1) / kSumTileTokens;
+
+    for (int i = tid; i < kSumWarps * NB; i += kSumThreads) (&w_hist[0][0])[i] = 0;
+    __syncthreads();
+
+    // ---- pass 1: histogram of the slice
+    int sc[4 * kSumLoads];
+    {
+        uint4 v[kSumLoads], nx[kSumLoads];
+        if (n_tiles > 0) sum_load_tile(row, lo + warp * kSumWarpTokens, lane, hi, v);
+        for (int it = 0; it < n_tiles; ++it) {
+            const int base = lo + it * kSumTileTokens + warp * kSumWarpTokens;
+            if (it + 1 < n_tiles) sum_load_tile(row, base + kSumTileTokens, lane, hi, nx);
+            sum_scores_of<G>(v, base, lane, hi, wb, q, sc);
+#pragma unroll
+            for (int e = 0; e < 4 * kSumLoads; ++e)
+                if (sc[e] >= 0) atomicAdd(&w_hist[warp][sc[e]], 1);
+            if (it + 1 < n_tiles) {
+#pragma unroll
+                for (int j = 0; j < kSumLoads; ++j) v[j] = nx[j];
+            }
+        }
+    }
+    __syncthreads();
+    for (int l = tid; l < NB; l += kSumThreads) {
+        int s = 0;
+#pragma unroll
+        for (int w = 0; w < kSumWarps; ++w) s += w_hist[w][l];
+        s_hist[l] = s;
+    }
+    cluster_sync_all();   // every CTA's histogram is complete and visible
+
+    // ---- merge: totals over the cluster and over the slices before this one
+    for (int l = tid; l < NB; l += kSumThreads) {
+        int tot = 0, bef = 0;
+#pragma unroll
+        for (uint32_t r = 0; r < (uint32_t)CS; ++r) {
+            const int x = ld_dsmem(&s_hist[l], r);
+            tot += x;
+            if (r < rank) bef += x;
+        }
+        s_tot[l] = tot;
+        s_bef[l] = bef;
+    }
+    cluster_arrive();     // done reading the others' shared memory; matched by the wait at the end
+    __syncthreads();
+
+    if (warp == 0) {      // threshold: lane l looks at levels [l * kPer, l * kPer + kPer)
+        const int l0 = lane * kPer, l1 = min(NB, l0 + kPer);
+        int mine = 0;
+        for (int l = l0; l < l1; ++l) mine += s_tot[l];
+        int suf = mine;   // tokens at the levels of lanes >= this one
+#pragma unroll
+        for (int dd = 1; dd < 32; dd <<= 1) {
+            const int o = __shfl_down_sync(0xffffffffu, suf, dd);
+            if (lane + dd < 32) suf += o;
+        }
+        int above = suf - mine, T = NB, r = 0;
+        bool found = false;
+        if (keep > 0) {
+            for (int l = l1 - 1; l >= l0; --l) {
+                const int here = s_tot[l];
+                if (!found && above < keep && keep <= above + here) { found = true; T = l; r = keep - above; }
+                above += here;
+            }
+        }
+        const unsigned who = __ballot_sync(0xffffffffu, found);
+        const int src = who ? (__ffs(who) - 1) : 0;
+        T = __shfl_sync(0xffffffffu, T, src);
+        r = __shfl_sync(0xffffffffu, r, src);
+        int gtb = 0;
+        for (int l = l0; l < l1; ++l)
+            if (l > T) gtb += s_bef[l];
+#pragma unroll
+        for (int dd = 16; dd > 0; dd >>= 1) gtb += __shfl_xor_sync(0xffffffffu, gtb, dd);
+        if (lane == 0) { s_T = T; s_r = r; s_gtb = gtb; s_eqb = (T < NB) ? s_bef[T] : 0; }
+    }
+    __syncthreads();
+    const int T = s_T, r = s_r;
+    if (a.hist_out && rank == 0)
+        for (int l = tid; l < NB; l += kSumThreads) a.hist_out[((long long)b * a.Hkv + g) * NB + l] = s_tot[l];
+
+    // ---- pass 2: the selected tokens of the slice, at their final positions
+    const int local_pos0 = wb.sink_end + keep;   // where the most recent tokens go
+    int run_g = s_gtb, run_q = s_eqb;            // tokens with S > T / S == T before the current tile
+    for (int it = 0; it < n_tiles; ++it) {
+        const int base = lo + it * kSumTileTokens + warp * kSumWarpTokens;
+        if (n_tiles != 1) {   // a slice of one tile still holds its scores in registers
+            uint4 v[kSumLoads];
+            sum_load_tile(row, base, lane, hi, v);
+            sum_scores_of<G>(v, base, lane, hi, wb, q, sc);
+        }
+        // packed counts (S > T in the low half, S == T in the high half) of this lane per load, then over the warp
+        int excl[kSumLoads], warp_total = 0;
+#pragma unroll
+        for (int j = 0; j < kSumLoads; ++j) {
+            int p = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) p += (sc[4 * j + e] > T ? 1 : 0) + (sc[4 * j + e] == T ? 0x10000 : 0);
+            int inc = p;
+#pragma unroll
+            for (int dd = 1; dd < 32; dd <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, inc, dd);
+                if (lane >= dd) inc += o;
+            }
+            excl[j] = warp_total + inc - p;
+            warp_total += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (lane == 0) s_wsum[it & 1][warp] = warp_total;
+        __syncthreads();
+        int before = 0, tile_total = 0;
+#pragma unroll
+        for (int w = 0; w < kSumWarps; ++w) {
+            const int x = s_wsum[it & 1][w];
+            if (w < warp) before += x;
+            tile_total += x;
+        }
+#pragma unroll
+        for (int j = 0; j < kSumLoads; ++j) {
+            int gb = run_g + ((before + excl[j]) & 0xffff), qb = run_q + ((before + excl[j]) >> 16);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int s = sc[4 * j + e], t = base + j * 128 + 4 * lane + e;
+                if (s > T) { list[wb.sink_end + gb + min(qb, r)] = t; ++gb; }
+                else if (s == T) { if (qb < r) list[wb.sink_end + gb + qb] = t; ++qb; }
+                else if (s == kSumForced) list[t < wb.sink_end ? t : local_pos0 + (t - wb.local_begin)] = t;
+            }
+        }
+        run_g += tile_total & 0xffff;
+        run_q += tile_total >> 16;
+    }
+
+    // ---- count and padding
+    const int cnt = nf + keep;
+    if (rank == 0 && tid == 0) a.count[(long long)b * a.Hkv + g] = cnt;
+    for (int i = cnt + (int)rank * kSumThreads + tid; i < a.k_max; i += CS * kSumThreads) list[i] = -1;
+    cluster_wait();
+}
+
+template <int G>
+static cudaError_t launch_sum_t(const SumArgs &a, int B, cudaStream_t st) {
+    constexpr int CS = 8;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(CS, a.Hkv, B);
+    cfg.blockDim = dim3(kSumThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, score_sum_select_kernel<G, CS>, a);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_score_topk_sum(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes, long long kc_sb,
+                                  long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq, int k_uniform,
+                                  int k_max, int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
+                                  int32_t *hist_out, cudaStream_t st, Windows win) {
+    if (B <= 0 || Hkv <= 0) return cudaSuccess;
+    SumArgs a;
+    a.q_codes = q_codes; a.k_codes = k_codes; a.kc_sb = kc_sb; a.kc_sh = kc_sh;
+    a.seq_lens = seq_lens; a.k_per_seq = k_per_seq; a.k_uniform = k_uniform; a.k_max = k_max;
+    a.Hq = Hq; a.Hkv = Hkv; a.idx = idx; a.idx_sb = idx_sb; a.idx_sh = idx_sh;
+    a.count = count; a.hist_out = hist_out; a.win = win;
+    switch (Hq / Hkv) {
+        case 1: return launch_sum_t<1>(a, B, st);
+        case 2: return launch_sum_t<2>(a, B, st);
+        case 4: return launch_sum_t<4>(a, B, st);
+        case 8: return launch_sum_t<8>(a, B, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+} // namespace ha

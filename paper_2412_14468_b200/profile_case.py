@@ -63,11 +63,21 @@ def score_only(args):
     for s in range(args.steps):
         _ = int(flush.sum())
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(200000)   # the GPU is busy while the host enqueues: the events bracket the kernels only
         e0.record()
         ha.ha_score_topk(shape, qc, kc, lens, None, k, n, k, idx, cnt, ws)
         e1.record()
         torch.cuda.synchronize()
         print(f"step {s}: {e0.elapsed_time(e1) * 1e3:.1f} us (plain launch, L2 flushed)")
+        if args.group_sum:   # the other group reduction: per-head scores added up
+            _ = int(flush.sum())
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda._sleep(200000)
+            e0.record()
+            ha.ha_score_topk_sum(shape, qc, kc, lens, None, k, k, idx, cnt)
+            e1.record()
+            torch.cuda.synchronize()
+            print(f"step {s} summed group scores: {e0.elapsed_time(e1) * 1e3:.1f} us (plain launch, L2 flushed)")
     print("signature bytes per step:", B * Hkv * n * 4)
 
 
@@ -119,6 +129,8 @@ def main():
                          "its split-K kernel also where few units with short rows would get the cluster kernel")
     ap.add_argument("--score-only", action="store_true",
                     help="SCORE + TOPK alone on random signatures (no K/V allocated: large batches stay small)")
+    ap.add_argument("--group-sum", action="store_true",
+                    help="with --score-only: also run ha_score_topk_sum (per-head scores added instead of maximised)")
     ap.add_argument("--score-wide", action="store_true",
                     help="stand-alone SCORE on signatures of 64..512 bits and the inner-product comparator on --tokens tokens")
     ap.add_argument("--tokens", type=int, default=1 << 23)

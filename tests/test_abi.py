@@ -119,6 +119,22 @@ def test_windows_and_prefill_arguments_are_checked_on_the_host(lib):
     assert lib.ha_encode_prefill(C.byref(m), 1, C.byref(t), 1, 8, 0, fake, 64, 64, ha.HA_PREFILL_TCGEN05, None, None) == ha.HA_OK
 
 
+def test_summed_group_score_arguments_are_checked_on_the_host(lib):
+    fake = 0x1000
+    s = ha.make_shape(1, 32, 8, 0.088)
+    call = lambda shape, q=fake, k=fake, sb=16, sh=16, lens=fake, k_uni=4, k_max=4, idx=fake, cnt=fake: \
+        lib.ha_score_topk_sum(C.byref(shape), q, k, sb, sh, lens, None, k_uni, k_max, idx, 0, 0, cnt, None, None)
+    assert call(s, q=None) == ha.HA_ERR_INVALID_ARG
+    assert call(s, idx=None) == ha.HA_ERR_INVALID_ARG
+    assert call(s, k=fake + 4) == ha.HA_ERR_INVALID_ARG          # signature rows not 16-byte aligned
+    assert call(s, sh=18) == ha.HA_ERR_INVALID_ARG
+    assert call(s, k_uni=-1) == ha.HA_ERR_INVALID_ARG
+    assert call(s, k_max=-1) == ha.HA_ERR_INVALID_ARG
+    assert call(ha.make_shape(1, 32, 8, 0.088, n_sink=128, n_local=128), k_max=255) == ha.HA_ERR_INVALID_ARG
+    assert call(ha.make_shape(1, 32, 5, 0.088)) in (ha.HA_ERR_INVALID_ARG, ha.HA_ERR_UNSUPPORTED)   # heads do not divide
+    assert call(ha.make_shape(0, 32, 8, 0.088)) == ha.HA_OK      # empty batch: no launch
+
+
 def test_wide_score_and_inner_product_arguments_are_checked_on_the_host(lib):
     fake = 0x1000
     assert lib.ha_score_wide(fake, fake, 100, 96, fake, None) == ha.HA_ERR_UNSUPPORTED        # width not 64/128/256/512

@@ -142,7 +142,7 @@ def test_encode_prefill_on_tensor_cores_matches_the_chain_up_to_its_margin(T, st
 
 # ---------------------------------------------------------------------------- SCORE + TOPK
 
-def _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, k_uniform=None, n_sink=0, n_local=0):
+def _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, k_uniform=None, n_sink=0, n_local=0, reduce="max"):
     B = len(lens)
     n_cap = kc_np.shape[2]
     k_max = max(max(ks) + n_sink + n_local, 1)
@@ -154,19 +154,24 @@ def _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, k_uniform=None, n_sink=0, n
     kp = None if k_uniform is not None else torch.tensor(ks, dtype=torch.int32, device=DEV)
     idx = torch.full((B, Hkv, k_max), -7, dtype=torch.int32, device=DEV)
     cnt = torch.full((B, Hkv), -7, dtype=torch.int32, device=DEV)
-    hist = torch.full((B, Hkv, 33), -7, dtype=torch.int32, device=DEV)
-    ha.ha_score_topk(shape, qc, kc, sl, kp, k_uniform if k_uniform is not None else 0, n_cap, k_max, idx, cnt, ws,
-                     hist_out=hist)
+    hist = torch.full((B, Hkv, 33 if reduce == "max" else 32 * (Hq // Hkv) + 1), -7, dtype=torch.int32, device=DEV)
+    if reduce == "max":
+        ha.ha_score_topk(shape, qc, kc, sl, kp, k_uniform if k_uniform is not None else 0, n_cap, k_max, idx, cnt, ws,
+                         hist_out=hist)
+    else:   # the per-head scores added up: a stand-alone entry without workspace
+        ha.ha_score_topk_sum(shape, qc, kc, sl, kp, k_uniform if k_uniform is not None else 0, k_max, idx, cnt,
+                             hist_out=hist)
     torch.cuda.synchronize()
     return idx.cpu().numpy(), cnt.cpu().numpy(), hist.cpu().numpy()
 
 
-def _check_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, n_sink=0, n_local=0, **kw):
-    idx, cnt, hist = _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, n_sink=n_sink, n_local=n_local, **kw)
+def _check_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, n_sink=0, n_local=0, reduce="max", **kw):
+    idx, cnt, hist = _run_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, n_sink=n_sink, n_local=n_local, reduce=reduce, **kw)
     G = Hq // Hkv
+    score_of = oracle.score if reduce == "max" else oracle.score_sum
     for b, (n, k) in enumerate(zip(lens, ks)):
         for g in range(Hkv):
-            s = oracle.score(qc_np[b, g * G:(g + 1) * G], kc_np[b, g, :n])
+            s = score_of(qc_np[b, g * G:(g + 1) * G], kc_np[b, g, :n])
             if n_sink == 0 and n_local == 0:
                 exp = oracle.topk(s, k)
                 assert cnt[b, g] == len(exp) == min(k, n)
@@ -180,7 +185,7 @@ def _check_score_topk(qc_np, kc_np, lens, ks, Hq, Hkv, n_sink=0, n_local=0, **kw
                 others = s[~forced]
             assert np.array_equal(idx[b, g, :len(exp)], exp), (b, g, n, k, n_sink, n_local)
             assert np.all(idx[b, g, len(exp):] == -1)
-            assert np.array_equal(hist[b, g], np.bincount(others, minlength=33))
+            assert np.array_equal(hist[b, g], np.bincount(others, minlength=hist.shape[2]))
 
 
 @pytest.mark.parametrize("G", [1, 4])
@@ -286,6 +291,65 @@ def test_score_topk_biased_bits_like_random_init_mappings():
     qbits = rng.random((1, Hq, 32)) < p1
     qc = (qbits * (1 << np.arange(32, dtype=np.uint64))).sum(-1).astype(np.uint32)
     _check_score_topk(qc, kc, [n], [1024], Hq, Hkv)
+
+
+# ---- the other group reduction: per-head scores added up (ha_score_topk_sum), 32 G + 1 levels
+
+@pytest.mark.parametrize("G", [1, 2, 4, 8])
+def test_score_topk_sum_sizes_ragged_tail_and_budgets(G):
+    rng = np.random.default_rng(105 + G)
+    Hkv, Hq = 2, 2 * G
+    lens = [0, 1, 5, 31, 32, 33, 1023, 2047, 4096 * 8, 4096 * 8 + 1, 5000, 70001]   # 32768: one full tile per CTA
+    n_cap = 70004
+    kc = rng.integers(0, 2 ** 32, size=(len(lens), Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    qc = rng.integers(0, 2 ** 32, size=(len(lens), Hq), dtype=np.uint64).astype(np.uint32)
+    for ks in ([n // 16 for n in lens], [n for n in lens], [n + 5 for n in lens], [1] * len(lens), [0] * len(lens),
+               [min(n, 777) for n in lens]):
+        _check_score_topk(qc, kc, lens, ks, Hq, Hkv, reduce="sum")
+
+
+def test_score_topk_sum_equals_the_maximum_variant_for_single_head_groups():
+    rng = np.random.default_rng(31)
+    lens, n_cap = [9000, 1, 33000], 33000
+    kc = rng.integers(0, 2 ** 32, size=(3, 4, n_cap), dtype=np.uint64).astype(np.uint32)
+    qc = rng.integers(0, 2 ** 32, size=(3, 4), dtype=np.uint64).astype(np.uint32)
+    ks = [500, 1, 2000]
+    a = _run_score_topk(qc, kc, lens, ks, 4, 4, reduce="max")
+    b = _run_score_topk(qc, kc, lens, ks, 4, 4, reduce="sum")
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
+
+
+def test_score_topk_sum_long_sequence_and_windows():
+    rng = np.random.default_rng(78)
+    Hkv, Hq = 1, 4
+    lens, n_cap = [600001, 131073, 9], 600004
+    kc = rng.integers(0, 2 ** 32, size=(len(lens), Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    qc = rng.integers(0, 2 ** 32, size=(len(lens), Hq), dtype=np.uint64).astype(np.uint32)
+    _check_score_topk(qc, kc, lens, [n // 32 for n in lens], Hq, Hkv, reduce="sum")
+    _check_score_topk(qc, kc, lens, [n // 32 for n in lens], Hq, Hkv, n_sink=128, n_local=128, reduce="sum")
+    _check_score_topk(qc, kc, lens, [3, lens[1], 20], Hq, Hkv, n_sink=5000, n_local=70000, reduce="sum")
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_score_topk_sum_random_shapes_budgets_windows_and_ties(seed):
+    rng = np.random.default_rng(9500 + seed)
+    B = int(rng.integers(1, 7))
+    Hkv = int(rng.choice([1, 2, 4]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    lens = [int(v) for v in rng.integers(0, int(rng.choice([40, 3000, 40000])), size=B)]
+    n_cap = (max(max(lens), 4) + 3) // 4 * 4
+    if seed % 3 == 0:   # few distinct signatures: long tie blocks
+        pool = rng.integers(0, 2 ** 32, size=5, dtype=np.uint64).astype(np.uint32)
+        kc = pool[rng.integers(0, 5, size=(B, Hkv, n_cap))]
+    else:
+        kc = rng.integers(0, 2 ** 32, size=(B, Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    qc = rng.integers(0, 2 ** 32, size=(B, Hkv * G), dtype=np.uint64).astype(np.uint32)
+    if seed % 4 == 1:
+        qc[:, :] = kc[:, :, 0].repeat(G, axis=1)[:, :Hkv * G]   # exact matches: the top level 32 G is reached
+    ks = [int(rng.integers(0, n + 10)) for n in lens]
+    n_sink, n_local = (0, 0) if seed % 2 == 0 else (int(rng.integers(0, 200)), int(rng.integers(0, 200)))
+    _check_score_topk(qc, kc, lens, ks, Hkv * G, Hkv, n_sink=n_sink, n_local=n_local, reduce="sum")
 
 
 # ---------------------------------------------------------------------------- GATHER-ATT / dense
