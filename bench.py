@@ -533,6 +533,41 @@ def main():
                 table[f"{n_tok}_tokens"] = row
                 torch.cuda.empty_cache()
             supplementary["score_latency_table"] = table
+
+            # SCORE + TOPK alone with the two group reductions (maximum: the layer-step's contract; sum: the stand-alone
+            # alternative), random signatures, L2-cold launches; the GPU is kept busy while the host enqueues, so the
+            # events bracket the kernels only
+            def cold_kernel_us(fn, iters=9):
+                ts = []
+                for _ in range(iters + 2):
+                    flush.fill_(1)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    torch.cuda._sleep(300000)
+                    e0.record()
+                    fn()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ts.append(e0.elapsed_time(e1) * 1e3)
+                return float(sorted(ts[2:])[len(ts[2:]) // 2])
+
+            red = {}
+            for name, (Bq, n_tok, kq) in {"c2": (1, 32768, 1024), "c3": (16, 32768, 2048), "batch64_32K": (64, 32768, 1024),
+                                          "c4": (1, 524288, 16384)}.items():
+                kc = torch.randint(-2**31, 2**31 - 1, (Bq, 8, n_tok), dtype=torch.int32, device=device, generator=gs)
+                qc = torch.randint(-2**31, 2**31 - 1, (Bq, 32), dtype=torch.int32, device=device, generator=gs)
+                shp = ha.make_shape(Bq, 32, 8, 1.0)
+                wsq = ha.alloc_workspace(shp, n_tok, kq, device=device)
+                ln = torch.full((Bq,), n_tok, dtype=torch.int32, device=device)
+                ix = torch.zeros(Bq, 8, kq, dtype=torch.int32, device=device)
+                ct = torch.zeros(Bq, 8, dtype=torch.int32, device=device)
+                nbytes = Bq * 8 * (n_tok * 4 + kq * 4)
+                t_max = cold_kernel_us(lambda: ha.ha_score_topk(shp, qc, kc, ln, None, kq, n_tok, kq, ix, ct, wsq))
+                t_sum = cold_kernel_us(lambda: ha.ha_score_topk_sum(shp, qc, kc, ln, None, kq, kq, ix, ct))
+                red[name] = {"algorithmic_bytes": nbytes,
+                             "max_over_heads": {"us": t_max, "frac": nbytes / t_max / 1e3 / peak},
+                             "sum_over_heads": {"us": t_sum, "frac": nbytes / t_sum / 1e3 / peak}}
+                del kc, ix, wsq
+            supplementary["score_topk_group_reductions"] = red
             del flush
             torch.cuda.empty_cache()
         except Exception as ex:

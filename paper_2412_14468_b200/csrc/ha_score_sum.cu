@@ -4,9 +4,9 @@
 // head; the layer-step reduces a group with the maximum (33 levels), this is the stand-alone alternative with
 // 32 G + 1 levels.
 //
-// One thread-block cluster per (sequence, KV head): the CTAs cut the signature row into equal contiguous slices.
+// One thread-block cluster (1 to 16 CTAs, by the number of units) per (sequence, KV head): the CTAs cut the signature row into equal contiguous slices.
 //   pass 1  every CTA streams its slice (16-byte loads, the next tile requested before the current one is counted)
-//           into per-warp histograms in shared memory;
+//           into a histogram in shared memory (one counter per level and lane);
 //   merge   the CTA histograms meet through distributed shared memory: every CTA reads all of them and derives the
 //           same threshold T (largest level with #{S >= T} >= k), r = k - #{S > T}, and how many tokens with
 //           S > T / S == T lie before its slice;
@@ -21,9 +21,8 @@ namespace ha {
 
 constexpr int kSumThreads = 256;
 constexpr int kSumWarps = kSumThreads / 32;
-constexpr int kSumLoads = 4;                                    // 16-byte loads per lane and tile
-constexpr int kSumWarpTokens = 32 * 4 * kSumLoads;              // 512 tokens per warp and tile
-constexpr int kSumTileTokens = kSumWarps * kSumWarpTokens;      // 4096 tokens per CTA and tile
+// A tile is LD 16-byte loads per lane: 128 LD tokens per warp, 1024 LD per CTA (LD = 4 where few CTAs run and each
+// must keep many bytes in flight, 2 where many CTAs share an SM and registers decide how many fit).
 constexpr int kSumForced = -2, kSumAbsent = -1;                 // score stand-ins: always in context / outside the slice
 
 struct SumArgs {
@@ -37,48 +36,80 @@ struct SumArgs {
     Windows win;
 };
 
-// Scores of the 16 tokens this lane owns in tile `it` of the slice [lo, hi): load j covers tokens
-// tile_base + j * 128 + 4 * lane .. + 3.
+// The summed score without one population count per head: for bit position i let c_i = number of the group's query
+// signatures with bit i set, d_i = G - c_i.  A key with bit i set agrees with c_i heads there, otherwise with d_i, so
+// S = sum_i (k_i ? c_i : d_i) = sum_p 2^p popc((k & C_p) | (~k & D_p)) with C_p / D_p the bit planes of c / d:
+// log2(G) + 1 population counts per token instead of G.
 template <int G>
-__device__ __forceinline__ void sum_scores_of(const uint4 (&v)[kSumLoads], int tile_base, int lane, int hi, WindowBounds wb,
-                                              const uint32_t (&q)[G], int (&sc)[4 * kSumLoads]) {
+struct SumPlanes {
+    static constexpr int P = (G == 1) ? 1 : (G == 2) ? 2 : (G == 4) ? 3 : 4;
+    uint32_t C[P], D[P];
+    __device__ __forceinline__ void build(const uint32_t (&q)[G]) {
 #pragma unroll
-    for (int j = 0; j < kSumLoads; ++j) {
+        for (int p = 0; p < P; ++p) { C[p] = 0u; D[p] = 0u; }
+#pragma unroll
+        for (int j = 0; j < G; ++j) {   // bit-sliced counters: add the one-bit numbers q_j (and their complements)
+            uint32_t carry_c = q[j], carry_d = ~q[j];
+#pragma unroll
+            for (int p = 0; p < P; ++p) {
+                const uint32_t tc = C[p] & carry_c, td = D[p] & carry_d;
+                C[p] ^= carry_c; D[p] ^= carry_d;
+                carry_c = tc; carry_d = td;
+            }
+        }
+    }
+    __device__ __forceinline__ int score(uint32_t k) const {
+        int s = 0;
+#pragma unroll
+        for (int p = 0; p < P; ++p) s += __popc((k & C[p]) | (~k & D[p])) << p;
+        return s;
+    }
+};
+
+// Scores of the 4 LD tokens this lane owns in a warp tile starting at `base`: load j covers tokens
+// base + j * 128 + 4 * lane .. + 3.  kEdge: the tile may touch the always-kept windows or the end of the slice.
+template <int G, int LD, bool kEdge>
+__device__ __forceinline__ void sum_scores_of(const uint4 (&v)[LD], int base, int lane, int hi, WindowBounds wb,
+                                              const SumPlanes<G> &pl, int (&sc)[4 * LD]) {
+#pragma unroll
+    for (int j = 0; j < LD; ++j) {
         const uint32_t c[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const int t = tile_base + j * 128 + 4 * lane + e;
-            int h = 0;
-#pragma unroll
-            for (int g = 0; g < G; ++g) h += __popc(c[e] ^ q[g]);
-            int s = 32 * G - h;
-            if (t < wb.sink_end || t >= wb.local_begin) s = kSumForced;
-            if (t >= hi) s = kSumAbsent;
+            int s = pl.score(c[e]);
+            if (kEdge) {
+                const int t = base + j * 128 + 4 * lane + e;
+                if (t < wb.sink_end || t >= wb.local_begin) s = kSumForced;
+                if (t >= hi) s = kSumAbsent;
+            }
             sc[4 * j + e] = s;
         }
     }
 }
 
-__device__ __forceinline__ void sum_load_tile(const uint32_t *row, int tile_base, int lane, int hi, uint4 (&v)[kSumLoads]) {
+template <int LD, bool kEdge>
+__device__ __forceinline__ void sum_load_tile(const uint32_t *row, int base, int lane, int hi, uint4 (&v)[LD]) {
 #pragma unroll
-    for (int j = 0; j < kSumLoads; ++j) {
-        const int t = tile_base + j * 128 + 4 * lane;
-        v[j] = (t < hi) ? load_codes4(row, t, hi) : make_uint4(0u, 0u, 0u, 0u);
+    for (int j = 0; j < LD; ++j) {
+        const int t = base + j * 128 + 4 * lane;
+        if (kEdge) v[j] = (t < hi) ? load_codes4(row, t, hi) : make_uint4(0u, 0u, 0u, 0u);
+        else v[j] = __ldg(reinterpret_cast<const uint4 *>(row + t));
     }
 }
 
-template <int G, int CS>
-__global__ void __launch_bounds__(kSumThreads) score_sum_select_kernel(const SumArgs a) {
+template <int G, int CS, int LD>
+__global__ void __launch_bounds__(kSumThreads, LD <= 2 ? 5 : 3) score_sum_select_kernel(const SumArgs a) {
+    constexpr int kWarpTokens = 128 * LD, kTileTokens = kSumWarps * kWarpTokens;
     constexpr int NB = 32 * G + 1;                      // score levels
     constexpr int kPer = (NB + 31) / 32;                // levels per lane in the threshold search
-    __shared__ int w_hist[kSumWarps][NB];               // pass 1: one histogram per warp
+    __shared__ __align__(16) int c_hist[NB][32];        // pass 1: one counter per (level, lane): no two lanes of a warp meet
     __shared__ int s_hist[NB];                          // this CTA's histogram, read by the whole cluster
     __shared__ int s_tot[NB], s_bef[NB];                // whole sequence / slices before this one
     __shared__ int s_wsum[2][kSumWarps];                // pass 2: packed (S > T, S == T) counts per warp, double buffered
     __shared__ int s_T, s_r, s_gtb, s_eqb;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t rank = cluster_rank();
+    const uint32_t rank = (CS > 1) ? cluster_rank() : 0u;
     const int g = blockIdx.y, b = blockIdx.z;
     const int n = max(a.seq_lens[b], 0);
     const WindowBounds wb = window_bounds(a.win, n);
@@ -88,58 +119,80 @@ __global__ void __launch_bounds__(kSumThreads) score_sum_select_kernel(const Sum
     const uint32_t *row = a.k_codes + (long long)b * a.kc_sb + (long long)g * a.kc_sh;
     int32_t *list = a.idx + (long long)b * a.idx_sb + (long long)g * a.idx_sh;
 
-    uint32_t q[G];
+    SumPlanes<G> pl;
+    {
+        uint32_t q[G];
 #pragma unroll
-    for (int j = 0; j < G; ++j) q[j] = __ldg(a.q_codes + (long long)b * a.Hq + (long long)g * G + j);
+        for (int j = 0; j < G; ++j) q[j] = __ldg(a.q_codes + (long long)b * a.Hq + (long long)g * G + j);
+        pl.build(q);
+    }
 
     // slice of this CTA: a multiple of four tokens, so that every 16-byte load stays inside it
     const int per = ((n + 3) / 4 + CS - 1) / CS * 4;
     const int lo = min(n, (int)rank * per), hi = min(n, lo + per);
-    const int n_tiles = (hi - lo + kSumTileTokens - 1) / kSumTileTokens;
+    const int n_tiles = (hi - lo + kTileTokens - 1) / kTileTokens;
+    const int plain_end = min(wb.local_begin, hi);      // warp tiles inside [sink_end, plain_end) need no per-token checks
+    auto is_edge = [&](int base) { return base < wb.sink_end || base + kWarpTokens > plain_end; };
 
-    for (int i = tid; i < kSumWarps * NB; i += kSumThreads) (&w_hist[0][0])[i] = 0;
+    for (int i = tid; i < NB * 8; i += kSumThreads) reinterpret_cast<uint4 *>(&c_hist[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
 
     // ---- pass 1: histogram of the slice
-    int sc[4 * kSumLoads];
+    int sc[4 * LD];
     {
-        uint4 v[kSumLoads], nx[kSumLoads];
-        if (n_tiles > 0) sum_load_tile(row, lo + warp * kSumWarpTokens, lane, hi, v);
+        uint4 v[LD], nx[LD];
+        auto load = [&](int base, uint4 (&dst)[LD]) {
+            if (is_edge(base)) sum_load_tile<LD, true>(row, base, lane, hi, dst);
+            else sum_load_tile<LD, false>(row, base, lane, hi, dst);
+        };
+        if (n_tiles > 0) load(lo + warp * kWarpTokens, v);
         for (int it = 0; it < n_tiles; ++it) {
-            const int base = lo + it * kSumTileTokens + warp * kSumWarpTokens;
-            if (it + 1 < n_tiles) sum_load_tile(row, base + kSumTileTokens, lane, hi, nx);
-            sum_scores_of<G>(v, base, lane, hi, wb, q, sc);
+            const int base = lo + it * kTileTokens + warp * kWarpTokens;
+            if (it + 1 < n_tiles) load(base + kTileTokens, nx);
+            if (is_edge(base)) {
+                sum_scores_of<G, LD, true>(v, base, lane, hi, wb, pl, sc);
 #pragma unroll
-            for (int e = 0; e < 4 * kSumLoads; ++e)
-                if (sc[e] >= 0) atomicAdd(&w_hist[warp][sc[e]], 1);
+                for (int e = 0; e < 4 * LD; ++e)
+                    if (sc[e] >= 0) atomicAdd(&c_hist[sc[e]][lane], 1);
+            } else {
+                sum_scores_of<G, LD, false>(v, base, lane, hi, wb, pl, sc);
+#pragma unroll
+                for (int e = 0; e < 4 * LD; ++e) atomicAdd(&c_hist[sc[e]][lane], 1);
+            }
             if (it + 1 < n_tiles) {
 #pragma unroll
-                for (int j = 0; j < kSumLoads; ++j) v[j] = nx[j];
+                for (int j = 0; j < LD; ++j) v[j] = nx[j];
             }
         }
     }
     __syncthreads();
-    for (int l = tid; l < NB; l += kSumThreads) {
+    for (int i = tid; i < (NB + 31) / 32 * 32 * 8; i += kSumThreads) {   // eight threads per level, four counters each
+        const int l = i >> 3;
         int s = 0;
-#pragma unroll
-        for (int w = 0; w < kSumWarps; ++w) s += w_hist[w][l];
-        s_hist[l] = s;
-    }
-    cluster_sync_all();   // every CTA's histogram is complete and visible
-
-    // ---- merge: totals over the cluster and over the slices before this one
-    for (int l = tid; l < NB; l += kSumThreads) {
-        int tot = 0, bef = 0;
-#pragma unroll
-        for (uint32_t r = 0; r < (uint32_t)CS; ++r) {
-            const int x = ld_dsmem(&s_hist[l], r);
-            tot += x;
-            if (r < rank) bef += x;
+        if (l < NB) {
+            const uint4 c4 = reinterpret_cast<const uint4 *>(&c_hist[l][0])[i & 7];
+            s = (int)(c4.x + c4.y + c4.z + c4.w);
         }
-        s_tot[l] = tot;
-        s_bef[l] = bef;
+        s += __shfl_xor_sync(0xffffffffu, s, 1);
+        s += __shfl_xor_sync(0xffffffffu, s, 2);
+        s += __shfl_xor_sync(0xffffffffu, s, 4);
+        if (l < NB && (i & 7) == 0) { s_hist[l] = s; if (CS == 1) { s_tot[l] = s; s_bef[l] = 0; } }
     }
-    cluster_arrive();     // done reading the others' shared memory; matched by the wait at the end
+    if (CS > 1) {
+        cluster_sync_all();   // every CTA's histogram is complete and visible
+        // ---- merge: totals over the cluster and over the slices before this one (all remote loads issued, then added)
+        for (int l = tid; l < NB; l += kSumThreads) {
+            int x[CS];
+#pragma unroll
+            for (int r = 0; r < CS; ++r) x[r] = ld_dsmem(&s_hist[l], (uint32_t)r);
+            int tot = 0, bef = 0;
+#pragma unroll
+            for (int r = 0; r < CS; ++r) { tot += x[r]; if (r < (int)rank) bef += x[r]; }
+            s_tot[l] = tot;
+            s_bef[l] = bef;
+        }
+        cluster_arrive();     // done reading the others' shared memory; matched by the wait at the end
+    }
     __syncthreads();
 
     if (warp == 0) {      // threshold: lane l looks at levels [l * kPer, l * kPer + kPer)
@@ -181,19 +234,26 @@ __global__ void __launch_bounds__(kSumThreads) score_sum_select_kernel(const Sum
     const int local_pos0 = wb.sink_end + keep;   // where the most recent tokens go
     int run_g = s_gtb, run_q = s_eqb;            // tokens with S > T / S == T before the current tile
     for (int it = 0; it < n_tiles; ++it) {
-        const int base = lo + it * kSumTileTokens + warp * kSumWarpTokens;
+        const int base = lo + it * kTileTokens + warp * kWarpTokens;
+        const bool edge = is_edge(base);
         if (n_tiles != 1) {   // a slice of one tile still holds its scores in registers
-            uint4 v[kSumLoads];
-            sum_load_tile(row, base, lane, hi, v);
-            sum_scores_of<G>(v, base, lane, hi, wb, q, sc);
+            uint4 v[LD];
+            if (edge) { sum_load_tile<LD, true>(row, base, lane, hi, v); sum_scores_of<G, LD, true>(v, base, lane, hi, wb, pl, sc); }
+            else { sum_load_tile<LD, false>(row, base, lane, hi, v); sum_scores_of<G, LD, false>(v, base, lane, hi, wb, pl, sc); }
         }
         // packed counts (S > T in the low half, S == T in the high half) of this lane per load, then over the warp
-        int excl[kSumLoads], warp_total = 0;
+        int excl[LD], warp_total = 0;
+        uint32_t wanted = 0;   // bit j: load j holds a token that may be written
 #pragma unroll
-        for (int j = 0; j < kSumLoads; ++j) {
+        for (int j = 0; j < LD; ++j) {
             int p = 0;
+            bool forced = false;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) p += (sc[4 * j + e] > T ? 1 : 0) + (sc[4 * j + e] == T ? 0x10000 : 0);
+            for (int e = 0; e < 4; ++e) {
+                p += (sc[4 * j + e] > T ? 1 : 0) + (sc[4 * j + e] == T ? 0x10000 : 0);
+                forced |= (sc[4 * j + e] == kSumForced);
+            }
+            if (p != 0 || (edge && forced)) wanted |= 1u << j;
             int inc = p;
 #pragma unroll
             for (int dd = 1; dd < 32; dd <<= 1) {
@@ -213,7 +273,8 @@ __global__ void __launch_bounds__(kSumThreads) score_sum_select_kernel(const Sum
             tile_total += x;
         }
 #pragma unroll
-        for (int j = 0; j < kSumLoads; ++j) {
+        for (int j = 0; j < LD; ++j) {
+            if (!(wanted & (1u << j))) continue;
             int gb = run_g + ((before + excl[j]) & 0xffff), qb = run_q + ((before + excl[j]) >> 16);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -231,12 +292,23 @@ __global__ void __launch_bounds__(kSumThreads) score_sum_select_kernel(const Sum
     const int cnt = nf + keep;
     if (rank == 0 && tid == 0) a.count[(long long)b * a.Hkv + g] = cnt;
     for (int i = cnt + (int)rank * kSumThreads + tid; i < a.k_max; i += CS * kSumThreads) list[i] = -1;
-    cluster_wait();
+    if (CS > 1) cluster_wait();
 }
 
-template <int G>
+template <int G, int CS, int LD>
 static cudaError_t launch_sum_t(const SumArgs &a, int B, cudaStream_t st) {
-    constexpr int CS = 8;
+    if (CS > 8) {   // clusters of more than 8 CTAs are an opt-in, per device
+        static bool allowed[64] = {};
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev < 0 || dev >= 64) dev = 0;
+        if (!allowed[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(score_sum_select_kernel<G, CS, LD>,
+                                                 cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            if (e != cudaSuccess) return e;
+            allowed[dev] = true;
+        }
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CS, a.Hkv, B);
     cfg.blockDim = dim3(kSumThreads);
@@ -249,10 +321,23 @@ static cudaError_t launch_sum_t(const SumArgs &a, int B, cudaStream_t st) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, score_sum_select_kernel<G, CS>, a);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, score_sum_select_kernel<G, CS, LD>, a);
     if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
+}
+
+// CTAs per unit: enough to give every SM about four CTAs, in clusters of at most 8 (16 for a handful of units, whose
+// sequences may be long).  The sequence lengths live on the device, so the choice looks at the unit count only;
+// a CTA whose slice is empty only takes part in the exchange.
+template <int G>
+static cudaError_t launch_sum_g(const SumArgs &a, int B, cudaStream_t st) {
+    const long long units = (long long)B * a.Hkv, want = 4LL * sm_count();
+    if (units * 8 < sm_count()) return launch_sum_t<G, 16, 4>(a, B, st);
+    if (units * 4 < want) return launch_sum_t<G, 8, 2>(a, B, st);
+    if (units * 2 < want) return launch_sum_t<G, 4, 2>(a, B, st);
+    if (units < want) return launch_sum_t<G, 2, 2>(a, B, st);
+    return launch_sum_t<G, 1, 2>(a, B, st);
 }
 
 cudaError_t launch_score_topk_sum(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes, long long kc_sb,
@@ -266,10 +351,10 @@ cudaError_t launch_score_topk_sum(int B, int Hq, int Hkv, const uint32_t *q_code
     a.Hq = Hq; a.Hkv = Hkv; a.idx = idx; a.idx_sb = idx_sb; a.idx_sh = idx_sh;
     a.count = count; a.hist_out = hist_out; a.win = win;
     switch (Hq / Hkv) {
-        case 1: return launch_sum_t<1>(a, B, st);
-        case 2: return launch_sum_t<2>(a, B, st);
-        case 4: return launch_sum_t<4>(a, B, st);
-        case 8: return launch_sum_t<8>(a, B, st);
+        case 1: return launch_sum_g<1>(a, B, st);
+        case 2: return launch_sum_g<2>(a, B, st);
+        case 4: return launch_sum_g<4>(a, B, st);
+        case 8: return launch_sum_g<8>(a, B, st);
         default: return cudaErrorInvalidValue;
     }
 }
