@@ -278,10 +278,14 @@ __global__ void __launch_bounds__(kSumThreads, LD <= 2 ? 5 : 3) score_sum_select
             int gb = run_g + ((before + excl[j]) & 0xffff), qb = run_q + ((before + excl[j]) >> 16);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
+                // a token with S > T, or one of the first r with S == T, lands behind everything selected before it:
+                // #{S > T before} + min(#{S == T before}, r)
                 const int s = sc[4 * j + e], t = base + j * 128 + 4 * lane + e;
-                if (s > T) { list[wb.sink_end + gb + min(qb, r)] = t; ++gb; }
-                else if (s == T) { if (qb < r) list[wb.sink_end + gb + qb] = t; ++qb; }
-                else if (s == kSumForced) list[t < wb.sink_end ? t : local_pos0 + (t - wb.local_begin)] = t;
+                const bool gt = s > T, eq = s == T;
+                if (gt || (eq && qb < r)) list[wb.sink_end + gb + min(qb, r)] = t;
+                gb += gt ? 1 : 0;
+                qb += eq ? 1 : 0;
+                if (edge && s == kSumForced) list[t < wb.sink_end ? t : local_pos0 + (t - wb.local_begin)] = t;
             }
         }
         run_g += tile_total & 0xffff;
