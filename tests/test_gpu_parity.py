@@ -331,6 +331,23 @@ def test_score_topk_sum_long_sequence_and_windows():
     _check_score_topk(qc, kc, lens, [3, lens[1], 20], Hq, Hkv, n_sink=5000, n_local=70000, reduce="sum")
 
 
+@pytest.mark.parametrize("B,Hkv", [(9, 2), (12, 2), (40, 2), (100, 2), (300, 2), (150, 4)])
+def test_score_topk_sum_every_cluster_size(B, Hkv):
+    """The cluster size follows the number of units: 16 CTAs up to 18 units, then 8, 4 (from 74), 2 (from 148) and
+    single CTAs (from 592), whose slices span several tiles here."""
+    rng = np.random.default_rng(600 + B)
+    G = 4
+    lens = [int(v) for v in rng.integers(0, 7000, size=B)]
+    lens[0], lens[-1] = 6999, 0
+    n_cap = 7000
+    kc = rng.integers(0, 2 ** 32, size=(B, Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    kc[1] = kc[1] & np.uint32(0x3)                      # four distinct signatures: long tie blocks across tiles
+    qc = rng.integers(0, 2 ** 32, size=(B, Hkv * G), dtype=np.uint64).astype(np.uint32)
+    ks = [int(rng.integers(0, n + 3)) for n in lens]
+    _check_score_topk(qc, kc, lens, ks, Hkv * G, Hkv, reduce="sum")
+    _check_score_topk(qc, kc, lens, [min(k, 500) for k in ks], Hkv * G, Hkv, n_sink=100, n_local=2100, reduce="sum")
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_score_topk_sum_random_shapes_budgets_windows_and_ties(seed):
     rng = np.random.default_rng(9500 + seed)
