@@ -241,19 +241,22 @@ __global__ void __launch_bounds__(kSumThreads, LD <= 2 ? 5 : 3) score_sum_select
             if (edge) { sum_load_tile<LD, true>(row, base, lane, hi, v); sum_scores_of<G, LD, true>(v, base, lane, hi, wb, pl, sc); }
             else { sum_load_tile<LD, false>(row, base, lane, hi, v); sum_scores_of<G, LD, false>(v, base, lane, hi, wb, pl, sc); }
         }
+        // bit i of the masks: token i of this lane (load i / 4, element i % 4) has S > T / S == T / is always kept
+        uint32_t gtm = 0, eqm = 0, fm = 0;
+#pragma unroll
+        for (int i = 0; i < 4 * LD; ++i) {
+            gtm |= (sc[i] > T ? 1u : 0u) << i;
+            eqm |= (sc[i] == T ? 1u : 0u) << i;
+            if (edge) fm |= (sc[i] == kSumForced ? 1u : 0u) << i;
+        }
         // packed counts (S > T in the low half, S == T in the high half) of this lane per load, then over the warp
         int excl[LD], warp_total = 0;
-        uint32_t wanted = 0;   // bit j: load j holds a token that may be written
 #pragma unroll
         for (int j = 0; j < LD; ++j) {
-            int p = 0;
-            bool forced = false;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                p += (sc[4 * j + e] > T ? 1 : 0) + (sc[4 * j + e] == T ? 0x10000 : 0);
-                forced |= (sc[4 * j + e] == kSumForced);
-            }
-            if (p != 0 || (edge && forced)) wanted |= 1u << j;
+            // bits set in the two nibbles, on the integer pipe (the population-count unit is the busy one here)
+            uint32_t v = ((gtm >> (4 * j)) & 15u) | (((eqm >> (4 * j)) & 15u) << 16);
+            v -= (v >> 1) & 0x00050005u;
+            const int p = (int)((v & 0x00030003u) + ((v >> 2) & 0x00030003u));
             int inc = p;
 #pragma unroll
             for (int dd = 1; dd < 32; dd <<= 1) {
@@ -272,21 +275,38 @@ __global__ void __launch_bounds__(kSumThreads, LD <= 2 ? 5 : 3) score_sum_select
             if (w < warp) before += x;
             tile_total += x;
         }
+        // A token with S > T, or one of the first r with S == T, lands behind everything selected before it:
+        // #{S > T before} + min(#{S == T before}, r).
+        if (LD >= 4) {
+            // few CTAs, each alone on its SM: only the few tokens at or above the threshold are visited
+            for (uint32_t m = gtm | eqm; m; m &= m - 1) {
+                const int i = __ffs(m) - 1, j = i >> 2, e = i & 3;
+                int ex = excl[0];
 #pragma unroll
-        for (int j = 0; j < LD; ++j) {
-            if (!(wanted & (1u << j))) continue;
-            int gb = run_g + ((before + excl[j]) & 0xffff), qb = run_q + ((before + excl[j]) >> 16);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                // a token with S > T, or one of the first r with S == T, lands behind everything selected before it:
-                // #{S > T before} + min(#{S == T before}, r)
-                const int s = sc[4 * j + e], t = base + j * 128 + 4 * lane + e;
-                const bool gt = s > T, eq = s == T;
-                if (gt || (eq && qb < r)) list[wb.sink_end + gb + min(qb, r)] = t;
-                gb += gt ? 1 : 0;
-                qb += eq ? 1 : 0;
-                if (edge && s == kSumForced) list[t < wb.sink_end ? t : local_pos0 + (t - wb.local_begin)] = t;
+                for (int jj = 1; jj < LD; ++jj)
+                    if (j == jj) ex = excl[jj];
+                const uint32_t low = (1u << e) - 1u;
+                const int gb = run_g + ((before + ex) & 0xffff) + __popc((gtm >> (4 * j)) & low);
+                const int qb = run_q + ((before + ex) >> 16) + __popc((eqm >> (4 * j)) & low);
+                if (((gtm >> i) & 1u) || qb < r) list[wb.sink_end + gb + min(qb, r)] = base + j * 128 + 4 * lane + e;
             }
+        } else {
+            // many CTAs per SM, bound by instruction issue: straight-line code, one predicated store per token
+#pragma unroll
+            for (int j = 0; j < LD; ++j) {
+                int gb = run_g + ((before + excl[j]) & 0xffff), qb = run_q + ((before + excl[j]) >> 16);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const bool gt = (gtm >> (4 * j + e)) & 1u, eq = (eqm >> (4 * j + e)) & 1u;
+                    if (gt || (eq && qb < r)) list[wb.sink_end + gb + min(qb, r)] = base + j * 128 + 4 * lane + e;
+                    gb += gt ? 1 : 0;
+                    qb += eq ? 1 : 0;
+                }
+            }
+        }
+        for (uint32_t m = fm; m; m &= m - 1) {   // edge tiles only
+            const int i = __ffs(m) - 1, t = base + (i >> 2) * 128 + 4 * lane + (i & 3);
+            list[t < wb.sink_end ? t : local_pos0 + (t - wb.local_begin)] = t;
         }
         run_g += tile_total & 0xffff;
         run_q += tile_total >> 16;
