@@ -10,8 +10,9 @@
 //   merge   the CTA histograms meet through distributed shared memory: every CTA reads all of them and derives the
 //           same threshold T (largest level with #{S >= T} >= k), r = k - #{S > T}, and how many tokens with
 //           S > T / S == T lie before its slice;
-//   pass 2  the slice is scored again (the signatures now come from L2; a slice of one tile keeps its scores in
-//           registers) and the selected tokens are written at their final positions: position = #{selected tokens
+//   pass 2  takes the scores of pass 1 from shared memory (one byte per token, groups of up to four heads, slices of up
+//           to 16384 / 65536 tokens; a one-tile slice keeps them in registers; anything else is scored again from L2)
+//           and the selected tokens are written at their final positions: position = #{selected tokens
 //           with a smaller index}, from a prefix sum over lanes, loads and warps.
 // Nothing is kept in global scratch.  Tokens that are always in context (first n_sink, most recent n_local) are
 // written without being scored, exactly as in the maximum variant.
@@ -34,6 +35,7 @@ struct SumArgs {
     long long idx_sb, idx_sh;
     int32_t *count, *hist_out;
     Windows win;
+    int cache_tokens;   // score bytes that fit in the dynamic shared memory of one CTA
 };
 
 // The summed score without one population count per head: for bit position i let c_i = number of the group's query
@@ -107,6 +109,10 @@ __global__ void __launch_bounds__(kSumThreads, LD <= 2 ? 5 : 3) score_sum_select
     __shared__ int s_tot[NB], s_bef[NB];                // whole sequence / slices before this one
     __shared__ int s_wsum[2][kSumWarps];                // pass 2: packed (S > T, S == T) counts per warp, double buffered
     __shared__ int s_T, s_r, s_gtb, s_eqb;
+    // Scores of pass 1, one byte per token (levels 0 .. 128: groups of up to four heads), for slices that fit: pass 2
+    // then neither reloads nor scores again, and compares four tokens per instruction.
+    extern __shared__ uint32_t s_sc[];
+    constexpr bool kCache = (G <= 4);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t rank = (CS > 1) ? cluster_rank() : 0u;
@@ -131,6 +137,7 @@ __global__ void __launch_bounds__(kSumThreads, LD <= 2 ? 5 : 3) score_sum_select
     const int per = ((n + 3) / 4 + CS - 1) / CS * 4;
     const int lo = min(n, (int)rank * per), hi = min(n, lo + per);
     const int n_tiles = (hi - lo + kTileTokens - 1) / kTileTokens;
+    const bool cached = kCache && n_tiles > 1 && hi - lo <= a.cache_tokens;   // a one-tile slice keeps its scores in registers
     const int plain_end = min(wb.local_begin, hi);      // warp tiles inside [sink_end, plain_end) need no per-token checks
     auto is_edge = [&](int base) { return base < wb.sink_end || base + kWarpTokens > plain_end; };
 
@@ -158,6 +165,12 @@ __global__ void __launch_bounds__(kSumThreads, LD <= 2 ? 5 : 3) score_sum_select
                 sum_scores_of<G, LD, false>(v, base, lane, hi, wb, pl, sc);
 #pragma unroll
                 for (int e = 0; e < 4 * LD; ++e) atomicAdd(&c_hist[sc[e]][lane], 1);
+                if (cached) {
+#pragma unroll
+                    for (int j = 0; j < LD; ++j)
+                        s_sc[(base - lo) / 4 + j * 32 + lane] = (uint32_t)sc[4 * j] | ((uint32_t)sc[4 * j + 1] << 8) |
+                                                                 ((uint32_t)sc[4 * j + 2] << 16) | ((uint32_t)sc[4 * j + 3] << 24);
+                }
             }
             if (it + 1 < n_tiles) {
 #pragma unroll
@@ -236,18 +249,28 @@ __global__ void __launch_bounds__(kSumThreads, LD <= 2 ? 5 : 3) score_sum_select
     for (int it = 0; it < n_tiles; ++it) {
         const int base = lo + it * kTileTokens + warp * kWarpTokens;
         const bool edge = is_edge(base);
-        if (n_tiles != 1) {   // a slice of one tile still holds its scores in registers
-            uint4 v[LD];
-            if (edge) { sum_load_tile<LD, true>(row, base, lane, hi, v); sum_scores_of<G, LD, true>(v, base, lane, hi, wb, pl, sc); }
-            else { sum_load_tile<LD, false>(row, base, lane, hi, v); sum_scores_of<G, LD, false>(v, base, lane, hi, wb, pl, sc); }
-        }
         // bit i of the masks: token i of this lane (load i / 4, element i % 4) has S > T / S == T / is always kept
         uint32_t gtm = 0, eqm = 0, fm = 0;
+        if (cached && !edge) {   // score bytes of pass 1, four tokens per comparison (T <= 129 fits a byte)
+            const uint32_t t4 = (uint32_t)T * 0x01010101u;
 #pragma unroll
-        for (int i = 0; i < 4 * LD; ++i) {
-            gtm |= (sc[i] > T ? 1u : 0u) << i;
-            eqm |= (sc[i] == T ? 1u : 0u) << i;
-            if (edge) fm |= (sc[i] == kSumForced ? 1u : 0u) << i;
+            for (int j = 0; j < LD; ++j) {
+                const uint32_t w = s_sc[(base - lo) / 4 + j * 32 + lane];
+                gtm |= high_bits_to_nibble(__vcmpgtu4(w, t4)) << (4 * j);
+                eqm |= high_bits_to_nibble(__vcmpeq4(w, t4)) << (4 * j);
+            }
+        } else {
+            if (n_tiles != 1) {   // a slice of one tile still holds its scores in registers
+                uint4 v[LD];
+                if (edge) { sum_load_tile<LD, true>(row, base, lane, hi, v); sum_scores_of<G, LD, true>(v, base, lane, hi, wb, pl, sc); }
+                else { sum_load_tile<LD, false>(row, base, lane, hi, v); sum_scores_of<G, LD, false>(v, base, lane, hi, wb, pl, sc); }
+            }
+#pragma unroll
+            for (int i = 0; i < 4 * LD; ++i) {
+                gtm |= (sc[i] > T ? 1u : 0u) << i;
+                eqm |= (sc[i] == T ? 1u : 0u) << i;
+                if (edge) fm |= (sc[i] == kSumForced ? 1u : 0u) << i;
+            }
         }
         // packed counts (S > T in the low half, S == T in the high half) of this lane per load, then over the warp
         int excl[LD], warp_total = 0;
@@ -333,10 +356,27 @@ static cudaError_t launch_sum_t(const SumArgs &a, int B, cudaStream_t st) {
             allowed[dev] = true;
         }
     }
+    // score bytes of pass 1 (groups of up to four heads): 16 KB where five CTAs share an SM; 64 KB in the few-CTA variant,
+    // which still lets two CTAs share an SM (with one per SM only seven clusters of 16 are resident at a time)
+    constexpr int kCacheBytes = (G > 4) ? 0 : (LD >= 4 ? 64 * 1024 : 16 * 1024);
+    if (kCacheBytes > 24 * 1024) {
+        static bool sized[64] = {};
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev < 0 || dev >= 64) dev = 0;
+        if (!sized[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(score_sum_select_kernel<G, CS, LD>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kCacheBytes);
+            if (e != cudaSuccess) return e;
+            sized[dev] = true;
+        }
+    }
+    SumArgs args = a;
+    args.cache_tokens = kCacheBytes;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CS, a.Hkv, B);
     cfg.blockDim = dim3(kSumThreads);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = kCacheBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -345,7 +385,7 @@ static cudaError_t launch_sum_t(const SumArgs &a, int B, cudaStream_t st) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, score_sum_select_kernel<G, CS, LD>, a);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, score_sum_select_kernel<G, CS, LD>, args);
     if (e != cudaSuccess) return e;
     count_launch();
     return cudaGetLastError();
@@ -373,7 +413,7 @@ cudaError_t launch_score_topk_sum(int B, int Hq, int Hkv, const uint32_t *q_code
     a.q_codes = q_codes; a.k_codes = k_codes; a.kc_sb = kc_sb; a.kc_sh = kc_sh;
     a.seq_lens = seq_lens; a.k_per_seq = k_per_seq; a.k_uniform = k_uniform; a.k_max = k_max;
     a.Hq = Hq; a.Hkv = Hkv; a.idx = idx; a.idx_sb = idx_sb; a.idx_sh = idx_sh;
-    a.count = count; a.hist_out = hist_out; a.win = win;
+    a.count = count; a.hist_out = hist_out; a.win = win; a.cache_tokens = 0;
     switch (Hq / Hkv) {
         case 1: return launch_sum_g<1>(a, B, st);
         case 2: return launch_sum_g<2>(a, B, st);

@@ -348,6 +348,27 @@ def test_score_topk_sum_every_cluster_size(B, Hkv):
     _check_score_topk(qc, kc, lens, [min(k, 500) for k in ks], Hkv * G, Hkv, n_sink=100, n_local=2100, reduce="sum")
 
 
+def test_score_topk_sum_slices_beyond_the_score_byte_cache():
+    """Slices of up to 16384 tokens (65536 in the few-CTA variant) keep one score byte per token in shared memory
+    between the passes; longer ones are scored twice.  Both kinds in one batch, and one sequence of over a million
+    tokens for the few-CTA variant."""
+    rng = np.random.default_rng(4242)
+    B, Hkv, G = 80, 2, 4                                # 160 units: clusters of 2
+    lens = [int(v) for v in rng.integers(0, 3000, size=B)]
+    lens[3], lens[40], lens[79] = 40000, 30000, 32769   # slices of 20000 (scored twice), 15000 and 16388 tokens
+    n_cap = 40000
+    kc = rng.integers(0, 2 ** 32, size=(B, Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    kc[3, 1] &= np.uint32(0x7)                          # tie blocks
+    qc = rng.integers(0, 2 ** 32, size=(B, Hkv * G), dtype=np.uint64).astype(np.uint32)
+    ks = [n // 16 for n in lens]
+    _check_score_topk(qc, kc, lens, ks, Hkv * G, Hkv, reduce="sum")
+    _check_score_topk(qc, kc, lens, ks, Hkv * G, Hkv, n_sink=128, n_local=128, reduce="sum")
+    n = 1100003                                         # 16 CTAs, slices of 68752 tokens
+    kc1 = rng.integers(0, 2 ** 32, size=(1, 1, n + 1), dtype=np.uint64).astype(np.uint32)
+    qc1 = rng.integers(0, 2 ** 32, size=(1, G), dtype=np.uint64).astype(np.uint32)
+    _check_score_topk(qc1, kc1, [n], [n // 64], G, 1, reduce="sum")
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_score_topk_sum_random_shapes_budgets_windows_and_ties(seed):
     rng = np.random.default_rng(9500 + seed)
