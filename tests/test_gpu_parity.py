@@ -660,6 +660,43 @@ def test_sparse_decode_step_matches_oracle(cfg):
     assert torch.equal(rp["idx"], r["idx"]) and torch.equal(rp["out"], r["out"])
 
 
+def test_step_from_entry_points_with_summed_group_scores():
+    """ENCODE, the summed-score SCORE + TOPK and GATHER-ATT chained through their entry points against the same chain
+    of oracle functions: the lists of ha_score_topk_sum feed ha_gather_attn unchanged."""
+    cfg = wl.Config("sum-chain", 58, 3, [300, 5000, 1], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8)
+    w = wl.make_workload(cfg, DEV)
+    B, Hq, Hkv, G = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, 4
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
+    ws = ha.alloc_workspace(shape, w["n_cap"], w["k_max"])
+    kc = torch.zeros(B, Hkv, (w["n_cap"] + 3) // 4 * 4, dtype=torch.int32, device=DEV)
+    qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+    ha.ha_encode(ha.Mapping(w["map_k"]), 1, w["K"], kc)
+    ha.ha_encode(ha.Mapping(w["map_q"]), G, w["q"], qc.unsqueeze(2))
+    idx = torch.zeros(B, Hkv, w["k_max"], dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=DEV)
+    out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=DEV)
+    ha.ha_score_topk_sum(shape, qc, kc, w["seq_lens"], w["k_per_seq"], 0, w["k_max"], idx, cnt)
+    ha.ha_gather_attn(shape, w["q"], w["K"], w["V"], w["seq_lens"], idx, cnt, w["k_max"], out, ws)
+    torch.cuda.synchronize()
+    assert ha.ha_read_device_status(ws) == 0
+    Kc = oracle_key_codes(w["K"], w["map_k"], w["lens"])
+    Qc = oracle_query_codes(w["q"], w["map_q"], Hkv)
+    assert np.array_equal(codes_np(qc), Qc)
+    qu, Ku, Vu = u16(w["q"]), u16(w["K"]), u16(w["V"])
+    differs = 0
+    for b, (n, k) in enumerate(zip(w["lens"], w["ks"])):
+        for g in range(Hkv):
+            s = oracle.score_sum(Qc[b, g * G:(g + 1) * G], Kc[b, g, :n])
+            exp = oracle.topk(s, k)
+            differs += int(not np.array_equal(exp, oracle.topk(oracle.score(Qc[b, g * G:(g + 1) * G], Kc[b, g, :n]), k)))
+            assert int(cnt[b, g]) == len(exp)
+            assert np.array_equal(idx[b, g, :len(exp)].cpu().numpy(), exp)
+            for j in range(G):
+                eo, _, _ = oracle.gather_attn(qu[b, g * G + j], Ku[b, g], Vu[b, g], exp, sm_scale=w["sm_scale"])
+                assert_out_close(u16(out[b, g * G + j]), eo)
+    assert differs > 0   # the two reductions pick different tokens on these inputs: the test would notice a mix-up
+
+
 @pytest.mark.parametrize("cfg", [
     wl.Config("win-ragged", 55, 3, [300, 2049, 1], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8),     # one fused launch
     wl.Config("win-batch", 56, 24, [900 + 37 * i for i in range(24)], None, 0.02, n_q_heads=8, n_kv_heads=2,
