@@ -175,6 +175,28 @@ int ha_score_topk_sum(const ha_shape *shape, const uint32_t *q_codes, const uint
                       int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, int32_t *hist_out,
                       void *stream);
 
+/* SCORE + TOPK and GATHER-ATT with one index list per QUERY head: no reduction over a GQA group at all.  Query head j
+ * scores the signatures of its KV head j / G by Eq. 1 (Section 4.1) and keeps its own top-k (Section 4), exactly what
+ * the paper defines for one head; GATHER-ATT then reads the K/V rows of KV head j / G through query head j's list, so
+ * the K/V traffic is G times that of the grouped entries.
+ *   ha_score_topk_per_head   arguments as ha_score_topk_sum, except
+ *       idx        out i32 [batch][n_q_heads][k_max] (strides given; idx_stride_h steps over QUERY heads)
+ *       count      out i32 [batch][n_q_heads]
+ *       hist_out   optional out i32 [batch][n_q_heads][33]
+ *     batch * n_q_heads must not exceed 65536 (else HA_ERR_UNSUPPORTED).
+ *   ha_gather_attn_per_head  arguments as ha_gather_attn with idx / count as above (contiguous K/V only); the
+ *     workspace must come from ha_workspace_bytes for the shape with n_kv_heads set to n_q_heads. */
+int ha_score_topk_per_head(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes,
+                           int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens,
+                           const int32_t *k_per_seq, int32_t k_uniform, int32_t k_max, int32_t *idx,
+                           int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, int32_t *hist_out,
+                           void *stream);
+int ha_gather_attn_per_head(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
+                            const ha_tensor *V, const int32_t *seq_lens, const int32_t *idx,
+                            int64_t idx_stride_b, int64_t idx_stride_h, const int32_t *count,
+                            int32_t k_max, uint16_t *out, float *lse, void *workspace, size_t ws_bytes,
+                            void *stream);
+
 /* GATHER-ATT — Section 4: out_j = sum_{i in I} softmax_I(sm_scale <q_j, k_i>) v_i for every
  * query head j, I = idx[b][j / G][0..count).  K/V rows are read in place through the indices
  * (Section 4.4).  fp32 accumulation, one rounding to bf16.

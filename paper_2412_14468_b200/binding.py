@@ -25,6 +25,7 @@ EXPORTS = [
     "ha_gather_attn_paged", "ha_sparse_decode_paged",
     "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
     "ha_score_wide", "ha_inner_products", "ha_sparse_decode_paged_host", "ha_score_topk_sum",
+    "ha_score_topk_per_head", "ha_gather_attn_per_head",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
 
@@ -69,6 +70,8 @@ def lib() -> C.CDLL:
         L.ha_encode_prefill.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, I32, P, P]
         L.ha_score_topk.argtypes = [P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64, P, P, P, SZ, P]
         L.ha_score_topk_sum.argtypes = [P, P, P, I64, I64, P, P, I32, I32, P, I64, I64, P, P, P]
+        L.ha_score_topk_per_head.argtypes = [P, P, P, I64, I64, P, P, I32, I32, P, I64, I64, P, P, P]
+        L.ha_gather_attn_per_head.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P, SZ, P]
         L.ha_gather_attn.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P, SZ, P]
         L.ha_gather_attn_paged.argtypes = [P, P, P, P, P, I64, I32, P, P, I64, I64, P, I32, P, P, P, SZ, P]
         L.ha_gather_attn_static.argtypes = [P, P, P, P, P, P, I64, I64, P, I32, P, P, P]
@@ -91,7 +94,7 @@ def lib() -> C.CDLL:
         for fn in ("ha_workspace_init", "ha_encode", "ha_score_topk", "ha_gather_attn", "ha_gather_attn_static", "ha_dense_decode",
                    "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status", "ha_score_wide",
                    "ha_inner_products", "ha_sparse_decode_paged_host", "ha_sparse_decode_paged", "ha_gather_attn_paged",
-                   "ha_encode_prefill", "ha_score_topk_sum"):
+                   "ha_encode_prefill", "ha_score_topk_sum", "ha_score_topk_per_head", "ha_gather_attn_per_head"):
             getattr(L, fn).restype = C.c_int
         _lib = L
     return _lib
@@ -253,6 +256,25 @@ def ha_score_topk_sum(shape: ha_shape, q_codes, k_codes, seq_lens, k_per_seq, k_
         C.byref(shape), q_codes.data_ptr(), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1),
         seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform, k_max, idx.data_ptr(), idx.stride(0), idx.stride(1),
         count.data_ptr(), _ptr(hist_out), _stream(stream)))
+
+
+def ha_score_topk_per_head(shape: ha_shape, q_codes, k_codes, seq_lens, k_per_seq, k_uniform: int, k_max: int, idx, count,
+                           hist_out=None, stream=None) -> None:
+    """One list per query head (no group reduction): idx int32 [B,Hq,k_max], count int32 [B,Hq], hist_out [B,Hq,33]."""
+    _check("ha_score_topk_per_head", lib().ha_score_topk_per_head(
+        C.byref(shape), q_codes.data_ptr(), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1),
+        seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform, k_max, idx.data_ptr(), idx.stride(0), idx.stride(1),
+        count.data_ptr(), _ptr(hist_out), _stream(stream)))
+
+
+def ha_gather_attn_per_head(shape: ha_shape, q, K, V, seq_lens, idx, count, k_max: int, out, workspace, lse=None,
+                            stream=None) -> None:
+    """GATHER-ATT through per-query-head lists; workspace sized for the shape with n_kv_heads = n_q_heads."""
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K), make_tensor(V)
+    _check("ha_gather_attn_per_head", lib().ha_gather_attn_per_head(
+        C.byref(shape), q.data_ptr(), C.byref(kt), C.byref(vt), seq_lens.data_ptr(), idx.data_ptr(), idx.stride(0),
+        idx.stride(1), count.data_ptr(), k_max, out.data_ptr(), _ptr(lse), p, n, _stream(stream)))
 
 
 def ha_gather_attn(shape: ha_shape, q, K, V, seq_lens, idx, count, k_max: int, out, workspace, lse=None,

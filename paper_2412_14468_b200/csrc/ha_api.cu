@@ -204,6 +204,47 @@ int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
     return HA_OK;
 }
 
+// ---- one list per QUERY head: no reduction over the group (the third reading of how a group selects)
+
+int ha_score_topk_per_head(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes, int64_t kc_stride_b,
+                           int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                           int32_t k_max, int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
+                           int32_t *hist_out, void *stream) {
+    HA_TRY(check_score_args(shape, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_uniform, k_per_seq, 0, k_max,
+                            idx, count));
+    if ((long long)shape->n_q_heads * shape->batch > kMaxUnits) return HA_ERR_UNSUPPORTED;
+    if (shape->batch == 0) return HA_OK;
+    HA_CUDA(launch_score_topk_sum(shape->batch, shape->n_q_heads, shape->n_kv_heads, q_codes, k_codes, kc_stride_b,
+                                  kc_stride_h, seq_lens, k_per_seq, k_uniform, k_max, idx, idx_stride_b, idx_stride_h,
+                                  count, hist_out, (cudaStream_t)stream, Windows{shape->n_sink, shape->n_local}, true));
+    return HA_OK;
+}
+
+int ha_gather_attn_per_head(const ha_shape *shape, const uint16_t *q, const ha_tensor *K, const ha_tensor *V,
+                            const int32_t *seq_lens, const int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h,
+                            const int32_t *count, int32_t k_max, uint16_t *out, float *lse, void *workspace,
+                            size_t ws_bytes, void *stream) {
+    HA_TRY(check_shape(shape));
+    HA_TRY(check_tensor(K));
+    HA_TRY(check_tensor(V));
+    if (!q || !seq_lens || !idx || !count || !out || k_max < 0) return HA_ERR_INVALID_ARG;
+    if ((uintptr_t)q & 15) return HA_ERR_INVALID_ARG;
+    ha_shape units = *shape;             // every query head is a unit: the scratch is laid out for that many
+    units.n_kv_heads = shape->n_q_heads;
+    HA_TRY(check_shape(&units));
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(&units, -1, workspace, ws_bytes, &L));
+    if (shape->batch == 0) return HA_OK;
+    int shift = 0;
+    while ((shape->n_kv_heads << shift) < shape->n_q_heads) ++shift;
+    HA_CUDA(launch_attention(true, shape->batch, shape->n_q_heads, shape->n_q_heads, shape->sm_scale, q, view(K), view(V),
+                             seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
+                             ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),
+                             ws_ptr<int32_t>(workspace, L.off_tickets), ws_ptr<uint32_t>(workspace, 0),
+                             (cudaStream_t)stream, 0, nullptr, 0, Windows{0, 0}, nullptr, 0, 0, shift));
+    return HA_OK;
+}
+
 int ha_gather_attn_paged(const ha_shape *shape, const uint16_t *q, const ha_tensor *K_pool, const ha_tensor *V_pool,
                          const int32_t *block_table, int64_t bt_stride_b, int32_t page_size, const int32_t *seq_lens,
                          const int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, const int32_t *count,

@@ -41,6 +41,7 @@ struct AttnArgs {
     long long bt_sb;
     int page_shift, page_rows;
     int max_items, Hq, Hkv, n_units, balanced;
+    int kv_shift;               // unit head h reads K/V head h >> kv_shift (0 unless every query head has its own list)
     float scale_log2;
     float *part_ml, *part_acc;
     int32_t *tickets;
@@ -182,8 +183,8 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attn_kernel(const AttnArgs a)
         const int start = blk_lo * kBlockTokens, end = min(cnt, blk_hi * kBlockTokens);
 
         const bool paged = kGather && a.block_table != nullptr;   // rows are then addressed from the pool's base
-        const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (paged ? 0LL : (long long)b * a.K.sb) + (long long)kvh * a.K.sh);
-        const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (paged ? 0LL : (long long)b * a.V.sb) + (long long)kvh * a.V.sh);
+        const unsigned char *Kb = reinterpret_cast<const unsigned char *>(a.K.ptr + (paged ? 0LL : (long long)b * a.K.sb) + (long long)(kvh >> a.kv_shift) * a.K.sh);
+        const unsigned char *Vb = reinterpret_cast<const unsigned char *>(a.V.ptr + (paged ? 0LL : (long long)b * a.V.sb) + (long long)(kvh >> a.kv_shift) * a.V.sh);
         const int32_t *pages = paged ? a.block_table + (long long)b * a.bt_sb : nullptr;
         const long long k_row = a.K.sn * 2, v_row = a.V.sn * 2;   // bytes
         const int32_t *list = kGather ? a.idx + (long long)b * a.idx_sb + (long long)kvh * a.idx_sh : nullptr;
@@ -453,8 +454,10 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              long long idx_sb, long long idx_sh, const int32_t *count, int max_items,
                              uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
                              uint32_t *status, cudaStream_t st, int count_from_k, const int32_t *k_per_seq,
-                             int k_uniform, Windows win, const int32_t *block_table, long long bt_sb, int page_shift) {
+                             int k_uniform, Windows win, const int32_t *block_table, long long bt_sb, int page_shift,
+                             int kv_shift) {
     AttnArgs a{};
+    a.kv_shift = kv_shift;
     a.win = win;
     a.block_table = block_table; a.bt_sb = bt_sb; a.page_shift = page_shift;
     a.page_rows = (block_table && K.sn > 0) ? (int)(K.sb / K.sn) : 0;

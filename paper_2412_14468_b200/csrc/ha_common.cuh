@@ -182,11 +182,12 @@ cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, c
                               int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
                               int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st, Windows win = Windows{0, 0});
 
-// SCORE + TOPK with the group's per-head scores added instead of maximised (one cluster per unit, no scratch).
+// SCORE + TOPK with the group's per-head scores added instead of maximised (one cluster per unit, no scratch);
+// per_head: no reduction at all, one list per QUERY head (idx, count, hist_out then have n_q_heads rows per sequence).
 cudaError_t launch_score_topk_sum(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes, long long kc_sb,
                                   long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq, int k_uniform,
                                   int k_max, int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
-                                  int32_t *hist_out, cudaStream_t st, Windows win = Windows{0, 0});
+                                  int32_t *hist_out, cudaStream_t st, Windows win = Windows{0, 0}, bool per_head = false);
 
 cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale, const uint16_t *q,
                              TensorView K, TensorView V, const int32_t *seq_lens, const int32_t *idx,
@@ -194,7 +195,8 @@ cudaError_t launch_attention(bool gather, int B, int Hq, int Hkv, float sm_scale
                              uint16_t *out, float *lse, float *part_ml, float *part_acc, int32_t *tickets,
                              uint32_t *status, cudaStream_t st, int count_from_k = 0,
                              const int32_t *k_per_seq = nullptr, int k_uniform = 0, Windows win = Windows{0, 0},
-                             const int32_t *block_table = nullptr, long long bt_sb = 0, int page_shift = 0);
+                             const int32_t *block_table = nullptr, long long bt_sb = 0, int page_shift = 0,
+                             int kv_shift = 0);   // kv_shift: unit head h reads K/V head h >> kv_shift
 
 // The whole layer-step in one launch (one cluster per unit); only for small batches.  v_new_host != NULL: q,
 // k_new and v_new are mapped host memory and the kernel appends the new K/V rows itself (host-buffer entry).

@@ -36,6 +36,7 @@ struct SumArgs {
     int32_t *count, *hist_out;
     Windows win;
     int cache_tokens;   // score bytes that fit in the dynamic shared memory of one CTA
+    int row_shift;      // unit head h scans the signature row of KV head h >> row_shift (per-query-head lists)
 };
 
 // The summed score without one population count per head: for bit position i let c_i = number of the group's query
@@ -122,7 +123,7 @@ __global__ void __launch_bounds__(kSumThreads, LD <= 2 ? 5 : 3) score_sum_select
     const int nf = forced_before(wb, n);
     const int kb = a.k_per_seq ? a.k_per_seq[b] : a.k_uniform;
     const int keep = max(0, min(min(kb, a.k_max - nf), n - nf));     // heavy tokens retrieved among the others
-    const uint32_t *row = a.k_codes + (long long)b * a.kc_sb + (long long)g * a.kc_sh;
+    const uint32_t *row = a.k_codes + (long long)b * a.kc_sb + (long long)(g >> a.row_shift) * a.kc_sh;
     int32_t *list = a.idx + (long long)b * a.idx_sb + (long long)g * a.idx_sh;
 
     SumPlanes<G> pl;
@@ -407,13 +408,20 @@ static cudaError_t launch_sum_g(const SumArgs &a, int B, cudaStream_t st) {
 cudaError_t launch_score_topk_sum(int B, int Hq, int Hkv, const uint32_t *q_codes, const uint32_t *k_codes, long long kc_sb,
                                   long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq, int k_uniform,
                                   int k_max, int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
-                                  int32_t *hist_out, cudaStream_t st, Windows win) {
+                                  int32_t *hist_out, cudaStream_t st, Windows win, bool per_head) {
     if (B <= 0 || Hkv <= 0) return cudaSuccess;
     SumArgs a;
     a.q_codes = q_codes; a.k_codes = k_codes; a.kc_sb = kc_sb; a.kc_sh = kc_sh;
     a.seq_lens = seq_lens; a.k_per_seq = k_per_seq; a.k_uniform = k_uniform; a.k_max = k_max;
     a.Hq = Hq; a.Hkv = Hkv; a.idx = idx; a.idx_sb = idx_sb; a.idx_sh = idx_sh;
-    a.count = count; a.hist_out = hist_out; a.win = win; a.cache_tokens = 0;
+    a.count = count; a.hist_out = hist_out; a.win = win; a.cache_tokens = 0; a.row_shift = 0;
+    if (per_head) {   // every query head is a unit of its own (one head per group) on the row of its KV head
+        int shift = 0;
+        while ((Hkv << shift) < Hq) ++shift;
+        a.Hkv = Hq;
+        a.row_shift = shift;
+        return launch_sum_g<1>(a, B, st);
+    }
     switch (Hq / Hkv) {
         case 1: return launch_sum_g<1>(a, B, st);
         case 2: return launch_sum_g<2>(a, B, st);

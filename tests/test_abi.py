@@ -135,6 +135,28 @@ def test_summed_group_score_arguments_are_checked_on_the_host(lib):
     assert call(ha.make_shape(0, 32, 8, 0.088)) == ha.HA_OK      # empty batch: no launch
 
 
+def test_per_query_head_arguments_are_checked_on_the_host(lib):
+    fake = 0x1000
+    s = ha.make_shape(2, 32, 8, 0.088)
+    t = ha.ha_tensor(fake, 1 << 20, 1 << 16, 128)
+    sel = lambda shape, q=fake, k=fake, k_max=4, idx=fake: \
+        lib.ha_score_topk_per_head(C.byref(shape), q, k, 16, 16, fake, None, 4, k_max, idx, 0, 0, fake, None, None)
+    assert sel(s, q=None) == ha.HA_ERR_INVALID_ARG
+    assert sel(s, idx=None) == ha.HA_ERR_INVALID_ARG
+    assert sel(s, k=fake + 4) == ha.HA_ERR_INVALID_ARG
+    assert sel(s, k_max=-1) == ha.HA_ERR_INVALID_ARG
+    assert sel(ha.make_shape(4096, 32, 8, 0.088)) == ha.HA_ERR_UNSUPPORTED      # more than 65536 query-head units
+    assert sel(ha.make_shape(0, 32, 8, 0.088)) == ha.HA_OK
+    att = lambda shape, q=fake, ws=fake, nbytes=1 << 30: \
+        lib.ha_gather_attn_per_head(C.byref(shape), q, C.byref(t), C.byref(t), fake, fake, 0, 0, fake, 4, fake, None, ws, nbytes, None)
+    assert att(s, q=None) == ha.HA_ERR_INVALID_ARG
+    assert att(s, ws=None) == ha.HA_ERR_WORKSPACE
+    # the scratch is laid out for one unit per query head: its size is that of the shape with n_kv_heads = n_q_heads
+    per_head = ha.ha_workspace_bytes(ha.make_shape(2, 32, 32, 0.088), 0, 64)
+    assert att(s, nbytes=per_head - 256) == ha.HA_ERR_WORKSPACE
+    assert att(ha.make_shape(0, 32, 8, 0.088), nbytes=per_head) == ha.HA_OK
+
+
 def test_wide_score_and_inner_product_arguments_are_checked_on_the_host(lib):
     fake = 0x1000
     assert lib.ha_score_wide(fake, fake, 100, 96, fake, None) == ha.HA_ERR_UNSUPPORTED        # width not 64/128/256/512

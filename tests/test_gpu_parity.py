@@ -697,6 +697,56 @@ def test_step_from_entry_points_with_summed_group_scores():
     assert differs > 0   # the two reductions pick different tokens on these inputs: the test would notice a mix-up
 
 
+@pytest.mark.parametrize("n_sink,n_local", [(0, 0), (16, 40)])
+@pytest.mark.parametrize("B,Hq,Hkv", [(3, 8, 2), (2, 16, 2), (30, 8, 4), (5, 4, 4)])
+def test_step_from_entry_points_with_one_list_per_query_head(B, Hq, Hkv, n_sink, n_local):
+    """No reduction over the group: every query head scores the signatures of its KV head by Eq. 1, keeps its own
+    top-k and attends through its own list (ha_score_topk_per_head + ha_gather_attn_per_head), against the oracle's
+    single-head score, top-k and GATHER-ATT."""
+    G = Hq // Hkv
+    lens = ([300, 5000, 1] + [int(v) for v in np.random.default_rng(B).integers(0, 2500, size=B)])[:B]
+    cfg = wl.Config("per-head", 59, B, lens, None, 0.02, n_q_heads=Hq, n_kv_heads=Hkv, sparsity=8)
+    w = wl.make_workload(cfg, DEV)
+    k_max = w["k_max"] + n_sink + n_local
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"], n_sink=n_sink, n_local=n_local)
+    ws = ha.alloc_workspace(ha.make_shape(B, Hq, Hq, w["sm_scale"]), w["n_cap"], k_max)   # one unit per query head
+    kc = torch.zeros(B, Hkv, (w["n_cap"] + 3) // 4 * 4, dtype=torch.int32, device=DEV)
+    qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+    ha.ha_encode(ha.Mapping(w["map_k"]), 1, w["K"], kc)
+    ha.ha_encode(ha.Mapping(w["map_q"]), G, w["q"], qc.unsqueeze(2))
+    idx = torch.full((B, Hq, k_max), -7, dtype=torch.int32, device=DEV)
+    cnt = torch.full((B, Hq), -7, dtype=torch.int32, device=DEV)
+    hist = torch.full((B, Hq, 33), -7, dtype=torch.int32, device=DEV)
+    out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(B, Hq, device=DEV)
+    ha.ha_score_topk_per_head(shape, qc, kc, w["seq_lens"], w["k_per_seq"], 0, k_max, idx, cnt, hist_out=hist)
+    ha.ha_gather_attn_per_head(shape, w["q"], w["K"], w["V"], w["seq_lens"], idx, cnt, k_max, out, ws, lse=lse)
+    torch.cuda.synchronize()
+    assert ha.ha_read_device_status(ws) == 0
+    Kc = oracle_key_codes(w["K"], w["map_k"], w["lens"])
+    Qc = oracle_query_codes(w["q"], w["map_q"], Hkv)
+    qu, Ku, Vu = u16(w["q"]), u16(w["K"]), u16(w["V"])
+    idx_np, cnt_np, hist_np = idx.cpu().numpy(), cnt.cpu().numpy(), hist.cpu().numpy()
+    lists_differ = 0
+    for b, (n, k) in enumerate(zip(w["lens"], w["ks"])):
+        for h in range(Hq):
+            s = oracle.score(Qc[b, h:h + 1], Kc[b, h // G, :n])
+            exp = oracle.topk_windows(s, k, n_sink, n_local) if (n_sink or n_local) else oracle.topk(s, k)
+            forced = np.zeros(n, bool)
+            forced[:n_sink] = True
+            forced[max(n - n_local, 0):] = bool(n_local)
+            assert cnt_np[b, h] == len(exp)
+            assert np.array_equal(idx_np[b, h, :len(exp)], exp), (b, h)
+            assert np.all(idx_np[b, h, len(exp):] == -1)
+            assert np.array_equal(hist_np[b, h], np.bincount(s[~forced], minlength=33))
+            lists_differ += int(h % G != 0 and not np.array_equal(exp, idx_np[b, h - 1, :cnt_np[b, h - 1]]))
+            eo, el, _ = oracle.gather_attn(qu[b, h], Ku[b, h // G], Vu[b, h // G], exp, sm_scale=w["sm_scale"])
+            assert_out_close(u16(out[b, h]), eo)
+            if len(exp):
+                assert abs(float(lse[b, h]) - el) < 1e-3
+    assert G == 1 or lists_differ > 0   # heads of one group really select on their own
+
+
 @pytest.mark.parametrize("cfg", [
     wl.Config("win-ragged", 55, 3, [300, 2049, 1], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8),     # one fused launch
     wl.Config("win-batch", 56, 24, [900 + 37 * i for i in range(24)], None, 0.02, n_q_heads=8, n_kv_heads=2,
