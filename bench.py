@@ -563,10 +563,28 @@ def main():
                 nbytes = Bq * 8 * (n_tok * 4 + kq * 4)
                 t_max = cold_kernel_us(lambda: ha.ha_score_topk(shp, qc, kc, ln, None, kq, n_tok, kq, ix, ct, wsq))
                 t_sum = cold_kernel_us(lambda: ha.ha_score_topk_sum(shp, qc, kc, ln, None, kq, kq, ix, ct))
+                ixh = torch.zeros(Bq, 32, kq, dtype=torch.int32, device=device)     # one list per query head
+                cth = torch.zeros(Bq, 32, dtype=torch.int32, device=device)
+                t_head = cold_kernel_us(lambda: ha.ha_score_topk_per_head(shp, qc, kc, ln, None, kq, kq, ixh, cth))
+                nbytes_head = Bq * 32 * (n_tok * 4 + kq * 4)                        # every query head scans its KV head's row
                 red[name] = {"algorithmic_bytes": nbytes,
                              "max_over_heads": {"us": t_max, "frac": nbytes / t_max / 1e3 / peak},
-                             "sum_over_heads": {"us": t_sum, "frac": nbytes / t_sum / 1e3 / peak}}
-                del kc, ix, wsq
+                             "sum_over_heads": {"us": t_sum, "frac": nbytes / t_sum / 1e3 / peak},
+                             "per_query_head": {"us": t_head, "bytes_read_by_the_sms": nbytes_head}}
+                if name == "c2":   # GATHER-ATT through the per-head lists against the grouped lists (4x the K/V rows)
+                    Kr = torch.empty(Bq, 8, n_tok, 128, device=device, dtype=torch.bfloat16).normal_(generator=gs)
+                    Vr = torch.empty(Bq, 8, n_tok, 128, device=device, dtype=torch.bfloat16).normal_(generator=gs)
+                    qr = torch.randn(Bq, 32, 128, device=device, generator=gs).to(torch.bfloat16)
+                    orr = torch.zeros(Bq, 32, 128, device=device, dtype=torch.bfloat16)
+                    wsh = ha.alloc_workspace(ha.make_shape(Bq, 32, 32, 1.0), n_tok, kq, device=device)
+                    ha.ha_score_topk(shp, qc, kc, ln, None, kq, n_tok, kq, ix, ct, wsq)
+                    t_gg = cold_kernel_us(lambda: ha.ha_gather_attn(shp, qr, Kr, Vr, ln, ix, ct, kq, orr, wsq))
+                    t_gh = cold_kernel_us(lambda: ha.ha_gather_attn_per_head(shp, qr, Kr, Vr, ln, ixh, cth, kq, orr, wsh))
+                    rows = Bq * 32 * kq * 512
+                    red[name]["gather_attn_grouped_lists_us"] = t_gg
+                    red[name]["gather_attn_per_head_lists"] = {"us": t_gh, "row_bytes": rows, "frac": rows / t_gh / 1e3 / peak}
+                    del Kr, Vr, wsh
+                del kc, ix, wsq, ixh
             supplementary["score_topk_group_reductions"] = red
             del flush
             torch.cuda.empty_cache()
