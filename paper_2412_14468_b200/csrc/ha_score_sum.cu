@@ -4,7 +4,8 @@
 // head; the layer-step reduces a group with the maximum (33 levels), this is the stand-alone alternative with
 // 32 G + 1 levels.
 //
-// One thread-block cluster (1 to 16 CTAs, by the number of units) per (sequence, KV head): the CTAs cut the signature row into equal contiguous slices.
+// One thread-block cluster (1 to 16 CTAs, by the number of units) per (sequence, KV head): the CTAs cut the
+// signature row into equal contiguous slices.
 //   pass 1  every CTA streams its slice (16-byte loads, the next tile requested before the current one is counted)
 //           into a histogram in shared memory (one counter per level and lane);
 //   merge   the CTA histograms meet through distributed shared memory: every CTA reads all of them and derives the
@@ -16,6 +17,8 @@
 //           with a smaller index}, from a prefix sum over lanes, loads and warps.
 // Nothing is kept in global scratch.  Tokens that are always in context (first n_sink, most recent n_local) are
 // written without being scored, exactly as in the maximum variant.
+// With groups of one head (G = 1, where sum, maximum and Eq. 1 coincide) and one unit per QUERY head the same kernel
+// gives every query head its own list on the signature row of its KV head (row_shift).
 #include "ha_score_dev.cuh"
 
 namespace ha {
