@@ -154,6 +154,29 @@ def make_workload(cfg: Union[str, Config], device: Union[str, torch.device] = "c
     }
 
 
+def shard_heads(w: Dict[str, object], rank: int, world: int) -> Dict[str, object]:
+    """Head-parallel split of one layer's inputs: rank r of `world` keeps KV heads [r * Hkv / world, (r + 1) * Hkv /
+    world), their query heads and their mapping networks; lengths and budgets are shared.  The (sequence, KV head)
+    units of the path are independent, so the shards need no exchange: every rank runs the whole step on its heads and
+    the outputs are the corresponding slices of the unsharded result.  K and V come back as strided views (the entry
+    points take strides), everything else contiguous."""
+    cfg = w["cfg"]
+    Hq, Hkv = cfg.n_q_heads, cfg.n_kv_heads
+    assert 0 <= rank < world and Hkv % world == 0, "the KV heads must divide evenly over the ranks"
+    hk, G = Hkv // world, Hq // Hkv
+    kv = slice(rank * hk, (rank + 1) * hk)
+    qh = slice(rank * hk * G, (rank + 1) * hk * G)
+    out = dict(w)
+    out["cfg"] = dataclasses.replace(cfg, n_q_heads=hk * G, n_kv_heads=hk)
+    out["q"] = w["q"][:, qh].contiguous()
+    out["K"], out["V"] = w["K"][:, kv], w["V"][:, kv]
+    out["k_new"], out["v_new"] = w["k_new"][:, kv].contiguous(), w["v_new"][:, kv].contiguous()
+    out["map_q"] = {k: v[kv].contiguous() for k, v in w["map_q"].items()}
+    out["map_k"] = {k: v[kv].contiguous() for k, v in w["map_k"].items()}
+    out["planted"] = [row[kv] for row in w["planted"]]
+    return out
+
+
 def algorithmic_bytes(lens: Sequence[int], ks: Sequence[int], n_q_heads: int = 32, n_kv_heads: int = 8) -> int:
     """Bytes one sparse layer-step must move: 4 B of key code per cached token, 512 B of K and V
     rows per selected token (per KV head), 512 B of q and out per query head."""

@@ -40,3 +40,54 @@ def test_single_process_passthrough():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.aggregate_over_ranks(3.5, 7.0) == (3.5, 7.0)
+
+
+# ---- head-parallel split: every rank runs the whole step on its KV heads, nothing is exchanged on the data path
+
+def _oracle_step(w):
+    import oracle
+    from paper_2412_14468_b200 import workloads as wl
+    from tests._util import oracle_key_codes, u16
+    Kc = oracle_key_codes(w["K"].contiguous(), w["map_k"], w["lens"])
+    return oracle.decode_step(u16(w["q"]), u16(w["k_new"]), u16(w["K"].contiguous()), u16(w["V"].contiguous()), Kc,
+                              wl.mapping_numpy(w["map_q"]), wl.mapping_numpy(w["map_k"]), w["lens"], w["ks"],
+                              sm_scale=w["sm_scale"], n_threads=1)
+
+
+def _head_worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2412_14468_b200 import workloads as wl
+    cfg = wl.Config("head-shards", 61, 2, [300, 77], None, 0.02, n_q_heads=8, n_kv_heads=4, sparsity=8)
+    w = wl.make_workload(cfg, "cpu")                       # the same seeded inputs on every rank
+    mine = _oracle_step(wl.shard_heads(w, rank, world))
+    out = torch.from_numpy(mine["out"].astype("int32"))    # bf16 bit patterns [B, Hq / world, 128]
+    idx = torch.from_numpy(mine["idx"].astype("int32"))
+    outs = [torch.empty_like(out) for _ in range(world)]
+    idxs = [torch.empty_like(idx) for _ in range(world)]
+    dist.all_gather(outs, out)                             # assembling the result is the only communication
+    dist.all_gather(idxs, idx)
+    ok = None
+    if rank == 0:
+        whole = _oracle_step(w)
+        ok = bool((torch.cat(outs, dim=1).numpy() == whole["out"].astype("int32")).all()
+                  and (torch.cat(idxs, dim=1).numpy() == whole["idx"].astype("int32")).all())
+    dist.barrier()
+    q.put((rank, ok))
+    dist.destroy_process_group()
+
+
+def test_head_parallel_shards_over_two_gloo_ranks_reassemble_the_whole_step():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 31500 + (os.getpid() % 2000)
+    procs = [ctx.Process(target=_head_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=240) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res == [(0, True), (1, None)]

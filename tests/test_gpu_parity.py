@@ -660,6 +660,28 @@ def test_sparse_decode_step_matches_oracle(cfg):
     assert torch.equal(rp["idx"], r["idx"]) and torch.equal(rp["out"], r["out"])
 
 
+@pytest.mark.parametrize("world", [2, 4])
+@pytest.mark.parametrize("B", [2, 20])          # one fused launch per shard / the three-kernel path
+def test_head_parallel_shards_reproduce_the_whole_step(B, world):
+    """The (sequence, KV head) units are independent: the step run on each rank's KV heads alone (strided K/V views,
+    sliced mappings) gives the slices of the unsharded result (signatures, lists and counts bit for bit, outputs to
+    rounding); no exchange exists on the data path."""
+    lens = ([700, 2049] + [500 + 61 * i for i in range(B)])[:B]
+    cfg = wl.Config("head-shards", 62, B, lens, None, 0.02, n_q_heads=16, n_kv_heads=4, sparsity=8)
+    w = wl.make_workload(cfg, DEV)
+    whole = _run_step(w)
+    hk, G = 4 // world, 4
+    for rank in range(world):
+        r = _run_step(wl.shard_heads(w, rank, world))
+        kv, qh = slice(rank * hk, (rank + 1) * hk), slice(rank * hk * G, (rank + 1) * hk * G)
+        assert torch.equal(r["idx"], whole["idx"][:, kv]) and torch.equal(r["cnt"], whole["cnt"][:, kv])
+        assert torch.equal(r["qc"], whole["qc"][:, qh]) and torch.equal(r["kc"], whole["kc"][:, kv])
+        # a shard may take another launch variant than the whole (fewer units): same index sets, while the fp32 sums
+        # are taken in another order
+        assert max_abs_diff_bf16(u16(r["out"]), u16(whole["out"][:, qh].contiguous())) <= OUT_AIM
+        assert float((r["lse"] - whole["lse"][:, qh]).abs().max()) < 1e-3
+
+
 def test_step_from_entry_points_with_summed_group_scores():
     """ENCODE, the summed-score SCORE + TOPK and GATHER-ATT chained through their entry points against the same chain
     of oracle functions: the lists of ha_score_topk_sum feed ha_gather_attn unchanged."""
