@@ -168,7 +168,8 @@ int ha_score_topk(const ha_shape *shape, const uint32_t *q_codes, const uint32_t
  * the idx / count outputs as in ha_score_topk; no workspace and no maximum sequence length are needed (any
  * seq_len >= 0), and
  *   hist_out   optional out i32 [batch][n_kv_heads][32 G + 1]: histogram of the summed scores (windows excluded).
- * The index lists feed ha_gather_attn unchanged. */
+ * The index lists feed ha_gather_attn unchanged.  A plain launch on `stream`; it can be captured into a CUDA graph after
+ * one call outside capture (which sets the kernel's attributes on this device). */
 int ha_score_topk_sum(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *k_codes,
                       int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens,
                       const int32_t *k_per_seq, int32_t k_uniform, int32_t k_max, int32_t *idx,

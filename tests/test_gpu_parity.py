@@ -369,6 +369,45 @@ def test_score_topk_sum_slices_beyond_the_score_byte_cache():
     _check_score_topk(qc1, kc1, [n], [n // 64], G, 1, reduce="sum")
 
 
+def test_score_topk_sum_and_per_head_replay_from_a_cuda_graph():
+    """Both stand-alone selections are plain launches on the caller's stream: captured once (after a first call that
+    sets the kernel attributes), replayed on new signatures."""
+    rng = np.random.default_rng(77)
+    B, Hq, Hkv, n, k = 2, 8, 2, 9000, 300
+    shape = ha.make_shape(B, Hq, Hkv, 1.0)
+    kc = torch.zeros(B, Hkv, n, dtype=torch.int32, device=DEV)
+    qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+    sl = torch.tensor([n, n - 77], dtype=torch.int32, device=DEV)
+    idx = torch.zeros(B, Hkv, k, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=DEV)
+    idx_h = torch.zeros(B, Hq, k, dtype=torch.int32, device=DEV)
+    cnt_h = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        ha.ha_score_topk_sum(shape, qc, kc, sl, None, k, k, idx, cnt, stream=st)
+        ha.ha_score_topk_per_head(shape, qc, kc, sl, None, k, k, idx_h, cnt_h, stream=st)
+        st.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=st):
+            ha.ha_score_topk_sum(shape, qc, kc, sl, None, k, k, idx, cnt, stream=st)
+            ha.ha_score_topk_per_head(shape, qc, kc, sl, None, k, k, idx_h, cnt_h, stream=st)
+    for rep in range(2):
+        kc_np = rng.integers(0, 2 ** 32, size=(B, Hkv, n), dtype=np.uint64).astype(np.uint32)
+        qc_np = rng.integers(0, 2 ** 32, size=(B, Hq), dtype=np.uint64).astype(np.uint32)
+        kc.copy_(torch.from_numpy(kc_np.view(np.int32)))
+        qc.copy_(torch.from_numpy(qc_np.view(np.int32)))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        for b, nb in enumerate([n, n - 77]):
+            for g in range(Hkv):
+                exp = oracle.topk(oracle.score_sum(qc_np[b, 4 * g:4 * g + 4], kc_np[b, g, :nb]), k)
+                assert np.array_equal(idx[b, g].cpu().numpy(), exp) and int(cnt[b, g]) == k
+            for h in range(Hq):
+                exp = oracle.topk(oracle.score(qc_np[b, h:h + 1], kc_np[b, h // 4, :nb]), k)
+                assert np.array_equal(idx_h[b, h].cpu().numpy(), exp) and int(cnt_h[b, h]) == k
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_score_topk_sum_random_shapes_budgets_windows_and_ties(seed):
     rng = np.random.default_rng(9500 + seed)
