@@ -32,7 +32,11 @@ if ROOT not in sys.path:
 
 METRIC = "sparse_decode_attn_us_per_layer_step"
 UNIT = "us"
-FUSED_KERNEL_TRAFFIC_C2 = 6552000   # dram__bytes_read.sum + write per launch, profiles/launch_list_bench_c2.md
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the step's kernel on this workload: NOT measured by this
+# run (a number taken under a profiler is never a bench value) but copied from the ncu capture named beside it
+TRAFFIC_FROM_PROFILE = {"bytes": 6552000, "source": "profiles/launch_list_bench_c2.md", "captured_at_commit": "aed5e69"}
+GATHER_TRAFFIC_FROM_PROFILE = {"bytes": 4275000, "source": "profiles/fused_step_kernel_c2.md", "captured_at_commit": "aed5e69"}
+MIN_TIMED_MS = 50.0                 # the timed region of `steps` steps is repeated until this much has been measured
 WORKLOAD = "c2: B=1, Hq=32, Hkv=8, d=128, ctx=32768, k=1024 (32x), 1% planted keys"
 
 
@@ -107,8 +111,10 @@ class ClockSampler:
 class Replica:
     """One layer's resident state on the device plus the per-step inputs and outputs."""
 
-    def __init__(self, cfg, seed, device, ha, wl, torch, windows=(0, 0)):
+    def __init__(self, cfg, seed, device, ha, wl, torch, windows=(0, 0), shard=None):
         w = wl.make_workload(cfg, device, seed=seed)
+        if shard is not None:                                      # (rank, world): this rank's KV heads of the workload
+            w = wl.shard_heads(w, shard[0], shard[1])
         w["k_max"] += windows[0] + windows[1]                     # index rows hold the always-kept tokens too
         self.w = w
         c = w["cfg"]
@@ -133,7 +139,7 @@ class Replica:
 
 
 class Bench:
-    def __init__(self, cfg_name, n_replicas, device, seed_base=None, windows=(0, 0)):
+    def __init__(self, cfg_name, n_replicas, device, seed_base=None, windows=(0, 0), shard=None):
         import torch
         from paper_2412_14468_b200 import binding as ha
         from paper_2412_14468_b200 import workloads as wl
@@ -142,7 +148,7 @@ class Bench:
         cfg = wl.CONFIGS[cfg_name] if isinstance(cfg_name, str) else cfg_name
         self.cfg = cfg
         base = (wl.BASE_SEED + cfg.index) if seed_base is None else seed_base
-        self.reps = [Replica(cfg, base + 100003 * r, device, ha, wl, torch, windows) for r in range(n_replicas)]
+        self.reps = [Replica(cfg, base + 100003 * r, device, ha, wl, torch, windows, shard) for r in range(n_replicas)]
         r0 = self.reps[0]
         self.ws = ha.alloc_workspace(r0.shape, max(r.w["n_cap"] for r in self.reps), max(r.w["k_max"] for r in self.reps),
                                      device=device)
@@ -192,9 +198,12 @@ class Bench:
                 fn(self.reps[(start + i) % len(self.reps)])
         return g, self.ha.ha_kernel_launches() - before
 
-    def time_steps(self, fn, steps, warmup, sampler=None, barrier=None):
-        """Times exactly `steps` calls of fn (graph replays of R steps + a tail graph); returns
-        (ms total, kernel launches in the timed region)."""
+    def time_steps(self, fn, steps, warmup, sampler=None, barrier=None, min_ms=MIN_TIMED_MS, stats=None):
+        """Times regions of exactly `steps` calls of fn (graph replays of R steps + a tail graph).  The region is
+        repeated, back to back on the stream with an event between two regions, until at least `min_ms` have been
+        measured (5 regions at least), so that a short `steps` never yields a single sub-millisecond sample.
+        Returns (MEDIAN ms per region, kernel launches in one region); `stats`, if given, receives min / median /
+        max ms per region and the number of regions."""
         torch = self.torch
         R = len(self.reps)
         fn(self.reps[0])                     # eager run first: surfaces errors outside capture
@@ -204,23 +213,38 @@ class Bench:
         g_tail, l_tail = (self.capture(fn, tail) if tail else (None, 0))
         wf, wt = divmod(max(warmup, 0), R)
         g_wtail = self.capture(fn, wt)[0] if wt else None
+
+        def region():
+            for _ in range(n_full):
+                g_full.replay()
+            if g_tail:
+                g_tail.replay()
+
         for _ in range(wf):
             g_full.replay()
         if g_wtail:
             g_wtail.replay()
-        torch.cuda.synchronize()
-        if barrier:
-            barrier()
+        # one untimed region: warms the graphs of the region itself and sizes the number of repeats
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        if sampler:
-            sampler.start()
         torch.cuda.synchronize()
         e0.record()
-        for _ in range(n_full):
-            g_full.replay()
-        if g_tail:
-            g_tail.replay()
+        region()
         e1.record()
+        torch.cuda.synchronize()
+        est = max(e0.elapsed_time(e1), 1e-3)
+        n_regions = int(min(4000, max(5, math.ceil(min_ms / est))))
+        if barrier:
+            barrier()
+        if sampler:
+            sampler.start()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_regions + 2)]
+        torch.cuda.synchronize()
+        ev[0].record()
+        region()                             # absorbs the host's launch latency on an idle GPU; not counted
+        for i in range(n_regions):
+            ev[i + 1].record()
+            region()
+        ev[n_regions + 1].record()
         if sampler:
             sampler.sample()
         torch.cuda.synchronize()
@@ -228,7 +252,11 @@ class Bench:
             sampler.stop()
         if barrier:
             barrier()
-        return e0.elapsed_time(e1), n_full * l_full + l_tail
+        ts = sorted(ev[i + 1].elapsed_time(ev[i + 2]) for i in range(n_regions))
+        med = ts[len(ts) // 2]
+        if stats is not None:
+            stats.update({"regions": n_regions, "ms_min": ts[0], "ms_median": med, "ms_max": ts[-1]})
+        return med, n_full * l_full + l_tail
 
 
 def aggregate_over_ranks(elapsed_ms: float, units: float, dist=None, device=None):
@@ -242,6 +270,52 @@ def aggregate_over_ranks(elapsed_ms: float, units: float, dist=None, device=None
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(u, op=dist.ReduceOp.SUM)
     return float(t.item()), float(u.item())
+
+
+def rank_env():
+    """(world size, rank, local rank) as the launcher (torch.distributed.run) exports them."""
+    return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def check_gpus_flag(gpus: int, world: int) -> str:
+    """What `--gpus N` asks for against the job this process is part of: "ok" (they agree), "spawn" (a plain
+    `python bench.py --gpus N` with N > 1: the ranks have to be launched first) or an error message."""
+    if gpus < 1:
+        return f"--gpus must be >= 1, got {gpus}"
+    if gpus == world:
+        return "ok"
+    if world == 1:
+        return "spawn"
+    return f"--gpus {gpus} disagrees with the launcher's WORLD_SIZE={world}: start N ranks for --gpus N"
+
+
+def init_ranks(backend: str, device=None):
+    """Joins the process group the launcher described in the environment (MASTER_ADDR / MASTER_PORT / RANK /
+    WORLD_SIZE); returns torch.distributed, or None for a single process."""
+    world, rank, _ = rank_env()
+    if world == 1:
+        return None
+    import torch.distributed as dist
+    kw = {"device_id": device} if (device is not None and backend == "nccl") else {}
+    dist.init_process_group(backend, rank=rank, world_size=world, **kw)
+    return dist
+
+
+def job_value(ms_region_local: float, steps: int, shard: str, dist=None, device=None):
+    """Whole-job figure of a multi-rank run from every rank's own time for `steps` layer-steps.
+    shard = "replicas": every rank runs its own copy of the workload (weak scaling); the job completes `world`
+    layer-steps per step time, so the job's us per layer-step is the slowest rank's step time / world.
+    shard = "heads": the ranks split the KV heads of ONE workload (strong scaling; no exchange on the data path);
+    a layer-step is complete when the slowest rank is, so the job's us per layer-step is that rank's step time.
+    Returns dict(us_per_step_rank_max, value, scaling, world)."""
+    world = dist.get_world_size() if (dist is not None and dist.is_initialized()) else 1
+    ms_max, total_steps = aggregate_over_ranks(ms_region_local, float(steps), dist, device)
+    us_rank = ms_max * 1e3 / steps
+    if shard == "heads":
+        return {"us_per_step_rank_max": us_rank, "value": us_rank, "scaling": "strong", "world": world,
+                "rank_steps_total": total_steps}
+    return {"us_per_step_rank_max": us_rank, "value": us_rank / world, "scaling": "weak", "world": world,
+            "rank_steps_total": total_steps}
 
 
 # ----------------------------------------------------------------------------- CPU oracle leg
@@ -299,39 +373,81 @@ def main():
     ap.add_argument("--warmup", type=int, default=4096)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--replicas", type=int, default=32)
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="N > 1: every rank runs its own copy of the workload (weak scaling, the default), or the ranks "
+                         "split the KV heads of one workload (strong scaling; the path has no exchange step either way)")
     ap.add_argument("--no-supplementary", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.impl == "reference":
+    world, rank, local = rank_env()
+    if args.impl == "reference":                            # rank 0 alone runs the oracle; nothing to launch
         return run_reference(args)
+    verdict = check_gpus_flag(args.gpus, world)
+    if verdict == "spawn":
+        # `python bench.py --gpus N` without a launcher: start the N ranks the way the driver does, one per GPU
+        port = 29000 + os.getpid() % 2000
+        os.execvp(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                   f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1", "--master-port", str(port),
+                                   os.path.abspath(__file__)] + sys.argv[1:])
+    elif verdict != "ok":
+        sys.exit("bench.py: " + verdict)
 
     import torch
     from paper_2412_14468_b200 import binding as ha
     from paper_2412_14468_b200 import workloads as wl
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if torch.cuda.device_count() < (local + 1):
+        sys.exit(f"bench.py: rank {rank} wants cuda:{local} but only {torch.cuda.device_count()} device(s) are visible")
     torch.cuda.set_device(local)
     device = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(device))
-    barrier = (lambda: dist.barrier()) if world > 1 else None
+    dist = init_ranks("nccl", torch.device(device))
+    barrier = (lambda: dist.barrier()) if dist is not None else None
+    if args.shard == "heads" and wl.CONFIGS["c2"].n_kv_heads % world != 0:
+        sys.exit(f"bench.py: --shard heads needs a rank count that divides the {wl.CONFIGS['c2'].n_kv_heads} KV heads")
 
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     peak, peak_kind = _peaks()
     R = args.replicas
-    bench = Bench("c2", R, device, seed_base=wl.BASE_SEED + 1 + 7919 * rank)
-    cfg = bench.cfg
+    by_heads = args.shard == "heads" and world > 1
+    # replicas: every rank its own seeds; heads: the same workload on every rank, each keeps its KV heads
+    bench = Bench("c2", R, device, seed_base=wl.BASE_SEED + 1 + (0 if by_heads else 7919 * rank),
+                  shard=(rank, world) if by_heads else None)
+    cfg = bench.reps[0].w["cfg"]
     lens, ks = bench.reps[0].w["lens"], bench.reps[0].w["ks"]
     alg_bytes = wl.algorithmic_bytes(lens, ks, cfg.n_q_heads, cfg.n_kv_heads)
 
-    # ---- headline: K layer-steps of the whole path, device-resident inputs
+    # ---- headline: regions of K layer-steps of the whole path, device-resident inputs
     sampler = ClockSampler(local)
-    ms, launches = bench.time_steps(bench.step, steps, warmup, sampler=sampler, barrier=barrier)
-    ms_max, units = aggregate_over_ranks(ms, float(steps), dist if world > 1 else None, device)
-    us_per_step = ms_max * 1e3 / steps                      # per rank
-    value = us_per_step / world                             # whole job: world layer-steps complete per step time
+    tstats = {}
+    ms, launches = bench.time_steps(bench.step, steps, warmup, sampler=sampler, barrier=barrier, stats=tstats)
+    job = job_value(ms, steps, args.shard if world > 1 else "replicas", dist, device)
+    us_per_step = job["us_per_step_rank_max"]               # per rank (max over ranks)
+    value = job["value"]                                    # whole job
+    us_min = tstats["ms_min"] * 1e3 / steps
+
+    # ---- the same step as a decode loop sees it: every layer-step behind an ordinary kernel that writes its q
+    # (a copy kernel without programmatic launch attributes standing in for the QKV projection), so that no part
+    # of a step can run under its predecessor.  `value` above is the steady state of back-to-back independent
+    # steps, whose prologues (weight fetch, signature requests) overlap the step in front.
+    q_src = [r.w["q"].clone() for r in bench.reps]
+
+    def q_writer(r):
+        r.w["q"].copy_(q_src[bench.reps.index(r)])
+
+    def isolated_step(r):
+        q_writer(r)
+        bench.step(r)
+
+    iso_steps = min(steps, 4096)
+    istats, wstats = {}, {}
+    t_iso, _ = bench.time_steps(isolated_step, iso_steps, min(warmup, 256), stats=istats)
+    t_wr, _ = bench.time_steps(q_writer, iso_steps, min(warmup, 256), stats=wstats)
+    latency_isolated_us = (t_iso - t_wr) * 1e3 / iso_steps
+    isolated = {"latency_isolated_us": latency_isolated_us, "step_plus_q_writer_us": t_iso * 1e3 / iso_steps,
+                "q_writer_alone_us": t_wr * 1e3 / iso_steps, "steps": iso_steps, "regions": istats["regions"],
+                "min_us": (istats["ms_min"] - wstats["ms_median"]) * 1e3 / iso_steps,
+                "how": "graph of [ordinary copy kernel writing q -> ha_sparse_decode] per layer-step, minus the same graph "
+                       "with the copy kernels alone"}
 
     # ---- per entry point (graphs over the same replicas), for the roofline of the dominant kernel
     sub_steps = min(steps, 8192)
@@ -346,6 +462,7 @@ def main():
     # (sequence, KV head)), so the timed region contains launches of that kernel only and its average
     # launch duration is the step time itself.
     achieved = alg_bytes / (us_per_step * 1e-6) / 1e9
+    achieved_isolated = alg_bytes / (latency_isolated_us * 1e-6) / 1e9
     g_us = parts["ha_gather_attn"]
     roofline = {
         "bound": "hbm",
@@ -354,13 +471,17 @@ def main():
         "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
         # dram__bytes_read.sum + dram__bytes_write.sum per launch of this kernel on this workload, from the
         # ncu launch list of this very command (profiles/launch_list_bench_c2.md)
-        "traffic": FUSED_KERNEL_TRAFFIC_C2 if launches_per_step < 1.5 else None,
+        "traffic": TRAFFIC_FROM_PROFILE["bytes"] if (launches_per_step < 1.5 and world == 1) else None,
+        "traffic_source": TRAFFIC_FROM_PROFILE if (launches_per_step < 1.5 and world == 1) else None,
         "algorithmic_bytes_per_launch": alg_bytes, "us_per_launch": us_per_step,
         "launches_per_step": launches_per_step,
+        "isolated": {"us_per_launch": latency_isolated_us, "achieved": achieved_isolated, "frac": achieved_isolated / peak},
         "standalone_entry_points": {
             "ha_gather_attn (gather_cluster_kernel<4,8>)": {"algorithmic_bytes": gather_bytes, "us": g_us,
                                                       "achieved": gather_bytes / (g_us * 1e-6) / 1e9,
-                                                      "frac": gather_bytes / (g_us * 1e-6) / 1e9 / peak, "traffic": 4275000},
+                                                      "frac": gather_bytes / (g_us * 1e-6) / 1e9 / peak,
+                                                      "traffic": GATHER_TRAFFIC_FROM_PROFILE["bytes"],
+                                                      "traffic_source": GATHER_TRAFFIC_FROM_PROFILE},
             "ha_score_topk (score_select_cluster_kernel<4,8>)": {"algorithmic_bytes": scan_bytes, "us": parts["ha_score_topk"],
                                                                     "achieved": scan_bytes / (parts["ha_score_topk"] * 1e-6) / 1e9},
             "ha_encode[q] (encode_vec_kernel<1>)": {"us": parts["ha_encode[q]"]},
@@ -383,10 +504,10 @@ def main():
         bench.step_host(bench.reps[i % R])
     e1.record()
     torch.cuda.synchronize()
-    e2e_ms, _ = aggregate_over_ranks(e0.elapsed_time(e1), float(e_steps), dist if world > 1 else None, device)
+    e2e_ms, _ = aggregate_over_ranks(e0.elapsed_time(e1), float(e_steps), dist, device)
     e2e_launches = bench.ha.ha_kernel_launches() - l0
     B = cfg.batch
-    e2e = {"value": e2e_ms * 1e3 / e_steps / world, "unit": UNIT, "steps": e_steps,
+    e2e = {"value": e2e_ms * 1e3 / e_steps / (1 if by_heads else world), "unit": UNIT, "steps": e_steps,
            "h2d_bytes_per_step": B * (cfg.n_q_heads + 2 * cfg.n_kv_heads) * 128 * 2,
            "d2h_bytes_per_step": B * cfg.n_q_heads * 128 * 2, "gpu_launches": e2e_launches}
 
@@ -411,6 +532,16 @@ def main():
                 l2, k2 = b2.reps[0].w["lens"], b2.reps[0].w["ks"]
                 ab = wl.algorithmic_bytes(l2, k2)
                 t_all, _ = b2.time_steps(b2.step, st, 20)
+                qs2 = [r.w["q"].clone() for r in b2.reps]           # the step behind an ordinary kernel that writes q
+
+                def wr2(r, b2=b2, qs2=qs2):
+                    r.w["q"].copy_(qs2[b2.reps.index(r)])
+
+                def iso2(r, b2=b2, wr2=wr2):
+                    wr2(r)
+                    b2.step(r)
+                t_iso2, _ = b2.time_steps(iso2, st, 20)
+                t_wr2, _ = b2.time_steps(wr2, st, 20)
                 t_sc, _ = b2.time_steps(b2.score_topk, st, 20)
                 t_ga, _ = b2.time_steps(b2.gather, st, 20)
                 t_de, _ = b2.time_steps(b2.dense, 40, 4)
@@ -418,7 +549,9 @@ def main():
                 gb = sum(8 * 512 * min(kk, nn) + 32 * 512 for nn, kk in zip(l2, k2))
                 supplementary[name] = {
                     "us_per_layer_step": us, "algorithmic_bytes": ab, "achieved_gbs": ab / (us * 1e-6) / 1e9,
-                    "frac": ab / (us * 1e-6) / 1e9 / peak, "score_topk_us": t_sc * 1e3 / st, "gather_attn_us": t_ga * 1e3 / st,
+                    "frac": ab / (us * 1e-6) / 1e9 / peak, "latency_isolated_us": (t_iso2 - t_wr2) * 1e3 / st,
+                    "frac_isolated": ab / ((t_iso2 - t_wr2) * 1e3 / st * 1e-6) / 1e9 / peak,
+                    "score_topk_us": t_sc * 1e3 / st, "gather_attn_us": t_ga * 1e3 / st,
                     "gather_attn_frac": gb / (t_ga * 1e3 / st * 1e-6) / 1e9 / peak,
                     "dense_us": t_de * 1e3 / 40, "dense_frac": wl.dense_bytes(l2) / (t_de * 1e3 / 40 * 1e-6) / 1e9 / peak,
                     "replicas": reps_n,
@@ -599,17 +732,27 @@ def main():
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-            "ms_per_step": us_per_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": us_per_step / 1e3, "higher_is_better": False, "scaling": job["scaling"], "vs_baseline": None,
+            "value_kind": "steady state of back-to-back independent layer-steps (median over the timed regions); "
+                          "latency_isolated_us is one step behind an ordinary kernel",
+            "latency_isolated_us": latency_isolated_us, "isolated": isolated,
+            "timing": {"regions": tstats["regions"], "steps_per_region": steps, "us_per_step_median": us_per_step,
+                       "us_per_step_min": us_min, "us_per_step_max": tstats["ms_max"] * 1e3 / steps,
+                       "timed_ms_total": tstats["ms_median"] * tstats["regions"]},
             "dtype": "bf16 in/out, fp32 accumulate; u32 signatures", "data": "synthetic",
             "config": {"workload": WORKLOAD, "replicas": R,
                        "l2": f"steps rotate over {R} layer replicas ({R * alg_bytes / 1e6:.0f} MB touched per rotation > 126 MB L2)",
-                       "launch": "CUDA graphs of ha_sparse_decode calls (one fused cluster kernel per step at this batch size)", "parallelism": f"replicas x{world}"},
+                       "launch": "CUDA graphs of ha_sparse_decode calls (one fused cluster kernel per step at this batch size); `value`: steps "
+                                 "back to back (their prologues overlap the step in front), `latency_isolated_us`: every step behind an "
+                                 "ordinary kernel that writes its q",
+                       "parallelism": (f"KV heads split over {world} ranks" if by_heads else f"replicas x{world}")},
             "clocks": sampler.summary(), "gpu_launches": launches, "e2e": e2e, "roofline": roofline,
             "cpu_baseline": cpu_baseline, "breakdown_us": parts, "dense_same_run": dense, "supplementary": supplementary,
             "paper_context": "A100: up to 4.3x (GPT-FAST) / 2.54x (FlashDecode) attention latency reduction at 32x",
         }
         print(json.dumps(line))
-    if world > 1:
+    if dist is not None:
+        dist.barrier()
         dist.destroy_process_group()
 
 

@@ -22,9 +22,16 @@
  *   - Kernels are launched with programmatic stream serialization: a kernel may start while its
  *     predecessor in the stream is finishing, and reads seq_lens, k_per_seq and the key signatures
  *     before it waits for that predecessor.  This is safe behind ordinary kernels and copies (they
- *     complete before anything of this library starts) and inside ha_sparse_decode; a caller whose
- *     own preceding kernel both writes those arrays AND releases its dependents early
- *     (griddepcontrol.launch_dependents) must release them only after the writes.
+ *     complete before anything of this library starts) and between calls of this library: the only
+ *     signatures a library kernel directly in front may still be writing are those of the appended
+ *     tokens, i.e. slot seq_len-1 (ha_encode with slot[b] = seq_len[b]-1, or this step's own k_new)
+ *     and slot seq_len-2 (a layer-step on the same cache for a sequence one token shorter), and every
+ *     scanning kernel reads these again after its wait.  A caller whose own preceding kernel both
+ *     writes those arrays AND releases its dependents early (griddepcontrol.launch_dependents) must
+ *     release them only after the writes.
+ *   - seq_lens[b] <= max_seq_len (where a call takes max_seq_len) and seq_lens[b] <= the number of
+ *     token slots of K, V and k_codes are the caller's promise.  SCORE + TOPK clamps a longer
+ *     sequence to max_seq_len; the append of the host-buffer entries and GATHER-ATT do not clamp.
  *   - Return value: HA_OK, or an HA_ERR_* code for errors detectable on the host (nothing is
  *     enqueued in that case).  Errors only visible on the device (an index outside the sequence)
  *     set a bit in the workspace status word, are skipped, and never trap.
@@ -52,7 +59,8 @@ extern "C" {
 
 /* bits of the device status word (ha_read_device_status) */
 #define HA_DEV_BAD_INDEX 1u /* an idx entry >= seq_len was met and skipped */
-#define HA_DEV_TIMEOUT 2u   /* reserved: a bounded wait gave up (no kernel here spins) */
+#define HA_DEV_TIMEOUT 2u   /* a bounded wait inside a kernel gave up (ha_encode_prefill's tensor-core path, the pipelined
+                               layer-step); the kernel returned early and its outputs are not valid */
 
 #define HA_HEAD_DIM 128
 #define HA_N_BITS 32
@@ -100,7 +108,9 @@ typedef struct ha_tensor {
 } ha_tensor;
 
 /* Bytes of workspace needed by every entry point for shapes up to (shape, max_seq_len, max_k).
- * Returns 0 if the shape is unsupported. */
+ * Returns 0 if the shape is unsupported.  The size depends on the batch, the head counts and
+ * max_seq_len; max_k (>= 0) is checked but does not enter the size, because index lists are the
+ * caller's own buffers. */
 size_t ha_workspace_bytes(const ha_shape *shape, int32_t max_seq_len, int32_t max_k);
 
 /* Clears the workspace header (device status word).  Call once after allocating the workspace

@@ -17,7 +17,7 @@
  *                    (Section 4.1), reported as 32 - Hamming distance; for grouped-query
  *                    attention the group score is the maximum over the query heads that
  *                    share the KV head (reduces to Eq. 1 when the group has one head).
- *   ora_score_sum    the other way to reduce Eq. 1 over a group (an option of ha_score_topk_grouped,
+ *   ora_score_sum    the other way to reduce Eq. 1 over a group (the stand-alone entry ha_score_topk_sum,
  *                    not of the layer-step): the per-head scores added up, 0 .. 32 G; the score
  *                    of the G query signatures concatenated against the key signature repeated.
  *   ora_score_wide   the same score for a signature of b = 64 .. 512 bits kept as b/64 packed

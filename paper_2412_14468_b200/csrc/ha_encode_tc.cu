@@ -558,7 +558,14 @@ __global__ void __launch_bounds__(kU_Threads, 1) encode_umma_kernel(const __grid
         tc_fence_before();
         group_sync(group);   // the group is done with this token buffer and with D before they are reused
     }
-    if (failed && gt == 0 && status) atomicOr(status, HA_DEV_TIMEOUT);
+    if (failed) {
+        // A group that gave up still has work in flight: the tile it prefetched into the other buffer and,
+        // after a timed-out MMA wait, the committed MMAs.  Give both one more bounded wait, so that nothing
+        // lands in shared or tensor memory that this CTA has already given back.
+        if (kTma && w + 2 < w_hi) mbar_wait_parity_bounded(smem_u32(&s_xbar[group][buf ^ 1]), xphase[buf ^ 1]);
+        mbar_wait_parity_bounded(bar, phase ^ 1u);   // returns at once when no MMA is outstanding
+        if (gt == 0 && status) atomicOr(status, HA_DEV_TIMEOUT);
+    }
     cp_async_wait<0>();
     tc_fence_before();
     __syncthreads();

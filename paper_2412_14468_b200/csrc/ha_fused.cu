@@ -400,15 +400,24 @@ __global__ void __launch_bounds__(kFusedThreads, S == 1 ? 2 : 1) fused_step_kern
 #pragma unroll
     for (int j = 0; j < G; ++j) qc[j] = s_codes[j];
     if (!kPreload) load_signatures();
-    if (has_new_key) {   // the appended token's signature replaces whatever the early request saw
-        const uint32_t kc = s_codes[G];
+    // Signatures that the early request may have seen in a stale state: slot n-1 (this step's appended token:
+    // encoded above, or, when the step has no k_new, possibly written by an ha_encode call directly in front)
+    // and slot n-2 (appended by a layer-step on the same cache directly in front, whose kernel lets this one
+    // start before it has stored its signature).  Everything older was complete before this kernel started.
+    auto replace_slot = [&](int t, uint32_t kc) {
 #pragma unroll
         for (int p = 0; p < kL; ++p) {
-            const int e = (n - 1) - (wbase + p * 4);
+            const int e = t - (wbase + p * 4);
             if (p < Lb && e >= 0 && e <= 3) {
                 if (e == 0) c[p].x = kc; else if (e == 1) c[p].y = kc; else if (e == 2) c[p].z = kc; else c[p].w = kc;
             }
         }
+    };
+    if (has_new_key) replace_slot(n - 1, s_codes[G]);
+    if (kPreload) {
+        const int lo = wbase, hi = wbase + 4 * Lb;   // this lane's tokens (contiguous)
+        if (!has_new_key && n - 1 >= lo && n - 1 < hi) replace_slot(n - 1, __ldcg(row + n - 1));
+        if (n - 2 >= lo && n - 2 < hi) replace_slot(n - 2, __ldcg(row + n - 2));
     }
 
     // ---------------- P2: SCORE, histogram, threshold, compaction

@@ -89,7 +89,8 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
         for (int j = 0; j < 4; ++j) {
             const int base = pass + j * 1024 + tid * 4;
             if (base < end) {
-                patch_token(cur[j], base, n - 1, row);   // the appended token may just have been written
+                patch_token(cur[j], base, n - 1, row);   // the appended token may just have been written,
+                patch_token(cur[j], base, n - 2, row);   // and the one before it by a layer-step directly in front
                 const int h0 = hamming(cur[j].x), h1 = hamming(cur[j].y), h2 = hamming(cur[j].z), h3 = hamming(cur[j].w);
                 // bytes 33 - h = score + 1 (0 = no token); no byte borrows because h <= 32
                 uint32_t s4 = 0x21212121u - ((uint32_t)h0 | ((uint32_t)h1 << 8) | ((uint32_t)h2 << 16) | ((uint32_t)h3 << 24));
@@ -327,13 +328,16 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
     if (tid < kBins + 3) s_hist[tid] = 0;
     pdl_launch_dependents();
     pdl_wait();
-    {   // the signature that the preceding ENCODE may just have written: re-read by the one lane that holds it
-        const int e_last = (n - 1) - wb;
+    // the signatures that a library kernel directly in front may just have written (slot n-1 by ENCODE, slot n-2
+    // by a layer-step for the sequence one token shorter): re-read by the one lane that holds them
+#pragma unroll
+    for (int back = 1; back <= 2; ++back) {
+        const int e_last = (n - back) - wb;
         if (e_last >= 0 && e_last < 512 && e_last < 256 * Rb && ((e_last & 255) >> 3) == lane) {
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
-                patch_token(c[2 * j], wb + j * 256 + lane * 8, n - 1, row);
-                patch_token(c[2 * j + 1], wb + j * 256 + lane * 8 + 4, n - 1, row);
+                patch_token(c[2 * j], wb + j * 256 + lane * 8, n - back, row);
+                patch_token(c[2 * j + 1], wb + j * 256 + lane * 8 + 4, n - back, row);
             }
         }
     }

@@ -1,6 +1,6 @@
 """Small, self-ending run of the decode path for profiler captures (ncu) and quick timing.
 
-    python -m paper_2412_14468_b200.profile_case --config c3 --batch 4 --steps 3
+    python profile_case.py --config c3 --batch 4 --steps 3
 
 Runs `steps` plain (un-graphed) layer-steps on one replica; inputs are larger than L2 for c3/c4
 style shapes but stay within a few GB.  Prints the CUDA-event time per step."""
@@ -11,8 +11,15 @@ import dataclasses
 
 import torch
 
-from . import binding as ha
-from . import workloads as wl
+import os
+import sys
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2412_14468_b200 import binding as ha  # noqa: E402
+from paper_2412_14468_b200 import workloads as wl  # noqa: E402
 
 
 def prefill(args):

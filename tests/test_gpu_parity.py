@@ -1016,6 +1016,59 @@ def test_step_edge_cases_empty_sequence_budget_above_length_and_no_new_key(reps)
         assert not u16(out)[0::4].any() and not u16(out)[3::4].any()          # empty selections give zeros
 
 
+@pytest.mark.parametrize("B", [1, 6, 40, 90])   # fused clusters of 8 / of 4 / three kernels / the pipelined kernel
+def test_append_by_a_separate_encode_call_and_consecutive_steps_on_one_cache(B):
+    """Library kernels start while the library kernel in front of them is finishing, and request signatures before they
+    wait for it.  Two sequences of calls in which that kernel writes a signature the next one needs: (1) the Section 4.1
+    append done by its own ha_encode call (slot = seq_len - 1) followed by a step without k_new; (2) two layer-steps back
+    to back on the same cache for lengths n and n + 1, the second of which needs the signature the first appended."""
+    lens = [2000 + 37 * b for b in range(B)]
+    cfg = wl.Config("append", 57, B, [n + 1 for n in lens], 128, 0.02, n_q_heads=8, n_kv_heads=2)
+    w = wl.make_workload(cfg, DEV)                                      # caches of n + 1 tokens per sequence
+    Hq, Hkv, n_cap = 8, 2, w["n_cap"]
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
+    ws = ha.alloc_workspace(shape, n_cap, 128)
+    mq, mk = ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"])
+    Kc = oracle_key_codes(w["K"], w["map_k"], [n + 1 for n in lens])
+    clean = torch.from_numpy(np.pad(Kc, ((0, 0), (0, 0), (0, (-Kc.shape[2]) % 4))).view(np.int32)).to(DEV)
+    stale = clean.clone()
+    ar = torch.arange(B, device=DEV)
+    len1 = torch.tensor(lens, dtype=torch.int32, device=DEV)            # first step: n tokens, appended token n - 1
+    len2 = len1 + 1                                                     # second step: n + 1 tokens, appended token n
+    slot1 = len1 - 1
+    stale[ar, :, len1.long() - 1] = 0x5A5A5A5A
+    stale[ar, :, len2.long() - 1] = 0x0F0F0F0F
+    k1 = w["K"][ar, :, len1.long() - 1].contiguous()
+    k2 = w["K"][ar, :, len2.long() - 1].contiguous()
+    kc = stale.clone()
+    qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+    idx = torch.zeros(B, Hkv, 128, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=DEV)
+    out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=DEV)
+    qu, Ku, Vu = u16(w["q"]), u16(w["K"]), u16(w["V"])
+    mqn, mkn = wl.mapping_numpy(w["map_q"]), wl.mapping_numpy(w["map_k"])
+    ref1 = oracle.decode_step(qu, None, Ku, Vu, Kc.copy(), mqn, mkn, lens, [128] * B, sm_scale=w["sm_scale"], n_threads=4)
+    ref2 = oracle.decode_step(qu, None, Ku, Vu, Kc.copy(), mqn, mkn, [n + 1 for n in lens], [128] * B,
+                              sm_scale=w["sm_scale"], n_threads=4)
+    for _ in range(10):
+        # (1) append by ha_encode, then the step without a new key
+        kc.copy_(stale)
+        ha.ha_encode(mk, 1, k1, kc, slot=slot1)
+        ha.ha_sparse_decode(shape, mq, None, w["q"], None, w["K"], w["V"], kc, len1, None, 128, n_cap, 128, qc, idx, cnt, out, ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(idx.cpu().numpy(), ref1["idx"]) and np.array_equal(cnt.cpu().numpy(), ref1["count"])
+        assert_out_close(u16(out), ref1["out"])
+        # (2) two steps back to back: n tokens, then n + 1 tokens
+        kc.copy_(stale)
+        ha.ha_sparse_decode(shape, mq, mk, w["q"], k1, w["K"], w["V"], kc, len1, None, 128, n_cap, 128, qc, idx, cnt, out, ws)
+        ha.ha_sparse_decode(shape, mq, mk, w["q"], k2, w["K"], w["V"], kc, len2, None, 128, n_cap, 128, qc, idx, cnt, out, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(kc, clean)                                   # both appended signatures are in place
+        assert np.array_equal(idx.cpu().numpy(), ref2["idx"]) and np.array_equal(cnt.cpu().numpy(), ref2["count"])
+        assert_out_close(u16(out), ref2["out"])
+    assert ha.ha_read_device_status(ws) == 0
+
+
 # ---------------------------------------------------------------- wide signatures (SCORE-latency table)
 
 def _wide_codes(rng, n, W):

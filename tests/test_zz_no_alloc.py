@@ -2,8 +2,9 @@
 instance a process whose memory pool already owns the whole GPU, or a plug-in that may only launch
 kernels): its scratch is a fixed array inside the library.  The test calls it through the C ABI
 twice in a row, on different inputs, and compares each result with ha_gather_attn (which uses a
-caller-allocated workspace) within the tolerance of the other attention tests; the second call
-shows that what the first one left in the shared array does no harm.  This file sorts last so that a
+caller-allocated workspace) and, head by head, with the CPU oracle's GATHER-ATT, within the
+tolerance of the other attention tests; the second call shows that what the first one left in the
+shared array does no harm.  This file sorts last so that a
 run that stops at the first failure has already run everything else; it also passes on its own."""
 import math
 
@@ -11,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2412_14468_b200 import binding as ha
 from tests._util import assert_out_close, u16
 
@@ -53,6 +55,17 @@ def test_static_scratch_entry_matches_workspace_entry_on_two_calls_in_a_row():
         both_inf = torch.isinf(lse_ref) & torch.isinf(lse_got)
         assert torch.equal(torch.isinf(lse_ref), torch.isinf(lse_got))
         assert float(((lse_ref - lse_got).abs()[~both_inf]).max()) < 1e-4
+        # ... and directly against the oracle, one query head at a time
+        qu, Ku, Vu, got_u, idx_np, cnt_np = u16(q), u16(K), u16(V), u16(got), idx.cpu().numpy(), cnt.cpu().numpy()
+        lse_np = lse_got.cpu().numpy()
+        G = Hq // Hkv
+        for b in range(B):
+            for h in range(Hq):
+                g = h // G
+                eo, el, _ = oracle.gather_attn(qu[b, h], Ku[b, g], Vu[b, g], idx_np[b, g, :cnt_np[b, g]],
+                                               sm_scale=1.0 / math.sqrt(128), n_valid=int(sl[b]))
+                assert_out_close(got_u[b, h], eo)
+                assert (np.isneginf(el) and np.isneginf(lse_np[b, h])) or abs(float(lse_np[b, h]) - el) < 1e-3
 
 
 def test_static_scratch_entry_rejects_problems_beyond_its_limit():
