@@ -80,8 +80,8 @@ size_t ha_workspace_bytes(const ha_shape *shape, int32_t max_seq_len, int32_t ma
 
 int ha_workspace_init(void *workspace, size_t ws_bytes, void *stream) {
     if (!workspace || ((uintptr_t)workspace & 255) || ws_bytes < kHeaderBytes) return HA_ERR_WORKSPACE;
-    // status word and the ticket counters (which every call leaves at zero again)
-    size_t n = kHeaderBytes + (size_t)kMaxUnits * 4;
+    // status and abort words, the ticket counters and the release counters (which every call leaves at zero again)
+    size_t n = kHeaderBytes + (size_t)3 * kMaxUnits * 4;
     if (n > ws_bytes) n = ws_bytes;
     HA_CUDA(cudaMemsetAsync(workspace, 0, n, (cudaStream_t)stream));
     return HA_OK;
@@ -342,6 +342,19 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
         jk.map = view(map_k);
     }
     HA_CUDA(launch_encode_vectors(jq, jk, st));
+    if (pipe_step_eligible(B, Hq, Hkv)) {
+        // SCORE + TOPK and GATHER-ATT in one persistent kernel: the scoring of later units runs under the row fetch of earlier ones
+        int32_t *counters = ws_ptr<int32_t>(workspace, L.off_tickets);
+        const size_t units = (size_t)B * Hkv;
+        HA_CUDA(launch_pipe_step(B, Hq, Hkv, shape->sm_scale, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq,
+                                 k_uniform, max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, q, view(K), view(V), out,
+                                 lse, counters, counters + units, counters + 2 * units, ws_ptr<int32_t>(workspace, L.off_hist),
+                                 ws_ptr<unsigned char>(workspace, L.off_scores), (long long)score_row_bytes(max_seq_len),
+                                 ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),
+                                 ws_ptr<uint32_t>(workspace, 0), st, Windows{shape->n_sink, shape->n_local}, block_table,
+                                 bt_stride_b, page_shift));
+        return HA_OK;
+    }
     HA_CUDA(launch_score_topk(B, Hq, Hkv, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
                               max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, nullptr,
                               ws_ptr<int32_t>(workspace, L.off_hist), ws_ptr<unsigned char>(workspace, L.off_scores), st,

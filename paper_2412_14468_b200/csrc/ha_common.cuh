@@ -26,7 +26,8 @@ constexpr int kMaxUnits = 65536;       // (sequence, KV head) pairs: bounds the 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t off_tickets;   // i32 [B][Hkv]  arrival counters of the split-K merge; zero between calls
+    size_t off_tickets;   // i32 [3][B][Hkv]  arrival counters of the split-K merge, then the two release counters per unit
+                          // of the pipelined step (first pass / second pass of SCORE + TOPK done); all zero between calls
     size_t off_hist;      // i32 [B][Hkv][kMaxChunks][33]   per-chunk score histograms
     size_t off_part_ml;   // f32 [slots][G][2]    split-K running max (log2 domain) and sum, slots = kMaxAttnCtas + B*Hkv
     size_t off_part_acc;  // f32 [slots][G][128]  split-K unnormalised outputs
@@ -35,16 +36,16 @@ struct WorkspaceLayout {
     size_t off_stage_v;   // bf16 [B][Hkv][128]
     size_t off_stage_out; // bf16 [B][Hq][128]
     size_t off_qcodes;    // u32 [B][Hq]
-    size_t off_scores;    // u8 [B][Hkv][round_up(max_seq_len, 16)]  group scores (long-sequence path only)
+    size_t off_scores;    // u8 [B][Hkv][round_up(max_seq_len, 256)]  group scores (long-sequence path, shared units of the pipelined step)
     size_t total;
 };
 
-inline size_t score_row_bytes(int max_seq_len) { return align_up((size_t)(max_seq_len > 0 ? max_seq_len : 0), 16); }
+inline size_t score_row_bytes(int max_seq_len) { return align_up((size_t)(max_seq_len > 0 ? max_seq_len : 0), 256); }
 
 inline WorkspaceLayout make_layout(int B, int Hq, int Hkv, int max_seq_len) {
     WorkspaceLayout L;
     size_t o = kHeaderBytes;
-    L.off_tickets = o;   o = align_up(o + (size_t)B * Hkv * 4, 256);
+    L.off_tickets = o;   o = align_up(o + (size_t)3 * B * Hkv * 4, 256);
     L.off_hist = o;      o = align_up(o + (size_t)B * Hkv * kMaxChunks * kBins * 4, 256);
     const size_t slots = (size_t)kMaxAttnCtas + (size_t)B * Hkv, G = (size_t)(Hq / (Hkv > 0 ? Hkv : 1));
     L.off_part_ml = o;   o = align_up(o + slots * G * 2 * 4, 256);
@@ -209,6 +210,17 @@ cudaError_t launch_fused_step(int B, int Hq, int Hkv, float sm_scale, const MapV
                               long long idx_sb, long long idx_sh, int32_t *count, uint16_t *out, float *lse,
                               cudaStream_t st, Windows win = Windows{0, 0}, const int32_t *block_table = nullptr,
                               long long bt_sb = 0, int page_shift = 0, const uint16_t *v_new_host = nullptr);
+
+// SCORE + TOPK and GATHER-ATT of a step in one persistent kernel whose SCORE warps run ahead of its GATHER warps
+// (steps of more units than the single-cluster kernel holds; the query signatures come from ENCODE in front).
+bool pipe_step_eligible(int B, int Hq, int Hkv);
+cudaError_t launch_pipe_step(int B, int Hq, int Hkv, float sm_scale, const uint32_t *q_codes, const uint32_t *k_codes,
+                             long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq, int k_uniform,
+                             int max_seq_len, int k_max, int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
+                             const uint16_t *q, TensorView K, TensorView V, uint16_t *out, float *lse, int32_t *tickets,
+                             int32_t *s1_done, int32_t *s2_done, int32_t *ws_hist, unsigned char *ws_scores, long long score_row,
+                             float *part_ml, float *part_acc, uint32_t *status, cudaStream_t st, Windows win = Windows{0, 0},
+                             const int32_t *block_table = nullptr, long long bt_sb = 0, int page_shift = 0);
 
 // Stand-alone GATHER-ATT with one 8-CTA cluster per unit (few units, short lists).
 bool gather_cluster_eligible(int B, int Hq, int Hkv, int k_max);

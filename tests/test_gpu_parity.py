@@ -700,7 +700,7 @@ def test_sparse_decode_step_matches_oracle(cfg):
 
 
 @pytest.mark.parametrize("world", [2, 4])
-@pytest.mark.parametrize("B", [2, 20])          # one fused launch per shard / the three-kernel path
+@pytest.mark.parametrize("B", [2, 20])          # one fused launch per shard / ENCODE + the pipelined kernel
 def test_head_parallel_shards_reproduce_the_whole_step(B, world):
     """The (sequence, KV head) units are independent: the step run on each rank's KV heads alone (strided K/V views,
     sliced mappings) gives the slices of the unsharded result (signatures, lists and counts bit for bit, outputs to
@@ -894,7 +894,7 @@ def test_sparse_decode_step_over_a_paged_cache(cfg, page_size):
 
 @pytest.mark.parametrize("seed", range(14))
 def test_sparse_decode_step_random_configs(seed):
-    """Seeded sweep over batch (both the fused launch and the three-kernel path), KV heads, group size, ragged
+    """Seeded sweep over batch (both the fused launch and ENCODE + the pipelined kernel), KV heads, group size, ragged
     lengths, sparsity and window sizes; everything the step returns is checked against the oracle."""
     rng = np.random.default_rng(7000 + seed)
     B = int(rng.integers(1, 13)) if seed < 8 else int(rng.integers(13, 110))   # up to 24 units / up to 220 units
@@ -923,22 +923,25 @@ def test_sparse_decode_step_random_configs(seed):
     # 60 units: clusters of 4 (two query vectors per encoding CTA, 32 tokens per thread)
     (wl.Config("fused-60-units", 84, 30, [1500 + 97 * i for i in range(30)], None, 0.02, n_q_heads=8, n_kv_heads=2,
                sparsity=8), 1),
-    # 100 units: more clusters of four than the device holds at once
+    # 100 units: more clusters of four than the device holds at once: ENCODE, then the pipelined kernel
     (wl.Config("split-100-units", 85, 50, [2500 + 301 * i for i in range(50)], None, 0.02, n_q_heads=16, n_kv_heads=2,
-               sparsity=16), 3),
+               sparsity=16), 2),
     # 6 units, budgets above 2048 rows: one fused launch of the two-stage variant, several blocks per warp
     (wl.Config("fused-large-k", 81, 3, [9000, 5000, 12001], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=2), 1),
     # 20 units with budgets of 1500 rows: more clusters than the two-stage variant holds at once, so the
     # one-stage variant takes them, two blocks per warp one after the other
     (wl.Config("fused-20-units-1500", 86, 10, [6000 + 7 * i for i in range(10)], None, 0.02, n_q_heads=8, n_kv_heads=2,
                sparsity=4), 1),
-    # 20 units with budgets above 2048 rows: three kernels
+    # 20 units with budgets above 2048 rows: ENCODE, then the pipelined kernel
     (wl.Config("split-large-k", 82, 10, [6000 + 7 * i for i in range(10)], None, 0.02, n_q_heads=8, n_kv_heads=2,
-               sparsity=2), 3),
+               sparsity=2), 2),
+    # 1200 units: beyond what the pipelined kernel's work split holds: ENCODE, SCORE + TOPK, GATHER-ATT as three kernels
+    (wl.Config("three-kernels-1200-units", 87, 600, [150 + (37 * i) % 200 for i in range(600)], None, 0.02, n_q_heads=4,
+               n_kv_heads=2, sparsity=8), 3),
 ])
 def test_sparse_decode_step_every_launch_variant(cfg, launches):
-    """The step picks the fused cluster kernel (one or two row stages per warp) or the three-kernel path from
-    the number of units and the budget; each choice gives the oracle's result."""
+    """The step picks the fused cluster kernel (one or two row stages per warp) or ENCODE followed by the pipelined
+    SCORE + TOPK + GATHER-ATT kernel from the number of units and the budget; each choice gives the oracle's result."""
     w = wl.make_workload(cfg, DEV)
     _run_step(w)                                   # first call: attributes, occupancy query
     before = ha.ha_kernel_launches()
@@ -963,6 +966,62 @@ def test_sparse_decode_step_every_launch_variant(cfg, launches):
     assert torch.equal(rh["idx"], r["idx"]) and torch.equal(rh["out"], r["out"])
 
 
+@pytest.mark.parametrize("name,B,Hq,Hkv,lens,sparsity,windows", [
+    # 120 ragged units, a few blocks each: most CTAs of the persistent kernel share units with their neighbours
+    ("ragged-120-units", 60, 8, 2, [1 + (997 * i) % 5000 for i in range(60)], 8, (0, 0)),
+    # 200 short units: several whole units per CTA, empty sequences and one-token sequences among them
+    ("short-200-units", 100, 4, 2, [(53 * i) % 300 for i in range(100)], 4, (0, 0)),
+    # 6 long units: every unit is scored by many CTAs, chunk by chunk, through the workspace
+    ("long-6-units", 3, 8, 2, [70001, 40000, 9], 16, (0, 0)),
+    # 128 units of 9000 tokens with half of them selected: units of more than 32768 / fewer tokens side by side
+    ("wide-budget-128-units", 64, 4, 2, [9000 - 13 * i for i in range(64)], 2, (0, 0)),
+    # one unit longer than the score bytes a CTA keeps in shared memory, owned by ONE CTA (tiny budgets around it)
+    ("owned-long-unit", 40, 4, 2, [40000] + [600] * 39, 1000, (0, 0)),
+    # always-kept windows on shared units; groups of one and of eight query heads
+    ("windows-150-units", 75, 16, 2, [300 + (211 * i) % 4000 for i in range(75)], 8, (16, 100)),
+    ("one-head-groups", 80, 2, 2, [1 + (389 * i) % 3000 for i in range(80)], 8, (0, 0)),
+    ("eight-head-groups", 40, 16, 2, [2000 + 77 * i for i in range(40)], 16, (3, 0)),
+])
+def test_pipelined_step_ragged_lengths_shared_and_owned_units(name, B, Hq, Hkv, lens, sparsity, windows):
+    """Steps that take the persistent SCORE + TOPK + GATHER-ATT kernel (more units than the single-cluster kernel holds,
+    or sequences beyond its length): whole units per CTA, units shared by neighbouring CTAs, units scored chunk by chunk
+    through the workspace, empty selections; run twice on the same workspace (the release counters must be back at
+    zero) and compared with the oracle on everything the step returns."""
+    cfg = wl.Config(name, 90 + len(name), B, lens, None, 0.02, n_q_heads=Hq, n_kv_heads=Hkv, sparsity=sparsity)
+    w = wl.make_workload(cfg, DEV)
+    n_sink, n_local = windows
+    before = ha.ha_kernel_launches()
+    r = _run_step(w, n_sink=n_sink, n_local=n_local)
+    assert ha.ha_kernel_launches() - before == 3            # prompt signatures, ENCODE of the step, the pipelined kernel
+    Kc = oracle_key_codes(w["K"], w["map_k"], w["lens"])
+    ref = oracle.decode_step(u16(w["q"]), u16(w["k_new"]), u16(w["K"]), u16(w["V"]), Kc.copy(),
+                             wl.mapping_numpy(w["map_q"]), wl.mapping_numpy(w["map_k"]), w["lens"], w["ks"],
+                             sm_scale=w["sm_scale"], n_threads=4, n_sink=n_sink, n_local=n_local)
+    assert np.array_equal(codes_np(r["qc"]), ref["qcodes"])
+    assert np.array_equal(r["cnt"].cpu().numpy(), ref["count"])
+    assert np.array_equal(r["idx"].cpu().numpy(), ref["idx"])
+    assert_out_close(u16(r["out"]), ref["out"])
+    got_lse = r["lse"].cpu().numpy().astype(np.float64)
+    finite = np.isfinite(ref["lse"])
+    assert np.array_equal(np.isneginf(got_lse), ~finite)
+    assert np.max(np.abs(got_lse[finite] - ref["lse"][finite]), initial=0.0) < 1e-3
+    # the same step three times in a row on ONE workspace: every call must find the counters at zero
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"], n_sink=n_sink, n_local=n_local)
+    k_max = w["k_max"] + n_sink + n_local
+    ws = ha.alloc_workspace(shape, w["n_cap"], k_max)
+    mq, mk = ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"])
+    for _ in range(3):
+        idx = torch.full((B, Hkv, k_max), 7, dtype=torch.int32, device=DEV)
+        cnt = torch.full((B, Hkv), 7, dtype=torch.int32, device=DEV)
+        out = torch.full((B, Hq, 128), 3.0, dtype=torch.bfloat16, device=DEV)
+        qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+        ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], r["kc"], w["seq_lens"], w["k_per_seq"], 0,
+                            w["n_cap"], k_max, qc, idx, cnt, out, ws)
+        torch.cuda.synchronize()
+        assert ha.ha_read_device_status(ws) == 0
+        assert torch.equal(idx, r["idx"]) and torch.equal(cnt, r["cnt"]) and torch.equal(out, r["out"])
+
+
 def test_k_equals_n_sparse_step_equals_dense_kernel():
     cfg = wl.Config("k=n", 52, 2, [1500, 900], None, 0.0, n_q_heads=8, n_kv_heads=2, sparsity=1)
     w = wl.make_workload(cfg, DEV)
@@ -975,7 +1034,7 @@ def test_k_equals_n_sparse_step_equals_dense_kernel():
     assert r["cnt"].cpu().tolist() == [[1500, 1500], [900, 900]]
 
 
-@pytest.mark.parametrize("reps", [1, 5, 12, 40])     # 8 / 40 units: fused kernel, clusters of 8 / 4; 96 and 320 units: three-kernel path
+@pytest.mark.parametrize("reps", [1, 5, 12, 40])     # 8 / 40 units: fused kernel, clusters of 8 / 4; 96 and 320 units: ENCODE + the pipelined kernel
 def test_step_edge_cases_empty_sequence_budget_above_length_and_no_new_key(reps):
     # one launch covers: an empty sequence, a one-token sequence, k > n, k = 0; then the same without a new key
     cfg = wl.Config("edges", 53, 4 * reps, [0, 1, 37, 2500] * reps, 64, 0.0, n_q_heads=8, n_kv_heads=2)
@@ -1016,7 +1075,7 @@ def test_step_edge_cases_empty_sequence_budget_above_length_and_no_new_key(reps)
         assert not u16(out)[0::4].any() and not u16(out)[3::4].any()          # empty selections give zeros
 
 
-@pytest.mark.parametrize("B", [1, 6, 40, 90])   # fused clusters of 8 / of 4 / three kernels / the pipelined kernel
+@pytest.mark.parametrize("B", [1, 6, 40, 90])   # fused clusters of 8 / of 4 / ENCODE + the pipelined kernel (80 and 180 units)
 def test_append_by_a_separate_encode_call_and_consecutive_steps_on_one_cache(B):
     """Library kernels start while the library kernel in front of them is finishing, and request signatures before they
     wait for it.  Two sequences of calls in which that kernel writes a signature the next one needs: (1) the Section 4.1
