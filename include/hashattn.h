@@ -59,8 +59,8 @@ extern "C" {
 
 /* bits of the device status word (ha_read_device_status) */
 #define HA_DEV_BAD_INDEX 1u /* an idx entry >= seq_len was met and skipped */
-#define HA_DEV_TIMEOUT 2u   /* a bounded wait inside a kernel gave up (ha_encode_prefill's tensor-core path, the pipelined
-                               layer-step); the kernel returned early and its outputs are not valid */
+#define HA_DEV_TIMEOUT 2u   /* a bounded wait inside a kernel gave up (ha_encode_prefill's tensor-core path,
+                               ha_sparse_decode_pipelined); the kernel returned early and its outputs are not valid */
 
 #define HA_HEAD_DIM 128
 #define HA_N_BITS 32
@@ -254,6 +254,24 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
                      int32_t k_uniform, int32_t max_seq_len, int32_t k_max, uint32_t *q_codes,
                      int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
                      uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream);
+
+/* The same layer-step (Section 4 recipe; Section 4.1 "Implementation") on another schedule: ENCODE, then ONE persistent
+ * kernel in which every SM's SCORE + TOPK warps run ahead of its GATHER-ATT warps over a range of (sequence, KV head)
+ * units, so that the bit counting of later units (Eq. 1) overlaps the K/V row fetch of earlier ones; units are released
+ * to the GATHER-ATT warps through counters in the workspace.  Arguments, outputs and results as ha_sparse_decode
+ * (signatures, counts and index lists bit-identical; outputs to fp32 reordering); contiguous K/V only;
+ * batch * n_kv_heads <= 1024 (else HA_ERR_UNSUPPORTED).  If a wait inside the kernel runs out (it never should: all
+ * CTAs are resident at once) the kernel ends early, raises HA_DEV_TIMEOUT in the workspace status word and the outputs
+ * must not be used; call ha_workspace_init before the workspace is used again.
+ * On B200 ha_sparse_decode is the faster of the two at every shape measured so far: scoring needs most of an SM's warp
+ * slots to keep its population-count unit busy, which the row fetch's registers and shared memory do not leave. */
+int ha_sparse_decode_pipelined(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k,
+                               const uint16_t *q, const uint16_t *k_new, const ha_tensor *K, const ha_tensor *V,
+                               uint32_t *k_codes, int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens,
+                               const int32_t *k_per_seq, int32_t k_uniform, int32_t max_seq_len, int32_t k_max,
+                               uint32_t *q_codes, int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h,
+                               int32_t *count, uint16_t *out, float *lse, void *workspace, size_t ws_bytes,
+                               void *stream);
 
 /* One whole layer-step over a paged K/V cache: ha_sparse_decode with K/V addressed as in
  * ha_gather_attn_paged (pools + block table + page_size); the signature cache k_codes stays contiguous. */

@@ -25,7 +25,7 @@ EXPORTS = [
     "ha_gather_attn_paged", "ha_sparse_decode_paged",
     "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
     "ha_score_wide", "ha_inner_products", "ha_sparse_decode_paged_host", "ha_score_topk_sum",
-    "ha_score_topk_per_head", "ha_gather_attn_per_head",
+    "ha_score_topk_per_head", "ha_gather_attn_per_head", "ha_sparse_decode_pipelined",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
 
@@ -78,6 +78,8 @@ def lib() -> C.CDLL:
         L.ha_dense_decode.argtypes = [P, P, P, P, P, I32, P, P, P, SZ, P]
         L.ha_sparse_decode.argtypes = [P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, P, I64, I64, P,
                                        P, P, P, SZ, P]
+        L.ha_sparse_decode_pipelined.argtypes = L.ha_sparse_decode.argtypes
+        L.ha_sparse_decode_pipelined.restype = C.c_int
         L.ha_sparse_decode_paged.argtypes = [P, P, P, P, P, P, P, P, I64, I32, P, I64, I64, P, P, I32, I32, I32, P, P, I64, I64,
                                              P, P, P, P, SZ, P]
         L.ha_sparse_decode_host.argtypes = [P, P, P, P, P, P, P, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64,
@@ -322,6 +324,19 @@ def ha_sparse_decode(shape: ha_shape, map_q: Mapping, map_k: Optional[Mapping], 
     p, n = _ws(workspace)
     kt, vt = make_tensor(K), make_tensor(V)
     _check("ha_sparse_decode", lib().ha_sparse_decode(
+        C.byref(shape), map_q.ref, None if map_k is None else map_k.ref, q.data_ptr(), _ptr(k_new), C.byref(kt),
+        C.byref(vt), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1), seq_lens.data_ptr(), _ptr(k_per_seq),
+        k_uniform, max_seq_len, k_max, q_codes.data_ptr(), idx.data_ptr(), idx.stride(0), idx.stride(1),
+        count.data_ptr(), out.data_ptr(), _ptr(lse), p, n, _stream(stream)))
+
+
+def ha_sparse_decode_pipelined(shape: ha_shape, map_q: Mapping, map_k: Optional[Mapping], q, k_new, K, V, k_codes, seq_lens,
+                               k_per_seq, k_uniform: int, max_seq_len: int, k_max: int, q_codes, idx, count, out, workspace,
+                               lse=None, stream=None) -> None:
+    """ha_sparse_decode on the schedule that runs SCORE + TOPK ahead of GATHER-ATT inside one persistent kernel."""
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K), make_tensor(V)
+    _check("ha_sparse_decode_pipelined", lib().ha_sparse_decode_pipelined(
         C.byref(shape), map_q.ref, None if map_k is None else map_k.ref, q.data_ptr(), _ptr(k_new), C.byref(kt),
         C.byref(vt), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1), seq_lens.data_ptr(), _ptr(k_per_seq),
         k_uniform, max_seq_len, k_max, q_codes.data_ptr(), idx.data_ptr(), idx.stride(0), idx.stride(1),

@@ -303,7 +303,7 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
                               int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
                               int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx, int64_t idx_stride_b,
                               int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse, void *workspace,
-                              size_t ws_bytes, void *stream, const uint16_t *v_new_host = nullptr) {
+                              size_t ws_bytes, void *stream, const uint16_t *v_new_host = nullptr, bool pipelined = false) {
     HA_TRY(check_score_args(shape, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_uniform, k_per_seq,
                             max_seq_len, k_max, idx, count));
     HA_TRY(check_mapping(map_q, shape->n_kv_heads));
@@ -317,7 +317,8 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
     cudaStream_t st = (cudaStream_t)stream;
     const int B = shape->batch, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
 
-    if (fused_step_eligible(B, Hq, Hkv, max_seq_len, k_max)) {
+    if (pipelined && !pipe_step_eligible(B, Hq, Hkv)) return HA_ERR_UNSUPPORTED;
+    if (!pipelined && fused_step_eligible(B, Hq, Hkv, max_seq_len, k_max)) {
         // small batch: the whole step is one cluster kernel
         HA_CUDA(launch_fused_step(B, Hq, Hkv, shape->sm_scale, view(map_q), k_new ? view(map_k) : MapView{}, q, k_new,
                                   view(K), view(V), k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
@@ -342,7 +343,7 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
         jk.map = view(map_k);
     }
     HA_CUDA(launch_encode_vectors(jq, jk, st));
-    if (pipe_step_eligible(B, Hq, Hkv)) {
+    if (pipelined) {
         // SCORE + TOPK and GATHER-ATT in one persistent kernel: the scoring of later units runs under the row fetch of earlier ones
         int32_t *counters = ws_ptr<int32_t>(workspace, L.off_tickets);
         const size_t units = (size_t)B * Hkv;
@@ -383,6 +384,17 @@ int ha_sparse_decode(const ha_shape *shape, const ha_mapping *map_q, const ha_ma
     return sparse_decode_impl(shape, map_q, map_k, q, k_new, K, V, nullptr, 0, 0, k_codes, kc_stride_b, kc_stride_h, seq_lens,
                               k_per_seq, k_uniform, max_seq_len, k_max, q_codes, idx, idx_stride_b, idx_stride_h, count, out,
                               lse, workspace, ws_bytes, stream);
+}
+
+int ha_sparse_decode_pipelined(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k, const uint16_t *q,
+                               const uint16_t *k_new, const ha_tensor *K, const ha_tensor *V, uint32_t *k_codes,
+                               int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
+                               int32_t k_uniform, int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx,
+                               int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse,
+                               void *workspace, size_t ws_bytes, void *stream) {
+    return sparse_decode_impl(shape, map_q, map_k, q, k_new, K, V, nullptr, 0, 0, k_codes, kc_stride_b, kc_stride_h, seq_lens,
+                              k_per_seq, k_uniform, max_seq_len, k_max, q_codes, idx, idx_stride_b, idx_stride_h, count, out,
+                              lse, workspace, ws_bytes, stream, nullptr, /*pipelined=*/true);
 }
 
 int ha_sparse_decode_paged(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k, const uint16_t *q,

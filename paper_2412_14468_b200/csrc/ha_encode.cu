@@ -163,6 +163,197 @@ static cudaError_t launch_vec_t(const EncodeJob &a, const EncodeJob &b, cudaStre
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ decode-step kernel for large batches
+//
+// From a few hundred vectors per step on, one output per thread wastes the shared-memory port: every weight is a
+// 2-byte load that serves a single fma chain per vector.  Here a CTA of 64 NG threads encodes a TILE of NG x VPT
+// vectors of one network with register tiling: a thread owns two neighbouring outputs of VPT
+// vectors, so a 4-byte weight load feeds 2 VPT chains and a 16-byte activation load (a warp-wide broadcast) feeds
+// four terms of two chains.  Chains stay what Eq. 2's network is defined as here: one fused multiply-add per term,
+// ascending input index, started from the bias; only their distribution over threads changes, so the signatures
+// are bit-identical to encode_vec_kernel's.  Weights arrive by the same three bulk copies, requested before the
+// programmatic-launch wait.
+constexpr int kTileMinVectors = 40;   // vectors per network (both sides together) from which the tiled kernel takes the step
+constexpr int kTileActLd = kD + 4;   // padded activation row (floats)
+
+template <int VPT, int NG>
+__global__ void __launch_bounds__(64 * NG) encode_tile_kernel(EncodeJob ja, EncodeJob jb) {
+    constexpr int TV = NG * VPT;   // vectors per tile: NG vector groups (64 threads each) x VPT
+    constexpr int kTileThreads = 64 * NG;
+    extern __shared__ __align__(128) unsigned char tile_smem[];
+    __shared__ __align__(8) unsigned long long s_bar[3];
+    uint16_t *sw1 = reinterpret_cast<uint16_t *>(tile_smem);
+    uint16_t *sw2 = sw1 + kD * kHid;
+    uint16_t *sw3 = sw2 + kHid * kHid;
+    float *actA = reinterpret_cast<float *>(sw3 + kHid * kBits);   // [TV][kTileActLd]
+    float *actB = actA + TV * kTileActLd;
+
+    int i = blockIdx.x;
+    const bool second = i >= ja.n_cta;
+    const EncodeJob &J = second ? jb : ja;
+    if (second) i -= ja.n_cta;
+    const int tiles_per_net = J.cta_per_net, net = i / tiles_per_net, tile = i % tiles_per_net;
+    const int hpk = J.heads_per_kv;
+    const int n_vec = J.batch * hpk;   // vectors of this network: t -> (b = t / hpk, head net*hpk + t % hpk)
+    const int t0 = tile * TV, nv = min(TV, n_vec - t0);
+    const int tid = threadIdx.x;
+
+    const uint16_t *g1 = J.map.w1 + (size_t)net * kD * kHid;
+    const uint16_t *g2 = J.map.w2 + (size_t)net * kHid * kHid;
+    const uint16_t *g3 = J.map.w3 + (size_t)net * kHid * kBits;
+    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(&s_bar[0]);
+    if (tid == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        mbar_init(bar0 + 16, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(bar0, kD * kHid * 2);
+        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw1), g1, kD * kHid * 2, bar0);
+        mbar_expect_tx(bar0 + 8, kHid * kHid * 2);
+        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw2), g2, kHid * kHid * 2, bar0 + 8);
+        mbar_expect_tx(bar0 + 16, kHid * kBits * 2);
+        bulk_g2s((uint32_t)__cvta_generic_to_shared(sw3), g3, kHid * kBits * 2, bar0 + 16);
+    }
+    // hidden layers: thread = (output pair op, vector group vg); last layer: thread = (output pair op3, vector v3)
+    const int op = tid & 63, vg = tid >> 6;
+    float b1[2], b2[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        b1[e] = J.map.b1 ? __ldg(J.map.b1 + net * kHid + 2 * op + e) : 0.0f;
+        b2[e] = J.map.b2 ? __ldg(J.map.b2 + net * kHid + 2 * op + e) : 0.0f;
+    }
+    pdl_wait();                 // the vectors may come from the kernel in front; the weights do not
+    pdl_launch_dependents();
+
+    // the tile's vectors -> fp32 rows (slots past the batch are zero rows; their signatures are dropped)
+    for (int e = tid; e < TV * (kD / 8); e += kTileThreads) {
+        const int v = e / (kD / 8), c = e % (kD / 8);
+        uint4 raw = make_uint4(0, 0, 0, 0);
+        if (v < nv) {
+            const int t = t0 + v;
+            const uint16_t *x = J.x + (long long)(t / hpk) * J.x_sb + (long long)(net * hpk + t % hpk) * J.x_sh;
+            raw = __ldg(reinterpret_cast<const uint4 *>(x) + c);
+        }
+        const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+        float *dst = actA + v * kTileActLd + c * 8;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            dst[2 * q] = __uint_as_float(r[q] << 16);
+            dst[2 * q + 1] = __uint_as_float(r[q] & 0xffff0000u);
+        }
+    }
+    __syncthreads();   // inputs and mbarrier inits visible
+
+    auto weights_ready = [&](int which, uint16_t *dst, const uint16_t *src, int n_elems) {
+        const bool ok = mbar_wait_bounded(bar0 + 8 * which);
+        if (__syncthreads_or(!ok)) {   // never seen: fetch the matrix with ordinary loads instead
+            for (int c = tid; c < n_elems / 8; c += kTileThreads)
+                reinterpret_cast<uint4 *>(dst)[c] = __ldg(reinterpret_cast<const uint4 *>(src) + c);
+            __syncthreads();
+        }
+    };
+    // one hidden layer: out[v][2 op + e] = relu(bias[e] + sum_k in[v][k] w[k][2 op + e]) for the VPT vectors of group vg
+    auto hidden = [&](const float *in, float *out, const uint16_t *w, const float (&bias)[2]) {
+        float z[VPT][2];
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) { z[v][0] = bias[0]; z[v][1] = bias[1]; }
+        const float *hin = in + (size_t)vg * VPT * kTileActLd;
+#pragma unroll 4
+        for (int k = 0; k < 128; k += 4) {
+            float wf[4][2];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const uint32_t wv = *reinterpret_cast<const uint32_t *>(w + (k + t) * kHid + 2 * op);
+                wf[t][0] = __uint_as_float(wv << 16);
+                wf[t][1] = __uint_as_float(wv & 0xffff0000u);
+            }
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) {
+                const float4 hv = *reinterpret_cast<const float4 *>(hin + v * kTileActLd + k);   // warp broadcast
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {   // ascending term index within every chain
+                    z[v][e] = __fmaf_rn(hv.x, wf[0][e], z[v][e]);
+                    z[v][e] = __fmaf_rn(hv.y, wf[1][e], z[v][e]);
+                    z[v][e] = __fmaf_rn(hv.z, wf[2][e], z[v][e]);
+                    z[v][e] = __fmaf_rn(hv.w, wf[3][e], z[v][e]);
+                }
+            }
+        }
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            float2 r;
+            r.x = (z[v][0] > 0.0f) ? z[v][0] : 0.0f;
+            r.y = (z[v][1] > 0.0f) ? z[v][1] : 0.0f;
+            *reinterpret_cast<float2 *>(out + (size_t)(vg * VPT + v) * kTileActLd + 2 * op) = r;
+        }
+    };
+    weights_ready(0, sw1, g1, kD * kHid);
+    hidden(actA, actB, sw1, b1);
+    __syncthreads();
+    weights_ready(1, sw2, g2, kHid * kHid);
+    hidden(actB, actA, sw2, b2);
+    __syncthreads();
+    weights_ready(2, sw3, g3, kHid * kBits);
+    // last layer, 32 outputs: thread (op3 = output pair, v3 = vector); a half-warp holds the 16 pairs of one vector
+    {
+        const int lane = tid & 31, op3 = tid & 15, v3 = tid >> 4;
+        if (v3 < TV) {   // warp-uniform (TV is 4, 8 or 16; the CTA has at least 16 TV threads)
+            float z0 = J.map.b3 ? __ldg(J.map.b3 + net * kBits + 2 * op3) : 0.0f;
+            float z1 = J.map.b3 ? __ldg(J.map.b3 + net * kBits + 2 * op3 + 1) : 0.0f;
+            const float *hin = actA + (size_t)v3 * kTileActLd;
+#pragma unroll 4
+            for (int k = 0; k < 128; k += 4) {
+                const float4 hv = *reinterpret_cast<const float4 *>(hin + k);
+                float wf[4][2];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const uint32_t wv = *reinterpret_cast<const uint32_t *>(sw3 + (k + t) * kBits + 2 * op3);
+                    wf[t][0] = __uint_as_float(wv << 16);
+                    wf[t][1] = __uint_as_float(wv & 0xffff0000u);
+                }
+                z0 = __fmaf_rn(hv.x, wf[0][0], z0); z1 = __fmaf_rn(hv.x, wf[0][1], z1);
+                z0 = __fmaf_rn(hv.y, wf[1][0], z0); z1 = __fmaf_rn(hv.y, wf[1][1], z1);
+                z0 = __fmaf_rn(hv.z, wf[2][0], z0); z1 = __fmaf_rn(hv.z, wf[2][1], z1);
+                z0 = __fmaf_rn(hv.w, wf[3][0], z0); z1 = __fmaf_rn(hv.w, wf[3][1], z1);
+            }
+            const uint32_t even = __ballot_sync(0xffffffffu, z0 > 0.0f), odd = __ballot_sync(0xffffffffu, z1 > 0.0f);
+            auto spread16 = [](uint32_t v) {   // bit i -> bit 2 i
+                v = (v | (v << 8)) & 0x00ff00ffu;
+                v = (v | (v << 4)) & 0x0f0f0f0fu;
+                v = (v | (v << 2)) & 0x33333333u;
+                v = (v | (v << 1)) & 0x55555555u;
+                return v;
+            };
+            const int shift = lane & 16;   // this half-warp's 16 bits of either ballot
+            const uint32_t code = spread16((even >> shift) & 0xffffu) | (spread16((odd >> shift) & 0xffffu) << 1);
+            if (op3 == 0 && v3 < nv) {
+                const int t = t0 + v3, b = t / hpk;
+                int slot = 0;
+                if (J.slot) slot = J.slot[b] - J.slot_minus_one;   // a negative slot skips the sequence
+                if (slot >= 0) J.codes[(long long)b * J.c_sb + (long long)(net * hpk + t % hpk) * J.c_sh + slot] = code;
+            }
+        }
+    }
+}
+
+template <int VPT, int NG>
+static cudaError_t launch_tile_t(const EncodeJob &a, const EncodeJob &b, cudaStream_t st) {
+    static_assert(64 * NG >= 16 * NG * VPT, "the last layer needs 16 threads per vector");
+    constexpr size_t smem = kVecWeightBytes + (size_t)2 * NG * VPT * kTileActLd * 4;
+    static bool done[64] = {};   // opt in to > 48 KB of shared memory once per device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(encode_tile_kernel<VPT, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        done[dev] = true;
+    }
+    cudaError_t e = launch_pdl(encode_tile_kernel<VPT, NG>, dim3(a.n_cta + b.n_cta), dim3(64 * NG), smem, st, a, b);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    return cudaGetLastError();
+}
+
 // `a` and `b` arrive with n_cta = the number of (sequence, network) pairs (0 = no such job); the item
 // width and the CTAs per network are chosen here: the smallest number m of vectors per CTA for which
 // all CTAs are resident at once (two CTAs of 76 KB fit one SM; a second wave would double the latency),
@@ -179,6 +370,24 @@ cudaError_t launch_encode_vectors(const EncodeJob &a_in, const EncodeJob &b_in, 
         vec_per_net[j] = J.batch * J.heads_per_kv;
     }
     const long long room = 2LL * sm_count();
+    if (vec_per_net[0] + vec_per_net[1] >= kTileMinVectors) {
+        // large batch: tiles of 4, 8 or 16 vectors per CTA, the smallest for which all CTAs are resident at once
+        int tv = 4;
+        auto tiles = [&](int t) {
+            long long n = 0;
+            for (int j = 0; j < 2; ++j) n += (long long)nets[j] * ((vec_per_net[j] + t - 1) / t);
+            return n;
+        };
+        while (tv < 16 && tiles(tv) > room) tv *= 2;
+        for (int j = 0; j < 2; ++j) {
+            EncodeJob &J = job[j];
+            J.cta_per_net = (vec_per_net[j] + tv - 1) / tv;   // tiles per network
+            J.n_cta = nets[j] * J.cta_per_net;
+        }
+        if (tv == 4) return launch_tile_t<1, 4>(job[0], job[1], st);
+        if (tv == 8) return launch_tile_t<2, 4>(job[0], job[1], st);
+        return launch_tile_t<4, 4>(job[0], job[1], st);
+    }
     auto ctas = [&](int m) {
         long long n = 0;
         for (int j = 0; j < 2; ++j) n += (long long)nets[j] * ((vec_per_net[j] + m - 1) / m);

@@ -3,11 +3,12 @@
 //
 // Why: at scale the two halves of the step are bound by different units of the SM.  SCORE (Eq. 1 as bitcount(xor),
 // Section 4.1) spends its time in the population-count pipe and the integer pipe; GATHER-ATT (Section 4) waits for
-// HBM.  Run one after the other, each leaves the other's resource idle.  Here every SM holds one CTA of twelve
-// warps with two roles:
-//   * four SCORE warps walk the units of the CTA's range: scores as one byte per token, a histogram per warp, the
-//     threshold of the standard top-k (Section 4), the index list in ascending token order (ties to the lowest
-//     index), then a release counter per unit;
+// HBM.  Run one after the other, each leaves the other's resource idle.  Here every SM holds one CTA of 24 warps
+// with two roles (the register file is re-divided between them with setmaxnreg: 48 registers per SCORE thread, 144
+// per GATHER thread):
+//   * sixteen SCORE warps walk the units of the CTA's range: scores as one byte per token, a histogram per group of
+//     four warps, the threshold of the standard top-k (Section 4), the index list in ascending token order (ties to
+//     the lowest index), then a release counter per unit;
 //   * eight GATHER warps follow them over the same range: each warp keeps a two-stage ring of 16-row blocks in flight
 //     (16-byte cp.async, a half-warp per 256-byte row), waits for a unit's counter before it touches the unit's list,
 //     and keeps requesting rows of the next unit while the states of the previous one are merged, so that the row
@@ -29,7 +30,9 @@
 namespace ha {
 
 constexpr int kPipeGatherWarps = 8;
-constexpr int kPipeScoreWarps = 4;
+constexpr int kPipeScoreWarps = 20;
+constexpr int kPipeScoreGroups = 5;                   // counter tables: one per four SCORE warps
+constexpr int kPipeGatherRegs = 152, kPipeScoreRegs = 40;   // per thread once the roles part (setmaxnreg); 8 x 32 x 144 + 16 x 32 x 48 = 768 x 80, what the CTA is launched with
 constexpr int kPipeGatherThreads = kPipeGatherWarps * 32;
 constexpr int kPipeScoreThreads = kPipeScoreWarps * 32;
 constexpr int kPipeThreads = kPipeGatherThreads + kPipeScoreThreads;
@@ -37,7 +40,7 @@ constexpr int kPipeStages = 2;                         // row blocks in flight p
 constexpr int kPipeWarpRing = kPipeStages * kStageBytes;
 constexpr int kPipeRingBytes = kPipeGatherWarps * kPipeWarpRing;
 constexpr int kPipeLocalTokens = 32768;                // score bytes of one chunk that fit in shared memory
-constexpr int kPipeHistBytes = kPipeScoreWarps * kBins * 32 * 4;
+constexpr int kPipeHistBytes = kPipeScoreGroups * kBins * 32 * 4;
 constexpr int kPipePrefBytes = (kMaxBalancedUnits + 4) * 4;
 constexpr int kPipeCntStride = 36;
 constexpr int kPipeSpinLimit = 1 << 22;                // polls of ~0.25 us each before a wait gives up
@@ -146,21 +149,27 @@ __device__ __forceinline__ int pipe_chunk_tokens(int n, int chunks) { return ((n
 struct ScoreJob {
     int u;
     int t0, t1;          // tokens of the unit that this CTA scores
-    int chunk, chunks;   // its chunk index and the number of chunks of the unit (1: the CTA owns the unit)
+    int chunk, chunks;   // its chunk index and the number of chunks of the unit
+    bool shared;         // the unit is shared with other CTAs: histograms meet in the workspace
     bool local;          // score bytes in shared memory (else in the workspace)
 };
 
+// Scoring needs many warps: a warp issues about one instruction in twelve cycles here (dependent population counts,
+// shared-memory reductions, loads), so the sixteen SCORE warps of a CTA together keep the population-count pipe busy
+// where four did not.  They get by with few registers (two rows of signatures in flight per warp), which leaves the
+// register file to the GATHER warps.
 template <int G>
 struct ScoreRole {
     const PipeArgs &a;
     unsigned char *s_local;      // kPipeLocalTokens score bytes
-    uint32_t *s_hist;            // [4][33][32] counters
-    int *s_cnt;                  // [4][kPipeCntStride] level counts of each warp's slice
-    int sw, lane;                // score warp 0..3
+    uint32_t *s_hist;            // [kPipeScoreGroups][33][32] counters: one table per group of four warps
+    int *s_cnt;                  // [kPipeScoreGroups][kPipeCntStride] level counts per table
+    int *s_wcnt;                 // [kPipeScoreWarps][2] numbers of tokens with S > T / S == T in each warp's slice
+    int sw, lane;                // score warp 0..15
     bool gave_up = false;
 
-    __device__ ScoreRole(const PipeArgs &a_, unsigned char *loc, uint32_t *hist, int *cnt, int sw_, int lane_)
-        : a(a_), s_local(loc), s_hist(hist), s_cnt(cnt), sw(sw_), lane(lane_) {}
+    __device__ ScoreRole(const PipeArgs &a_, unsigned char *loc, uint32_t *hist, int *cnt, int *wcnt, int sw_, int lane_)
+        : a(a_), s_local(loc), s_hist(hist), s_cnt(cnt), s_wcnt(wcnt), sw(sw_), lane(lane_) {}
 
     __device__ __forceinline__ unsigned char *bytes_of(const ScoreJob &j) const {
         // byte of token t at base[t - j.t0]
@@ -174,11 +183,13 @@ struct ScoreRole {
         w1 = min(j.t1, w0 + per);
     }
 
-    // Pass 1: score bytes (score + 1; 0 = no token; kForcedByte = always kept) and the warp's level counts.
+    // Pass 1: score bytes (score + 1; 0 = no token; kForcedByte = always kept) and the level counts of the job.
+    // Ends with the job's counts in s_cnt (valid after the role barrier inside).
     __device__ void pass1(const ScoreJob &j, const PipeUnit &pu) {
-        uint32_t *hist = s_hist + sw * kBins * 32;
-        for (int i = lane; i < kBins * 32; i += 32) hist[i] = 0u;
-        __syncwarp();
+        const int grp = sw >> 2, st = sw * 32 + lane;
+        for (int i = st; i < kPipeScoreGroups * kBins * 32; i += kPipeScoreThreads) s_hist[i] = 0u;
+        bar_sync(2, kPipeScoreThreads);
+        uint32_t *hist = s_hist + grp * kBins * 32;
         int w0, w1;
         warp_range(j, w0, w1);
         const int n = pu.n;
@@ -213,112 +224,75 @@ struct ScoreRole {
             return s4;
         };
         const int n_rows = (w1 - w0 + 255) / 256;
-        constexpr int kRows = 4;   // rows per batch; the next batch is requested before the current one is scored
-        auto load_rows = [&](uint4 (&c)[2 * kRows], int r0) {
-#pragma unroll
-            for (int r = 0; r < kRows; ++r) {
-                const int t = w0 + (r0 + r) * 256 + lane * 8;
-                if (r0 + r < n_rows && t + 8 <= n) {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(row + t);
-                    c[2 * r] = __ldcg(src);
-                    c[2 * r + 1] = __ldcg(src + 1);
-                } else {
-                    c[2 * r] = (r0 + r < n_rows && t < n) ? load_codes4(row, t, n) : make_uint4(0, 0, 0, 0);
-                    c[2 * r + 1] = (r0 + r < n_rows && t + 4 < n) ? load_codes4(row, t + 4, n) : make_uint4(0, 0, 0, 0);
-                }
+        auto load_row = [&](int r, uint4 &lo, uint4 &hi) {
+            const int t = w0 + r * 256 + lane * 8;
+            if (r < n_rows && t + 8 <= n) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(row + t);
+                lo = __ldcg(src);
+                hi = __ldcg(src + 1);
+            } else {
+                lo = (r < n_rows && t < n) ? load_codes4(row, t, n) : make_uint4(0, 0, 0, 0);
+                hi = (r < n_rows && t + 4 < n) ? load_codes4(row, t + 4, n) : make_uint4(0, 0, 0, 0);
             }
         };
-        uint4 cur[2 * kRows], nxt[2 * kRows];
-        load_rows(cur, 0);
-        for (int r0 = 0; r0 < n_rows; r0 += kRows) {
-            if (r0 + kRows < n_rows) load_rows(nxt, r0 + kRows);
-#pragma unroll
-            for (int r = 0; r < kRows; ++r) {
-                const int t = w0 + (r0 + r) * 256 + lane * 8;
-                if (r0 + r < n_rows) {
-                    const bool whole = t + 8 <= w1 && t >= pu.wbd.sink_end && t + 8 <= pu.wbd.local_begin;
-                    uint2 w;
-                    w.x = score_word(cur[2 * r], t, whole);
-                    w.y = score_word(cur[2 * r + 1], t + 4, whole);
-                    *reinterpret_cast<uint2 *>(sc + (t - j.t0)) = w;
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < 2 * kRows; ++r) cur[r] = nxt[r];
+        uint4 c0, c1, n0, n1;   // the row being scored and the one behind it, requested a row ahead
+        load_row(0, c0, c1);
+        for (int r = 0; r < n_rows; ++r) {
+            load_row(r + 1, n0, n1);
+            const int t = w0 + r * 256 + lane * 8;
+            const bool whole = t + 8 <= w1 && t >= pu.wbd.sink_end && t + 8 <= pu.wbd.local_begin;
+            uint2 w;
+            w.x = score_word(c0, t, whole);
+            w.y = score_word(c1, t + 4, whole);
+            *reinterpret_cast<uint2 *>(sc + (t - j.t0)) = w;
+            c0 = n0; c1 = n1;
         }
-        __syncwarp();
-        // level counts of this warp's slice: lane l adds the 32 counters of level l (rotated start: no bank conflict)
-        int c = 0;
-#pragma unroll 8
-        for (int jj = 0; jj < 32; ++jj) c += (int)hist[lane * 32 + ((jj + lane) & 31)];
-        int c32 = (int)hist[32 * 32 + lane];
-#pragma unroll
-        for (int dd = 16; dd > 0; dd >>= 1) c32 += __shfl_xor_sync(0xffffffffu, c32, dd);
-        s_cnt[sw * kPipeCntStride + lane] = c;
-        if (lane == 0) s_cnt[sw * kPipeCntStride + 32] = c32;
-    }
-
-    // level counts of the whole job (lane l: level l; level 32 in every lane); call after a role barrier
-    __device__ __forceinline__ void job_counts(int &tot, int &tot32) const {
-        tot = 0; tot32 = 0;
-#pragma unroll
-        for (int w = 0; w < kPipeScoreWarps; ++w) { tot += s_cnt[w * kPipeCntStride + lane]; tot32 += s_cnt[w * kPipeCntStride + 32]; }
-    }
-
-    // Publishes the chunk's histogram (units shared by several CTAs).  All four warps call it after pass1.
-    __device__ void publish_chunk(const ScoreJob &j) {
         bar_sync(2, kPipeScoreThreads);
-        if (sw == 0) {
-            int tot, tot32;
-            job_counts(tot, tot32);
-            int32_t *h = a.ws_hist + ((long long)j.u * kMaxChunks + j.chunk) * kBins;
-            h[lane] = tot;
-            if (lane == 0) h[32] = tot32;
-            __threadfence();
-        }
-        __syncwarp();
-        // the score bytes of this chunk wait in the workspace: make them visible before the counter moves
-        __threadfence();
-        bar_sync(2, kPipeScoreThreads);
-        if (sw == 0 && lane == 0) atomicAdd(a.s1_done + j.u, 1);
-    }
-
-    // Pass 2: threshold, this warp's part of the index list, the unit's count and padding, release.
-    // own_counts: s_cnt still holds this job's level counts (pass1 directly in front); else they are recounted
-    // from the score bytes.
-    __device__ void pass2(const ScoreJob &j, const PipeUnit &pu, bool own_counts) {
-        int w0, w1;
-        warp_range(j, w0, w1);
-        const unsigned char *sc = bytes_of(j);
-        if (!own_counts) {
-            // the warp's level counts again, from its score bytes (a shared unit's chunk, scored a while ago)
-            uint32_t *hist = s_hist + sw * kBins * 32;
-            for (int i = lane; i < kBins * 32; i += 32) hist[i] = 0u;
-            __syncwarp();
-            const uint32_t base = (uint32_t)__cvta_generic_to_shared(hist + lane);
-            for (int t = w0 + lane * 16; t < w1; t += 512) {
-                const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(sc + (t - j.t0)));
-                const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const uint32_t byte = (wv[e >> 2] >> (8 * (e & 3))) & 0xffu;
-                    if (byte >= 1u && byte <= 33u) asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(base + (byte - 1u) * 128u) : "memory");
-                }
-            }
-            __syncwarp();
+        // level counts per table: warp g folds table g (lane l adds the 32 counters of level l, rotated start: no bank conflict)
+        if (sw < kPipeScoreGroups) {
+            const uint32_t *hg = s_hist + sw * kBins * 32;
             int c = 0;
 #pragma unroll 8
-            for (int jj = 0; jj < 32; ++jj) c += (int)hist[lane * 32 + ((jj + lane) & 31)];
-            int c32 = (int)hist[32 * 32 + lane];
+            for (int jj = 0; jj < 32; ++jj) c += (int)hg[lane * 32 + ((jj + lane) & 31)];
+            int c32 = (int)hg[32 * 32 + lane];
 #pragma unroll
             for (int dd = 16; dd > 0; dd >>= 1) c32 += __shfl_xor_sync(0xffffffffu, c32, dd);
             s_cnt[sw * kPipeCntStride + lane] = c;
             if (lane == 0) s_cnt[sw * kPipeCntStride + 32] = c32;
         }
         bar_sync(2, kPipeScoreThreads);
-        int tot, tot32, bef = 0, bef32 = 0;
-        if (j.chunks == 1) {
+    }
+
+    // level counts of the whole job (lane l: level l; level 32 in every lane)
+    __device__ __forceinline__ void job_counts(int &tot, int &tot32) const {
+        tot = 0; tot32 = 0;
+#pragma unroll
+        for (int w = 0; w < kPipeScoreGroups; ++w) { tot += s_cnt[w * kPipeCntStride + lane]; tot32 += s_cnt[w * kPipeCntStride + 32]; }
+    }
+
+    // Publishes the chunk's histogram (units shared by several CTAs).  All warps call it directly after pass1.
+    __device__ void publish_chunk(const ScoreJob &j) {
+        if (sw == 0) {
+            int tot, tot32;
             job_counts(tot, tot32);
+            int32_t *h = a.ws_hist + ((long long)j.u * kMaxChunks + j.chunk) * kBins;
+            h[lane] = tot;
+            if (lane == 0) h[32] = tot32;
+        }
+        // the score bytes of this chunk wait in the workspace: they and the histogram are visible before the counter moves
+        __threadfence();
+        bar_sync(2, kPipeScoreThreads);
+        if (sw == 0 && lane == 0) atomicAdd(a.s1_done + j.u, 1);
+    }
+
+    // Pass 2: threshold, this warp's part of the index list, the unit's count and padding, release.
+    __device__ void pass2(const ScoreJob &j, const PipeUnit &pu) {
+        int w0, w1;
+        warp_range(j, w0, w1);
+        const unsigned char *sc = bytes_of(j);
+        int tot, tot32, bef = 0, bef32 = 0;
+        if (!j.shared) {
+            job_counts(tot, tot32);   // pass1 directly in front
         } else {
             pipe_wait(a.s1_done + j.u, j.chunks, a.status, gave_up, 1, j.u);
             tot = 0; tot32 = 0;
@@ -331,35 +305,54 @@ struct ScoreRole {
         }
         int T, r, gt_before, eq_before;
         find_threshold(tot, bef, tot32, bef32, pu.keep_rest, lane, T, r, gt_before, eq_before);
-        // tokens of this job that lie before this warp's slice: S > T / S == T from the warps' level counts
-        int run_gt = gt_before + forced_before(pu.wbd, w0), run_eq = eq_before;
-        for (int w = 0; w < sw; ++w) {
-            const int cl = s_cnt[w * kPipeCntStride + lane], c32 = s_cnt[w * kPipeCntStride + 32];
-            int g = (lane > T) ? cl : 0;
+        // Per byte b = score + 1 (0 = no token): b + 127 - (T+1) sets bit 7 iff score > T, b + 128 - (T+1) iff
+        // score >= T (no byte sum reaches 256); always-kept tokens (kForcedByte) count as S > T for every T.
+        const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
+        const uint32_t c_gt = 0x7f7f7f7fu - T4, c_ge = 0x80808080u - T4;
+        const int written_end = w0 + (w1 - w0 + 255) / 256 * 256;   // pass 1 wrote whole rows (zero bytes past the slice)
+        auto flags32 = [&](int first, uint32_t &gt, uint32_t &eq) {      // flags of tokens first .. first + 31
+            gt = 0u;
+            uint32_t ge = 0u;
+            if (first < written_end) {
+                const uint4 *p = reinterpret_cast<const uint4 *>(sc + (first - j.t0));
+                const uint4 v0 = j.local ? p[0] : __ldcg(p), v1 = j.local ? p[1] : __ldcg(p + 1);
+                const uint32_t wv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
 #pragma unroll
-            for (int dd = 16; dd > 0; dd >>= 1) g += __shfl_xor_sync(0xffffffffu, g, dd);
-            if (T < 32) { run_gt += g + c32; run_eq += __shfl_sync(0xffffffffu, cl, T & 31); }
-            else if (T == 32) run_eq += c32;
+                for (int e = 0; e < 8; ++e) {
+                    gt |= high_bits_to_nibble(wv[e] + c_gt) << (4 * e);
+                    ge |= high_bits_to_nibble(wv[e] + c_ge) << (4 * e);
+                }
+            }
+            eq = ge ^ gt;
+        };
+        // sweep A: how many tokens of this warp's slice lie above / at the threshold
+        int mine_gt = 0, mine_eq = 0;
+        if (pu.keep > 0) {
+            for (int tile = w0; tile < w1; tile += 1024) {
+                uint32_t gt, eq;
+                flags32(tile + lane * 32, gt, eq);
+                mine_gt += __popc(gt);
+                mine_eq += __popc(eq);
+            }
+#pragma unroll
+            for (int dd = 16; dd > 0; dd >>= 1) {
+                mine_gt += __shfl_xor_sync(0xffffffffu, mine_gt, dd);
+                mine_eq += __shfl_xor_sync(0xffffffffu, mine_eq, dd);
+            }
         }
+        if (lane == 0) { s_wcnt[2 * sw] = mine_gt; s_wcnt[2 * sw + 1] = mine_eq; }
+        bar_sync(2, kPipeScoreThreads);
         int32_t *list = a.idx + (long long)pu.b * a.idx_sb + (long long)pu.kvh * a.idx_sh;
         if (pu.keep > 0 && w0 < w1) {
-            const uint32_t T4 = (uint32_t)(T + 1) * 0x01010101u;
-            const uint32_t c_gt = 0x7f7f7f7fu - T4, c_ge = 0x80808080u - T4;
-            const int written_end = w0 + (w1 - w0 + 255) / 256 * 256;   // pass 1 wrote whole rows (zero bytes past the slice)
+            // tokens before this warp's slice: scored ones of earlier chunks (histograms), always-kept ones before the
+            // job (closed form), and everything flagged in the slices of the warps in front
+            int run_gt = gt_before + forced_before(pu.wbd, j.t0), run_eq = eq_before;
+            for (int w = 0; w < sw; ++w) { run_gt += s_wcnt[2 * w]; run_eq += s_wcnt[2 * w + 1]; }
+            // sweep B: the selected tokens at their final positions
             for (int tile = w0; tile < w1; tile += 1024) {              // warp-uniform
                 const int first = tile + lane * 32;
-                uint32_t gt = 0u, ge = 0u;
-                if (first < written_end) {
-                    const uint4 *p = reinterpret_cast<const uint4 *>(sc + (first - j.t0));
-                    const uint4 v0 = j.local ? p[0] : __ldcg(p), v1 = j.local ? p[1] : __ldcg(p + 1);
-                    const uint32_t wv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        gt |= high_bits_to_nibble(wv[e] + c_gt) << (4 * e);
-                        ge |= high_bits_to_nibble(wv[e] + c_ge) << (4 * e);
-                    }
-                }
-                const uint32_t eq = ge ^ gt;
+                uint32_t gt, eq;
+                flags32(first, gt, eq);
                 const int packed = __popc(gt) | (__popc(eq) << 16);
                 int inc = packed;
 #pragma unroll
@@ -398,7 +391,8 @@ __global__ void __launch_bounds__(kPipeThreads, 1) pipe_step_kernel(const PipeAr
     unsigned char *s_local = psm + kPipeRingBytes + pipe_scratch_bytes(G);
     uint32_t *s_hist = reinterpret_cast<uint32_t *>(s_local + kPipeLocalTokens);
     int *s_pref = reinterpret_cast<int *>(reinterpret_cast<unsigned char *>(s_hist) + kPipeHistBytes);   // [n_units + 1]
-    __shared__ int s_cnt[kPipeScoreWarps * kPipeCntStride];
+    __shared__ int s_cnt[kPipeScoreGroups * kPipeCntStride];
+    __shared__ int s_wcnt[2 * kPipeScoreWarps];
     __shared__ float s_m[kPipeGatherWarps][8], s_l[kPipeGatherWarps][8];
     __shared__ uint32_t s_mask[kPipeGatherWarps][kPipeStages];
     __shared__ int s_last;
@@ -445,7 +439,8 @@ __global__ void __launch_bounds__(kPipeThreads, 1) pipe_step_kernel(const PipeAr
     if (warp >= kPipeGatherWarps) {
         // ================================================================ SCORE warps
         const int sw = warp - kPipeGatherWarps;
-        ScoreRole<G> S(a, s_local, s_hist, s_cnt, sw, lane);
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPipeScoreRegs));
+        ScoreRole<G> S(a, s_local, s_hist, s_cnt, s_wcnt, sw, lane);
         // units without a single selected token take no part in the split: count, padding, zero output
         for (int v = cta; v < a.n_units; v += P) {
             if (s_pref[v + 1] != s_pref[v]) continue;
@@ -465,10 +460,11 @@ __global__ void __launch_bounds__(kPipeThreads, 1) pipe_step_kernel(const PipeAr
             const PipeSplit sp = pipe_split(s_pref[u], s_pref[u + 1], T, Pe);
             j.u = u;
             if (sp.n_parts == 1) {
-                j.chunk = 0; j.chunks = 1; j.t0 = 0; j.t1 = pu.n;
+                j.chunk = 0; j.chunks = 1; j.t0 = 0; j.t1 = pu.n; j.shared = false;
                 j.local = pu.n <= kPipeLocalTokens;
                 return true;
             }
+            j.shared = true;
             j.chunks = pipe_chunks(pu.n, sp.n_parts);
             j.chunk = cta - sp.c_first;
             if (j.chunk >= j.chunks) return false;
@@ -497,8 +493,10 @@ __global__ void __launch_bounds__(kPipeThreads, 1) pipe_step_kernel(const PipeAr
             have_l = job_of(u_last, jl, pl, false);
             if (have_l) { S.pass1(jl, pl); S.publish_chunk(jl); }
         }
-        // 2. second pass of the first unit (the GATHER warps need its list first)
-        if (have_f) S.pass2(jf, pf, /*own_counts=*/!have_l);
+        // 2. their second passes: the GATHER warps here need the first unit's list first, and a neighbour's need the last
+        // unit's (it is the first of its range)
+        if (have_f) S.pass2(jf, pf);
+        if (have_l) S.pass2(jl, pl);
         // 3. the units inside the range, in order
         for (int u = u_first + (first_shared ? 1 : 0); u <= u_last - (last_shared ? 1 : 0); ++u) {
             if (s_pref[u + 1] == s_pref[u]) continue;
@@ -506,14 +504,13 @@ __global__ void __launch_bounds__(kPipeThreads, 1) pipe_step_kernel(const PipeAr
             PipeUnit pu;
             job_of(u, j, pu, false);
             S.pass1(j, pu);
-            S.pass2(j, pu, true);
+            S.pass2(j, pu);
         }
-        // 4. second pass of the last unit
-        if (have_l) S.pass2(jl, pl, false);
         return;
     }
 
     // ==================================================================== GATHER warps
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kPipeGatherRegs));
     if (x_lo >= x_hi) return;
     const int g = lane >> 2, c = lane & 3;
     unsigned char *my_ring = ring + warp * kPipeWarpRing;

@@ -619,7 +619,7 @@ def test_gather_attn_over_a_paged_cache(page_size):
 
 # ---------------------------------------------------------------------------- whole step
 
-def _run_step(w, host=False, pinned=True, n_sink=0, n_local=0, prepared=False):
+def _run_step(w, host=False, pinned=True, n_sink=0, n_local=0, prepared=False, pipelined=False):
     cfg = w["cfg"]
     B, Hq, Hkv = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads
     shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"], n_sink=n_sink, n_local=n_local)
@@ -659,8 +659,9 @@ def _run_step(w, host=False, pinned=True, n_sink=0, n_local=0, prepared=False):
         out = ho.to(DEV)
         lse = None
     else:
-        ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
-                            w["n_cap"], w["k_max"], qc, idx, cnt, out, ws, lse=lse)
+        step = ha.ha_sparse_decode_pipelined if pipelined else ha.ha_sparse_decode
+        step(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
+             w["n_cap"], w["k_max"], qc, idx, cnt, out, ws, lse=lse)
     torch.cuda.synchronize()
     assert ha.ha_read_device_status(ws) == 0
     return dict(kc=kc, qc=qc, idx=idx, cnt=cnt, out=out, lse=lse)
@@ -700,7 +701,7 @@ def test_sparse_decode_step_matches_oracle(cfg):
 
 
 @pytest.mark.parametrize("world", [2, 4])
-@pytest.mark.parametrize("B", [2, 20])          # one fused launch per shard / ENCODE + the pipelined kernel
+@pytest.mark.parametrize("B", [2, 20])          # one fused launch per shard / the three-kernel path
 def test_head_parallel_shards_reproduce_the_whole_step(B, world):
     """The (sequence, KV head) units are independent: the step run on each rank's KV heads alone (strided K/V views,
     sliced mappings) gives the slices of the unsharded result (signatures, lists and counts bit for bit, outputs to
@@ -894,7 +895,7 @@ def test_sparse_decode_step_over_a_paged_cache(cfg, page_size):
 
 @pytest.mark.parametrize("seed", range(14))
 def test_sparse_decode_step_random_configs(seed):
-    """Seeded sweep over batch (both the fused launch and ENCODE + the pipelined kernel), KV heads, group size, ragged
+    """Seeded sweep over batch (both the fused launch and the three-kernel path), KV heads, group size, ragged
     lengths, sparsity and window sizes; everything the step returns is checked against the oracle."""
     rng = np.random.default_rng(7000 + seed)
     B = int(rng.integers(1, 13)) if seed < 8 else int(rng.integers(13, 110))   # up to 24 units / up to 220 units
@@ -923,25 +924,25 @@ def test_sparse_decode_step_random_configs(seed):
     # 60 units: clusters of 4 (two query vectors per encoding CTA, 32 tokens per thread)
     (wl.Config("fused-60-units", 84, 30, [1500 + 97 * i for i in range(30)], None, 0.02, n_q_heads=8, n_kv_heads=2,
                sparsity=8), 1),
-    # 100 units: more clusters of four than the device holds at once: ENCODE, then the pipelined kernel
+    # 100 units: more clusters of four than the device holds at once
     (wl.Config("split-100-units", 85, 50, [2500 + 301 * i for i in range(50)], None, 0.02, n_q_heads=16, n_kv_heads=2,
-               sparsity=16), 2),
+               sparsity=16), 3),
     # 6 units, budgets above 2048 rows: one fused launch of the two-stage variant, several blocks per warp
     (wl.Config("fused-large-k", 81, 3, [9000, 5000, 12001], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=2), 1),
     # 20 units with budgets of 1500 rows: more clusters than the two-stage variant holds at once, so the
     # one-stage variant takes them, two blocks per warp one after the other
     (wl.Config("fused-20-units-1500", 86, 10, [6000 + 7 * i for i in range(10)], None, 0.02, n_q_heads=8, n_kv_heads=2,
                sparsity=4), 1),
-    # 20 units with budgets above 2048 rows: ENCODE, then the pipelined kernel
+    # 20 units with budgets above 2048 rows: three kernels
     (wl.Config("split-large-k", 82, 10, [6000 + 7 * i for i in range(10)], None, 0.02, n_q_heads=8, n_kv_heads=2,
-               sparsity=2), 2),
-    # 1200 units: beyond what the pipelined kernel's work split holds: ENCODE, SCORE + TOPK, GATHER-ATT as three kernels
+               sparsity=2), 3),
+    # 1200 units: more than the balanced work split of GATHER-ATT holds: one CTA per unit
     (wl.Config("three-kernels-1200-units", 87, 600, [150 + (37 * i) % 200 for i in range(600)], None, 0.02, n_q_heads=4,
                n_kv_heads=2, sparsity=8), 3),
 ])
 def test_sparse_decode_step_every_launch_variant(cfg, launches):
-    """The step picks the fused cluster kernel (one or two row stages per warp) or ENCODE followed by the pipelined
-    SCORE + TOPK + GATHER-ATT kernel from the number of units and the budget; each choice gives the oracle's result."""
+    """The step picks the fused cluster kernel (one or two row stages per warp) or the three-kernel path from
+    the number of units and the budget; each choice gives the oracle's result."""
     w = wl.make_workload(cfg, DEV)
     _run_step(w)                                   # first call: attributes, occupancy query
     before = ha.ha_kernel_launches()
@@ -983,15 +984,15 @@ def test_sparse_decode_step_every_launch_variant(cfg, launches):
     ("eight-head-groups", 40, 16, 2, [2000 + 77 * i for i in range(40)], 16, (3, 0)),
 ])
 def test_pipelined_step_ragged_lengths_shared_and_owned_units(name, B, Hq, Hkv, lens, sparsity, windows):
-    """Steps that take the persistent SCORE + TOPK + GATHER-ATT kernel (more units than the single-cluster kernel holds,
-    or sequences beyond its length): whole units per CTA, units shared by neighbouring CTAs, units scored chunk by chunk
-    through the workspace, empty selections; run twice on the same workspace (the release counters must be back at
-    zero) and compared with the oracle on everything the step returns."""
+    """ha_sparse_decode_pipelined (ENCODE, then the persistent SCORE + TOPK + GATHER-ATT kernel): whole units per CTA, units
+    shared by neighbouring CTAs, units scored chunk by chunk through the workspace, empty selections; compared with the
+    oracle on everything the step returns, then run three times on one workspace (the release counters must be back
+    at zero after every call)."""
     cfg = wl.Config(name, 90 + len(name), B, lens, None, 0.02, n_q_heads=Hq, n_kv_heads=Hkv, sparsity=sparsity)
     w = wl.make_workload(cfg, DEV)
     n_sink, n_local = windows
     before = ha.ha_kernel_launches()
-    r = _run_step(w, n_sink=n_sink, n_local=n_local)
+    r = _run_step(w, n_sink=n_sink, n_local=n_local, pipelined=True)
     assert ha.ha_kernel_launches() - before == 3            # prompt signatures, ENCODE of the step, the pipelined kernel
     Kc = oracle_key_codes(w["K"], w["map_k"], w["lens"])
     ref = oracle.decode_step(u16(w["q"]), u16(w["k_new"]), u16(w["K"]), u16(w["V"]), Kc.copy(),
@@ -1015,11 +1016,15 @@ def test_pipelined_step_ragged_lengths_shared_and_owned_units(name, B, Hq, Hkv, 
         cnt = torch.full((B, Hkv), 7, dtype=torch.int32, device=DEV)
         out = torch.full((B, Hq, 128), 3.0, dtype=torch.bfloat16, device=DEV)
         qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
-        ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], r["kc"], w["seq_lens"], w["k_per_seq"], 0,
-                            w["n_cap"], k_max, qc, idx, cnt, out, ws)
+        ha.ha_sparse_decode_pipelined(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], r["kc"], w["seq_lens"], w["k_per_seq"],
+                                      0, w["n_cap"], k_max, qc, idx, cnt, out, ws)
         torch.cuda.synchronize()
         assert ha.ha_read_device_status(ws) == 0
         assert torch.equal(idx, r["idx"]) and torch.equal(cnt, r["cnt"]) and torch.equal(out, r["out"])
+    # ... and ha_sparse_decode itself (fused or three kernels) returns the same lists
+    r2 = _run_step(w, n_sink=n_sink, n_local=n_local)
+    assert torch.equal(r2["idx"], r["idx"]) and torch.equal(r2["cnt"], r["cnt"]) and torch.equal(r2["qc"], r["qc"])
+    assert max_abs_diff_bf16(u16(r2["out"]), u16(r["out"])) <= OUT_AIM
 
 
 def test_k_equals_n_sparse_step_equals_dense_kernel():
@@ -1034,7 +1039,7 @@ def test_k_equals_n_sparse_step_equals_dense_kernel():
     assert r["cnt"].cpu().tolist() == [[1500, 1500], [900, 900]]
 
 
-@pytest.mark.parametrize("reps", [1, 5, 12, 40])     # 8 / 40 units: fused kernel, clusters of 8 / 4; 96 and 320 units: ENCODE + the pipelined kernel
+@pytest.mark.parametrize("reps", [1, 5, 12, 40])     # 8 / 40 units: fused kernel, clusters of 8 / 4; 96 and 320 units: three-kernel path
 def test_step_edge_cases_empty_sequence_budget_above_length_and_no_new_key(reps):
     # one launch covers: an empty sequence, a one-token sequence, k > n, k = 0; then the same without a new key
     cfg = wl.Config("edges", 53, 4 * reps, [0, 1, 37, 2500] * reps, 64, 0.0, n_q_heads=8, n_kv_heads=2)
@@ -1075,7 +1080,7 @@ def test_step_edge_cases_empty_sequence_budget_above_length_and_no_new_key(reps)
         assert not u16(out)[0::4].any() and not u16(out)[3::4].any()          # empty selections give zeros
 
 
-@pytest.mark.parametrize("B", [1, 6, 40, 90])   # fused clusters of 8 / of 4 / ENCODE + the pipelined kernel (80 and 180 units)
+@pytest.mark.parametrize("B", [1, 6, 40, 90])   # fused clusters of 8 / of 4 / three kernels (80 and 180 units)
 def test_append_by_a_separate_encode_call_and_consecutive_steps_on_one_cache(B):
     """Library kernels start while the library kernel in front of them is finishing, and request signatures before they
     wait for it.  Two sequences of calls in which that kernel writes a signature the next one needs: (1) the Section 4.1
