@@ -66,6 +66,32 @@ def encode(x, w1, w2, w3, b1=None, b2=None, b3=None, return_z3=False):
     return (codes, z3) if return_z3 else codes
 
 
+def encode_wide(x, w1, w2, w3, b1=None, b2=None, b3=None, return_z3=False):
+    """Eq. 2 at b = w3.shape[1] bits (a multiple of 64).  x: uint16 [n,128]; w3: uint16 [128,b]; codes uint64 [n, b/64]
+    with bit j of a signature = bit j % 64 of word j // 64."""
+    x = _u16(x).reshape(-1, D)
+    n = x.shape[0]
+    w1, w2, w3 = _u16(w1), _u16(w2), _u16(w3)
+    n_bits = w3.shape[1]
+    assert w1.shape == (D, HID) and w2.shape == (HID, HID) and w3.shape == (HID, n_bits) and n_bits % 64 == 0
+    bs = [None if b is None else np.ascontiguousarray(b, dtype=np.float32) for b in (b1, b2, b3)]
+    codes = np.zeros((n, n_bits // 64), dtype=np.uint64)
+    z3 = np.zeros((n, n_bits), dtype=np.float32) if return_z3 else None
+    lib().ora_encode_wide(_p(x), C.c_int64(n), C.c_int64(D), _p(w1), _p(w2), _p(w3), _p(bs[0]), _p(bs[1]), _p(bs[2]),
+                          C.c_int32(n_bits), _p(codes), _p(z3))
+    return (codes, z3) if return_z3 else codes
+
+
+def score_wide_group(qcodes, kcodes) -> np.ndarray:
+    """Group score at b bits: the maximum over the group's query signatures (qcodes uint64 [G, W]) of the pinned
+    single-query score_wide, as the 32-bit layer-step reduces a GQA group; kcodes uint64 [n, W]."""
+    qcodes = np.ascontiguousarray(qcodes, dtype=np.uint64)
+    best = score_wide(qcodes[0], kcodes)
+    for j in range(1, qcodes.shape[0]):
+        best = np.maximum(best, score_wide(qcodes[j], kcodes))
+    return best
+
+
 def score(qcodes, kcodes) -> np.ndarray:
     """Eq. 1 as 32 - Hamming, maximum over the query codes of one GQA group."""
     qcodes = np.ascontiguousarray(qcodes, dtype=np.uint32).reshape(-1)

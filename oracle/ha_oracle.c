@@ -24,6 +24,10 @@
  *                    64-bit integers (the setting of the SCORE-latency table, "Latency of
  *                    SCORE computation"): b - Hamming distance, one query signature against n
  *                    key signatures, counted bit by bit.
+ *   ora_encode_wide  Eq. 2 at b = 64 .. 512 bits (the signature widths of the bit-width study and of the
+ *                    SCORE-latency table): the same network with a last layer of 128 x b, the b sign bits packed
+ *                    into b/64 64-bit integers, bit j of the signature = bit j % 64 of word j / 64 (the order that
+ *                    ora_score_wide reads).  Same arithmetic as ora_encode, output by output.
  *   ora_inner_products  the comparator column of that table: the inner product of one query
  *                    with each of n keys of 128 16-bit floats (bf16 here), in float64.
  *   ora_topk         "the standard top-k on these scores" (Section 4): sort by
@@ -136,6 +140,45 @@ void ora_encode(const uint16_t *x, int64_t n_vec, int64_t x_stride,
             for (int o = 0; o < HA_BITS; ++o) z3_out[r * HA_BITS + o] = z[o];
     }
     free(W1); free(W2); free(W3);
+}
+
+/* Eq. 2 with a last layer of n_bits outputs (n_bits a multiple of 64): w3 bf16 [128][n_bits], b3 fp32 [n_bits] or
+ * NULL; codes out, uint64 [n_vec][n_bits / 64]; z3_out optional fp32 [n_vec][n_bits].  Layers 1 and 2 and the
+ * arithmetic of every output (fmaf chain, ascending input index, from the bias) are those of ora_encode. */
+void ora_encode_wide(const uint16_t *x, int64_t n_vec, int64_t x_stride,
+                     const uint16_t *w1, const uint16_t *w2, const uint16_t *w3,
+                     const float *b1, const float *b2, const float *b3, int32_t n_bits,
+                     uint64_t *codes, float *z3_out) {
+    const int n_words = n_bits / 64;
+    float *W1 = (float *)malloc(sizeof(float) * HA_D * HA_HID);
+    float *W2 = (float *)malloc(sizeof(float) * HA_HID * HA_HID);
+    float *W3 = (float *)malloc(sizeof(float) * HA_HID * (size_t)n_bits);
+    float *z3 = (float *)malloc(sizeof(float) * (size_t)n_bits);
+    for (int i = 0; i < HA_D * HA_HID; ++i) W1[i] = bf16_to_f32(w1[i]);
+    for (int i = 0; i < HA_HID * HA_HID; ++i) W2[i] = bf16_to_f32(w2[i]);
+    for (int i = 0; i < HA_HID * n_bits; ++i) W3[i] = bf16_to_f32(w3[i]);
+    for (int64_t r = 0; r < n_vec; ++r) {
+        float h0[HA_D], h1[HA_HID], h2[HA_HID], z[HA_HID];
+        const uint16_t *xr = x + r * x_stride;
+        for (int k = 0; k < HA_D; ++k) h0[k] = bf16_to_f32(xr[k]);
+        for (int o = 0; o < HA_HID; ++o) z[o] = b1 ? b1[o] : 0.0f;
+        for (int k = 0; k < HA_D; ++k)
+            for (int o = 0; o < HA_HID; ++o) z[o] = fmaf(h0[k], W1[k * HA_HID + o], z[o]);
+        for (int o = 0; o < HA_HID; ++o) h1[o] = (z[o] > 0.0f) ? z[o] : 0.0f;
+        for (int o = 0; o < HA_HID; ++o) z[o] = b2 ? b2[o] : 0.0f;
+        for (int k = 0; k < HA_HID; ++k)
+            for (int o = 0; o < HA_HID; ++o) z[o] = fmaf(h1[k], W2[k * HA_HID + o], z[o]);
+        for (int o = 0; o < HA_HID; ++o) h2[o] = (z[o] > 0.0f) ? z[o] : 0.0f;
+        for (int o = 0; o < n_bits; ++o) z3[o] = b3 ? b3[o] : 0.0f;
+        for (int k = 0; k < HA_HID; ++k)
+            for (int o = 0; o < n_bits; ++o) z3[o] = fmaf(h2[k], W3[(size_t)k * n_bits + o], z3[o]);
+        for (int w = 0; w < n_words; ++w) codes[r * n_words + w] = 0;
+        for (int o = 0; o < n_bits; ++o)
+            if (z3[o] > 0.0f) codes[r * n_words + o / 64] |= ((uint64_t)1 << (o % 64));
+        if (z3_out)
+            for (int o = 0; o < n_bits; ++o) z3_out[r * n_bits + o] = z3[o];
+    }
+    free(W1); free(W2); free(W3); free(z3);
 }
 
 /* ---------------------------------------------------------------- SCORE (Eq. 1) */
