@@ -37,7 +37,7 @@
  *     set a bit in the workspace status word, are skipped, and never trap.
  *   - Fixed by the method's configuration (Section 5.2; abstract): head_dim = 128, signature
  *     width b = 32 bits, mapping network 128x128 - 128x128 - 128x32.  Other values return
- *     HA_ERR_UNSUPPORTED.  n_q_heads must be a multiple of n_kv_heads with a group size
+ *     HA_ERR_UNSUPPORTED, except in the entry points named *_wide, which take b = 64 .. 512.  n_q_heads must be a multiple of n_kv_heads with a group size
  *     G = n_q_heads / n_kv_heads <= 8; query head j uses KV head j / G.
  */
 #ifndef HASHATTN_H
@@ -356,6 +356,34 @@ int ha_gather_attn_static(const ha_shape *shape, const uint16_t *q, const ha_ten
  * inner product, not a step of ha_sparse_decode (whose signatures have 32 bits). */
 int ha_score_wide(const uint64_t *q_code, const uint64_t *k_codes, int64_t n, int32_t n_bits,
                   uint16_t *scores, void *stream);
+
+/* ENCODE -> SCORE -> TOPK at signatures of b = 64, 128, 256 or 512 bits (the widths of the paper's study of the number
+ * of bits and of its SCORE-latency table, which keeps them as packed 64-bit integers).  The index lists and counts have
+ * the layout of ha_score_topk's and feed ha_gather_attn unchanged.
+ *
+ * ha_encode_wide — Eq. 2 with a last layer of 128 x b: map->n_bits = b, map->w3 bf16 [n_kv_heads][128][b], map->b3 fp32
+ *   [n_kv_heads][b] or NULL; layers 1 and 2, the arithmetic of every output (fp32 fused multiply-add chain, ascending
+ *   input index, from the bias) and the arguments as ha_encode, except
+ *   codes   out, 64-bit words [batch][n_heads][tokens][b / 64] (8-byte aligned; c_stride_b, c_stride_h in words); bit j
+ *           of a signature is bit j % 64 of word j / 64; with `slot` (n_tokens == 1) the signature of sequence b goes
+ *           to token slot[b] (slot[b] < 0 skips b).
+ * ha_score_topk_wide — Eq. 1 as s = b - bitcount(k_code xor q_code) (Section 4.1), 0 .. b, group score = max over the
+ *   G query heads of the KV head, then the standard top-k (Section 4), ties to the lowest token index; always-kept
+ *   windows (shape->n_sink / n_local) as in ha_score_topk.
+ *   q_codes   words [batch][n_q_heads][b / 64]
+ *   k_codes   words [batch][n_kv_heads][>= seq_len][b / 64], 16-byte aligned (kc_stride_b, kc_stride_h in words)
+ *   hist_out  optional out i32 [batch][n_kv_heads][b + 1]: histogram of the group scores (windows excluded)
+ *   workspace at least ha_workspace_bytes_wide(shape, max_seq_len) bytes, 256-byte aligned; needs no initialisation;
+ *             calls that share it must be ordered on one stream. */
+int ha_encode_wide(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, int32_t batch, int32_t n_heads,
+                   int32_t n_tokens, uint64_t *codes, int64_t c_stride_b, int64_t c_stride_h, const int32_t *slot,
+                   void *stream);
+size_t ha_workspace_bytes_wide(const ha_shape *shape, int32_t max_seq_len);
+int ha_score_topk_wide(const ha_shape *shape, int32_t n_bits, const uint64_t *q_codes, const uint64_t *k_codes,
+                       int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
+                       int32_t k_uniform, int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
+                       int64_t idx_stride_h, int32_t *count, int32_t *hist_out, void *workspace, size_t ws_bytes,
+                       void *stream);
 
 /* The comparator column of the same table: dots[i] = <q, K[i]> for one query and n keys of 128 bf16
  * components ("128 x 16Float"), fp32 accumulation.

@@ -26,6 +26,7 @@ EXPORTS = [
     "ha_gather_attn_static", "ha_dense_decode", "ha_sparse_decode", "ha_sparse_decode_host", "ha_read_device_status",
     "ha_score_wide", "ha_inner_products", "ha_sparse_decode_paged_host", "ha_score_topk_sum",
     "ha_score_topk_per_head", "ha_gather_attn_per_head", "ha_sparse_decode_pipelined",
+    "ha_encode_wide", "ha_workspace_bytes_wide", "ha_score_topk_wide",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
 
@@ -88,6 +89,12 @@ def lib() -> C.CDLL:
         L.ha_sparse_decode_paged_host.argtypes = [P, P, P, P, P, P, P, P, P, I64, I32, P, I64, I64, P, P, I32, I32, I32, P,
                                                   I64, I64, P, P, P, SZ, P]
         L.ha_score_wide.argtypes = [P, P, I64, I32, P, P]
+        L.ha_encode_wide.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, P, P]
+        L.ha_encode_wide.restype = C.c_int
+        L.ha_workspace_bytes_wide.restype = SZ
+        L.ha_workspace_bytes_wide.argtypes = [P, I32]
+        L.ha_score_topk_wide.argtypes = [P, I32, P, P, I64, I64, P, P, I32, I32, I32, P, I64, I64, P, P, P, SZ, P]
+        L.ha_score_topk_wide.restype = C.c_int
         L.ha_inner_products.argtypes = [P, P, I64, I64, P, P]
         L.ha_kernel_launches.restype = C.c_uint64
         L.ha_status_string.restype = C.c_char_p
@@ -118,6 +125,61 @@ def ha_score_wide(q_code: torch.Tensor, k_codes: torch.Tensor, n_bits: int, scor
     assert k_codes.dim() == 2 and k_codes.shape[1] * 64 == n_bits == q_code.numel() * 64 and scores.numel() == n
     _check("ha_score_wide", lib().ha_score_wide(q_code.data_ptr(), k_codes.data_ptr(), n, n_bits, scores.data_ptr(),
                                                 _stream(stream)))
+
+
+class MappingWide:
+    """Device-resident weights of one side's mapping networks with a last layer of 128 x n_bits (64 .. 512)."""
+
+    def __init__(self, weights: Dict[str, torch.Tensor]):
+        self.t = {k: _dev(weights[k], torch.bfloat16, k).contiguous() for k in ("w1", "w2", "w3")}
+        for k in ("b1", "b2", "b3"):
+            b = weights.get(k)
+            self.t[k] = None if b is None else _dev(b, torch.float32, k).contiguous()
+        hkv, n_bits = self.t["w1"].shape[0], self.t["w3"].shape[2]
+        assert tuple(self.t["w1"].shape) == (hkv, 128, 128) and tuple(self.t["w2"].shape) == (hkv, 128, 128)
+        assert tuple(self.t["w3"].shape) == (hkv, 128, n_bits)
+        self.n_bits = n_bits
+        self.struct = ha_mapping(hkv, 128, 128, n_bits, _ptr(self.t["w1"]), _ptr(self.t["w2"]), _ptr(self.t["w3"]),
+                                 _ptr(self.t["b1"]), _ptr(self.t["b2"]), _ptr(self.t["b3"]))
+
+    @property
+    def ref(self):
+        return C.byref(self.struct)
+
+
+def ha_encode_wide(mapping: "MappingWide", heads_per_kv: int, x: torch.Tensor, codes: torch.Tensor,
+                   slot: Optional[torch.Tensor] = None, stream=None) -> None:
+    """x: bf16 [B,H,T,128] (or [B,H,128]); codes: int64 [B,H,>=T,n_bits/64] (the packed 64-bit words, contiguous per token)."""
+    xt = make_tensor(x)
+    B, H = x.shape[0], x.shape[1]
+    T = 1 if x.dim() == 3 else x.shape[2]
+    _dev(codes, torch.int64, "codes")
+    assert codes.dim() == 4 and codes.stride(3) == 1 and codes.stride(2) == codes.shape[3] == mapping.n_bits // 64
+    _check("ha_encode_wide", lib().ha_encode_wide(mapping.ref, heads_per_kv, C.byref(xt), B, H, T, codes.data_ptr(),
+                                                  codes.stride(0), codes.stride(1), _ptr(slot), _stream(stream)))
+
+
+def ha_workspace_bytes_wide(shape: ha_shape, max_seq_len: int) -> int:
+    n = int(lib().ha_workspace_bytes_wide(C.byref(shape), max_seq_len))
+    if n == 0:
+        raise HashAttnError("ha_workspace_bytes_wide", HA_ERR_UNSUPPORTED)
+    return n
+
+
+def alloc_workspace_wide(shape: ha_shape, max_seq_len: int, device="cuda") -> torch.Tensor:
+    return torch.empty(ha_workspace_bytes_wide(shape, max_seq_len), dtype=torch.uint8, device=device)
+
+
+def ha_score_topk_wide(shape: ha_shape, n_bits: int, q_codes, k_codes, seq_lens, k_per_seq, k_uniform: int, max_seq_len: int,
+                       k_max: int, idx, count, workspace, hist_out=None, stream=None) -> None:
+    """q_codes int64 [B,Hq,W]; k_codes int64 [B,Hkv,N,W] (W = n_bits/64 words per token); idx int32 [B,Hkv,k_max]."""
+    _dev(q_codes, torch.int64, "q_codes"); _dev(k_codes, torch.int64, "k_codes")
+    assert q_codes.is_contiguous() and k_codes.dim() == 4 and k_codes.stride(3) == 1 and k_codes.stride(2) == k_codes.shape[3]
+    p, n = _ws(workspace)
+    _check("ha_score_topk_wide", lib().ha_score_topk_wide(
+        C.byref(shape), n_bits, q_codes.data_ptr(), k_codes.data_ptr(), k_codes.stride(0), k_codes.stride(1),
+        seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform, max_seq_len, k_max, idx.data_ptr(), idx.stride(0), idx.stride(1),
+        count.data_ptr(), _ptr(hist_out), p, n, _stream(stream)))
 
 
 def ha_inner_products(q: torch.Tensor, K: torch.Tensor, dots: torch.Tensor, stream=None) -> None:

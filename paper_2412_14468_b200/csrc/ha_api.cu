@@ -527,6 +527,52 @@ int ha_score_wide(const uint64_t *q_code, const uint64_t *k_codes, int64_t n, in
     return HA_OK;
 }
 
+static bool wide_bits_ok(int32_t n_bits) { return n_bits == 64 || n_bits == 128 || n_bits == 256 || n_bits == 512; }
+
+int ha_encode_wide(const ha_mapping *map, int32_t heads_per_kv, const ha_tensor *x, int32_t batch, int32_t n_heads,
+                   int32_t n_tokens, uint64_t *codes, int64_t c_stride_b, int64_t c_stride_h, const int32_t *slot,
+                   void *stream) {
+    if (!map || !map->w1 || !map->w2 || !map->w3) return HA_ERR_INVALID_ARG;
+    if (map->in_dim != kD || map->hid_dim != kHid || !wide_bits_ok(map->n_bits)) return HA_ERR_UNSUPPORTED;
+    if (map->n_kv_heads <= 0 || (((uintptr_t)map->w1 | (uintptr_t)map->w2 | (uintptr_t)map->w3) & 15)) return HA_ERR_INVALID_ARG;
+    HA_TRY(check_tensor(x));
+    if (!codes || ((uintptr_t)codes & 7) || batch < 0 || n_heads <= 0 || n_tokens < 0 || heads_per_kv <= 0) return HA_ERR_INVALID_ARG;
+    if (n_heads % heads_per_kv != 0 || n_heads / heads_per_kv != map->n_kv_heads) return HA_ERR_INVALID_ARG;
+    if (slot && n_tokens != 1) return HA_ERR_INVALID_ARG;
+    if (batch > 65535 || n_heads > 65535) return HA_ERR_UNSUPPORTED;
+    if (batch == 0 || n_tokens == 0) return HA_OK;
+    HA_CUDA(launch_encode_wide(view(map), map->n_bits, heads_per_kv, view(x), batch, n_heads, n_tokens, codes, c_stride_b,
+                               c_stride_h, slot, (cudaStream_t)stream));
+    return HA_OK;
+}
+
+size_t ha_workspace_bytes_wide(const ha_shape *shape, int32_t max_seq_len) {
+    if (check_shape(shape) != HA_OK || max_seq_len < 0) return 0;
+    return wide_workspace_bytes(shape->batch, shape->n_kv_heads, max_seq_len);
+}
+
+int ha_score_topk_wide(const ha_shape *shape, int32_t n_bits, const uint64_t *q_codes, const uint64_t *k_codes,
+                       int64_t kc_stride_b, int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq,
+                       int32_t k_uniform, int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
+                       int64_t idx_stride_h, int32_t *count, int32_t *hist_out, void *workspace, size_t ws_bytes,
+                       void *stream) {
+    HA_TRY(check_shape(shape));
+    if (!wide_bits_ok(n_bits)) return HA_ERR_UNSUPPORTED;
+    if (!q_codes || !k_codes || !seq_lens || !idx || !count) return HA_ERR_INVALID_ARG;
+    if (max_seq_len < 0 || k_max < 0 || (!k_per_seq && k_uniform < 0)) return HA_ERR_INVALID_ARG;
+    if (((uintptr_t)k_codes & 15) || ((uintptr_t)q_codes & 7)) return HA_ERR_INVALID_ARG;
+    if (n_bits > 64 && ((kc_stride_b & 1) || (kc_stride_h & 1))) return HA_ERR_INVALID_ARG;   // 16-byte loads
+    if ((long long)shape->n_sink + shape->n_local > k_max) return HA_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255)) return HA_ERR_WORKSPACE;
+    if (ws_bytes < wide_workspace_bytes(shape->batch, shape->n_kv_heads, max_seq_len)) return HA_ERR_WORKSPACE;
+    if (shape->batch == 0) return HA_OK;
+    HA_CUDA(launch_score_topk_wide(shape->batch, shape->n_q_heads, shape->n_kv_heads, n_bits, q_codes, k_codes, kc_stride_b,
+                                   kc_stride_h, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx, idx_stride_b,
+                                   idx_stride_h, count, hist_out, workspace, (cudaStream_t)stream,
+                                   Windows{shape->n_sink, shape->n_local}));
+    return HA_OK;
+}
+
 int ha_inner_products(const uint16_t *q, const uint16_t *K, int64_t n, int64_t row_stride, float *dots, void *stream) {
     if (n < 0 || !q || (n > 0 && (!K || !dots)) || row_stride < kD || (row_stride & 7)) return HA_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(K) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(dots) & 3))

@@ -230,6 +230,15 @@ cudaError_t launch_gather_cluster(int B, int Hq, int Hkv, float sm_scale, const 
                                   cudaStream_t st, const int32_t *block_table = nullptr, long long bt_sb = 0,
                                   int page_shift = 0);
 
+// Signatures of 64 .. 512 bits through ENCODE and SCORE + TOPK (packed 64-bit words; strides in words).
+cudaError_t launch_encode_wide(const MapView &map, int n_bits, int heads_per_kv, TensorView x, int B, int H, int T,
+                               uint64_t *codes, long long c_sb, long long c_sh, const int32_t *slot, cudaStream_t st);
+size_t wide_workspace_bytes(int B, int Hkv, int max_seq_len);
+cudaError_t launch_score_topk_wide(int B, int Hq, int Hkv, int n_bits, const uint64_t *q_codes, const uint64_t *k_codes,
+                                   long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
+                                   int k_uniform, int max_seq_len, int k_max, int32_t *idx, long long idx_sb, long long idx_sh,
+                                   int32_t *count, int32_t *hist_out, void *workspace, cudaStream_t st, Windows win);
+
 cudaError_t launch_score_wide(const uint64_t *q_code, const uint64_t *k_codes, long long n, int n_words, uint16_t *scores,
                               cudaStream_t st);
 cudaError_t launch_inner_products(const uint16_t *q, const uint16_t *K, long long n, long long row_stride, float *dots,

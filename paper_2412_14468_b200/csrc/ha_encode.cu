@@ -584,3 +584,127 @@ cudaError_t launch_encode_bulk(const MapView &map, int heads_per_kv, TensorView 
 }
 
 } // namespace ha
+
+// ------------------------------------------------------------------ signatures of 64 to 512 bits
+//
+// Eq. 2 with a last layer of 128 x b (the widths of the bit-width study and of the SCORE-latency table): the token
+// tile, the two hidden layers and the arithmetic of every output are those of encode_bulk_kernel; the last layer
+// runs block by block over 32 outputs at a time (its 128 x 32 slice of W3 staged in shared memory), and block c
+// becomes the 32-bit half c % 2 of word c / 2 of the packed signature (bit j = bit j % 64 of word j / 64).
+namespace ha {
+
+__global__ void __launch_bounds__(kBulkThreads) encode_bulk_wide_kernel(MapView map, int n_bits, int heads_per_kv, TensorView x,
+                                                                       int T, uint32_t *codes32, long long c_sb,
+                                                                       long long c_sh, const int32_t *slot) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    uint16_t *sw1 = reinterpret_cast<uint16_t *>(smem);
+    uint16_t *sw2 = sw1 + kD * kHid;
+    uint16_t *sw3 = sw2 + kHid * kHid;                     // one 128 x 32 block of the last layer at a time
+    float *actA = reinterpret_cast<float *>(sw3 + kHid * kBits);
+    float *actB = actA + kTile * kActLd;
+
+    const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int net = h / heads_per_kv;
+    const int tid = threadIdx.x;
+    const int t0 = tile * kTile;
+    const int nt = min(kTile, T - t0);
+    const int n_words = n_bits / 64;
+    {
+        const uint4 *g1 = reinterpret_cast<const uint4 *>(map.w1 + (size_t)net * kD * kHid);
+        const uint4 *g2 = reinterpret_cast<const uint4 *>(map.w2 + (size_t)net * kHid * kHid);
+        uint4 *s1 = reinterpret_cast<uint4 *>(sw1), *s2 = reinterpret_cast<uint4 *>(sw2);
+        for (int i = tid; i < kD * kHid / 8; i += kBulkThreads) s1[i] = __ldg(g1 + i);
+        for (int i = tid; i < kHid * kHid / 8; i += kBulkThreads) s2[i] = __ldg(g2 + i);
+    }
+    const uint16_t *xb = x.ptr + (long long)b * x.sb + (long long)h * x.sh;
+    for (int i = tid; i < kTile * (kD / 8); i += kBulkThreads) {
+        const int t = i / (kD / 8), c = i % (kD / 8);
+        uint4 raw = make_uint4(0, 0, 0, 0);
+        if (t < nt) raw = __ldg(reinterpret_cast<const uint4 *>(xb + (long long)(t0 + t) * x.sn) + c);
+        const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+        float *dst = actA + t * kActLd + c * 8;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            dst[2 * e] = __uint_as_float(r[e] << 16);
+            dst[2 * e + 1] = __uint_as_float(r[e] & 0xffff0000u);
+        }
+    }
+    __syncthreads();
+    const int oq = tid & 31, tg = tid >> 5;
+    bulk_hidden_layer(actA, actB, sw1, map.b1 ? map.b1 + net * kHid : nullptr, oq, tg);
+    __syncthreads();
+    bulk_hidden_layer(actB, actA, sw2, map.b2 ? map.b2 + net * kHid : nullptr, oq, tg);
+    __syncthreads();
+
+    const int lane = tid & 31, op = tid & 15, tq = tid >> 4;
+    const uint16_t *g3 = map.w3 + (size_t)net * kHid * n_bits;
+    // the token slot a signature goes to: its position in the tile, or the append slot of its sequence (T == 1)
+    long long tok_base = t0;
+    bool write_ok = true;
+    if (slot) { const int sl = slot[b]; write_ok = sl >= 0; tok_base = sl; }
+    uint32_t *cb = codes32 + 2 * ((long long)b * c_sb + (long long)h * c_sh + tok_base * n_words);
+    for (int blk = 0; blk < n_bits / 32; ++blk) {
+        // W3[:, 32 blk .. 32 blk + 31]: 128 rows of 64 bytes, one 16-byte piece per thread
+        {
+            const int r = tid >> 2, pc = tid & 3;
+            reinterpret_cast<uint4 *>(sw3)[tid] = __ldg(reinterpret_cast<const uint4 *>(g3 + (size_t)r * n_bits + 32 * blk) + pc);
+        }
+        __syncthreads();
+        float z[4][2];
+        const float b0 = map.b3 ? map.b3[net * n_bits + 32 * blk + 2 * op] : 0.0f;
+        const float b1 = map.b3 ? map.b3[net * n_bits + 32 * blk + 2 * op + 1] : 0.0f;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) { z[t][0] = b0; z[t][1] = b1; }
+        const float *hin = actA + (size_t)tq * 4 * kActLd;
+#pragma unroll 4
+        for (int k = 0; k < 128; k += 4) {
+            float wf[4][2];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t wv = *reinterpret_cast<const uint32_t *>(sw3 + (k + i) * kBits + 2 * op);
+                wf[i][0] = __uint_as_float(wv << 16);
+                wf[i][1] = __uint_as_float(wv & 0xffff0000u);
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const float4 hv = *reinterpret_cast<const float4 *>(hin + t * kActLd + k);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    z[t][j] = __fmaf_rn(hv.x, wf[0][j], z[t][j]);
+                    z[t][j] = __fmaf_rn(hv.y, wf[1][j], z[t][j]);
+                    z[t][j] = __fmaf_rn(hv.z, wf[2][j], z[t][j]);
+                    z[t][j] = __fmaf_rn(hv.w, wf[3][j], z[t][j]);
+                }
+            }
+        }
+        auto spread16 = [](uint32_t v) {   // bit i -> bit 2 i
+            v = (v | (v << 8)) & 0x00ff00ffu;
+            v = (v | (v << 4)) & 0x0f0f0f0fu;
+            v = (v | (v << 2)) & 0x33333333u;
+            v = (v | (v << 1)) & 0x55555555u;
+            return v;
+        };
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const uint32_t even = __ballot_sync(0xffffffffu, z[t][0] > 0.0f), odd = __ballot_sync(0xffffffffu, z[t][1] > 0.0f);
+            const int shift = lane & 16;
+            const uint32_t code = spread16((even >> shift) & 0xffffu) | (spread16((odd >> shift) & 0xffffu) << 1);
+            const int tok = tq * 4 + t;
+            if (op == 0 && tok < nt && write_ok) cb[2 * ((long long)tok * n_words) + blk] = code;
+        }
+        __syncthreads();   // the block of W3 is overwritten by the next one
+    }
+}
+
+cudaError_t launch_encode_wide(const MapView &map, int n_bits, int heads_per_kv, TensorView x, int B, int H, int T,
+                               uint64_t *codes, long long c_sb, long long c_sh, const int32_t *slot, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(encode_bulk_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBulkSmem);
+    if (e != cudaSuccess) return e;
+    dim3 grid((T + kTile - 1) / kTile, H, B);
+    encode_bulk_wide_kernel<<<grid, kBulkThreads, kBulkSmem, st>>>(map, n_bits, heads_per_kv, x, T, reinterpret_cast<uint32_t *>(codes),
+                                                                  c_sb, c_sh, slot);
+    count_launch();
+    return cudaGetLastError();
+}
+
+} // namespace ha

@@ -1175,3 +1175,141 @@ def test_inner_products_match_the_oracle(n, stride):
     # 128 products of magnitude ~1 accumulated in fp32: error far below 1e-3
     assert np.max(np.abs(got[:n] - ref)) < 1e-3
     assert got[n] == 123.0
+
+
+# ---------------------------------------------------------------- wide signatures through ENCODE -> SCORE -> TOPK
+
+def _wide_mapping(hkv, n_bits, seed):
+    g = torch.Generator(DEV).manual_seed(seed)
+    m = wl.make_mapping(hkv, g, DEV)
+    bound = 1.0 / np.sqrt(128)
+    m["w3"] = ((torch.rand(hkv, 128, n_bits, device=DEV, generator=g) * 2 - 1) * bound).to(torch.bfloat16)
+    m["b3"] = (torch.rand(hkv, n_bits, device=DEV, generator=g) * 2 - 1) * bound
+    return m
+
+
+@pytest.mark.parametrize("n_bits", [64, 128, 256, 512])
+@pytest.mark.parametrize("T", [1, 77, 300])
+def test_encode_wide_is_bit_exact(n_bits, T):
+    """ha_encode_wide against the oracle's Eq. 2 with a 128 x b last layer: every word of every signature, for the
+    query side (heads sharing a network) and strided inputs, and the append into a token slot."""
+    B, Hkv, G, W = 2, 2, 2, n_bits // 64
+    m = _wide_mapping(Hkv, n_bits, 900 + n_bits)
+    mp = ha.MappingWide(m)
+    mn = wl.mapping_numpy(m)
+    g = torch.Generator(DEV).manual_seed(77 + T)
+    xs = torch.randn(B, Hkv * G, T + 3, 128, device=DEV, generator=g).to(torch.bfloat16)
+    x = xs[:, :, 1:T + 1]                                         # strided view
+    codes = torch.zeros(B, Hkv * G, T, W, dtype=torch.int64, device=DEV)
+    ha.ha_encode_wide(mp, G, x, codes)
+    torch.cuda.synchronize()
+    got = codes.cpu().numpy().view(np.uint64)
+    xu = u16(x.contiguous())
+    for b in range(B):
+        for h in range(Hkv * G):
+            net = h // G
+            ref = oracle.encode_wide(xu[b, h], mn["w1"][net], mn["w2"][net], mn["w3"][net], mn["b1"][net], mn["b2"][net], mn["b3"][net])
+            assert np.array_equal(got[b, h], ref), (b, h)
+    if T == 1:                                                    # append: one new vector per (sequence, head) into slot[b]
+        cache = torch.full((B, Hkv * G, 9, W), -1, dtype=torch.int64, device=DEV)
+        slot = torch.tensor([4, -1], dtype=torch.int32, device=DEV)
+        ha.ha_encode_wide(mp, G, x[:, :, 0], cache, slot=slot)
+        torch.cuda.synchronize()
+        c = cache.cpu().numpy()
+        assert np.array_equal(c[0, :, 4].view(np.uint64), got[0, :, 0]) and (c[1] == -1).all() and (c[0, :, :4] == -1).all()
+
+
+def _check_score_topk_wide(n_bits, qc, kc, lens, ks, Hq, Hkv, n_sink=0, n_local=0):
+    B, W, G = len(lens), n_bits // 64, Hq // Hkv
+    n_cap = kc.shape[2]
+    k_max = max(max(ks), 1) + n_sink + n_local
+    shape = ha.make_shape(B, Hq, Hkv, 1.0, n_sink=n_sink, n_local=n_local)
+    ws = ha.alloc_workspace_wide(shape, n_cap)
+    idx = torch.full((B, Hkv, k_max), 7, dtype=torch.int32, device=DEV)
+    cnt = torch.full((B, Hkv), 7, dtype=torch.int32, device=DEV)
+    hist = torch.full((B, Hkv, n_bits + 1), -1, dtype=torch.int32, device=DEV)
+    for _ in range(2):                                            # twice on one workspace: the histograms are cleared per call
+        ha.ha_score_topk_wide(shape, n_bits, torch.from_numpy(qc.view(np.int64)).to(DEV), torch.from_numpy(kc.view(np.int64)).to(DEV),
+                              torch.tensor(lens, dtype=torch.int32, device=DEV), torch.tensor(ks, dtype=torch.int32, device=DEV),
+                              0, n_cap, k_max, idx, cnt, ws, hist_out=hist)
+    torch.cuda.synchronize()
+    idx_np, cnt_np, hist_np = idx.cpu().numpy(), cnt.cpu().numpy(), hist.cpu().numpy()
+    for b, n in enumerate(lens):
+        for g in range(Hkv):
+            s = oracle.score_wide_group(qc[b, g * G:(g + 1) * G], kc[b, g, :n]) if n else np.zeros(0, np.int32)
+            ref = oracle.topk_windows(s, ks[b], n_sink, n_local) if (n_sink or n_local) else oracle.topk(s, ks[b])
+            assert cnt_np[b, g] == len(ref), (b, g, cnt_np[b, g], len(ref))
+            assert np.array_equal(idx_np[b, g, :len(ref)], ref), (b, g)
+            assert (idx_np[b, g, len(ref):] == -1).all()
+            others = np.ones(n, bool)
+            others[:min(n_sink, n)] = False
+            others[max(n - n_local, min(n_sink, n)):] = False
+            assert np.array_equal(hist_np[b, g], np.bincount(s[others], minlength=n_bits + 1))
+    return idx_np
+
+
+@pytest.mark.parametrize("n_bits", [64, 128, 256, 512])
+@pytest.mark.parametrize("G", [1, 4])
+def test_score_topk_wide_sizes_ragged_tail_budgets_and_ties(n_bits, G):
+    rng = np.random.default_rng(n_bits + G)
+    W, Hkv = n_bits // 64, 2
+    lens = [0, 1, 15, 4097, 20000, 70001]
+    ks = [3, 5, 20, 300, 0, 9000]
+    n_cap = max(lens) + 5
+    kc = _wide_codes(rng, len(lens) * Hkv * n_cap, W).reshape(len(lens), Hkv, n_cap, W)
+    qc = _wide_codes(rng, len(lens) * Hkv * G, W).reshape(len(lens), Hkv * G, W)
+    kc[3, :, 100:400] = kc[3, :, 99:100]                          # a block of equal signatures: ties decided by token index
+    kc[5, 0, 5000] = qc[5, 0]                                     # an exact match: the top level b
+    flip = rng.integers(0, 64, size=(n_cap,))                     # near matches at every distance from 1 on
+    kc[5, 1, :] = qc[5, G]
+    for t in range(0, 3000):
+        kc[5, 1, t, (t // 64) % W] ^= np.uint64(((1 << (t % 64 + 1)) - 1) & (2**64 - 1))
+    _check_score_topk_wide(n_bits, qc, kc, lens, ks, Hkv * G, Hkv)
+
+
+@pytest.mark.parametrize("n_sink,n_local", [(128, 128), (3, 0), (5000, 70000)])
+def test_score_topk_wide_with_always_kept_windows(n_sink, n_local):
+    rng = np.random.default_rng(7)
+    n_bits, W, Hkv, G = 128, 2, 2, 2
+    lens = [100, 6000, 150001]
+    ks = [10, 700, 2000]
+    n_cap = max(lens)
+    kc = _wide_codes(rng, len(lens) * Hkv * n_cap, W).reshape(len(lens), Hkv, n_cap, W)
+    qc = _wide_codes(rng, len(lens) * Hkv * G, W).reshape(len(lens), Hkv * G, W)
+    _check_score_topk_wide(n_bits, qc, kc, lens, ks, Hkv * G, Hkv, n_sink, n_local)
+
+
+@pytest.mark.parametrize("n_bits", [64, 256])
+def test_step_from_entry_points_at_wide_signatures(n_bits):
+    """ENCODE -> SCORE -> TOPK -> GATHER-ATT chained through the wide entry points against the same chain of oracle
+    functions (Section 4 recipe at b = 64 / 256 bits): the index lists of ha_score_topk_wide feed ha_gather_attn."""
+    cfg = wl.Config("wide-chain", 59, 3, [300, 5000, 1], None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8)
+    w = wl.make_workload(cfg, DEV)
+    B, Hq, Hkv, G, W = 3, 8, 2, 4, n_bits // 64
+    mq, mk = _wide_mapping(Hkv, n_bits, 31), _wide_mapping(Hkv, n_bits, 32)
+    n_cap, k_max = w["n_cap"], w["k_max"]
+    kc = torch.zeros(B, Hkv, n_cap, W, dtype=torch.int64, device=DEV)
+    qc = torch.zeros(B, Hq, 1, W, dtype=torch.int64, device=DEV)
+    ha.ha_encode_wide(ha.MappingWide(mk), 1, w["K"], kc)
+    ha.ha_encode_wide(ha.MappingWide(mq), G, w["q"], qc)
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
+    idx = torch.zeros(B, Hkv, k_max, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=DEV)
+    out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=DEV)
+    ha.ha_score_topk_wide(shape, n_bits, qc.reshape(B, Hq, W), kc, w["seq_lens"], w["k_per_seq"], 0, n_cap, k_max, idx, cnt,
+                          ha.alloc_workspace_wide(shape, n_cap))
+    ha.ha_gather_attn(shape, w["q"], w["K"], w["V"], w["seq_lens"], idx, cnt, k_max, out, ha.alloc_workspace(shape, n_cap, k_max))
+    torch.cuda.synchronize()
+    qu, Ku, Vu = u16(w["q"]), u16(w["K"]), u16(w["V"])
+    mqn, mkn = wl.mapping_numpy(mq), wl.mapping_numpy(mk)
+    idx_np, cnt_np = idx.cpu().numpy(), cnt.cpu().numpy()
+    for b, n in enumerate(w["lens"]):
+        for g in range(Hkv):
+            kcodes = oracle.encode_wide(Ku[b, g, :n], mkn["w1"][g], mkn["w2"][g], mkn["w3"][g], mkn["b1"][g], mkn["b2"][g], mkn["b3"][g])
+            qcodes = oracle.encode_wide(qu[b, g * G:(g + 1) * G], mqn["w1"][g], mqn["w2"][g], mqn["w3"][g], mqn["b1"][g], mqn["b2"][g], mqn["b3"][g])
+            assert np.array_equal(kc[b, g, :n].cpu().numpy().view(np.uint64), kcodes)
+            ref = oracle.topk(oracle.score_wide_group(qcodes, kcodes), w["ks"][b])
+            assert cnt_np[b, g] == len(ref) and np.array_equal(idx_np[b, g, :len(ref)], ref)
+            for j in range(G):
+                eo, _, _ = oracle.gather_attn(qu[b, g * G + j], Ku[b, g], Vu[b, g], ref, sm_scale=w["sm_scale"], n_valid=n)
+                assert_out_close(u16(out[b, g * G + j]), eo)
