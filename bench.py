@@ -641,6 +641,19 @@ def main():
                     ts.append(e0.elapsed_time(e1) * 1e3)
                 return float(sorted(ts[2:])[len(ts[2:]) // 2])
 
+            def cold_kernel_us(fn, iters=9):
+                ts = []
+                for _ in range(iters + 2):
+                    flush.fill_(1)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    torch.cuda._sleep(300000)
+                    e0.record()
+                    fn()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ts.append(e0.elapsed_time(e1) * 1e3)
+                return float(sorted(ts[2:])[len(ts[2:]) // 2])
+
             table = {}
             gs = torch.Generator(device).manual_seed(wl.BASE_SEED + 77)
             for n_tok, pm in paper_ms.items():
@@ -667,22 +680,39 @@ def main():
                 torch.cuda.empty_cache()
             supplementary["score_latency_table"] = table
 
+            # the same table through SCORE + TOPK (ha_score_topk_wide: one query head, k = n / 32, L2-cold launches): what a
+            # decode step pays for selection at each signature width, beside the 32-bit selection of the layer-step
+            sel = {}
+            for n_tok in paper_ms:
+                row = {}
+                shp1 = ha.make_shape(1, 1, 1, 1.0)
+                ln = torch.full((1,), n_tok, dtype=torch.int32, device=device)
+                kq = n_tok // 32
+                ix = torch.zeros(1, 1, kq, dtype=torch.int32, device=device)
+                ct = torch.zeros(1, 1, dtype=torch.int32, device=device)
+                kc32 = torch.randint(-2**31, 2**31 - 1, (1, 1, n_tok), dtype=torch.int32, device=device, generator=gs)
+                qc32 = torch.randint(-2**31, 2**31 - 1, (1, 1), dtype=torch.int32, device=device, generator=gs)
+                ws32 = ha.alloc_workspace(shp1, n_tok, kq, device=device)
+                us = cold_kernel_us(lambda: ha.ha_score_topk(shp1, qc32, kc32, ln, None, kq, n_tok, kq, ix, ct, ws32))
+                row["hamming_32bit"] = {"us": us, "gbs": n_tok * 4 / us / 1e3, "frac": n_tok * 4 / us / 1e3 / peak}
+                del kc32, ws32
+                wsw = ha.alloc_workspace_wide(shp1, n_tok, device=device)
+                for bits in (64, 128, 256, 512):
+                    W = bits // 64
+                    kcw = torch.randint(-2**63, 2**63 - 1, (1, 1, n_tok, W), dtype=torch.int64, device=device, generator=gs)
+                    qcw = torch.randint(-2**63, 2**63 - 1, (1, 1, W), dtype=torch.int64, device=device, generator=gs)
+                    us = cold_kernel_us(lambda: ha.ha_score_topk_wide(shp1, bits, qcw, kcw, ln, None, kq, n_tok, kq, ix, ct, wsw))
+                    nbytes = n_tok * 8 * W
+                    row[f"hamming_{bits}bit"] = {"us": us, "signature_gbs": nbytes / us / 1e3, "frac": nbytes / us / 1e3 / peak}
+                    del kcw
+                sel[f"{n_tok}_tokens"] = row
+                del wsw
+                torch.cuda.empty_cache()
+            supplementary["score_topk_latency_by_signature_width"] = sel
+
             # SCORE + TOPK alone with the two group reductions (maximum: the layer-step's contract; sum: the stand-alone
             # alternative), random signatures, L2-cold launches; the GPU is kept busy while the host enqueues, so the
             # events bracket the kernels only
-            def cold_kernel_us(fn, iters=9):
-                ts = []
-                for _ in range(iters + 2):
-                    flush.fill_(1)
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    torch.cuda._sleep(300000)
-                    e0.record()
-                    fn()
-                    e1.record()
-                    torch.cuda.synchronize()
-                    ts.append(e0.elapsed_time(e1) * 1e3)
-                return float(sorted(ts[2:])[len(ts[2:]) // 2])
-
             red = {}
             for name, (Bq, n_tok, kq) in {"c2": (1, 32768, 1024), "c3": (16, 32768, 2048), "batch64_32K": (64, 32768, 1024),
                                           "c4": (1, 524288, 16384)}.items():

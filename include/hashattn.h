@@ -228,8 +228,8 @@ int ha_gather_attn(const ha_shape *shape, const uint16_t *q, const ha_tensor *K,
  *                   number of rows per page stride (stride_b / stride_n, an integer)
  *   block_table     i32 [batch][>= ceil(seq_len / page_size)] page numbers (device)
  *   page_size       power of two (1 = every token its own page)
- * The index lists hold logical token numbers, exactly as ha_score_topk writes them (the signature cache
- * stays one contiguous array per sequence and KV head: 4 bytes per token). */
+ * The index lists hold logical token numbers, exactly as ha_score_topk writes them (here the signature cache
+ * stays one contiguous array per sequence and KV head; the *_paged entries further down page it too). */
 int ha_gather_attn_paged(const ha_shape *shape, const uint16_t *q, const ha_tensor *K_pool,
                          const ha_tensor *V_pool, const int32_t *block_table, int64_t bt_stride_b,
                          int32_t page_size, const int32_t *seq_lens, const int32_t *idx,
@@ -315,6 +315,50 @@ int ha_sparse_decode_paged_host(const ha_shape *shape, const ha_mapping *map_q, 
                                 int32_t k_uniform, int32_t max_seq_len, int32_t k_max, int32_t *idx,
                                 int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
                                 uint16_t *out_host, void *workspace, size_t ws_bytes, void *stream);
+
+/* The signature cache in pages as well (Section 4.1 "Implementation": signatures are computed and cached along with the
+ * KV cache; the paper's vLLM integration, Section 4.4, keeps that cache in pages).  code_pool holds the 32-bit signatures
+ * as [n_pages][n_kv_heads][page_size] addressed by element strides (cp_stride_page, cp_stride_head; multiples of 4 and a
+ * 16-byte aligned base when page_size >= 4), with the SAME block table and page size as the K/V pools: the signature of
+ * token t of sequence b and KV head h is
+ *     code_pool[block_table[b * bt_stride_b + t / page_size] * cp_stride_page + h * cp_stride_head + t % page_size].
+ * page_size is a power of two; 16 makes a page one 64-byte segment per head, 1 gives every token its own page.
+ * Index lists hold logical token numbers and are bit-identical to those over a contiguous cache.
+ *   ha_score_topk_paged            ha_score_topk over the pool (arguments otherwise the same)
+ *   ha_score_topk_per_head_paged   ha_score_topk_per_head over the pool; unlike its contiguous form it takes
+ *                                  max_seq_len and a workspace from ha_workspace_bytes for the shape with n_kv_heads
+ *                                  set to n_q_heads
+ *   ha_gather_attn_per_head_paged  ha_gather_attn_per_head over paged K/V pools (as ha_gather_attn_paged)
+ *   ha_encode_append_paged         the append of Section 4.1 into the pool: signature of k_new [batch][n_kv_heads][128]
+ *                                  (phi_kv) written at token seq_lens[b] - 1 of sequence b (skipped if that is < 0)
+ *   ha_sparse_decode_paged_codes   the whole layer-step with K, V and the signatures all paged (ENCODE with the append
+ *                                  into the pool, SCORE + TOPK, GATHER-ATT as separate kernels) */
+int ha_score_topk_paged(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *code_pool, int64_t cp_stride_page,
+                        int64_t cp_stride_head, const int32_t *block_table, int64_t bt_stride_b, int32_t page_size,
+                        const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform, int32_t max_seq_len,
+                        int32_t k_max, int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
+                        int32_t *hist_out, void *workspace, size_t ws_bytes, void *stream);
+int ha_score_topk_per_head_paged(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *code_pool,
+                                 int64_t cp_stride_page, int64_t cp_stride_head, const int32_t *block_table,
+                                 int64_t bt_stride_b, int32_t page_size, const int32_t *seq_lens, const int32_t *k_per_seq,
+                                 int32_t k_uniform, int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
+                                 int64_t idx_stride_h, int32_t *count, int32_t *hist_out, void *workspace, size_t ws_bytes,
+                                 void *stream);
+int ha_gather_attn_per_head_paged(const ha_shape *shape, const uint16_t *q, const ha_tensor *K_pool,
+                                  const ha_tensor *V_pool, const int32_t *block_table, int64_t bt_stride_b,
+                                  int32_t page_size, const int32_t *seq_lens, const int32_t *idx, int64_t idx_stride_b,
+                                  int64_t idx_stride_h, const int32_t *count, int32_t k_max, uint16_t *out, float *lse,
+                                  void *workspace, size_t ws_bytes, void *stream);
+int ha_encode_append_paged(const ha_mapping *map, const uint16_t *k_new, int32_t batch, uint32_t *code_pool,
+                           int64_t cp_stride_page, int64_t cp_stride_head, const int32_t *block_table, int64_t bt_stride_b,
+                           int32_t page_size, const int32_t *seq_lens, void *stream);
+int ha_sparse_decode_paged_codes(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k, const uint16_t *q,
+                                 const uint16_t *k_new, const ha_tensor *K_pool, const ha_tensor *V_pool,
+                                 uint32_t *code_pool, int64_t cp_stride_page, int64_t cp_stride_head,
+                                 const int32_t *block_table, int64_t bt_stride_b, int32_t page_size, const int32_t *seq_lens,
+                                 const int32_t *k_per_seq, int32_t k_uniform, int32_t max_seq_len, int32_t k_max,
+                                 uint32_t *q_codes, int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count,
+                                 uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream);
 
 /* GATHER-ATT without a caller-provided workspace.  (The paper has no counterpart of this entry
  * point; it exists for integration reasons only.)

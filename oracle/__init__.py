@@ -183,6 +183,16 @@ def unpage_rows(pool, block_table_row, page_size: int, head: int, n: int) -> np.
     return np.ascontiguousarray(pool[pages, head, t % page_size, :])
 
 
+def unpage_codes(pool, block_table_row, page_size: int, head: int, n: int) -> np.ndarray:
+    """Signatures 0..n-1 of one sequence and KV head out of a paged signature cache: pool is uint32 [n_pages, Hkv,
+    page_size]; token t lives in page block_table_row[t // page_size] at slot t % page_size.  Paging is storage only:
+    SCORE + TOPK over a paged cache is score / topk over these signatures."""
+    pool = np.ascontiguousarray(pool, dtype=np.uint32)
+    t = np.arange(n)
+    pages = np.asarray(block_table_row, dtype=np.int64)[t // page_size]
+    return np.ascontiguousarray(pool[pages, head, t % page_size])
+
+
 def dense(q, K, V, n=None, sm_scale=None):
     """SDPA for one query over tokens 0..n-1."""
     return gather_attn(q, K, V, None, sm_scale=sm_scale, n_valid=n)

@@ -27,6 +27,8 @@ EXPORTS = [
     "ha_score_wide", "ha_inner_products", "ha_sparse_decode_paged_host", "ha_score_topk_sum",
     "ha_score_topk_per_head", "ha_gather_attn_per_head", "ha_sparse_decode_pipelined",
     "ha_encode_wide", "ha_workspace_bytes_wide", "ha_score_topk_wide",
+    "ha_score_topk_paged", "ha_score_topk_per_head_paged", "ha_gather_attn_per_head_paged", "ha_encode_append_paged",
+    "ha_sparse_decode_paged_codes",
     "ha_kernel_launches", "ha_status_string", "ha_version",
 ]
 
@@ -89,6 +91,15 @@ def lib() -> C.CDLL:
         L.ha_sparse_decode_paged_host.argtypes = [P, P, P, P, P, P, P, P, P, I64, I32, P, I64, I64, P, P, I32, I32, I32, P,
                                                   I64, I64, P, P, P, SZ, P]
         L.ha_score_wide.argtypes = [P, P, I64, I32, P, P]
+        L.ha_score_topk_paged.argtypes = [P, P, P, I64, I64, P, I64, I32, P, P, I32, I32, I32, P, I64, I64, P, P, P, SZ, P]
+        L.ha_score_topk_per_head_paged.argtypes = L.ha_score_topk_paged.argtypes
+        L.ha_gather_attn_per_head_paged.argtypes = L.ha_gather_attn_paged.argtypes
+        L.ha_encode_append_paged.argtypes = [P, P, I32, P, I64, I64, P, I64, I32, P, P]
+        L.ha_sparse_decode_paged_codes.argtypes = [P, P, P, P, P, P, P, P, I64, I64, P, I64, I32, P, P, I32, I32, I32, P, P,
+                                                   I64, I64, P, P, P, P, SZ, P]
+        for fn in ("ha_score_topk_paged", "ha_score_topk_per_head_paged", "ha_gather_attn_per_head_paged",
+                   "ha_encode_append_paged", "ha_sparse_decode_paged_codes"):
+            getattr(L, fn).restype = C.c_int
         L.ha_encode_wide.argtypes = [P, I32, P, I32, I32, I32, P, I64, I64, P, P]
         L.ha_encode_wide.restype = C.c_int
         L.ha_workspace_bytes_wide.restype = SZ
@@ -358,6 +369,67 @@ def ha_gather_attn_paged(shape: ha_shape, q, K_pool, V_pool, block_table, page_s
     _check("ha_gather_attn_paged", lib().ha_gather_attn_paged(
         C.byref(shape), q.data_ptr(), C.byref(kt), C.byref(vt), block_table.data_ptr(), block_table.stride(0), page_size,
         seq_lens.data_ptr(), idx.data_ptr(), idx.stride(0), idx.stride(1), count.data_ptr(), k_max, out.data_ptr(),
+        _ptr(lse), p, n, _stream(stream)))
+
+
+def _pool(code_pool: torch.Tensor):
+    """int32 [n_pages, Hkv, page_size] signature pool -> (pointer, page stride, head stride, page size)."""
+    _dev(code_pool, torch.int32, "code_pool")
+    assert code_pool.dim() == 3 and code_pool.stride(2) == 1
+    return code_pool.data_ptr(), code_pool.stride(0), code_pool.stride(1), code_pool.shape[2]
+
+
+def ha_score_topk_paged(shape: ha_shape, q_codes, code_pool, block_table, seq_lens, k_per_seq, k_uniform: int, max_seq_len: int,
+                        k_max: int, idx, count, workspace, hist_out=None, per_head: bool = False, stream=None) -> None:
+    """ha_score_topk (per_head: ha_score_topk_per_head) over a paged signature pool int32 [n_pages, Hkv, page_size]."""
+    p, n = _ws(workspace)
+    cp, sp, sh, ps = _pool(code_pool)
+    fn = lib().ha_score_topk_per_head_paged if per_head else lib().ha_score_topk_paged
+    _check("ha_score_topk_per_head_paged" if per_head else "ha_score_topk_paged", fn(
+        C.byref(shape), q_codes.data_ptr(), cp, sp, sh, block_table.data_ptr(), block_table.stride(0), ps, seq_lens.data_ptr(),
+        _ptr(k_per_seq), k_uniform, max_seq_len, k_max, idx.data_ptr(), idx.stride(0), idx.stride(1), count.data_ptr(),
+        _ptr(hist_out), p, n, _stream(stream)))
+
+
+def ha_score_topk_per_head_paged(shape: ha_shape, q_codes, code_pool, block_table, seq_lens, k_per_seq, k_uniform: int,
+                                 max_seq_len: int, k_max: int, idx, count, workspace, hist_out=None, stream=None) -> None:
+    """ha_score_topk_per_head over a paged signature pool; workspace sized for the shape with n_kv_heads = n_q_heads."""
+    ha_score_topk_paged(shape, q_codes, code_pool, block_table, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx, count,
+                        workspace, hist_out=hist_out, per_head=True, stream=stream)
+
+
+def ha_gather_attn_per_head_paged(shape: ha_shape, q, K_pool, V_pool, block_table, page_size: int, seq_lens, idx, count,
+                                  k_max: int, out, workspace, lse=None, stream=None) -> None:
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K_pool), make_tensor(V_pool)
+    _check("ha_gather_attn_per_head_paged", lib().ha_gather_attn_per_head_paged(
+        C.byref(shape), q.data_ptr(), C.byref(kt), C.byref(vt), block_table.data_ptr(), block_table.stride(0), page_size,
+        seq_lens.data_ptr(), idx.data_ptr(), idx.stride(0), idx.stride(1), count.data_ptr(), k_max, out.data_ptr(),
+        _ptr(lse), p, n, _stream(stream)))
+
+
+def ha_encode_append_paged(mapping: Mapping, k_new, code_pool, block_table, seq_lens, stream=None) -> None:
+    """Signature of k_new bf16 [B, Hkv, 128] written at token seq_lens[b] - 1 of sequence b in the paged pool."""
+    cp, sp, sh, ps = _pool(code_pool)
+    _dev(k_new, torch.bfloat16, "k_new")
+    assert k_new.is_contiguous()
+    _check("ha_encode_append_paged", lib().ha_encode_append_paged(
+        mapping.ref, k_new.data_ptr(), k_new.shape[0], cp, sp, sh, block_table.data_ptr(), block_table.stride(0), ps,
+        seq_lens.data_ptr(), _stream(stream)))
+
+
+def ha_sparse_decode_paged_codes(shape: ha_shape, map_q: Mapping, map_k: Optional[Mapping], q, k_new, K_pool, V_pool, code_pool,
+                                 block_table, seq_lens, k_per_seq, k_uniform: int, max_seq_len: int, k_max: int, q_codes, idx,
+                                 count, out, workspace, lse=None, stream=None) -> None:
+    """The whole step with K, V (bf16 [n_pages, Hkv, page_size, 128]) and the signatures (int32 [n_pages, Hkv, page_size])
+    all paged through one block table int32 [B, pages]."""
+    p, n = _ws(workspace)
+    kt, vt = make_tensor(K_pool), make_tensor(V_pool)
+    cp, sp, sh, ps = _pool(code_pool)
+    _check("ha_sparse_decode_paged_codes", lib().ha_sparse_decode_paged_codes(
+        C.byref(shape), map_q.ref, None if map_k is None else map_k.ref, q.data_ptr(), _ptr(k_new), C.byref(kt), C.byref(vt),
+        cp, sp, sh, block_table.data_ptr(), block_table.stride(0), ps, seq_lens.data_ptr(), _ptr(k_per_seq), k_uniform,
+        max_seq_len, k_max, q_codes.data_ptr(), idx.data_ptr(), idx.stride(0), idx.stride(1), count.data_ptr(), out.data_ptr(),
         _ptr(lse), p, n, _stream(stream)))
 
 

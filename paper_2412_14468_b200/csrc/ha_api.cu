@@ -303,11 +303,14 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
                               int64_t kc_stride_h, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
                               int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx, int64_t idx_stride_b,
                               int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse, void *workspace,
-                              size_t ws_bytes, void *stream, const uint16_t *v_new_host = nullptr, bool pipelined = false) {
+                              size_t ws_bytes, void *stream, const uint16_t *v_new_host = nullptr, bool pipelined = false,
+                              CodePages code_pages = CodePages{nullptr, 0, 0, 0, 0}) {
     HA_TRY(check_score_args(shape, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_uniform, k_per_seq,
                             max_seq_len, k_max, idx, count));
     HA_TRY(check_mapping(map_q, shape->n_kv_heads));
     if (k_new) HA_TRY(check_mapping(map_k, shape->n_kv_heads));
+    const bool codes_paged = code_pages.table != nullptr;   // then only the kernel-by-kernel path knows the layout
+    if (codes_paged && (pipelined || v_new_host)) return HA_ERR_UNSUPPORTED;
     HA_TRY(check_tensor(K));
     HA_TRY(check_tensor(V));
     if (!q || !out || ((uintptr_t)q & 15)) return HA_ERR_INVALID_ARG;
@@ -318,7 +321,7 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
     const int B = shape->batch, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
 
     if (pipelined && !pipe_step_eligible(B, Hq, Hkv)) return HA_ERR_UNSUPPORTED;
-    if (!pipelined && fused_step_eligible(B, Hq, Hkv, max_seq_len, k_max)) {
+    if (!pipelined && !codes_paged && fused_step_eligible(B, Hq, Hkv, max_seq_len, k_max)) {
         // small batch: the whole step is one cluster kernel
         HA_CUDA(launch_fused_step(B, Hq, Hkv, shape->sm_scale, view(map_q), k_new ? view(map_k) : MapView{}, q, k_new,
                                   view(K), view(V), k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
@@ -341,6 +344,7 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
         jk.slot = seq_lens; jk.slot_minus_one = 1;
         jk.n_heads = Hkv; jk.heads_per_kv = 1; jk.n_cta = B * Hkv;
         jk.map = view(map_k);
+        jk.pages = code_pages;
     }
     HA_CUDA(launch_encode_vectors(jq, jk, st));
     if (pipelined) {
@@ -359,7 +363,7 @@ static int sparse_decode_impl(const ha_shape *shape, const ha_mapping *map_q, co
     HA_CUDA(launch_score_topk(B, Hq, Hkv, q_codes, k_codes, kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform,
                               max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, nullptr,
                               ws_ptr<int32_t>(workspace, L.off_hist), ws_ptr<unsigned char>(workspace, L.off_scores), st,
-                              Windows{shape->n_sink, shape->n_local}));
+                              Windows{shape->n_sink, shape->n_local}, code_pages));
     if (gather_cluster_eligible(B, Hq, Hkv, k_max)) {
         // up to a cluster per unit resident at once and short lists: GATHER-ATT with the states merged in shared memory
         HA_CUDA(launch_gather_cluster(B, Hq, Hkv, shape->sm_scale, q, view(K), view(V), seq_lens, idx, idx_stride_b,
@@ -414,6 +418,129 @@ int ha_sparse_decode_paged(const ha_shape *shape, const ha_mapping *map_q, const
     return sparse_decode_impl(shape, map_q, map_k, q, k_new, K_pool, V_pool, block_table, bt_stride_b, shift, k_codes,
                               kc_stride_b, kc_stride_h, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, q_codes, idx,
                               idx_stride_b, idx_stride_h, count, out, lse, workspace, ws_bytes, stream);
+}
+
+// ---- paged signature cache: the signatures live in a pool beside the K/V pools, addressed by the same block table
+
+static int check_code_pool(const uint32_t *code_pool, int64_t cp_stride_page, int64_t cp_stride_head, const int32_t *block_table,
+                           int32_t page_size, CodePages *cp, int64_t bt_stride_b) {
+    if (!code_pool || !block_table) return HA_ERR_INVALID_ARG;
+    if (page_size <= 0 || (page_size & (page_size - 1)) || page_size > 65536) return HA_ERR_INVALID_ARG;
+    // pages of four tokens or more are read sixteen bytes at a time
+    if (((uintptr_t)code_pool & 15) || (page_size >= 4 && ((cp_stride_page & 3) || (cp_stride_head & 3)))) return HA_ERR_INVALID_ARG;
+    int shift = 0;
+    while ((1 << shift) < page_size) ++shift;
+    *cp = CodePages{block_table, (long long)bt_stride_b, (long long)cp_stride_page, (long long)cp_stride_head, shift};
+    return HA_OK;
+}
+
+int ha_score_topk_paged(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *code_pool, int64_t cp_stride_page,
+                        int64_t cp_stride_head, const int32_t *block_table, int64_t bt_stride_b, int32_t page_size,
+                        const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform, int32_t max_seq_len, int32_t k_max,
+                        int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, int32_t *count, int32_t *hist_out,
+                        void *workspace, size_t ws_bytes, void *stream) {
+    CodePages cp;
+    HA_TRY(check_code_pool(code_pool, cp_stride_page, cp_stride_head, block_table, page_size, &cp, bt_stride_b));
+    HA_TRY(check_score_args(shape, q_codes, code_pool, 0, 0, seq_lens, k_uniform, k_per_seq, max_seq_len, k_max, idx, count));
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(shape, max_seq_len, workspace, ws_bytes, &L));
+    if (shape->batch == 0) return HA_OK;
+    HA_CUDA(launch_score_topk(shape->batch, shape->n_q_heads, shape->n_kv_heads, q_codes, code_pool, 0, 0, seq_lens, k_per_seq,
+                              k_uniform, max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, hist_out,
+                              ws_ptr<int32_t>(workspace, L.off_hist), ws_ptr<unsigned char>(workspace, L.off_scores),
+                              (cudaStream_t)stream, Windows{shape->n_sink, shape->n_local}, cp));
+    return HA_OK;
+}
+
+int ha_score_topk_per_head_paged(const ha_shape *shape, const uint32_t *q_codes, const uint32_t *code_pool,
+                                 int64_t cp_stride_page, int64_t cp_stride_head, const int32_t *block_table,
+                                 int64_t bt_stride_b, int32_t page_size, const int32_t *seq_lens, const int32_t *k_per_seq,
+                                 int32_t k_uniform, int32_t max_seq_len, int32_t k_max, int32_t *idx, int64_t idx_stride_b,
+                                 int64_t idx_stride_h, int32_t *count, int32_t *hist_out, void *workspace, size_t ws_bytes,
+                                 void *stream) {
+    CodePages cp;
+    HA_TRY(check_code_pool(code_pool, cp_stride_page, cp_stride_head, block_table, page_size, &cp, bt_stride_b));
+    HA_TRY(check_score_args(shape, q_codes, code_pool, 0, 0, seq_lens, k_uniform, k_per_seq, max_seq_len, k_max, idx, count));
+    ha_shape units = *shape;             // every query head is a unit: the scratch is laid out for that many
+    units.n_kv_heads = shape->n_q_heads;
+    HA_TRY(check_shape(&units));
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(&units, max_seq_len, workspace, ws_bytes, &L));
+    if (shape->batch == 0) return HA_OK;
+    int shift = 0;
+    while ((shape->n_kv_heads << shift) < shape->n_q_heads) ++shift;
+    HA_CUDA(launch_score_topk(shape->batch, shape->n_q_heads, shape->n_kv_heads, q_codes, code_pool, 0, 0, seq_lens, k_per_seq,
+                              k_uniform, max_seq_len, k_max, idx, idx_stride_b, idx_stride_h, count, hist_out,
+                              ws_ptr<int32_t>(workspace, L.off_hist), ws_ptr<unsigned char>(workspace, L.off_scores),
+                              (cudaStream_t)stream, Windows{shape->n_sink, shape->n_local}, cp, shift));
+    return HA_OK;
+}
+
+int ha_gather_attn_per_head_paged(const ha_shape *shape, const uint16_t *q, const ha_tensor *K_pool, const ha_tensor *V_pool,
+                                  const int32_t *block_table, int64_t bt_stride_b, int32_t page_size, const int32_t *seq_lens,
+                                  const int32_t *idx, int64_t idx_stride_b, int64_t idx_stride_h, const int32_t *count,
+                                  int32_t k_max, uint16_t *out, float *lse, void *workspace, size_t ws_bytes, void *stream) {
+    HA_TRY(check_shape(shape));
+    HA_TRY(check_tensor(K_pool));
+    HA_TRY(check_tensor(V_pool));
+    if (!q || !block_table || !seq_lens || !idx || !count || !out || k_max < 0 || ((uintptr_t)q & 15)) return HA_ERR_INVALID_ARG;
+    if (page_size <= 0 || (page_size & (page_size - 1)) || page_size > 65536) return HA_ERR_INVALID_ARG;
+    if (K_pool->stride_b % K_pool->stride_n != 0 || V_pool->stride_b % V_pool->stride_n != 0 ||
+        K_pool->stride_b / K_pool->stride_n != V_pool->stride_b / V_pool->stride_n)
+        return HA_ERR_INVALID_ARG;
+    ha_shape units = *shape;
+    units.n_kv_heads = shape->n_q_heads;
+    HA_TRY(check_shape(&units));
+    WorkspaceLayout L;
+    HA_TRY(check_workspace(&units, -1, workspace, ws_bytes, &L));
+    if (shape->batch == 0) return HA_OK;
+    int kv_shift = 0, page_shift = 0;
+    while ((shape->n_kv_heads << kv_shift) < shape->n_q_heads) ++kv_shift;
+    while ((1 << page_shift) < page_size) ++page_shift;
+    HA_CUDA(launch_attention(true, shape->batch, shape->n_q_heads, shape->n_q_heads, shape->sm_scale, q, view(K_pool), view(V_pool),
+                             seq_lens, idx, idx_stride_b, idx_stride_h, count, k_max, out, lse,
+                             ws_ptr<float>(workspace, L.off_part_ml), ws_ptr<float>(workspace, L.off_part_acc),
+                             ws_ptr<int32_t>(workspace, L.off_tickets), ws_ptr<uint32_t>(workspace, 0), (cudaStream_t)stream, 0,
+                             nullptr, 0, Windows{0, 0}, block_table, bt_stride_b, page_shift, kv_shift));
+    return HA_OK;
+}
+
+int ha_encode_append_paged(const ha_mapping *map, const uint16_t *k_new, int32_t batch, uint32_t *code_pool,
+                           int64_t cp_stride_page, int64_t cp_stride_head, const int32_t *block_table, int64_t bt_stride_b,
+                           int32_t page_size, const int32_t *seq_lens, void *stream) {
+    HA_TRY(check_mapping(map, 0));
+    CodePages cp;
+    HA_TRY(check_code_pool(code_pool, cp_stride_page, cp_stride_head, block_table, page_size, &cp, bt_stride_b));
+    if (!k_new || ((uintptr_t)k_new & 15) || !seq_lens || batch < 0 || batch > 65535) return HA_ERR_INVALID_ARG;
+    if (batch == 0) return HA_OK;
+    const int Hkv = map->n_kv_heads;
+    EncodeJob jk{};
+    jk.x = k_new; jk.x_sb = (long long)Hkv * kD; jk.x_sh = kD;
+    jk.codes = code_pool; jk.slot = seq_lens; jk.slot_minus_one = 1;
+    jk.n_heads = Hkv; jk.heads_per_kv = 1; jk.n_cta = batch * Hkv;
+    jk.map = view(map);
+    jk.pages = cp;
+    EncodeJob none{};
+    HA_CUDA(launch_encode_vectors(jk, none, (cudaStream_t)stream));
+    return HA_OK;
+}
+
+int ha_sparse_decode_paged_codes(const ha_shape *shape, const ha_mapping *map_q, const ha_mapping *map_k, const uint16_t *q,
+                                 const uint16_t *k_new, const ha_tensor *K_pool, const ha_tensor *V_pool, uint32_t *code_pool,
+                                 int64_t cp_stride_page, int64_t cp_stride_head, const int32_t *block_table, int64_t bt_stride_b,
+                                 int32_t page_size, const int32_t *seq_lens, const int32_t *k_per_seq, int32_t k_uniform,
+                                 int32_t max_seq_len, int32_t k_max, uint32_t *q_codes, int32_t *idx, int64_t idx_stride_b,
+                                 int64_t idx_stride_h, int32_t *count, uint16_t *out, float *lse, void *workspace,
+                                 size_t ws_bytes, void *stream) {
+    if (!K_pool || !V_pool) return HA_ERR_INVALID_ARG;
+    CodePages cp;
+    HA_TRY(check_code_pool(code_pool, cp_stride_page, cp_stride_head, block_table, page_size, &cp, bt_stride_b));
+    if (K_pool->stride_n <= 0 || V_pool->stride_n <= 0 || K_pool->stride_b % K_pool->stride_n != 0 ||
+        V_pool->stride_b % V_pool->stride_n != 0 || K_pool->stride_b / K_pool->stride_n != V_pool->stride_b / V_pool->stride_n)
+        return HA_ERR_INVALID_ARG;
+    return sparse_decode_impl(shape, map_q, map_k, q, k_new, K_pool, V_pool, block_table, bt_stride_b, cp.shift, code_pool, 0, 0,
+                              seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, q_codes, idx, idx_stride_b, idx_stride_h, count,
+                              out, lse, workspace, ws_bytes, stream, nullptr, false, cp);
 }
 
 // Both host-buffer entries: block_table == NULL is the contiguous cache, else K / V are pools (page_shift = log2 of

@@ -140,6 +140,15 @@ inline int forced_before(WindowBounds w, int p) {
     return (p < w.sink_end ? p : w.sink_end) + (p > w.local_begin ? p - w.local_begin : 0);
 }
 
+// A paged signature cache (the paper's vLLM integration keeps the KV cache, and with it the signatures of Section 4.1,
+// in pages addressed through a block table): token t of sequence b and KV head h is the 32-bit word
+// pool[table[b * bt_sb + (t >> shift)] * page_stride + h * head_stride + (t & (2^shift - 1))].  table == NULL: contiguous.
+struct CodePages {
+    const int32_t *table;
+    long long bt_sb, page_stride, head_stride;
+    int shift;
+};
+
 // One batch of single vectors to encode (decode step): CTA i handles sequence i / n_nets and
 // network i % n_nets, i.e. the heads_per_kv (<= 8) heads that share that network.
 struct EncodeJob {
@@ -152,7 +161,17 @@ struct EncodeJob {
     int n_heads, heads_per_kv, n_cta;   // n_cta = batch * n_heads / heads_per_kv
     int batch, cta_per_net;  // filled in by the launcher: sequences, and CTAs that share one network's items
     MapView map;
+    CodePages pages;         // pages.table != NULL: `codes` is a paged pool and the slot a token of the sequence
 };
+#ifdef __CUDACC__
+// where the signature of (sequence b, head h, token slot) is stored
+__device__ __forceinline__ uint32_t *encode_slot_ptr(const EncodeJob &J, int b, int h, int slot) {
+    if (J.pages.table)
+        return J.codes + (long long)J.pages.table[(long long)b * J.pages.bt_sb + (slot >> J.pages.shift)] * J.pages.page_stride +
+               (long long)h * J.pages.head_stride + (slot & ((1 << J.pages.shift) - 1));
+    return J.codes + (long long)b * J.c_sb + (long long)h * J.c_sh + slot;
+}
+#endif
 
 // Number of SMs of the current device (cached per device).
 inline int sm_count() {
@@ -181,7 +200,10 @@ cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, c
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens,
                               const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max,
                               int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
-                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st, Windows win = Windows{0, 0});
+                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st, Windows win = Windows{0, 0},
+                              CodePages pages = CodePages{nullptr, 0, 0, 0, 0}, int row_shift = -1);
+// pages.table != NULL: k_codes is a paged pool (always the two-kernel path); row_shift >= 0: one unit per QUERY head
+// (Hq units per sequence, groups of one head), whose signature row is that of KV head h >> row_shift.
 
 // SCORE + TOPK with the group's per-head scores added instead of maximised (one cluster per unit, no scratch);
 // per_head: no reduction at all, one list per QUERY head (idx, count, hist_out then have n_q_heads rows per sequence).

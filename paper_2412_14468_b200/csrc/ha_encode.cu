@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(kVecThreads) encode_vec_kernel(EncodeJob ja, E
                         int slot = 0;
                         if (J.slot) slot = J.slot[b] - J.slot_minus_one;   // a negative slot skips the sequence
                         if (lane == 0 && slot >= 0)
-                            J.codes[(long long)b * J.c_sb + (long long)(net * hpk + t % hpk) * J.c_sh + slot] = code;
+                            *encode_slot_ptr(J, b, net * hpk + t % hpk, slot) = code;
                     }
                 }
             }
@@ -330,7 +330,7 @@ __global__ void __launch_bounds__(64 * NG) encode_tile_kernel(EncodeJob ja, Enco
                 const int t = t0 + v3, b = t / hpk;
                 int slot = 0;
                 if (J.slot) slot = J.slot[b] - J.slot_minus_one;   // a negative slot skips the sequence
-                if (slot >= 0) J.codes[(long long)b * J.c_sb + (long long)(net * hpk + t % hpk) * J.c_sh + slot] = code;
+                if (slot >= 0) *encode_slot_ptr(J, b, net * hpk + t % hpk, slot) = code;
             }
         }
     }

@@ -24,6 +24,31 @@ __device__ __forceinline__ void patch_token(uint4 &v, int base, int last, const 
     if (e == 0) v.x = c; else if (e == 1) v.y = c; else if (e == 2) v.z = c; else v.w = c;
 }
 
+// The same two helpers over a paged signature cache (pool_head = pool + h * head_stride, table_b = the sequence's row of
+// the block table).  Pages of at least four tokens hold an aligned group of four in one piece; smaller pages are read
+// token by token.
+__device__ __forceinline__ uint4 load_codes4_paged(const CodePages &cp, const uint32_t *pool_head, const int32_t *table_b,
+                                                   int base, int n) {
+    if (cp.shift >= 2) {
+        const uint32_t *p = pool_head + (long long)__ldg(table_b + (base >> cp.shift)) * cp.page_stride + (base & ((1 << cp.shift) - 1));
+        return load_codes4(p - base, base, n);
+    }
+    uint32_t v[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int t = base + i;
+        if (t < n) v[i] = __ldg(pool_head + (long long)__ldg(table_b + (t >> cp.shift)) * cp.page_stride + (t & ((1 << cp.shift) - 1)));
+    }
+    return make_uint4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void patch_token_paged(uint4 &v, int base, int last, const CodePages &cp, const uint32_t *pool_head,
+                                                  const int32_t *table_b) {
+    const int e = last - base;
+    if (e < 0 || e > 3) return;
+    const uint32_t c = __ldcg(pool_head + (long long)__ldg(table_b + (last >> cp.shift)) * cp.page_stride + (last & ((1 << cp.shift) - 1)));
+    if (e == 0) v.x = c; else if (e == 1) v.y = c; else if (e == 2) v.z = c; else v.w = c;
+}
+
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));

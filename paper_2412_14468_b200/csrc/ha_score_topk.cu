@@ -37,16 +37,21 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
                                                                  int max_seq_len, int Hq, int Hkv,
                                                                  int chunk_tokens, long long score_row,
                                                                  unsigned char *__restrict__ ws_scores,
-                                                                 int32_t *__restrict__ ws_hist, Windows win) {
+                                                                 int32_t *__restrict__ ws_hist, Windows win, CodePages cp,
+                                                                 int row_shift) {
     __shared__ __align__(16) uint32_t c_hist[kBins][32];
     __shared__ int s_hist[kBins + 3];
     __shared__ uint32_t s_qc[G];
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    const int kvh = row_shift >= 0 ? (g >> row_shift) : g;   // the KV head whose signatures this unit scans
+    const bool paged = cp.table != nullptr;
+    const int32_t *table_b = paged ? cp.table + (long long)b * cp.bt_sb : nullptr;
     const int n = min(seq_lens[b], max_seq_len);
     const int start = chunk * chunk_tokens;
     if (start >= n) return;
     const int tid = threadIdx.x, lane = tid & 31;
-    const uint32_t *row = k_codes + (long long)b * kc_sb + (long long)g * kc_sh;
+    // contiguous cache: the unit's row; paged cache: the pool from this head's offset on
+    const uint32_t *row = paged ? k_codes + (long long)kvh * cp.head_stride : k_codes + (long long)b * kc_sb + (long long)kvh * kc_sh;
     uint32_t *srow = reinterpret_cast<uint32_t *>(ws_scores + ((long long)b * Hkv + g) * score_row);
     const int end = min(n, start + chunk_tokens);
     const WindowBounds wbd = window_bounds(win, n);   // always-kept tokens: byte kForcedByte, not counted
@@ -56,7 +61,8 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int base = pass + j * 1024 + tid * 4;
-            c[j] = (base < end) ? load_codes4(row, base, end) : make_uint4(0, 0, 0, 0);
+            if (base >= end) c[j] = make_uint4(0, 0, 0, 0);
+            else c[j] = paged ? load_codes4_paged(cp, row, table_b, base, end) : load_codes4(row, base, end);
         }
     };
     uint4 cur[4], nxt[4];
@@ -89,8 +95,13 @@ __global__ void __launch_bounds__(kScanThreads) scan_score_kernel(const uint32_t
         for (int j = 0; j < 4; ++j) {
             const int base = pass + j * 1024 + tid * 4;
             if (base < end) {
-                patch_token(cur[j], base, n - 1, row);   // the appended token may just have been written,
-                patch_token(cur[j], base, n - 2, row);   // and the one before it by a layer-step directly in front
+                if (paged) {
+                    patch_token_paged(cur[j], base, n - 1, cp, row, table_b);
+                    patch_token_paged(cur[j], base, n - 2, cp, row, table_b);
+                } else {
+                    patch_token(cur[j], base, n - 1, row);   // the appended token may just have been written,
+                    patch_token(cur[j], base, n - 2, row);   // and the one before it by a layer-step directly in front
+                }
                 const int h0 = hamming(cur[j].x), h1 = hamming(cur[j].y), h2 = hamming(cur[j].z), h3 = hamming(cur[j].w);
                 // bytes 33 - h = score + 1 (0 = no token); no byte borrows because h <= 32
                 uint32_t s4 = 0x21212121u - ((uint32_t)h0 | ((uint32_t)h1 << 8) | ((uint32_t)h2 << 16) | ((uint32_t)h3 << 24));
@@ -513,8 +524,8 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
                             long long kc_sb, long long kc_sh, const int32_t *seq_lens, const int32_t *k_per_seq,
                             int k_uniform, int max_seq_len, int k_max, int32_t *idx, long long idx_sb,
                             long long idx_sh, int32_t *count, int32_t *hist_out, int32_t *ws_hist,
-                            unsigned char *ws_scores, cudaStream_t st, Windows win) {
-    if (max_seq_len <= kClusterMaxSeq) {
+                            unsigned char *ws_scores, cudaStream_t st, Windows win, CodePages cp, int row_shift) {
+    if (max_seq_len <= kClusterMaxSeq && !cp.table && row_shift < 0) {
         // Fused path: one cluster per unit.  Cluster size: the largest of 8, 4, 2 whose grid still fits
         // the GPU in one wave (about six 256-thread CTAs per SM), so that small batches get the most
         // parallelism per sequence and large batches the most work per cluster barrier; a lane then
@@ -537,7 +548,7 @@ static cudaError_t launch_g(int B, int Hq, int Hkv, const uint32_t *q_codes, con
     const long long score_row = (long long)score_row_bytes(max_seq_len);
     dim3 grid(n_chunks, Hkv, B);
     cudaError_t e = launch_pdl(scan_score_kernel<G>, grid, dim3(kScanThreads), 0, st, q_codes, k_codes, kc_sb, kc_sh,
-                               seq_lens, max_seq_len, Hq, Hkv, chunk_tokens, score_row, ws_scores, ws_hist, win);
+                               seq_lens, max_seq_len, Hq, Hkv, chunk_tokens, score_row, ws_scores, ws_hist, win, cp, row_shift);
     if (e != cudaSuccess) return e;
     e = launch_pdl(select_kernel, grid, dim3(kScanThreads), 0, st, seq_lens, max_seq_len, k_per_seq, k_uniform, k_max,
                    Hkv, chunk_tokens, score_row, (const unsigned char *)ws_scores, (const int32_t *)ws_hist, idx, idx_sb,
@@ -551,9 +562,14 @@ cudaError_t launch_score_topk(int B, int Hq, int Hkv, const uint32_t *q_codes, c
                               long long kc_sb, long long kc_sh, const int32_t *seq_lens,
                               const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max,
                               int32_t *idx, long long idx_sb, long long idx_sh, int32_t *count,
-                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st, Windows win) {
+                              int32_t *hist_out, int32_t *ws_hist, unsigned char *ws_scores, cudaStream_t st, Windows win,
+                              CodePages cp, int row_shift) {
+    if (row_shift >= 0) {   // one unit per query head: groups of one head over Hq unit heads
+        return launch_g<1>(B, Hq, Hq, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx, idx_sb,
+                           idx_sh, count, hist_out, ws_hist, ws_scores, st, win, cp, row_shift);
+    }
 #define HA_ARGS B, Hq, Hkv, q_codes, k_codes, kc_sb, kc_sh, seq_lens, k_per_seq, k_uniform, max_seq_len, k_max, idx, \
-                idx_sb, idx_sh, count, hist_out, ws_hist, ws_scores, st, win
+                idx_sb, idx_sh, count, hist_out, ws_hist, ws_scores, st, win, cp, -1
     switch (Hq / Hkv) {
         case 1: return launch_g<1>(HA_ARGS);
         case 2: return launch_g<2>(HA_ARGS);

@@ -1313,3 +1313,126 @@ def test_step_from_entry_points_at_wide_signatures(n_bits):
             for j in range(G):
                 eo, _, _ = oracle.gather_attn(qu[b, g * G + j], Ku[b, g], Vu[b, g], ref, sm_scale=w["sm_scale"], n_valid=n)
                 assert_out_close(u16(out[b, g * G + j]), eo)
+
+
+# ---------------------------------------------------------------- paged signature cache
+
+def _page_codes(codes_np, lens, page_size, rng):
+    """Scatter contiguous signatures [B, Hkv, n_cap] over a pool [n_pages, Hkv, page_size]; returns (pool, block table)."""
+    B, Hkv, n_cap = codes_np.shape
+    pps = (n_cap + page_size - 1) // page_size
+    perm = rng.permutation(B * pps + 5)[:B * pps].reshape(B, pps).astype(np.int32)
+    pool = np.full((B * pps + 5, Hkv, page_size), 0x7BADC0DE, np.uint32)
+    padded = np.pad(codes_np, ((0, 0), (0, 0), (0, pps * page_size - n_cap)))
+    for b in range(B):
+        pool[perm[b]] = padded[b].reshape(Hkv, pps, page_size).transpose(1, 0, 2)
+    return pool, perm
+
+
+@pytest.mark.parametrize("page_size", [1, 2, 16, 64])
+def test_score_topk_over_a_paged_signature_cache(page_size):
+    """ha_score_topk_paged and ha_score_topk_per_head_paged: lists, counts and histograms bit-identical to the oracle's
+    on the un-paged signatures (paging is storage only), for ragged lengths, windows and ties."""
+    rng = np.random.default_rng(100 + page_size)
+    B, Hq, Hkv, G = 4, 8, 2, 4
+    lens = [0, 37, 4100, 9000]
+    ks = [4, 10, 300, 1000]
+    n_cap = 9003
+    codes = rng.integers(0, 2**32, size=(B, Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    codes[2, :, 500:900] = codes[2, :, 499:500]                         # a tie block
+    qc = rng.integers(0, 2**32, size=(B, Hq), dtype=np.uint64).astype(np.uint32)
+    pool, table = _page_codes(codes, lens, page_size, rng)
+    for b in range(B):                                                  # the pool round-trips through the oracle's reader
+        for h in range(Hkv):
+            assert np.array_equal(oracle.unpage_codes(pool, table[b], page_size, h, lens[b]), codes[b, h, :lens[b]])
+    pool_t = torch.from_numpy(pool.view(np.int32)).to(DEV)
+    table_t = torch.from_numpy(table).to(DEV)
+    qc_t = torch.from_numpy(qc.view(np.int32)).to(DEV)
+    sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    kp = torch.tensor(ks, dtype=torch.int32, device=DEV)
+    for n_sink, n_local in ((0, 0), (3, 40)):
+        k_max = max(ks) + n_sink + n_local
+        shape = ha.make_shape(B, Hq, Hkv, 1.0, n_sink=n_sink, n_local=n_local)
+        pick = lambda s, k: oracle.topk_windows(s, k, n_sink, n_local) if (n_sink or n_local) else oracle.topk(s, k)
+        # grouped (maximum over the group)
+        ws = ha.alloc_workspace(shape, n_cap, k_max)
+        idx = torch.full((B, Hkv, k_max), 5, dtype=torch.int32, device=DEV)
+        cnt = torch.full((B, Hkv), 5, dtype=torch.int32, device=DEV)
+        ha.ha_score_topk_paged(shape, qc_t, pool_t, table_t, sl, kp, 0, n_cap, k_max, idx, cnt, ws)
+        # one list per query head
+        wsh = ha.alloc_workspace(ha.make_shape(B, Hq, Hq, 1.0), n_cap, k_max)
+        idxh = torch.full((B, Hq, k_max), 5, dtype=torch.int32, device=DEV)
+        cnth = torch.full((B, Hq), 5, dtype=torch.int32, device=DEV)
+        ha.ha_score_topk_paged(shape, qc_t, pool_t, table_t, sl, kp, 0, n_cap, k_max, idxh, cnth, wsh, per_head=True)
+        torch.cuda.synchronize()
+        idx_np, cnt_np, idxh_np, cnth_np = idx.cpu().numpy(), cnt.cpu().numpy(), idxh.cpu().numpy(), cnth.cpu().numpy()
+        for b, n in enumerate(lens):
+            for g in range(Hkv):
+                ref = pick(oracle.score(qc[b, g * G:(g + 1) * G], codes[b, g, :n]), ks[b])
+                assert cnt_np[b, g] == len(ref) and np.array_equal(idx_np[b, g, :len(ref)], ref) and (idx_np[b, g, len(ref):] == -1).all()
+                for j in range(G):
+                    h = g * G + j
+                    refh = pick(oracle.score(qc[b, h:h + 1], codes[b, g, :n]), ks[b])
+                    assert cnth_np[b, h] == len(refh) and np.array_equal(idxh_np[b, h, :len(refh)], refh)
+
+
+@pytest.mark.parametrize("page_size,B", [(1, 3), (16, 3), (16, 20)])
+def test_whole_step_with_keys_values_and_signatures_all_paged(page_size, B):
+    """ha_sparse_decode_paged_codes (K, V and signatures behind one block table, the appended signature written into the
+    pool) returns the lists and outputs of ha_sparse_decode over the contiguous caches; ha_encode_append_paged and the
+    per-head entries over the same pools agree with their contiguous forms."""
+    lens = ([700, 2049, 33] + [500 + 61 * i for i in range(B)])[:B]
+    cfg = wl.Config("all-paged", 63, B, lens, None, 0.02, n_q_heads=8, n_kv_heads=2, sparsity=8)
+    w = wl.make_workload(cfg, DEV)
+    Hq, Hkv, n_cap, k_max = 8, 2, w["n_cap"], w["k_max"]
+    ref = _run_step(w)                                                  # contiguous caches (checked against the oracle elsewhere)
+    rng = np.random.default_rng(5 + page_size)
+    pps = (n_cap + page_size - 1) // page_size
+    table = torch.from_numpy(rng.permutation(B * pps + 3)[:B * pps].reshape(B, pps).astype(np.int32)).to(DEV)
+
+    def paged(X, fill):                                                 # [B, Hkv, n_cap, ...] -> pool [pages, Hkv, page_size, ...]
+        tail = X.shape[3:]
+        P = torch.full((B * pps + 3, Hkv, page_size) + tuple(tail), fill, dtype=X.dtype, device=DEV)
+        pad = torch.zeros((B, Hkv, pps * page_size - n_cap) + tuple(tail), dtype=X.dtype, device=DEV)
+        Xp = torch.cat([X, pad], dim=2).reshape((B, Hkv, pps, page_size) + tuple(tail)).transpose(1, 2)
+        P[table.reshape(-1).long()] = Xp.reshape((B * pps, Hkv, page_size) + tuple(tail))
+        return P
+
+    Kp, Vp = paged(w["K"], 0), paged(w["V"], 0)
+    kc_clean = ref["kc"][:, :, :n_cap]
+    stale = kc_clean.clone()
+    for b in range(B):
+        stale[b, :, lens[b] - 1] = 0x0BADF00D                           # the step must write the appended signature into the pool
+    Cp = paged(stale, 0x11111111)
+    shape = ha.make_shape(B, Hq, Hkv, w["sm_scale"])
+    ws = ha.alloc_workspace(shape, n_cap, k_max)
+    mq, mk = ha.Mapping(w["map_q"]), ha.Mapping(w["map_k"])
+    qc = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+    idx = torch.zeros(B, Hkv, k_max, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(B, Hkv, dtype=torch.int32, device=DEV)
+    out = torch.zeros(B, Hq, 128, dtype=torch.bfloat16, device=DEV)
+    ha.ha_sparse_decode_paged_codes(shape, mq, mk, w["q"], w["k_new"], Kp, Vp, Cp, table, w["seq_lens"], w["k_per_seq"], 0, n_cap,
+                                    k_max, qc, idx, cnt, out, ws)
+    torch.cuda.synchronize()
+    assert ha.ha_read_device_status(ws) == 0
+    assert torch.equal(idx, ref["idx"]) and torch.equal(cnt, ref["cnt"]) and torch.equal(qc, ref["qc"])
+    assert max_abs_diff_bf16(u16(out), u16(ref["out"])) <= OUT_AIM
+    assert torch.equal(Cp, paged(kc_clean, 0x11111111))                 # every appended signature sits in its page slot
+    # the stand-alone append into the pool
+    Cp2 = paged(stale, 0x11111111)
+    ha.ha_encode_append_paged(mk, w["k_new"], Cp2, table, w["seq_lens"])
+    torch.cuda.synchronize()
+    assert torch.equal(Cp2, Cp)
+    # one list per query head over the pools against the contiguous per-head entries
+    idxh = torch.zeros(B, Hq, k_max, dtype=torch.int32, device=DEV)
+    cnth = torch.zeros(B, Hq, dtype=torch.int32, device=DEV)
+    idxr, cntr = torch.zeros_like(idxh), torch.zeros_like(cnth)
+    outh, outr = torch.zeros_like(out), torch.zeros_like(out)
+    wsh = ha.alloc_workspace(ha.make_shape(B, Hq, Hq, w["sm_scale"]), n_cap, k_max)
+    ha.ha_score_topk_paged(shape, qc, Cp, table, w["seq_lens"], w["k_per_seq"], 0, n_cap, k_max, idxh, cnth, wsh, per_head=True)
+    ha.ha_gather_attn_per_head_paged(shape, w["q"], Kp, Vp, table, page_size, w["seq_lens"], idxh, cnth, k_max, outh, wsh)
+    kc_c = torch.nn.functional.pad(kc_clean, (0, (-n_cap) % 4)).contiguous()
+    ha.ha_score_topk_per_head(shape, qc, kc_c, w["seq_lens"], w["k_per_seq"], 0, k_max, idxr, cntr)
+    ha.ha_gather_attn_per_head(shape, w["q"], w["K"], w["V"], w["seq_lens"], idxr, cntr, k_max, outr, wsh)
+    torch.cuda.synchronize()
+    assert torch.equal(idxh, idxr) and torch.equal(cnth, cntr) and torch.equal(outh, outr)

@@ -161,3 +161,23 @@ def test_topk_all_equal_scores_takes_lowest_indices():
     assert oracle.topk(np.full(100, 17), 10).tolist() == list(range(10))
     assert oracle.topk(np.full(5, 0), 10).tolist() == list(range(5))
     assert oracle.topk(np.array([], dtype=np.int32), 4).tolist() == []
+
+
+def test_unpaging_signatures_is_storage_only():
+    """A paged signature cache read back through its block table gives the signatures that were put in, whatever the
+    page order and page size, so scores and selections over it are those over the contiguous cache."""
+    rng = np.random.default_rng(15)
+    n, Hkv = 75, 3
+    codes = rng.integers(0, 2**32, size=(Hkv, n), dtype=np.uint64).astype(np.uint32)
+    q = rng.integers(0, 2**32, size=2, dtype=np.uint64).astype(np.uint32)
+    for ps in (1, 4, 16, 64):
+        n_pages = (n + ps - 1) // ps
+        perm = rng.permutation(n_pages + 4)[:n_pages]                 # pages scattered over a larger pool
+        pool = np.full((n_pages + 4, Hkv, ps), 0xDEADBEEF, np.uint32)
+        for t in range(n):
+            pool[perm[t // ps], :, t % ps] = codes[:, t]
+        for h in range(Hkv):
+            back = oracle.unpage_codes(pool, perm, ps, h, n)
+            assert np.array_equal(back, codes[h])
+            assert np.array_equal(oracle.topk(oracle.score(q, back), 9), oracle.topk(oracle.score(q, codes[h]), 9))
+        assert np.array_equal(oracle.unpage_codes(pool, perm, ps, 1, 10), codes[1, :10])   # a prefix of the sequence
