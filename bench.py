@@ -556,6 +556,13 @@ def main():
                     "dense_us": t_de * 1e3 / 40, "dense_frac": wl.dense_bytes(l2) / (t_de * 1e3 / 40 * 1e-6) / 1e9 / peak,
                     "replicas": reps_n,
                 }
+                if name in ("sweep_B64_32K_32x", "c5"):   # the other schedule of the step: scoring ahead of the row fetch in one kernel
+                    def step_pipelined(r, b2=b2):
+                        w = r.w
+                        ha.ha_sparse_decode_pipelined(r.shape, r.mq, r.mk, w["q"], w["k_new"], w["K"], w["V"], r.kc, w["seq_lens"],
+                                                      w["k_per_seq"], 0, w["n_cap"], w["k_max"], r.qc, r.idx, r.cnt, r.out, b2.ws)
+                    t_pp, _ = b2.time_steps(step_pipelined, st, 20)
+                    supplementary[name]["pipelined_step_us"] = t_pp * 1e3 / st
                 if name == "c3":   # the same lists over a paged copy of K/V (pages of 16 tokens scattered over a pool)
                     ps, pools = 16, []
                     for r in b2.reps:
@@ -577,7 +584,23 @@ def main():
                                                 r.out, b2.ws)
                     t_pg, _ = b2.time_steps(gather_paged, st, 20)
                     supplementary[name]["gather_attn_paged16_us"] = t_pg * 1e3 / st
-                    del pools
+                    # ... and the signatures in pages of 16 behind the same block tables (one 64-byte segment per page and head)
+                    cpools = []
+                    for r, (_, _, perm) in zip(b2.reps, pools):
+                        Bn, Hk, Np = r.kc.shape
+                        pps = perm.shape[1]
+                        Cp = torch.zeros(Bn * pps, Hk, ps, dtype=torch.int32, device=device)
+                        Cp[perm.reshape(-1).long()] = torch.nn.functional.pad(r.kc, (0, pps * ps - Np)) \
+                            .reshape(Bn, Hk, pps, ps).permute(0, 2, 1, 3).reshape(Bn * pps, Hk, ps)
+                        cpools.append(Cp)
+
+                    def score_paged(r):
+                        i = b2.reps.index(r)
+                        ha.ha_score_topk_paged(r.shape, r.qc, cpools[i], pools[i][2], r.w["seq_lens"], r.w["k_per_seq"], 0,
+                                               r.w["n_cap"], r.w["k_max"], r.idx, r.cnt, b2.ws)
+                    t_sp, _ = b2.time_steps(score_paged, st, 20)
+                    supplementary[name]["score_topk_paged16_us"] = t_sp * 1e3 / st
+                    del pools, cpools
                 del b2
                 torch.cuda.empty_cache()
             except Exception as ex:   # supplementary numbers never take the headline down

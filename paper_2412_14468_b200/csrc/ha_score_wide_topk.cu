@@ -23,6 +23,7 @@ constexpr int kWideHistStride = 520;
 constexpr int kWideTokensPerThread = 16;
 constexpr int kWidePass = kWideThreads * kWideTokensPerThread;   // tokens of one pass of a CTA
 constexpr uint32_t kWideForced = 0xFFFFu;
+constexpr int kWideMaxChunks = 1024;           // chunks per unit: a single long sequence still fills the device
 
 struct WideArgs {
     const uint64_t *q_codes, *k_codes;
@@ -34,7 +35,7 @@ struct WideArgs {
     long long idx_sb, idx_sh;
     int32_t *count, *hist_out;
     int32_t *unit_hist;            // [units][kWideHistStride], zero before the scan
-    int32_t *chunk_counts;         // [units][kMaxChunks][2]
+    int32_t *chunk_counts;         // [units][kWideMaxChunks][2]
     uint16_t *scores;              // [units][score_row]
     long long score_row;
 };
@@ -92,7 +93,10 @@ __global__ void __launch_bounds__(kWideThreads) wide_scan_kernel(const WideArgs 
         const int score = a.n_bits - best;
         const bool forced = t < wu.wbd.sink_end || t >= wu.wbd.local_begin;
         srow[t] = forced ? (uint16_t)kWideForced : (uint16_t)score;
-        if (!forced) atomicAdd(&s_hist[warp][score], 1);
+        // unrelated signatures crowd into a few levels around b / 2: lanes with the same score add once, together
+        const int key = forced ? -1 : score;
+        const unsigned peers = __match_any_sync(__activemask(), key);
+        if (key >= 0 && (int)(__ffs(peers) - 1) == (tid & 31)) atomicAdd(&s_hist[warp][score], __popc(peers));
     }
     __syncthreads();
     int32_t *uh = a.unit_hist + (long long)unit * kWideHistStride;
@@ -184,7 +188,7 @@ __global__ void __launch_bounds__(kWideThreads) wide_count_kernel(const WideArgs
     if (tid < 2) {
         int s = 0;
         for (int w = 0; w < kWideThreads / 32; ++w) s += s_red[tid][w];
-        a.chunk_counts[((long long)unit * kMaxChunks + chunk) * 2 + tid] = s;
+        a.chunk_counts[((long long)unit * kWideMaxChunks + chunk) * 2 + tid] = s;
     }
 }
 
@@ -209,7 +213,7 @@ __global__ void __launch_bounds__(kWideThreads) wide_write_kernel(const WideArgs
     } else if (warp <= 2) {   // tokens above / at the threshold in the chunks before this one
         const int which = warp - 1;
         int s = 0;
-        for (int c = lane; c < chunk; c += 32) s += __ldcg(a.chunk_counts + ((long long)unit * kMaxChunks + c) * 2 + which);
+        for (int c = lane; c < chunk; c += 32) s += __ldcg(a.chunk_counts + ((long long)unit * kWideMaxChunks + c) * 2 + which);
 #pragma unroll
         for (int dd = 16; dd > 0; dd >>= 1) s += __shfl_xor_sync(0xffffffffu, s, dd);
         if (lane == 0) s_before[which] = s;
@@ -265,7 +269,7 @@ WideLayout wide_layout(int B, int Hkv, int max_seq_len) {
     const size_t units = (size_t)B * Hkv;
     size_t o = kHeaderBytes;
     L.off_hist = o;   o = align_up(o + units * kWideHistStride * 4, 256);
-    L.off_counts = o; o = align_up(o + units * kMaxChunks * 2 * 4, 256);
+    L.off_counts = o; o = align_up(o + units * kWideMaxChunks * 2 * 4, 256);
     L.score_row = align_up((size_t)(max_seq_len > 0 ? max_seq_len : 0), 256);
     L.off_scores = o; o = align_up(o + units * L.score_row * 2, 256);
     L.total = o;
@@ -287,13 +291,13 @@ cudaError_t launch_score_topk_wide(int B, int Hq, int Hkv, int n_bits, const uin
     a.chunk_counts = reinterpret_cast<int32_t *>(ws + L.off_counts);
     a.scores = reinterpret_cast<uint16_t *>(ws + L.off_scores);
     a.score_row = (long long)L.score_row;
-    // chunks of whole passes, about four CTAs per SM when there is that much work, at most kMaxChunks per unit
+    // chunks of whole passes, about eight CTAs per SM when there is that much work, at most kWideMaxChunks per unit
     const long long units = (long long)B * Hkv, n = max_seq_len > 0 ? max_seq_len : 1;
-    long long per_unit = 4LL * sm_count() / (units > 0 ? units : 1);
+    long long per_unit = 8LL * sm_count() / (units > 0 ? units : 1);
     if (per_unit < 1) per_unit = 1;
-    if (per_unit > kMaxChunks) per_unit = kMaxChunks;
+    if (per_unit > kWideMaxChunks) per_unit = kWideMaxChunks;
     long long c = (n + per_unit - 1) / per_unit;
-    const long long c_min = (n + kMaxChunks - 1) / kMaxChunks;
+    const long long c_min = (n + kWideMaxChunks - 1) / kWideMaxChunks;
     if (c < c_min) c = c_min;
     if (c < kWidePass) c = kWidePass;
     a.chunk_tokens = (int)((c + kWidePass - 1) / kWidePass * kWidePass);
