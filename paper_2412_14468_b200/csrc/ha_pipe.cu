@@ -1,12 +1,13 @@
 // SCORE + TOPK and GATHER-ATT of a layer-step in ONE persistent kernel, for steps with too many (sequence, KV head)
-// units for the single-cluster kernel of ha_fused.cu.
+// units for the single-cluster kernel of ha_fused.cu (entry point ha_sparse_decode_pipelined; ha_sparse_decode itself runs
+// such steps as three kernels, which is the faster schedule on B200: see the note on scoring further down).
 //
 // Why: at scale the two halves of the step are bound by different units of the SM.  SCORE (Eq. 1 as bitcount(xor),
 // Section 4.1) spends its time in the population-count pipe and the integer pipe; GATHER-ATT (Section 4) waits for
-// HBM.  Run one after the other, each leaves the other's resource idle.  Here every SM holds one CTA of 24 warps
-// with two roles (the register file is re-divided between them with setmaxnreg: 48 registers per SCORE thread, 144
-// per GATHER thread):
-//   * sixteen SCORE warps walk the units of the CTA's range: scores as one byte per token, a histogram per group of
+// HBM.  Run one after the other, each leaves the other's resource idle.  Here every SM holds one CTA of 28 warps
+// with two roles (the register file is re-divided between them with setmaxnreg: 40 registers per SCORE thread, 152
+// per GATHER thread, out of the 72 per thread the CTA is launched with):
+//   * twenty SCORE warps walk the units of the CTA's range: scores as one byte per token, a histogram per group of
 //     four warps, the threshold of the standard top-k (Section 4), the index list in ascending token order (ties to
 //     the lowest index), then a release counter per unit;
 //   * eight GATHER warps follow them over the same range: each warp keeps a two-stage ring of 16-row blocks in flight
@@ -32,7 +33,7 @@ namespace ha {
 constexpr int kPipeGatherWarps = 8;
 constexpr int kPipeScoreWarps = 20;
 constexpr int kPipeScoreGroups = 5;                   // counter tables: one per four SCORE warps
-constexpr int kPipeGatherRegs = 152, kPipeScoreRegs = 40;   // per thread once the roles part (setmaxnreg); 8 x 32 x 144 + 16 x 32 x 48 = 768 x 80, what the CTA is launched with
+constexpr int kPipeGatherRegs = 152, kPipeScoreRegs = 40;   // per thread once the roles part (setmaxnreg): 8 x 32 x 152 + 20 x 32 x 40 = 896 x 72, exactly what the CTA is launched with (a role can only take what the other gave back)
 constexpr int kPipeGatherThreads = kPipeGatherWarps * 32;
 constexpr int kPipeScoreThreads = kPipeScoreWarps * 32;
 constexpr int kPipeThreads = kPipeGatherThreads + kPipeScoreThreads;
@@ -155,8 +156,8 @@ struct ScoreJob {
 };
 
 // Scoring needs many warps: a warp issues about one instruction in twelve cycles here (dependent population counts,
-// shared-memory reductions, loads), so the sixteen SCORE warps of a CTA together keep the population-count pipe busy
-// where four did not.  They get by with few registers (two rows of signatures in flight per warp), which leaves the
+// shared-memory reductions, loads), so the twenty SCORE warps of a CTA together keep the population-count pipe far busier
+// than four did (and still less busy than the 48 warps per SM of the stand-alone kernel).  They get by with few registers (two rows of signatures in flight per warp), which leaves the
 // register file to the GATHER warps.
 template <int G>
 struct ScoreRole {

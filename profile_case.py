@@ -120,6 +120,64 @@ def score_wide(args):
             print(f"step {s} {name:14s}: {us:9.1f} us  {nbytes / us / 1e3:8.1f} GB/s (plain launch, L2 flushed)")
 
 
+def encode_only(args):
+    """ENCODE of one decode step alone (queries through phi_q, appended keys through phi_kv): a few KB of inputs."""
+    cfg = wl.CONFIGS[args.config]
+    B = args.batch if args.batch is not None else cfg.batch
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    Hq, Hkv = cfg.n_q_heads, cfg.n_kv_heads
+    g = torch.Generator(dev).manual_seed(wl.BASE_SEED + 79)
+    mq, mk = ha.Mapping(wl.make_mapping(Hkv, g, dev)), ha.Mapping(wl.make_mapping(Hkv, g, dev))
+    q = torch.randn(B, Hq, 128, device=dev, generator=g).to(torch.bfloat16)
+    k = torch.randn(B, Hkv, 128, device=dev, generator=g).to(torch.bfloat16)
+    qc = torch.zeros(B, Hq, 1, dtype=torch.int32, device=dev)
+    kc = torch.zeros(B, Hkv, 1, dtype=torch.int32, device=dev)
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+    for s in range(args.steps):
+        _ = int(flush.sum())
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ha.ha_encode(mq, Hq // Hkv, q, qc)
+        ha.ha_encode(mk, 1, k, kc)
+        e1.record()
+        torch.cuda.synchronize()
+        print(f"step {s}: {e0.elapsed_time(e1) * 1e3:.1f} us for {B * Hq} + {B * Hkv} vectors (plain launches, L2 flushed)")
+
+
+def score_topk_wide(args):
+    """SCORE + TOPK at signatures of 64 .. 512 bits: one query head over --tokens tokens, k = n / 32."""
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    n = args.tokens
+    g = torch.Generator(dev).manual_seed(wl.BASE_SEED + 6)
+    shape = ha.make_shape(1, 1, 1, 1.0)
+    ln = torch.full((1,), n, dtype=torch.int32, device=dev)
+    kq = n // 32
+    idx = torch.zeros(1, 1, kq, dtype=torch.int32, device=dev)
+    cnt = torch.zeros(1, 1, dtype=torch.int32, device=dev)
+    ws = ha.alloc_workspace_wide(shape, n, device=dev)
+    flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+    cases = []
+    for bits in (64, 512):
+        W = bits // 64
+        kc = torch.randint(-2**63, 2**63 - 1, (1, 1, n, W), dtype=torch.int64, device=dev, generator=g)
+        qc = torch.randint(-2**63, 2**63 - 1, (1, 1, W), dtype=torch.int64, device=dev, generator=g)
+        cases.append((bits, kc, qc))
+    torch.cuda.synchronize()
+    for s in range(args.steps):
+        for bits, kc, qc in cases:
+            _ = int(flush.sum())
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ha.ha_score_topk_wide(shape, bits, qc, kc, ln, None, kq, n, kq, idx, cnt, ws)
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3
+            print(f"step {s} {bits:3d} bit: {us:9.1f} us  {n * bits / 8 / us / 1e3:8.1f} GB/s of signatures (plain launches, L2 flushed)")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="c3")
@@ -140,10 +198,19 @@ def main():
                     help="with --score-only: also run ha_score_topk_sum (per-head scores added instead of maximised)")
     ap.add_argument("--score-wide", action="store_true",
                     help="stand-alone SCORE on signatures of 64..512 bits and the inner-product comparator on --tokens tokens")
+    ap.add_argument("--score-topk-wide", action="store_true",
+                    help="SCORE + TOPK on signatures of 64 and 512 bits (ha_score_topk_wide) on --tokens tokens")
+    ap.add_argument("--encode-only", action="store_true", help="ENCODE of one decode step alone (--batch sequences)")
+    ap.add_argument("--pipelined", action="store_true",
+                    help="run the step through ha_sparse_decode_pipelined (SCORE + TOPK ahead of GATHER-ATT in one persistent kernel)")
     ap.add_argument("--tokens", type=int, default=1 << 23)
     args = ap.parse_args()
     if args.score_wide:
         return score_wide(args)
+    if args.score_topk_wide:
+        return score_topk_wide(args)
+    if args.encode_only:
+        return encode_only(args)
     if args.score_only:
         return score_only(args)
     if args.prefill:
@@ -178,8 +245,9 @@ def main():
             ha.ha_score_topk(shape, qc, kc, w["seq_lens"], w["k_per_seq"], 0, w["n_cap"], w["k_max"], idx, cnt, ws)
             ha.ha_gather_attn(shape, w["q"], w["K"], w["V"], w["seq_lens"], idx, cnt, row_width, out, ws)
         else:
-            ha.ha_sparse_decode(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
-                                w["n_cap"], w["k_max"], qc, idx, cnt, out, ws)
+            step = ha.ha_sparse_decode_pipelined if args.pipelined else ha.ha_sparse_decode
+            step(shape, mq, mk, w["q"], w["k_new"], w["K"], w["V"], kc, w["seq_lens"], w["k_per_seq"], 0,
+                 w["n_cap"], w["k_max"], qc, idx, cnt, out, ws)
         e1.record()
         if args.dense:
             ha.ha_dense_decode(shape, w["q"], w["K"], w["V"], w["seq_lens"], w["n_cap"], out, ws)
