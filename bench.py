@@ -35,7 +35,7 @@ UNIT = "us"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the step's kernel on this workload: NOT measured by this
 # run (a number taken under a profiler is never a bench value) but copied from the ncu capture named beside it
 TRAFFIC_FROM_PROFILE = {"bytes": 6555553, "source": "profiles/launch_list_bench_c2.md", "captured_at_commit": "220b429"}
-GATHER_TRAFFIC_FROM_PROFILE = {"bytes": 4275000, "source": "profiles/fused_step_kernel_c2.md", "captured_at_commit": "aed5e69"}
+GATHER_TRAFFIC_FROM_PROFILE = {"bytes": 4275000, "source": "profiles/launch_list_bench_c2.md", "captured_at_commit": "aed5e69"}
 MIN_TIMED_MS = 50.0                 # the timed region of `steps` steps is repeated until this much has been measured
 WORKLOAD = "c2: B=1, Hq=32, Hkv=8, d=128, ctx=32768, k=1024 (32x), 1% planted keys"
 
