@@ -497,10 +497,46 @@ static cudaError_t launch_cluster_t(int rows, int B, int Hq, int Hkv, const uint
                                     const int32_t *k_per_seq, int k_uniform, int max_seq_len, int k_max, int32_t *idx,
                                     long long idx_sb, long long idx_sh, int32_t *count, int32_t *hist_out,
                                     cudaStream_t st, Windows win) {
+    static bool opted[64] = {};   // opt in to the padded shared-memory sizes once per device
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev >= 0 && dev < 64 && !opted[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(score_select_cluster_kernel<G, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+            if (e != cudaSuccess) return e;
+            opted[dev] = true;
+        }
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CS, Hkv, B);
     cfg.blockDim = dim3(kScanThreads);
     cfg.dynamicSmemBytes = (size_t)rows * 2048;   // one score byte per token of the CTA's slice (<= 16 KB)
+    {
+        // Launched behind another kernel, the CTAs land wherever room appears first, and an SM that takes six of them
+        // while others hold two sets the kernel's time (the population-count unit is shared by the CTAs of an SM).
+        // When the grid needs fewer than six CTAs per SM, shared memory is requested as if each CTA needed a whole
+        // share of the SM, so that no SM can take more than ceil(CTAs / SMs).  Clusters of 4 or 8 need some slack
+        // for that (all CTAs of a cluster are placed together): without it the cap only delays their placement.
+        const int n_ctas = CS * Hkv * B, n_sm = sm_count();
+        const int cap = (n_ctas + n_sm - 1) / n_sm;   // CTAs per SM
+        const bool slack = CS == 2 || 2 * (cap * n_sm - n_ctas) >= n_sm;
+        if (n_ctas > n_sm && cap < 6 && slack) {
+            static size_t pad[64][6] = {};   // per device and cap: the least dynamic shared memory with which only `cap` CTAs fit
+            int dev = 0;
+            cudaGetDevice(&dev);
+            if (dev < 0 || dev >= 64) dev = 0;
+            if (!pad[dev][cap]) {
+                size_t found = 0;
+                for (size_t kb = 8; kb <= 100 && !found; ++kb) {
+                    int occ = 0;
+                    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, score_select_cluster_kernel<G, CS>, kScanThreads, kb * 1024) != cudaSuccess) break;
+                    if (occ <= cap) found = kb * 1024;
+                }
+                pad[dev][cap] = found ? found : 1;
+            }
+            if (pad[dev][cap] > cfg.dynamicSmemBytes) cfg.dynamicSmemBytes = pad[dev][cap];
+        }
+    }
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
