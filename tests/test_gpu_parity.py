@@ -213,6 +213,22 @@ def test_score_topk_long_sequences(lens, n_cap):
         _check_score_topk(qc, kc, lens, ks, Hq, Hkv)
 
 
+@pytest.mark.parametrize("B,Hkv,G,n_hi", [(16, 8, 4, 2100), (30, 8, 2, 9000), (40, 4, 4, 2100), (14, 8, 1, 30000)])
+def test_score_topk_grids_that_are_launched_with_a_cap_on_ctas_per_sm(B, Hkv, G, n_hi):
+    """Batches whose cluster grid needs fewer than six CTAs per SM are launched with padded shared memory (at most
+    ceil(CTAs / SMs) CTAs per SM): clusters of 4, 2, 4 and 8 here, ragged lengths, same lists as the oracle."""
+    rng = np.random.default_rng(500 + B)
+    Hq = Hkv * G
+    lens = [int(v) for v in rng.integers(1, n_hi, size=B)]
+    lens[0], lens[-1] = n_hi, 0
+    n_cap = (n_hi + 3) // 4 * 4
+    kc = rng.integers(0, 2 ** 32, size=(B, Hkv, n_cap), dtype=np.uint64).astype(np.uint32)
+    qc = rng.integers(0, 2 ** 32, size=(B, Hq), dtype=np.uint64).astype(np.uint32)
+    for ks in ([n // 16 for n in lens], [min(n, 300) for n in lens]):
+        _check_score_topk(qc, kc, lens, ks, Hq, Hkv)
+    _check_score_topk(qc, kc, lens, [n // 32 for n in lens], Hq, Hkv, n_sink=7, n_local=33)
+
+
 @pytest.mark.parametrize("n_sink,n_local", [(128, 128), (1, 0), (0, 3), (5000, 7), (300, 70000)])
 def test_score_topk_with_always_kept_windows(n_sink, n_local):
     """First n_sink and most recent n_local tokens always selected, the budget on top (Section 5, baselines):
