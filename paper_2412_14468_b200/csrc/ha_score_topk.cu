@@ -334,6 +334,12 @@ __global__ void __launch_bounds__(kScanThreads, 6) score_select_cluster_kernel(
     uint4 c[4];   // two rows
     load_row(0, c[0], c[1], true);
     load_row(1, c[2], c[3], true);
+    // the other rows of this warp start their way from HBM to L2 now (one request per 128-byte line, no registers): the
+    // loads that follow turn by turn then wait for L2 only, which is what counts when few CTAs share the SM
+    for (int p = 2; p < Rb; ++p) {
+        const int t = wb + p * 256 + lane * 8;
+        if ((lane & 3) == 0 && t < n) asm volatile("prefetch.global.L2 [%0];" ::"l"(row + t));
+    }
     for (int i = tid; i < kBins * 32 / 4; i += kScanThreads)
         reinterpret_cast<uint4 *>(&c_hist[0][0])[i] = make_uint4(0u, 0u, 0u, 0u);
     if (tid < kBins + 3) s_hist[tid] = 0;
