@@ -57,6 +57,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         with ThreadPoolExecutor(max_workers=min(len(todo), os.cpu_count() or 4)) as ex:
             list(ex.map(compile_one, todo))
     objs = [_obj(s) for s in sources()]
+    for stale in set(glob.glob(os.path.join(OBJ, "*.o"))) - set(objs):   # objects of sources that no longer exist
+        os.remove(stale)
     if todo or force or _stale(LIB, objs):
         subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB] + objs, check=True)
     return LIB
