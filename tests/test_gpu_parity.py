@@ -529,6 +529,29 @@ def test_gather_attn_with_smaller_clusters(B):
     _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128), expect_flag=ha.HA_DEV_BAD_INDEX)
 
 
+@pytest.mark.parametrize("ragged", [False, True])
+def test_gather_attn_equal_lists_on_most_of_the_ctas_are_taken_as_whole_units(ragged):
+    """240 units (more than the cluster kernel takes, at least three quarters of the split-K kernel's CTAs): lists of
+    equal length are attended to one whole unit per CTA, a batch with one shorter list by the balanced split; both
+    against the oracle."""
+    B, Hkv, G, n_cap, k_max = 60, 4, 2, 700, 200
+    Hq = Hkv * G
+    rng = np.random.default_rng(91)
+    lens = [n_cap] * B
+    q, K, V = _attn_inputs(B, Hq, Hkv, n_cap, 92)
+    idx = np.full((B, Hkv, k_max), -1, np.int32)
+    cnt = np.full((B, Hkv), k_max, np.int32)
+    for b in range(B):
+        for g in range(Hkv):
+            idx[b, g] = np.sort(rng.choice(n_cap, size=k_max, replace=False))
+    if ragged:
+        cnt[17, 2] = 37
+        idx[17, 2, 37:] = -1
+    before = ha.ha_kernel_launches()
+    _check_gather(q, K, V, lens, idx, cnt, 1.0 / math.sqrt(128))
+    assert ha.ha_kernel_launches() - before == 1
+
+
 @pytest.mark.parametrize("width", [64, 2100])   # both stand-alone gather kernels (see test_gather_attn_random_lists)
 def test_gather_attn_padding_invalid_and_unsorted_indices(width):
     Hq, Hkv, n_cap = 8, 2, 500
