@@ -524,7 +524,7 @@ def main():
         del bench
         torch.cuda.empty_cache()
         cases = [("c3", wl.CONFIGS["c3"], 2, 400), ("c4", wl.CONFIGS["c4"], 2, 400), ("c5", wl.CONFIGS["c5"], 2, 200)]
-        for bsz in (4, 8, 16, 64):   # batch sweep at the headline shape: 32K context, 32x
+        for bsz in (4, 8, 16, 32, 64):   # batch sweep at the headline shape: 32K context, 32x
             cases.append((f"sweep_B{bsz}_32K_32x", wl.Config(f"sweep{bsz}", 10 + bsz, bsz, 32768, 1024, 0.01), 2 if bsz >= 16 else 8, 400))
         for name, cfg_s, reps_n, st in cases:
             try:
