@@ -17,6 +17,7 @@
 // split into bf16 hi + lo parts so the weights keep ~16 bits), softmax online in fp32 in the log2
 // domain.  At ~4 FLOP/B the kernel is bound by HBM; the tensor cores only keep the instruction
 // count out of the way.
+#include <atomic>
 #include "ha_attn_dev.cuh"
 
 namespace ha {
@@ -574,15 +575,15 @@ extern "C" int ha_gather_attn_static(const ha_shape *shape, const uint16_t *q, c
 
     // Set-up, once per device: in host code the array's name is only a stand-in for the symbol; the
     // device address that a kernel can use has to be asked for, with the device current.
-    static void *scratch_of_device[64] = {};
+    static std::atomic<void *> scratch_of_device[64];   // zero-initialised; two threads that race store the same address
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HA_ERR_CUDA;
-    if (!scratch_of_device[dev]) {
-        void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return HA_ERR_CUDA;
-        scratch_of_device[dev] = p;
+    void *scratch = scratch_of_device[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || !scratch) return HA_ERR_CUDA;
+        scratch_of_device[dev].store(scratch, std::memory_order_release);
     }
-    unsigned char *base = reinterpret_cast<unsigned char *>(scratch_of_device[dev]);
+    unsigned char *base = reinterpret_cast<unsigned char *>(scratch);
     cudaStream_t st = (cudaStream_t)stream;
     // the array keeps whatever the last call left: the status word and the ticket counters must start at zero
     if (cudaMemsetAsync(base, 0, kStaticMlOff, st) != cudaSuccess) return HA_ERR_CUDA;
